@@ -1,0 +1,362 @@
+"""Pins of the CPU oracle against things other than itself: closed forms, invariants,
+library routines on special cases, brute force on tiny inputs and the values the paper
+prints (tests/golden).  A plausible mistake in the oracle (dropped term, wrong sign or
+index, transposed operand) fails at least one of these."""
+import itertools
+import os
+
+import numpy as np
+import pytest
+
+from oracle import accordion_oracle as orc
+from paper_2010_16248_b200 import workloads as wl
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden", "data_sent_tables.txt")
+
+
+def _layers(table):
+    return [(int(table.offset[l]), int(table.rows[l]), int(table.cols[l]), int(table.kind[l]))
+            for l in range(table.n_layers)]
+
+
+# ------------------------------------------------------------------ controller
+def test_alg1_truth_table():
+    # (prev_norm, curr_norm, lr_curr, lr_next) -> level, eta = 0.5; boundary cases are exactly representable
+    cases = [
+        (1.0, 0.5, 0.1, 0.1, orc.LOW),    # ratio exactly eta: ">=" -> critical
+        (1.0, 1.5, 0.1, 0.1, orc.LOW),    # growth counts too (absolute value)
+        (1.0, 0.75, 0.1, 0.1, orc.HIGH),
+        (1.0, 1.25, 0.1, 0.1, orc.HIGH),
+        (1.0, 1.0, 0.1, 0.01, orc.LOW),   # LR decay forces the low level
+        (1.0, 1.0, 0.1, 0.2, orc.HIGH),   # LR increase does not
+        (4.0, 1.0, 0.1, 0.1, orc.LOW),
+        (0.0, 0.0, 0.1, 0.1, orc.LOW),    # ||prev|| = 0: product form, 0 >= 0
+        (0.0, 3.0, 0.1, 0.1, orc.LOW),
+    ]
+    for a, b, lc, ln, want in cases:
+        level, prev = orc.detect_regime(np.array([b * b]), np.array([a * a]), lc, ln, 0.5)
+        assert level[0] == want, (a, b, lc, ln)
+        assert prev[0] == b * b
+    level, prev = orc.detect_regime(np.array([9.0]), np.array([-1.0]), 0.1, 0.1, 0.5)
+    assert level[0] == orc.LOW and prev[0] == 9.0  # no previous window
+
+
+def test_detector_scale_invariance_and_per_layer_independence():
+    rng = np.random.default_rng(0)
+    prev = rng.uniform(0.1, 4.0, 50)
+    curr = rng.uniform(0.1, 4.0, 50)
+    l1, _ = orc.detect_regime(curr, prev, 0.1, 0.1, 0.5)
+    l2, _ = orc.detect_regime(curr * 64.0, prev * 64.0, 0.1, 0.1, 0.5)
+    assert np.array_equal(l1, l2)
+    want = (np.abs(np.sqrt(prev) - np.sqrt(curr)) / np.sqrt(prev) >= 0.5).astype(np.uint8)
+    assert np.array_equal(l1, want)
+    assert 0 < l1.sum() < 50
+
+
+def test_layer_norms_closed_form_and_library():
+    table = wl.make_table([("a", (3, 5)), ("b", (7,)), ("c", (4, 4))])
+    layers = _layers(table)
+    buf = np.zeros(table.stride, np.float32)
+    buf[0:15] = 1.0                      # ||ones(15)||^2 = 15
+    buf[16:23] = np.arange(1, 8)         # 1^2+..+7^2 = 140
+    rng = np.random.default_rng(1)
+    c = rng.standard_normal(16).astype(np.float32)
+    buf[24:40] = c
+    n2 = orc.layer_norms2(buf, layers)
+    assert n2[0] == 15.0 and n2[1] == 140.0
+    assert np.isclose(np.sqrt(n2[2]), np.linalg.norm(c.astype(np.float64)), rtol=1e-14)
+
+
+def test_accumulate_sums_decider_gradients():
+    table = wl.make_table([("a", (2, 3)), ("b", (5,))])
+    layers = _layers(table)
+    delta = np.zeros(table.stride)
+    g1 = np.arange(table.stride, dtype=np.float32)
+    g2 = np.ones(table.stride, np.float32)
+    orc.accumulate(delta, g1, layers)
+    orc.accumulate(delta, g2, layers)
+    for (off, r, c, k) in layers:
+        assert np.array_equal(delta[off:off + r * c], (g1 + g2)[off:off + r * c].astype(np.float64))
+    assert delta[6] == 0.0 and delta[7] == 0.0  # padding between layers untouched
+
+
+def test_c1_schedule_known_answer():
+    """Config 1: scale doubles at iteration 10, checks after iterations 4, 9, 14, 19.
+    Levels: LOW before the first check and after it (no previous window), HIGH after the
+    second (equal windows), LOW after the third (window norm doubled: ratio 1 >= 0.5),
+    HIGH after the fourth (equal again)."""
+    w = wl.workload(1, scale=4)
+    layers = _layers(w.table)
+    stream = wl.GradientStream(w)
+    delta = np.zeros(w.table.stride)
+    prev = -np.ones(1)
+    levels = []
+    level = np.ones(1, np.uint8)
+    for t in range(w.n_iters):
+        levels.append(int(level[0]))
+        g = stream.grads(t).numpy()
+        orc.accumulate(delta, g[0], layers)
+        if (t + 1) % w.check_every == 0:
+            level, prev = orc.detect_regime(orc.layer_norms2(delta, layers), prev, 0.1, 0.1, w.eta)
+            delta[:] = 0
+    assert levels == [1] * 5 + [1] * 5 + [0] * 5 + [1] * 5
+    assert int(level[0]) == 0
+
+
+# ------------------------------------------------------------------ PowerSGD
+def _rand_problem(rng, n, m, W, rank_low, err_scale=0.3):
+    table = wl.make_table([("w", (n, m)), ("b", (5,))])
+    layers = _layers(table)
+    grads = np.zeros((W, table.stride), np.float32)
+    err = np.zeros((W, table.stride), np.float32)
+    grads[:, :n * m] = rng.standard_normal((W, n * m))
+    err[:, :n * m] = err_scale * rng.standard_normal((W, n * m))
+    grads[:, layers[1][0]:layers[1][0] + 5] = rng.standard_normal((W, 5))
+    q = [rng.standard_normal((m, rank_low)).astype(np.float32), None]
+    return table, layers, grads, err, q
+
+
+def test_powersgd_exact_recovery_of_rank_r():
+    rng = np.random.default_rng(2)
+    n, m, W = 12, 9, 3
+    for r in (1, 2, 4):
+        table, layers, grads, err, q = _rand_problem(rng, n, m, W, r)
+        # small-integer factors: the product is exactly representable in fp32, so the rank is exactly r
+        B = rng.integers(-4, 5, (n, r)).astype(np.float64) @ rng.integers(-4, 5, (r, m)).astype(np.float64)
+        assert np.linalg.matrix_rank(B) == r
+        grads[:, :n * m] = B.astype(np.float32).reshape(-1)
+        err[:] = 0
+        M = grads[0, :n * m].astype(np.float64).reshape(n, m)
+        out, e, qn, ph = orc.powersgd_step(grads, err, q, [1, 1], layers, r, 1, gs_eps=0.0)
+        assert np.allclose(out[:n * m].reshape(n, m), M, atol=1e-12 * np.abs(M).max())
+        assert np.abs(e[:, :n * m]).max() < 1e-12 * np.abs(M).max()
+
+
+def test_powersgd_matches_qr_and_projection():
+    rng = np.random.default_rng(3)
+    n, m, W, r = 10, 7, 4, 3
+    table, layers, grads, err, q = _rand_problem(rng, n, m, W, r)
+    out, e, qn, ph = orc.powersgd_step(grads, err, q, [1, 1], layers, r, 1, gs_eps=0.0)
+    Mw = [(grads[w, :n * m].astype(np.float64) + err[w, :n * m].astype(np.float64)).reshape(n, m) for w in range(W)]
+    Mbar = sum(Mw) / W
+    # P^ is the thin-QR factor of Mbar Q with R's diagonal made positive (library routine)
+    Qf, R = np.linalg.qr(Mbar @ q[0].astype(np.float64))
+    Qf = Qf * np.sign(np.diag(R))
+    assert np.allclose(ph[0], Qf, atol=1e-10)
+    assert np.allclose(ph[0].T @ ph[0], np.eye(r), atol=1e-12)
+    # A = P^ P^T Mbar ; Q_new = Mbar^T P^
+    A = out[:n * m].reshape(n, m)
+    assert np.allclose(A, Qf @ Qf.T @ Mbar, atol=1e-12)
+    assert np.allclose(qn[0], Mbar.T @ Qf, atol=1e-12)
+    # error-feedback invariant per worker and orthogonality of the mean residual to P^
+    for w in range(W):
+        assert np.allclose(A + e[w, :n * m].reshape(n, m), Mw[w], atol=1e-13)
+    assert np.abs(Qf.T @ (sum(e[w, :n * m].reshape(n, m) for w in range(W)) / W)).max() < 1e-12
+    # VECTOR layer: plain mean, no memory
+    off = layers[1][0]
+    assert np.allclose(out[off:off + 5], grads[:, off:off + 5].astype(np.float64).mean(0), atol=1e-15)
+    assert np.all(e[:, off:off + 5] == 0)
+
+
+def test_powersgd_rank_levels_and_untouched_columns():
+    rng = np.random.default_rng(4)
+    n, m, W = 8, 6, 2
+    table, layers, grads, err, q = _rand_problem(rng, n, m, W, 2)
+    _, _, qn_hi, ph_hi = orc.powersgd_step(grads, err, q, [0, 0], layers, 2, 1)
+    assert ph_hi[0].shape == (n, 1)
+    assert np.array_equal(qn_hi[0][:, 1], q[0][:, 1].astype(np.float64))  # column beyond the rank keeps its value
+    _, _, qn_lo, ph_lo = orc.powersgd_step(grads, err, q, [1, 1], layers, 2, 1)
+    assert ph_lo[0].shape == (n, 2)
+    assert np.allclose(ph_lo[0][:, 0], ph_hi[0][:, 0])
+
+
+def test_powersgd_symmetries():
+    rng = np.random.default_rng(5)
+    n, m, W, r = 9, 11, 3, 2
+    table, layers, grads, err, q = _rand_problem(rng, n, m, W, r)
+    out, e, qn, ph = orc.powersgd_step(grads, err, q, [1, 1], layers, r, 1, gs_eps=0.0)
+    perm = [2, 0, 1]
+    out_p, e_p, qn_p, ph_p = orc.powersgd_step(grads[perm], err[perm], q, [1, 1], layers, r, 1, gs_eps=0.0)
+    assert np.allclose(out, out_p, atol=1e-13) and np.allclose(e[perm], e_p, atol=1e-13)
+    c = 8.0  # power of two: exact scaling
+    out_s, e_s, qn_s, ph_s = orc.powersgd_step(grads * c, err * c, q, [1, 1], layers, r, 1, gs_eps=0.0)
+    assert np.allclose(out_s, c * out, rtol=1e-12, atol=1e-14)
+    assert np.allclose(ph_s[0], ph[0], atol=1e-12)
+
+
+@pytest.mark.parametrize("power", [1.0, 0.5])
+def test_powersgd_power_iteration_reaches_best_rank_r_error(power):
+    """Repeating the step on a fixed M with the memory reset is subspace iteration: the
+    error converges to the optimal sqrt(sum_{i>r} s_i^2), known in closed form for the
+    synthetic spectra s_i = i^-1 and i^-0.5."""
+    rng = np.random.default_rng(6)
+    n, m, r, rho = 40, 30, 2, 30
+    U, _ = np.linalg.qr(rng.standard_normal((n, rho)))
+    V, _ = np.linalg.qr(rng.standard_normal((m, rho)))
+    s = np.arange(1, rho + 1, dtype=np.float64) ** (-power)
+    M = (U * s) @ V.T
+    table = wl.make_table([("w", (n, m))])
+    layers = _layers(table)
+    grads = np.zeros((1, table.stride), np.float32)
+    grads[0, :n * m] = M.reshape(-1)
+    M32 = grads[0, :n * m].astype(np.float64).reshape(n, m)
+    s32 = np.linalg.svd(M32, compute_uv=False)
+    best = np.sqrt(np.sum(s32[r:] ** 2))
+    assert np.isclose(best, np.sqrt(np.sum(s[r:] ** 2)), rtol=1e-5)
+    q = [rng.standard_normal((m, r)).astype(np.float32)]
+    err0 = np.zeros_like(grads)
+    last = None
+    for it in range(400):
+        out, e, q, ph = orc.powersgd_step(grads, err0, q, [1], layers, r, 1, gs_eps=0.0)
+        last = np.linalg.norm(e[0, :n * m])
+    assert last >= best * (1 - 1e-12)
+    assert np.isclose(last, best, rtol=1e-6)
+
+
+def test_gram_schmidt_zero_column_is_finite():
+    P = np.zeros((5, 2))
+    P[:, 0] = 1.0
+    out = orc.gram_schmidt(P, 1e-8)
+    assert np.all(np.isfinite(out)) and np.all(out[:, 1] == 0)
+
+
+# ------------------------------------------------------------------ TopK
+def _order_key(v, i):
+    bits = np.float32(v).view(np.uint32) & np.uint32(0x7FFFFFFF)
+    return (-int(bits), i)
+
+
+def _brute_force_topk(vals, k):
+    """The kept set is the unique size-k subset in which every member precedes every
+    non-member in the order (larger |v| first, then lower index): enumerate subsets."""
+    n = len(vals)
+    found = None
+    for S in itertools.combinations(range(n), k):
+        rest = [i for i in range(n) if i not in S]
+        worst_in = max(_order_key(vals[i], i) for i in S)
+        if all(worst_in < _order_key(vals[j], j) for j in rest):
+            assert found is None
+            found = S
+    return np.array(found)
+
+
+def test_topk_brute_force_tiny():
+    rng = np.random.default_rng(7)
+    for trial in range(30):
+        n = int(rng.integers(1, 11))
+        k = int(rng.integers(1, n + 1))
+        v = rng.integers(-3, 4, n).astype(np.float32) * np.float32(0.5)  # many ties, zeros, signs
+        got = orc.topk_select(v, k)
+        assert np.array_equal(got, _brute_force_topk(v, k)), (v, k)
+
+
+def test_topk_equals_python_sort():
+    rng = np.random.default_rng(8)
+    v = rng.standard_normal(500).astype(np.float32)
+    v[rng.integers(0, 500, 60)] = np.float32(0.75)
+    v[rng.integers(0, 500, 60)] = np.float32(-0.75)
+    v[rng.integers(0, 500, 20)] = np.float32(-0.0)
+    for k in (1, 7, 50, 137, 499, 500):
+        want = sorted(sorted(range(500), key=lambda i: _order_key(v[i], i))[:k])
+        assert np.array_equal(orc.topk_select(v, k), np.array(want))
+
+
+def test_topk_degenerate_inputs():
+    assert np.array_equal(orc.topk_select(np.zeros(10, np.float32), 4), np.arange(4))
+    assert np.array_equal(orc.topk_select(np.full(10, -2.5, np.float32), 3), np.arange(3))
+    v = np.array([0.0, -0.0, 0.0, 1.0], np.float32)
+    assert np.array_equal(orc.topk_select(v, 3), np.array([0, 1, 3]))  # -0.0 ties with +0.0
+    assert np.array_equal(orc.topk_select(v, 4), np.arange(4))
+    assert orc.topk_count(1728, 100) == 17 and orc.topk_count(50, 100) == 1 and orc.topk_count(21630700, 1000) == 2163070
+
+
+def test_topk_step_invariants():
+    rng = np.random.default_rng(9)
+    table = wl.make_table([("a", (13, 17)), ("v", (6,)), ("b", (8, 25))])
+    layers = _layers(table)
+    W = 3
+    grads = np.zeros((W, table.stride), np.float32)
+    err = np.zeros((W, table.stride), np.float32)
+    for (off, r, c, k) in layers:
+        grads[:, off:off + r * c] = rng.standard_normal((W, r * c))
+        if k == orc.MATRIX:
+            err[:, off:off + r * c] = 0.5 * rng.standard_normal((W, r * c))
+    grads[:, 3] = grads[:, 40]  # some exact ties in the gradient
+    level = [1, 0, 0]
+    vals, idx, counts, out, e = orc.topk_step(grads, err, level, layers, 1000, 100)
+    for l, (off, r, c, kind) in enumerate(layers):
+        size = r * c
+        if kind == orc.VECTOR:
+            assert np.allclose(out[off:off + size], grads[:, off:off + size].astype(np.float64).mean(0))
+            continue
+        k = max(1, size * (1000 if level[l] else 100) // 10000)
+        acc = np.zeros(size)
+        for w in range(W):
+            M = grads[w, off:off + size] + err[w, off:off + size]   # fp32 add
+            assert M.dtype == np.float32
+            assert counts[w, l] == k == len(idx[w][l]) == len(vals[w][l])
+            assert np.all(np.diff(idx[w][l]) > 0)
+            kept = np.zeros(size, bool); kept[idx[w][l]] = True
+            assert np.abs(M[kept]).min() >= np.abs(M[~kept]).max()
+            # bitwise error-feedback invariant: scatter(idx, val) + e' == M
+            rec = e[w, off:off + size].copy()
+            assert np.all(rec[kept].view(np.uint32) == 0)           # +0.0 exactly
+            rec[idx[w][l]] = vals[w][l]
+            assert np.array_equal(rec.view(np.uint32), M.view(np.uint32))
+            acc[idx[w][l]] += vals[w][l].astype(np.float64)
+        assert np.allclose(out[off:off + size], acc / W, rtol=0, atol=1e-15)
+
+
+def test_topk_tie_at_threshold_keeps_lower_indices():
+    v = np.array([1, 5, 1, 1, 7, 1, 1], np.float32)
+    v[2] = -1
+    assert np.array_equal(orc.topk_select(v, 4), np.array([0, 1, 2, 4]))
+
+
+# ------------------------------------------------------------------ tables of the paper
+def _golden():
+    rows, params = [], []
+    with open(GOLDEN) as f:
+        for line in f:
+            line = line.strip()
+            if not line or line.startswith("#"):
+                continue
+            t = line.split()
+            if t[0] == "params":
+                params.append((t[1], int(t[2]), int(t[3])))
+            else:
+                rows.append((t[0], int(t[1]), t[2], t[3], float(t[4]), t[5]))
+    return rows, params
+
+
+def _table(model, classes):
+    return wl.make_table(wl.shapes_resnet18(classes) if model == "resnet18" else wl.shapes_vgg19bn(classes))
+
+
+def test_parameter_totals_match_appendix_g():
+    _, params = _golden()
+    assert len(params) == 3
+    for model, classes, total in params:
+        assert _table(model, classes).n_params == total
+    assert wl.make_table(wl.shapes_lstm()).n_params == 50065078
+    t = _table("resnet18", 100)
+    assert int((t.kind == wl.MATRIX).sum()) == 21 and int((t.kind == wl.VECTOR).sum()) == 41
+
+
+def test_data_sent_matches_tables():
+    rows, _ = _golden()
+    assert len(rows) == 7
+    iters = 300 * 98
+    for model, classes, comp, setting, value, unit in rows:
+        table = _table(model, classes)
+        layers = _layers(table)
+        L = len(layers)
+        if comp == "powersgd":
+            r = int(setting[4:])
+            per_it = orc.floats_sent_per_iteration(layers, [1] * L, "powersgd", 4, rank_low=r, rank_high=r)
+            got = per_it * iters / 1e6
+            assert abs(got - value) <= 0.11, (model, setting, got, value)  # printed to 0.1 M floats
+        else:
+            per_it = orc.floats_sent_per_iteration(layers, [1] * L, "topk", 4, topk_low_bp=1000)
+            got = per_it * iters / 1e9
+            assert abs(got - value) / value < 1e-3, (got, value)
