@@ -1,0 +1,164 @@
+/*
+ * acc.h -- C ABI of the Accordion gradient-compression step for NVIDIA B200 (sm_100a).
+ *
+ * The library runs, for W simulated data-parallel workers whose gradients sit in one GPU's
+ * memory, the per-iteration step that Accordion (arXiv 2010.16248) drives:
+ *
+ *   - error-feedback accumulation          M_w = g_w + e_w           (the "memory term", Section 5.2)
+ *   - gradient accumulation + layer norms  for the critical-regime test (Section 4.2)
+ *   - the regime test itself               Algorithm 1
+ *   - the compressor at the chosen level   PowerSGD rank r, or TopK K%   (Section 5, first paragraph)
+ *   - the mean over workers of the compressed gradients   (update rule of Section 3)
+ *
+ * General rules, valid for every entry point unless it says otherwise:
+ *   * Pointers named in "Device pointers" below are DEVICE pointers owned by the caller; the library
+ *     never allocates or frees device memory.  `cfg`, `layers`, and every `int64_t*` / `size_t*`
+ *     out-parameter are HOST pointers.
+ *   * Every device buffer must be 16-byte aligned (ACC_EALIGN otherwise).
+ *   * Calls are asynchronous on `stream` (a cudaStream_t passed as void*; NULL = default stream),
+ *     never synchronise the device, and return an int status: ACC_OK or one of the ACC_E* codes.
+ *     Calls on one context must be ordered on one stream (or otherwise serialised by the caller):
+ *     they share the context's scratch memory.
+ *   * Layout.  All per-parameter buffers use one flat per-worker layout given by the layer table:
+ *     layer l occupies elements [offset_l, offset_l + rows_l*cols_l) of each worker's slice, each
+ *     offset a multiple of 4 elements; worker w's slice starts at element w*worker_stride
+ *     (worker_stride a multiple of 4).  MATRIX layers are row-major rows x cols (convolution weights
+ *     viewed as out x (in*k*k), the view that reproduces the "Data Sent" columns of Tables 1-2);
+ *     VECTOR layers (1-D tensors) are never compressed and carry no error memory (Appendix F).
+ *   * level[l] = 1 selects the low-compression level l_low (rank_low / topk_low_bp),
+ *     level[l] = 0 the high-compression level l_high (rank_high / topk_high_bp)  (Section 4.2).
+ */
+#ifndef ACC_H_
+#define ACC_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define ACC_OK 0
+#define ACC_EINVAL 1      /* bad argument / inconsistent configuration            */
+#define ACC_EALIGN 2      /* a pointer, offset or stride is not 16-byte aligned    */
+#define ACC_EWORKSPACE 3  /* workspace missing or too small                        */
+#define ACC_ECUDA 4       /* a CUDA runtime call or kernel launch reported an error */
+
+#define ACC_MATRIX 0
+#define ACC_VECTOR 1
+#define ACC_MAX_RANK 4    /* ranks are interleaved in groups of ACC_MAX_RANK floats  */
+
+#define ACC_COMPRESSOR_POWERSGD 0
+#define ACC_COMPRESSOR_TOPK 1
+
+typedef struct {
+  int64_t offset; /* first element of the layer inside a worker's slice; multiple of 4 */
+  int32_t rows;   /* MATRIX: rows; VECTOR: 1                                           */
+  int32_t cols;   /* MATRIX: cols; VECTOR: length                                      */
+  int32_t kind;   /* ACC_MATRIX or ACC_VECTOR                                          */
+  int32_t reserved;
+} acc_layer_desc;
+
+typedef struct {
+  int32_t n_workers;            /* W >= 1                                                        */
+  int32_t n_layers;             /* L >= 1                                                        */
+  const acc_layer_desc* layers; /* HOST array [L], copied by acc_create                          */
+  int64_t worker_stride;        /* elements between consecutive workers' slices                  */
+  int32_t rank_low, rank_high;  /* PowerSGD ranks, 1 <= rank_high <= rank_low <= ACC_MAX_RANK    */
+  int32_t topk_low_bp;          /* TopK fraction at l_low in basis points (1000 = 10 %)          */
+  int32_t topk_high_bp;         /* TopK fraction at l_high; 1 <= high <= low <= 10000            */
+  float eta;                    /* detection threshold of Algorithm 1 (the paper uses 0.5)       */
+  float gs_eps;                 /* Gram-Schmidt divides by (norm + gs_eps)                       */
+  int32_t decider;              /* worker whose raw gradient is accumulated for the detector     */
+  int32_t flags;                /* must be 0                                                     */
+} acc_config;
+
+typedef struct acc_ctx acc_ctx;
+
+/* Bytes of device scratch memory acc_create needs for this configuration (HOST out-parameter). */
+int acc_workspace_bytes(const acc_config* cfg, size_t* bytes);
+
+/* Validates cfg, copies the layer table and the launch tables into `workspace` (DEVICE memory of at
+ * least acc_workspace_bytes bytes, 256-byte aligned, owned by the caller and kept alive until
+ * acc_destroy) and returns a context.  Synchronous (blocking copies on the current device).        */
+int acc_create(const acc_config* cfg, void* workspace, size_t workspace_bytes, acc_ctx** out);
+int acc_destroy(acc_ctx* ctx);
+
+/* Factor layout of PowerSGD.  q holds, for every MATRIX layer, cols_l rows of ACC_MAX_RANK floats
+ * (row j = Q[j, 0..3], rank-interleaved); p_hat holds rows_l rows of ACC_MAX_RANK floats.  The block
+ * of layer l starts at row q_row[l] / p_row[l] (-1 for VECTOR layers).  Any out-pointer may be NULL.
+ * q_rows / p_rows: total rows, i.e. the buffers hold 4*q_rows and 4*p_rows floats.                 */
+int acc_factor_layout(const acc_ctx* ctx, int64_t* q_row /*[L]*/, int64_t* p_row /*[L]*/,
+                      int64_t* q_rows, int64_t* p_rows);
+
+/* Packed TopK layout.  A worker's packed region has `capacity` entries; the segment of MATRIX layer l
+ * starts at seg_offset[l] (-1 for VECTOR layers) and has room for k_low[l] entries.  Worker w's
+ * region starts at entry w*capacity of `vals` and `idx`.                                          */
+int acc_topk_layout(const acc_ctx* ctx, int64_t* seg_offset /*[L]*/, int64_t* k_low /*[L]*/,
+                    int64_t* k_high /*[L]*/, int64_t* capacity);
+
+/* Error-feedback accumulation on its own (Section 5.2: compressors run "with memory"):
+ *   err_w <- g_w + err_w  on MATRIX layers, in fp32 (one IEEE add), for every worker;
+ *   delta <- delta + g_decider on every layer when delta != NULL (gradient accumulation of the
+ *   detector, Section 4.2 "Computational and memory overhead").
+ * Device pointers: grads [W][worker_stride] (read), err [W][worker_stride] (in: e, out: M),
+ * delta [worker_stride] or NULL.                                                                   */
+int acc_error_feedback(acc_ctx* ctx, const float* grads, float* err, float* delta, void* stream);
+
+/* Per-layer squared L2 norms (Section 4.2: "After each epoch, norms are calculated"):
+ *   norm2[b*L + l] = sum of squares of layer l in buffer b, b < n_bufs <= W, accumulated in fp64 in a
+ *   fixed order (bit-reproducible).  Device pointers: buf [n_bufs][buf_stride] (read),
+ *   norm2 [n_bufs*L] doubles (written).                                                            */
+int acc_layer_norms(acc_ctx* ctx, const float* buf, int64_t buf_stride, int32_t n_bufs, double* norm2,
+                    void* stream);
+
+/* Critical-regime test, Algorithm 1, per layer, on the device:
+ *   a = sqrt(norm2_prev[l]), b = sqrt(norm2_curr[l]);
+ *   level[l] = 1 (l_low)  if norm2_prev[l] < 0 (no earlier window), or |a - b| >= eta*a, or
+ *              lr_next < lr_curr;  else 0 (l_high).
+ *   Then norm2_prev[l] <- norm2_curr[l] and, when delta != NULL, delta <- 0 (new window).
+ * Device pointers: norm2_curr [L] doubles (read), norm2_prev [L] doubles (in/out), level [L] bytes
+ * (written), delta [worker_stride] or NULL (cleared).                                              */
+int acc_detect_regime(acc_ctx* ctx, const double* norm2_curr, double* norm2_prev, float lr_curr,
+                      float lr_next, uint8_t* level, float* delta, void* stream);
+
+/* One PowerSGD step with error feedback (the compressor of Section 5.2, applied per MATRIX layer at
+ * rank r = rank_low if level[l] else rank_high), all workers, mean over workers (Section 3):
+ *   M_w = g_w + e_w;  P = mean_w M_w Q[:, :r];  P^ = modified Gram-Schmidt(P) (divide by norm + gs_eps);
+ *   Q[:, :r] <- mean_w M_w^T P^;  A = P^ Q[:, :r]^T;  out[l] = A;  e_w <- M_w - A.
+ *   VECTOR layers: out[l] = mean_w g_w[l].  delta != NULL: delta += g_decider (all layers).
+ * Columns r..3 of q and p_hat keep their previous contents.
+ * Device pointers: grads [W][worker_stride] (read), err [W][worker_stride] (in/out),
+ * q [4*q_rows] (in: warm start, out: new Q), p_hat [4*p_rows] (out: P^), level [L] bytes (read),
+ * out [worker_stride] (written), delta [worker_stride] or NULL.                                    */
+int acc_powersgd_step(acc_ctx* ctx, const float* grads, float* err, float* q, float* p_hat,
+                      const uint8_t* level, float* out, float* delta, void* stream);
+
+/* One TopK step with error feedback (the sparsifier of Section 5.3, per MATRIX layer and worker,
+ * k = max(1, floor(rows*cols*K_bp/10000)), K_bp = topk_low_bp if level[l] else topk_high_bp):
+ *   M_w = g_w + e_w (fp32);  keep the k entries of largest |M_w| -- compared as 31-bit patterns,
+ *   ties broken by lower index --;  vals/idx <- kept values (bit copies) and layer-local indices in
+ *   ascending index order;  counts[w*L + l] = k;  e_w <- M_w with the kept entries set to +0.0;
+ *   out[l] = (1/W) sum_w scatter(idx_w, val_w)  (workers added in order, bit-reproducible).
+ *   VECTOR layers: out[l] = mean_w g_w[l], counts = 0.  delta != NULL: delta += g_decider.
+ * Device pointers: grads, err, level, out, delta as above; vals [W*capacity] floats,
+ * idx [W*capacity] int32, counts [W*L] int32 (see acc_topk_layout).                                */
+int acc_topk_step(acc_ctx* ctx, const float* grads, float* err, const uint8_t* level, float* vals,
+                  int32_t* idx, int32_t* counts, float* out, float* delta, void* stream);
+
+/* Floats one iteration communicates at the given HOST level array, following the "Data Sent"
+ * accounting of Tables 1-4: PowerSGD r*(rows+cols) per MATRIX layer, TopK 2*k*W per MATRIX layer
+ * (values + indices gathered from every worker), plus every VECTOR element once.  Returns -1 on a
+ * bad argument.  Host-only helper.                                                                 */
+int64_t acc_floats_sent(const acc_config* cfg, const uint8_t* level_host, int32_t compressor);
+
+/* Number of kernels the last *_step / acc_error_feedback / acc_layer_norms / acc_detect_regime call
+ * on this context launched (for launch accounting in benchmarks).                                  */
+int32_t acc_last_launch_count(const acc_ctx* ctx);
+
+const char* acc_strerror(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ACC_H_ */

@@ -1,0 +1,215 @@
+"""ctypes binding of the C-ABI library (include/acc.h): argument marshalling only.
+
+Every step of the path runs in the library's CUDA kernels.  torch is used for device
+memory and streams.  There is no CPU fallback: loading fails loudly when the library
+has not been built, and every call checks that its tensors live on a CUDA device.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional
+
+import numpy as np
+import torch
+
+from . import build as _build
+
+ACC_OK = 0
+ACC_MATRIX, ACC_VECTOR = 0, 1
+ACC_MAX_RANK = 4
+POWERSGD, TOPK = 0, 1
+
+
+class AccError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {lib().acc_strerror(status).decode()} (status {status})")
+
+
+class acc_layer_desc(C.Structure):
+    _fields_ = [("offset", C.c_int64), ("rows", C.c_int32), ("cols", C.c_int32), ("kind", C.c_int32),
+                ("reserved", C.c_int32)]
+
+
+class acc_config(C.Structure):
+    _fields_ = [("n_workers", C.c_int32), ("n_layers", C.c_int32), ("layers", C.POINTER(acc_layer_desc)),
+                ("worker_stride", C.c_int64), ("rank_low", C.c_int32), ("rank_high", C.c_int32),
+                ("topk_low_bp", C.c_int32), ("topk_high_bp", C.c_int32), ("eta", C.c_float),
+                ("gs_eps", C.c_float), ("decider", C.c_int32), ("flags", C.c_int32)]
+
+
+EXPORTS = ["acc_workspace_bytes", "acc_create", "acc_destroy", "acc_factor_layout", "acc_topk_layout",
+           "acc_error_feedback", "acc_layer_norms", "acc_detect_regime", "acc_powersgd_step", "acc_topk_step",
+           "acc_floats_sent", "acc_last_launch_count", "acc_strerror"]
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """Loads libacc.so (built in-tree by ``build.build_library``); raises if it is missing."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    path = _build.LIB_PATH
+    if not os.path.exists(path):
+        raise RuntimeError(f"{path} not found: build it with `python -m paper_2010_16248_b200.build` "
+                           "(there is no CPU fallback)")
+    L = C.CDLL(path)
+    vp, i32, i64, f32 = C.c_void_p, C.c_int32, C.c_int64, C.c_float
+    L.acc_workspace_bytes.argtypes = [C.POINTER(acc_config), C.POINTER(C.c_size_t)]
+    L.acc_create.argtypes = [C.POINTER(acc_config), vp, C.c_size_t, C.POINTER(vp)]
+    L.acc_destroy.argtypes = [vp]
+    L.acc_factor_layout.argtypes = [vp, C.POINTER(i64), C.POINTER(i64), C.POINTER(i64), C.POINTER(i64)]
+    L.acc_topk_layout.argtypes = [vp, C.POINTER(i64), C.POINTER(i64), C.POINTER(i64), C.POINTER(i64)]
+    L.acc_error_feedback.argtypes = [vp, vp, vp, vp, vp]
+    L.acc_layer_norms.argtypes = [vp, vp, i64, i32, vp, vp]
+    L.acc_detect_regime.argtypes = [vp, vp, vp, f32, f32, vp, vp, vp]
+    L.acc_powersgd_step.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp]
+    L.acc_topk_step.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
+    L.acc_floats_sent.argtypes = [C.POINTER(acc_config), C.POINTER(C.c_uint8), i32]
+    L.acc_floats_sent.restype = i64
+    L.acc_last_launch_count.argtypes = [vp]
+    L.acc_last_launch_count.restype = i32
+    L.acc_strerror.argtypes = [C.c_int]
+    L.acc_strerror.restype = C.c_char_p
+    for name in EXPORTS:
+        if name not in ("acc_floats_sent", "acc_last_launch_count", "acc_strerror"):
+            getattr(L, name).restype = C.c_int
+    _lib = L
+    return L
+
+
+def make_config(table, n_workers, rank_low=2, rank_high=1, topk_low_bp=1000, topk_high_bp=100, eta=0.5,
+                gs_eps=1e-8, decider=0, worker_stride=None):
+    """Builds an ``acc_config`` (plus the array it points to) from a workloads.LayerTable."""
+    L = table.n_layers
+    arr = (acc_layer_desc * L)()
+    for l in range(L):
+        arr[l].offset = int(table.offset[l]); arr[l].rows = int(table.rows[l]); arr[l].cols = int(table.cols[l])
+        arr[l].kind = int(table.kind[l]); arr[l].reserved = 0
+    cfg = acc_config(n_workers, L, arr, int(worker_stride if worker_stride is not None else table.stride),
+                     rank_low, rank_high, topk_low_bp, topk_high_bp, eta, gs_eps, decider, 0)
+    cfg._keepalive = arr
+    return cfg
+
+
+def acc_floats_sent(cfg: acc_config, level, compressor: int) -> int:
+    lv = (C.c_uint8 * cfg.n_layers)(*[int(x) for x in level])
+    return int(lib().acc_floats_sent(C.byref(cfg), lv, compressor))
+
+
+def _ptr(t: Optional[torch.Tensor], dtype=None) -> Optional[int]:
+    if t is None:
+        return None
+    if not t.is_cuda:
+        raise ValueError("expected a CUDA tensor (the library has no CPU path)")
+    if not t.is_contiguous():
+        raise ValueError("expected a contiguous tensor")
+    if dtype is not None and t.dtype != dtype:
+        raise ValueError(f"expected dtype {dtype}, got {t.dtype}")
+    return t.data_ptr()
+
+
+def _stream(stream) -> Optional[int]:
+    s = torch.cuda.current_stream() if stream is None else stream
+    return s.cuda_stream or None
+
+
+class Context:
+    """Owns the workspace tensor and the ``acc_ctx``; methods mirror the C entry points."""
+
+    def __init__(self, table, n_workers, device="cuda", **cfg_kwargs):
+        self.table = table
+        self.device = torch.device(device)
+        self.cfg = make_config(table, n_workers, **cfg_kwargs)
+        self.n_workers, self.n_layers, self.stride = n_workers, table.n_layers, int(self.cfg.worker_stride)
+        L = lib()
+        nbytes = C.c_size_t(0)
+        st = L.acc_workspace_bytes(C.byref(self.cfg), C.byref(nbytes))
+        if st != ACC_OK:
+            raise AccError(st, "acc_workspace_bytes")
+        self.workspace_bytes = int(nbytes.value)
+        with torch.cuda.device(self.device):
+            self.workspace = torch.zeros(max(self.workspace_bytes, 256), dtype=torch.uint8, device=self.device)
+            h = C.c_void_p()
+            st = L.acc_create(C.byref(self.cfg), self.workspace.data_ptr(), self.workspace_bytes, C.byref(h))
+        if st != ACC_OK:
+            raise AccError(st, "acc_create")
+        self._h = h
+        n = self.n_layers
+        qr, pr = (C.c_int64 * n)(), (C.c_int64 * n)()
+        qn, pn = C.c_int64(), C.c_int64()
+        L.acc_factor_layout(self._h, qr, pr, C.byref(qn), C.byref(pn))
+        self.q_row, self.p_row = np.array(qr[:], np.int64), np.array(pr[:], np.int64)
+        self.q_rows, self.p_rows = int(qn.value), int(pn.value)
+        so, kl, kh, cap = (C.c_int64 * n)(), (C.c_int64 * n)(), (C.c_int64 * n)(), C.c_int64()
+        L.acc_topk_layout(self._h, so, kl, kh, C.byref(cap))
+        self.seg_offset, self.k_low, self.k_high = (np.array(a[:], np.int64) for a in (so, kl, kh))
+        self.capacity = int(cap.value)
+
+    def close(self):
+        if getattr(self, "_h", None):
+            lib().acc_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def _check(self, st, where):
+        if st != ACC_OK:
+            raise AccError(st, where)
+
+    # --- entry points -------------------------------------------------------------------------
+    def acc_error_feedback(self, grads, err, delta=None, stream=None):
+        self._check(lib().acc_error_feedback(self._h, _ptr(grads, torch.float32), _ptr(err, torch.float32),
+                                             _ptr(delta, torch.float32), _stream(stream)), "acc_error_feedback")
+
+    def acc_layer_norms(self, buf, n_bufs, norm2, buf_stride=None, stream=None):
+        stride = int(buf_stride if buf_stride is not None else self.stride)
+        self._check(lib().acc_layer_norms(self._h, _ptr(buf, torch.float32), stride, n_bufs,
+                                          _ptr(norm2, torch.float64), _stream(stream)), "acc_layer_norms")
+
+    def acc_detect_regime(self, norm2_curr, norm2_prev, lr_curr, lr_next, level, delta=None, stream=None):
+        self._check(lib().acc_detect_regime(self._h, _ptr(norm2_curr, torch.float64), _ptr(norm2_prev, torch.float64),
+                                            float(lr_curr), float(lr_next), _ptr(level, torch.uint8),
+                                            _ptr(delta, torch.float32), _stream(stream)), "acc_detect_regime")
+
+    def acc_powersgd_step(self, grads, err, q, p_hat, level, out, delta=None, stream=None):
+        self._check(lib().acc_powersgd_step(self._h, _ptr(grads, torch.float32), _ptr(err, torch.float32),
+                                            _ptr(q, torch.float32), _ptr(p_hat, torch.float32),
+                                            _ptr(level, torch.uint8), _ptr(out, torch.float32),
+                                            _ptr(delta, torch.float32), _stream(stream)), "acc_powersgd_step")
+
+    def acc_topk_step(self, grads, err, level, vals, idx, counts, out, delta=None, stream=None):
+        self._check(lib().acc_topk_step(self._h, _ptr(grads, torch.float32), _ptr(err, torch.float32),
+                                        _ptr(level, torch.uint8), _ptr(vals, torch.float32), _ptr(idx, torch.int32),
+                                        _ptr(counts, torch.int32), _ptr(out, torch.float32),
+                                        _ptr(delta, torch.float32), _stream(stream)), "acc_topk_step")
+
+    def last_launch_count(self) -> int:
+        return int(lib().acc_last_launch_count(self._h))
+
+    # --- buffer helpers (allocation and layout conversion only) -------------------------------
+    def new_q(self, q_list=None):
+        """Device q buffer ``[q_rows, 4]``; filled from per-layer ``[m, r]`` tensors when given."""
+        q = torch.zeros(self.q_rows, ACC_MAX_RANK, dtype=torch.float32, device=self.device)
+        if q_list is not None:
+            for l, ql in enumerate(q_list):
+                if ql is not None:
+                    r0 = int(self.q_row[l])
+                    q[r0:r0 + ql.shape[0], :ql.shape[1]] = ql.to(self.device)
+        return q
+
+    def new_p(self):
+        return torch.zeros(self.p_rows, ACC_MAX_RANK, dtype=torch.float32, device=self.device)
+
+    def new_topk_buffers(self):
+        W = self.n_workers
+        vals = torch.zeros(W * self.capacity, dtype=torch.float32, device=self.device)
+        idx = torch.zeros(W * self.capacity, dtype=torch.int32, device=self.device)
+        counts = torch.zeros(W * self.n_layers, dtype=torch.int32, device=self.device)
+        return vals, idx, counts

@@ -1,0 +1,295 @@
+// C-ABI entry points: configuration checks, launch-table planning, workspace layout.
+#include <algorithm>
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "acc_internal.cuh"
+
+namespace acc {
+
+static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+static int topk_count(long long size, int bp) {
+  long long k = size * (long long)bp / 10000;
+  return (int)std::max<long long>(1, k);
+}
+
+static int validate(const acc_config* cfg) {
+  if (!cfg || !cfg->layers) return ACC_EINVAL;
+  if (cfg->n_workers < 1 || cfg->n_workers > 1024 || cfg->n_layers < 1) return ACC_EINVAL;
+  if (cfg->flags != 0) return ACC_EINVAL;
+  if (cfg->rank_high < 1 || cfg->rank_low < cfg->rank_high || cfg->rank_low > ACC_MAX_RANK) return ACC_EINVAL;
+  if (cfg->topk_high_bp < 1 || cfg->topk_low_bp < cfg->topk_high_bp || cfg->topk_low_bp > 10000) return ACC_EINVAL;
+  if (!(cfg->eta >= 0.f) || !(cfg->gs_eps >= 0.f)) return ACC_EINVAL;
+  if (cfg->decider < 0 || cfg->decider >= cfg->n_workers) return ACC_EINVAL;
+  if (cfg->worker_stride < 4) return ACC_EINVAL;
+  if (cfg->worker_stride % 4 != 0) return ACC_EALIGN;
+  long long prev_end = 0;
+  long long rows_total = 0, cols_total = 0;
+  for (int l = 0; l < cfg->n_layers; ++l) {
+    const acc_layer_desc& d = cfg->layers[l];
+    if (d.kind != ACC_MATRIX && d.kind != ACC_VECTOR) return ACC_EINVAL;
+    if (d.rows < 1 || d.cols < 1) return ACC_EINVAL;
+    if (d.kind == ACC_VECTOR && d.rows != 1) return ACC_EINVAL;
+    if (d.offset < 0) return ACC_EINVAL;
+    if (d.offset % 4 != 0) return ACC_EALIGN;
+    long long size = (long long)d.rows * d.cols;
+    if (size >= (1ll << 31) - kTile) return ACC_EINVAL;          // layer-local indices are int32
+    if (d.offset < prev_end) return ACC_EINVAL;                  // layers in order, no overlap
+    prev_end = d.offset + size;
+    if (prev_end > cfg->worker_stride) return ACC_EINVAL;
+    if (d.kind == ACC_MATRIX) { rows_total += d.rows; cols_total += d.cols; }
+  }
+  if (rows_total >= (1ll << 31) || cols_total >= (1ll << 31)) return ACC_EINVAL;
+  return ACC_OK;
+}
+
+static int make_plan(const acc_config* cfg, Plan& p) {
+  int st = validate(cfg);
+  if (st != ACC_OK) return st;
+  const int L = cfg->n_layers, W = cfg->n_workers;
+  p.layers.resize(L);
+  for (int l = 0; l < L; ++l) {
+    const acc_layer_desc& d = cfg->layers[l];
+    DevLayer& o = p.layers[l];
+    memset(&o, 0, sizeof(o));
+    o.offset = d.offset; o.rows = d.rows; o.cols = d.cols; o.kind = d.kind;
+    o.q_row = o.p_row = o.mat = -1; o.seg_off = -1; o.part_base = -1;
+    o.vec = (d.cols % 4 == 0) ? 4 : (d.cols % 2 == 0) ? 2 : 1;
+    const long long size = (long long)d.rows * d.cols;
+    // flat tiles
+    o.tile0 = (int)p.tiles.size();
+    for (long long e = 0; e < size; e += kTile) {
+      Tile t{l, (int)e, (int)std::min<long long>(kTile, size - e)};
+      if (d.kind == ACC_VECTOR) p.vec_tiles.push_back((int)p.tiles.size());
+      p.tiles.push_back(t);
+    }
+    o.ntiles = (int)p.tiles.size() - o.tile0;
+    if (d.kind != ACC_MATRIX) continue;
+    o.mat = p.n_mat++;
+    p.mat_layers.push_back(l);
+    o.q_row = (int)p.q_rows; p.q_rows += d.cols;
+    o.p_row = (int)p.p_rows; p.p_rows += d.rows;
+    o.k_low = topk_count(size, cfg->topk_low_bp);
+    o.k_high = topk_count(size, cfg->topk_high_bp);
+    o.seg_off = p.capacity; p.capacity += o.k_low;
+    // row slabs of the row-wise passes: about kRowSlabElems elements per worker, whole rows,
+    // a multiple of 8 rows (one row per warp of a 256-thread block) where the layer allows it
+    int rs = std::max(1, kRowSlabElems / d.cols);
+    if (rs >= 8) rs = rs / 8 * 8;
+    rs = std::min(rs, d.rows);
+    for (int r0 = 0; r0 < d.rows; r0 += rs) p.row_items.push_back(RowItem{l, r0, std::min(rs, d.rows - r0)});
+    // row slabs x column blocks of the Q-partial pass (each thread owns `vec` adjacent columns)
+    o.slab_rows = std::min(d.rows, std::max(32, (d.rows + 127) / 128));
+    o.nslabs = (d.rows + o.slab_rows - 1) / o.slab_rows;
+    o.part_base = p.part_f4; p.part_f4 += (long long)o.nslabs * d.cols;
+    const int cb = kColBlockThreads * o.vec;
+    for (int s = 0; s < o.nslabs; ++s)
+      for (int c0 = 0; c0 < d.cols; c0 += cb)
+        p.col_items.push_back(ColItem{l, s, s * o.slab_rows, std::min(o.slab_rows, d.rows - s * o.slab_rows), c0});
+  }
+  // biggest row items first so that the tail of the grid is made of small ones
+  std::stable_sort(p.row_items.begin(), p.row_items.end(), [&](const RowItem& a, const RowItem& b) {
+    return (long long)a.nrows * p.layers[a.layer].cols > (long long)b.nrows * p.layers[b.layer].cols;
+  });
+  const size_t nt = p.tiles.size();
+  const size_t seg = (size_t)W * std::max(p.n_mat, 1);
+  size_t o = 0;
+  auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes, 256); return at; };
+  p.o_layers = take(sizeof(DevLayer) * L);
+  p.o_row_items = take(sizeof(RowItem) * std::max<size_t>(1, p.row_items.size()));
+  p.o_col_items = take(sizeof(ColItem) * std::max<size_t>(1, p.col_items.size()));
+  p.o_tiles = take(sizeof(Tile) * nt);
+  p.o_mat_layers = take(sizeof(int) * std::max<size_t>(1, p.mat_layers.size()));
+  p.o_vec_tiles = take(sizeof(int) * std::max<size_t>(1, p.vec_tiles.size()));
+  p.o_part = take(sizeof(float4) * std::max<long long>(1, p.part_f4));
+  p.o_norm_part = take(sizeof(double) * (size_t)W * nt);
+  p.o_hist = o;
+  take(sizeof(unsigned) * seg * kBins1);
+  take(sizeof(unsigned) * seg * kBins2);
+  take(sizeof(unsigned) * seg * kBins3);
+  p.hist_bytes = o - p.o_hist;
+  p.o_sel = take(sizeof(Select) * seg);
+  p.o_tile_cnt = take(sizeof(int2) * (size_t)W * nt);
+  p.o_tile_h3 = take(sizeof(unsigned short) * (size_t)W * nt * kBins3);
+  p.o_tile_pre = take(sizeof(int2) * (size_t)W * nt);
+  p.total = o;
+  return ACC_OK;
+}
+
+static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+}  // namespace acc
+
+using namespace acc;
+
+extern "C" {
+
+int acc_workspace_bytes(const acc_config* cfg, size_t* bytes) {
+  if (!bytes) return ACC_EINVAL;
+  Plan p;
+  int st = make_plan(cfg, p);
+  if (st != ACC_OK) return st;
+  *bytes = p.total;
+  return ACC_OK;
+}
+
+int acc_create(const acc_config* cfg, void* workspace, size_t workspace_bytes, acc_ctx** out) {
+  if (!out) return ACC_EINVAL;
+  *out = nullptr;
+  acc_ctx* ctx = new (std::nothrow) acc_ctx();
+  if (!ctx) return ACC_EINVAL;
+  int st = make_plan(cfg, ctx->plan);
+  if (st != ACC_OK) { delete ctx; return st; }
+  if (!workspace || workspace_bytes < ctx->plan.total) { delete ctx; return ACC_EWORKSPACE; }
+  if (reinterpret_cast<uintptr_t>(workspace) & 255u) { delete ctx; return ACC_EALIGN; }
+  ctx->cfg = *cfg;
+  ctx->host_layers.assign(cfg->layers, cfg->layers + cfg->n_layers);
+  ctx->cfg.layers = ctx->host_layers.data();
+  ctx->ws = static_cast<char*>(workspace);
+  Plan& p = ctx->plan;
+  char* ws = ctx->ws;
+  ctx->d_layers = reinterpret_cast<DevLayer*>(ws + p.o_layers);
+  ctx->d_row_items = reinterpret_cast<RowItem*>(ws + p.o_row_items);
+  ctx->d_col_items = reinterpret_cast<ColItem*>(ws + p.o_col_items);
+  ctx->d_tiles = reinterpret_cast<Tile*>(ws + p.o_tiles);
+  ctx->d_mat_layers = reinterpret_cast<int*>(ws + p.o_mat_layers);
+  ctx->d_vec_tiles = reinterpret_cast<int*>(ws + p.o_vec_tiles);
+  ctx->d_part = reinterpret_cast<float4*>(ws + p.o_part);
+  ctx->d_norm_part = reinterpret_cast<double*>(ws + p.o_norm_part);
+  const size_t seg = (size_t)cfg->n_workers * std::max(p.n_mat, 1);
+  ctx->d_hist1 = reinterpret_cast<unsigned*>(ws + p.o_hist);
+  ctx->d_hist2 = ctx->d_hist1 + (align_up(sizeof(unsigned) * seg * kBins1, 256) / sizeof(unsigned));
+  ctx->d_hist3 = ctx->d_hist2 + (align_up(sizeof(unsigned) * seg * kBins2, 256) / sizeof(unsigned));
+  ctx->d_sel = reinterpret_cast<Select*>(ws + p.o_sel);
+  ctx->d_tile_cnt = reinterpret_cast<int2*>(ws + p.o_tile_cnt);
+  ctx->d_tile_h3 = reinterpret_cast<unsigned short*>(ws + p.o_tile_h3);
+  ctx->d_tile_pre = reinterpret_cast<int2*>(ws + p.o_tile_pre);
+
+  cudaError_t e = cudaSuccess;
+  auto up = [&](void* dst, const void* src, size_t bytes) {
+    if (e == cudaSuccess && bytes) e = cudaMemcpy(dst, src, bytes, cudaMemcpyHostToDevice);
+  };
+  up(ctx->d_layers, p.layers.data(), sizeof(DevLayer) * p.layers.size());
+  up(ctx->d_row_items, p.row_items.data(), sizeof(RowItem) * p.row_items.size());
+  up(ctx->d_col_items, p.col_items.data(), sizeof(ColItem) * p.col_items.size());
+  up(ctx->d_tiles, p.tiles.data(), sizeof(Tile) * p.tiles.size());
+  up(ctx->d_mat_layers, p.mat_layers.data(), sizeof(int) * p.mat_layers.size());
+  up(ctx->d_vec_tiles, p.vec_tiles.data(), sizeof(int) * p.vec_tiles.size());
+  int dev = 0;
+  if (e == cudaSuccess) e = cudaGetDevice(&dev);
+  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, dev);
+  if (e != cudaSuccess) { delete ctx; return ACC_ECUDA; }
+  *out = ctx;
+  return ACC_OK;
+}
+
+int acc_destroy(acc_ctx* ctx) {
+  if (!ctx) return ACC_EINVAL;
+  delete ctx;
+  return ACC_OK;
+}
+
+int acc_factor_layout(const acc_ctx* ctx, int64_t* q_row, int64_t* p_row, int64_t* q_rows, int64_t* p_rows) {
+  if (!ctx) return ACC_EINVAL;
+  for (int l = 0; l < ctx->cfg.n_layers; ++l) {
+    if (q_row) q_row[l] = ctx->plan.layers[l].q_row;
+    if (p_row) p_row[l] = ctx->plan.layers[l].p_row;
+  }
+  if (q_rows) *q_rows = ctx->plan.q_rows;
+  if (p_rows) *p_rows = ctx->plan.p_rows;
+  return ACC_OK;
+}
+
+int acc_topk_layout(const acc_ctx* ctx, int64_t* seg_offset, int64_t* k_low, int64_t* k_high, int64_t* capacity) {
+  if (!ctx) return ACC_EINVAL;
+  for (int l = 0; l < ctx->cfg.n_layers; ++l) {
+    const DevLayer& d = ctx->plan.layers[l];
+    if (seg_offset) seg_offset[l] = d.seg_off;
+    if (k_low) k_low[l] = d.kind == ACC_MATRIX ? d.k_low : 0;
+    if (k_high) k_high[l] = d.kind == ACC_MATRIX ? d.k_high : 0;
+  }
+  if (capacity) *capacity = ctx->plan.capacity;
+  return ACC_OK;
+}
+
+static int finish(cudaError_t e) { return e == cudaSuccess ? ACC_OK : ACC_ECUDA; }
+
+int acc_error_feedback(acc_ctx* ctx, const float* grads, float* err, float* delta, void* stream) {
+  if (!ctx || !grads || !err) return ACC_EINVAL;
+  if (!aligned16(grads) || !aligned16(err) || !aligned16(delta)) return ACC_EALIGN;
+  ctx->last_launches = 0;
+  return finish(launch_error_feedback(ctx, grads, err, delta, static_cast<cudaStream_t>(stream)));
+}
+
+int acc_layer_norms(acc_ctx* ctx, const float* buf, int64_t buf_stride, int32_t n_bufs, double* norm2, void* stream) {
+  if (!ctx || !buf || !norm2 || n_bufs < 1 || n_bufs > ctx->cfg.n_workers) return ACC_EINVAL;
+  if (n_bufs > 1 && buf_stride < ctx->cfg.worker_stride) return ACC_EINVAL;
+  if (!aligned16(buf) || (n_bufs > 1 && buf_stride % 4 != 0) || (reinterpret_cast<uintptr_t>(norm2) & 7u)) return ACC_EALIGN;
+  ctx->last_launches = 0;
+  return finish(launch_layer_norms(ctx, buf, buf_stride, n_bufs, norm2, static_cast<cudaStream_t>(stream)));
+}
+
+int acc_detect_regime(acc_ctx* ctx, const double* norm2_curr, double* norm2_prev, float lr_curr, float lr_next,
+                      uint8_t* level, float* delta, void* stream) {
+  if (!ctx || !norm2_curr || !norm2_prev || !level) return ACC_EINVAL;
+  if (!aligned16(delta)) return ACC_EALIGN;
+  ctx->last_launches = 0;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  cudaError_t e = launch_detect(ctx, norm2_curr, norm2_prev, lr_curr, lr_next, level, s);
+  if (e == cudaSuccess && delta) e = cudaMemsetAsync(delta, 0, sizeof(float) * (size_t)ctx->cfg.worker_stride, s);
+  return finish(e);
+}
+
+int acc_powersgd_step(acc_ctx* ctx, const float* grads, float* err, float* q, float* p_hat, const uint8_t* level,
+                      float* out, float* delta, void* stream) {
+  if (!ctx || !grads || !err || !q || !p_hat || !level || !out) return ACC_EINVAL;
+  if (!aligned16(grads) || !aligned16(err) || !aligned16(q) || !aligned16(p_hat) || !aligned16(out) ||
+      !aligned16(delta))
+    return ACC_EALIGN;
+  ctx->last_launches = 0;
+  return finish(launch_powersgd(ctx, grads, err, q, p_hat, level, out, delta, static_cast<cudaStream_t>(stream)));
+}
+
+int acc_topk_step(acc_ctx* ctx, const float* grads, float* err, const uint8_t* level, float* vals, int32_t* idx,
+                  int32_t* counts, float* out, float* delta, void* stream) {
+  if (!ctx || !grads || !err || !level || !vals || !idx || !counts || !out) return ACC_EINVAL;
+  if (!aligned16(grads) || !aligned16(err) || !aligned16(vals) || !aligned16(idx) || !aligned16(out) ||
+      !aligned16(delta))
+    return ACC_EALIGN;
+  ctx->last_launches = 0;
+  return finish(launch_topk(ctx, grads, err, level, vals, idx, counts, out, delta, static_cast<cudaStream_t>(stream)));
+}
+
+int64_t acc_floats_sent(const acc_config* cfg, const uint8_t* level_host, int32_t compressor) {
+  if (!level_host || validate(cfg) != ACC_OK) return -1;
+  if (compressor != ACC_COMPRESSOR_POWERSGD && compressor != ACC_COMPRESSOR_TOPK) return -1;
+  int64_t total = 0;
+  for (int l = 0; l < cfg->n_layers; ++l) {
+    const acc_layer_desc& d = cfg->layers[l];
+    const long long size = (long long)d.rows * d.cols;
+    if (d.kind == ACC_VECTOR) { total += size; continue; }
+    if (compressor == ACC_COMPRESSOR_POWERSGD) {
+      total += (int64_t)(level_host[l] ? cfg->rank_low : cfg->rank_high) * (d.rows + d.cols);
+    } else {
+      total += 2ll * topk_count(size, level_host[l] ? cfg->topk_low_bp : cfg->topk_high_bp) * cfg->n_workers;
+    }
+  }
+  return total;
+}
+
+int32_t acc_last_launch_count(const acc_ctx* ctx) { return ctx ? ctx->last_launches : -1; }
+
+const char* acc_strerror(int status) {
+  switch (status) {
+    case ACC_OK: return "ok";
+    case ACC_EINVAL: return "invalid argument or configuration";
+    case ACC_EALIGN: return "pointer, offset or stride not 16-byte aligned";
+    case ACC_EWORKSPACE: return "workspace missing or too small";
+    case ACC_ECUDA: return "CUDA runtime or launch error";
+    default: return "unknown status";
+  }
+}
+
+}  // extern "C"

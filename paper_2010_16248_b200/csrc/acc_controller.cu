@@ -1,0 +1,124 @@
+// Error-feedback add, detector accumulation, per-layer norms and the regime test (Section 4.2, Algorithm 1).
+#include "acc_internal.cuh"
+
+namespace acc {
+
+// One block per (tile, worker): err <- g + err on MATRIX tiles; delta += g for the deciding worker.
+__global__ void __launch_bounds__(256) ef_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict__ tiles,
+                                                 const float* __restrict__ grads, float* __restrict__ err,
+                                                 float* __restrict__ delta, long long stride, int decider) {
+  const Tile t = tiles[blockIdx.x];
+  const int w = blockIdx.y;
+  const DevLayer L = layers[t.layer];
+  const bool is_mat = L.kind == ACC_MATRIX;
+  const bool acc_delta = (delta != nullptr) && (w == decider);
+  if (!is_mat && !acc_delta) return;
+  const long long base = L.offset + t.elem0;
+  const float* g = grads + (long long)w * stride + base;
+  float* e = err + (long long)w * stride + base;
+  float* d = delta + base;
+  const int n4 = t.nelem >> 2;
+  for (int i = threadIdx.x; i < n4; i += blockDim.x) {
+    const float4 gv = ld_stream4(g + 4 * i);
+    if (is_mat) {
+      const float4 ev = ld_stream4(e + 4 * i);
+      st_stream4(e + 4 * i, make_float4(gv.x + ev.x, gv.y + ev.y, gv.z + ev.z, gv.w + ev.w));
+    }
+    if (acc_delta) {
+      float4 dv = *reinterpret_cast<const float4*>(d + 4 * i);
+      dv.x += gv.x; dv.y += gv.y; dv.z += gv.z; dv.w += gv.w;
+      *reinterpret_cast<float4*>(d + 4 * i) = dv;
+    }
+  }
+  for (int i = 4 * n4 + threadIdx.x; i < t.nelem; i += blockDim.x) {
+    const float gv = g[i];
+    if (is_mat) e[i] = gv + e[i];
+    if (acc_delta) d[i] += gv;
+  }
+}
+
+// One block per (tile, buffer): fp64 sum of squares of the tile, reduced in a fixed order.
+__global__ void __launch_bounds__(256) norm_partial_kernel(const DevLayer* __restrict__ layers,
+                                                           const Tile* __restrict__ tiles,
+                                                           const float* __restrict__ buf, long long stride,
+                                                           double* __restrict__ part, int n_tiles) {
+  __shared__ double sm[8];
+  const Tile t = tiles[blockIdx.x];
+  const int b = blockIdx.y;
+  const float* x = buf + (long long)b * stride + layers[t.layer].offset + t.elem0;
+  double acc = 0.0;
+  const int n4 = t.nelem >> 2;
+  for (int i = threadIdx.x; i < n4; i += blockDim.x) {
+    const float4 v = ld_stream4(x + 4 * i);
+    acc += (double)v.x * v.x;
+    acc += (double)v.y * v.y;
+    acc += (double)v.z * v.z;
+    acc += (double)v.w * v.w;
+  }
+  for (int i = 4 * n4 + threadIdx.x; i < t.nelem; i += blockDim.x) acc += (double)x[i] * x[i];
+  acc = warp_sum(acc);
+  if ((threadIdx.x & 31) == 0) sm[threadIdx.x >> 5] = acc;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double s = 0.0;
+    for (int i = 0; i < (int)(blockDim.x >> 5); ++i) s += sm[i];
+    part[(long long)b * n_tiles + blockIdx.x] = s;
+  }
+}
+
+// One warp per (layer, buffer): sums the layer's tile partials in a fixed order.
+__global__ void norm_final_kernel(const DevLayer* __restrict__ layers, const double* __restrict__ part,
+                                  double* __restrict__ norm2, int n_layers, int n_tiles) {
+  const int l = blockIdx.x, b = blockIdx.y;
+  const DevLayer L = layers[l];
+  double acc = 0.0;
+  for (int i = threadIdx.x; i < L.ntiles; i += 32) acc += part[(long long)b * n_tiles + L.tile0 + i];
+  acc = warp_sum(acc);
+  if (threadIdx.x == 0) norm2[(long long)b * n_layers + l] = acc;
+}
+
+// Algorithm 1 per layer, in product form so that a zero previous norm needs no division.
+__global__ void detect_kernel(const double* __restrict__ n2c, double* __restrict__ n2p, float lr_curr, float lr_next,
+                              double eta, uint8_t* __restrict__ level, int n_layers) {
+  const int l = blockIdx.x * blockDim.x + threadIdx.x;
+  if (l >= n_layers) return;
+  const double cur = n2c[l], prev = n2p[l];
+  uint8_t lv;
+  if (prev < 0.0) {
+    lv = 1;
+  } else {
+    const double a = sqrt(prev), b = sqrt(cur);
+    lv = (fabs(a - b) >= eta * a || lr_next < lr_curr) ? 1 : 0;
+  }
+  level[l] = lv;
+  n2p[l] = cur;
+}
+
+cudaError_t launch_error_feedback(acc_ctx* ctx, const float* grads, float* err, float* delta, cudaStream_t s) {
+  dim3 grid((unsigned)ctx->plan.tiles.size(), (unsigned)ctx->cfg.n_workers);
+  ef_kernel<<<grid, 256, 0, s>>>(ctx->d_layers, ctx->d_tiles, grads, err, delta, ctx->cfg.worker_stride,
+                                 ctx->cfg.decider);
+  ctx->last_launches += 1;
+  return cudaGetLastError();
+}
+
+cudaError_t launch_layer_norms(acc_ctx* ctx, const float* buf, long long stride, int n_bufs, double* norm2,
+                               cudaStream_t s) {
+  const int nt = (int)ctx->plan.tiles.size();
+  norm_partial_kernel<<<dim3((unsigned)nt, (unsigned)n_bufs), 256, 0, s>>>(ctx->d_layers, ctx->d_tiles, buf, stride,
+                                                                          ctx->d_norm_part, nt);
+  norm_final_kernel<<<dim3((unsigned)ctx->cfg.n_layers, (unsigned)n_bufs), 32, 0, s>>>(
+      ctx->d_layers, ctx->d_norm_part, norm2, ctx->cfg.n_layers, nt);
+  ctx->last_launches += 2;
+  return cudaGetLastError();
+}
+
+cudaError_t launch_detect(acc_ctx* ctx, const double* n2c, double* n2p, float lr_curr, float lr_next, uint8_t* level,
+                          cudaStream_t s) {
+  const int L = ctx->cfg.n_layers;
+  detect_kernel<<<(L + 127) / 128, 128, 0, s>>>(n2c, n2p, lr_curr, lr_next, (double)ctx->cfg.eta, level, L);
+  ctx->last_launches += 1;
+  return cudaGetLastError();
+}
+
+}  // namespace acc

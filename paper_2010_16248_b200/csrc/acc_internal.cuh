@@ -1,0 +1,118 @@
+// Internal declarations shared by the CUDA translation units of the library.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <vector>
+
+#include "acc.h"
+
+namespace acc {
+
+constexpr int kTile = 8192;        // elements per flat tile (TopK / EF / norms); multiple of 4
+constexpr int kBins1 = 4096;       // radix-select level 1: key bits [30:19]
+constexpr int kBins2 = 4096;       // level 2: key bits [18:7]
+constexpr int kBins3 = 128;        // level 3: key bits [6:0]
+constexpr int kRowSlabElems = 8192;  // target elements per (row-slab, worker) of the row-wise kernels
+constexpr int kColBlockThreads = 256;
+
+// One layer, device-side view.
+struct DevLayer {
+  long long offset;   // element offset inside a worker's slice
+  int rows, cols, kind;
+  int q_row, p_row;   // first row of the layer's block in q / p_hat (MATRIX), else -1
+  int vec;            // widest vector width (4, 2, 1) at which every row start is aligned
+  int mat;            // index among MATRIX layers, else -1
+  int tile0, ntiles;  // flat tiles of this layer: [tile0, tile0 + ntiles)
+  int k_low, k_high;  // TopK counts
+  long long seg_off;  // first packed entry of the layer inside a worker's packed region
+  long long part_base;  // first float4 of the layer's Q partials
+  int slab_rows, nslabs;  // row slabs of the Q-partial pass
+};
+
+struct RowItem { int layer, row0, nrows; };            // row slab of a MATRIX layer
+struct ColItem { int layer, slab, row0, nrows, col0; };  // (row slab, column block) of a MATRIX layer
+struct Tile { int layer, elem0, nelem; };              // flat tile, never spans layers
+
+// Per (worker, MATRIX layer) state of the radix select.
+struct Select {
+  unsigned b1, b2;      // chosen buckets of level 1 and 2
+  unsigned tau;         // 31-bit key of the k-th largest magnitude
+  int k, k1, k2, need;  // k wanted; still wanted inside bucket b1 / (b1,b2); ties (key == tau) to keep
+  int pad;
+};
+
+struct Plan {
+  std::vector<DevLayer> layers;
+  std::vector<RowItem> row_items;
+  std::vector<ColItem> col_items;
+  std::vector<Tile> tiles;
+  std::vector<int> mat_layers;   // layer index of each MATRIX layer
+  std::vector<int> vec_tiles;    // tile indices that belong to VECTOR layers
+  long long q_rows = 0, p_rows = 0, capacity = 0, part_f4 = 0;
+  int n_mat = 0;
+  // workspace offsets (bytes)
+  size_t o_layers = 0, o_row_items = 0, o_col_items = 0, o_tiles = 0, o_mat_layers = 0, o_vec_tiles = 0,
+         o_part = 0, o_norm_part = 0, o_hist = 0, o_sel = 0, o_tile_cnt = 0, o_tile_h3 = 0, o_tile_pre = 0,
+         hist_bytes = 0, total = 0;
+};
+
+}  // namespace acc
+
+struct acc_ctx {
+  acc_config cfg;
+  std::vector<acc_layer_desc> host_layers;
+  acc::Plan plan;
+  char* ws = nullptr;
+  int sm_count = 148;
+  int last_launches = 0;
+  // device views into the workspace
+  acc::DevLayer* d_layers = nullptr;
+  acc::RowItem* d_row_items = nullptr;
+  acc::ColItem* d_col_items = nullptr;
+  acc::Tile* d_tiles = nullptr;
+  int* d_mat_layers = nullptr;
+  int* d_vec_tiles = nullptr;
+  float4* d_part = nullptr;
+  double* d_norm_part = nullptr;
+  unsigned* d_hist1 = nullptr;
+  unsigned* d_hist2 = nullptr;
+  unsigned* d_hist3 = nullptr;
+  acc::Select* d_sel = nullptr;
+  int2* d_tile_cnt = nullptr;
+  unsigned short* d_tile_h3 = nullptr;
+  int2* d_tile_pre = nullptr;
+};
+
+namespace acc {
+
+// Kernel launchers (one per translation unit).  Each returns a cudaError_t from cudaGetLastError and
+// adds the number of kernels it launched to ctx->last_launches.
+cudaError_t launch_error_feedback(acc_ctx* ctx, const float* grads, float* err, float* delta, cudaStream_t s);
+cudaError_t launch_layer_norms(acc_ctx* ctx, const float* buf, long long stride, int n_bufs, double* norm2,
+                               cudaStream_t s);
+cudaError_t launch_detect(acc_ctx* ctx, const double* n2c, double* n2p, float lr_curr, float lr_next,
+                          uint8_t* level, cudaStream_t s);
+cudaError_t launch_powersgd(acc_ctx* ctx, const float* grads, float* err, float* q, float* p_hat,
+                            const uint8_t* level, float* out, float* delta, cudaStream_t s);
+cudaError_t launch_topk(acc_ctx* ctx, const float* grads, float* err, const uint8_t* level, float* vals,
+                        int32_t* idx, int32_t* counts, float* out, float* delta, cudaStream_t s);
+
+// ---- small device helpers -------------------------------------------------------------------------
+__device__ __forceinline__ float4 ld_stream4(const float* p) { return __ldcs(reinterpret_cast<const float4*>(p)); }
+__device__ __forceinline__ float ld_stream1(const float* p) { return __ldcs(p); }
+__device__ __forceinline__ void st_stream4(float* p, float4 v) { __stcs(reinterpret_cast<float4*>(p), v); }
+
+__device__ __forceinline__ double warp_sum(double v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+}  // namespace acc

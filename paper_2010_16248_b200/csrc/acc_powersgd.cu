@@ -1,0 +1,334 @@
+// PowerSGD rank-r step with error feedback over W workers (compressor of Section 5.2).
+//
+// Because every product of the step is linear in the workers' matrices, the factors only depend on
+// the mean matrix  Mbar = (1/W) sum_w (g_w + e_w):   P = Mbar Q,  Q' = Mbar^T P^,  A = P^ Q'^T.
+// The project pass therefore reads every worker's g and e once, writes M_w back over e_w, and keeps
+// Mbar (1/W of the data) in `out` for the second product; only the residual pass touches the
+// per-worker data again.
+#include "acc_internal.cuh"
+
+namespace acc {
+
+struct RowGeom {
+  long long start;  // element index of the row inside a worker's slice
+  int head, nbody4, tail;
+};
+
+__device__ __forceinline__ RowGeom row_geom(const DevLayer& L, int row) {
+  RowGeom g;
+  g.start = L.offset + (long long)row * L.cols;
+  int h = (int)((4 - (g.start & 3)) & 3);
+  g.head = h < L.cols ? h : L.cols;
+  g.nbody4 = (L.cols - g.head) >> 2;
+  g.tail = L.cols - g.head - 4 * g.nbody4;
+  return g;
+}
+
+// out = mean_w g_w on one tile of a VECTOR layer; delta += g_decider.
+__device__ void vector_mean_tile(const Tile& t, const DevLayer& L, const float* __restrict__ grads,
+                                 float* __restrict__ out, float* __restrict__ delta, long long stride, int W,
+                                 int decider, float inv_w) {
+  const long long base = L.offset + t.elem0;
+  for (int i = threadIdx.x; i < t.nelem; i += blockDim.x) {
+    float acc = 0.f;
+    for (int w = 0; w < W; ++w) {
+      const float g = grads[(long long)w * stride + base + i];
+      acc += g;
+      if (delta != nullptr && w == decider) delta[base + i] += g;
+    }
+    out[base + i] = acc * inv_w;
+  }
+}
+
+// Pass 1.  One block per row slab (one warp per row), all workers:
+//   M_w = g_w + e_w -> err;  Mbar = mean_w M_w -> out;  P[row, :] = Mbar[row, :] . Q   (first r ranks);
+//   delta += g_decider.  Blocks beyond the row items handle the VECTOR tiles.
+template <int WB>
+__global__ void __launch_bounds__(256)
+psgd_project_kernel(const DevLayer* __restrict__ layers, const RowItem* __restrict__ items, int n_items,
+                    const Tile* __restrict__ tiles, const int* __restrict__ vec_tiles,
+                    const float* __restrict__ grads, float* __restrict__ err, const float* __restrict__ q,
+                    float* __restrict__ p, const uint8_t* __restrict__ level, float* __restrict__ out,
+                    float* __restrict__ delta, long long stride, int W, int decider, float inv_w, int rank_low,
+                    int rank_high) {
+  if ((int)blockIdx.x >= n_items) {
+    const Tile t = tiles[vec_tiles[blockIdx.x - n_items]];
+    vector_mean_tile(t, layers[t.layer], grads, out, delta, stride, W, decider, inv_w);
+    return;
+  }
+  const RowItem it = items[blockIdx.x];
+  const DevLayer L = layers[it.layer];
+  const int r = level[it.layer] ? rank_low : rank_high;
+  const float4* __restrict__ Q4 = reinterpret_cast<const float4*>(q) + L.q_row;
+  float4* __restrict__ P4 = reinterpret_cast<float4*>(p) + L.p_row;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  for (int row = it.row0 + warp; row < it.row0 + it.nrows; row += 8) {
+    const RowGeom rg = row_geom(L, row);
+    float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+    for (int t = lane; t < rg.nbody4; t += 32) {
+      const int col = rg.head + 4 * t;
+      const long long idx = rg.start + col;
+      float4 mb = make_float4(0.f, 0.f, 0.f, 0.f);
+      for (int w0 = 0; w0 < W; w0 += WB) {
+        float4 g[WB], e[WB];
+#pragma unroll
+        for (int b = 0; b < WB; ++b)
+          if (w0 + b < W) {
+            g[b] = ld_stream4(grads + (long long)(w0 + b) * stride + idx);
+            e[b] = ld_stream4(err + (long long)(w0 + b) * stride + idx);
+          }
+#pragma unroll
+        for (int b = 0; b < WB; ++b)
+          if (w0 + b < W) {
+            const float4 m = make_float4(g[b].x + e[b].x, g[b].y + e[b].y, g[b].z + e[b].z, g[b].w + e[b].w);
+            *reinterpret_cast<float4*>(err + (long long)(w0 + b) * stride + idx) = m;
+            mb.x += m.x; mb.y += m.y; mb.z += m.z; mb.w += m.w;
+            if (delta != nullptr && w0 + b == decider) {
+              float4 d = *reinterpret_cast<const float4*>(delta + idx);
+              d.x += g[b].x; d.y += g[b].y; d.z += g[b].z; d.w += g[b].w;
+              *reinterpret_cast<float4*>(delta + idx) = d;
+            }
+          }
+      }
+      mb.x *= inv_w; mb.y *= inv_w; mb.z *= inv_w; mb.w *= inv_w;
+      *reinterpret_cast<float4*>(out + idx) = mb;
+      const float4 q0 = __ldg(Q4 + col), q1 = __ldg(Q4 + col + 1), q2 = __ldg(Q4 + col + 2), q3 = __ldg(Q4 + col + 3);
+      a0 = fmaf(mb.x, q0.x, a0); a1 = fmaf(mb.x, q0.y, a1); a2 = fmaf(mb.x, q0.z, a2); a3 = fmaf(mb.x, q0.w, a3);
+      a0 = fmaf(mb.y, q1.x, a0); a1 = fmaf(mb.y, q1.y, a1); a2 = fmaf(mb.y, q1.z, a2); a3 = fmaf(mb.y, q1.w, a3);
+      a0 = fmaf(mb.z, q2.x, a0); a1 = fmaf(mb.z, q2.y, a1); a2 = fmaf(mb.z, q2.z, a2); a3 = fmaf(mb.z, q2.w, a3);
+      a0 = fmaf(mb.w, q3.x, a0); a1 = fmaf(mb.w, q3.y, a1); a2 = fmaf(mb.w, q3.z, a2); a3 = fmaf(mb.w, q3.w, a3);
+    }
+    if (lane < rg.head + rg.tail) {  // the unaligned ends of the row, one element per lane
+      const int col = lane < rg.head ? lane : rg.head + 4 * rg.nbody4 + (lane - rg.head);
+      const long long idx = rg.start + col;
+      float mb = 0.f;
+      for (int w = 0; w < W; ++w) {
+        const float g = grads[(long long)w * stride + idx];
+        const float m = g + err[(long long)w * stride + idx];
+        err[(long long)w * stride + idx] = m;
+        mb += m;
+        if (delta != nullptr && w == decider) delta[idx] += g;
+      }
+      mb *= inv_w;
+      out[idx] = mb;
+      const float4 q0 = __ldg(Q4 + col);
+      a0 = fmaf(mb, q0.x, a0); a1 = fmaf(mb, q0.y, a1); a2 = fmaf(mb, q0.z, a2); a3 = fmaf(mb, q0.w, a3);
+    }
+    a0 = warp_sum(a0); a1 = warp_sum(a1); a2 = warp_sum(a2); a3 = warp_sum(a3);
+    if (lane == 0) {
+      float4 pv = P4[row];
+      pv.x = a0;
+      if (r > 1) pv.y = a1;
+      if (r > 2) pv.z = a2;
+      if (r > 3) pv.w = a3;
+      P4[row] = pv;
+    }
+  }
+}
+
+// Deterministic block-wide sum of doubles; every thread gets the result.
+__device__ __forceinline__ double block_sum(double v, double* sm) {
+  v = warp_sum(v);
+  __syncthreads();
+  if ((threadIdx.x & 31) == 0) sm[threadIdx.x >> 5] = v;
+  __syncthreads();
+  double s = 0.0;
+  const int nw = blockDim.x >> 5;
+  for (int i = 0; i < nw; ++i) s += sm[i];
+  return s;
+}
+
+// Pass 2.  One block per MATRIX layer: modified Gram-Schmidt on the first r columns of P, in place.
+__global__ void __launch_bounds__(1024)
+psgd_orthonormalise_kernel(const DevLayer* __restrict__ layers, const int* __restrict__ mat_layers,
+                           float* __restrict__ p, const uint8_t* __restrict__ level, int rank_low, int rank_high,
+                           float eps) {
+  __shared__ double sm[32];
+  const int l = mat_layers[blockIdx.x];
+  const DevLayer L = layers[l];
+  const int r = level[l] ? rank_low : rank_high;
+  float* P = p + 4ll * L.p_row;
+  const int n = L.rows;
+  for (int c = 0; c < r; ++c) {
+    for (int j = 0; j < c; ++j) {
+      double part = 0.0;
+      for (int i = threadIdx.x; i < n; i += blockDim.x) part += (double)P[4 * i + j] * (double)P[4 * i + c];
+      const float dot = (float)block_sum(part, sm);
+      for (int i = threadIdx.x; i < n; i += blockDim.x) P[4 * i + c] = fmaf(-dot, P[4 * i + j], P[4 * i + c]);
+    }
+    double part = 0.0;
+    for (int i = threadIdx.x; i < n; i += blockDim.x) part += (double)P[4 * i + c] * (double)P[4 * i + c];
+    const double nrm = sqrt(block_sum(part, sm));
+    const float inv = (float)(1.0 / (nrm + (double)eps));
+    for (int i = threadIdx.x; i < n; i += blockDim.x) P[4 * i + c] *= inv;
+  }
+}
+
+template <int VEC>
+struct VecT;
+template <> struct VecT<4> { using type = float4; };
+template <> struct VecT<2> { using type = float2; };
+template <> struct VecT<1> { using type = float; };
+
+template <int VEC>
+__device__ __forceinline__ void qpart_cols(const ColItem& it, const DevLayer& L, const float* __restrict__ mbar,
+                                           const float4* __restrict__ P4, float4* __restrict__ part) {
+  using V = typename VecT<VEC>::type;
+  const int col = it.col0 + (int)threadIdx.x * VEC;
+  if (col >= L.cols) return;
+  float acc[VEC][4];
+#pragma unroll
+  for (int e = 0; e < VEC; ++e) acc[e][0] = acc[e][1] = acc[e][2] = acc[e][3] = 0.f;
+  const float* base = mbar + L.offset + (long long)it.row0 * L.cols + col;
+  const float4* pr = P4 + it.row0;
+#pragma unroll 8
+  for (int i = 0; i < it.nrows; ++i) {
+    const V mv = *reinterpret_cast<const V*>(base + (long long)i * L.cols);
+    const float4 pv = __ldg(pr + i);
+    const float* m = reinterpret_cast<const float*>(&mv);
+#pragma unroll
+    for (int e = 0; e < VEC; ++e) {
+      acc[e][0] = fmaf(m[e], pv.x, acc[e][0]);
+      acc[e][1] = fmaf(m[e], pv.y, acc[e][1]);
+      acc[e][2] = fmaf(m[e], pv.z, acc[e][2]);
+      acc[e][3] = fmaf(m[e], pv.w, acc[e][3]);
+    }
+  }
+  float4* dst = part + L.part_base + (long long)it.slab * L.cols + col;
+#pragma unroll
+  for (int e = 0; e < VEC; ++e) dst[e] = make_float4(acc[e][0], acc[e][1], acc[e][2], acc[e][3]);
+}
+
+// Pass 3.  One block per (row slab, column block): partial Q' = Mbar[slab]^T P^[slab]; each thread owns
+// `vec` adjacent columns and walks the slab's rows.
+__global__ void __launch_bounds__(kColBlockThreads)
+psgd_qpartial_kernel(const DevLayer* __restrict__ layers, const ColItem* __restrict__ items,
+                     const float* __restrict__ mbar, const float* __restrict__ p, float4* __restrict__ part) {
+  const ColItem it = items[blockIdx.x];
+  const DevLayer L = layers[it.layer];
+  const float4* P4 = reinterpret_cast<const float4*>(p) + L.p_row;
+  if (L.vec == 4) qpart_cols<4>(it, L, mbar, P4, part);
+  else if (L.vec == 2) qpart_cols<2>(it, L, mbar, P4, part);
+  else qpart_cols<1>(it, L, mbar, P4, part);
+}
+
+// Pass 4.  Sums the slab partials of 32 columns in a fixed order and stores the first r ranks of Q'.
+__global__ void __launch_bounds__(256)
+psgd_qreduce_kernel(const DevLayer* __restrict__ layers, const int* __restrict__ mat_layers,
+                    const float4* __restrict__ part, float* __restrict__ q, const uint8_t* __restrict__ level,
+                    int rank_low, int rank_high) {
+  __shared__ float4 sm[8][32];
+  const int l = mat_layers[blockIdx.y];
+  const DevLayer L = layers[l];
+  if ((int)blockIdx.x * 32 >= L.cols) return;
+  const int cx = threadIdx.x & 31, gy = threadIdx.x >> 5;
+  const int col = blockIdx.x * 32 + cx;
+  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+  if (col < L.cols) {
+    for (int s = gy; s < L.nslabs; s += 8) {
+      const float4 v = part[L.part_base + (long long)s * L.cols + col];
+      acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+    }
+  }
+  sm[gy][cx] = acc;
+  __syncthreads();
+  if (gy == 0 && col < L.cols) {
+    float4 t = sm[0][cx];
+    for (int g = 1; g < 8; ++g) { t.x += sm[g][cx].x; t.y += sm[g][cx].y; t.z += sm[g][cx].z; t.w += sm[g][cx].w; }
+    const int r = level[l] ? rank_low : rank_high;
+    float4* Q4 = reinterpret_cast<float4*>(q) + L.q_row;
+    float4 qv = Q4[col];
+    qv.x = t.x;
+    if (r > 1) qv.y = t.y;
+    if (r > 2) qv.z = t.z;
+    if (r > 3) qv.w = t.w;
+    Q4[col] = qv;
+  }
+}
+
+__device__ __forceinline__ float lowrank_entry(const float4& pv, const float4& qv, int r) {
+  float a = pv.x * qv.x;
+  if (r > 1) a = fmaf(pv.y, qv.y, a);
+  if (r > 2) a = fmaf(pv.z, qv.z, a);
+  if (r > 3) a = fmaf(pv.w, qv.w, a);
+  return a;
+}
+
+// Pass 5.  One block per row slab (one warp per row): A = P^ Q'^T -> out;  e_w = M_w - A -> err.
+template <int WB>
+__global__ void __launch_bounds__(256)
+psgd_residual_kernel(const DevLayer* __restrict__ layers, const RowItem* __restrict__ items,
+                     float* __restrict__ err, const float* __restrict__ q, const float* __restrict__ p,
+                     const uint8_t* __restrict__ level, float* __restrict__ out, long long stride, int W,
+                     int rank_low, int rank_high) {
+  const RowItem it = items[blockIdx.x];
+  const DevLayer L = layers[it.layer];
+  const int r = level[it.layer] ? rank_low : rank_high;
+  const float4* __restrict__ Q4 = reinterpret_cast<const float4*>(q) + L.q_row;
+  const float4* __restrict__ P4 = reinterpret_cast<const float4*>(p) + L.p_row;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  for (int row = it.row0 + warp; row < it.row0 + it.nrows; row += 8) {
+    const RowGeom rg = row_geom(L, row);
+    const float4 pv = __ldg(P4 + row);
+    for (int t = lane; t < rg.nbody4; t += 32) {
+      const int col = rg.head + 4 * t;
+      const long long idx = rg.start + col;
+      float4 a;
+      a.x = lowrank_entry(pv, __ldg(Q4 + col), r);
+      a.y = lowrank_entry(pv, __ldg(Q4 + col + 1), r);
+      a.z = lowrank_entry(pv, __ldg(Q4 + col + 2), r);
+      a.w = lowrank_entry(pv, __ldg(Q4 + col + 3), r);
+      for (int w0 = 0; w0 < W; w0 += WB) {
+        float4 m[WB];
+#pragma unroll
+        for (int b = 0; b < WB; ++b)
+          if (w0 + b < W) m[b] = ld_stream4(err + (long long)(w0 + b) * stride + idx);
+#pragma unroll
+        for (int b = 0; b < WB; ++b)
+          if (w0 + b < W)
+            st_stream4(err + (long long)(w0 + b) * stride + idx,
+                       make_float4(m[b].x - a.x, m[b].y - a.y, m[b].z - a.z, m[b].w - a.w));
+      }
+      st_stream4(out + idx, a);
+    }
+    if (lane < rg.head + rg.tail) {
+      const int col = lane < rg.head ? lane : rg.head + 4 * rg.nbody4 + (lane - rg.head);
+      const long long idx = rg.start + col;
+      const float a = lowrank_entry(pv, __ldg(Q4 + col), r);
+      for (int w = 0; w < W; ++w) err[(long long)w * stride + idx] -= a;
+      out[idx] = a;
+    }
+  }
+}
+
+cudaError_t launch_powersgd(acc_ctx* ctx, const float* grads, float* err, float* q, float* p_hat,
+                            const uint8_t* level, float* out, float* delta, cudaStream_t s) {
+  const Plan& pl = ctx->plan;
+  const acc_config& c = ctx->cfg;
+  const int n_items = (int)pl.row_items.size();
+  const int n_vec = (int)pl.vec_tiles.size();
+  const float inv_w = 1.0f / (float)c.n_workers;
+  if (n_items + n_vec > 0) {
+    psgd_project_kernel<4><<<n_items + n_vec, 256, 0, s>>>(
+        ctx->d_layers, ctx->d_row_items, n_items, ctx->d_tiles, ctx->d_vec_tiles, grads, err, q, p_hat, level, out,
+        delta, c.worker_stride, c.n_workers, c.decider, inv_w, c.rank_low, c.rank_high);
+    ctx->last_launches += 1;
+  }
+  if (pl.n_mat > 0) {
+    psgd_orthonormalise_kernel<<<pl.n_mat, 1024, 0, s>>>(ctx->d_layers, ctx->d_mat_layers, p_hat, level, c.rank_low,
+                                                        c.rank_high, c.gs_eps);
+    psgd_qpartial_kernel<<<(unsigned)pl.col_items.size(), kColBlockThreads, 0, s>>>(ctx->d_layers, ctx->d_col_items,
+                                                                                    out, p_hat, ctx->d_part);
+    int max_cols = 0;
+    for (int l : pl.mat_layers) max_cols = max_cols > pl.layers[l].cols ? max_cols : pl.layers[l].cols;
+    psgd_qreduce_kernel<<<dim3((max_cols + 31) / 32, pl.n_mat), 256, 0, s>>>(ctx->d_layers, ctx->d_mat_layers,
+                                                                            ctx->d_part, q, level, c.rank_low,
+                                                                            c.rank_high);
+    psgd_residual_kernel<4><<<n_items, 256, 0, s>>>(ctx->d_layers, ctx->d_row_items, err, q, p_hat, level, out,
+                                                    c.worker_stride, c.n_workers, c.rank_low, c.rank_high);
+    ctx->last_launches += 4;
+  }
+  return cudaGetLastError();
+}
+
+}  // namespace acc

@@ -1,0 +1,473 @@
+// TopK-K% sparsification with error feedback (sparsifier of Section 5.3), exact and order-preserving.
+//
+// Selection is a three-level radix select on the 31-bit magnitude pattern key = bits(M) & 0x7fffffff
+// (12 + 12 + 7 bits, shared-memory histograms), followed by an ordered compaction:
+//   ef_hist1   M = g + e -> err, level-1 histogram per (worker, layer)                [reads g, e; writes M]
+//   pick1      bucket b1 holding the k-th largest key
+//   hist2      level-2 histogram of the keys inside b1, per-tile count of keys above b1        [reads M]
+//   pick2      bucket b2
+//   hist3      per-tile level-3 histogram of the keys with prefix (b1,b2), per-tile count above [reads M]
+//   pick3scan  threshold tau, number of ties to keep, exclusive per-tile prefix of (above, ties)
+//   select     keep key > tau and the lowest-index `need` of key == tau; write (val, idx) in index
+//              order, zero the kept entries of err, accumulate out = mean_w kept                [reads M]
+// No floating-point atomics and no inter-block waiting: same input, same bits.
+#include "acc_internal.cuh"
+
+namespace acc {
+
+__device__ __forceinline__ unsigned key_of(float v) { return __float_as_uint(v) & 0x7fffffffu; }
+
+// Pass A.  Persistent blocks over (worker, tile) in worker-major order; the shared histogram is flushed
+// when the (worker, layer) segment changes.
+__global__ void __launch_bounds__(256)
+topk_ef_hist1_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict__ tiles, int n_tiles, int n_mat,
+                     const float* __restrict__ grads, float* __restrict__ err, float* __restrict__ delta,
+                     long long stride, int W, int decider, unsigned* __restrict__ hist1) {
+  __shared__ unsigned h[kBins1];
+  for (int b = threadIdx.x; b < kBins1; b += blockDim.x) h[b] = 0;
+  __syncthreads();
+  const long long V = (long long)W * n_tiles;
+  const long long v0 = V * blockIdx.x / gridDim.x, v1 = V * (blockIdx.x + 1) / gridDim.x;
+  int cur = -1;
+  for (long long v = v0; v < v1; ++v) {
+    const int w = (int)(v / n_tiles);
+    const Tile t = tiles[(int)(v % n_tiles)];
+    const DevLayer L = layers[t.layer];
+    if (L.kind != ACC_MATRIX) continue;
+    const int seg = w * n_mat + L.mat;
+    if (seg != cur) {
+      __syncthreads();
+      if (cur >= 0)
+        for (int b = threadIdx.x; b < kBins1; b += blockDim.x) {
+          const unsigned c = h[b];
+          if (c) { atomicAdd(&hist1[(long long)cur * kBins1 + b], c); h[b] = 0; }
+        }
+      __syncthreads();
+      cur = seg;
+    }
+    const long long base = L.offset + t.elem0;
+    const float* g = grads + (long long)w * stride + base;
+    float* e = err + (long long)w * stride + base;
+    const bool acc_delta = delta != nullptr && w == decider;
+    const int n4 = t.nelem >> 2;
+#pragma unroll 4
+    for (int i = threadIdx.x; i < n4; i += blockDim.x) {
+      const float4 gv = ld_stream4(g + 4 * i);
+      const float4 ev = ld_stream4(e + 4 * i);
+      const float4 m = make_float4(gv.x + ev.x, gv.y + ev.y, gv.z + ev.z, gv.w + ev.w);
+      *reinterpret_cast<float4*>(e + 4 * i) = m;
+      atomicAdd(&h[key_of(m.x) >> 19], 1u);
+      atomicAdd(&h[key_of(m.y) >> 19], 1u);
+      atomicAdd(&h[key_of(m.z) >> 19], 1u);
+      atomicAdd(&h[key_of(m.w) >> 19], 1u);
+      if (acc_delta) {
+        float4 d = *reinterpret_cast<const float4*>(delta + base + 4 * i);
+        d.x += gv.x; d.y += gv.y; d.z += gv.z; d.w += gv.w;
+        *reinterpret_cast<float4*>(delta + base + 4 * i) = d;
+      }
+    }
+    for (int i = 4 * n4 + threadIdx.x; i < t.nelem; i += blockDim.x) {
+      const float gv = g[i];
+      const float m = gv + e[i];
+      e[i] = m;
+      atomicAdd(&h[key_of(m) >> 19], 1u);
+      if (acc_delta) delta[base + i] += gv;
+    }
+  }
+  __syncthreads();
+  if (cur >= 0)
+    for (int b = threadIdx.x; b < kBins1; b += blockDim.x) {
+      const unsigned c = h[b];
+      if (c) atomicAdd(&hist1[(long long)cur * kBins1 + b], c);
+    }
+}
+
+// Finds, scanning from the top bin, the bin that holds the `want`-th largest key (1-based).
+// Single-thread helper over `nbins` counters; returns the bin and the count of keys in higher bins.
+__device__ void pick_from_top(const unsigned* __restrict__ hist, int nbins, long long want, unsigned* bin,
+                              long long* above) {
+  long long cum = 0;
+  int b = nbins - 1;
+  for (; b > 0; --b) {
+    const long long c = hist[b];
+    if (cum + c >= want) break;
+    cum += c;
+  }
+  *bin = (unsigned)b;
+  *above = cum;
+}
+
+// Block-parallel version for the 4096-bin levels: each of 256 threads owns 16 consecutive bins.
+__device__ void pick_from_top_block(const unsigned* __restrict__ hist, long long want, unsigned* bin,
+                                    long long* above, unsigned* sm_sums) {
+  const int tid = threadIdx.x;
+  unsigned s = 0;
+  for (int i = 0; i < 16; ++i) s += hist[tid * 16 + i];
+  sm_sums[tid] = s;
+  __syncthreads();
+  if (tid == 0) {
+    long long cum = 0;
+    int t = 255;
+    for (; t > 0; --t) {
+      if (cum + sm_sums[t] >= want) break;
+      cum += sm_sums[t];
+    }
+    int b = t * 16 + 15;
+    for (; b > t * 16; --b) {
+      const long long c = hist[b];
+      if (cum + c >= want) break;
+      cum += c;
+    }
+    *bin = (unsigned)b;
+    *above = cum;
+  }
+  __syncthreads();
+}
+
+// One block per (worker, MATRIX layer).
+__global__ void __launch_bounds__(256)
+topk_pick1_kernel(const DevLayer* __restrict__ layers, const int* __restrict__ mat_layers, int n_mat, int n_layers,
+                  const uint8_t* __restrict__ level, const unsigned* __restrict__ hist1, Select* __restrict__ sel,
+                  int32_t* __restrict__ counts) {
+  __shared__ unsigned sums[256];
+  __shared__ unsigned bin;
+  __shared__ long long above;
+  const int seg = blockIdx.x, w = seg / n_mat, l = mat_layers[seg % n_mat];
+  const DevLayer L = layers[l];
+  const int k = level[l] ? L.k_low : L.k_high;
+  pick_from_top_block(hist1 + (long long)seg * kBins1, k, &bin, &above, sums);
+  if (threadIdx.x == 0) {
+    Select s;
+    s.b1 = bin; s.b2 = 0; s.tau = 0; s.k = k; s.k1 = k - (int)above; s.k2 = 0; s.need = 0; s.pad = 0;
+    sel[seg] = s;
+    counts[w * n_layers + l] = k;
+  }
+}
+
+__global__ void __launch_bounds__(256)
+topk_pick2_kernel(int n_mat, const unsigned* __restrict__ hist2, Select* __restrict__ sel) {
+  __shared__ unsigned sums[256];
+  __shared__ unsigned bin;
+  __shared__ long long above;
+  const int seg = blockIdx.x;
+  const int k1 = sel[seg].k1;
+  pick_from_top_block(hist2 + (long long)seg * kBins2, k1, &bin, &above, sums);
+  if (threadIdx.x == 0) { sel[seg].b2 = bin; sel[seg].k2 = k1 - (int)above; }
+}
+
+// Pass C.  Level-2 histogram of the keys whose level-1 bin is b1; per tile, how many keys lie in higher bins.
+__global__ void __launch_bounds__(256)
+topk_hist2_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict__ tiles, int n_tiles, int n_mat,
+                  const float* __restrict__ err, long long stride, int W, const Select* __restrict__ sel,
+                  unsigned* __restrict__ hist2, int2* __restrict__ tile_cnt) {
+  __shared__ unsigned h[kBins2];
+  __shared__ int cnt;
+  for (int b = threadIdx.x; b < kBins2; b += blockDim.x) h[b] = 0;
+  if (threadIdx.x == 0) cnt = 0;
+  __syncthreads();
+  const long long V = (long long)W * n_tiles;
+  const long long v0 = V * blockIdx.x / gridDim.x, v1 = V * (blockIdx.x + 1) / gridDim.x;
+  int cur = -1;
+  unsigned b1 = 0;
+  for (long long v = v0; v < v1; ++v) {
+    const int w = (int)(v / n_tiles), ti = (int)(v % n_tiles);
+    const Tile t = tiles[ti];
+    const DevLayer L = layers[t.layer];
+    if (L.kind != ACC_MATRIX) continue;
+    const int seg = w * n_mat + L.mat;
+    if (seg != cur) {
+      __syncthreads();
+      if (cur >= 0)
+        for (int b = threadIdx.x; b < kBins2; b += blockDim.x) {
+          const unsigned c = h[b];
+          if (c) { atomicAdd(&hist2[(long long)cur * kBins2 + b], c); h[b] = 0; }
+        }
+      __syncthreads();
+      cur = seg;
+      b1 = sel[seg].b1;
+    }
+    const float* m = err + (long long)w * stride + L.offset + t.elem0;
+    int above = 0;
+    const int n4 = t.nelem >> 2;
+#pragma unroll 4
+    for (int i = threadIdx.x; i < n4; i += blockDim.x) {
+      const float4 mv = ld_stream4(m + 4 * i);
+      const unsigned k0 = key_of(mv.x), k1 = key_of(mv.y), k2 = key_of(mv.z), k3 = key_of(mv.w);
+      above += ((k0 >> 19) > b1) + ((k1 >> 19) > b1) + ((k2 >> 19) > b1) + ((k3 >> 19) > b1);
+      if ((k0 >> 19) == b1) atomicAdd(&h[(k0 >> 7) & 0xfffu], 1u);
+      if ((k1 >> 19) == b1) atomicAdd(&h[(k1 >> 7) & 0xfffu], 1u);
+      if ((k2 >> 19) == b1) atomicAdd(&h[(k2 >> 7) & 0xfffu], 1u);
+      if ((k3 >> 19) == b1) atomicAdd(&h[(k3 >> 7) & 0xfffu], 1u);
+    }
+    for (int i = 4 * n4 + threadIdx.x; i < t.nelem; i += blockDim.x) {
+      const unsigned k0 = key_of(m[i]);
+      above += (k0 >> 19) > b1;
+      if ((k0 >> 19) == b1) atomicAdd(&h[(k0 >> 7) & 0xfffu], 1u);
+    }
+    above = __reduce_add_sync(0xffffffffu, above);
+    if ((threadIdx.x & 31) == 0 && above) atomicAdd(&cnt, above);
+    __syncthreads();
+    if (threadIdx.x == 0) { tile_cnt[(long long)w * n_tiles + ti].x = cnt; cnt = 0; }
+    __syncthreads();
+  }
+  __syncthreads();
+  if (cur >= 0)
+    for (int b = threadIdx.x; b < kBins2; b += blockDim.x) {
+      const unsigned c = h[b];
+      if (c) atomicAdd(&hist2[(long long)cur * kBins2 + b], c);
+    }
+}
+
+// Pass C'.  One block per (tile, worker): level-3 histogram of the keys with 24-bit prefix (b1, b2), kept
+// per tile (16-bit counters) and summed per segment; per-tile count of keys in bin b1 above b2.
+__global__ void __launch_bounds__(256)
+topk_hist3_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict__ tiles, int n_tiles, int n_mat,
+                  const float* __restrict__ err, long long stride, const Select* __restrict__ sel,
+                  unsigned* __restrict__ hist3, int2* __restrict__ tile_cnt, unsigned short* __restrict__ tile_h3) {
+  __shared__ unsigned h[kBins3];
+  __shared__ int cnt;
+  const int ti = blockIdx.x, w = blockIdx.y;
+  const Tile t = tiles[ti];
+  const DevLayer L = layers[t.layer];
+  if (L.kind != ACC_MATRIX) return;
+  if (threadIdx.x < kBins3) h[threadIdx.x] = 0;
+  if (threadIdx.x == 0) cnt = 0;
+  __syncthreads();
+  const int seg = w * n_mat + L.mat;
+  const Select s = sel[seg];
+  const unsigned prefix = (s.b1 << 12) | s.b2;
+  const float* m = err + (long long)w * stride + L.offset + t.elem0;
+  int above = 0;
+  const int n4 = t.nelem >> 2;
+#pragma unroll 4
+  for (int i = threadIdx.x; i < n4; i += blockDim.x) {
+    const float4 mv = ld_stream4(m + 4 * i);
+    const unsigned k[4] = {key_of(mv.x), key_of(mv.y), key_of(mv.z), key_of(mv.w)};
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const unsigned p = k[e] >> 7;
+      above += ((p >> 12) == s.b1) && (p > prefix);
+      if (p == prefix) atomicAdd(&h[k[e] & 127u], 1u);
+    }
+  }
+  for (int i = 4 * n4 + threadIdx.x; i < t.nelem; i += blockDim.x) {
+    const unsigned k0 = key_of(m[i]), p = k0 >> 7;
+    above += ((p >> 12) == s.b1) && (p > prefix);
+    if (p == prefix) atomicAdd(&h[k0 & 127u], 1u);
+  }
+  above = __reduce_add_sync(0xffffffffu, above);
+  if ((threadIdx.x & 31) == 0 && above) atomicAdd(&cnt, above);
+  __syncthreads();
+  if (threadIdx.x == 0) tile_cnt[(long long)w * n_tiles + ti].y = cnt;
+  if (threadIdx.x < kBins3) {
+    const unsigned c = h[threadIdx.x];
+    tile_h3[((long long)w * n_tiles + ti) * kBins3 + threadIdx.x] = (unsigned short)c;
+    if (c) atomicAdd(&hist3[(long long)seg * kBins3 + threadIdx.x], c);
+  }
+}
+
+// One block per (worker, MATRIX layer): final threshold and the exclusive prefix, over the layer's tiles
+// in index order, of (keys above tau, keys equal to tau).
+__global__ void __launch_bounds__(256)
+topk_pick3_scan_kernel(const DevLayer* __restrict__ layers, const int* __restrict__ mat_layers, int n_mat,
+                       int n_tiles, const unsigned* __restrict__ hist3, Select* __restrict__ sel,
+                       const int2* __restrict__ tile_cnt, const unsigned short* __restrict__ tile_h3,
+                       int2* __restrict__ tile_pre) {
+  __shared__ unsigned b3s;
+  __shared__ int2 chunk_sum[256];
+  const int seg = blockIdx.x, w = seg / n_mat, l = mat_layers[seg % n_mat];
+  const DevLayer L = layers[l];
+  if (threadIdx.x == 0) {
+    Select s = sel[seg];
+    unsigned bin;
+    long long above;
+    pick_from_top(hist3 + (long long)seg * kBins3, kBins3, s.k2, &bin, &above);
+    s.tau = (s.b1 << 19) | (s.b2 << 7) | bin;
+    s.need = s.k2 - (int)above;
+    sel[seg] = s;
+    b3s = bin;
+  }
+  __syncthreads();
+  const unsigned b3 = b3s;
+  const int per = (L.ntiles + 255) / 256;
+  const int t0 = min(L.ntiles, (int)threadIdx.x * per), t1 = min(L.ntiles, t0 + per);
+  const long long tb = (long long)w * n_tiles + L.tile0;
+  int2 sum = make_int2(0, 0);
+  for (int t = t0; t < t1; ++t) {
+    const int2 c = tile_cnt[tb + t];
+    const unsigned short* h = tile_h3 + (tb + t) * kBins3;
+    int above = c.x + c.y;
+    for (unsigned b = b3 + 1; b < (unsigned)kBins3; ++b) above += h[b];
+    sum.x += above;
+    sum.y += h[b3];
+  }
+  chunk_sum[threadIdx.x] = sum;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int2 run = make_int2(0, 0);
+    for (int i = 0; i < 256; ++i) {
+      const int2 c = chunk_sum[i];
+      chunk_sum[i] = run;
+      run.x += c.x; run.y += c.y;
+    }
+  }
+  __syncthreads();
+  int2 run = chunk_sum[threadIdx.x];
+  for (int t = t0; t < t1; ++t) {
+    const int2 c = tile_cnt[tb + t];
+    const unsigned short* h = tile_h3 + (tb + t) * kBins3;
+    int above = c.x + c.y;
+    for (unsigned b = b3 + 1; b < (unsigned)kBins3; ++b) above += h[b];
+    tile_pre[tb + t] = run;
+    run.x += above;
+    run.y += h[b3];
+  }
+}
+
+// Pass E.  One block per tile, all workers in order.  Warp `wi` owns float4s [wi*256, wi*256+256) of the
+// tile; lane handles float4 j*32+lane of that range for j = 0..7, so (j, lane, element) is index order.
+__global__ void __launch_bounds__(256)
+topk_select_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict__ tiles, int n_tiles, int n_mat,
+                   const float* __restrict__ grads, float* __restrict__ err, const Select* __restrict__ sel,
+                   const int2* __restrict__ tile_pre, float* __restrict__ vals, int32_t* __restrict__ idx,
+                   float* __restrict__ out, float* __restrict__ delta, long long stride, long long capacity, int W,
+                   int decider, float inv_w) {
+  __shared__ unsigned wtot[8];
+  const int ti = blockIdx.x;
+  const Tile t = tiles[ti];
+  const DevLayer L = layers[t.layer];
+  const long long base = L.offset + t.elem0;
+  if (L.kind != ACC_MATRIX) {  // VECTOR layer: plain mean, detector accumulation
+    for (int i = threadIdx.x; i < t.nelem; i += blockDim.x) {
+      float acc = 0.f;
+      for (int w = 0; w < W; ++w) {
+        const float g = grads[(long long)w * stride + base + i];
+        acc += g;
+        if (delta != nullptr && w == decider) delta[base + i] += g;
+      }
+      out[base + i] = acc * inv_w;
+    }
+    return;
+  }
+  const int wi = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  float oacc[8][4];
+#pragma unroll
+  for (int j = 0; j < 8; ++j) oacc[j][0] = oacc[j][1] = oacc[j][2] = oacc[j][3] = 0.f;
+  for (int w = 0; w < W; ++w) {
+    const Select s = sel[w * n_mat + L.mat];
+    const int2 pre = tile_pre[(long long)w * n_tiles + ti];
+    float* m = err + (long long)w * stride + base;
+    float mv[8][4];
+    unsigned am[8], tm[8];  // 4-bit masks: key > tau, key == tau
+    unsigned incl[8];       // inclusive lane scan of (above | ties << 16) per j
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const int e0 = 4 * (wi * 256 + j * 32 + lane);
+      if (e0 + 3 < t.nelem) {
+        const float4 v = *reinterpret_cast<const float4*>(m + e0);
+        mv[j][0] = v.x; mv[j][1] = v.y; mv[j][2] = v.z; mv[j][3] = v.w;
+      } else {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) mv[j][e] = (e0 + e < t.nelem) ? m[e0 + e] : 0.f;
+      }
+    }
+    unsigned carry = 0;  // (above | ties << 16) of this warp's earlier j
+    unsigned base_j[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const int e0 = 4 * (wi * 256 + j * 32 + lane);
+      unsigned a = 0, tt = 0;
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const unsigned k = key_of(mv[j][e]);
+        const bool valid = e0 + e < t.nelem;
+        a |= (unsigned)(valid && k > s.tau) << e;
+        tt |= (unsigned)(valid && k == s.tau) << e;
+      }
+      am[j] = a; tm[j] = tt;
+      unsigned c = __popc(a) | (__popc(tt) << 16);
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const unsigned n = __shfl_up_sync(0xffffffffu, c, o);
+        if (lane >= o) c += n;
+      }
+      incl[j] = c;
+      base_j[j] = carry;
+      carry += __shfl_sync(0xffffffffu, c, 31);
+    }
+    __syncthreads();  // previous worker's readers of wtot are done
+    if (lane == 0) wtot[wi] = carry;
+    __syncthreads();
+    unsigned wbase = 0;
+    for (int i = 0; i < wi; ++i) wbase += wtot[i];
+    const long long seg = (long long)w * capacity + L.seg_off;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      if ((am[j] | tm[j]) == 0) continue;
+      const int e0 = 4 * (wi * 256 + j * 32 + lane);
+      const unsigned excl = wbase + base_j[j] + incl[j] - (__popc(am[j]) | (__popc(tm[j]) << 16));
+      int above_before = pre.x + (int)(excl & 0xffffu);
+      int ties_before = pre.y + (int)(excl >> 16);
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const bool is_a = (am[j] >> e) & 1u, is_t = (tm[j] >> e) & 1u;
+        if (is_a || (is_t && ties_before < s.need)) {
+          const int pos = above_before + min(ties_before, s.need);
+          vals[seg + pos] = mv[j][e];
+          idx[seg + pos] = t.elem0 + e0 + e;
+          m[e0 + e] = 0.f;
+          oacc[j][e] += mv[j][e];
+        }
+        above_before += is_a;
+        ties_before += is_t;
+      }
+    }
+  }
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    const int e0 = 4 * (wi * 256 + j * 32 + lane);
+    if (e0 + 3 < t.nelem) {
+      *reinterpret_cast<float4*>(out + base + e0) =
+          make_float4(oacc[j][0] * inv_w, oacc[j][1] * inv_w, oacc[j][2] * inv_w, oacc[j][3] * inv_w);
+    } else {
+#pragma unroll
+      for (int e = 0; e < 4; ++e)
+        if (e0 + e < t.nelem) out[base + e0 + e] = oacc[j][e] * inv_w;
+    }
+  }
+}
+
+cudaError_t launch_topk(acc_ctx* ctx, const float* grads, float* err, const uint8_t* level, float* vals,
+                        int32_t* idx, int32_t* counts, float* out, float* delta, cudaStream_t s) {
+  const Plan& pl = ctx->plan;
+  const acc_config& c = ctx->cfg;
+  const int nt = (int)pl.tiles.size(), W = c.n_workers, n_mat = pl.n_mat;
+  const float inv_w = 1.0f / (float)W;
+  cudaError_t e = cudaMemsetAsync(ctx->ws + pl.o_hist, 0, pl.hist_bytes, s);
+  if (e != cudaSuccess) return e;
+  e = cudaMemsetAsync(counts, 0, sizeof(int32_t) * (size_t)W * c.n_layers, s);
+  if (e != cudaSuccess) return e;
+  if (n_mat > 0) {
+    const long long V = (long long)W * nt;
+    const int grid = (int)(V < (long long)ctx->sm_count * 8 ? V : (long long)ctx->sm_count * 8);
+    topk_ef_hist1_kernel<<<grid, 256, 0, s>>>(ctx->d_layers, ctx->d_tiles, nt, n_mat, grads, err, delta,
+                                              c.worker_stride, W, c.decider, ctx->d_hist1);
+    topk_pick1_kernel<<<W * n_mat, 256, 0, s>>>(ctx->d_layers, ctx->d_mat_layers, n_mat, c.n_layers, level,
+                                                ctx->d_hist1, ctx->d_sel, counts);
+    topk_hist2_kernel<<<grid, 256, 0, s>>>(ctx->d_layers, ctx->d_tiles, nt, n_mat, err, c.worker_stride, W,
+                                           ctx->d_sel, ctx->d_hist2, ctx->d_tile_cnt);
+    topk_pick2_kernel<<<W * n_mat, 256, 0, s>>>(n_mat, ctx->d_hist2, ctx->d_sel);
+    topk_hist3_kernel<<<dim3(nt, W), 256, 0, s>>>(ctx->d_layers, ctx->d_tiles, nt, n_mat, err, c.worker_stride,
+                                                  ctx->d_sel, ctx->d_hist3, ctx->d_tile_cnt, ctx->d_tile_h3);
+    topk_pick3_scan_kernel<<<W * n_mat, 256, 0, s>>>(ctx->d_layers, ctx->d_mat_layers, n_mat, nt, ctx->d_hist3,
+                                                     ctx->d_sel, ctx->d_tile_cnt, ctx->d_tile_h3, ctx->d_tile_pre);
+    ctx->last_launches += 6;
+  }
+  topk_select_kernel<<<nt, 256, 0, s>>>(ctx->d_layers, ctx->d_tiles, nt, n_mat, grads, err, ctx->d_sel,
+                                        ctx->d_tile_pre, vals, idx, out, delta, c.worker_stride, pl.capacity, W,
+                                        c.decider, inv_w);
+  ctx->last_launches += 1;
+  return cudaGetLastError();
+}
+
+}  // namespace acc

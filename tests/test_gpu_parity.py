@@ -1,0 +1,266 @@
+"""Parity of the CUDA path (through the C-ABI) against the CPU oracle on the same seeded inputs.
+
+Integer / index / byte results (TopK indices, counts, packed value bits, error-memory bits after
+TopK, regime decisions) must be bit-exact; float results must match to a relative Frobenius error
+of at most 1e-4 per layer."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import accordion_oracle as orc
+from paper_2010_16248_b200 import binding, workloads as wl
+from tests import helpers as H
+
+pytestmark = pytest.mark.gpu
+
+
+def _table_mixed():
+    # several tiles per layer (tile = 8192 elements), ragged tails, rows that are not multiples of 4,
+    # rows only 8-byte aligned (cols = 650), a tiny layer (27 columns), vectors in between
+    return wl.make_table([
+        ("conv1.weight", (64, 27)), ("bn1.weight", (64,)), ("bn1.bias", (64,)),
+        ("lstm.weight", (37, 650)), ("b0", (13,)),
+        ("conv2.weight", (128, 1152)), ("wide.weight", (9, 4608)), ("b1", (8200,)),
+        ("fc.weight", (100, 512)), ("odd.weight", (33, 333)), ("few.weight", (5, 7)), ("thin.weight", (300, 6)),
+    ])
+
+
+def _random_inputs(table, W, seed, err_scale=0.5):
+    g = torch.Generator(device="cuda").manual_seed(seed)
+    grads = torch.zeros(W, table.stride, device="cuda")
+    err = torch.zeros(W, table.stride, device="cuda")
+    for l, sl in table.slices():
+        scale = 10.0 ** (-(l % 4))
+        grads[:, sl] = torch.randn(W, sl.stop - sl.start, generator=g, device="cuda") * scale
+        if table.kind[l] == wl.MATRIX:
+            err[:, sl] = torch.randn(W, sl.stop - sl.start, generator=g, device="cuda") * scale * err_scale
+    return grads, err
+
+
+# ------------------------------------------------------------------ error feedback, norms, detector
+@pytest.mark.parametrize("W", [1, 3])
+def test_error_feedback_bit_exact(W):
+    table = _table_mixed()
+    ctx = binding.Context(table, W)
+    grads, err = _random_inputs(table, W, 1)
+    delta = torch.randn(table.stride, device="cuda")
+    e0, d0 = err.clone(), delta.clone()
+    ctx.acc_error_feedback(grads, err, delta)
+    torch.cuda.synchronize()
+    M = orc.error_feedback(grads.cpu().numpy(), e0.cpu().numpy(), H.layers_of(table), fp32=True)
+    err_h, d_h = err.cpu().numpy(), delta.cpu().numpy()
+    g_h, d0_h = grads.cpu().numpy(), d0.cpu().numpy()
+    for l, (off, r, c, kind) in enumerate(H.layers_of(table)):
+        sl = slice(off, off + r * c)
+        if kind == orc.MATRIX:
+            assert np.array_equal(err_h[:, sl].view(np.uint32), M[:, sl].view(np.uint32))
+        else:
+            assert np.array_equal(err_h[:, sl], e0.cpu().numpy()[:, sl])
+        assert np.array_equal(d_h[sl], d0_h[sl] + g_h[0, sl])  # one fp32 add per element
+    # no delta: err only
+    err2 = e0.clone()
+    ctx.acc_error_feedback(grads, err2, None)
+    torch.cuda.synchronize()
+    assert torch.equal(err2, err)
+
+
+def test_layer_norms_match_oracle():
+    table = _table_mixed()
+    W = 3
+    ctx = binding.Context(table, W)
+    grads, _ = _random_inputs(table, W, 2)
+    n2 = torch.zeros(W * table.n_layers, dtype=torch.float64, device="cuda")
+    ctx.acc_layer_norms(grads, W, n2)
+    n2b = torch.zeros_like(n2)
+    ctx.acc_layer_norms(grads, W, n2b)
+    torch.cuda.synchronize()
+    assert torch.equal(n2, n2b)  # bit-reproducible
+    got = n2.cpu().numpy().reshape(W, -1)
+    for w in range(W):
+        want = orc.layer_norms2(grads[w].cpu().numpy(), H.layers_of(table))
+        assert np.allclose(got[w], want, rtol=1e-12, atol=0)
+    one = torch.zeros(table.n_layers, dtype=torch.float64, device="cuda")
+    ctx.acc_layer_norms(grads[1], 1, one)
+    torch.cuda.synchronize()
+    assert np.array_equal(one.cpu().numpy(), got[1])
+
+
+def test_detect_regime_truth_table_and_random():
+    L = 300
+    table = wl.make_table([(f"v{i}", (4,)) for i in range(L)])
+    ctx = binding.Context(table, 1, eta=0.5)
+    rng = np.random.default_rng(3)
+    prev = rng.uniform(0.0, 4.0, L)
+    curr = rng.uniform(0.0, 4.0, L)
+    # exactly representable boundary cases (a, b) -> |a-b| vs 0.5 a
+    cases = [(1.0, 0.5), (1.0, 1.5), (1.0, 0.75), (1.0, 1.25), (4.0, 1.0), (0.0, 0.0), (0.0, 3.0), (2.0, 1.0), (2.0, 3.0)]
+    for i, (a, b) in enumerate(cases):
+        prev[i], curr[i] = a * a, b * b
+    prev[20:30] = -1.0  # no previous window
+    for lr_next in (0.1, 0.01):
+        p = torch.tensor(prev, device="cuda"); c = torch.tensor(curr, device="cuda")
+        level = torch.full((L,), 7, dtype=torch.uint8, device="cuda")
+        delta = torch.ones(table.stride, device="cuda")
+        ctx.acc_detect_regime(c, p, 0.1, lr_next, level, delta)
+        torch.cuda.synchronize()
+        want, want_prev = orc.detect_regime(curr, prev, 0.1, lr_next, np.float32(0.5))
+        assert np.array_equal(level.cpu().numpy(), want)
+        assert np.array_equal(p.cpu().numpy(), want_prev)
+        assert float(delta.abs().max()) == 0.0
+    assert list(want[:9]) == [1] * 9  # lr decay: all low
+    want, _ = orc.detect_regime(curr, prev, 0.1, 0.1, 0.5)
+    assert list(want[:9]) == [1, 1, 0, 0, 1, 1, 1, 1, 1]
+
+
+# ------------------------------------------------------------------ PowerSGD
+@pytest.mark.parametrize("W,rank_low,rank_high", [(1, 2, 1), (2, 2, 1), (3, 3, 2), (4, 4, 1), (8, 4, 4), (5, 1, 1)])
+def test_powersgd_step_matches_oracle(W, rank_low, rank_high):
+    table = _table_mixed()
+    ctx = binding.Context(table, W, rank_low=rank_low, rank_high=rank_high, gs_eps=1e-8)
+    grads, err = _random_inputs(table, W, 10 + W)
+    q = ctx.new_q(wl.initial_q(table, 4, seed=W))  # ranks beyond rank_low hold values that must survive
+    p = ctx.new_p()
+    p.fill_(3.25)
+    level = torch.tensor([(l * 7 + W) % 3 != 0 for l in range(table.n_layers)], dtype=torch.uint8, device="cuda")
+    out = torch.full((table.stride,), float("nan"), device="cuda")
+    delta = torch.zeros(table.stride, device="cuda")
+    for it in range(3):  # three consecutive steps: warm start, memory carried over
+        e0, q0 = err.clone(), q.clone()
+        ctx.acc_powersgd_step(grads, err, q, p, level, out, delta)
+        torch.cuda.synchronize()
+        H.check_powersgd_against_oracle(ctx, table, grads, e0, q0, level, out, err, q, p, rank_low, rank_high, 1e-8)
+        grads, _ = _random_inputs(table, W, 100 + it)
+    assert ctx.last_launch_count() == 5
+
+
+def test_powersgd_invariants_and_exact_recovery():
+    table = wl.make_table([("a", (48, 650)), ("v", (10,)), ("b", (200, 96))])
+    W, r = 4, 2
+    ctx = binding.Context(table, W, rank_low=r, rank_high=1, gs_eps=0.0)
+    rng = np.random.default_rng(5)
+    grads = torch.zeros(W, table.stride, device="cuda")
+    for l, sl in table.slices():
+        if table.kind[l] == wl.MATRIX:
+            n, m = int(table.rows[l]), int(table.cols[l])
+            B = rng.integers(-4, 5, (n, r)).astype(np.float64) @ rng.integers(-4, 5, (r, m)).astype(np.float64)
+            grads[:, sl] = torch.tensor(B.reshape(-1), dtype=torch.float32, device="cuda")
+    err = torch.zeros_like(grads)
+    q = ctx.new_q(wl.initial_q(table, r))
+    p = ctx.new_p()
+    level = torch.ones(table.n_layers, dtype=torch.uint8, device="cuda")
+    out = torch.zeros(table.stride, device="cuda")
+    ctx.acc_powersgd_step(grads, err, q, p, level, out)
+    torch.cuda.synchronize()
+    for l, sl in table.slices():
+        if table.kind[l] != wl.MATRIX:
+            continue
+        M = grads[0, sl]
+        assert float((out[sl] - M).norm() / M.norm()) < 1e-5           # rank-r input is recovered
+        assert float(err[:, sl].norm() / M.norm()) < 1e-5
+        n = int(table.rows[l])
+        ph = p[ctx.p_row[l]:ctx.p_row[l] + n, :r].double()
+        assert torch.allclose(ph.T @ ph, torch.eye(r, device="cuda", dtype=torch.float64), atol=1e-5)
+    # error-feedback invariant A + e'_w = g_w + e_w on random data
+    grads2, err2 = _random_inputs(table, W, 6)
+    M = grads2 + err2
+    ctx.acc_powersgd_step(grads2, err2, q, p, level, out)
+    torch.cuda.synchronize()
+    for l, sl in table.slices():
+        if table.kind[l] == wl.MATRIX:
+            for w in range(W):
+                assert float((out[sl] + err2[w, sl] - M[w, sl]).norm() / M[w, sl].norm()) < 1e-6
+
+
+# ------------------------------------------------------------------ TopK
+@pytest.mark.parametrize("W,low_bp,high_bp", [(1, 1000, 100), (3, 1000, 100), (4, 2500, 200), (2, 10000, 9900), (2, 1, 1)])
+def test_topk_step_bit_exact(W, low_bp, high_bp):
+    table = _table_mixed()
+    ctx = binding.Context(table, W, topk_low_bp=low_bp, topk_high_bp=high_bp)
+    grads, err = _random_inputs(table, W, 20 + W)
+    level = torch.tensor([(l * 5 + W) % 2 for l in range(table.n_layers)], dtype=torch.uint8, device="cuda")
+    vals, idx, counts = ctx.new_topk_buffers()
+    out = torch.full((table.stride,), float("nan"), device="cuda")
+    for it in range(3):  # memory carried over: kept entries are +0.0 in the next add
+        e0 = err.clone()
+        ctx.acc_topk_step(grads, err, level, vals, idx, counts, out)
+        torch.cuda.synchronize()
+        H.check_topk_against_oracle(ctx, table, grads, e0, level, vals, idx, counts, out, err, low_bp, high_bp)
+        grads, _ = _random_inputs(table, W, 200 + it)
+    assert ctx.last_launch_count() == 7
+
+
+def test_topk_ties_zeros_and_degenerate_layers():
+    table = wl.make_table([
+        ("ties", (40, 650)),       # many exact duplicates around the threshold
+        ("zeros", (30, 1000)),     # all zero: keeps the k lowest indices
+        ("sparse", (500, 64)),     # row-sparse: k exceeds the non-zeros, filled with zeros by index
+        ("equal", (3, 4097)),      # all equal magnitude, mixed sign
+        ("small", (2, 3)), ("v", (7,)),
+        ("quant", (64, 640)),      # few distinct values: ties at every level of the radix select
+    ])
+    W = 3
+    ctx = binding.Context(table, W, topk_low_bp=1000, topk_high_bp=100)
+    g = torch.Generator(device="cuda").manual_seed(7)
+    grads = torch.zeros(W, table.stride, device="cuda")
+    sl = {table.names[l]: s for l, s in table.slices()}
+    n = sl["ties"].stop - sl["ties"].start
+    base = torch.randn(W, n, generator=g, device="cuda")
+    dup = torch.randint(0, n, (W, n // 3), generator=g, device="cuda")
+    src = torch.randint(0, n, (W, n // 3), generator=g, device="cuda")
+    sign = torch.randint(0, 2, (W, n // 3), generator=g, device="cuda").float() * 2 - 1
+    base.scatter_(1, dup, torch.gather(base, 1, src).abs() * sign)
+    grads[:, sl["ties"]] = base
+    rows = torch.randperm(500, generator=g, device="cuda")[:10]
+    sp = torch.zeros(W, 500, 64, device="cuda")
+    sp[:, rows] = torch.randn(W, 10, 64, generator=g, device="cuda")
+    grads[:, sl["sparse"]] = sp.reshape(W, -1)
+    ne = sl["equal"].stop - sl["equal"].start
+    grads[:, sl["equal"]] = (torch.randint(0, 2, (W, ne), generator=g, device="cuda").float() * 2 - 1) * 0.375
+    grads[:, sl["small"]] = torch.randn(W, 6, generator=g, device="cuda")
+    grads[:, sl["v"]] = torch.randn(W, 7, generator=g, device="cuda")
+    nq = sl["quant"].stop - sl["quant"].start
+    grads[:, sl["quant"]] = torch.randint(-3, 4, (W, nq), generator=g, device="cuda").float() * 0.25
+    err = torch.zeros_like(grads)
+    err[:, sl["zeros"]] = -0.0
+    for level_val in (1, 0):
+        level = torch.full((table.n_layers,), level_val, dtype=torch.uint8, device="cuda")
+        e = err.clone()
+        vals, idx, counts = ctx.new_topk_buffers()
+        out = torch.zeros(table.stride, device="cuda")
+        ctx.acc_topk_step(grads, e, level, vals, idx, counts, out)
+        torch.cuda.synchronize()
+        H.check_topk_against_oracle(ctx, table, grads, err, level, vals, idx, counts, out, e, 1000, 100)
+
+
+def test_topk_is_bit_reproducible():
+    table = _table_mixed()
+    W = 4
+    ctx = binding.Context(table, W)
+    grads, err = _random_inputs(table, W, 31)
+    level = torch.ones(table.n_layers, dtype=torch.uint8, device="cuda")
+    res = []
+    for rep in range(2):
+        e = err.clone()
+        vals, idx, counts = ctx.new_topk_buffers()
+        out = torch.zeros(table.stride, device="cuda")
+        ctx.acc_topk_step(grads, e, level, vals, idx, counts, out)
+        torch.cuda.synchronize()
+        res.append((e, vals, idx, counts, out))
+    for a, b in zip(res[0], res[1]):
+        assert torch.equal(a, b)
+
+
+# ------------------------------------------------------------------ argument checks (no kernels run)
+def test_bad_arguments_are_rejected():
+    table = _table_mixed()
+    ctx = binding.Context(table, 2)
+    grads, err = _random_inputs(table, 2, 1)
+    with pytest.raises(binding.AccError) as ei:
+        ctx.acc_error_feedback(grads.view(-1)[1:-3].view(-1), err)  # misaligned pointer
+    assert ei.value.status == 2
+    with pytest.raises(ValueError):
+        ctx.acc_error_feedback(grads.cpu(), err)
+    with pytest.raises(binding.AccError):
+        binding.Context(table, 2, rank_low=5)
+    with pytest.raises(binding.AccError):
+        binding.Context(table, 2, topk_low_bp=50, topk_high_bp=100)

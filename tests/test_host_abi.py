@@ -1,0 +1,75 @@
+"""CPU-side checks of the C-ABI library: it loads, exports every symbol include/acc.h declares, and its
+host-only entry points (configuration checks, workspace sizing, communication accounting) behave."""
+import ctypes as C
+import os
+import re
+
+import pytest
+
+from oracle import accordion_oracle as orc
+from paper_2010_16248_b200 import binding, build, workloads as wl
+from tests import helpers as H
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    build.build_library()
+    return binding.lib()
+
+
+def _declared():
+    text = open(os.path.join(ROOT, "include", "acc.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(acc_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol(lib):
+    names = _declared()
+    assert len(names) >= 13
+    for n in names:
+        assert hasattr(lib, n), f"{n} declared in acc.h but not exported"
+    assert set(names) == set(binding.EXPORTS)
+
+
+def test_workspace_sizing_and_config_validation(lib):
+    table = wl.make_table(wl.shapes_resnet18(100))
+    cfg = binding.make_config(table, 4)
+    n = C.c_size_t()
+    assert lib.acc_workspace_bytes(C.byref(cfg), C.byref(n)) == 0 and n.value > 0
+    small = n.value
+    cfg8 = binding.make_config(table, 8)
+    assert lib.acc_workspace_bytes(C.byref(cfg8), C.byref(n)) == 0 and n.value > small
+    bad = [dict(rank_low=5), dict(rank_low=1, rank_high=2), dict(topk_low_bp=0, topk_high_bp=0),
+           dict(topk_low_bp=20000), dict(decider=4), dict(eta=-1.0), dict(worker_stride=table.stride - 4)]
+    for kw in bad:
+        c = binding.make_config(table, 4, **kw)
+        assert lib.acc_workspace_bytes(C.byref(c), C.byref(n)) == 1, kw
+    c = binding.make_config(table, 4, worker_stride=table.stride + 2)
+    assert lib.acc_workspace_bytes(C.byref(c), C.byref(n)) == 2            # stride not a multiple of 4
+    c = binding.make_config(table, 4)
+    c.layers[3].offset += 1
+    assert lib.acc_workspace_bytes(C.byref(c), C.byref(n)) == 2            # misaligned layer
+    c = binding.make_config(table, 4)
+    c.layers[5].offset = c.layers[4].offset                               # overlapping layers
+    assert lib.acc_workspace_bytes(C.byref(c), C.byref(n)) == 1
+    h = C.c_void_p()
+    assert lib.acc_create(C.byref(cfg), None, 0, C.byref(h)) == 3          # no workspace
+    assert lib.acc_strerror(3).decode().startswith("workspace")
+
+
+def test_floats_sent_matches_oracle_and_tables(lib):
+    for shapes, W, rl, rh in ((wl.shapes_resnet18(10), 4, 2, 1), (wl.shapes_vgg19bn(10), 4, 4, 1)):
+        table = wl.make_table(shapes)
+        layers = H.layers_of(table)
+        cfg = binding.make_config(table, W, rank_low=rl, rank_high=rh)
+        for lv in (0, 1):
+            level = [lv] * table.n_layers
+            for comp, name in ((binding.POWERSGD, "powersgd"), (binding.TOPK, "topk")):
+                want = orc.floats_sent_per_iteration(layers, level, name, W, rl, rh, 1000, 100)
+                assert binding.acc_floats_sent(cfg, level, comp) == want
+    # Table 1, ResNet-18 / CIFAR-10, rank 2: 2418.4 million floats over 300 epochs x 98 iterations
+    table = wl.make_table(wl.shapes_resnet18(10))
+    cfg = binding.make_config(table, 4, rank_low=2, rank_high=1)
+    assert abs(binding.acc_floats_sent(cfg, [1] * table.n_layers, binding.POWERSGD) * 29400 / 1e6 - 2418.4) < 0.1
