@@ -42,7 +42,7 @@ def test_workspace_sizing_and_config_validation(lib):
     cfg8 = binding.make_config(table, 8)
     assert lib.acc_workspace_bytes(C.byref(cfg8), C.byref(n)) == 0 and n.value > small
     bad = [dict(rank_low=5), dict(rank_low=1, rank_high=2), dict(topk_low_bp=0, topk_high_bp=0),
-           dict(topk_low_bp=20000), dict(decider=4), dict(eta=-1.0), dict(worker_stride=table.stride - 4)]
+           dict(topk_low_bp=20000), dict(decider=4), dict(eta=-1.0), dict(worker_stride=table.stride // 8 * 4)]
     for kw in bad:
         c = binding.make_config(table, 4, **kw)
         assert lib.acc_workspace_bytes(C.byref(c), C.byref(n)) == 1, kw
