@@ -1,0 +1,363 @@
+#!/usr/bin/env python
+"""Benchmark of the Accordion gradient-compression step on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config 5] [--impl reference]
+
+One "step" is one pass of the whole hot path over one batch of synthetic worker gradients: the
+PowerSGD step and the TopK step of the workload (each with its own error memory, both with error
+feedback, the first also accumulating the detector's gradient), plus -- every `check_every` steps --
+the layer norms and the regime test that sets the per-layer levels for the following steps.
+
+metric = GB/s of gradient processed: each compressor pass consumes the W workers' gradients once, so a
+step processes (number of compressors) x 4 x W x N bytes.  Prints ONE JSON line (rank 0).
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+import torch  # noqa: E402
+
+METRIC = "compression_step_gradient_throughput"
+UNIT = "GB/s"
+RING = 4  # pre-generated gradient batches cycled through the steps (each far larger than L2)
+REF_LAYER = "rnn.weight_hh_l0"
+
+
+def _peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    return 6650.0, "fallback (6.65 TB/s, no MEASURED_PEAKS.json)"
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons of one GPU while the timed region runs."""
+
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append((time.time(), line.strip()))
+
+    def stop(self, t0, t1):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=2)
+        except Exception:
+            pass
+        rows = [l for (t, l) in self.lines if t0 <= t <= t1 + 0.15] or [l for (_, l) in self.lines]
+        sm, mx, reasons, power = [], [], set(), []
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for l in rows:
+            f = [x.strip() for x in l.split(",")]
+            if len(f) < 8:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1])); power.append(float(f[2]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[4:8]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "power_w": float(np.median(power)) if power else None, "samples": len(sm),
+                "reasons": sorted(reasons)}
+
+
+def _kernel_alg_bytes(name, units):
+    """Algorithmic bytes one launch of a streaming kernel must move, per MATRIX parameter-worker
+    (fp32): reads + writes that the method itself requires of that pass."""
+    per_unit = {
+        "psgd_project_kernel": 12.0,    # read g, read e, write M
+        "psgd_residual_kernel": 8.0,    # read M, write e'
+        "topk_ef_hist1_kernel": 12.0,   # read g, read e, write M
+        "topk_hist2_kernel": 4.0,       # read M
+        "topk_hist3_kernel": 4.0,       # read M
+        "topk_select_kernel": 4.0,      # read M (+ sparse writes, not counted)
+        "ef_kernel": 12.0,
+    }
+    return per_unit.get(name, 0.0) * units
+
+
+def run_reference(args, rank, world):
+    """Times the CPU oracle, as it stands, on a bounded sample of the workload (one LSTM gate matrix
+    with all workers, both compressors)."""
+    if rank != 0:
+        return
+    from oracle import accordion_oracle as orc
+    from paper_2010_16248_b200 import workloads as wl
+    from tests import helpers as H
+    w = wl.workload(args.config)
+    full = w.table
+    li = full.names.index(REF_LAYER) if REF_LAYER in full.names else int(np.argmax(full.kind == wl.MATRIX))
+    n, m = int(full.rows[li]), int(full.cols[li])
+    sub = wl.make_table([(full.names[li], (n, m))])
+    layers = H.layers_of(sub)
+    rng = np.random.default_rng(1234)
+    W = w.n_workers
+    batches = [rng.standard_normal((W, sub.stride)).astype(np.float32) for _ in range(2)]
+    err_p = np.zeros((W, sub.stride), np.float32)
+    err_t = np.zeros((W, sub.stride), np.float32)
+    q = [rng.standard_normal((m, w.rank_low)).astype(np.float32)]
+    level = np.ones(1, np.uint8)
+    delta = np.zeros(sub.stride)
+    prev = -np.ones(1)
+
+    def step(t):
+        nonlocal err_p, err_t, q, level, prev
+        g = batches[t % 2]
+        orc.accumulate(delta, g[0], layers)
+        n_comp = 0
+        if "powersgd" in w.compressors:
+            _, e, qn, _ = orc.powersgd_step(g, err_p, q, level, layers, w.rank_low, w.rank_high)
+            err_p, q = e.astype(np.float32), [x.astype(np.float32) for x in qn]
+            n_comp += 1
+        if "topk" in w.compressors:
+            _, _, _, _, err_t = orc.topk_step(g, err_t, level, layers, w.topk_low_bp, w.topk_high_bp)
+            n_comp += 1
+        if (t + 1) % w.check_every == 0:
+            level, prev = orc.detect_regime(orc.layer_norms2(delta, layers), prev, 0.1, 0.1, w.eta)
+            delta[:] = 0
+        return n_comp
+
+    for t in range(args.warmup):
+        step(t)
+    t0 = time.perf_counter()
+    n_comp = 0
+    for t in range(args.steps):
+        n_comp = step(args.warmup + t)
+    dt = time.perf_counter() - t0
+    bytes_per_step = n_comp * 4.0 * W * n * m
+    value = bytes_per_step * args.steps / dt / 1e9
+    try:
+        from threadpoolctl import threadpool_info
+        cores = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        cores = 1
+    sample = f"layer {full.names[li]} ({n}x{m}) of {w.name}, all {W} workers, {n_comp} compressor passes per step"
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": w.name, "sample": sample},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def cpu_baseline(w, seconds_budget=20.0):
+    """The oracle timed on the host cores on a bounded sample (same sample as --impl reference)."""
+    ns = argparse.Namespace(config=w.config_id, warmup=1, steps=3, gpus=1)
+    import io
+    from contextlib import redirect_stdout
+    buf = io.StringIO()
+    with redirect_stdout(buf):
+        run_reference(ns, 0, 1)
+    return json.loads(buf.getvalue().strip().splitlines()[-1])["cpu_baseline"]
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--config", type=int, default=5, help="BASELINE config 1..5 (default: 5, the largest gradient set)")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--e2e-steps", type=int, default=8)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        run_reference(args, rank, world)
+        return
+
+    import torch.distributed as dist
+    from paper_2010_16248_b200 import build, pipeline, workloads as wl
+    if rank == 0:
+        build.build_library()
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU path)"
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+        dist.barrier()
+
+    w = wl.workload(args.config)
+    table, W = w.table, w.n_workers
+    n_comp = len(w.compressors)
+    stream_gen = wl.GradientStream(w, device=dev)
+    # independent replicas: every rank draws its own gradient batches
+    ring = [stream_gen.grads(1000 * rank + t) for t in range(RING)]
+    eng = pipeline.AccordionStep(table, W, w.compressors, w.rank_low, w.rank_high, w.topk_low_bp, w.topk_high_bp,
+                                 w.eta, 1e-8, w.check_every, device=dev)
+    n_mat = table.n_matrix_params
+    grad_bytes_step = n_comp * 4.0 * W * table.n_params
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    step_no = 0
+
+    def run_steps(k, events=None):
+        nonlocal step_no
+        for i in range(k):
+            if events is not None:
+                events[i][0].record()
+            eng.step(ring[step_no % RING])
+            if events is not None:
+                events[i][1].record()
+            step_no += 1
+
+    # ---- warm-up, then the timed region (device-resident inputs)
+    run_steps(args.warmup)
+    barrier()
+    K = args.steps
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    if sampler:
+        sampler.start()
+        time.sleep(0.25)
+    barrier()
+    launches0 = eng.launches
+    t0 = time.time()
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    start.record()
+    run_steps(K, ev)
+    stop.record()
+    barrier()
+    t1 = time.time()
+    clocks = sampler.stop(t0, t1) if sampler else None
+    total_ms = start.elapsed_time(stop)
+    gpu_launches = eng.launches - launches0
+    per_step = np.array([a.elapsed_time(b) for a, b in ev])
+    if world > 1:
+        t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    ms_per_step = total_ms / K
+    value = grad_bytes_step * world / (ms_per_step * 1e-3) / 1e9
+
+    # ---- same K steps again with per-kernel CUDA events (on the launching stream) for the roofline
+    eng.ctx.acc_profile_enable(True)
+    run_steps(K)
+    torch.cuda.synchronize()
+    prof = eng.ctx.acc_profile_read()
+    eng.ctx.acc_profile_enable(False)
+    peak, peak_src = _peaks()
+    units = W * n_mat
+    total_k_ms = sum(ms for ms, _ in prof.values())
+    kernels = {}
+    for name, (ms, cnt) in sorted(prof.items(), key=lambda kv: -kv[1][0]):
+        alg = _kernel_alg_bytes(name, units)
+        avg = ms / cnt
+        kernels[name] = {"launches": cnt, "ms_total": round(ms, 4), "share": round(ms / total_k_ms, 4),
+                         "avg_ms": round(avg, 5),
+                         "alg_gbs": round(alg / (avg * 1e-3) / 1e9, 1) if alg else None}
+    dom = next(iter(kernels))
+    dom_alg = _kernel_alg_bytes(dom, units)
+    dom_avg_ms = prof[dom][0] / prof[dom][1]
+    achieved = dom_alg / (dom_avg_ms * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "kernel": dom, "achieved": round(achieved, 1), "peak": peak, "unit": "GB/s",
+                "frac": round(achieved / peak, 4), "peak_source": peak_src, "traffic": TRAFFIC.get((args.config, dom)),
+                "alg_bytes_per_launch": dom_alg,
+                "step_frac_of_12B": round(n_comp * 12.0 * units / (ms_per_step * 1e-3) / 1e9 / peak, 4)}
+
+    # ---- end to end: host (pinned) gradients -> device every step, result read back to the host
+    e2e = None
+    ke = max(1, min(args.e2e_steps, K))
+    host = [torch.empty(W, table.stride, dtype=torch.float32).pin_memory() for _ in range(2)]
+    for i in range(2):
+        host[i].copy_(ring[i])
+    outs_host = [torch.empty(table.stride, dtype=torch.float32).pin_memory() for _ in eng.outputs()]
+    stage = torch.empty_like(ring[0])
+
+    def e2e_step(i):
+        stage.copy_(host[i % 2], non_blocking=True)
+        eng.step(stage)
+        for oh, od in zip(outs_host, eng.outputs()):
+            oh.copy_(od, non_blocking=True)
+
+    e2e_step(0)
+    barrier()
+    s2, e2 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    s2.record()
+    for i in range(ke):
+        e2e_step(i + 1)
+    e2.record()
+    barrier()
+    e2e_ms = s2.elapsed_time(e2)
+    if world > 1:
+        t = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    e2e = {"value": grad_bytes_step * world / (e2e_ms / ke * 1e-3) / 1e9, "unit": UNIT, "steps": ke,
+           "ms_per_step": e2e_ms / ke, "h2d_bytes_per_step": int(4 * W * table.stride),
+           "d2h_bytes_per_step": int(4 * table.stride * len(outs_host))}
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        cpu = cpu_baseline(w)
+
+    if rank == 0:
+        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": args.warmup,
+                "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+                "dtype": "f32", "data": "synthetic",
+                "config": {"workload": w.name, "n_workers": W, "params": table.n_params,
+                           "compressors": list(w.compressors), "rank_low_high": [w.rank_low, w.rank_high],
+                           "topk_bp_low_high": [w.topk_low_bp, w.topk_high_bp], "check_every": w.check_every,
+                           "gradient_bytes_per_step": grad_bytes_step,
+                           "l2_policy": f"inputs larger than L2: {RING} gradient batches of "
+                                        f"{4 * W * table.stride / 1e6:.0f} MB cycled, no flush",
+                           "multi_gpu": "independent replicas, no collective"},
+                "clocks": clocks, "e2e": e2e, "gpu_launches": gpu_launches,
+                "roofline": roofline, "cpu_baseline": cpu,
+                "step_ms": {"median": float(np.median(per_step)), "min": float(per_step.min()),
+                            "max": float(per_step.max())},
+                "kernels": kernels}
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per launch of the dominant kernel, from the
+# ncu captures summarised under profiles/ ; keyed by (config, kernel).
+TRAFFIC = {}
+
+if __name__ == "__main__":
+    main()

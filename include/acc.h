@@ -156,6 +156,18 @@ int64_t acc_floats_sent(const acc_config* cfg, const uint8_t* level_host, int32_
  * on this context launched (for launch accounting in benchmarks).                                  */
 int32_t acc_last_launch_count(const acc_ctx* ctx);
 
+/* Per-kernel timing aid (no counterpart in the paper).  While enabled, every kernel the library
+ * launches on this context is bracketed by CUDA events on its stream.  acc_profile_read waits for the
+ * recorded events (blocks the host until those kernels finished), writes per kernel the summed
+ * duration in milliseconds and the number of launches since the last read into HOST arrays of
+ * n >= acc_profile_kernel_count() entries, and clears the record.  Kernel i is named
+ * acc_profile_kernel_name(i).  Event records cost about a microsecond each: leave profiling off
+ * when timing whole steps.                                                                          */
+int acc_profile_enable(acc_ctx* ctx, int32_t enable);
+int acc_profile_read(acc_ctx* ctx, double* ms, int32_t* launches, int32_t n);
+int32_t acc_profile_kernel_count(void);
+const char* acc_profile_kernel_name(int32_t i);
+
 const char* acc_strerror(int status);
 
 #ifdef __cplusplus

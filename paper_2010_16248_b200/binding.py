@@ -41,7 +41,8 @@ class acc_config(C.Structure):
 
 EXPORTS = ["acc_workspace_bytes", "acc_create", "acc_destroy", "acc_factor_layout", "acc_topk_layout",
            "acc_error_feedback", "acc_layer_norms", "acc_detect_regime", "acc_powersgd_step", "acc_topk_step",
-           "acc_floats_sent", "acc_last_launch_count", "acc_strerror"]
+           "acc_floats_sent", "acc_last_launch_count", "acc_strerror", "acc_profile_enable", "acc_profile_read",
+           "acc_profile_kernel_count", "acc_profile_kernel_name"]
 
 _lib = None
 
@@ -73,8 +74,15 @@ def lib() -> C.CDLL:
     L.acc_last_launch_count.restype = i32
     L.acc_strerror.argtypes = [C.c_int]
     L.acc_strerror.restype = C.c_char_p
+    L.acc_profile_enable.argtypes = [vp, i32]
+    L.acc_profile_read.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(i32), i32]
+    L.acc_profile_kernel_count.argtypes = []
+    L.acc_profile_kernel_count.restype = i32
+    L.acc_profile_kernel_name.argtypes = [i32]
+    L.acc_profile_kernel_name.restype = C.c_char_p
     for name in EXPORTS:
-        if name not in ("acc_floats_sent", "acc_last_launch_count", "acc_strerror"):
+        if name not in ("acc_floats_sent", "acc_last_launch_count", "acc_strerror", "acc_profile_kernel_count",
+                        "acc_profile_kernel_name"):
             getattr(L, name).restype = C.c_int
     _lib = L
     return L
@@ -189,6 +197,16 @@ class Context:
                                         _ptr(level, torch.uint8), _ptr(vals, torch.float32), _ptr(idx, torch.int32),
                                         _ptr(counts, torch.int32), _ptr(out, torch.float32),
                                         _ptr(delta, torch.float32), _stream(stream)), "acc_topk_step")
+
+    def acc_profile_enable(self, enable: bool):
+        self._check(lib().acc_profile_enable(self._h, int(bool(enable))), "acc_profile_enable")
+
+    def acc_profile_read(self):
+        """{kernel name: (milliseconds, launches)} since the last read; waits for the recorded kernels."""
+        n = int(lib().acc_profile_kernel_count())
+        ms, cnt = (C.c_double * n)(), (C.c_int32 * n)()
+        self._check(lib().acc_profile_read(self._h, ms, cnt, n), "acc_profile_read")
+        return {lib().acc_profile_kernel_name(i).decode(): (float(ms[i]), int(cnt[i])) for i in range(n) if cnt[i]}
 
     def last_launch_count(self) -> int:
         return int(lib().acc_last_launch_count(self._h))

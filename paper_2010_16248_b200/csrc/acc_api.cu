@@ -187,6 +187,7 @@ int acc_create(const acc_config* cfg, void* workspace, size_t workspace_bytes, a
 
 int acc_destroy(acc_ctx* ctx) {
   if (!ctx) return ACC_EINVAL;
+  for (ProfSlot& sl : ctx->prof_slots) { cudaEventDestroy(sl.a); cudaEventDestroy(sl.b); }
   delete ctx;
   return ACC_OK;
 }
@@ -277,6 +278,40 @@ int64_t acc_floats_sent(const acc_config* cfg, const uint8_t* level_host, int32_
     }
   }
   return total;
+}
+
+int acc_profile_enable(acc_ctx* ctx, int32_t enable) {
+  if (!ctx) return ACC_EINVAL;
+  ctx->prof = enable != 0;
+  ctx->prof_used = 0;
+  return ACC_OK;
+}
+
+int acc_profile_read(acc_ctx* ctx, double* ms, int32_t* launches, int32_t n) {
+  if (!ctx || !ms || !launches || n < PH_COUNT) return ACC_EINVAL;
+  for (int i = 0; i < n; ++i) { ms[i] = 0.0; launches[i] = 0; }
+  for (size_t i = 0; i < ctx->prof_used; ++i) {
+    const ProfSlot& sl = ctx->prof_slots[i];
+    float t = 0.f;
+    if (cudaEventSynchronize(sl.b) != cudaSuccess || cudaEventElapsedTime(&t, sl.a, sl.b) != cudaSuccess)
+      return ACC_ECUDA;
+    ms[sl.phase] += (double)t;
+    launches[sl.phase] += 1;
+  }
+  ctx->prof_used = 0;
+  return ACC_OK;
+}
+
+int32_t acc_profile_kernel_count(void) { return PH_COUNT; }
+
+const char* acc_profile_kernel_name(int32_t i) {
+  static const char* names[PH_COUNT] = {
+      "ef_kernel", "norm_partial_kernel", "norm_final_kernel", "detect_kernel",
+      "psgd_project_kernel", "psgd_orthonormalise_kernel", "psgd_qpartial_kernel", "psgd_qreduce_kernel",
+      "psgd_residual_kernel",
+      "topk_ef_hist1_kernel", "topk_pick1_kernel", "topk_hist2_kernel", "topk_pick2_kernel", "topk_hist3_kernel",
+      "topk_pick3_scan_kernel", "topk_select_kernel"};
+  return (i >= 0 && i < PH_COUNT) ? names[i] : "";
 }
 
 int32_t acc_last_launch_count(const acc_ctx* ctx) { return ctx ? ctx->last_launches : -1; }

@@ -96,28 +96,37 @@ __global__ void detect_kernel(const double* __restrict__ n2c, double* __restrict
 
 cudaError_t launch_error_feedback(acc_ctx* ctx, const float* grads, float* err, float* delta, cudaStream_t s) {
   dim3 grid((unsigned)ctx->plan.tiles.size(), (unsigned)ctx->cfg.n_workers);
-  ef_kernel<<<grid, 256, 0, s>>>(ctx->d_layers, ctx->d_tiles, grads, err, delta, ctx->cfg.worker_stride,
-                                 ctx->cfg.decider);
-  ctx->last_launches += 1;
+  {
+    PhaseTimer pt(ctx, PH_EF, s);
+    ef_kernel<<<grid, 256, 0, s>>>(ctx->d_layers, ctx->d_tiles, grads, err, delta, ctx->cfg.worker_stride,
+                                   ctx->cfg.decider);
+  }
   return cudaGetLastError();
 }
 
 cudaError_t launch_layer_norms(acc_ctx* ctx, const float* buf, long long stride, int n_bufs, double* norm2,
                                cudaStream_t s) {
   const int nt = (int)ctx->plan.tiles.size();
-  norm_partial_kernel<<<dim3((unsigned)nt, (unsigned)n_bufs), 256, 0, s>>>(ctx->d_layers, ctx->d_tiles, buf, stride,
-                                                                          ctx->d_norm_part, nt);
-  norm_final_kernel<<<dim3((unsigned)ctx->cfg.n_layers, (unsigned)n_bufs), 32, 0, s>>>(
-      ctx->d_layers, ctx->d_norm_part, norm2, ctx->cfg.n_layers, nt);
-  ctx->last_launches += 2;
+  {
+    PhaseTimer pt(ctx, PH_NORM_PARTIAL, s);
+    norm_partial_kernel<<<dim3((unsigned)nt, (unsigned)n_bufs), 256, 0, s>>>(ctx->d_layers, ctx->d_tiles, buf, stride,
+                                                                            ctx->d_norm_part, nt);
+  }
+  {
+    PhaseTimer pt(ctx, PH_NORM_FINAL, s);
+    norm_final_kernel<<<dim3((unsigned)ctx->cfg.n_layers, (unsigned)n_bufs), 32, 0, s>>>(
+        ctx->d_layers, ctx->d_norm_part, norm2, ctx->cfg.n_layers, nt);
+  }
   return cudaGetLastError();
 }
 
 cudaError_t launch_detect(acc_ctx* ctx, const double* n2c, double* n2p, float lr_curr, float lr_next, uint8_t* level,
                           cudaStream_t s) {
   const int L = ctx->cfg.n_layers;
-  detect_kernel<<<(L + 127) / 128, 128, 0, s>>>(n2c, n2p, lr_curr, lr_next, (double)ctx->cfg.eta, level, L);
-  ctx->last_launches += 1;
+  {
+    PhaseTimer pt(ctx, PH_DETECT, s);
+    detect_kernel<<<(L + 127) / 128, 128, 0, s>>>(n2c, n2p, lr_curr, lr_next, (double)ctx->cfg.eta, level, L);
+  }
   return cudaGetLastError();
 }
 

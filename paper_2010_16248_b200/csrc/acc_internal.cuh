@@ -43,6 +43,16 @@ struct Select {
   int pad;
 };
 
+// Kernels of the library, for per-kernel timing (acc_profile_*).
+enum Phase {
+  PH_EF = 0, PH_NORM_PARTIAL, PH_NORM_FINAL, PH_DETECT,
+  PH_PSGD_PROJECT, PH_PSGD_ORTHO, PH_PSGD_QPARTIAL, PH_PSGD_QREDUCE, PH_PSGD_RESIDUAL,
+  PH_TOPK_EF_HIST1, PH_TOPK_PICK1, PH_TOPK_HIST2, PH_TOPK_PICK2, PH_TOPK_HIST3, PH_TOPK_PICK3_SCAN, PH_TOPK_SELECT,
+  PH_COUNT
+};
+
+struct ProfSlot { int phase; cudaEvent_t a, b; };
+
 struct Plan {
   std::vector<DevLayer> layers;
   std::vector<RowItem> row_items;
@@ -67,6 +77,9 @@ struct acc_ctx {
   char* ws = nullptr;
   int sm_count = 148;
   int last_launches = 0;
+  bool prof = false;                 // per-kernel event timing on
+  std::vector<acc::ProfSlot> prof_slots;
+  size_t prof_used = 0;
   // device views into the workspace
   acc::DevLayer* d_layers = nullptr;
   acc::RowItem* d_row_items = nullptr;
@@ -98,6 +111,24 @@ cudaError_t launch_powersgd(acc_ctx* ctx, const float* grads, float* err, float*
                             const uint8_t* level, float* out, float* delta, cudaStream_t s);
 cudaError_t launch_topk(acc_ctx* ctx, const float* grads, float* err, const uint8_t* level, float* vals,
                         int32_t* idx, int32_t* counts, float* out, float* delta, cudaStream_t s);
+
+// Brackets one kernel launch with CUDA events on its stream when profiling is on; counts the launch.
+struct PhaseTimer {
+  acc_ctx* ctx; cudaStream_t s; ProfSlot* slot = nullptr;
+  PhaseTimer(acc_ctx* c, int phase, cudaStream_t st) : ctx(c), s(st) {
+    ctx->last_launches += 1;
+    if (!ctx->prof) return;
+    if (ctx->prof_used == ctx->prof_slots.size()) {
+      ProfSlot n{phase, nullptr, nullptr};
+      if (cudaEventCreate(&n.a) != cudaSuccess || cudaEventCreate(&n.b) != cudaSuccess) return;
+      ctx->prof_slots.push_back(n);
+    }
+    slot = &ctx->prof_slots[ctx->prof_used++];
+    slot->phase = phase;
+    cudaEventRecord(slot->a, s);
+  }
+  ~PhaseTimer() { if (slot) cudaEventRecord(slot->b, s); }
+};
 
 // ---- small device helpers -------------------------------------------------------------------------
 __device__ __forceinline__ float4 ld_stream4(const float* p) { return __ldcs(reinterpret_cast<const float4*>(p)); }

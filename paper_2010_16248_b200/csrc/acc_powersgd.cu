@@ -309,24 +309,34 @@ cudaError_t launch_powersgd(acc_ctx* ctx, const float* grads, float* err, float*
   const int n_vec = (int)pl.vec_tiles.size();
   const float inv_w = 1.0f / (float)c.n_workers;
   if (n_items + n_vec > 0) {
+    PhaseTimer pt(ctx, PH_PSGD_PROJECT, s);
     psgd_project_kernel<4><<<n_items + n_vec, 256, 0, s>>>(
         ctx->d_layers, ctx->d_row_items, n_items, ctx->d_tiles, ctx->d_vec_tiles, grads, err, q, p_hat, level, out,
         delta, c.worker_stride, c.n_workers, c.decider, inv_w, c.rank_low, c.rank_high);
-    ctx->last_launches += 1;
   }
   if (pl.n_mat > 0) {
-    psgd_orthonormalise_kernel<<<pl.n_mat, 1024, 0, s>>>(ctx->d_layers, ctx->d_mat_layers, p_hat, level, c.rank_low,
-                                                        c.rank_high, c.gs_eps);
-    psgd_qpartial_kernel<<<(unsigned)pl.col_items.size(), kColBlockThreads, 0, s>>>(ctx->d_layers, ctx->d_col_items,
-                                                                                    out, p_hat, ctx->d_part);
+    {
+      PhaseTimer pt(ctx, PH_PSGD_ORTHO, s);
+      psgd_orthonormalise_kernel<<<pl.n_mat, 1024, 0, s>>>(ctx->d_layers, ctx->d_mat_layers, p_hat, level,
+                                                          c.rank_low, c.rank_high, c.gs_eps);
+    }
+    {
+      PhaseTimer pt(ctx, PH_PSGD_QPARTIAL, s);
+      psgd_qpartial_kernel<<<(unsigned)pl.col_items.size(), kColBlockThreads, 0, s>>>(
+          ctx->d_layers, ctx->d_col_items, out, p_hat, ctx->d_part);
+    }
     int max_cols = 0;
     for (int l : pl.mat_layers) max_cols = max_cols > pl.layers[l].cols ? max_cols : pl.layers[l].cols;
-    psgd_qreduce_kernel<<<dim3((max_cols + 31) / 32, pl.n_mat), 256, 0, s>>>(ctx->d_layers, ctx->d_mat_layers,
-                                                                            ctx->d_part, q, level, c.rank_low,
-                                                                            c.rank_high);
-    psgd_residual_kernel<4><<<n_items, 256, 0, s>>>(ctx->d_layers, ctx->d_row_items, err, q, p_hat, level, out,
-                                                    c.worker_stride, c.n_workers, c.rank_low, c.rank_high);
-    ctx->last_launches += 4;
+    {
+      PhaseTimer pt(ctx, PH_PSGD_QREDUCE, s);
+      psgd_qreduce_kernel<<<dim3((max_cols + 31) / 32, pl.n_mat), 256, 0, s>>>(
+          ctx->d_layers, ctx->d_mat_layers, ctx->d_part, q, level, c.rank_low, c.rank_high);
+    }
+    {
+      PhaseTimer pt(ctx, PH_PSGD_RESIDUAL, s);
+      psgd_residual_kernel<4><<<n_items, 256, 0, s>>>(ctx->d_layers, ctx->d_row_items, err, q, p_hat, level, out,
+                                                      c.worker_stride, c.n_workers, c.rank_low, c.rank_high);
+    }
   }
   return cudaGetLastError();
 }

@@ -450,23 +450,43 @@ cudaError_t launch_topk(acc_ctx* ctx, const float* grads, float* err, const uint
   if (n_mat > 0) {
     const long long V = (long long)W * nt;
     const int grid = (int)(V < (long long)ctx->sm_count * 8 ? V : (long long)ctx->sm_count * 8);
-    topk_ef_hist1_kernel<<<grid, 256, 0, s>>>(ctx->d_layers, ctx->d_tiles, nt, n_mat, grads, err, delta,
-                                              c.worker_stride, W, c.decider, ctx->d_hist1);
-    topk_pick1_kernel<<<W * n_mat, 256, 0, s>>>(ctx->d_layers, ctx->d_mat_layers, n_mat, c.n_layers, level,
-                                                ctx->d_hist1, ctx->d_sel, counts);
-    topk_hist2_kernel<<<grid, 256, 0, s>>>(ctx->d_layers, ctx->d_tiles, nt, n_mat, err, c.worker_stride, W,
-                                           ctx->d_sel, ctx->d_hist2, ctx->d_tile_cnt);
-    topk_pick2_kernel<<<W * n_mat, 256, 0, s>>>(n_mat, ctx->d_hist2, ctx->d_sel);
-    topk_hist3_kernel<<<dim3(nt, W), 256, 0, s>>>(ctx->d_layers, ctx->d_tiles, nt, n_mat, err, c.worker_stride,
-                                                  ctx->d_sel, ctx->d_hist3, ctx->d_tile_cnt, ctx->d_tile_h3);
-    topk_pick3_scan_kernel<<<W * n_mat, 256, 0, s>>>(ctx->d_layers, ctx->d_mat_layers, n_mat, nt, ctx->d_hist3,
-                                                     ctx->d_sel, ctx->d_tile_cnt, ctx->d_tile_h3, ctx->d_tile_pre);
-    ctx->last_launches += 6;
+    {
+      PhaseTimer pt(ctx, PH_TOPK_EF_HIST1, s);
+      topk_ef_hist1_kernel<<<grid, 256, 0, s>>>(ctx->d_layers, ctx->d_tiles, nt, n_mat, grads, err, delta,
+                                                c.worker_stride, W, c.decider, ctx->d_hist1);
+    }
+    {
+      PhaseTimer pt(ctx, PH_TOPK_PICK1, s);
+      topk_pick1_kernel<<<W * n_mat, 256, 0, s>>>(ctx->d_layers, ctx->d_mat_layers, n_mat, c.n_layers, level,
+                                                  ctx->d_hist1, ctx->d_sel, counts);
+    }
+    {
+      PhaseTimer pt(ctx, PH_TOPK_HIST2, s);
+      topk_hist2_kernel<<<grid, 256, 0, s>>>(ctx->d_layers, ctx->d_tiles, nt, n_mat, err, c.worker_stride, W,
+                                             ctx->d_sel, ctx->d_hist2, ctx->d_tile_cnt);
+    }
+    {
+      PhaseTimer pt(ctx, PH_TOPK_PICK2, s);
+      topk_pick2_kernel<<<W * n_mat, 256, 0, s>>>(n_mat, ctx->d_hist2, ctx->d_sel);
+    }
+    {
+      PhaseTimer pt(ctx, PH_TOPK_HIST3, s);
+      topk_hist3_kernel<<<dim3(nt, W), 256, 0, s>>>(ctx->d_layers, ctx->d_tiles, nt, n_mat, err, c.worker_stride,
+                                                    ctx->d_sel, ctx->d_hist3, ctx->d_tile_cnt, ctx->d_tile_h3);
+    }
+    {
+      PhaseTimer pt(ctx, PH_TOPK_PICK3_SCAN, s);
+      topk_pick3_scan_kernel<<<W * n_mat, 256, 0, s>>>(ctx->d_layers, ctx->d_mat_layers, n_mat, nt, ctx->d_hist3,
+                                                       ctx->d_sel, ctx->d_tile_cnt, ctx->d_tile_h3,
+                                                       ctx->d_tile_pre);
+    }
   }
-  topk_select_kernel<<<nt, 256, 0, s>>>(ctx->d_layers, ctx->d_tiles, nt, n_mat, grads, err, ctx->d_sel,
-                                        ctx->d_tile_pre, vals, idx, out, delta, c.worker_stride, pl.capacity, W,
-                                        c.decider, inv_w);
-  ctx->last_launches += 1;
+  {
+    PhaseTimer pt(ctx, PH_TOPK_SELECT, s);
+    topk_select_kernel<<<nt, 256, 0, s>>>(ctx->d_layers, ctx->d_tiles, nt, n_mat, grads, err, ctx->d_sel,
+                                          ctx->d_tile_pre, vals, idx, out, delta, c.worker_stride, pl.capacity, W,
+                                          c.decider, inv_w);
+  }
   return cudaGetLastError();
 }
 

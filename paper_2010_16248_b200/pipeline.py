@@ -1,0 +1,72 @@
+"""Sequencing of the C-ABI calls for one training run: state buffers and the detection cadence.
+
+``AccordionStep`` owns the persistent state of the path (error memories, PowerSGD factors, the
+detector's accumulator and norms, the per-layer level array) as device tensors and issues, per
+iteration, the compressor step(s) and -- every ``check_every`` iterations -- the norm and regime
+kernels (Section 4.2: accumulate during the window, take norms at its end, Algorithm 1).  All
+arithmetic happens in the library's kernels; nothing here reads results back to the host.
+"""
+from __future__ import annotations
+
+from typing import Optional, Sequence
+
+import torch
+
+from . import binding
+from . import workloads as wl
+
+
+class AccordionStep:
+    def __init__(self, table: wl.LayerTable, n_workers: int, compressors: Sequence[str] = ("powersgd",),
+                 rank_low=2, rank_high=1, topk_low_bp=1000, topk_high_bp=100, eta=0.5, gs_eps=1e-8,
+                 check_every=10, decider=0, q_init=None, device="cuda"):
+        self.table, self.W = table, n_workers
+        self.compressors = tuple(compressors)
+        self.check_every = check_every
+        self.device = torch.device(device)
+        self.ctx = binding.Context(table, n_workers, device=device, rank_low=rank_low, rank_high=rank_high,
+                                   topk_low_bp=topk_low_bp, topk_high_bp=topk_high_bp, eta=eta, gs_eps=gs_eps,
+                                   decider=decider)
+        dev, L, stride = self.device, table.n_layers, table.stride
+        self.level = torch.ones(L, dtype=torch.uint8, device=dev)  # before the first check: low compression
+        self.delta = torch.zeros(stride, device=dev)
+        self.norm2_curr = torch.zeros(L, dtype=torch.float64, device=dev)
+        self.norm2_prev = torch.full((L,), -1.0, dtype=torch.float64, device=dev)
+        self.t = 0
+        self.launches = 0
+        if "powersgd" in self.compressors:
+            self.err_psgd = torch.zeros(n_workers, stride, device=dev)
+            self.q = self.ctx.new_q(q_init if q_init is not None else wl.initial_q(table, rank_low, device=dev))
+            self.p_hat = self.ctx.new_p()
+            self.out_psgd = torch.zeros(stride, device=dev)
+        if "topk" in self.compressors:
+            self.err_topk = torch.zeros(n_workers, stride, device=dev)
+            self.vals, self.idx, self.counts = self.ctx.new_topk_buffers()
+            self.out_topk = torch.zeros(stride, device=dev)
+
+    def step(self, grads: torch.Tensor, lr_curr: float = 0.1, lr_next: float = 0.1, stream=None):
+        """One iteration on device-resident gradients ``[W, stride]``."""
+        c = self.ctx
+        delta: Optional[torch.Tensor] = self.delta  # accumulated once per iteration, by the first compressor
+        if "powersgd" in self.compressors:
+            c.acc_powersgd_step(grads, self.err_psgd, self.q, self.p_hat, self.level, self.out_psgd, delta, stream)
+            self.launches += c.last_launch_count()
+            delta = None
+        if "topk" in self.compressors:
+            c.acc_topk_step(grads, self.err_topk, self.level, self.vals, self.idx, self.counts, self.out_topk,
+                            delta, stream)
+            self.launches += c.last_launch_count()
+        self.t += 1
+        if self.t % self.check_every == 0:
+            c.acc_layer_norms(self.delta, 1, self.norm2_curr, stream=stream)
+            self.launches += c.last_launch_count()
+            c.acc_detect_regime(self.norm2_curr, self.norm2_prev, lr_curr, lr_next, self.level, self.delta, stream)
+            self.launches += c.last_launch_count()
+
+    def outputs(self):
+        outs = []
+        if "powersgd" in self.compressors:
+            outs.append(self.out_psgd)
+        if "topk" in self.compressors:
+            outs.append(self.out_topk)
+        return outs
