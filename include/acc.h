@@ -43,6 +43,7 @@ extern "C" {
 #define ACC_EALIGN 2      /* a pointer, offset or stride is not 16-byte aligned    */
 #define ACC_EWORKSPACE 3  /* workspace missing or too small                        */
 #define ACC_ECUDA 4       /* a CUDA runtime call or kernel launch reported an error */
+#define ACC_ETOOBIG 5     /* size beyond the fixed capacity of acc_sumsq_static    */
 
 #define ACC_MATRIX 0
 #define ACC_VECTOR 1
@@ -155,6 +156,31 @@ int64_t acc_floats_sent(const acc_config* cfg, const uint8_t* level_host, int32_
 /* Number of kernels the last *_step / acc_error_feedback / acc_layer_norms / acc_detect_regime call
  * on this context launched (for launch accounting in benchmarks).                                  */
 int32_t acc_last_launch_count(const acc_ctx* ctx);
+
+/* Squared L2 norm of one flat fp32 buffer without any caller-provided scratch (the paper has no
+ * counterpart; the value is what acc_layer_norms returns for a single layer covering the buffer,
+ * e.g. the whole-model gradient norm).
+ *
+ * Who needs it: callers that cannot allocate device memory and have no workspace to pass -- code
+ * that runs inside another framework's fixed memory budget, a plugin that is only handed tensors,
+ * a loop that cannot afford the device-wide synchronisation an allocation implies.  Every other
+ * entry point needs the workspace given to acc_create; this one keeps its reduction scratch in a
+ * device array built into the library (256 KB on every GPU that loads the library, held until the
+ * process exits).  It performs no allocation of any kind.
+ *
+ *   *norm2 = sum_i buf[i]^2, i < n, accumulated in fp64 in a fixed order (bit-reproducible).
+ *
+ * Device pointers: buf [n] floats, 16-byte aligned (read); norm2: one double (written).
+ * Limits and rules:
+ *   - 1 <= n <= ACC_STATIC_NORM_MAX_ELEMS, otherwise ACC_ETOOBIG (nothing is launched).
+ *   - The first call on each device looks up the array's device address (once per device, with
+ *     that device current); make that first call outside any stream capture.
+ *   - All calls on a device share the one array, and it keeps the previous call's partial sums.
+ *     Nothing in it needs clearing (each call overwrites every slot it later reads), but two calls
+ *     that overlap on the GPU -- different streams, no ordering between them -- race on it and
+ *     return garbage: order them on one stream or with events.                                      */
+#define ACC_STATIC_NORM_MAX_ELEMS (1 << 28)
+int acc_sumsq_static(const float* buf, int64_t n, double* norm2, void* stream);
 
 /* Per-kernel timing aid (no counterpart in the paper).  While enabled, every kernel the library
  * launches on this context is bracketed by CUDA events on its stream.  acc_profile_read waits for the

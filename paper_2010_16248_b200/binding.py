@@ -42,7 +42,7 @@ class acc_config(C.Structure):
 EXPORTS = ["acc_workspace_bytes", "acc_create", "acc_destroy", "acc_factor_layout", "acc_topk_layout",
            "acc_error_feedback", "acc_layer_norms", "acc_detect_regime", "acc_powersgd_step", "acc_topk_step",
            "acc_floats_sent", "acc_last_launch_count", "acc_strerror", "acc_profile_enable", "acc_profile_read",
-           "acc_profile_kernel_count", "acc_profile_kernel_name"]
+           "acc_profile_kernel_count", "acc_profile_kernel_name", "acc_sumsq_static"]
 
 _lib = None
 
@@ -80,6 +80,7 @@ def lib() -> C.CDLL:
     L.acc_profile_kernel_count.restype = i32
     L.acc_profile_kernel_name.argtypes = [i32]
     L.acc_profile_kernel_name.restype = C.c_char_p
+    L.acc_sumsq_static.argtypes = [vp, i64, vp, vp]
     for name in EXPORTS:
         if name not in ("acc_floats_sent", "acc_last_launch_count", "acc_strerror", "acc_profile_kernel_count",
                         "acc_profile_kernel_name"):
@@ -105,6 +106,17 @@ def make_config(table, n_workers, rank_low=2, rank_high=1, topk_low_bp=1000, top
 def acc_floats_sent(cfg: acc_config, level, compressor: int) -> int:
     lv = (C.c_uint8 * cfg.n_layers)(*[int(x) for x in level])
     return int(lib().acc_floats_sent(C.byref(cfg), lv, compressor))
+
+
+def acc_sumsq_static(buf: torch.Tensor, n: int, norm2: torch.Tensor, stream=None) -> None:
+    """Squared L2 norm of the first ``n`` floats of ``buf`` into the one-element fp64 tensor ``norm2``.
+
+    For callers that cannot allocate device memory or supply a workspace: the reduction scratch is a
+    fixed array inside the library, so this call allocates nothing (neither do these few lines).
+    ``n`` is limited to 2**28 elements; calls that overlap on the GPU share the scratch and race."""
+    st = lib().acc_sumsq_static(_ptr(buf, torch.float32), int(n), _ptr(norm2, torch.float64), _stream(stream))
+    if st != ACC_OK:
+        raise AccError(st, "acc_sumsq_static")
 
 
 def _ptr(t: Optional[torch.Tensor], dtype=None) -> Optional[int]:

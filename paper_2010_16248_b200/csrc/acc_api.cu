@@ -323,6 +323,7 @@ const char* acc_strerror(int status) {
     case ACC_EALIGN: return "pointer, offset or stride not 16-byte aligned";
     case ACC_EWORKSPACE: return "workspace missing or too small";
     case ACC_ECUDA: return "CUDA runtime or launch error";
+    case ACC_ETOOBIG: return "size exceeds the capacity of the built-in scratch array (ACC_STATIC_NORM_MAX_ELEMS)";
     default: return "unknown status";
   }
 }
