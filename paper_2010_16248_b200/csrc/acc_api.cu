@@ -76,8 +76,7 @@ static int make_plan(const acc_config* cfg, Plan& p) {
     o.seg_off = p.capacity; p.capacity += o.k_low;
     // row slabs of the row-wise passes: about kRowSlabElems elements per worker, whole rows,
     // a multiple of 8 rows (one row per warp of a 256-thread block) where the layer allows it
-    int rs = std::max(1, kRowSlabElems / d.cols);
-    if (rs >= 8) rs = rs / 8 * 8;
+    int rs = std::max(8, kRowSlabElems / d.cols / 8 * 8);
     rs = std::min(rs, d.rows);
     for (int r0 = 0; r0 < d.rows; r0 += rs) p.row_items.push_back(RowItem{l, r0, std::min(rs, d.rows - r0)});
     // row slabs x column blocks of the Q-partial pass (each thread owns `vec` adjacent columns)
@@ -310,7 +309,7 @@ const char* acc_profile_kernel_name(int32_t i) {
       "psgd_project_kernel", "psgd_orthonormalise_kernel", "psgd_qpartial_kernel", "psgd_qreduce_kernel",
       "psgd_residual_kernel",
       "topk_ef_hist1_kernel", "topk_pick1_kernel", "topk_hist2_kernel", "topk_pick2_kernel", "topk_hist3_kernel",
-      "topk_pick3_scan_kernel", "topk_select_kernel"};
+      "topk_pick3_scan_kernel", "topk_select_kernel", "topk_decompress_kernel"};
   return (i >= 0 && i < PH_COUNT) ? names[i] : "";
 }
 

@@ -48,6 +48,7 @@ enum Phase {
   PH_EF = 0, PH_NORM_PARTIAL, PH_NORM_FINAL, PH_DETECT,
   PH_PSGD_PROJECT, PH_PSGD_ORTHO, PH_PSGD_QPARTIAL, PH_PSGD_QREDUCE, PH_PSGD_RESIDUAL,
   PH_TOPK_EF_HIST1, PH_TOPK_PICK1, PH_TOPK_HIST2, PH_TOPK_PICK2, PH_TOPK_HIST3, PH_TOPK_PICK3_SCAN, PH_TOPK_SELECT,
+  PH_TOPK_DECOMPRESS,
   PH_COUNT
 };
 

@@ -9,7 +9,8 @@
 //   hist3      per-tile level-3 histogram of the keys with prefix (b1,b2), per-tile count above [reads M]
 //   pick3scan  threshold tau, number of ties to keep, exclusive per-tile prefix of (above, ties)
 //   select     keep key > tau and the lowest-index `need` of key == tau; write (val, idx) in index
-//              order, zero the kept entries of err, accumulate out = mean_w kept                [reads M]
+//              order, zero the kept entries of err                                              [reads M]
+//   decompress out = (1/W) sum_w scatter(idx_w, val_w), accumulated per tile in shared memory [reads packed]
 // No floating-point atomics and no inter-block waiting: same input, same bits.
 #include "acc_internal.cuh"
 
@@ -266,8 +267,9 @@ topk_hist3_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict__ 
   }
 }
 
-// One block per (worker, MATRIX layer): final threshold and the exclusive prefix, over the layer's tiles
-// in index order, of (keys above tau, keys equal to tau).
+// One block per (worker, MATRIX layer): final threshold tau and number of ties to keep; then, per tile of
+// the layer, (keys above tau, keys equal to tau) from the per-tile counters, and their exclusive prefix in
+// index order.
 __global__ void __launch_bounds__(256)
 topk_pick3_scan_kernel(const DevLayer* __restrict__ layers, const int* __restrict__ mat_layers, int n_mat,
                        int n_tiles, const unsigned* __restrict__ hist3, Select* __restrict__ sel,
@@ -289,17 +291,32 @@ topk_pick3_scan_kernel(const DevLayer* __restrict__ layers, const int* __restric
   }
   __syncthreads();
   const unsigned b3 = b3s;
+  const long long tb = (long long)w * n_tiles + L.tile0;
+  // phase 1: one warp per tile turns the tile's level-3 histogram into (above, ties)
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  for (int t = warp; t < L.ntiles; t += 8) {
+    const unsigned short* h = tile_h3 + (tb + t) * kBins3;
+    int above = 0;
+#pragma unroll
+    for (int i = 0; i < kBins3 / 32; ++i) {
+      const unsigned b = i * 32 + lane;
+      const int c = h[b];
+      above += b > b3 ? c : 0;
+    }
+    above = __reduce_add_sync(0xffffffffu, above);
+    if (lane == 0) {
+      const int2 c = tile_cnt[tb + t];
+      tile_pre[tb + t] = make_int2(c.x + c.y + above, (int)h[b3]);
+    }
+  }
+  __syncthreads();
+  // phase 2: exclusive scan over the layer's tiles (each thread owns a contiguous chunk)
   const int per = (L.ntiles + 255) / 256;
   const int t0 = min(L.ntiles, (int)threadIdx.x * per), t1 = min(L.ntiles, t0 + per);
-  const long long tb = (long long)w * n_tiles + L.tile0;
   int2 sum = make_int2(0, 0);
   for (int t = t0; t < t1; ++t) {
-    const int2 c = tile_cnt[tb + t];
-    const unsigned short* h = tile_h3 + (tb + t) * kBins3;
-    int above = c.x + c.y;
-    for (unsigned b = b3 + 1; b < (unsigned)kBins3; ++b) above += h[b];
-    sum.x += above;
-    sum.y += h[b3];
+    const int2 c = tile_pre[tb + t];
+    sum.x += c.x; sum.y += c.y;
   }
   chunk_sum[threadIdx.x] = sum;
   __syncthreads();
@@ -314,127 +331,145 @@ topk_pick3_scan_kernel(const DevLayer* __restrict__ layers, const int* __restric
   __syncthreads();
   int2 run = chunk_sum[threadIdx.x];
   for (int t = t0; t < t1; ++t) {
-    const int2 c = tile_cnt[tb + t];
-    const unsigned short* h = tile_h3 + (tb + t) * kBins3;
-    int above = c.x + c.y;
-    for (unsigned b = b3 + 1; b < (unsigned)kBins3; ++b) above += h[b];
+    const int2 c = tile_pre[tb + t];
     tile_pre[tb + t] = run;
-    run.x += above;
-    run.y += h[b3];
+    run.x += c.x; run.y += c.y;
   }
 }
 
-// Pass E.  One block per tile, all workers in order.  Warp `wi` owns float4s [wi*256, wi*256+256) of the
-// tile; lane handles float4 j*32+lane of that range for j = 0..7, so (j, lane, element) is index order.
-__global__ void __launch_bounds__(256)
+// Pass E.  One block per (tile, worker).  Warp `wi` owns float4s [wi*256, wi*256+256) of the tile; lane
+// handles float4 j*32+lane of that range for j = 0..7, so (j, lane, element) is index order.  Writes the
+// kept (value, index) pairs at their final positions and zeroes them in err.
+__global__ void __launch_bounds__(256, 3)
 topk_select_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict__ tiles, int n_tiles, int n_mat,
-                   const float* __restrict__ grads, float* __restrict__ err, const Select* __restrict__ sel,
-                   const int2* __restrict__ tile_pre, float* __restrict__ vals, int32_t* __restrict__ idx,
-                   float* __restrict__ out, float* __restrict__ delta, long long stride, long long capacity, int W,
-                   int decider, float inv_w) {
+                   float* __restrict__ err, const Select* __restrict__ sel, const int2* __restrict__ tile_pre,
+                   float* __restrict__ vals, int32_t* __restrict__ idx, long long stride, long long capacity) {
   __shared__ unsigned wtot[8];
-  const int ti = blockIdx.x;
+  const int ti = blockIdx.x, w = blockIdx.y;
   const Tile t = tiles[ti];
   const DevLayer L = layers[t.layer];
-  const long long base = L.offset + t.elem0;
-  if (L.kind != ACC_MATRIX) {  // VECTOR layer: plain mean, detector accumulation
-    for (int i = threadIdx.x; i < t.nelem; i += blockDim.x) {
-      float acc = 0.f;
-      for (int w = 0; w < W; ++w) {
-        const float g = grads[(long long)w * stride + base + i];
-        acc += g;
-        if (delta != nullptr && w == decider) delta[base + i] += g;
-      }
-      out[base + i] = acc * inv_w;
-    }
-    return;
-  }
+  if (L.kind != ACC_MATRIX) return;
   const int wi = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  float oacc[8][4];
-#pragma unroll
-  for (int j = 0; j < 8; ++j) oacc[j][0] = oacc[j][1] = oacc[j][2] = oacc[j][3] = 0.f;
-  for (int w = 0; w < W; ++w) {
-    const Select s = sel[w * n_mat + L.mat];
-    const int2 pre = tile_pre[(long long)w * n_tiles + ti];
-    float* m = err + (long long)w * stride + base;
-    float mv[8][4];
-    unsigned am[8], tm[8];  // 4-bit masks: key > tau, key == tau
-    unsigned incl[8];       // inclusive lane scan of (above | ties << 16) per j
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      const int e0 = 4 * (wi * 256 + j * 32 + lane);
-      if (e0 + 3 < t.nelem) {
-        const float4 v = *reinterpret_cast<const float4*>(m + e0);
-        mv[j][0] = v.x; mv[j][1] = v.y; mv[j][2] = v.z; mv[j][3] = v.w;
-      } else {
-#pragma unroll
-        for (int e = 0; e < 4; ++e) mv[j][e] = (e0 + e < t.nelem) ? m[e0 + e] : 0.f;
-      }
-    }
-    unsigned carry = 0;  // (above | ties << 16) of this warp's earlier j
-    unsigned base_j[8];
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      const int e0 = 4 * (wi * 256 + j * 32 + lane);
-      unsigned a = 0, tt = 0;
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const unsigned k = key_of(mv[j][e]);
-        const bool valid = e0 + e < t.nelem;
-        a |= (unsigned)(valid && k > s.tau) << e;
-        tt |= (unsigned)(valid && k == s.tau) << e;
-      }
-      am[j] = a; tm[j] = tt;
-      unsigned c = __popc(a) | (__popc(tt) << 16);
-#pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        const unsigned n = __shfl_up_sync(0xffffffffu, c, o);
-        if (lane >= o) c += n;
-      }
-      incl[j] = c;
-      base_j[j] = carry;
-      carry += __shfl_sync(0xffffffffu, c, 31);
-    }
-    __syncthreads();  // previous worker's readers of wtot are done
-    if (lane == 0) wtot[wi] = carry;
-    __syncthreads();
-    unsigned wbase = 0;
-    for (int i = 0; i < wi; ++i) wbase += wtot[i];
-    const long long seg = (long long)w * capacity + L.seg_off;
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      if ((am[j] | tm[j]) == 0) continue;
-      const int e0 = 4 * (wi * 256 + j * 32 + lane);
-      const unsigned excl = wbase + base_j[j] + incl[j] - (__popc(am[j]) | (__popc(tm[j]) << 16));
-      int above_before = pre.x + (int)(excl & 0xffffu);
-      int ties_before = pre.y + (int)(excl >> 16);
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const bool is_a = (am[j] >> e) & 1u, is_t = (tm[j] >> e) & 1u;
-        if (is_a || (is_t && ties_before < s.need)) {
-          const int pos = above_before + min(ties_before, s.need);
-          vals[seg + pos] = mv[j][e];
-          idx[seg + pos] = t.elem0 + e0 + e;
-          m[e0 + e] = 0.f;
-          oacc[j][e] += mv[j][e];
-        }
-        above_before += is_a;
-        ties_before += is_t;
-      }
-    }
-  }
+  const Select s = sel[w * n_mat + L.mat];
+  const int2 pre = tile_pre[(long long)w * n_tiles + ti];
+  float* m = err + (long long)w * stride + L.offset + t.elem0;
+  float4 mv[8];
 #pragma unroll
   for (int j = 0; j < 8; ++j) {
     const int e0 = 4 * (wi * 256 + j * 32 + lane);
     if (e0 + 3 < t.nelem) {
-      *reinterpret_cast<float4*>(out + base + e0) =
-          make_float4(oacc[j][0] * inv_w, oacc[j][1] * inv_w, oacc[j][2] * inv_w, oacc[j][3] * inv_w);
+      mv[j] = ld_stream4(m + e0);
     } else {
-#pragma unroll
-      for (int e = 0; e < 4; ++e)
-        if (e0 + e < t.nelem) out[base + e0 + e] = oacc[j][e] * inv_w;
+      mv[j].x = e0 < t.nelem ? m[e0] : 0.f;
+      mv[j].y = e0 + 1 < t.nelem ? m[e0 + 1] : 0.f;
+      mv[j].z = e0 + 2 < t.nelem ? m[e0 + 2] : 0.f;
+      mv[j].w = 0.f;
     }
   }
+  unsigned am = 0, tm = 0;  // 4 bits per j: key > tau, key == tau
+  unsigned excl[8];         // exclusive prefix inside the warp of (above | ties << 16), per j
+  unsigned carry = 0;
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    const int e0 = 4 * (wi * 256 + j * 32 + lane);
+    const float v[4] = {mv[j].x, mv[j].y, mv[j].z, mv[j].w};
+    unsigned a = 0, tt = 0;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const unsigned k = key_of(v[e]);
+      const bool valid = e0 + e < t.nelem;
+      a |= (unsigned)(valid && k > s.tau) << e;
+      tt |= (unsigned)(valid && k == s.tau) << e;
+    }
+    am |= a << (4 * j);
+    tm |= tt << (4 * j);
+    const unsigned own = __popc(a) | (__popc(tt) << 16);
+    unsigned c = own;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const unsigned n = __shfl_up_sync(0xffffffffu, c, o);
+      if (lane >= o) c += n;
+    }
+    excl[j] = carry + c - own;
+    carry += __shfl_sync(0xffffffffu, c, 31);
+  }
+  if (lane == 0) wtot[wi] = carry;
+  __syncthreads();
+  if ((am | tm) == 0) return;
+  unsigned wbase = 0;
+  for (int i = 0; i < wi; ++i) wbase += wtot[i];
+  const long long seg = (long long)w * capacity + L.seg_off;
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    const unsigned a = (am >> (4 * j)) & 15u, tt = (tm >> (4 * j)) & 15u;
+    if ((a | tt) == 0) continue;
+    const int e0 = 4 * (wi * 256 + j * 32 + lane);
+    const unsigned ex = wbase + excl[j];
+    int above_before = pre.x + (int)(ex & 0xffffu);
+    int ties_before = pre.y + (int)(ex >> 16);
+    const float v[4] = {mv[j].x, mv[j].y, mv[j].z, mv[j].w};
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const bool is_a = (a >> e) & 1u, is_t = (tt >> e) & 1u;
+      if (is_a || (is_t && ties_before < s.need)) {
+        const int pos = above_before + min(ties_before, s.need);
+        vals[seg + pos] = v[e];
+        idx[seg + pos] = t.elem0 + e0 + e;
+        m[e0 + e] = 0.f;
+      }
+      above_before += is_a;
+      ties_before += is_t;
+    }
+  }
+}
+
+// Pass F.  Scatter-decompress and average: one block per tile; the tile of `out` is accumulated in shared
+// memory from every worker's packed entries that fall into it, workers in order (fixed fp32 order), then
+// scaled by 1/W.  VECTOR tiles: out = mean_w g_w, delta += g_decider.
+__global__ void __launch_bounds__(256)
+topk_decompress_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict__ tiles, int n_tiles, int n_mat,
+                       const float* __restrict__ grads, const Select* __restrict__ sel,
+                       const int2* __restrict__ tile_pre, const float* __restrict__ vals,
+                       const int32_t* __restrict__ idx, float* __restrict__ out, float* __restrict__ delta,
+                       long long stride, long long capacity, int W, int decider, float inv_w) {
+  __shared__ float acc[kTile];
+  const int ti = blockIdx.x;
+  const Tile t = tiles[ti];
+  const DevLayer L = layers[t.layer];
+  const long long base = L.offset + t.elem0;
+  if (L.kind != ACC_MATRIX) {
+    for (int i = threadIdx.x; i < t.nelem; i += blockDim.x) {
+      float a = 0.f;
+      for (int w = 0; w < W; ++w) {
+        const float g = grads[(long long)w * stride + base + i];
+        a += g;
+        if (delta != nullptr && w == decider) delta[base + i] += g;
+      }
+      out[base + i] = a * inv_w;
+    }
+    return;
+  }
+  for (int i = threadIdx.x; i < kTile; i += blockDim.x) acc[i] = 0.f;
+  __syncthreads();
+  const bool last = ti == L.tile0 + L.ntiles - 1;
+  for (int w = 0; w < W; ++w) {
+    const Select s = sel[w * n_mat + L.mat];
+    const int2 p0 = tile_pre[(long long)w * n_tiles + ti];
+    const int start = p0.x + min(p0.y, s.need);
+    int end = s.k;
+    if (!last) {
+      const int2 p1 = tile_pre[(long long)w * n_tiles + ti + 1];
+      end = p1.x + min(p1.y, s.need);
+    }
+    const long long seg = (long long)w * capacity + L.seg_off;
+    for (int i = start + threadIdx.x; i < end; i += blockDim.x) acc[idx[seg + i] - t.elem0] += vals[seg + i];
+    __syncthreads();
+  }
+  const int n4 = t.nelem >> 2;
+  for (int i = threadIdx.x; i < n4; i += blockDim.x)
+    st_stream4(out + base + 4 * i, make_float4(acc[4 * i] * inv_w, acc[4 * i + 1] * inv_w, acc[4 * i + 2] * inv_w,
+                                               acc[4 * i + 3] * inv_w));
+  for (int i = 4 * n4 + threadIdx.x; i < t.nelem; i += blockDim.x) out[base + i] = acc[i] * inv_w;
 }
 
 cudaError_t launch_topk(acc_ctx* ctx, const float* grads, float* err, const uint8_t* level, float* vals,
@@ -481,11 +516,16 @@ cudaError_t launch_topk(acc_ctx* ctx, const float* grads, float* err, const uint
                                                        ctx->d_tile_pre);
     }
   }
-  {
+  if (n_mat > 0) {
     PhaseTimer pt(ctx, PH_TOPK_SELECT, s);
-    topk_select_kernel<<<nt, 256, 0, s>>>(ctx->d_layers, ctx->d_tiles, nt, n_mat, grads, err, ctx->d_sel,
-                                          ctx->d_tile_pre, vals, idx, out, delta, c.worker_stride, pl.capacity, W,
-                                          c.decider, inv_w);
+    topk_select_kernel<<<dim3(nt, W), 256, 0, s>>>(ctx->d_layers, ctx->d_tiles, nt, n_mat, err, ctx->d_sel,
+                                                   ctx->d_tile_pre, vals, idx, c.worker_stride, pl.capacity);
+  }
+  {
+    PhaseTimer pt(ctx, PH_TOPK_DECOMPRESS, s);
+    topk_decompress_kernel<<<nt, 256, 0, s>>>(ctx->d_layers, ctx->d_tiles, nt, n_mat, grads, ctx->d_sel,
+                                              ctx->d_tile_pre, vals, idx, out, delta, c.worker_stride, pl.capacity,
+                                              W, c.decider, inv_w);
   }
   return cudaGetLastError();
 }
