@@ -97,7 +97,7 @@ def _kernel_alg_bytes(name, units):
     (fp32): reads + writes that the method itself requires of that pass."""
     per_unit = {
         "psgd_project_kernel": 12.0,    # read g, read e, write M
-        "psgd_residual_kernel": 8.0,    # read M, write e'
+        "psgd_residual_kernel": 8.0,    # read M, write e' (eager mode; in lazy mode it only writes out)
         "topk_ef_hist1_kernel": 12.0,   # read g, read e, write M
         "topk_hist2_kernel": 4.0,       # read M
         "topk_hist3_kernel": 4.0,       # read M
@@ -193,6 +193,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=8)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--eager", action="store_true", help="PowerSGD: materialise the error memory every step")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -221,7 +222,7 @@ def main():
     # independent replicas: every rank draws its own gradient batches
     ring = [stream_gen.grads(1000 * rank + t) for t in range(RING)]
     eng = pipeline.AccordionStep(table, W, w.compressors, w.rank_low, w.rank_high, w.topk_low_bp, w.topk_high_bp,
-                                 w.eta, 1e-8, w.check_every, device=dev)
+                                 w.eta, 1e-8, w.check_every, device=dev, lazy_residual=not args.eager)
     n_mat = table.n_matrix_params
     grad_bytes_step = n_comp * 4.0 * W * table.n_params
 
@@ -340,6 +341,7 @@ def main():
                 "config": {"workload": w.name, "n_workers": W, "params": table.n_params,
                            "compressors": list(w.compressors), "rank_low_high": [w.rank_low, w.rank_high],
                            "topk_bp_low_high": [w.topk_low_bp, w.topk_high_bp], "check_every": w.check_every,
+                           "powersgd_residual": "eager" if args.eager else "lazy (applied on the next load)",
                            "gradient_bytes_per_step": grad_bytes_step,
                            "l2_policy": f"inputs larger than L2: {RING} gradient batches of "
                                         f"{4 * W * table.stride / 1e6:.0f} MB cycled, no flush",

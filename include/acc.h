@@ -49,6 +49,9 @@ extern "C" {
 #define ACC_VECTOR 1
 #define ACC_MAX_RANK 4    /* ranks are interleaved in groups of ACC_MAX_RANK floats  */
 
+/* acc_config.flags */
+#define ACC_FLAG_LAZY_RESIDUAL 1 /* PowerSGD keeps M_w in err and applies -A on the next load (see acc_powersgd_step) */
+
 #define ACC_COMPRESSOR_POWERSGD 0
 #define ACC_COMPRESSOR_TOPK 1
 
@@ -71,7 +74,7 @@ typedef struct {
   float eta;                    /* detection threshold of Algorithm 1 (the paper uses 0.5)       */
   float gs_eps;                 /* Gram-Schmidt divides by (norm + gs_eps)                       */
   int32_t decider;              /* worker whose raw gradient is accumulated for the detector     */
-  int32_t flags;                /* must be 0                                                     */
+  int32_t flags;                /* 0 or ACC_FLAG_LAZY_RESIDUAL                                   */
 } acc_config;
 
 typedef struct acc_ctx acc_ctx;
@@ -131,9 +134,21 @@ int acc_detect_regime(acc_ctx* ctx, const double* norm2_curr, double* norm2_prev
  * Columns r..3 of q and p_hat keep their previous contents.
  * Device pointers: grads [W][worker_stride] (read), err [W][worker_stride] (in/out),
  * q [4*q_rows] (in: warm start, out: new Q), p_hat [4*p_rows] (out: P^), level [L] bytes (read),
- * out [worker_stride] (written), delta [worker_stride] or NULL.                                    */
+ * out [worker_stride] (written), delta [worker_stride] or NULL.
+ *
+ * With ACC_FLAG_LAZY_RESIDUAL the subtraction e_w <- M_w - A is deferred: after the call err holds M_w,
+ * and the next acc_powersgd_step subtracts the A of this step (recomputed from p_hat and q, in the same
+ * fp32 operation order) while it loads err, so every later result is bit-identical to the eager mode's
+ * and one full read + write of err per step is saved.  Between steps the caller must leave err, q and
+ * p_hat untouched; acc_powersgd_flush materialises the error memory.                                 */
 int acc_powersgd_step(acc_ctx* ctx, const float* grads, float* err, float* q, float* p_hat,
                       const uint8_t* level, float* out, float* delta, void* stream);
+
+/* Lazy mode only (ACC_EINVAL otherwise): err_w <- err_w - P^ Q^T for the residual still pending from the
+ * last acc_powersgd_step, for every MATRIX layer and worker; afterwards err is the error memory e_w of
+ * the eager mode and nothing is pending.  A no-op per layer when nothing is pending.
+ * Device pointers: err [W][worker_stride] (in/out), q, p_hat (read).                                */
+int acc_powersgd_flush(acc_ctx* ctx, float* err, const float* q, const float* p_hat, void* stream);
 
 /* One TopK step with error feedback (the sparsifier of Section 5.3, per MATRIX layer and worker,
  * k = max(1, floor(rows*cols*K_bp/10000)), K_bp = topk_low_bp if level[l] else topk_high_bp):

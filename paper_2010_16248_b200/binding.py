@@ -18,6 +18,7 @@ from . import build as _build
 ACC_OK = 0
 ACC_MATRIX, ACC_VECTOR = 0, 1
 ACC_MAX_RANK = 4
+ACC_FLAG_LAZY_RESIDUAL = 1
 POWERSGD, TOPK = 0, 1
 
 
@@ -42,7 +43,7 @@ class acc_config(C.Structure):
 EXPORTS = ["acc_workspace_bytes", "acc_create", "acc_destroy", "acc_factor_layout", "acc_topk_layout",
            "acc_error_feedback", "acc_layer_norms", "acc_detect_regime", "acc_powersgd_step", "acc_topk_step",
            "acc_floats_sent", "acc_last_launch_count", "acc_strerror", "acc_profile_enable", "acc_profile_read",
-           "acc_profile_kernel_count", "acc_profile_kernel_name", "acc_sumsq_static"]
+           "acc_profile_kernel_count", "acc_profile_kernel_name", "acc_sumsq_static", "acc_powersgd_flush"]
 
 _lib = None
 
@@ -81,6 +82,7 @@ def lib() -> C.CDLL:
     L.acc_profile_kernel_name.argtypes = [i32]
     L.acc_profile_kernel_name.restype = C.c_char_p
     L.acc_sumsq_static.argtypes = [vp, i64, vp, vp]
+    L.acc_powersgd_flush.argtypes = [vp, vp, vp, vp, vp]
     for name in EXPORTS:
         if name not in ("acc_floats_sent", "acc_last_launch_count", "acc_strerror", "acc_profile_kernel_count",
                         "acc_profile_kernel_name"):
@@ -90,7 +92,7 @@ def lib() -> C.CDLL:
 
 
 def make_config(table, n_workers, rank_low=2, rank_high=1, topk_low_bp=1000, topk_high_bp=100, eta=0.5,
-                gs_eps=1e-8, decider=0, worker_stride=None):
+                gs_eps=1e-8, decider=0, worker_stride=None, flags=0):
     """Builds an ``acc_config`` (plus the array it points to) from a workloads.LayerTable."""
     L = table.n_layers
     arr = (acc_layer_desc * L)()
@@ -98,7 +100,7 @@ def make_config(table, n_workers, rank_low=2, rank_high=1, topk_low_bp=1000, top
         arr[l].offset = int(table.offset[l]); arr[l].rows = int(table.rows[l]); arr[l].cols = int(table.cols[l])
         arr[l].kind = int(table.kind[l]); arr[l].reserved = 0
     cfg = acc_config(n_workers, L, arr, int(worker_stride if worker_stride is not None else table.stride),
-                     rank_low, rank_high, topk_low_bp, topk_high_bp, eta, gs_eps, decider, 0)
+                     rank_low, rank_high, topk_low_bp, topk_high_bp, eta, gs_eps, decider, flags)
     cfg._keepalive = arr
     return cfg
 
@@ -203,6 +205,10 @@ class Context:
                                             _ptr(q, torch.float32), _ptr(p_hat, torch.float32),
                                             _ptr(level, torch.uint8), _ptr(out, torch.float32),
                                             _ptr(delta, torch.float32), _stream(stream)), "acc_powersgd_step")
+
+    def acc_powersgd_flush(self, err, q, p_hat, stream=None):
+        self._check(lib().acc_powersgd_flush(self._h, _ptr(err, torch.float32), _ptr(q, torch.float32),
+                                             _ptr(p_hat, torch.float32), _stream(stream)), "acc_powersgd_flush")
 
     def acc_topk_step(self, grads, err, level, vals, idx, counts, out, delta=None, stream=None):
         self._check(lib().acc_topk_step(self._h, _ptr(grads, torch.float32), _ptr(err, torch.float32),

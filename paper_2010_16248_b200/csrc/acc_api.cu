@@ -18,7 +18,7 @@ static int topk_count(long long size, int bp) {
 static int validate(const acc_config* cfg) {
   if (!cfg || !cfg->layers) return ACC_EINVAL;
   if (cfg->n_workers < 1 || cfg->n_workers > 1024 || cfg->n_layers < 1) return ACC_EINVAL;
-  if (cfg->flags != 0) return ACC_EINVAL;
+  if (cfg->flags & ~ACC_FLAG_LAZY_RESIDUAL) return ACC_EINVAL;
   if (cfg->rank_high < 1 || cfg->rank_low < cfg->rank_high || cfg->rank_low > ACC_MAX_RANK) return ACC_EINVAL;
   if (cfg->topk_high_bp < 1 || cfg->topk_low_bp < cfg->topk_high_bp || cfg->topk_low_bp > 10000) return ACC_EINVAL;
   if (!(cfg->eta >= 0.f) || !(cfg->gs_eps >= 0.f)) return ACC_EINVAL;
@@ -76,7 +76,14 @@ static int make_plan(const acc_config* cfg, Plan& p) {
     o.seg_off = p.capacity; p.capacity += o.k_low;
     // row slabs of the row-wise passes: about kRowSlabElems elements per worker, whole rows,
     // a multiple of 8 rows (one row per warp of a 256-thread block) where the layer allows it
-    int rs = std::max(8, kRowSlabElems / d.cols / 8 * 8);
+    // lanes per row: a full warp (512 contiguous bytes per access) unless the row is shorter than that;
+    // narrower groups on long rows scatter each access over several DRAM pages and measured slower
+    {
+      const int nf4 = std::max(1, d.cols / 4);
+      o.lpr = nf4 > 16 ? 32 : nf4 > 8 ? 16 : 8;
+    }
+    const int rows_per_pass = 8 * (32 / o.lpr);  // rows a 256-thread block has in flight
+    int rs = std::max(rows_per_pass, kRowSlabElems / d.cols / rows_per_pass * rows_per_pass);
     rs = std::min(rs, d.rows);
     for (int r0 = 0; r0 < d.rows; r0 += rs) p.row_items.push_back(RowItem{l, r0, std::min(rs, d.rows - r0)});
     // row slabs x column blocks of the Q-partial pass (each thread owns `vec` adjacent columns)
@@ -103,6 +110,7 @@ static int make_plan(const acc_config* cfg, Plan& p) {
   p.o_mat_layers = take(sizeof(int) * std::max<size_t>(1, p.mat_layers.size()));
   p.o_vec_tiles = take(sizeof(int) * std::max<size_t>(1, p.vec_tiles.size()));
   p.o_part = take(sizeof(float4) * std::max<long long>(1, p.part_f4));
+  p.o_pending = take(sizeof(int) * L);
   p.o_norm_part = take(sizeof(double) * (size_t)W * nt);
   p.o_hist = o;
   take(sizeof(unsigned) * seg * kBins1);
@@ -156,6 +164,7 @@ int acc_create(const acc_config* cfg, void* workspace, size_t workspace_bytes, a
   ctx->d_mat_layers = reinterpret_cast<int*>(ws + p.o_mat_layers);
   ctx->d_vec_tiles = reinterpret_cast<int*>(ws + p.o_vec_tiles);
   ctx->d_part = reinterpret_cast<float4*>(ws + p.o_part);
+  ctx->d_pending = reinterpret_cast<int*>(ws + p.o_pending);
   ctx->d_norm_part = reinterpret_cast<double*>(ws + p.o_norm_part);
   const size_t seg = (size_t)cfg->n_workers * std::max(p.n_mat, 1);
   ctx->d_hist1 = reinterpret_cast<unsigned*>(ws + p.o_hist);
@@ -176,6 +185,7 @@ int acc_create(const acc_config* cfg, void* workspace, size_t workspace_bytes, a
   up(ctx->d_tiles, p.tiles.data(), sizeof(Tile) * p.tiles.size());
   up(ctx->d_mat_layers, p.mat_layers.data(), sizeof(int) * p.mat_layers.size());
   up(ctx->d_vec_tiles, p.vec_tiles.data(), sizeof(int) * p.vec_tiles.size());
+  if (e == cudaSuccess) e = cudaMemset(ctx->d_pending, 0, sizeof(int) * cfg->n_layers);
   int dev = 0;
   if (e == cudaSuccess) e = cudaGetDevice(&dev);
   if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, dev);
@@ -252,6 +262,14 @@ int acc_powersgd_step(acc_ctx* ctx, const float* grads, float* err, float* q, fl
   return finish(launch_powersgd(ctx, grads, err, q, p_hat, level, out, delta, static_cast<cudaStream_t>(stream)));
 }
 
+int acc_powersgd_flush(acc_ctx* ctx, float* err, const float* q, const float* p_hat, void* stream) {
+  if (!ctx || !err || !q || !p_hat) return ACC_EINVAL;
+  if (!(ctx->cfg.flags & ACC_FLAG_LAZY_RESIDUAL)) return ACC_EINVAL;
+  if (!aligned16(err) || !aligned16(q) || !aligned16(p_hat)) return ACC_EALIGN;
+  ctx->last_launches = 0;
+  return finish(launch_powersgd_flush(ctx, err, q, p_hat, static_cast<cudaStream_t>(stream)));
+}
+
 int acc_topk_step(acc_ctx* ctx, const float* grads, float* err, const uint8_t* level, float* vals, int32_t* idx,
                   int32_t* counts, float* out, float* delta, void* stream) {
   if (!ctx || !grads || !err || !level || !vals || !idx || !counts || !out) return ACC_EINVAL;
@@ -309,7 +327,7 @@ const char* acc_profile_kernel_name(int32_t i) {
       "psgd_project_kernel", "psgd_orthonormalise_kernel", "psgd_qpartial_kernel", "psgd_qreduce_kernel",
       "psgd_residual_kernel",
       "topk_ef_hist1_kernel", "topk_pick1_kernel", "topk_hist2_kernel", "topk_pick2_kernel", "topk_hist3_kernel",
-      "topk_pick3_scan_kernel", "topk_select_kernel", "topk_decompress_kernel"};
+      "topk_pick3_scan_kernel", "topk_select_kernel", "topk_decompress_kernel", "psgd_flush_kernel"};
   return (i >= 0 && i < PH_COUNT) ? names[i] : "";
 }
 

@@ -23,6 +23,7 @@ struct DevLayer {
   int rows, cols, kind;
   int q_row, p_row;   // first row of the layer's block in q / p_hat (MATRIX), else -1
   int vec;            // widest vector width (4, 2, 1) at which every row start is aligned
+  int lpr;            // lanes per row (8, 16 or 32) of the row-wise kernels
   int mat;            // index among MATRIX layers, else -1
   int tile0, ntiles;  // flat tiles of this layer: [tile0, tile0 + ntiles)
   int k_low, k_high;  // TopK counts
@@ -48,7 +49,7 @@ enum Phase {
   PH_EF = 0, PH_NORM_PARTIAL, PH_NORM_FINAL, PH_DETECT,
   PH_PSGD_PROJECT, PH_PSGD_ORTHO, PH_PSGD_QPARTIAL, PH_PSGD_QREDUCE, PH_PSGD_RESIDUAL,
   PH_TOPK_EF_HIST1, PH_TOPK_PICK1, PH_TOPK_HIST2, PH_TOPK_PICK2, PH_TOPK_HIST3, PH_TOPK_PICK3_SCAN, PH_TOPK_SELECT,
-  PH_TOPK_DECOMPRESS,
+  PH_TOPK_DECOMPRESS, PH_PSGD_FLUSH,
   PH_COUNT
 };
 
@@ -65,7 +66,7 @@ struct Plan {
   int n_mat = 0;
   // workspace offsets (bytes)
   size_t o_layers = 0, o_row_items = 0, o_col_items = 0, o_tiles = 0, o_mat_layers = 0, o_vec_tiles = 0,
-         o_part = 0, o_norm_part = 0, o_hist = 0, o_sel = 0, o_tile_cnt = 0, o_tile_h3 = 0, o_tile_pre = 0,
+         o_part = 0, o_pending = 0, o_norm_part = 0, o_hist = 0, o_sel = 0, o_tile_cnt = 0, o_tile_h3 = 0, o_tile_pre = 0,
          hist_bytes = 0, total = 0;
 };
 
@@ -89,6 +90,7 @@ struct acc_ctx {
   int* d_mat_layers = nullptr;
   int* d_vec_tiles = nullptr;
   float4* d_part = nullptr;
+  int* d_pending = nullptr;          // lazy PowerSGD: rank of the residual not yet applied to err, per layer
   double* d_norm_part = nullptr;
   unsigned* d_hist1 = nullptr;
   unsigned* d_hist2 = nullptr;
@@ -110,6 +112,7 @@ cudaError_t launch_detect(acc_ctx* ctx, const double* n2c, double* n2p, float lr
                           uint8_t* level, cudaStream_t s);
 cudaError_t launch_powersgd(acc_ctx* ctx, const float* grads, float* err, float* q, float* p_hat,
                             const uint8_t* level, float* out, float* delta, cudaStream_t s);
+cudaError_t launch_powersgd_flush(acc_ctx* ctx, float* err, const float* q, const float* p_hat, cudaStream_t s);
 cudaError_t launch_topk(acc_ctx* ctx, const float* grads, float* err, const uint8_t* level, float* vals,
                         int32_t* idx, int32_t* counts, float* out, float* delta, cudaStream_t s);
 

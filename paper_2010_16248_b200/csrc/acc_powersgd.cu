@@ -40,17 +40,34 @@ __device__ void vector_mean_tile(const Tile& t, const DevLayer& L, const float* 
   }
 }
 
-// Pass 1.  One block per row slab (one warp per row), all workers:
+__device__ __forceinline__ float lowrank_entry(const float4& pv, const float4& qv, int r) {
+  float a = pv.x * qv.x;
+  if (r > 1) a = fmaf(pv.y, qv.y, a);
+  if (r > 2) a = fmaf(pv.z, qv.z, a);
+  if (r > 3) a = fmaf(pv.w, qv.w, a);
+  return a;
+}
+
+// Sum over the `lpr` consecutive lanes of a row group (lpr = 8, 16 or 32); every lane of the warp calls it.
+__device__ __forceinline__ float group_sum(float v, int lpr) {
+  for (int o = lpr >> 1; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+// Pass 1.  One block per row slab, all workers.  A group of `lpr` lanes owns a row (8*32/lpr rows in
+// flight per block):
+//   e_w = err_w                               (eager: err holds the error memory)
+//   e_w = err_w - P^_prev Q^T  (first rp ranks) (lazy: err holds last step's M_w, residual still pending)
 //   M_w = g_w + e_w -> err;  Mbar = mean_w M_w -> out;  P[row, :] = Mbar[row, :] . Q   (first r ranks);
 //   delta += g_decider.  Blocks beyond the row items handle the VECTOR tiles.
-template <int WB>
-__global__ void __launch_bounds__(256)
+template <int WB, bool LAZY>
+__global__ void __launch_bounds__(256, 3)
 psgd_project_kernel(const DevLayer* __restrict__ layers, const RowItem* __restrict__ items, int n_items,
                     const Tile* __restrict__ tiles, const int* __restrict__ vec_tiles,
                     const float* __restrict__ grads, float* __restrict__ err, const float* __restrict__ q,
-                    float* __restrict__ p, const uint8_t* __restrict__ level, float* __restrict__ out,
-                    float* __restrict__ delta, long long stride, int W, int decider, float inv_w, int rank_low,
-                    int rank_high) {
+                    float* __restrict__ p, const uint8_t* __restrict__ level, const int* __restrict__ pending,
+                    float* __restrict__ out, float* __restrict__ delta, long long stride, int W, int decider,
+                    float inv_w, int rank_low, int rank_high) {
   if ((int)blockIdx.x >= n_items) {
     const Tile t = tiles[vec_tiles[blockIdx.x - n_items]];
     vector_mean_tile(t, layers[t.layer], grads, out, delta, stride, W, decider, inv_w);
@@ -59,63 +76,84 @@ psgd_project_kernel(const DevLayer* __restrict__ layers, const RowItem* __restri
   const RowItem it = items[blockIdx.x];
   const DevLayer L = layers[it.layer];
   const int r = level[it.layer] ? rank_low : rank_high;
+  const int rp = LAZY ? pending[it.layer] : 0;
   const float4* __restrict__ Q4 = reinterpret_cast<const float4*>(q) + L.q_row;
   float4* __restrict__ P4 = reinterpret_cast<float4*>(p) + L.p_row;
+  const int lpr = L.lpr, groups = 32 / lpr;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  for (int row = it.row0 + warp; row < it.row0 + it.nrows; row += 8) {
-    const RowGeom rg = row_geom(L, row);
+  const int g = lane / lpr, gl = lane - g * lpr;
+  const int row_end = it.row0 + it.nrows;
+  for (int r0 = it.row0 + warp * groups; r0 < row_end; r0 += 8 * groups) {
+    const int row = r0 + g;
+    const bool valid = row < row_end;
     float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
-    for (int t = lane; t < rg.nbody4; t += 32) {
-      const int col = rg.head + 4 * t;
-      const long long idx = rg.start + col;
-      float4 mb = make_float4(0.f, 0.f, 0.f, 0.f);
-      for (int w0 = 0; w0 < W; w0 += WB) {
-        float4 g[WB], e[WB];
+    if (valid) {
+      const RowGeom rg = row_geom(L, row);
+      float4 pp = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (LAZY && rp > 0) pp = P4[row];
+      for (int t = gl; t < rg.nbody4; t += lpr) {
+        const int col = rg.head + 4 * t;
+        const long long idx = rg.start + col;
+        const float4 q0 = __ldg(Q4 + col), q1 = __ldg(Q4 + col + 1), q2 = __ldg(Q4 + col + 2), q3 = __ldg(Q4 + col + 3);
+        float4 corr = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (LAZY && rp > 0) {
+          corr.x = lowrank_entry(pp, q0, rp); corr.y = lowrank_entry(pp, q1, rp);
+          corr.z = lowrank_entry(pp, q2, rp); corr.w = lowrank_entry(pp, q3, rp);
+        }
+        float4 mb = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int w0 = 0; w0 < W; w0 += WB) {
+          float4 gv[WB], ev[WB];
 #pragma unroll
-        for (int b = 0; b < WB; ++b)
-          if (w0 + b < W) {
-            g[b] = ld_stream4(grads + (long long)(w0 + b) * stride + idx);
-            e[b] = ld_stream4(err + (long long)(w0 + b) * stride + idx);
-          }
-#pragma unroll
-        for (int b = 0; b < WB; ++b)
-          if (w0 + b < W) {
-            const float4 m = make_float4(g[b].x + e[b].x, g[b].y + e[b].y, g[b].z + e[b].z, g[b].w + e[b].w);
-            *reinterpret_cast<float4*>(err + (long long)(w0 + b) * stride + idx) = m;
-            mb.x += m.x; mb.y += m.y; mb.z += m.z; mb.w += m.w;
-            if (delta != nullptr && w0 + b == decider) {
-              float4 d = *reinterpret_cast<const float4*>(delta + idx);
-              d.x += g[b].x; d.y += g[b].y; d.z += g[b].z; d.w += g[b].w;
-              *reinterpret_cast<float4*>(delta + idx) = d;
+          for (int b = 0; b < WB; ++b)
+            if (w0 + b < W) {
+              gv[b] = ld_stream4(grads + (long long)(w0 + b) * stride + idx);
+              ev[b] = ld_stream4(err + (long long)(w0 + b) * stride + idx);
             }
-          }
+#pragma unroll
+          for (int b = 0; b < WB; ++b)
+            if (w0 + b < W) {
+              float4 e = ev[b];
+              if (LAZY && rp > 0) { e.x -= corr.x; e.y -= corr.y; e.z -= corr.z; e.w -= corr.w; }
+              const float4 m = make_float4(gv[b].x + e.x, gv[b].y + e.y, gv[b].z + e.z, gv[b].w + e.w);
+              if (LAZY) st_stream4(err + (long long)(w0 + b) * stride + idx, m);
+              else *reinterpret_cast<float4*>(err + (long long)(w0 + b) * stride + idx) = m;
+              mb.x += m.x; mb.y += m.y; mb.z += m.z; mb.w += m.w;
+              if (delta != nullptr && w0 + b == decider) {
+                float4 d = *reinterpret_cast<const float4*>(delta + idx);
+                d.x += gv[b].x; d.y += gv[b].y; d.z += gv[b].z; d.w += gv[b].w;
+                *reinterpret_cast<float4*>(delta + idx) = d;
+              }
+            }
+        }
+        mb.x *= inv_w; mb.y *= inv_w; mb.z *= inv_w; mb.w *= inv_w;
+        *reinterpret_cast<float4*>(out + idx) = mb;
+        a0 = fmaf(mb.x, q0.x, a0); a1 = fmaf(mb.x, q0.y, a1); a2 = fmaf(mb.x, q0.z, a2); a3 = fmaf(mb.x, q0.w, a3);
+        a0 = fmaf(mb.y, q1.x, a0); a1 = fmaf(mb.y, q1.y, a1); a2 = fmaf(mb.y, q1.z, a2); a3 = fmaf(mb.y, q1.w, a3);
+        a0 = fmaf(mb.z, q2.x, a0); a1 = fmaf(mb.z, q2.y, a1); a2 = fmaf(mb.z, q2.z, a2); a3 = fmaf(mb.z, q2.w, a3);
+        a0 = fmaf(mb.w, q3.x, a0); a1 = fmaf(mb.w, q3.y, a1); a2 = fmaf(mb.w, q3.z, a2); a3 = fmaf(mb.w, q3.w, a3);
       }
-      mb.x *= inv_w; mb.y *= inv_w; mb.z *= inv_w; mb.w *= inv_w;
-      *reinterpret_cast<float4*>(out + idx) = mb;
-      const float4 q0 = __ldg(Q4 + col), q1 = __ldg(Q4 + col + 1), q2 = __ldg(Q4 + col + 2), q3 = __ldg(Q4 + col + 3);
-      a0 = fmaf(mb.x, q0.x, a0); a1 = fmaf(mb.x, q0.y, a1); a2 = fmaf(mb.x, q0.z, a2); a3 = fmaf(mb.x, q0.w, a3);
-      a0 = fmaf(mb.y, q1.x, a0); a1 = fmaf(mb.y, q1.y, a1); a2 = fmaf(mb.y, q1.z, a2); a3 = fmaf(mb.y, q1.w, a3);
-      a0 = fmaf(mb.z, q2.x, a0); a1 = fmaf(mb.z, q2.y, a1); a2 = fmaf(mb.z, q2.z, a2); a3 = fmaf(mb.z, q2.w, a3);
-      a0 = fmaf(mb.w, q3.x, a0); a1 = fmaf(mb.w, q3.y, a1); a2 = fmaf(mb.w, q3.z, a2); a3 = fmaf(mb.w, q3.w, a3);
-    }
-    if (lane < rg.head + rg.tail) {  // the unaligned ends of the row, one element per lane
-      const int col = lane < rg.head ? lane : rg.head + 4 * rg.nbody4 + (lane - rg.head);
-      const long long idx = rg.start + col;
-      float mb = 0.f;
-      for (int w = 0; w < W; ++w) {
-        const float g = grads[(long long)w * stride + idx];
-        const float m = g + err[(long long)w * stride + idx];
-        err[(long long)w * stride + idx] = m;
-        mb += m;
-        if (delta != nullptr && w == decider) delta[idx] += g;
+      if (gl < rg.head + rg.tail) {  // the unaligned ends of the row, one element per lane
+        const int col = gl < rg.head ? gl : rg.head + 4 * rg.nbody4 + (gl - rg.head);
+        const long long idx = rg.start + col;
+        const float4 q0 = __ldg(Q4 + col);
+        const float corr = (LAZY && rp > 0) ? lowrank_entry(pp, q0, rp) : 0.f;
+        float mb = 0.f;
+        for (int w = 0; w < W; ++w) {
+          const float gv = grads[(long long)w * stride + idx];
+          float e = err[(long long)w * stride + idx];
+          if (LAZY && rp > 0) e -= corr;
+          const float m = gv + e;
+          err[(long long)w * stride + idx] = m;
+          mb += m;
+          if (delta != nullptr && w == decider) delta[idx] += gv;
+        }
+        mb *= inv_w;
+        out[idx] = mb;
+        a0 = fmaf(mb, q0.x, a0); a1 = fmaf(mb, q0.y, a1); a2 = fmaf(mb, q0.z, a2); a3 = fmaf(mb, q0.w, a3);
       }
-      mb *= inv_w;
-      out[idx] = mb;
-      const float4 q0 = __ldg(Q4 + col);
-      a0 = fmaf(mb, q0.x, a0); a1 = fmaf(mb, q0.y, a1); a2 = fmaf(mb, q0.z, a2); a3 = fmaf(mb, q0.w, a3);
     }
-    a0 = warp_sum(a0); a1 = warp_sum(a1); a2 = warp_sum(a2); a3 = warp_sum(a3);
-    if (lane == 0) {
+    a0 = group_sum(a0, lpr); a1 = group_sum(a1, lpr); a2 = group_sum(a2, lpr); a3 = group_sum(a3, lpr);
+    if (valid && gl == 0) {
       float4 pv = P4[row];
       pv.x = a0;
       if (r > 1) pv.y = a1;
@@ -141,12 +179,13 @@ __device__ __forceinline__ double block_sum(double v, double* sm) {
 // Pass 2.  One block per MATRIX layer: modified Gram-Schmidt on the first r columns of P, in place.
 __global__ void __launch_bounds__(1024)
 psgd_orthonormalise_kernel(const DevLayer* __restrict__ layers, const int* __restrict__ mat_layers,
-                           float* __restrict__ p, const uint8_t* __restrict__ level, int rank_low, int rank_high,
-                           float eps) {
+                           float* __restrict__ p, const uint8_t* __restrict__ level, int* __restrict__ pending,
+                           int rank_low, int rank_high, float eps) {
   __shared__ double sm[32];
   const int l = mat_layers[blockIdx.x];
   const DevLayer L = layers[l];
   const int r = level[l] ? rank_low : rank_high;
+  if (pending != nullptr && threadIdx.x == 0) pending[l] = r;  // lazy mode: this step's residual stays pending
   float* P = p + 4ll * L.p_row;
   const int n = L.rows;
   for (int c = 0; c < r; ++c) {
@@ -246,31 +285,29 @@ psgd_qreduce_kernel(const DevLayer* __restrict__ layers, const int* __restrict__
   }
 }
 
-__device__ __forceinline__ float lowrank_entry(const float4& pv, const float4& qv, int r) {
-  float a = pv.x * qv.x;
-  if (r > 1) a = fmaf(pv.y, qv.y, a);
-  if (r > 2) a = fmaf(pv.z, qv.z, a);
-  if (r > 3) a = fmaf(pv.w, qv.w, a);
-  return a;
-}
-
-// Pass 5.  One block per row slab (one warp per row): A = P^ Q'^T -> out;  e_w = M_w - A -> err.
-template <int WB>
+// Pass 5.  One block per row slab, a group of `lpr` lanes per row:  A = P^ Q'^T (first r ranks);
+//   WRITE_OUT: out = A;   UPDATE_ERR: err_w -= A for every worker.
+// Eager step: both (r from the level).  Lazy step: WRITE_OUT only.  Flush: UPDATE_ERR only, r = pending rank.
+template <int WB, bool WRITE_OUT, bool UPDATE_ERR>
 __global__ void __launch_bounds__(256)
 psgd_residual_kernel(const DevLayer* __restrict__ layers, const RowItem* __restrict__ items,
                      float* __restrict__ err, const float* __restrict__ q, const float* __restrict__ p,
-                     const uint8_t* __restrict__ level, float* __restrict__ out, long long stride, int W,
-                     int rank_low, int rank_high) {
+                     const uint8_t* __restrict__ level, const int* __restrict__ pending, float* __restrict__ out,
+                     long long stride, int W, int rank_low, int rank_high) {
   const RowItem it = items[blockIdx.x];
   const DevLayer L = layers[it.layer];
-  const int r = level[it.layer] ? rank_low : rank_high;
+  const int r = pending != nullptr ? pending[it.layer] : (level[it.layer] ? rank_low : rank_high);
+  if (r == 0) return;
   const float4* __restrict__ Q4 = reinterpret_cast<const float4*>(q) + L.q_row;
   const float4* __restrict__ P4 = reinterpret_cast<const float4*>(p) + L.p_row;
+  const int lpr = L.lpr, groups = 32 / lpr;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  for (int row = it.row0 + warp; row < it.row0 + it.nrows; row += 8) {
+  const int g = lane / lpr, gl = lane - g * lpr;
+  const int row_end = it.row0 + it.nrows;
+  for (int row = it.row0 + warp * groups + g; row < row_end; row += 8 * groups) {
     const RowGeom rg = row_geom(L, row);
     const float4 pv = __ldg(P4 + row);
-    for (int t = lane; t < rg.nbody4; t += 32) {
+    for (int t = gl; t < rg.nbody4; t += lpr) {
       const int col = rg.head + 4 * t;
       const long long idx = rg.start + col;
       float4 a;
@@ -278,27 +315,36 @@ psgd_residual_kernel(const DevLayer* __restrict__ layers, const RowItem* __restr
       a.y = lowrank_entry(pv, __ldg(Q4 + col + 1), r);
       a.z = lowrank_entry(pv, __ldg(Q4 + col + 2), r);
       a.w = lowrank_entry(pv, __ldg(Q4 + col + 3), r);
-      for (int w0 = 0; w0 < W; w0 += WB) {
-        float4 m[WB];
+      if (UPDATE_ERR) {
+        for (int w0 = 0; w0 < W; w0 += WB) {
+          float4 m[WB];
 #pragma unroll
-        for (int b = 0; b < WB; ++b)
-          if (w0 + b < W) m[b] = ld_stream4(err + (long long)(w0 + b) * stride + idx);
+          for (int b = 0; b < WB; ++b)
+            if (w0 + b < W) m[b] = ld_stream4(err + (long long)(w0 + b) * stride + idx);
 #pragma unroll
-        for (int b = 0; b < WB; ++b)
-          if (w0 + b < W)
-            st_stream4(err + (long long)(w0 + b) * stride + idx,
-                       make_float4(m[b].x - a.x, m[b].y - a.y, m[b].z - a.z, m[b].w - a.w));
+          for (int b = 0; b < WB; ++b)
+            if (w0 + b < W)
+              st_stream4(err + (long long)(w0 + b) * stride + idx,
+                         make_float4(m[b].x - a.x, m[b].y - a.y, m[b].z - a.z, m[b].w - a.w));
+        }
       }
-      st_stream4(out + idx, a);
+      if (WRITE_OUT) st_stream4(out + idx, a);
     }
-    if (lane < rg.head + rg.tail) {
-      const int col = lane < rg.head ? lane : rg.head + 4 * rg.nbody4 + (lane - rg.head);
+    if (gl < rg.head + rg.tail) {
+      const int col = gl < rg.head ? gl : rg.head + 4 * rg.nbody4 + (gl - rg.head);
       const long long idx = rg.start + col;
       const float a = lowrank_entry(pv, __ldg(Q4 + col), r);
-      for (int w = 0; w < W; ++w) err[(long long)w * stride + idx] -= a;
-      out[idx] = a;
+      if (UPDATE_ERR)
+        for (int w = 0; w < W; ++w) err[(long long)w * stride + idx] -= a;
+      if (WRITE_OUT) out[idx] = a;
     }
   }
+}
+
+// Lazy mode only: after a flush no residual is pending.
+__global__ void psgd_clear_pending_kernel(int* __restrict__ pending, int n_layers) {
+  const int l = blockIdx.x * blockDim.x + threadIdx.x;
+  if (l < n_layers) pending[l] = 0;
 }
 
 cudaError_t launch_powersgd(acc_ctx* ctx, const float* grads, float* err, float* q, float* p_hat,
@@ -308,17 +354,24 @@ cudaError_t launch_powersgd(acc_ctx* ctx, const float* grads, float* err, float*
   const int n_items = (int)pl.row_items.size();
   const int n_vec = (int)pl.vec_tiles.size();
   const float inv_w = 1.0f / (float)c.n_workers;
+  const bool lazy = (c.flags & ACC_FLAG_LAZY_RESIDUAL) != 0;
   if (n_items + n_vec > 0) {
     PhaseTimer pt(ctx, PH_PSGD_PROJECT, s);
-    psgd_project_kernel<4><<<n_items + n_vec, 256, 0, s>>>(
-        ctx->d_layers, ctx->d_row_items, n_items, ctx->d_tiles, ctx->d_vec_tiles, grads, err, q, p_hat, level, out,
-        delta, c.worker_stride, c.n_workers, c.decider, inv_w, c.rank_low, c.rank_high);
+    if (lazy)
+      psgd_project_kernel<4, true><<<n_items + n_vec, 256, 0, s>>>(
+          ctx->d_layers, ctx->d_row_items, n_items, ctx->d_tiles, ctx->d_vec_tiles, grads, err, q, p_hat, level,
+          ctx->d_pending, out, delta, c.worker_stride, c.n_workers, c.decider, inv_w, c.rank_low, c.rank_high);
+    else
+      psgd_project_kernel<4, false><<<n_items + n_vec, 256, 0, s>>>(
+          ctx->d_layers, ctx->d_row_items, n_items, ctx->d_tiles, ctx->d_vec_tiles, grads, err, q, p_hat, level,
+          nullptr, out, delta, c.worker_stride, c.n_workers, c.decider, inv_w, c.rank_low, c.rank_high);
   }
   if (pl.n_mat > 0) {
     {
       PhaseTimer pt(ctx, PH_PSGD_ORTHO, s);
       psgd_orthonormalise_kernel<<<pl.n_mat, 1024, 0, s>>>(ctx->d_layers, ctx->d_mat_layers, p_hat, level,
-                                                          c.rank_low, c.rank_high, c.gs_eps);
+                                                          lazy ? ctx->d_pending : nullptr, c.rank_low, c.rank_high,
+                                                          c.gs_eps);
     }
     {
       PhaseTimer pt(ctx, PH_PSGD_QPARTIAL, s);
@@ -334,9 +387,32 @@ cudaError_t launch_powersgd(acc_ctx* ctx, const float* grads, float* err, float*
     }
     {
       PhaseTimer pt(ctx, PH_PSGD_RESIDUAL, s);
-      psgd_residual_kernel<4><<<n_items, 256, 0, s>>>(ctx->d_layers, ctx->d_row_items, err, q, p_hat, level, out,
-                                                      c.worker_stride, c.n_workers, c.rank_low, c.rank_high);
+      if (lazy)
+        psgd_residual_kernel<4, true, false><<<n_items, 256, 0, s>>>(
+            ctx->d_layers, ctx->d_row_items, err, q, p_hat, level, nullptr, out, c.worker_stride, c.n_workers,
+            c.rank_low, c.rank_high);
+      else
+        psgd_residual_kernel<4, true, true><<<n_items, 256, 0, s>>>(
+            ctx->d_layers, ctx->d_row_items, err, q, p_hat, level, nullptr, out, c.worker_stride, c.n_workers,
+            c.rank_low, c.rank_high);
     }
+  }
+  return cudaGetLastError();
+}
+
+cudaError_t launch_powersgd_flush(acc_ctx* ctx, float* err, const float* q, const float* p_hat, cudaStream_t s) {
+  const Plan& pl = ctx->plan;
+  const acc_config& c = ctx->cfg;
+  const int n_items = (int)pl.row_items.size();
+  if (n_items > 0) {
+    {
+      PhaseTimer pt(ctx, PH_PSGD_FLUSH, s);
+      psgd_residual_kernel<4, false, true><<<n_items, 256, 0, s>>>(
+          ctx->d_layers, ctx->d_row_items, err, q, p_hat, nullptr, ctx->d_pending, nullptr, c.worker_stride,
+          c.n_workers, c.rank_low, c.rank_high);
+    }
+    ctx->last_launches += 1;
+    psgd_clear_pending_kernel<<<(c.n_layers + 127) / 128, 128, 0, s>>>(ctx->d_pending, c.n_layers);
   }
   return cudaGetLastError();
 }

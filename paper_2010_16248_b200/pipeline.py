@@ -19,14 +19,15 @@ from . import workloads as wl
 class AccordionStep:
     def __init__(self, table: wl.LayerTable, n_workers: int, compressors: Sequence[str] = ("powersgd",),
                  rank_low=2, rank_high=1, topk_low_bp=1000, topk_high_bp=100, eta=0.5, gs_eps=1e-8,
-                 check_every=10, decider=0, q_init=None, device="cuda"):
+                 check_every=10, decider=0, q_init=None, device="cuda", lazy_residual=False):
         self.table, self.W = table, n_workers
         self.compressors = tuple(compressors)
         self.check_every = check_every
         self.device = torch.device(device)
         self.ctx = binding.Context(table, n_workers, device=device, rank_low=rank_low, rank_high=rank_high,
                                    topk_low_bp=topk_low_bp, topk_high_bp=topk_high_bp, eta=eta, gs_eps=gs_eps,
-                                   decider=decider)
+                                   decider=decider,
+                                   flags=binding.ACC_FLAG_LAZY_RESIDUAL if lazy_residual else 0)
         dev, L, stride = self.device, table.n_layers, table.stride
         self.level = torch.ones(L, dtype=torch.uint8, device=dev)  # before the first check: low compression
         self.delta = torch.zeros(stride, device=dev)

@@ -264,3 +264,44 @@ def test_bad_arguments_are_rejected():
         binding.Context(table, 2, rank_low=5)
     with pytest.raises(binding.AccError):
         binding.Context(table, 2, topk_low_bp=50, topk_high_bp=100)
+
+
+# ------------------------------------------------------------------ PowerSGD, lazy residual
+@pytest.mark.parametrize("W,rank_low,rank_high", [(2, 2, 1), (8, 4, 1), (3, 3, 2)])
+def test_powersgd_lazy_residual_is_bit_identical_to_eager(W, rank_low, rank_high):
+    """With ACC_FLAG_LAZY_RESIDUAL err holds M_w between steps; out, q and p_hat of every step and the
+    flushed error memory must equal the eager mode's bit for bit, also when the level (rank) changes
+    between steps; the eager mode itself is checked against the oracle above."""
+    table = _table_mixed()
+    eager = binding.Context(table, W, rank_low=rank_low, rank_high=rank_high)
+    lazy = binding.Context(table, W, rank_low=rank_low, rank_high=rank_high, flags=binding.ACC_FLAG_LAZY_RESIDUAL)
+    grads, err0 = _random_inputs(table, W, 40 + W)
+    state = []
+    for ctx in (eager, lazy):
+        state.append(dict(err=err0.clone(), q=ctx.new_q(wl.initial_q(table, 4, seed=3)), p=ctx.new_p(),
+                          out=torch.zeros(table.stride, device="cuda"), delta=torch.zeros(table.stride, device="cuda")))
+    for it in range(4):
+        level = torch.tensor([(l + it) % 2 for l in range(table.n_layers)], dtype=torch.uint8, device="cuda")
+        for ctx, st in zip((eager, lazy), state):
+            ctx.acc_powersgd_step(grads, st["err"], st["q"], st["p"], level, st["out"], st["delta"])
+        torch.cuda.synchronize()
+        for name in ("out", "q", "p", "delta"):
+            assert torch.equal(state[0][name], state[1][name]), f"step {it}: {name} differs"
+        grads, _ = _random_inputs(table, W, 300 + it)
+    lazy.acc_powersgd_flush(state[1]["err"], state[1]["q"], state[1]["p"])
+    torch.cuda.synchronize()
+    assert torch.equal(state[0]["err"], state[1]["err"])
+    # a second flush has nothing pending and changes nothing
+    before = state[1]["err"].clone()
+    lazy.acc_powersgd_flush(state[1]["err"], state[1]["q"], state[1]["p"])
+    torch.cuda.synchronize()
+    assert torch.equal(before, state[1]["err"])
+    # and the run continues identically after a flush
+    for ctx, st in zip((eager, lazy), state):
+        ctx.acc_powersgd_step(grads, st["err"], st["q"], st["p"], level, st["out"], None)
+    lazy.acc_powersgd_flush(state[1]["err"], state[1]["q"], state[1]["p"])
+    torch.cuda.synchronize()
+    for name in ("out", "q", "p", "err"):
+        assert torch.equal(state[0][name], state[1][name]), name
+    with pytest.raises(binding.AccError):
+        eager.acc_powersgd_flush(state[0]["err"], state[0]["q"], state[0]["p"])
