@@ -99,7 +99,8 @@ def _kernel_alg_bytes(name, units):
         "psgd_project_kernel": 12.0,    # read g, read e, write M
         "psgd_residual_kernel": 8.0,    # read M, write e' (eager mode; in lazy mode it only writes out)
         "topk_ef_hist1_kernel": 12.0,   # read g, read e, write M
-        "topk_hist2_kernel": 4.0,       # read M
+        "topk_collect_kernel": 4.0,     # read M
+        "topk_hist2_kernel": 4.0,       # read M (dense path only)
         "topk_hist3_kernel": 4.0,       # read M
         "topk_select_kernel": 4.0,      # read M (+ sparse writes, not counted)
         "ef_kernel": 12.0,

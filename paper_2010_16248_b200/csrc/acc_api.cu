@@ -74,6 +74,8 @@ static int make_plan(const acc_config* cfg, Plan& p) {
     o.k_low = topk_count(size, cfg->topk_low_bp);
     o.k_high = topk_count(size, cfg->topk_high_bp);
     o.seg_off = p.capacity; p.capacity += o.k_low;
+    o.cand_cap = (int)std::max<long long>(64, (size / 8 + 3) / 4 * 4);
+    o.cand_base = p.cand_total; p.cand_total += o.cand_cap;
     // row slabs of the row-wise passes: about kRowSlabElems elements per worker, whole rows,
     // a multiple of 8 rows (one row per warp of a 256-thread block) where the layer allows it
     // lanes per row: a full warp (512 contiguous bytes per access) unless the row is shorter than that;
@@ -116,8 +118,11 @@ static int make_plan(const acc_config* cfg, Plan& p) {
   take(sizeof(unsigned) * seg * kBins1);
   take(sizeof(unsigned) * seg * kBins2);
   take(sizeof(unsigned) * seg * kBins3);
+  take(sizeof(unsigned) * seg);  // candidate counters, cleared with the histograms
   p.hist_bytes = o - p.o_hist;
   p.o_sel = take(sizeof(Select) * seg);
+  p.o_cand = take(sizeof(unsigned) * (size_t)W * std::max<long long>(1, p.cand_total));
+  p.o_tile_cand = take(sizeof(int2) * (size_t)W * nt);
   p.o_tile_cnt = take(sizeof(int2) * (size_t)W * nt);
   p.o_tile_h3 = take(sizeof(unsigned short) * (size_t)W * nt * kBins3);
   p.o_tile_pre = take(sizeof(int2) * (size_t)W * nt);
@@ -170,7 +175,10 @@ int acc_create(const acc_config* cfg, void* workspace, size_t workspace_bytes, a
   ctx->d_hist1 = reinterpret_cast<unsigned*>(ws + p.o_hist);
   ctx->d_hist2 = ctx->d_hist1 + (align_up(sizeof(unsigned) * seg * kBins1, 256) / sizeof(unsigned));
   ctx->d_hist3 = ctx->d_hist2 + (align_up(sizeof(unsigned) * seg * kBins2, 256) / sizeof(unsigned));
+  ctx->d_seg_cand = ctx->d_hist3 + (align_up(sizeof(unsigned) * seg * kBins3, 256) / sizeof(unsigned));
   ctx->d_sel = reinterpret_cast<Select*>(ws + p.o_sel);
+  ctx->d_cand = reinterpret_cast<unsigned*>(ws + p.o_cand);
+  ctx->d_tile_cand = reinterpret_cast<int2*>(ws + p.o_tile_cand);
   ctx->d_tile_cnt = reinterpret_cast<int2*>(ws + p.o_tile_cnt);
   ctx->d_tile_h3 = reinterpret_cast<unsigned short*>(ws + p.o_tile_h3);
   ctx->d_tile_pre = reinterpret_cast<int2*>(ws + p.o_tile_pre);
@@ -327,7 +335,8 @@ const char* acc_profile_kernel_name(int32_t i) {
       "psgd_project_kernel", "psgd_orthonormalise_kernel", "psgd_qpartial_kernel", "psgd_qreduce_kernel",
       "psgd_residual_kernel",
       "topk_ef_hist1_kernel", "topk_pick1_kernel", "topk_hist2_kernel", "topk_pick2_kernel", "topk_hist3_kernel",
-      "topk_pick3_scan_kernel", "topk_select_kernel", "topk_decompress_kernel", "psgd_flush_kernel"};
+      "topk_pick3_scan_kernel", "topk_select_kernel", "topk_decompress_kernel", "psgd_flush_kernel",
+      "topk_collect_kernel"};
   return (i >= 0 && i < PH_COUNT) ? names[i] : "";
 }
 

@@ -28,6 +28,8 @@ struct DevLayer {
   int tile0, ntiles;  // flat tiles of this layer: [tile0, tile0 + ntiles)
   int k_low, k_high;  // TopK counts
   long long seg_off;  // first packed entry of the layer inside a worker's packed region
+  long long cand_base;  // first slot of the layer's candidate keys inside a worker's candidate region
+  int cand_cap;         // slots of that list (the list path is taken when bucket b1 fits)
   long long part_base;  // first float4 of the layer's Q partials
   int slab_rows, nslabs;  // row slabs of the Q-partial pass
 };
@@ -41,15 +43,16 @@ struct Select {
   unsigned b1, b2;      // chosen buckets of level 1 and 2
   unsigned tau;         // 31-bit key of the k-th largest magnitude
   int k, k1, k2, need;  // k wanted; still wanted inside bucket b1 / (b1,b2); ties (key == tau) to keep
-  int pad;
+  int mode;             // kSelDense: levels 2-3 read M;  kSelList: they read the collected keys of bucket b1
 };
+constexpr int kSelDense = 0, kSelList = 1;
 
 // Kernels of the library, for per-kernel timing (acc_profile_*).
 enum Phase {
   PH_EF = 0, PH_NORM_PARTIAL, PH_NORM_FINAL, PH_DETECT,
   PH_PSGD_PROJECT, PH_PSGD_ORTHO, PH_PSGD_QPARTIAL, PH_PSGD_QREDUCE, PH_PSGD_RESIDUAL,
   PH_TOPK_EF_HIST1, PH_TOPK_PICK1, PH_TOPK_HIST2, PH_TOPK_PICK2, PH_TOPK_HIST3, PH_TOPK_PICK3_SCAN, PH_TOPK_SELECT,
-  PH_TOPK_DECOMPRESS, PH_PSGD_FLUSH,
+  PH_TOPK_DECOMPRESS, PH_PSGD_FLUSH, PH_TOPK_COLLECT,
   PH_COUNT
 };
 
@@ -62,11 +65,11 @@ struct Plan {
   std::vector<Tile> tiles;
   std::vector<int> mat_layers;   // layer index of each MATRIX layer
   std::vector<int> vec_tiles;    // tile indices that belong to VECTOR layers
-  long long q_rows = 0, p_rows = 0, capacity = 0, part_f4 = 0;
+  long long q_rows = 0, p_rows = 0, capacity = 0, part_f4 = 0, cand_total = 0;
   int n_mat = 0;
   // workspace offsets (bytes)
   size_t o_layers = 0, o_row_items = 0, o_col_items = 0, o_tiles = 0, o_mat_layers = 0, o_vec_tiles = 0,
-         o_part = 0, o_pending = 0, o_norm_part = 0, o_hist = 0, o_sel = 0, o_tile_cnt = 0, o_tile_h3 = 0, o_tile_pre = 0,
+         o_part = 0, o_pending = 0, o_norm_part = 0, o_hist = 0, o_sel = 0, o_cand = 0, o_tile_cand = 0, o_tile_cnt = 0, o_tile_h3 = 0, o_tile_pre = 0,
          hist_bytes = 0, total = 0;
 };
 
@@ -96,6 +99,9 @@ struct acc_ctx {
   unsigned* d_hist2 = nullptr;
   unsigned* d_hist3 = nullptr;
   acc::Select* d_sel = nullptr;
+  unsigned* d_seg_cand = nullptr;    // per (worker, layer): candidate slots handed out this step
+  unsigned* d_cand = nullptr;        // candidate keys, [W][cand_total]
+  int2* d_tile_cand = nullptr;       // per (worker, tile): (first slot, count) inside the segment's list
   int2* d_tile_cnt = nullptr;
   unsigned short* d_tile_h3 = nullptr;
   int2* d_tile_pre = nullptr;

@@ -3,10 +3,14 @@
 // Selection is a three-level radix select on the 31-bit magnitude pattern key = bits(M) & 0x7fffffff
 // (12 + 12 + 7 bits, shared-memory histograms), followed by an ordered compaction:
 //   ef_hist1   M = g + e -> err, level-1 histogram per (worker, layer)                [reads g, e; writes M]
-//   pick1      bucket b1 holding the k-th largest key
-//   hist2      level-2 histogram of the keys inside b1, per-tile count of keys above b1        [reads M]
+//   pick1      bucket b1 holding the k-th largest key; list path if the keys of b1 fit the candidate list
+//   collect    (list path) keys of bucket b1 -> per-tile ranges of the segment's candidate list,
+//              per-tile count of keys above b1                                                  [reads M]
+//   hist2      level-2 histogram of the keys inside b1 (dense path: reads M and also counts the keys
+//              above b1 per tile; list path: reads the collected keys)
 //   pick2      bucket b2
-//   hist3      per-tile level-3 histogram of the keys with prefix (b1,b2), per-tile count above [reads M]
+//   hist3      per-tile level-3 histogram of the keys with prefix (b1,b2), per-tile count above
+//              (dense path: reads M; list path: reads the collected keys)
 //   pick3scan  threshold tau, number of ties to keep, exclusive per-tile prefix of (above, ties)
 //   select     keep key > tau and the lowest-index `need` of key == tau; write (val, idx) in index
 //              order, zero the kept entries of err                                              [reads M]
@@ -139,7 +143,8 @@ topk_pick1_kernel(const DevLayer* __restrict__ layers, const int* __restrict__ m
   pick_from_top_block(hist1 + (long long)seg * kBins1, k, &bin, &above, sums);
   if (threadIdx.x == 0) {
     Select s;
-    s.b1 = bin; s.b2 = 0; s.tau = 0; s.k = k; s.k1 = k - (int)above; s.k2 = 0; s.need = 0; s.pad = 0;
+    s.b1 = bin; s.b2 = 0; s.tau = 0; s.k = k; s.k1 = k - (int)above; s.k2 = 0; s.need = 0;
+    s.mode = hist1[(long long)seg * kBins1 + bin] <= (unsigned)L.cand_cap ? kSelList : kSelDense;
     sel[seg] = s;
     counts[w * n_layers + l] = k;
   }
@@ -156,10 +161,91 @@ topk_pick2_kernel(int n_mat, const unsigned* __restrict__ hist2, Select* __restr
   if (threadIdx.x == 0) { sel[seg].b2 = bin; sel[seg].k2 = k1 - (int)above; }
 }
 
+// List path.  One block per (tile, worker) of a segment in list mode: the tile's keys of bucket b1 go to a
+// range of the segment's candidate list (reserved with one atomic per tile; the order of the ranges does
+// not matter, the keys are only counted later), and the keys above b1 are counted.
+__global__ void __launch_bounds__(256, 3)
+topk_collect_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict__ tiles, int n_tiles, int n_mat,
+                    const float* __restrict__ err, long long stride, const Select* __restrict__ sel,
+                    unsigned* __restrict__ seg_cand, unsigned* __restrict__ cand, int2* __restrict__ tile_cand,
+                    long long cand_total, int2* __restrict__ tile_cnt) {
+  __shared__ unsigned wsum[8];
+  __shared__ unsigned s_start;
+  const int ti = blockIdx.x, w = blockIdx.y;
+  const Tile t = tiles[ti];
+  const DevLayer L = layers[t.layer];
+  if (L.kind != ACC_MATRIX) return;
+  const int seg = w * n_mat + L.mat;
+  const Select s = sel[seg];
+  if (s.mode != kSelList) return;
+  const float* m = err + (long long)w * stride + L.offset + t.elem0;
+  const int wi = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  float4 mv[8];
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    const int e0 = 4 * (j * 256 + (int)threadIdx.x);
+    if (e0 + 3 < t.nelem) {
+      mv[j] = ld_stream4(m + e0);
+    } else {  // ragged end of the layer: absent elements are masked out by `valid` below
+      mv[j].x = e0 < t.nelem ? m[e0] : 0.f;
+      mv[j].y = e0 + 1 < t.nelem ? m[e0 + 1] : 0.f;
+      mv[j].z = e0 + 2 < t.nelem ? m[e0 + 2] : 0.f;
+      mv[j].w = 0.f;
+    }
+  }
+  unsigned inb = 0;  // 4 bits per j: key in bucket b1
+  int above = 0;
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    const int e0 = 4 * (j * 256 + (int)threadIdx.x);
+    const float v[4] = {mv[j].x, mv[j].y, mv[j].z, mv[j].w};
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const unsigned b = key_of(v[e]) >> 19;
+      const bool valid = e0 + e < t.nelem;
+      above += valid && b > s.b1;
+      inb |= (unsigned)(valid && b == s.b1) << (4 * j + e);
+    }
+  }
+  // block-wide exclusive prefix of (candidates | above << 16)
+  const unsigned own = (unsigned)__popc(inb) | ((unsigned)above << 16);
+  unsigned c = own;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const unsigned n = __shfl_up_sync(0xffffffffu, c, o);
+    if (lane >= o) c += n;
+  }
+  if (lane == 31) wsum[wi] = c;
+  __syncthreads();
+  unsigned wbase = 0, total = 0;
+  for (int i = 0; i < 8; ++i) {
+    if (i < wi) wbase += wsum[i];
+    total += wsum[i];
+  }
+  if (threadIdx.x == 0) {
+    const unsigned n_cand = total & 0xffffu;
+    const unsigned start = n_cand ? atomicAdd(&seg_cand[seg], n_cand) : 0u;
+    s_start = start;
+    tile_cand[(long long)w * n_tiles + ti] = make_int2((int)start, (int)n_cand);
+    tile_cnt[(long long)w * n_tiles + ti].x = (int)(total >> 16);
+  }
+  __syncthreads();
+  if (inb == 0) return;
+  unsigned* dst = cand + (long long)w * cand_total + L.cand_base + s_start + ((wbase + c - own) & 0xffffu);
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    const float v[4] = {mv[j].x, mv[j].y, mv[j].z, mv[j].w};
+#pragma unroll
+    for (int e = 0; e < 4; ++e)
+      if ((inb >> (4 * j + e)) & 1u) *dst++ = key_of(v[e]);
+  }
+}
+
 // Pass C.  Level-2 histogram of the keys whose level-1 bin is b1; per tile, how many keys lie in higher bins.
 __global__ void __launch_bounds__(256)
 topk_hist2_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict__ tiles, int n_tiles, int n_mat,
                   const float* __restrict__ err, long long stride, int W, const Select* __restrict__ sel,
+                  const unsigned* __restrict__ cand, const int2* __restrict__ tile_cand, long long cand_total,
                   unsigned* __restrict__ hist2, int2* __restrict__ tile_cnt) {
   __shared__ unsigned h[kBins2];
   __shared__ int cnt;
@@ -168,7 +254,7 @@ topk_hist2_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict__ 
   __syncthreads();
   const long long V = (long long)W * n_tiles;
   const long long v0 = V * blockIdx.x / gridDim.x, v1 = V * (blockIdx.x + 1) / gridDim.x;
-  int cur = -1;
+  int cur = -1, mode = kSelDense;
   unsigned b1 = 0;
   for (long long v = v0; v < v1; ++v) {
     const int w = (int)(v / n_tiles), ti = (int)(v % n_tiles);
@@ -186,6 +272,13 @@ topk_hist2_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict__ 
       __syncthreads();
       cur = seg;
       b1 = sel[seg].b1;
+      mode = sel[seg].mode;
+    }
+    if (mode == kSelList) {  // the tile's keys of bucket b1 were collected; its count above b1 is already known
+      const int2 tc = tile_cand[(long long)w * n_tiles + ti];
+      const unsigned* c = cand + (long long)w * cand_total + L.cand_base + tc.x;
+      for (int i = threadIdx.x; i < tc.y; i += blockDim.x) atomicAdd(&h[(c[i] >> 7) & 0xfffu], 1u);
+      continue;
     }
     const float* m = err + (long long)w * stride + L.offset + t.elem0;
     int above = 0;
@@ -224,6 +317,7 @@ topk_hist2_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict__ 
 __global__ void __launch_bounds__(256)
 topk_hist3_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict__ tiles, int n_tiles, int n_mat,
                   const float* __restrict__ err, long long stride, const Select* __restrict__ sel,
+                  const unsigned* __restrict__ cand, const int2* __restrict__ tile_cand, long long cand_total,
                   unsigned* __restrict__ hist3, int2* __restrict__ tile_cnt, unsigned short* __restrict__ tile_h3) {
   __shared__ unsigned h[kBins3];
   __shared__ int cnt;
@@ -239,22 +333,32 @@ topk_hist3_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict__ 
   const unsigned prefix = (s.b1 << 12) | s.b2;
   const float* m = err + (long long)w * stride + L.offset + t.elem0;
   int above = 0;
-  const int n4 = t.nelem >> 2;
-#pragma unroll 4
-  for (int i = threadIdx.x; i < n4; i += blockDim.x) {
-    const float4 mv = ld_stream4(m + 4 * i);
-    const unsigned k[4] = {key_of(mv.x), key_of(mv.y), key_of(mv.z), key_of(mv.w)};
-#pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      const unsigned p = k[e] >> 7;
-      above += ((p >> 12) == s.b1) && (p > prefix);
-      if (p == prefix) atomicAdd(&h[k[e] & 127u], 1u);
+  if (s.mode == kSelList) {
+    const int2 tc = tile_cand[(long long)w * n_tiles + ti];
+    const unsigned* c = cand + (long long)w * cand_total + L.cand_base + tc.x;
+    for (int i = threadIdx.x; i < tc.y; i += blockDim.x) {
+      const unsigned k0 = c[i], p = k0 >> 7;  // every collected key lies in bucket b1
+      above += p > prefix;
+      if (p == prefix) atomicAdd(&h[k0 & 127u], 1u);
     }
-  }
-  for (int i = 4 * n4 + threadIdx.x; i < t.nelem; i += blockDim.x) {
-    const unsigned k0 = key_of(m[i]), p = k0 >> 7;
-    above += ((p >> 12) == s.b1) && (p > prefix);
-    if (p == prefix) atomicAdd(&h[k0 & 127u], 1u);
+  } else {
+    const int n4 = t.nelem >> 2;
+#pragma unroll 4
+    for (int i = threadIdx.x; i < n4; i += blockDim.x) {
+      const float4 mv = ld_stream4(m + 4 * i);
+      const unsigned k[4] = {key_of(mv.x), key_of(mv.y), key_of(mv.z), key_of(mv.w)};
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const unsigned p = k[e] >> 7;
+        above += ((p >> 12) == s.b1) && (p > prefix);
+        if (p == prefix) atomicAdd(&h[k[e] & 127u], 1u);
+      }
+    }
+    for (int i = 4 * n4 + threadIdx.x; i < t.nelem; i += blockDim.x) {
+      const unsigned k0 = key_of(m[i]), p = k0 >> 7;
+      above += ((p >> 12) == s.b1) && (p > prefix);
+      if (p == prefix) atomicAdd(&h[k0 & 127u], 1u);
+    }
   }
   above = __reduce_add_sync(0xffffffffu, above);
   if ((threadIdx.x & 31) == 0 && above) atomicAdd(&cnt, above);
@@ -496,9 +600,16 @@ cudaError_t launch_topk(acc_ctx* ctx, const float* grads, float* err, const uint
                                                   ctx->d_hist1, ctx->d_sel, counts);
     }
     {
+      PhaseTimer pt(ctx, PH_TOPK_COLLECT, s);
+      topk_collect_kernel<<<dim3(nt, W), 256, 0, s>>>(ctx->d_layers, ctx->d_tiles, nt, n_mat, err, c.worker_stride,
+                                                      ctx->d_sel, ctx->d_seg_cand, ctx->d_cand, ctx->d_tile_cand,
+                                                      pl.cand_total, ctx->d_tile_cnt);
+    }
+    {
       PhaseTimer pt(ctx, PH_TOPK_HIST2, s);
       topk_hist2_kernel<<<grid, 256, 0, s>>>(ctx->d_layers, ctx->d_tiles, nt, n_mat, err, c.worker_stride, W,
-                                             ctx->d_sel, ctx->d_hist2, ctx->d_tile_cnt);
+                                             ctx->d_sel, ctx->d_cand, ctx->d_tile_cand, pl.cand_total,
+                                             ctx->d_hist2, ctx->d_tile_cnt);
     }
     {
       PhaseTimer pt(ctx, PH_TOPK_PICK2, s);
@@ -507,7 +618,8 @@ cudaError_t launch_topk(acc_ctx* ctx, const float* grads, float* err, const uint
     {
       PhaseTimer pt(ctx, PH_TOPK_HIST3, s);
       topk_hist3_kernel<<<dim3(nt, W), 256, 0, s>>>(ctx->d_layers, ctx->d_tiles, nt, n_mat, err, c.worker_stride,
-                                                    ctx->d_sel, ctx->d_hist3, ctx->d_tile_cnt, ctx->d_tile_h3);
+                                                    ctx->d_sel, ctx->d_cand, ctx->d_tile_cand, pl.cand_total,
+                                                    ctx->d_hist3, ctx->d_tile_cnt, ctx->d_tile_h3);
     }
     {
       PhaseTimer pt(ctx, PH_TOPK_PICK3_SCAN, s);
