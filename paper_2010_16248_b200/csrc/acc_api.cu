@@ -85,9 +85,20 @@ static int make_plan(const acc_config* cfg, Plan& p) {
       o.lpr = nf4 > 16 ? 32 : nf4 > 8 ? 16 : 8;
     }
     const int rows_per_pass = 8 * (32 / o.lpr);  // rows a 256-thread block has in flight
-    int rs = std::max(rows_per_pass, kRowSlabElems / d.cols / rows_per_pass * rows_per_pass);
+    // wide rows are cut into column chunks (multiples of 128 columns) so that items stay small enough to
+    // balance over the SMs; each chunk then yields a partial row of P, summed by the orthonormalise pass
+    o.nchunks = d.cols > kColChunk + kColChunk / 2 ? (d.cols + kColChunk - 1) / kColChunk : 1;
+    const int chunk_w = o.nchunks == 1 ? d.cols : ((d.cols + o.nchunks - 1) / o.nchunks + 127) / 128 * 128;
+    o.ppart_base = -1;
+    if (o.nchunks > 1) { o.ppart_base = p.ppart_f4; p.ppart_f4 += (long long)d.rows * o.nchunks; }
+    int rs = std::max(rows_per_pass, kRowSlabElems / std::min(d.cols, chunk_w) / rows_per_pass * rows_per_pass);
     rs = std::min(rs, d.rows);
-    for (int r0 = 0; r0 < d.rows; r0 += rs) p.row_items.push_back(RowItem{l, r0, std::min(rs, d.rows - r0)});
+    for (int r0 = 0; r0 < d.rows; r0 += rs)
+      for (int ch = 0; ch < o.nchunks; ++ch) {
+        const int c0 = ch * chunk_w;
+        if (c0 >= d.cols) break;
+        p.row_items.push_back(RowItem{l, r0, std::min(rs, d.rows - r0), c0, std::min(chunk_w, d.cols - c0), ch});
+      }
     // row slabs x column blocks of the Q-partial pass (each thread owns `vec` adjacent columns)
     o.slab_rows = std::min(d.rows, std::max(32, (d.rows + 127) / 128));
     o.nslabs = (d.rows + o.slab_rows - 1) / o.slab_rows;
@@ -99,7 +110,7 @@ static int make_plan(const acc_config* cfg, Plan& p) {
   }
   // biggest row items first so that the tail of the grid is made of small ones
   std::stable_sort(p.row_items.begin(), p.row_items.end(), [&](const RowItem& a, const RowItem& b) {
-    return (long long)a.nrows * p.layers[a.layer].cols > (long long)b.nrows * p.layers[b.layer].cols;
+    return (long long)a.nrows * a.ncols > (long long)b.nrows * b.ncols;
   });
   const size_t nt = p.tiles.size();
   const size_t seg = (size_t)W * std::max(p.n_mat, 1);
@@ -112,6 +123,7 @@ static int make_plan(const acc_config* cfg, Plan& p) {
   p.o_mat_layers = take(sizeof(int) * std::max<size_t>(1, p.mat_layers.size()));
   p.o_vec_tiles = take(sizeof(int) * std::max<size_t>(1, p.vec_tiles.size()));
   p.o_part = take(sizeof(float4) * std::max<long long>(1, p.part_f4));
+  p.o_ppart = take(sizeof(float4) * std::max<long long>(1, p.ppart_f4));
   p.o_pending = take(sizeof(int) * L);
   p.o_norm_part = take(sizeof(double) * (size_t)W * nt);
   p.o_hist = o;
@@ -169,6 +181,7 @@ int acc_create(const acc_config* cfg, void* workspace, size_t workspace_bytes, a
   ctx->d_mat_layers = reinterpret_cast<int*>(ws + p.o_mat_layers);
   ctx->d_vec_tiles = reinterpret_cast<int*>(ws + p.o_vec_tiles);
   ctx->d_part = reinterpret_cast<float4*>(ws + p.o_part);
+  ctx->d_ppart = reinterpret_cast<float4*>(ws + p.o_ppart);
   ctx->d_pending = reinterpret_cast<int*>(ws + p.o_pending);
   ctx->d_norm_part = reinterpret_cast<double*>(ws + p.o_norm_part);
   const size_t seg = (size_t)cfg->n_workers * std::max(p.n_mat, 1);
@@ -335,8 +348,8 @@ const char* acc_profile_kernel_name(int32_t i) {
       "psgd_project_kernel", "psgd_orthonormalise_kernel", "psgd_qpartial_kernel", "psgd_qreduce_kernel",
       "psgd_residual_kernel",
       "topk_ef_hist1_kernel", "topk_pick1_kernel", "topk_hist2_kernel", "topk_pick2_kernel", "topk_hist3_kernel",
-      "topk_pick3_scan_kernel", "topk_select_kernel", "topk_decompress_kernel", "psgd_flush_kernel",
-      "topk_collect_kernel"};
+      "topk_tile_scan_kernel", "topk_select_kernel", "topk_decompress_kernel", "psgd_flush_kernel",
+      "topk_collect_kernel", "topk_pick3_kernel", "topk_tile_counts_kernel"};
   return (i >= 0 && i < PH_COUNT) ? names[i] : "";
 }
 

@@ -16,6 +16,7 @@ constexpr int kBins2 = 4096;       // level 2: key bits [18:7]
 constexpr int kBins3 = 128;        // level 3: key bits [6:0]
 constexpr int kRowSlabElems = 8192;  // target elements per (row-slab, worker) of the row-wise kernels
 constexpr int kColBlockThreads = 256;
+constexpr int kColChunk = 1152;      // widest column chunk of a row-wise item
 
 // One layer, device-side view.
 struct DevLayer {
@@ -24,6 +25,8 @@ struct DevLayer {
   int q_row, p_row;   // first row of the layer's block in q / p_hat (MATRIX), else -1
   int vec;            // widest vector width (4, 2, 1) at which every row start is aligned
   int lpr;            // lanes per row (8, 16 or 32) of the row-wise kernels
+  int nchunks;        // column chunks of the row-wise kernels (wide rows are split for load balance)
+  long long ppart_base;  // first float4 of the layer's per-chunk partial P rows (nchunks > 1)
   int mat;            // index among MATRIX layers, else -1
   int tile0, ntiles;  // flat tiles of this layer: [tile0, tile0 + ntiles)
   int k_low, k_high;  // TopK counts
@@ -34,7 +37,7 @@ struct DevLayer {
   int slab_rows, nslabs;  // row slabs of the Q-partial pass
 };
 
-struct RowItem { int layer, row0, nrows; };            // row slab of a MATRIX layer
+struct RowItem { int layer, row0, nrows, col0, ncols, chunk; };  // row slab x column chunk of a MATRIX layer
 struct ColItem { int layer, slab, row0, nrows, col0; };  // (row slab, column block) of a MATRIX layer
 struct Tile { int layer, elem0, nelem; };              // flat tile, never spans layers
 
@@ -52,7 +55,7 @@ enum Phase {
   PH_EF = 0, PH_NORM_PARTIAL, PH_NORM_FINAL, PH_DETECT,
   PH_PSGD_PROJECT, PH_PSGD_ORTHO, PH_PSGD_QPARTIAL, PH_PSGD_QREDUCE, PH_PSGD_RESIDUAL,
   PH_TOPK_EF_HIST1, PH_TOPK_PICK1, PH_TOPK_HIST2, PH_TOPK_PICK2, PH_TOPK_HIST3, PH_TOPK_PICK3_SCAN, PH_TOPK_SELECT,
-  PH_TOPK_DECOMPRESS, PH_PSGD_FLUSH, PH_TOPK_COLLECT,
+  PH_TOPK_DECOMPRESS, PH_PSGD_FLUSH, PH_TOPK_COLLECT, PH_TOPK_PICK3, PH_TOPK_TILE_COUNTS,
   PH_COUNT
 };
 
@@ -65,11 +68,11 @@ struct Plan {
   std::vector<Tile> tiles;
   std::vector<int> mat_layers;   // layer index of each MATRIX layer
   std::vector<int> vec_tiles;    // tile indices that belong to VECTOR layers
-  long long q_rows = 0, p_rows = 0, capacity = 0, part_f4 = 0, cand_total = 0;
+  long long q_rows = 0, p_rows = 0, capacity = 0, part_f4 = 0, cand_total = 0, ppart_f4 = 0;
   int n_mat = 0;
   // workspace offsets (bytes)
   size_t o_layers = 0, o_row_items = 0, o_col_items = 0, o_tiles = 0, o_mat_layers = 0, o_vec_tiles = 0,
-         o_part = 0, o_pending = 0, o_norm_part = 0, o_hist = 0, o_sel = 0, o_cand = 0, o_tile_cand = 0, o_tile_cnt = 0, o_tile_h3 = 0, o_tile_pre = 0,
+         o_part = 0, o_ppart = 0, o_pending = 0, o_norm_part = 0, o_hist = 0, o_sel = 0, o_cand = 0, o_tile_cand = 0, o_tile_cnt = 0, o_tile_h3 = 0, o_tile_pre = 0,
          hist_bytes = 0, total = 0;
 };
 
@@ -93,6 +96,7 @@ struct acc_ctx {
   int* d_mat_layers = nullptr;
   int* d_vec_tiles = nullptr;
   float4* d_part = nullptr;
+  float4* d_ppart = nullptr;         // per-chunk partial rows of P for layers whose rows are split
   int* d_pending = nullptr;          // lazy PowerSGD: rank of the residual not yet applied to err, per layer
   double* d_norm_part = nullptr;
   unsigned* d_hist1 = nullptr;

@@ -9,18 +9,20 @@
 
 namespace acc {
 
+// One row of an item (columns [col0, col0 + ncols) of the layer's row): scalar head up to the first
+// 16-byte boundary, aligned float4 body, scalar tail.  Column indices below are relative to col0.
 struct RowGeom {
-  long long start;  // element index of the row inside a worker's slice
+  long long start;  // element index of the first column of the chunk inside a worker's slice
   int head, nbody4, tail;
 };
 
-__device__ __forceinline__ RowGeom row_geom(const DevLayer& L, int row) {
+__device__ __forceinline__ RowGeom row_geom(const DevLayer& L, const RowItem& it, int row) {
   RowGeom g;
-  g.start = L.offset + (long long)row * L.cols;
+  g.start = L.offset + (long long)row * L.cols + it.col0;
   int h = (int)((4 - (g.start & 3)) & 3);
-  g.head = h < L.cols ? h : L.cols;
-  g.nbody4 = (L.cols - g.head) >> 2;
-  g.tail = L.cols - g.head - 4 * g.nbody4;
+  g.head = h < it.ncols ? h : it.ncols;
+  g.nbody4 = (it.ncols - g.head) >> 2;
+  g.tail = it.ncols - g.head - 4 * g.nbody4;
   return g;
 }
 
@@ -65,9 +67,9 @@ __global__ void __launch_bounds__(256, 3)
 psgd_project_kernel(const DevLayer* __restrict__ layers, const RowItem* __restrict__ items, int n_items,
                     const Tile* __restrict__ tiles, const int* __restrict__ vec_tiles,
                     const float* __restrict__ grads, float* __restrict__ err, const float* __restrict__ q,
-                    float* __restrict__ p, const uint8_t* __restrict__ level, const int* __restrict__ pending,
-                    float* __restrict__ out, float* __restrict__ delta, long long stride, int W, int decider,
-                    float inv_w, int rank_low, int rank_high) {
+                    float* __restrict__ p, float4* __restrict__ p_part, const uint8_t* __restrict__ level,
+                    const int* __restrict__ pending, float* __restrict__ out, float* __restrict__ delta,
+                    long long stride, int W, int decider, float inv_w, int rank_low, int rank_high) {
   if ((int)blockIdx.x >= n_items) {
     const Tile t = tiles[vec_tiles[blockIdx.x - n_items]];
     vector_mean_tile(t, layers[t.layer], grads, out, delta, stride, W, decider, inv_w);
@@ -77,7 +79,7 @@ psgd_project_kernel(const DevLayer* __restrict__ layers, const RowItem* __restri
   const DevLayer L = layers[it.layer];
   const int r = level[it.layer] ? rank_low : rank_high;
   const int rp = LAZY ? pending[it.layer] : 0;
-  const float4* __restrict__ Q4 = reinterpret_cast<const float4*>(q) + L.q_row;
+  const float4* __restrict__ Q4 = reinterpret_cast<const float4*>(q) + L.q_row + it.col0;
   float4* __restrict__ P4 = reinterpret_cast<float4*>(p) + L.p_row;
   const int lpr = L.lpr, groups = 32 / lpr;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -88,7 +90,7 @@ psgd_project_kernel(const DevLayer* __restrict__ layers, const RowItem* __restri
     const bool valid = row < row_end;
     float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
     if (valid) {
-      const RowGeom rg = row_geom(L, row);
+      const RowGeom rg = row_geom(L, it, row);
       float4 pp = make_float4(0.f, 0.f, 0.f, 0.f);
       if (LAZY && rp > 0) pp = P4[row];
       for (int t = gl; t < rg.nbody4; t += lpr) {
@@ -154,12 +156,16 @@ psgd_project_kernel(const DevLayer* __restrict__ layers, const RowItem* __restri
     }
     a0 = group_sum(a0, lpr); a1 = group_sum(a1, lpr); a2 = group_sum(a2, lpr); a3 = group_sum(a3, lpr);
     if (valid && gl == 0) {
-      float4 pv = P4[row];
-      pv.x = a0;
-      if (r > 1) pv.y = a1;
-      if (r > 2) pv.z = a2;
-      if (r > 3) pv.w = a3;
-      P4[row] = pv;
+      if (L.nchunks > 1) {  // partial row of this column chunk; summed over chunks before orthonormalising
+        p_part[L.ppart_base + (long long)row * L.nchunks + it.chunk] = make_float4(a0, a1, a2, a3);
+      } else {
+        float4 pv = P4[row];
+        pv.x = a0;
+        if (r > 1) pv.y = a1;
+        if (r > 2) pv.z = a2;
+        if (r > 3) pv.w = a3;
+        P4[row] = pv;
+      }
     }
   }
 }
@@ -179,8 +185,9 @@ __device__ __forceinline__ double block_sum(double v, double* sm) {
 // Pass 2.  One block per MATRIX layer: modified Gram-Schmidt on the first r columns of P, in place.
 __global__ void __launch_bounds__(1024)
 psgd_orthonormalise_kernel(const DevLayer* __restrict__ layers, const int* __restrict__ mat_layers,
-                           float* __restrict__ p, const uint8_t* __restrict__ level, int* __restrict__ pending,
-                           int rank_low, int rank_high, float eps) {
+                           float* __restrict__ p, const float4* __restrict__ p_part,
+                           const uint8_t* __restrict__ level, int* __restrict__ pending, int rank_low, int rank_high,
+                           float eps) {
   __shared__ double sm[32];
   const int l = mat_layers[blockIdx.x];
   const DevLayer L = layers[l];
@@ -188,6 +195,17 @@ psgd_orthonormalise_kernel(const DevLayer* __restrict__ layers, const int* __res
   if (pending != nullptr && threadIdx.x == 0) pending[l] = r;  // lazy mode: this step's residual stays pending
   float* P = p + 4ll * L.p_row;
   const int n = L.rows;
+  if (L.nchunks > 1) {  // rows split into column chunks: P = sum of the chunk partials, in chunk order
+    for (int i = threadIdx.x; i < n; i += blockDim.x) {
+      const float4* pp = p_part + L.ppart_base + (long long)i * L.nchunks;
+      float4 acc = pp[0];
+      for (int ch = 1; ch < L.nchunks; ++ch) { acc.x += pp[ch].x; acc.y += pp[ch].y; acc.z += pp[ch].z; acc.w += pp[ch].w; }
+      P[4 * i] = acc.x;
+      if (r > 1) P[4 * i + 1] = acc.y;
+      if (r > 2) P[4 * i + 2] = acc.z;
+      if (r > 3) P[4 * i + 3] = acc.w;
+    }
+  }
   for (int c = 0; c < r; ++c) {
     for (int j = 0; j < c; ++j) {
       double part = 0.0;
@@ -298,14 +316,14 @@ psgd_residual_kernel(const DevLayer* __restrict__ layers, const RowItem* __restr
   const DevLayer L = layers[it.layer];
   const int r = pending != nullptr ? pending[it.layer] : (level[it.layer] ? rank_low : rank_high);
   if (r == 0) return;
-  const float4* __restrict__ Q4 = reinterpret_cast<const float4*>(q) + L.q_row;
+  const float4* __restrict__ Q4 = reinterpret_cast<const float4*>(q) + L.q_row + it.col0;
   const float4* __restrict__ P4 = reinterpret_cast<const float4*>(p) + L.p_row;
   const int lpr = L.lpr, groups = 32 / lpr;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = lane / lpr, gl = lane - g * lpr;
   const int row_end = it.row0 + it.nrows;
   for (int row = it.row0 + warp * groups + g; row < row_end; row += 8 * groups) {
-    const RowGeom rg = row_geom(L, row);
+    const RowGeom rg = row_geom(L, it, row);
     const float4 pv = __ldg(P4 + row);
     for (int t = gl; t < rg.nbody4; t += lpr) {
       const int col = rg.head + 4 * t;
@@ -359,17 +377,17 @@ cudaError_t launch_powersgd(acc_ctx* ctx, const float* grads, float* err, float*
     PhaseTimer pt(ctx, PH_PSGD_PROJECT, s);
     if (lazy)
       psgd_project_kernel<4, true><<<n_items + n_vec, 256, 0, s>>>(
-          ctx->d_layers, ctx->d_row_items, n_items, ctx->d_tiles, ctx->d_vec_tiles, grads, err, q, p_hat, level,
-          ctx->d_pending, out, delta, c.worker_stride, c.n_workers, c.decider, inv_w, c.rank_low, c.rank_high);
+          ctx->d_layers, ctx->d_row_items, n_items, ctx->d_tiles, ctx->d_vec_tiles, grads, err, q, p_hat, ctx->d_ppart,
+          level, ctx->d_pending, out, delta, c.worker_stride, c.n_workers, c.decider, inv_w, c.rank_low, c.rank_high);
     else
       psgd_project_kernel<4, false><<<n_items + n_vec, 256, 0, s>>>(
-          ctx->d_layers, ctx->d_row_items, n_items, ctx->d_tiles, ctx->d_vec_tiles, grads, err, q, p_hat, level,
-          nullptr, out, delta, c.worker_stride, c.n_workers, c.decider, inv_w, c.rank_low, c.rank_high);
+          ctx->d_layers, ctx->d_row_items, n_items, ctx->d_tiles, ctx->d_vec_tiles, grads, err, q, p_hat, ctx->d_ppart,
+          level, nullptr, out, delta, c.worker_stride, c.n_workers, c.decider, inv_w, c.rank_low, c.rank_high);
   }
   if (pl.n_mat > 0) {
     {
       PhaseTimer pt(ctx, PH_PSGD_ORTHO, s);
-      psgd_orthonormalise_kernel<<<pl.n_mat, 1024, 0, s>>>(ctx->d_layers, ctx->d_mat_layers, p_hat, level,
+      psgd_orthonormalise_kernel<<<pl.n_mat, 1024, 0, s>>>(ctx->d_layers, ctx->d_mat_layers, p_hat, ctx->d_ppart, level,
                                                           lazy ? ctx->d_pending : nullptr, c.rank_low, c.rank_high,
                                                           c.gs_eps);
     }

@@ -11,7 +11,8 @@
 //   pick2      bucket b2
 //   hist3      per-tile level-3 histogram of the keys with prefix (b1,b2), per-tile count above
 //              (dense path: reads M; list path: reads the collected keys)
-//   pick3scan  threshold tau, number of ties to keep, exclusive per-tile prefix of (above, ties)
+//   pick3      threshold tau and the number of ties to keep
+//   tilecounts per tile (keys above tau, keys equal to tau);  tilescan: their exclusive prefix per layer
 //   select     keep key > tau and the lowest-index `need` of key == tau; write (val, idx) in index
 //              order, zero the kept entries of err                                              [reads M]
 //   decompress out = (1/W) sum_w scatter(idx_w, val_w), accumulated per tile in shared memory [reads packed]
@@ -164,27 +165,17 @@ topk_pick2_kernel(int n_mat, const unsigned* __restrict__ hist2, Select* __restr
 // List path.  One block per (tile, worker) of a segment in list mode: the tile's keys of bucket b1 go to a
 // range of the segment's candidate list (reserved with one atomic per tile; the order of the ranges does
 // not matter, the keys are only counted later), and the keys above b1 are counted.
-__global__ void __launch_bounds__(256, 3)
-topk_collect_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict__ tiles, int n_tiles, int n_mat,
-                    const float* __restrict__ err, long long stride, const Select* __restrict__ sel,
-                    unsigned* __restrict__ seg_cand, unsigned* __restrict__ cand, int2* __restrict__ tile_cand,
-                    long long cand_total, int2* __restrict__ tile_cnt) {
-  __shared__ unsigned wsum[8];
-  __shared__ unsigned s_start;
-  const int ti = blockIdx.x, w = blockIdx.y;
-  const Tile t = tiles[ti];
-  const DevLayer L = layers[t.layer];
-  if (L.kind != ACC_MATRIX) return;
-  const int seg = w * n_mat + L.mat;
-  const Select s = sel[seg];
-  if (s.mode != kSelList) return;
-  const float* m = err + (long long)w * stride + L.offset + t.elem0;
+template <bool FULL>
+__device__ __forceinline__ void collect_tile(const Tile& t, const Select& s, const float* __restrict__ m,
+                                             unsigned* __restrict__ seg_counter, unsigned* __restrict__ seg_list,
+                                             int2* __restrict__ tile_cand_out, int2* __restrict__ tile_cnt_out,
+                                             unsigned* wsum, unsigned* s_start) {
   const int wi = threadIdx.x >> 5, lane = threadIdx.x & 31;
   float4 mv[8];
 #pragma unroll
   for (int j = 0; j < 8; ++j) {
     const int e0 = 4 * (j * 256 + (int)threadIdx.x);
-    if (e0 + 3 < t.nelem) {
+    if (FULL || e0 + 3 < t.nelem) {
       mv[j] = ld_stream4(m + e0);
     } else {  // ragged end of the layer: absent elements are masked out by `valid` below
       mv[j].x = e0 < t.nelem ? m[e0] : 0.f;
@@ -193,7 +184,7 @@ topk_collect_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict_
       mv[j].w = 0.f;
     }
   }
-  unsigned inb = 0;  // 4 bits per j: key in bucket b1
+  unsigned inb = 0;  // one bit per element of this thread: key in bucket b1
   int above = 0;
 #pragma unroll
   for (int j = 0; j < 8; ++j) {
@@ -202,7 +193,7 @@ topk_collect_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict_
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
       const unsigned b = key_of(v[e]) >> 19;
-      const bool valid = e0 + e < t.nelem;
+      const bool valid = FULL || e0 + e < t.nelem;
       above += valid && b > s.b1;
       inb |= (unsigned)(valid && b == s.b1) << (4 * j + e);
     }
@@ -224,14 +215,14 @@ topk_collect_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict_
   }
   if (threadIdx.x == 0) {
     const unsigned n_cand = total & 0xffffu;
-    const unsigned start = n_cand ? atomicAdd(&seg_cand[seg], n_cand) : 0u;
-    s_start = start;
-    tile_cand[(long long)w * n_tiles + ti] = make_int2((int)start, (int)n_cand);
-    tile_cnt[(long long)w * n_tiles + ti].x = (int)(total >> 16);
+    const unsigned start = n_cand ? atomicAdd(seg_counter, n_cand) : 0u;
+    *s_start = start;
+    *tile_cand_out = make_int2((int)start, (int)n_cand);
+    tile_cnt_out->x = (int)(total >> 16);
   }
   __syncthreads();
   if (inb == 0) return;
-  unsigned* dst = cand + (long long)w * cand_total + L.cand_base + s_start + ((wbase + c - own) & 0xffffu);
+  unsigned* dst = seg_list + *s_start + ((wbase + c - own) & 0xffffu);
 #pragma unroll
   for (int j = 0; j < 8; ++j) {
     const float v[4] = {mv[j].x, mv[j].y, mv[j].z, mv[j].w};
@@ -239,6 +230,27 @@ topk_collect_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict_
     for (int e = 0; e < 4; ++e)
       if ((inb >> (4 * j + e)) & 1u) *dst++ = key_of(v[e]);
   }
+}
+
+__global__ void __launch_bounds__(256, 3)
+topk_collect_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict__ tiles, int n_tiles, int n_mat,
+                    const float* __restrict__ err, long long stride, const Select* __restrict__ sel,
+                    unsigned* __restrict__ seg_cand, unsigned* __restrict__ cand, int2* __restrict__ tile_cand,
+                    long long cand_total, int2* __restrict__ tile_cnt) {
+  __shared__ unsigned wsum[8];
+  __shared__ unsigned s_start;
+  const int ti = blockIdx.x, w = blockIdx.y;
+  const Tile t = tiles[ti];
+  const DevLayer L = layers[t.layer];
+  if (L.kind != ACC_MATRIX) return;
+  const int seg = w * n_mat + L.mat;
+  const Select s = sel[seg];
+  if (s.mode != kSelList) return;
+  const float* m = err + (long long)w * stride + L.offset + t.elem0;
+  unsigned* list = cand + (long long)w * cand_total + L.cand_base;
+  const long long v = (long long)w * n_tiles + ti;
+  if (t.nelem == kTile) collect_tile<true>(t, s, m, seg_cand + seg, list, tile_cand + v, tile_cnt + v, wsum, &s_start);
+  else collect_tile<false>(t, s, m, seg_cand + seg, list, tile_cand + v, tile_cnt + v, wsum, &s_start);
 }
 
 // Pass C.  Level-2 histogram of the keys whose level-1 bin is b1; per tile, how many keys lie in higher bins.
@@ -371,50 +383,78 @@ topk_hist3_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict__ 
   }
 }
 
-// One block per (worker, MATRIX layer): final threshold tau and number of ties to keep; then, per tile of
-// the layer, (keys above tau, keys equal to tau) from the per-tile counters, and their exclusive prefix in
-// index order.
+// One warp per (worker, MATRIX layer): bucket b3 of level 3, hence the threshold tau and the number of ties
+// (key == tau) to keep.  Lane l owns bins 4l..4l+3; a suffix sum over the lanes locates the bin.
 __global__ void __launch_bounds__(256)
-topk_pick3_scan_kernel(const DevLayer* __restrict__ layers, const int* __restrict__ mat_layers, int n_mat,
-                       int n_tiles, const unsigned* __restrict__ hist3, Select* __restrict__ sel,
-                       const int2* __restrict__ tile_cnt, const unsigned short* __restrict__ tile_h3,
-                       int2* __restrict__ tile_pre) {
-  __shared__ unsigned b3s;
+topk_pick3_kernel(int n_seg, const unsigned* __restrict__ hist3, Select* __restrict__ sel) {
+  const int seg = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+  if (seg >= n_seg) return;
+  const uint4 c4 = *reinterpret_cast<const uint4*>(hist3 + (long long)seg * kBins3 + 4 * lane);
+  const unsigned c[4] = {c4.x, c4.y, c4.z, c4.w};
+  const unsigned own = c[0] + c[1] + c[2] + c[3];
+  const unsigned want = (unsigned)sel[seg].k2;
+  unsigned suf = own;  // sum over lanes >= this one
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const unsigned n = __shfl_down_sync(0xffffffffu, suf, o);
+    if (lane + o < 32) suf += n;
+  }
+  const unsigned hit = __ballot_sync(0xffffffffu, suf >= want);
+  const int top = hit ? 31 - __clz((int)hit) : 0;  // highest lane whose suffix reaches `want`
+  if (lane == top) {
+    unsigned cum = suf - own;
+    int i = 3;
+    for (; i > 0; --i) {
+      if (cum + c[i] >= want) break;
+      cum += c[i];
+    }
+    Select s = sel[seg];
+    s.tau = (s.b1 << 19) | (s.b2 << 7) | (unsigned)(4 * lane + i);
+    s.need = s.k2 - (int)cum;
+    sel[seg] = s;
+  }
+}
+
+// One warp per (tile, worker): (keys above tau, keys equal to tau) of the tile, from its counters and its
+// level-3 histogram.
+__global__ void __launch_bounds__(256)
+topk_tile_counts_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict__ tiles, int n_tiles, int n_mat,
+                        int W, const Select* __restrict__ sel, const int2* __restrict__ tile_cnt,
+                        const unsigned short* __restrict__ tile_h3, int2* __restrict__ tile_pre) {
+  const long long v = (long long)blockIdx.x * 8 + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  if (v >= (long long)W * n_tiles) return;
+  const int w = (int)(v / n_tiles), ti = (int)(v % n_tiles);
+  const DevLayer L = layers[tiles[ti].layer];
+  if (L.kind != ACC_MATRIX) return;
+  const unsigned b3 = sel[w * n_mat + L.mat].tau & 127u;
+  const unsigned short* h = tile_h3 + v * kBins3;
+  const uint2 raw = *reinterpret_cast<const uint2*>(h + 4 * lane);  // bins 4*lane .. 4*lane+3
+  const unsigned c[4] = {raw.x & 0xffffu, raw.x >> 16, raw.y & 0xffffu, raw.y >> 16};
+  int above = 0, ties = 0;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const unsigned b = 4 * lane + i;
+    above += b > b3 ? (int)c[i] : 0;
+    ties += b == b3 ? (int)c[i] : 0;
+  }
+  above = __reduce_add_sync(0xffffffffu, above);
+  ties = __reduce_add_sync(0xffffffffu, ties);
+  if (lane == 0) {
+    const int2 c0 = tile_cnt[v];
+    tile_pre[v] = make_int2(c0.x + c0.y + above, ties);
+  }
+}
+
+// One block per (worker, MATRIX layer): exclusive prefix, over the layer's tiles in index order, of the
+// per-tile (above, ties) counts, in place.
+__global__ void __launch_bounds__(256)
+topk_tile_scan_kernel(const DevLayer* __restrict__ layers, const int* __restrict__ mat_layers, int n_mat,
+                      int n_tiles, int2* __restrict__ tile_pre) {
   __shared__ int2 chunk_sum[256];
   const int seg = blockIdx.x, w = seg / n_mat, l = mat_layers[seg % n_mat];
   const DevLayer L = layers[l];
-  if (threadIdx.x == 0) {
-    Select s = sel[seg];
-    unsigned bin;
-    long long above;
-    pick_from_top(hist3 + (long long)seg * kBins3, kBins3, s.k2, &bin, &above);
-    s.tau = (s.b1 << 19) | (s.b2 << 7) | bin;
-    s.need = s.k2 - (int)above;
-    sel[seg] = s;
-    b3s = bin;
-  }
-  __syncthreads();
-  const unsigned b3 = b3s;
   const long long tb = (long long)w * n_tiles + L.tile0;
-  // phase 1: one warp per tile turns the tile's level-3 histogram into (above, ties)
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  for (int t = warp; t < L.ntiles; t += 8) {
-    const unsigned short* h = tile_h3 + (tb + t) * kBins3;
-    int above = 0;
-#pragma unroll
-    for (int i = 0; i < kBins3 / 32; ++i) {
-      const unsigned b = i * 32 + lane;
-      const int c = h[b];
-      above += b > b3 ? c : 0;
-    }
-    above = __reduce_add_sync(0xffffffffu, above);
-    if (lane == 0) {
-      const int2 c = tile_cnt[tb + t];
-      tile_pre[tb + t] = make_int2(c.x + c.y + above, (int)h[b3]);
-    }
-  }
-  __syncthreads();
-  // phase 2: exclusive scan over the layer's tiles (each thread owns a contiguous chunk)
   const int per = (L.ntiles + 255) / 256;
   const int t0 = min(L.ntiles, (int)threadIdx.x * per), t1 = min(L.ntiles, t0 + per);
   int2 sum = make_int2(0, 0);
@@ -441,9 +481,102 @@ topk_pick3_scan_kernel(const DevLayer* __restrict__ layers, const int* __restric
   }
 }
 
+__device__ __forceinline__ unsigned warp_incl_scan(unsigned c, int lane) {
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const unsigned n = __shfl_up_sync(0xffffffffu, c, o);
+    if (lane >= o) c += n;
+  }
+  return c;
+}
+
 // Pass E.  One block per (tile, worker).  Warp `wi` owns float4s [wi*256, wi*256+256) of the tile; lane
 // handles float4 j*32+lane of that range for j = 0..7, so (j, lane, element) is index order.  Writes the
 // kept (value, index) pairs at their final positions and zeroes them in err.
+// Per-j lane counts are at most 4 and their warp prefixes at most 128, so four j share one 32-bit scan.
+template <bool FULL>
+__device__ __forceinline__ void select_tile(const Tile& t, const DevLayer& L, const Select& s, const int2 pre,
+                                            float* __restrict__ m, float* __restrict__ vals,
+                                            int32_t* __restrict__ idx, long long seg, unsigned* wtot) {
+  const int wi = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  float4 mv[8];
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    const int e0 = 4 * (wi * 256 + j * 32 + lane);
+    if (FULL || e0 + 3 < t.nelem) {
+      mv[j] = ld_stream4(m + e0);
+    } else {
+      mv[j].x = e0 < t.nelem ? m[e0] : 0.f;
+      mv[j].y = e0 + 1 < t.nelem ? m[e0 + 1] : 0.f;
+      mv[j].z = e0 + 2 < t.nelem ? m[e0 + 2] : 0.f;
+      mv[j].w = 0.f;
+    }
+  }
+  unsigned am = 0, tm = 0;                   // 4 bits per j: key > tau, key == tau
+  unsigned ca[2] = {0, 0}, ct[2] = {0, 0};   // one byte per j: counts of this lane
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    const int e0 = 4 * (wi * 256 + j * 32 + lane);
+    const unsigned k[4] = {key_of(mv[j].x), key_of(mv[j].y), key_of(mv[j].z), key_of(mv[j].w)};
+    unsigned a = 0, tt = 0;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const bool valid = FULL || e0 + e < t.nelem;
+      a |= (unsigned)(valid && k[e] > s.tau) << e;
+      tt |= (unsigned)(valid && k[e] == s.tau) << e;
+    }
+    am |= a << (4 * j);
+    tm |= tt << (4 * j);
+    ca[j >> 2] |= (unsigned)__popc(a) << (8 * (j & 3));
+    ct[j >> 2] |= (unsigned)__popc(tt) << (8 * (j & 3));
+  }
+  unsigned ia[2], it[2] = {0, 0};
+  ia[0] = warp_incl_scan(ca[0], lane);
+  ia[1] = warp_incl_scan(ca[1], lane);
+  const bool any_tie = __any_sync(0xffffffffu, tm != 0);
+  if (any_tie) {
+    it[0] = warp_incl_scan(ct[0], lane);
+    it[1] = warp_incl_scan(ct[1], lane);
+  }
+  const unsigned ta0 = __shfl_sync(0xffffffffu, ia[0], 31), ta1 = __shfl_sync(0xffffffffu, ia[1], 31);
+  const unsigned tt0 = __shfl_sync(0xffffffffu, it[0], 31), tt1 = __shfl_sync(0xffffffffu, it[1], 31);
+  // byte sums: totals of the warp
+  const unsigned wa = __dp4a(ta0, 0x01010101u, 0u) + __dp4a(ta1, 0x01010101u, 0u);
+  const unsigned wt = __dp4a(tt0, 0x01010101u, 0u) + __dp4a(tt1, 0x01010101u, 0u);
+  if (lane == 0) wtot[wi] = wa | (wt << 16);
+  __syncthreads();
+  if ((am | tm) == 0) return;
+  unsigned wbase = 0;
+  for (int i = 0; i < wi; ++i) wbase += wtot[i];
+  int base_a = pre.x + (int)(wbase & 0xffffu), base_t = pre.y + (int)(wbase >> 16);
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    const unsigned a = (am >> (4 * j)) & 15u, tt = (tm >> (4 * j)) & 15u;
+    const unsigned sh = 8 * (j & 3);
+    const unsigned tot_a = ((j < 4 ? ta0 : ta1) >> sh) & 0xffu, tot_t = ((j < 4 ? tt0 : tt1) >> sh) & 0xffu;
+    if (a | tt) {
+      const int e0 = 4 * (wi * 256 + j * 32 + lane);
+      int above_before = base_a + (int)((ia[j >> 2] >> sh) & 0xffu) - __popc(a);
+      int ties_before = base_t + (int)((it[j >> 2] >> sh) & 0xffu) - __popc(tt);
+      const float v[4] = {mv[j].x, mv[j].y, mv[j].z, mv[j].w};
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const bool is_a = (a >> e) & 1u, is_t = (tt >> e) & 1u;
+        if (is_a || (is_t && ties_before < s.need)) {
+          const int pos = above_before + min(ties_before, s.need);
+          vals[seg + pos] = v[e];
+          idx[seg + pos] = t.elem0 + e0 + e;
+          m[e0 + e] = 0.f;
+        }
+        above_before += is_a;
+        ties_before += is_t;
+      }
+    }
+    base_a += (int)tot_a;
+    base_t += (int)tot_t;
+  }
+}
+
 __global__ void __launch_bounds__(256, 3)
 topk_select_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict__ tiles, int n_tiles, int n_mat,
                    float* __restrict__ err, const Select* __restrict__ sel, const int2* __restrict__ tile_pre,
@@ -453,78 +586,12 @@ topk_select_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict__
   const Tile t = tiles[ti];
   const DevLayer L = layers[t.layer];
   if (L.kind != ACC_MATRIX) return;
-  const int wi = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const Select s = sel[w * n_mat + L.mat];
   const int2 pre = tile_pre[(long long)w * n_tiles + ti];
   float* m = err + (long long)w * stride + L.offset + t.elem0;
-  float4 mv[8];
-#pragma unroll
-  for (int j = 0; j < 8; ++j) {
-    const int e0 = 4 * (wi * 256 + j * 32 + lane);
-    if (e0 + 3 < t.nelem) {
-      mv[j] = ld_stream4(m + e0);
-    } else {
-      mv[j].x = e0 < t.nelem ? m[e0] : 0.f;
-      mv[j].y = e0 + 1 < t.nelem ? m[e0 + 1] : 0.f;
-      mv[j].z = e0 + 2 < t.nelem ? m[e0 + 2] : 0.f;
-      mv[j].w = 0.f;
-    }
-  }
-  unsigned am = 0, tm = 0;  // 4 bits per j: key > tau, key == tau
-  unsigned excl[8];         // exclusive prefix inside the warp of (above | ties << 16), per j
-  unsigned carry = 0;
-#pragma unroll
-  for (int j = 0; j < 8; ++j) {
-    const int e0 = 4 * (wi * 256 + j * 32 + lane);
-    const float v[4] = {mv[j].x, mv[j].y, mv[j].z, mv[j].w};
-    unsigned a = 0, tt = 0;
-#pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      const unsigned k = key_of(v[e]);
-      const bool valid = e0 + e < t.nelem;
-      a |= (unsigned)(valid && k > s.tau) << e;
-      tt |= (unsigned)(valid && k == s.tau) << e;
-    }
-    am |= a << (4 * j);
-    tm |= tt << (4 * j);
-    const unsigned own = __popc(a) | (__popc(tt) << 16);
-    unsigned c = own;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      const unsigned n = __shfl_up_sync(0xffffffffu, c, o);
-      if (lane >= o) c += n;
-    }
-    excl[j] = carry + c - own;
-    carry += __shfl_sync(0xffffffffu, c, 31);
-  }
-  if (lane == 0) wtot[wi] = carry;
-  __syncthreads();
-  if ((am | tm) == 0) return;
-  unsigned wbase = 0;
-  for (int i = 0; i < wi; ++i) wbase += wtot[i];
   const long long seg = (long long)w * capacity + L.seg_off;
-#pragma unroll
-  for (int j = 0; j < 8; ++j) {
-    const unsigned a = (am >> (4 * j)) & 15u, tt = (tm >> (4 * j)) & 15u;
-    if ((a | tt) == 0) continue;
-    const int e0 = 4 * (wi * 256 + j * 32 + lane);
-    const unsigned ex = wbase + excl[j];
-    int above_before = pre.x + (int)(ex & 0xffffu);
-    int ties_before = pre.y + (int)(ex >> 16);
-    const float v[4] = {mv[j].x, mv[j].y, mv[j].z, mv[j].w};
-#pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      const bool is_a = (a >> e) & 1u, is_t = (tt >> e) & 1u;
-      if (is_a || (is_t && ties_before < s.need)) {
-        const int pos = above_before + min(ties_before, s.need);
-        vals[seg + pos] = v[e];
-        idx[seg + pos] = t.elem0 + e0 + e;
-        m[e0 + e] = 0.f;
-      }
-      above_before += is_a;
-      ties_before += is_t;
-    }
-  }
+  if (t.nelem == kTile) select_tile<true>(t, L, s, pre, m, vals, idx, seg, wtot);
+  else select_tile<false>(t, L, s, pre, m, vals, idx, seg, wtot);
 }
 
 // Pass F.  Scatter-decompress and average: one block per tile; the tile of `out` is accumulated in shared
@@ -622,10 +689,17 @@ cudaError_t launch_topk(acc_ctx* ctx, const float* grads, float* err, const uint
                                                     ctx->d_hist3, ctx->d_tile_cnt, ctx->d_tile_h3);
     }
     {
+      PhaseTimer pt(ctx, PH_TOPK_PICK3, s);
+      topk_pick3_kernel<<<(W * n_mat + 7) / 8, 256, 0, s>>>(W * n_mat, ctx->d_hist3, ctx->d_sel);
+    }
+    {
+      PhaseTimer pt(ctx, PH_TOPK_TILE_COUNTS, s);
+      topk_tile_counts_kernel<<<(unsigned)(((long long)W * nt + 7) / 8), 256, 0, s>>>(
+          ctx->d_layers, ctx->d_tiles, nt, n_mat, W, ctx->d_sel, ctx->d_tile_cnt, ctx->d_tile_h3, ctx->d_tile_pre);
+    }
+    {
       PhaseTimer pt(ctx, PH_TOPK_PICK3_SCAN, s);
-      topk_pick3_scan_kernel<<<W * n_mat, 256, 0, s>>>(ctx->d_layers, ctx->d_mat_layers, n_mat, nt, ctx->d_hist3,
-                                                       ctx->d_sel, ctx->d_tile_cnt, ctx->d_tile_h3,
-                                                       ctx->d_tile_pre);
+      topk_tile_scan_kernel<<<W * n_mat, 256, 0, s>>>(ctx->d_layers, ctx->d_mat_layers, n_mat, nt, ctx->d_tile_pre);
     }
   }
   if (n_mat > 0) {
