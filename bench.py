@@ -206,7 +206,7 @@ def main():
         return
 
     import torch.distributed as dist
-    from paper_2010_16248_b200 import build, pipeline, workloads as wl
+    from paper_2010_16248_b200 import build, dist_util, pipeline, workloads as wl
     if rank == 0:
         build.build_library()
     assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU path)"
@@ -221,7 +221,7 @@ def main():
     n_comp = len(w.compressors)
     stream_gen = wl.GradientStream(w, device=dev)
     # independent replicas: every rank draws its own gradient batches
-    ring = [stream_gen.grads(1000 * rank + t) for t in range(RING)]
+    ring = [stream_gen.grads(dist_util.replica_seed_offset(rank) + t) for t in range(RING)]
     eng = pipeline.AccordionStep(table, W, w.compressors, w.rank_low, w.rank_high, w.topk_low_bp, w.topk_high_bp,
                                  w.eta, 1e-8, w.check_every, device=dev, lazy_residual=not args.eager)
     n_mat = table.n_matrix_params
@@ -267,12 +267,9 @@ def main():
     total_ms = start.elapsed_time(stop)
     gpu_launches = eng.launches - launches0
     per_step = np.array([a.elapsed_time(b) for a, b in ev])
-    if world > 1:
-        t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = dist_util.max_over_ranks(total_ms, dev)
     ms_per_step = total_ms / K
-    value = grad_bytes_step * world / (ms_per_step * 1e-3) / 1e9
+    value = dist_util.whole_job_throughput(grad_bytes_step, ms_per_step, world) / 1e9
 
     # ---- same K steps again with per-kernel CUDA events (on the launching stream) for the roofline
     eng.ctx.acc_profile_enable(True)
@@ -323,11 +320,8 @@ def main():
     e2.record()
     barrier()
     e2e_ms = s2.elapsed_time(e2)
-    if world > 1:
-        t = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
-    e2e = {"value": grad_bytes_step * world / (e2e_ms / ke * 1e-3) / 1e9, "unit": UNIT, "steps": ke,
+    e2e_ms = dist_util.max_over_ranks(e2e_ms, dev)
+    e2e = {"value": dist_util.whole_job_throughput(grad_bytes_step, e2e_ms / ke, world) / 1e9, "unit": UNIT, "steps": ke,
            "ms_per_step": e2e_ms / ke, "h2d_bytes_per_step": int(4 * W * table.stride),
            "d2h_bytes_per_step": int(4 * table.stride * len(outs_host))}
 

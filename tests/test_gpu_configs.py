@@ -1,0 +1,155 @@
+"""The five BASELINE configurations on the GPU against the oracle.
+
+Protocol.  TopK and the controller are bit-reproducible, so they run free over the iterations and must
+match exactly (levels, indices, counts, packed value bits, error memory).  PowerSGD is compared per step
+from synchronised state: the oracle is fed the GPU's own error memory, Q and levels from just before
+the call (fp32 and fp64 trajectories may drift apart through the memory when singular values are
+close).  Reduced-size versions of each configuration run many iterations across a scale jump; the
+full-size versions run a few steps in the launch configuration bench.py times (lazy residual), with
+the oracle restricted to sampled layers / workers where it would otherwise take minutes."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import accordion_oracle as orc
+from paper_2010_16248_b200 import binding, pipeline, workloads as wl
+from tests import helpers as H
+
+pytestmark = pytest.mark.gpu
+
+
+class OracleController:
+    """Oracle-side mirror of the detection cadence (accumulate, norms, Algorithm 1 every check_every)."""
+
+    def __init__(self, table, check_every, eta):
+        self.layers = H.layers_of(table)
+        self.delta = np.zeros(table.stride)
+        self.prev = -np.ones(table.n_layers)
+        self.level = np.ones(table.n_layers, np.uint8)
+        self.check_every, self.eta, self.t = check_every, eta, 0
+
+    def step(self, g_decider, lr_curr=0.1, lr_next=0.1):
+        orc.accumulate(self.delta, g_decider, self.layers)
+        self.t += 1
+        if self.t % self.check_every == 0:
+            n2 = orc.layer_norms2(self.delta, self.layers)
+            self.level, self.prev = orc.detect_regime(n2, self.prev, lr_curr, lr_next, np.float32(self.eta))
+            self.delta[:] = 0
+
+
+def _run_config(w, iters, t0=0, lazy=False, topk_layers=None, topk_workers=None, psgd_check=None):
+    """Runs `iters` iterations of workload `w` starting at stream iteration t0; checks every TopK step and
+    every level decision exactly, and the PowerSGD steps listed in psgd_check (default: all).  With
+    lazy=True a second engine in lazy-residual mode (the mode bench.py times) runs in lockstep and must
+    reproduce the eager engine's out, Q and P^ bit for bit at every step, and its error memory after a
+    final flush."""
+    table, W = w.table, w.n_workers
+    stream = wl.GradientStream(w, device="cuda")
+    eng = pipeline.AccordionStep(table, W, w.compressors, w.rank_low, w.rank_high, w.topk_low_bp, w.topk_high_bp,
+                                 w.eta, 1e-8, w.check_every)
+    lz = None
+    if lazy and "powersgd" in w.compressors:
+        lz = pipeline.AccordionStep(table, W, ("powersgd",), w.rank_low, w.rank_high, w.topk_low_bp, w.topk_high_bp,
+                                    w.eta, 1e-8, w.check_every, lazy_residual=True)
+    ctl = OracleController(table, w.check_every, w.eta)
+    seen_levels = set()
+    for i in range(iters):
+        grads = stream.grads(t0 + i)
+        level_before = eng.level.clone()
+        assert np.array_equal(level_before.cpu().numpy(), ctl.level), f"iteration {i}: levels differ"
+        seen_levels.update(int(x) for x in ctl.level[table.kind == wl.MATRIX])
+        if "powersgd" in w.compressors:
+            e0, q0 = eng.err_psgd.clone(), eng.q.clone()
+        if "topk" in w.compressors:
+            et0 = eng.err_topk.clone()
+        eng.step(grads)
+        if lz is not None:
+            lz.step(grads)
+        torch.cuda.synchronize()
+        if lz is not None:
+            assert torch.equal(lz.level, eng.level)
+            for name in ("out_psgd", "q", "p_hat"):
+                assert torch.equal(getattr(lz, name), getattr(eng, name)), f"iteration {i}: lazy {name} differs"
+        if "powersgd" in w.compressors and (psgd_check is None or i in psgd_check):
+            H.check_powersgd_against_oracle(eng.ctx, table, grads, e0, q0, level_before, eng.out_psgd, eng.err_psgd,
+                                            eng.q, eng.p_hat, w.rank_low, w.rank_high, 1e-8)
+        if "topk" in w.compressors:
+            H.check_topk_against_oracle(eng.ctx, table, grads, et0, level_before, eng.vals, eng.idx, eng.counts,
+                                        eng.out_topk, eng.err_topk, w.topk_low_bp, w.topk_high_bp,
+                                        layers_subset=topk_layers, workers_subset=topk_workers)
+        ctl.step(grads[0].cpu().numpy())
+    if lz is not None:
+        lz.ctx.acc_powersgd_flush(lz.err_psgd, lz.q, lz.p_hat)
+        torch.cuda.synchronize()
+        assert torch.equal(lz.err_psgd, eng.err_psgd), "flushed lazy error memory differs from the eager one"
+    return seen_levels
+
+
+# ------------------------------------------------------------------ config 1, full size, all 20 iterations
+def test_config1_full_run():
+    w = wl.workload(1)
+    levels = []
+    table, W = w.table, w.n_workers
+    stream = wl.GradientStream(w, device="cuda")
+    eng = pipeline.AccordionStep(table, W, w.compressors, w.rank_low, w.rank_high, w.topk_low_bp, w.topk_high_bp,
+                                 w.eta, 1e-8, w.check_every)
+    ctl = OracleController(table, w.check_every, w.eta)
+    worst = 0.0
+    for t in range(w.n_iters):
+        grads = stream.grads(t)
+        lv = eng.level.clone()
+        levels.append(int(lv[0]))
+        assert np.array_equal(lv.cpu().numpy(), ctl.level)
+        e0, q0, et0 = eng.err_psgd.clone(), eng.q.clone(), eng.err_topk.clone()
+        eng.step(grads)
+        torch.cuda.synchronize()
+        worst = max(worst, H.check_powersgd_against_oracle(eng.ctx, table, grads, e0, q0, lv, eng.out_psgd,
+                                                           eng.err_psgd, eng.q, eng.p_hat, w.rank_low, w.rank_high,
+                                                           1e-8))
+        H.check_topk_against_oracle(eng.ctx, table, grads, et0, lv, eng.vals, eng.idx, eng.counts, eng.out_topk,
+                                    eng.err_topk, w.topk_low_bp, w.topk_high_bp)
+        ctl.step(grads[0].cpu().numpy())
+    # known answer of the schedule: the detector lags the scale jump at iteration 10 by one window
+    assert levels == [1] * 10 + [0] * 5 + [1] * 5
+    assert int(eng.level[0]) == 0 and worst < H.REL_TOL
+
+
+# ------------------------------------------------------------------ reduced-size configs across a scale jump
+@pytest.mark.parametrize("config,scale", [(2, 4), (3, 4), (4, 4), (5, 16)])
+def test_reduced_configs_across_scale_jump(config, scale):
+    w = wl.workload(config, scale=scale)
+    # iterations 80..119 of the schedule: windows [80,90) [90,100) equal -> HIGH, jump at 100 -> LOW at 110
+    seen = _run_config(w, iters=40, t0=80, psgd_check=set(range(0, 40, 3)) | {19, 20, 21, 29, 30, 31, 39})
+    assert seen == {0, 1}, "both compression levels must have been exercised"
+
+
+def test_reduced_config2_lazy_residual():
+    w = wl.workload(2, scale=4)
+    _run_config(w, iters=25, t0=90, lazy=True, psgd_check=set(range(25)))
+
+
+# ------------------------------------------------------------------ full-size configs, bench launch configuration
+@pytest.mark.parametrize("config", [2, 4])
+def test_full_size_powersgd(config):
+    w = wl.workload(config)
+    _run_config(w, iters=3, t0=0, lazy=True)
+
+
+def test_full_size_config3_topk():
+    w = wl.workload(3)
+    big = [l for l in range(w.table.n_layers) if w.table.kind[l] == wl.MATRIX]
+    # every matrix layer for worker 0, plus all workers on the first conv, the largest conv and the classifier
+    _run_config(w, iters=2, t0=0, topk_workers=[0])
+    sizes = w.table.sizes
+    sample = [big[0], int(np.argmax(sizes)), big[-1]]
+    _run_config(w, iters=2, t0=0, topk_layers=sample)
+
+
+def test_full_size_config5_sampled():
+    """LSTM set, W = 8: PowerSGD (lazy) checked on every layer for two steps; TopK checked on the row-sparse
+    encoder (k exceeds its non-zeros: filled with zeros by lowest index), one gate matrix and the decoder
+    for two workers."""
+    w = wl.workload(5)
+    names = w.table.names
+    sample = [names.index("encoder.weight"), names.index("rnn.weight_hh_l1"), names.index("decoder.weight")]
+    _run_config(w, iters=2, t0=0, lazy=True, topk_layers=sample, topk_workers=[0, 5])

@@ -1,0 +1,98 @@
+"""CPU tests of the input generators (structure and determinism of the synthetic gradients) and of the
+multi-process plumbing of the benchmark (world_size 2, gloo)."""
+import os
+
+import numpy as np
+import pytest
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+from paper_2010_16248_b200 import dist_util, workloads as wl
+
+
+def test_tables_are_aligned_and_disjoint():
+    for c in range(1, 6):
+        t = wl.workload(c, scale=8).table
+        assert np.all(t.offset % 4 == 0) and t.stride % 64 == 0
+        ends = t.offset + t.sizes
+        assert np.all(t.offset[1:] >= ends[:-1]) and ends[-1] <= t.stride
+
+
+def test_streams_are_deterministic_and_padding_is_zero():
+    for c in (1, 2, 3, 5):
+        w = wl.workload(c, scale=8)
+        a = wl.GradientStream(w).grads(7)
+        b = wl.GradientStream(w).grads(7)
+        assert torch.equal(a, b)
+        assert not torch.equal(a, wl.GradientStream(w).grads(8))
+        mask = torch.ones(w.table.stride, dtype=torch.bool)
+        for l, sl in w.table.slices():
+            mask[sl] = False
+        assert float(a[:, mask].abs().max()) == 0.0 if mask.any() else True
+        assert a.shape == (w.n_workers, w.table.stride) and a.dtype == torch.float32
+
+
+def test_scale_jumps_double_the_norm():
+    w = wl.workload(2, scale=8)
+    s = wl.GradientStream(w)
+    n99, n100 = s.grads(99).norm().item(), s.grads(100).norm().item()
+    assert 1.8 < n100 / n99 < 2.2
+    assert w.amplitude(0) == 2.0 and w.amplitude(100) == 4.0 and w.amplitude(150) == 8.0
+
+
+def test_topk_workload_has_exact_ties_and_outliers():
+    w = wl.workload(3, scale=4)
+    g = wl.GradientStream(w).grads(0)
+    l = int(np.argmax(w.table.sizes))
+    off, size = int(w.table.offset[l]), int(w.table.sizes[l])
+    x = g[0, off:off + size].abs().numpy()
+    uniq = np.unique(x)
+    assert size - len(uniq) >= size // 1500          # ~0.1 % of the coordinates duplicate a magnitude
+    assert (x > 6 * np.median(x)).mean() > 0.01     # heavy-tailed support carrying the mean
+
+
+def test_lstm_encoder_gradient_is_row_sparse():
+    w = wl.workload(5, scale=16)
+    g = wl.GradientStream(w).grads(3)
+    l = w.table.names.index("encoder.weight")
+    off, n, m = int(w.table.offset[l]), int(w.table.rows[l]), int(w.table.cols[l])
+    for wk in (0, w.n_workers - 1):
+        rows = g[wk, off:off + n * m].view(n, m)
+        nz = int((rows.abs().sum(1) > 0).sum())
+        assert nz == max(1, n * 2 // 100)
+    assert not torch.equal(g[0, off:off + n * m], g[1, off:off + n * m])
+
+
+def _rank_main(rank, world, port, out):
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        ms = dist_util.max_over_ranks(10.0 + 5.0 * rank)
+        w = wl.workload(1, scale=8)
+        g = wl.GradientStream(w).grads(dist_util.replica_seed_offset(rank))
+        sums = [torch.zeros(1, dtype=torch.float64) for _ in range(world)]
+        dist.all_gather(sums, g.double().sum().reshape(1))
+        dist.barrier()
+        out[rank] = (ms, [float(x) for x in sums])
+    finally:
+        dist.destroy_process_group()
+
+
+def test_two_rank_replicas_gloo():
+    world = 2
+    ctx = mp.get_context("spawn")
+    out = ctx.Manager().dict()
+    port = 29500 + os.getpid() % 2000
+    procs = [ctx.Process(target=_rank_main, args=(r, world, port, out)) for r in range(world)]
+    for p in procs:
+        p.start()
+    for p in procs:
+        p.join(120)
+        assert p.exitcode == 0
+    assert out[0][0] == out[1][0] == 15.0                       # slowest rank decides
+    assert out[0][1] == out[1][1] and out[0][1][0] != out[0][1][1]  # ranks drew different batches
+    # whole-job throughput: both ranks' units over the slowest rank's time
+    assert dist_util.whole_job_throughput(100.0, 15.0, world) == pytest.approx(2 * 100.0 / 0.015)
+    assert dist_util.max_over_ranks(3.0) == 3.0                 # no process group: identity
