@@ -131,8 +131,10 @@ static int make_plan(const acc_config* cfg, Plan& p) {
   take(sizeof(unsigned) * seg * kBins2);
   take(sizeof(unsigned) * seg * kBins3);
   take(sizeof(unsigned) * seg);  // candidate counters, cleared with the histograms
+  take(sizeof(unsigned) * seg);  // overflow flags of the predicted collection, likewise
   p.hist_bytes = o - p.o_hist;
   p.o_sel = take(sizeof(Select) * seg);
+  p.o_pred = take(sizeof(unsigned) * 2 * seg);
   p.o_cand = take(sizeof(unsigned) * (size_t)W * std::max<long long>(1, p.cand_total));
   p.o_tile_cand = take(sizeof(int2) * (size_t)W * nt);
   p.o_tile_cnt = take(sizeof(int2) * (size_t)W * nt);
@@ -189,6 +191,8 @@ int acc_create(const acc_config* cfg, void* workspace, size_t workspace_bytes, a
   ctx->d_hist2 = ctx->d_hist1 + (align_up(sizeof(unsigned) * seg * kBins1, 256) / sizeof(unsigned));
   ctx->d_hist3 = ctx->d_hist2 + (align_up(sizeof(unsigned) * seg * kBins2, 256) / sizeof(unsigned));
   ctx->d_seg_cand = ctx->d_hist3 + (align_up(sizeof(unsigned) * seg * kBins3, 256) / sizeof(unsigned));
+  ctx->d_seg_flag = ctx->d_seg_cand + (align_up(sizeof(unsigned) * seg, 256) / sizeof(unsigned));
+  ctx->d_pred = reinterpret_cast<unsigned*>(ws + p.o_pred);
   ctx->d_sel = reinterpret_cast<Select*>(ws + p.o_sel);
   ctx->d_cand = reinterpret_cast<unsigned*>(ws + p.o_cand);
   ctx->d_tile_cand = reinterpret_cast<int2*>(ws + p.o_tile_cand);
@@ -207,6 +211,7 @@ int acc_create(const acc_config* cfg, void* workspace, size_t workspace_bytes, a
   up(ctx->d_mat_layers, p.mat_layers.data(), sizeof(int) * p.mat_layers.size());
   up(ctx->d_vec_tiles, p.vec_tiles.data(), sizeof(int) * p.vec_tiles.size());
   if (e == cudaSuccess) e = cudaMemset(ctx->d_pending, 0, sizeof(int) * cfg->n_layers);
+  if (e == cudaSuccess) e = cudaMemset(ctx->d_pred, 0xff, sizeof(unsigned) * 2 * seg);  // no prediction yet
   int dev = 0;
   if (e == cudaSuccess) e = cudaGetDevice(&dev);
   if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, dev);

@@ -48,7 +48,8 @@ struct Select {
   int k, k1, k2, need;  // k wanted; still wanted inside bucket b1 / (b1,b2); ties (key == tau) to keep
   int mode;             // kSelDense: levels 2-3 read M;  kSelList: they read the collected keys of bucket b1
 };
-constexpr int kSelDense = 0, kSelList = 1;
+constexpr int kSelDense = 0, kSelList = 1, kSelListPred = 2;  // ListPred: the list was filled by pass A
+constexpr int kPredTileCap = 2048;  // keys one tile may hand to a predicted list (more: overflow, fall back)
 
 // Kernels of the library, for per-kernel timing (acc_profile_*).
 enum Phase {
@@ -72,7 +73,7 @@ struct Plan {
   int n_mat = 0;
   // workspace offsets (bytes)
   size_t o_layers = 0, o_row_items = 0, o_col_items = 0, o_tiles = 0, o_mat_layers = 0, o_vec_tiles = 0,
-         o_part = 0, o_ppart = 0, o_pending = 0, o_norm_part = 0, o_hist = 0, o_sel = 0, o_cand = 0, o_tile_cand = 0, o_tile_cnt = 0, o_tile_h3 = 0, o_tile_pre = 0,
+         o_part = 0, o_ppart = 0, o_pending = 0, o_norm_part = 0, o_hist = 0, o_sel = 0, o_pred = 0, o_cand = 0, o_tile_cand = 0, o_tile_cnt = 0, o_tile_h3 = 0, o_tile_pre = 0,
          hist_bytes = 0, total = 0;
 };
 
@@ -104,6 +105,8 @@ struct acc_ctx {
   unsigned* d_hist3 = nullptr;
   acc::Select* d_sel = nullptr;
   unsigned* d_seg_cand = nullptr;    // per (worker, layer): candidate slots handed out this step
+  unsigned* d_seg_flag = nullptr;    // per (worker, layer): 1 if pass A's collection overflowed this step
+  unsigned* d_pred = nullptr;        // [2][W * n_mat]: predicted threshold bucket per level, kept across steps
   unsigned* d_cand = nullptr;        // candidate keys, [W][cand_total]
   int2* d_tile_cand = nullptr;       // per (worker, tile): (first slot, count) inside the segment's list
   int2* d_tile_cnt = nullptr;

@@ -3,7 +3,9 @@
 // Selection is a three-level radix select on the 31-bit magnitude pattern key = bits(M) & 0x7fffffff
 // (12 + 12 + 7 bits, shared-memory histograms), followed by an ordered compaction:
 //   ef_hist1   M = g + e -> err, level-1 histogram per (worker, layer)                [reads g, e; writes M]
-//   pick1      bucket b1 holding the k-th largest key; list path if the keys of b1 fit the candidate list
+//              (+ keys of the buckets around the predicted threshold bucket -> candidate list)
+//   pick1      bucket b1 holding the k-th largest key; predicted-list path if pass A's prediction held,
+//              else list path if the keys of b1 fit the candidate list, else dense path
 //   collect    (list path) keys of bucket b1 -> per-tile ranges of the segment's candidate list,
 //              per-tile count of keys above b1                                                  [reads M]
 //   hist2      level-2 histogram of the keys inside b1 (dense path: reads M and also counts the keys
@@ -23,21 +25,44 @@ namespace acc {
 
 __device__ __forceinline__ unsigned key_of(float v) { return __float_as_uint(v) & 0x7fffffffu; }
 
+// A prediction word: level-1 bucket of the threshold at the segment's last step at this level, and the
+// half-width (in buckets) of the band collected around it.
+constexpr unsigned kPredInvalid = 0xffffffffu;
+__device__ __forceinline__ bool pred_band(unsigned word, unsigned* lo, unsigned* hi) {
+  if (word == kPredInvalid) return false;
+  const unsigned b = word & 0xffffu, hw = word >> 16;
+  *lo = b > hw ? b - hw : 1u;  // bucket 0 (zeros, denormals) is never collected
+  *hi = b + hw < (unsigned)kBins1 ? b + hw : (unsigned)kBins1 - 1u;
+  return *lo <= *hi;
+}
+
 // Pass A.  Persistent blocks over (worker, tile) in worker-major order; the shared histogram is flushed
-// when the (worker, layer) segment changes.
+// when the (worker, layer) segment changes.  Where a prediction of the threshold's level-1 bucket exists
+// (the bucket of the previous step at the same level), the keys of the buckets around it are collected
+// on the fly into the segment's candidate list, so that no further pass over M is needed to refine the
+// threshold when the prediction holds (checked exactly by pick1).
 __global__ void __launch_bounds__(256)
 topk_ef_hist1_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict__ tiles, int n_tiles, int n_mat,
                      const float* __restrict__ grads, float* __restrict__ err, float* __restrict__ delta,
-                     long long stride, int W, int decider, unsigned* __restrict__ hist1) {
+                     long long stride, int W, int decider, const uint8_t* __restrict__ level,
+                     const unsigned* __restrict__ pred, unsigned* __restrict__ hist1,
+                     unsigned* __restrict__ seg_cand, unsigned* __restrict__ seg_flag, unsigned* __restrict__ cand,
+                     int2* __restrict__ tile_cand, long long cand_total, int2* __restrict__ tile_cnt) {
   __shared__ unsigned h[kBins1];
+  __shared__ unsigned s_buf[kPredTileCap];
+  __shared__ unsigned s_cnt, s_start;
+  __shared__ int s_above;
   for (int b = threadIdx.x; b < kBins1; b += blockDim.x) h[b] = 0;
+  if (threadIdx.x == 0) { s_cnt = 0; s_above = 0; }
   __syncthreads();
   const long long V = (long long)W * n_tiles;
   const long long v0 = V * blockIdx.x / gridDim.x, v1 = V * (blockIdx.x + 1) / gridDim.x;
   int cur = -1;
+  bool collect = false;
+  unsigned blo = 1, bhi = 0;
   for (long long v = v0; v < v1; ++v) {
-    const int w = (int)(v / n_tiles);
-    const Tile t = tiles[(int)(v % n_tiles)];
+    const int w = (int)(v / n_tiles), ti = (int)(v % n_tiles);
+    const Tile t = tiles[ti];
     const DevLayer L = layers[t.layer];
     if (L.kind != ACC_MATRIX) continue;
     const int seg = w * n_mat + L.mat;
@@ -50,22 +75,34 @@ topk_ef_hist1_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict
         }
       __syncthreads();
       cur = seg;
+      collect = pred_band(pred[(level[t.layer] ? 1 : 0) * W * n_mat + seg], &blo, &bhi);
     }
     const long long base = L.offset + t.elem0;
     const float* g = grads + (long long)w * stride + base;
     float* e = err + (long long)w * stride + base;
     const bool acc_delta = delta != nullptr && w == decider;
     const int n4 = t.nelem >> 2;
+    const unsigned span = bhi - blo;
+    int above = 0;
 #pragma unroll 4
     for (int i = threadIdx.x; i < n4; i += blockDim.x) {
       const float4 gv = ld_stream4(g + 4 * i);
       const float4 ev = ld_stream4(e + 4 * i);
       const float4 m = make_float4(gv.x + ev.x, gv.y + ev.y, gv.z + ev.z, gv.w + ev.w);
       *reinterpret_cast<float4*>(e + 4 * i) = m;
-      atomicAdd(&h[key_of(m.x) >> 19], 1u);
-      atomicAdd(&h[key_of(m.y) >> 19], 1u);
-      atomicAdd(&h[key_of(m.z) >> 19], 1u);
-      atomicAdd(&h[key_of(m.w) >> 19], 1u);
+      const unsigned k[4] = {key_of(m.x), key_of(m.y), key_of(m.z), key_of(m.w)};
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const unsigned bin = k[q] >> 19;
+        atomicAdd(&h[bin], 1u);
+        if (collect) {
+          above += bin > bhi;
+          if (bin - blo <= span) {
+            const unsigned slot = atomicAdd(&s_cnt, 1u);
+            if (slot < (unsigned)kPredTileCap) s_buf[slot] = k[q];
+          }
+        }
+      }
       if (acc_delta) {
         float4 d = *reinterpret_cast<const float4*>(delta + base + 4 * i);
         d.x += gv.x; d.y += gv.y; d.z += gv.z; d.w += gv.w;
@@ -76,8 +113,40 @@ topk_ef_hist1_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict
       const float gv = g[i];
       const float m = gv + e[i];
       e[i] = m;
-      atomicAdd(&h[key_of(m) >> 19], 1u);
+      const unsigned kk = key_of(m), bin = kk >> 19;
+      atomicAdd(&h[bin], 1u);
+      if (collect) {
+        above += bin > bhi;
+        if (bin - blo <= span) {
+          const unsigned slot = atomicAdd(&s_cnt, 1u);
+          if (slot < (unsigned)kPredTileCap) s_buf[slot] = kk;
+        }
+      }
       if (acc_delta) delta[base + i] += gv;
+    }
+    if (collect) {  // hand the tile's collected keys over to the segment's list
+      above = __reduce_add_sync(0xffffffffu, above);
+      if ((threadIdx.x & 31) == 0 && above) atomicAdd(&s_above, above);
+      __syncthreads();
+      if (threadIdx.x == 0) {
+        unsigned n = s_cnt, start = 0;
+        if (n > (unsigned)kPredTileCap) {
+          atomicOr(&seg_flag[seg], 1u);
+          n = 0;
+        } else if (n) {
+          start = atomicAdd(&seg_cand[seg], n);
+          if (start + n > (unsigned)L.cand_cap) { atomicOr(&seg_flag[seg], 1u); n = 0; }
+        }
+        s_start = start;
+        s_cnt = n;
+        tile_cand[(long long)w * n_tiles + ti] = make_int2((int)start, (int)n);
+        tile_cnt[(long long)w * n_tiles + ti].x = s_above;
+      }
+      __syncthreads();
+      unsigned* dst = cand + (long long)w * cand_total + L.cand_base + s_start;
+      for (unsigned i = threadIdx.x; i < s_cnt; i += blockDim.x) dst[i] = s_buf[i];
+      __syncthreads();
+      if (threadIdx.x == 0) { s_cnt = 0; s_above = 0; }
     }
   }
   __syncthreads();
@@ -130,22 +199,43 @@ __device__ void pick_from_top_block(const unsigned* __restrict__ hist, long long
   __syncthreads();
 }
 
-// One block per (worker, MATRIX layer).
+// One block per (worker, MATRIX layer): level-1 bucket b1 of the threshold, and how levels 2-3 will read
+// the keys of that bucket: from the list collected by pass A if its prediction held (b1 inside the collected
+// band, no overflow), else from a list the collect pass builds if the bucket fits, else from M itself.
+// Also records b1 as the next prediction for this (level, segment).
 __global__ void __launch_bounds__(256)
 topk_pick1_kernel(const DevLayer* __restrict__ layers, const int* __restrict__ mat_layers, int n_mat, int n_layers,
-                  const uint8_t* __restrict__ level, const unsigned* __restrict__ hist1, Select* __restrict__ sel,
-                  int32_t* __restrict__ counts) {
+                  int W, const uint8_t* __restrict__ level, const unsigned* __restrict__ hist1,
+                  Select* __restrict__ sel, int32_t* __restrict__ counts, unsigned* __restrict__ pred,
+                  unsigned* __restrict__ seg_cand, const unsigned* __restrict__ seg_flag) {
   __shared__ unsigned sums[256];
   __shared__ unsigned bin;
   __shared__ long long above;
   const int seg = blockIdx.x, w = seg / n_mat, l = mat_layers[seg % n_mat];
   const DevLayer L = layers[l];
-  const int k = level[l] ? L.k_low : L.k_high;
+  const int lv = level[l] ? 1 : 0;
+  const int k = lv ? L.k_low : L.k_high;
   pick_from_top_block(hist1 + (long long)seg * kBins1, k, &bin, &above, sums);
   if (threadIdx.x == 0) {
     Select s;
     s.b1 = bin; s.b2 = 0; s.tau = 0; s.k = k; s.k1 = k - (int)above; s.k2 = 0; s.need = 0;
-    s.mode = hist1[(long long)seg * kBins1 + bin] <= (unsigned)L.cand_cap ? kSelList : kSelDense;
+    unsigned* pw = pred + (long long)lv * W * n_mat + seg;
+    const unsigned word = *pw;
+    unsigned blo, bhi;
+    const bool had_band = pred_band(word, &blo, &bhi);
+    const bool overflow = seg_flag[seg] != 0;
+    const bool fits = hist1[(long long)seg * kBins1 + bin] <= (unsigned)L.cand_cap;
+    if (had_band && !overflow && bin >= blo && bin <= bhi) {
+      s.mode = kSelListPred;
+    } else {
+      seg_cand[seg] = 0;  // whatever pass A collected is of no use
+      s.mode = fits ? kSelList : kSelDense;
+    }
+    // next prediction: narrow the band after an overflow; none for the zero bucket or for buckets that
+    // do not fit the list
+    unsigned hw = had_band ? (word >> 16) : 1u;
+    if (had_band && overflow) hw = 0;
+    *pw = (!fits || bin == 0) ? kPredInvalid : (bin | (hw << 16));
     sel[seg] = s;
     counts[w * n_layers + l] = k;
   }
@@ -286,10 +376,13 @@ topk_hist2_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict__ 
       b1 = sel[seg].b1;
       mode = sel[seg].mode;
     }
-    if (mode == kSelList) {  // the tile's keys of bucket b1 were collected; its count above b1 is already known
+    if (mode != kSelDense) {  // the tile's keys of bucket b1 were collected; its count above is already known
       const int2 tc = tile_cand[(long long)w * n_tiles + ti];
       const unsigned* c = cand + (long long)w * cand_total + L.cand_base + tc.x;
-      for (int i = threadIdx.x; i < tc.y; i += blockDim.x) atomicAdd(&h[(c[i] >> 7) & 0xfffu], 1u);
+      for (int i = threadIdx.x; i < tc.y; i += blockDim.x) {
+        const unsigned kk = c[i];  // a predicted band may hold keys of neighbouring buckets
+        if ((kk >> 19) == b1) atomicAdd(&h[(kk >> 7) & 0xfffu], 1u);
+      }
       continue;
     }
     const float* m = err + (long long)w * stride + L.offset + t.elem0;
@@ -345,11 +438,11 @@ topk_hist3_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict__ 
   const unsigned prefix = (s.b1 << 12) | s.b2;
   const float* m = err + (long long)w * stride + L.offset + t.elem0;
   int above = 0;
-  if (s.mode == kSelList) {
+  if (s.mode != kSelDense) {
     const int2 tc = tile_cand[(long long)w * n_tiles + ti];
     const unsigned* c = cand + (long long)w * cand_total + L.cand_base + tc.x;
     for (int i = threadIdx.x; i < tc.y; i += blockDim.x) {
-      const unsigned k0 = c[i], p = k0 >> 7;  // every collected key lies in bucket b1
+      const unsigned k0 = c[i], p = k0 >> 7;  // collected keys: bucket b1, or a predicted band around it
       above += p > prefix;
       if (p == prefix) atomicAdd(&h[k0 & 127u], 1u);
     }
@@ -659,12 +752,15 @@ cudaError_t launch_topk(acc_ctx* ctx, const float* grads, float* err, const uint
     {
       PhaseTimer pt(ctx, PH_TOPK_EF_HIST1, s);
       topk_ef_hist1_kernel<<<grid, 256, 0, s>>>(ctx->d_layers, ctx->d_tiles, nt, n_mat, grads, err, delta,
-                                                c.worker_stride, W, c.decider, ctx->d_hist1);
+                                                c.worker_stride, W, c.decider, level, ctx->d_pred, ctx->d_hist1,
+                                                ctx->d_seg_cand, ctx->d_seg_flag, ctx->d_cand, ctx->d_tile_cand,
+                                                pl.cand_total, ctx->d_tile_cnt);
     }
     {
       PhaseTimer pt(ctx, PH_TOPK_PICK1, s);
-      topk_pick1_kernel<<<W * n_mat, 256, 0, s>>>(ctx->d_layers, ctx->d_mat_layers, n_mat, c.n_layers, level,
-                                                  ctx->d_hist1, ctx->d_sel, counts);
+      topk_pick1_kernel<<<W * n_mat, 256, 0, s>>>(ctx->d_layers, ctx->d_mat_layers, n_mat, c.n_layers, W, level,
+                                                  ctx->d_hist1, ctx->d_sel, counts, ctx->d_pred, ctx->d_seg_cand,
+                                                  ctx->d_seg_flag);
     }
     {
       PhaseTimer pt(ctx, PH_TOPK_COLLECT, s);
