@@ -78,29 +78,11 @@ static int make_plan(const acc_config* cfg, Plan& p) {
     o.cand_base = p.cand_total; p.cand_total += o.cand_cap;
     // row slabs of the row-wise passes: about kRowSlabElems elements per worker, whole rows,
     // a multiple of 8 rows (one row per warp of a 256-thread block) where the layer allows it
-    // lanes per row: a full warp (512 contiguous bytes per access) unless the row is shorter than that;
-    // narrower groups on long rows scatter each access over several DRAM pages and measured slower
-    {
-      const int nf4 = std::max(1, d.cols / 4);
-      o.lpr = nf4 > 16 ? 32 : nf4 > 8 ? 16 : 8;
-    }
-    const int rows_per_pass = 8 * (32 / o.lpr);  // rows a 256-thread block has in flight
-    // wide rows are cut into column chunks (multiples of 128 columns) so that items stay small enough to
-    // balance over the SMs; each chunk then yields a partial row of P, summed by the orthonormalise pass
-    o.nchunks = d.cols > kColChunk + kColChunk / 2 ? (d.cols + kColChunk - 1) / kColChunk : 1;
-    const int chunk_w = o.nchunks == 1 ? d.cols : ((d.cols + o.nchunks - 1) / o.nchunks + 127) / 128 * 128;
-    o.ppart_base = -1;
-    if (o.nchunks > 1) { o.ppart_base = p.ppart_f4; p.ppart_f4 += (long long)d.rows * o.nchunks; }
-    int rs = std::max(rows_per_pass, kRowSlabElems / std::min(d.cols, chunk_w) / rows_per_pass * rows_per_pass);
-    rs = std::min(rs, d.rows);
-    for (int r0 = 0; r0 < d.rows; r0 += rs)
-      for (int ch = 0; ch < o.nchunks; ++ch) {
-        const int c0 = ch * chunk_w;
-        if (c0 >= d.cols) break;
-        p.row_items.push_back(RowItem{l, r0, std::min(rs, d.rows - r0), c0, std::min(chunk_w, d.cols - c0), ch});
-      }
+    // partial rows of P: one slot per tile a row can touch
+    o.nslots = (d.cols - 1) / kTile + 2;
+    o.ppart_base = p.ppart_f4; p.ppart_f4 += (long long)d.rows * o.nslots;
     // row slabs x column blocks of the Q-partial pass (each thread owns `vec` adjacent columns)
-    o.slab_rows = std::min(d.rows, std::max(32, (d.rows + 127) / 128));
+    o.slab_rows = std::min(d.rows, std::min(64, std::max(32, (d.rows + 511) / 512)));
     o.nslabs = (d.rows + o.slab_rows - 1) / o.slab_rows;
     o.part_base = p.part_f4; p.part_f4 += (long long)o.nslabs * d.cols;
     const int cb = kColBlockThreads * o.vec;
@@ -108,16 +90,11 @@ static int make_plan(const acc_config* cfg, Plan& p) {
       for (int c0 = 0; c0 < d.cols; c0 += cb)
         p.col_items.push_back(ColItem{l, s, s * o.slab_rows, std::min(o.slab_rows, d.rows - s * o.slab_rows), c0});
   }
-  // biggest row items first so that the tail of the grid is made of small ones
-  std::stable_sort(p.row_items.begin(), p.row_items.end(), [&](const RowItem& a, const RowItem& b) {
-    return (long long)a.nrows * a.ncols > (long long)b.nrows * b.ncols;
-  });
   const size_t nt = p.tiles.size();
   const size_t seg = (size_t)W * std::max(p.n_mat, 1);
   size_t o = 0;
   auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes, 256); return at; };
   p.o_layers = take(sizeof(DevLayer) * L);
-  p.o_row_items = take(sizeof(RowItem) * std::max<size_t>(1, p.row_items.size()));
   p.o_col_items = take(sizeof(ColItem) * std::max<size_t>(1, p.col_items.size()));
   p.o_tiles = take(sizeof(Tile) * nt);
   p.o_mat_layers = take(sizeof(int) * std::max<size_t>(1, p.mat_layers.size()));
@@ -177,7 +154,6 @@ int acc_create(const acc_config* cfg, void* workspace, size_t workspace_bytes, a
   Plan& p = ctx->plan;
   char* ws = ctx->ws;
   ctx->d_layers = reinterpret_cast<DevLayer*>(ws + p.o_layers);
-  ctx->d_row_items = reinterpret_cast<RowItem*>(ws + p.o_row_items);
   ctx->d_col_items = reinterpret_cast<ColItem*>(ws + p.o_col_items);
   ctx->d_tiles = reinterpret_cast<Tile*>(ws + p.o_tiles);
   ctx->d_mat_layers = reinterpret_cast<int*>(ws + p.o_mat_layers);
@@ -205,7 +181,6 @@ int acc_create(const acc_config* cfg, void* workspace, size_t workspace_bytes, a
     if (e == cudaSuccess && bytes) e = cudaMemcpy(dst, src, bytes, cudaMemcpyHostToDevice);
   };
   up(ctx->d_layers, p.layers.data(), sizeof(DevLayer) * p.layers.size());
-  up(ctx->d_row_items, p.row_items.data(), sizeof(RowItem) * p.row_items.size());
   up(ctx->d_col_items, p.col_items.data(), sizeof(ColItem) * p.col_items.size());
   up(ctx->d_tiles, p.tiles.data(), sizeof(Tile) * p.tiles.size());
   up(ctx->d_mat_layers, p.mat_layers.data(), sizeof(int) * p.mat_layers.size());

@@ -14,9 +14,7 @@ constexpr int kTile = 8192;        // elements per flat tile (TopK / EF / norms)
 constexpr int kBins1 = 4096;       // radix-select level 1: key bits [30:19]
 constexpr int kBins2 = 4096;       // level 2: key bits [18:7]
 constexpr int kBins3 = 128;        // level 3: key bits [6:0]
-constexpr int kRowSlabElems = 8192;  // target elements per (row-slab, worker) of the row-wise kernels
 constexpr int kColBlockThreads = 256;
-constexpr int kColChunk = 1152;      // widest column chunk of a row-wise item
 
 // One layer, device-side view.
 struct DevLayer {
@@ -24,9 +22,8 @@ struct DevLayer {
   int rows, cols, kind;
   int q_row, p_row;   // first row of the layer's block in q / p_hat (MATRIX), else -1
   int vec;            // widest vector width (4, 2, 1) at which every row start is aligned
-  int lpr;            // lanes per row (8, 16 or 32) of the row-wise kernels
-  int nchunks;        // column chunks of the row-wise kernels (wide rows are split for load balance)
-  long long ppart_base;  // first float4 of the layer's per-chunk partial P rows (nchunks > 1)
+  int nslots;         // tiles a row of this layer can touch: (cols - 1) / 8192 + 2
+  long long ppart_base;  // first float4 of the layer's partial P rows, [rows][nslots]
   int mat;            // index among MATRIX layers, else -1
   int tile0, ntiles;  // flat tiles of this layer: [tile0, tile0 + ntiles)
   int k_low, k_high;  // TopK counts
@@ -37,7 +34,6 @@ struct DevLayer {
   int slab_rows, nslabs;  // row slabs of the Q-partial pass
 };
 
-struct RowItem { int layer, row0, nrows, col0, ncols, chunk; };  // row slab x column chunk of a MATRIX layer
 struct ColItem { int layer, slab, row0, nrows, col0; };  // (row slab, column block) of a MATRIX layer
 struct Tile { int layer, elem0, nelem; };              // flat tile, never spans layers
 
@@ -64,7 +60,6 @@ struct ProfSlot { int phase; cudaEvent_t a, b; };
 
 struct Plan {
   std::vector<DevLayer> layers;
-  std::vector<RowItem> row_items;
   std::vector<ColItem> col_items;
   std::vector<Tile> tiles;
   std::vector<int> mat_layers;   // layer index of each MATRIX layer
@@ -72,7 +67,7 @@ struct Plan {
   long long q_rows = 0, p_rows = 0, capacity = 0, part_f4 = 0, cand_total = 0, ppart_f4 = 0;
   int n_mat = 0;
   // workspace offsets (bytes)
-  size_t o_layers = 0, o_row_items = 0, o_col_items = 0, o_tiles = 0, o_mat_layers = 0, o_vec_tiles = 0,
+  size_t o_layers = 0, o_col_items = 0, o_tiles = 0, o_mat_layers = 0, o_vec_tiles = 0,
          o_part = 0, o_ppart = 0, o_pending = 0, o_norm_part = 0, o_hist = 0, o_sel = 0, o_pred = 0, o_cand = 0, o_tile_cand = 0, o_tile_cnt = 0, o_tile_h3 = 0, o_tile_pre = 0,
          hist_bytes = 0, total = 0;
 };
@@ -91,13 +86,12 @@ struct acc_ctx {
   size_t prof_used = 0;
   // device views into the workspace
   acc::DevLayer* d_layers = nullptr;
-  acc::RowItem* d_row_items = nullptr;
   acc::ColItem* d_col_items = nullptr;
   acc::Tile* d_tiles = nullptr;
   int* d_mat_layers = nullptr;
   int* d_vec_tiles = nullptr;
   float4* d_part = nullptr;
-  float4* d_ppart = nullptr;         // per-chunk partial rows of P for layers whose rows are split
+  float4* d_ppart = nullptr;         // partial rows of P, one slot per tile a row touches
   int* d_pending = nullptr;          // lazy PowerSGD: rank of the residual not yet applied to err, per layer
   double* d_norm_part = nullptr;
   unsigned* d_hist1 = nullptr;

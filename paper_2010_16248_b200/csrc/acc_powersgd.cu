@@ -3,27 +3,36 @@
 // Because every product of the step is linear in the workers' matrices, the factors only depend on
 // the mean matrix  Mbar = (1/W) sum_w (g_w + e_w):   P = Mbar Q,  Q' = Mbar^T P^,  A = P^ Q'^T.
 // The project pass therefore reads every worker's g and e once, writes M_w back over e_w, and keeps
-// Mbar (1/W of the data) in `out` for the second product; only the residual pass touches the
-// per-worker data again.
+// Mbar (1/W of the data) in `out` for the second product.
+//
+// The streaming passes work on flat 8192-element tiles of a layer (the same tiles as the TopK path):
+// every access is a fully coalesced, 16-byte aligned float4 whatever the row length, and all blocks carry
+// the same load.  Row structure only enters through the factors: element i of a layer sits in row i / m,
+// column i % m, and the rows a tile cuts are reduced from shared memory afterwards.
 #include "acc_internal.cuh"
 
 namespace acc {
 
-// One row of an item (columns [col0, col0 + ncols) of the layer's row): scalar head up to the first
-// 16-byte boundary, aligned float4 body, scalar tail.  Column indices below are relative to col0.
-struct RowGeom {
-  long long start;  // element index of the first column of the chunk inside a worker's slice
-  int head, nbody4, tail;
-};
+__device__ __forceinline__ float lowrank_entry(const float4& pv, const float4& qv, int r) {
+  float a = pv.x * qv.x;
+  if (r > 1) a = fmaf(pv.y, qv.y, a);
+  if (r > 2) a = fmaf(pv.z, qv.z, a);
+  if (r > 3) a = fmaf(pv.w, qv.w, a);
+  return a;
+}
 
-__device__ __forceinline__ RowGeom row_geom(const DevLayer& L, const RowItem& it, int row) {
-  RowGeom g;
-  g.start = L.offset + (long long)row * L.cols + it.col0;
-  int h = (int)((4 - (g.start & 3)) & 3);
-  g.head = h < it.ncols ? h : it.ncols;
-  g.nbody4 = (it.ncols - g.head) >> 2;
-  g.tail = it.ncols - g.head - 4 * g.nbody4;
-  return g;
+// A = P^[row] . Q[col] (first r ranks) for the four consecutive elements that start at layer element e_idx.
+__device__ __forceinline__ float4 lowrank4(const float4* __restrict__ P4, const float4* __restrict__ Q4, int m,
+                                           int e_idx, int r) {
+  int row = e_idx / m, col = e_idx - row * m;
+  float4 pv = __ldg(P4 + row);
+  float a[4];
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    a[e] = lowrank_entry(pv, __ldg(Q4 + col), r);
+    if (++col == m && e < 3) { col = 0; ++row; pv = __ldg(P4 + row); }
+  }
+  return make_float4(a[0], a[1], a[2], a[3]);
 }
 
 // out = mean_w g_w on one tile of a VECTOR layer; delta += g_decider.
@@ -42,131 +51,103 @@ __device__ void vector_mean_tile(const Tile& t, const DevLayer& L, const float* 
   }
 }
 
-__device__ __forceinline__ float lowrank_entry(const float4& pv, const float4& qv, int r) {
-  float a = pv.x * qv.x;
-  if (r > 1) a = fmaf(pv.y, qv.y, a);
-  if (r > 2) a = fmaf(pv.z, qv.z, a);
-  if (r > 3) a = fmaf(pv.w, qv.w, a);
-  return a;
-}
-
-// Sum over the `lpr` consecutive lanes of a row group (lpr = 8, 16 or 32); every lane of the warp calls it.
-__device__ __forceinline__ float group_sum(float v, int lpr) {
-  for (int o = lpr >> 1; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-  return v;
-}
-
-// Pass 1.  One block per row slab, all workers.  A group of `lpr` lanes owns a row (8*32/lpr rows in
-// flight per block):
-//   e_w = err_w                               (eager: err holds the error memory)
+// Pass 1.  One block per tile, all workers:
+//   e_w = err_w                                 (eager: err holds the error memory)
 //   e_w = err_w - P^_prev Q^T  (first rp ranks) (lazy: err holds last step's M_w, residual still pending)
-//   M_w = g_w + e_w -> err;  Mbar = mean_w M_w -> out;  P[row, :] = Mbar[row, :] . Q   (first r ranks);
-//   delta += g_decider.  Blocks beyond the row items handle the VECTOR tiles.
+//   M_w = g_w + e_w -> err;  Mbar = mean_w M_w -> out and shared memory;  delta += g_decider;
+// then, for every row the tile cuts, the partial dot products Mbar[row, cols in tile] . Q go to the row's
+// slot for this tile in p_part (a row touches (m-1)/8192 + 2 tiles at most; the orthonormalise pass adds
+// the slots in order).
 template <int WB, bool LAZY>
 __global__ void __launch_bounds__(256, 3)
-psgd_project_kernel(const DevLayer* __restrict__ layers, const RowItem* __restrict__ items, int n_items,
-                    const Tile* __restrict__ tiles, const int* __restrict__ vec_tiles,
+psgd_project_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict__ tiles,
                     const float* __restrict__ grads, float* __restrict__ err, const float* __restrict__ q,
-                    float* __restrict__ p, float4* __restrict__ p_part, const uint8_t* __restrict__ level,
+                    const float* __restrict__ p, float4* __restrict__ p_part, const uint8_t* __restrict__ level,
                     const int* __restrict__ pending, float* __restrict__ out, float* __restrict__ delta,
-                    long long stride, int W, int decider, float inv_w, int rank_low, int rank_high) {
-  if ((int)blockIdx.x >= n_items) {
-    const Tile t = tiles[vec_tiles[blockIdx.x - n_items]];
-    vector_mean_tile(t, layers[t.layer], grads, out, delta, stride, W, decider, inv_w);
+                    long long stride, int W, int decider, float inv_w) {
+  __shared__ __align__(16) float s_mbar[kTile];
+  const Tile t = tiles[blockIdx.x];
+  const DevLayer L = layers[t.layer];
+  if (L.kind != ACC_MATRIX) {
+    vector_mean_tile(t, L, grads, out, delta, stride, W, decider, inv_w);
     return;
   }
-  const RowItem it = items[blockIdx.x];
-  const DevLayer L = layers[it.layer];
-  const int r = level[it.layer] ? rank_low : rank_high;
-  const int rp = LAZY ? pending[it.layer] : 0;
-  const float4* __restrict__ Q4 = reinterpret_cast<const float4*>(q) + L.q_row + it.col0;
-  float4* __restrict__ P4 = reinterpret_cast<float4*>(p) + L.p_row;
-  const int lpr = L.lpr, groups = 32 / lpr;
+  const int rp = LAZY ? pending[t.layer] : 0;
+  const int m = L.cols;
+  const float4* __restrict__ Q4 = reinterpret_cast<const float4*>(q) + L.q_row;
+  const float4* __restrict__ P4 = reinterpret_cast<const float4*>(p) + L.p_row;
+  const long long base = L.offset + t.elem0;
+  const int n4 = t.nelem >> 2;
+  for (int f = threadIdx.x; f < n4; f += blockDim.x) {
+    const long long idx = base + 4 * f;
+    float4 corr = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (LAZY && rp > 0) corr = lowrank4(P4, Q4, m, t.elem0 + 4 * f, rp);
+    float4 mb = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int w0 = 0; w0 < W; w0 += WB) {
+      float4 gv[WB], ev[WB];
+#pragma unroll
+      for (int b = 0; b < WB; ++b)
+        if (w0 + b < W) {
+          gv[b] = ld_stream4(grads + (long long)(w0 + b) * stride + idx);
+          ev[b] = ld_stream4(err + (long long)(w0 + b) * stride + idx);
+        }
+#pragma unroll
+      for (int b = 0; b < WB; ++b)
+        if (w0 + b < W) {
+          float4 e = ev[b];
+          if (LAZY && rp > 0) { e.x -= corr.x; e.y -= corr.y; e.z -= corr.z; e.w -= corr.w; }
+          const float4 mw = make_float4(gv[b].x + e.x, gv[b].y + e.y, gv[b].z + e.z, gv[b].w + e.w);
+          if (LAZY) st_stream4(err + (long long)(w0 + b) * stride + idx, mw);
+          else *reinterpret_cast<float4*>(err + (long long)(w0 + b) * stride + idx) = mw;
+          mb.x += mw.x; mb.y += mw.y; mb.z += mw.z; mb.w += mw.w;
+          if (delta != nullptr && w0 + b == decider) {
+            float4 d = *reinterpret_cast<const float4*>(delta + idx);
+            d.x += gv[b].x; d.y += gv[b].y; d.z += gv[b].z; d.w += gv[b].w;
+            *reinterpret_cast<float4*>(delta + idx) = d;
+          }
+        }
+    }
+    mb.x *= inv_w; mb.y *= inv_w; mb.z *= inv_w; mb.w *= inv_w;
+    *reinterpret_cast<float4*>(out + idx) = mb;
+    *reinterpret_cast<float4*>(s_mbar + 4 * f) = mb;
+  }
+  for (int i = 4 * n4 + threadIdx.x; i < t.nelem; i += blockDim.x) {  // last 1-3 elements of the layer
+    const long long idx = base + i;
+    const int e_idx = t.elem0 + i, row = e_idx / m, col = e_idx - row * m;
+    const float corr = (LAZY && rp > 0) ? lowrank_entry(__ldg(P4 + row), __ldg(Q4 + col), rp) : 0.f;
+    float mb = 0.f;
+    for (int w = 0; w < W; ++w) {
+      const float gv = grads[(long long)w * stride + idx];
+      float e = err[(long long)w * stride + idx];
+      if (LAZY && rp > 0) e -= corr;
+      const float mw = gv + e;
+      err[(long long)w * stride + idx] = mw;
+      mb += mw;
+      if (delta != nullptr && w == decider) delta[idx] += gv;
+    }
+    mb *= inv_w;
+    out[idx] = mb;
+    s_mbar[i] = mb;
+  }
+  __syncthreads();
+  // partial rows of P from the tile in shared memory: one warp per row piece
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int g = lane / lpr, gl = lane - g * lpr;
-  const int row_end = it.row0 + it.nrows;
-  for (int r0 = it.row0 + warp * groups; r0 < row_end; r0 += 8 * groups) {
-    const int row = r0 + g;
-    const bool valid = row < row_end;
+  const int first_row = t.elem0 / m, last_row = (t.elem0 + t.nelem - 1) / m;
+  const int tile_in_layer = t.elem0 / kTile;
+  for (int row = first_row + warp; row <= last_row; row += 8) {
+    const int row_begin = row * m;
+    const int lo = max(row_begin, t.elem0) - t.elem0, hi = min(row_begin + m, t.elem0 + t.nelem) - t.elem0;
+    const float4* qr = Q4 + (t.elem0 + lo - row_begin);
     float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
-    if (valid) {
-      const RowGeom rg = row_geom(L, it, row);
-      float4 pp = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (LAZY && rp > 0) pp = P4[row];
-      for (int t = gl; t < rg.nbody4; t += lpr) {
-        const int col = rg.head + 4 * t;
-        const long long idx = rg.start + col;
-        const float4 q0 = __ldg(Q4 + col), q1 = __ldg(Q4 + col + 1), q2 = __ldg(Q4 + col + 2), q3 = __ldg(Q4 + col + 3);
-        float4 corr = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (LAZY && rp > 0) {
-          corr.x = lowrank_entry(pp, q0, rp); corr.y = lowrank_entry(pp, q1, rp);
-          corr.z = lowrank_entry(pp, q2, rp); corr.w = lowrank_entry(pp, q3, rp);
-        }
-        float4 mb = make_float4(0.f, 0.f, 0.f, 0.f);
-        for (int w0 = 0; w0 < W; w0 += WB) {
-          float4 gv[WB], ev[WB];
-#pragma unroll
-          for (int b = 0; b < WB; ++b)
-            if (w0 + b < W) {
-              gv[b] = ld_stream4(grads + (long long)(w0 + b) * stride + idx);
-              ev[b] = ld_stream4(err + (long long)(w0 + b) * stride + idx);
-            }
-#pragma unroll
-          for (int b = 0; b < WB; ++b)
-            if (w0 + b < W) {
-              float4 e = ev[b];
-              if (LAZY && rp > 0) { e.x -= corr.x; e.y -= corr.y; e.z -= corr.z; e.w -= corr.w; }
-              const float4 m = make_float4(gv[b].x + e.x, gv[b].y + e.y, gv[b].z + e.z, gv[b].w + e.w);
-              if (LAZY) st_stream4(err + (long long)(w0 + b) * stride + idx, m);
-              else *reinterpret_cast<float4*>(err + (long long)(w0 + b) * stride + idx) = m;
-              mb.x += m.x; mb.y += m.y; mb.z += m.z; mb.w += m.w;
-              if (delta != nullptr && w0 + b == decider) {
-                float4 d = *reinterpret_cast<const float4*>(delta + idx);
-                d.x += gv[b].x; d.y += gv[b].y; d.z += gv[b].z; d.w += gv[b].w;
-                *reinterpret_cast<float4*>(delta + idx) = d;
-              }
-            }
-        }
-        mb.x *= inv_w; mb.y *= inv_w; mb.z *= inv_w; mb.w *= inv_w;
-        *reinterpret_cast<float4*>(out + idx) = mb;
-        a0 = fmaf(mb.x, q0.x, a0); a1 = fmaf(mb.x, q0.y, a1); a2 = fmaf(mb.x, q0.z, a2); a3 = fmaf(mb.x, q0.w, a3);
-        a0 = fmaf(mb.y, q1.x, a0); a1 = fmaf(mb.y, q1.y, a1); a2 = fmaf(mb.y, q1.z, a2); a3 = fmaf(mb.y, q1.w, a3);
-        a0 = fmaf(mb.z, q2.x, a0); a1 = fmaf(mb.z, q2.y, a1); a2 = fmaf(mb.z, q2.z, a2); a3 = fmaf(mb.z, q2.w, a3);
-        a0 = fmaf(mb.w, q3.x, a0); a1 = fmaf(mb.w, q3.y, a1); a2 = fmaf(mb.w, q3.z, a2); a3 = fmaf(mb.w, q3.w, a3);
-      }
-      if (gl < rg.head + rg.tail) {  // the unaligned ends of the row, one element per lane
-        const int col = gl < rg.head ? gl : rg.head + 4 * rg.nbody4 + (gl - rg.head);
-        const long long idx = rg.start + col;
-        const float4 q0 = __ldg(Q4 + col);
-        const float corr = (LAZY && rp > 0) ? lowrank_entry(pp, q0, rp) : 0.f;
-        float mb = 0.f;
-        for (int w = 0; w < W; ++w) {
-          const float gv = grads[(long long)w * stride + idx];
-          float e = err[(long long)w * stride + idx];
-          if (LAZY && rp > 0) e -= corr;
-          const float m = gv + e;
-          err[(long long)w * stride + idx] = m;
-          mb += m;
-          if (delta != nullptr && w == decider) delta[idx] += gv;
-        }
-        mb *= inv_w;
-        out[idx] = mb;
-        a0 = fmaf(mb, q0.x, a0); a1 = fmaf(mb, q0.y, a1); a2 = fmaf(mb, q0.z, a2); a3 = fmaf(mb, q0.w, a3);
-      }
+    for (int i = lo + lane; i < hi; i += 32) {
+      const float v = s_mbar[i];
+      const float4 qv = __ldg(qr + (i - lo));
+      a0 = fmaf(v, qv.x, a0); a1 = fmaf(v, qv.y, a1); a2 = fmaf(v, qv.z, a2); a3 = fmaf(v, qv.w, a3);
     }
-    a0 = group_sum(a0, lpr); a1 = group_sum(a1, lpr); a2 = group_sum(a2, lpr); a3 = group_sum(a3, lpr);
-    if (valid && gl == 0) {
-      if (L.nchunks > 1) {  // partial row of this column chunk; summed over chunks before orthonormalising
-        p_part[L.ppart_base + (long long)row * L.nchunks + it.chunk] = make_float4(a0, a1, a2, a3);
-      } else {
-        float4 pv = P4[row];
-        pv.x = a0;
-        if (r > 1) pv.y = a1;
-        if (r > 2) pv.z = a2;
-        if (r > 3) pv.w = a3;
-        P4[row] = pv;
-      }
-    }
+    a0 = warp_sum(a0); a1 = warp_sum(a1); a2 = warp_sum(a2); a3 = warp_sum(a3);
+    if (lane == 0)
+      p_part[L.ppart_base + (long long)row * L.nslots + (tile_in_layer - row_begin / kTile)] =
+          make_float4(a0, a1, a2, a3);
   }
 }
 
@@ -195,17 +176,20 @@ psgd_orthonormalise_kernel(const DevLayer* __restrict__ layers, const int* __res
   if (pending != nullptr && threadIdx.x == 0) pending[l] = r;  // lazy mode: this step's residual stays pending
   float* P = p + 4ll * L.p_row;
   const int n = L.rows;
-  if (L.nchunks > 1) {  // rows split into column chunks: P = sum of the chunk partials, in chunk order
-    for (int i = threadIdx.x; i < n; i += blockDim.x) {
-      const float4* pp = p_part + L.ppart_base + (long long)i * L.nchunks;
-      float4 acc = pp[0];
-      for (int ch = 1; ch < L.nchunks; ++ch) { acc.x += pp[ch].x; acc.y += pp[ch].y; acc.z += pp[ch].z; acc.w += pp[ch].w; }
-      P[4 * i] = acc.x;
-      if (r > 1) P[4 * i + 1] = acc.y;
-      if (r > 2) P[4 * i + 2] = acc.z;
-      if (r > 3) P[4 * i + 3] = acc.w;
+  // P[i] = sum, in tile order, of the partial rows the project pass left for the tiles row i touches
+  for (int i = threadIdx.x; i < n; i += blockDim.x) {
+    const int first_tile = (i * L.cols) / kTile, last_tile = (i * L.cols + L.cols - 1) / kTile;
+    const float4* pp = p_part + L.ppart_base + (long long)i * L.nslots;
+    float4 acc = pp[0];
+    for (int sl = 1; sl <= last_tile - first_tile; ++sl) {
+      acc.x += pp[sl].x; acc.y += pp[sl].y; acc.z += pp[sl].z; acc.w += pp[sl].w;
     }
+    P[4 * i] = acc.x;
+    if (r > 1) P[4 * i + 1] = acc.y;
+    if (r > 2) P[4 * i + 2] = acc.z;
+    if (r > 3) P[4 * i + 3] = acc.w;
   }
+  __syncthreads();
   for (int c = 0; c < r; ++c) {
     for (int j = 0; j < c; ++j) {
       double part = 0.0;
@@ -303,59 +287,49 @@ psgd_qreduce_kernel(const DevLayer* __restrict__ layers, const int* __restrict__
   }
 }
 
-// Pass 5.  One block per row slab, a group of `lpr` lanes per row:  A = P^ Q'^T (first r ranks);
+// Pass 5.  One block per tile:  A = P^ Q'^T (first r ranks) at every element of the tile;
 //   WRITE_OUT: out = A;   UPDATE_ERR: err_w -= A for every worker.
 // Eager step: both (r from the level).  Lazy step: WRITE_OUT only.  Flush: UPDATE_ERR only, r = pending rank.
 template <int WB, bool WRITE_OUT, bool UPDATE_ERR>
 __global__ void __launch_bounds__(256)
-psgd_residual_kernel(const DevLayer* __restrict__ layers, const RowItem* __restrict__ items,
-                     float* __restrict__ err, const float* __restrict__ q, const float* __restrict__ p,
-                     const uint8_t* __restrict__ level, const int* __restrict__ pending, float* __restrict__ out,
-                     long long stride, int W, int rank_low, int rank_high) {
-  const RowItem it = items[blockIdx.x];
-  const DevLayer L = layers[it.layer];
-  const int r = pending != nullptr ? pending[it.layer] : (level[it.layer] ? rank_low : rank_high);
+psgd_residual_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict__ tiles, float* __restrict__ err,
+                     const float* __restrict__ q, const float* __restrict__ p, const uint8_t* __restrict__ level,
+                     const int* __restrict__ pending, float* __restrict__ out, long long stride, int W,
+                     int rank_low, int rank_high) {
+  const Tile t = tiles[blockIdx.x];
+  const DevLayer L = layers[t.layer];
+  if (L.kind != ACC_MATRIX) return;
+  const int r = pending != nullptr ? pending[t.layer] : (level[t.layer] ? rank_low : rank_high);
   if (r == 0) return;
-  const float4* __restrict__ Q4 = reinterpret_cast<const float4*>(q) + L.q_row + it.col0;
+  const int m = L.cols;
+  const float4* __restrict__ Q4 = reinterpret_cast<const float4*>(q) + L.q_row;
   const float4* __restrict__ P4 = reinterpret_cast<const float4*>(p) + L.p_row;
-  const int lpr = L.lpr, groups = 32 / lpr;
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int g = lane / lpr, gl = lane - g * lpr;
-  const int row_end = it.row0 + it.nrows;
-  for (int row = it.row0 + warp * groups + g; row < row_end; row += 8 * groups) {
-    const RowGeom rg = row_geom(L, it, row);
-    const float4 pv = __ldg(P4 + row);
-    for (int t = gl; t < rg.nbody4; t += lpr) {
-      const int col = rg.head + 4 * t;
-      const long long idx = rg.start + col;
-      float4 a;
-      a.x = lowrank_entry(pv, __ldg(Q4 + col), r);
-      a.y = lowrank_entry(pv, __ldg(Q4 + col + 1), r);
-      a.z = lowrank_entry(pv, __ldg(Q4 + col + 2), r);
-      a.w = lowrank_entry(pv, __ldg(Q4 + col + 3), r);
-      if (UPDATE_ERR) {
-        for (int w0 = 0; w0 < W; w0 += WB) {
-          float4 m[WB];
+  const long long base = L.offset + t.elem0;
+  const int n4 = t.nelem >> 2;
+  for (int f = threadIdx.x; f < n4; f += blockDim.x) {
+    const long long idx = base + 4 * f;
+    const float4 a = lowrank4(P4, Q4, m, t.elem0 + 4 * f, r);
+    if (UPDATE_ERR) {
+      for (int w0 = 0; w0 < W; w0 += WB) {
+        float4 mw[WB];
 #pragma unroll
-          for (int b = 0; b < WB; ++b)
-            if (w0 + b < W) m[b] = ld_stream4(err + (long long)(w0 + b) * stride + idx);
+        for (int b = 0; b < WB; ++b)
+          if (w0 + b < W) mw[b] = ld_stream4(err + (long long)(w0 + b) * stride + idx);
 #pragma unroll
-          for (int b = 0; b < WB; ++b)
-            if (w0 + b < W)
-              st_stream4(err + (long long)(w0 + b) * stride + idx,
-                         make_float4(m[b].x - a.x, m[b].y - a.y, m[b].z - a.z, m[b].w - a.w));
-        }
+        for (int b = 0; b < WB; ++b)
+          if (w0 + b < W)
+            st_stream4(err + (long long)(w0 + b) * stride + idx,
+                       make_float4(mw[b].x - a.x, mw[b].y - a.y, mw[b].z - a.z, mw[b].w - a.w));
       }
-      if (WRITE_OUT) st_stream4(out + idx, a);
     }
-    if (gl < rg.head + rg.tail) {
-      const int col = gl < rg.head ? gl : rg.head + 4 * rg.nbody4 + (gl - rg.head);
-      const long long idx = rg.start + col;
-      const float a = lowrank_entry(pv, __ldg(Q4 + col), r);
-      if (UPDATE_ERR)
-        for (int w = 0; w < W; ++w) err[(long long)w * stride + idx] -= a;
-      if (WRITE_OUT) out[idx] = a;
-    }
+    if (WRITE_OUT) st_stream4(out + idx, a);
+  }
+  for (int i = 4 * n4 + threadIdx.x; i < t.nelem; i += blockDim.x) {
+    const int e_idx = t.elem0 + i, row = e_idx / m, col = e_idx - row * m;
+    const float a = lowrank_entry(__ldg(P4 + row), __ldg(Q4 + col), r);
+    if (UPDATE_ERR)
+      for (int w = 0; w < W; ++w) err[(long long)w * stride + base + i] -= a;
+    if (WRITE_OUT) out[base + i] = a;
   }
 }
 
@@ -369,27 +343,26 @@ cudaError_t launch_powersgd(acc_ctx* ctx, const float* grads, float* err, float*
                             const uint8_t* level, float* out, float* delta, cudaStream_t s) {
   const Plan& pl = ctx->plan;
   const acc_config& c = ctx->cfg;
-  const int n_items = (int)pl.row_items.size();
-  const int n_vec = (int)pl.vec_tiles.size();
+  const int nt = (int)pl.tiles.size();
   const float inv_w = 1.0f / (float)c.n_workers;
   const bool lazy = (c.flags & ACC_FLAG_LAZY_RESIDUAL) != 0;
-  if (n_items + n_vec > 0) {
+  {
     PhaseTimer pt(ctx, PH_PSGD_PROJECT, s);
     if (lazy)
-      psgd_project_kernel<4, true><<<n_items + n_vec, 256, 0, s>>>(
-          ctx->d_layers, ctx->d_row_items, n_items, ctx->d_tiles, ctx->d_vec_tiles, grads, err, q, p_hat, ctx->d_ppart,
-          level, ctx->d_pending, out, delta, c.worker_stride, c.n_workers, c.decider, inv_w, c.rank_low, c.rank_high);
+      psgd_project_kernel<4, true><<<nt, 256, 0, s>>>(ctx->d_layers, ctx->d_tiles, grads, err, q, p_hat, ctx->d_ppart,
+                                                      level, ctx->d_pending, out, delta, c.worker_stride,
+                                                      c.n_workers, c.decider, inv_w);
     else
-      psgd_project_kernel<4, false><<<n_items + n_vec, 256, 0, s>>>(
-          ctx->d_layers, ctx->d_row_items, n_items, ctx->d_tiles, ctx->d_vec_tiles, grads, err, q, p_hat, ctx->d_ppart,
-          level, nullptr, out, delta, c.worker_stride, c.n_workers, c.decider, inv_w, c.rank_low, c.rank_high);
+      psgd_project_kernel<4, false><<<nt, 256, 0, s>>>(ctx->d_layers, ctx->d_tiles, grads, err, q, p_hat,
+                                                       ctx->d_ppart, level, nullptr, out, delta, c.worker_stride,
+                                                       c.n_workers, c.decider, inv_w);
   }
   if (pl.n_mat > 0) {
     {
       PhaseTimer pt(ctx, PH_PSGD_ORTHO, s);
-      psgd_orthonormalise_kernel<<<pl.n_mat, 1024, 0, s>>>(ctx->d_layers, ctx->d_mat_layers, p_hat, ctx->d_ppart, level,
-                                                          lazy ? ctx->d_pending : nullptr, c.rank_low, c.rank_high,
-                                                          c.gs_eps);
+      psgd_orthonormalise_kernel<<<pl.n_mat, 1024, 0, s>>>(ctx->d_layers, ctx->d_mat_layers, p_hat, ctx->d_ppart,
+                                                          level, lazy ? ctx->d_pending : nullptr, c.rank_low,
+                                                          c.rank_high, c.gs_eps);
     }
     {
       PhaseTimer pt(ctx, PH_PSGD_QPARTIAL, s);
@@ -406,13 +379,13 @@ cudaError_t launch_powersgd(acc_ctx* ctx, const float* grads, float* err, float*
     {
       PhaseTimer pt(ctx, PH_PSGD_RESIDUAL, s);
       if (lazy)
-        psgd_residual_kernel<4, true, false><<<n_items, 256, 0, s>>>(
-            ctx->d_layers, ctx->d_row_items, err, q, p_hat, level, nullptr, out, c.worker_stride, c.n_workers,
-            c.rank_low, c.rank_high);
+        psgd_residual_kernel<4, true, false><<<nt, 256, 0, s>>>(ctx->d_layers, ctx->d_tiles, err, q, p_hat, level,
+                                                                nullptr, out, c.worker_stride, c.n_workers,
+                                                                c.rank_low, c.rank_high);
       else
-        psgd_residual_kernel<4, true, true><<<n_items, 256, 0, s>>>(
-            ctx->d_layers, ctx->d_row_items, err, q, p_hat, level, nullptr, out, c.worker_stride, c.n_workers,
-            c.rank_low, c.rank_high);
+        psgd_residual_kernel<4, true, true><<<nt, 256, 0, s>>>(ctx->d_layers, ctx->d_tiles, err, q, p_hat, level,
+                                                               nullptr, out, c.worker_stride, c.n_workers,
+                                                               c.rank_low, c.rank_high);
     }
   }
   return cudaGetLastError();
@@ -421,13 +394,13 @@ cudaError_t launch_powersgd(acc_ctx* ctx, const float* grads, float* err, float*
 cudaError_t launch_powersgd_flush(acc_ctx* ctx, float* err, const float* q, const float* p_hat, cudaStream_t s) {
   const Plan& pl = ctx->plan;
   const acc_config& c = ctx->cfg;
-  const int n_items = (int)pl.row_items.size();
-  if (n_items > 0) {
+  const int nt = (int)pl.tiles.size();
+  if (pl.n_mat > 0) {
     {
       PhaseTimer pt(ctx, PH_PSGD_FLUSH, s);
-      psgd_residual_kernel<4, false, true><<<n_items, 256, 0, s>>>(
-          ctx->d_layers, ctx->d_row_items, err, q, p_hat, nullptr, ctx->d_pending, nullptr, c.worker_stride,
-          c.n_workers, c.rank_low, c.rank_high);
+      psgd_residual_kernel<4, false, true><<<nt, 256, 0, s>>>(ctx->d_layers, ctx->d_tiles, err, q, p_hat, nullptr,
+                                                              ctx->d_pending, nullptr, c.worker_stride, c.n_workers,
+                                                              c.rank_low, c.rank_high);
     }
     ctx->last_launches += 1;
     psgd_clear_pending_kernel<<<(c.n_layers + 127) / 128, 128, 0, s>>>(ctx->d_pending, c.n_layers);
