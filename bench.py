@@ -292,7 +292,8 @@ def main():
     dom_avg_ms = prof[dom][0] / prof[dom][1]
     achieved = dom_alg / (dom_avg_ms * 1e-3) / 1e9
     roofline = {"bound": "hbm", "kernel": dom, "achieved": round(achieved, 1), "peak": peak, "unit": "GB/s",
-                "frac": round(achieved / peak, 4), "peak_source": peak_src, "traffic": TRAFFIC.get((args.config, dom)),
+                "frac": round(achieved / peak, 4), "peak_source": peak_src, "traffic": (TRAFFIC_PER_UNIT[dom] * units if dom in TRAFFIC_PER_UNIT else None),
+                "traffic_source": TRAFFIC_SOURCE.get(dom),
                 "alg_bytes_per_launch": dom_alg,
                 "step_frac_of_12B": round(n_comp * 12.0 * units / (ms_per_step * 1e-3) / 1e9 / peak, 4)}
 
@@ -352,9 +353,12 @@ def main():
         dist.destroy_process_group()
 
 
-# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per launch of the dominant kernel, from the
-# ncu captures summarised under profiles/ ; keyed by (config, kernel).
-TRAFFIC = {}
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per MATRIX parameter-worker, from the ncu captures
+# summarised under profiles/; a launch's traffic is this figure times the units it processes (the kernels
+# stream every element once, so traffic grows in proportion).
+TRAFFIC_PER_UNIT = {"psgd_project_kernel": 13.15, "topk_ef_hist1_kernel": 12.92}
+TRAFFIC_SOURCE = {"psgd_project_kernel": "ncu on config 4 (profiles/psgd_project_kernel_config4_traffic.md), scaled by units",
+                  "topk_ef_hist1_kernel": "ncu on config 3 (profiles/topk_kernels_config3_resnet18.md), scaled by units"}
 
 if __name__ == "__main__":
     main()
