@@ -49,15 +49,19 @@ topk_ef_hist1_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict
                      unsigned* __restrict__ seg_cand, unsigned* __restrict__ seg_flag, unsigned* __restrict__ cand,
                      int2* __restrict__ tile_cand, long long cand_total, int2* __restrict__ tile_cnt) {
   __shared__ unsigned h[kBins1];
-  __shared__ unsigned s_buf[kPredTileCap];
-  __shared__ unsigned s_cnt, s_start;
-  __shared__ int s_above;
+  // three staging buffers for the collected keys: a tile's keys are copied out while the next tile is
+  // being processed and the buffer is reused two tiles later, so one barrier per tile is enough
+  __shared__ unsigned s_buf[3][kPredTileCap];
+  __shared__ unsigned s_cnt[3], s_n[3];
+  __shared__ int s_above[3];
+  __shared__ long long s_dst[3];
   for (int b = threadIdx.x; b < kBins1; b += blockDim.x) h[b] = 0;
-  if (threadIdx.x == 0) { s_cnt = 0; s_above = 0; }
+  if (threadIdx.x < 3) { s_cnt[threadIdx.x] = 0; s_above[threadIdx.x] = 0; s_n[threadIdx.x] = 0; }
   __syncthreads();
   const long long V = (long long)W * n_tiles;
   const long long v0 = V * blockIdx.x / gridDim.x, v1 = V * (blockIdx.x + 1) / gridDim.x;
   int cur = -1;
+  int cb = 0, pend = -1;  // staging buffer in use; buffer waiting to be copied out
   bool collect = false;
   unsigned blo = 1, bhi = 0;
   for (long long v = v0; v < v1; ++v) {
@@ -83,6 +87,8 @@ topk_ef_hist1_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict
     const bool acc_delta = delta != nullptr && w == decider;
     const int n4 = t.nelem >> 2;
     const unsigned span = bhi - blo;
+    unsigned* buf = s_buf[cb];
+    unsigned* cnt = &s_cnt[cb];
     int above = 0;
 #pragma unroll 4
     for (int i = threadIdx.x; i < n4; i += blockDim.x) {
@@ -98,8 +104,8 @@ topk_ef_hist1_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict
         if (collect) {
           above += bin > bhi;
           if (bin - blo <= span) {
-            const unsigned slot = atomicAdd(&s_cnt, 1u);
-            if (slot < (unsigned)kPredTileCap) s_buf[slot] = k[q];
+            const unsigned slot = atomicAdd(cnt, 1u);
+            if (slot < (unsigned)kPredTileCap) buf[slot] = k[q];
           }
         }
       }
@@ -118,18 +124,25 @@ topk_ef_hist1_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict
       if (collect) {
         above += bin > bhi;
         if (bin - blo <= span) {
-          const unsigned slot = atomicAdd(&s_cnt, 1u);
-          if (slot < (unsigned)kPredTileCap) s_buf[slot] = kk;
+          const unsigned slot = atomicAdd(cnt, 1u);
+          if (slot < (unsigned)kPredTileCap) buf[slot] = kk;
         }
       }
       if (acc_delta) delta[base + i] += gv;
     }
     if (collect) {  // hand the tile's collected keys over to the segment's list
       above = __reduce_add_sync(0xffffffffu, above);
-      if ((threadIdx.x & 31) == 0 && above) atomicAdd(&s_above, above);
+      if ((threadIdx.x & 31) == 0 && above) atomicAdd(&s_above[cb], above);
+      const int nb = cb == 2 ? 0 : cb + 1;
+      if (threadIdx.x == 0) { s_cnt[nb] = 0; s_above[nb] = 0; }  // free since the barrier of the previous tile
       __syncthreads();
+      if (pend >= 0) {  // copy out the previous tile's keys (its range was published before this barrier)
+        unsigned* dst = cand + s_dst[pend];
+        const unsigned n = s_n[pend];
+        for (unsigned i = threadIdx.x; i < n; i += blockDim.x) dst[i] = s_buf[pend][i];
+      }
       if (threadIdx.x == 0) {
-        unsigned n = s_cnt, start = 0;
+        unsigned n = s_cnt[cb], start = 0;
         if (n > (unsigned)kPredTileCap) {
           atomicOr(&seg_flag[seg], 1u);
           n = 0;
@@ -137,19 +150,21 @@ topk_ef_hist1_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict
           start = atomicAdd(&seg_cand[seg], n);
           if (start + n > (unsigned)L.cand_cap) { atomicOr(&seg_flag[seg], 1u); n = 0; }
         }
-        s_start = start;
-        s_cnt = n;
+        s_n[cb] = n;
+        s_dst[cb] = (long long)w * cand_total + L.cand_base + start;
         tile_cand[(long long)w * n_tiles + ti] = make_int2((int)start, (int)n);
-        tile_cnt[(long long)w * n_tiles + ti].x = s_above;
+        tile_cnt[(long long)w * n_tiles + ti].x = s_above[cb];
       }
-      __syncthreads();
-      unsigned* dst = cand + (long long)w * cand_total + L.cand_base + s_start;
-      for (unsigned i = threadIdx.x; i < s_cnt; i += blockDim.x) dst[i] = s_buf[i];
-      __syncthreads();
-      if (threadIdx.x == 0) { s_cnt = 0; s_above = 0; }
+      pend = cb;
+      cb = nb;
     }
   }
   __syncthreads();
+  if (pend >= 0) {
+    unsigned* dst = cand + s_dst[pend];
+    const unsigned n = s_n[pend];
+    for (unsigned i = threadIdx.x; i < n; i += blockDim.x) dst[i] = s_buf[pend][i];
+  }
   if (cur >= 0)
     for (int b = threadIdx.x; b < kBins1; b += blockDim.x) {
       const unsigned c = h[b];
