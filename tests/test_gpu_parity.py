@@ -305,3 +305,26 @@ def test_powersgd_lazy_residual_is_bit_identical_to_eager(W, rank_low, rank_high
         assert torch.equal(state[0][name], state[1][name]), name
     with pytest.raises(binding.AccError):
         eager.acc_powersgd_flush(state[0]["err"], state[0]["q"], state[0]["p"])
+
+
+def test_topk_threshold_prediction_hits_and_misses():
+    """The step predicts the threshold's bucket from the previous step at the same level.  Sequence of
+    gradient scales that makes the prediction hold (same scale), miss upwards (x10: exact list path),
+    miss downwards (x0.1: the histogram below the predicted band was not counted, redo path) and switch
+    level in between; every step must still match the oracle bit for bit."""
+    table = _table_mixed()
+    W = 2
+    ctx = binding.Context(table, W)
+    vals, idx, counts = ctx.new_topk_buffers()
+    out = torch.zeros(table.stride, device="cuda")
+    base, _ = _random_inputs(table, W, 77, err_scale=0.0)
+    steps = [(1.0, 1), (1.0, 1), (0.1, 1), (0.1, 1), (10.0, 1), (10.0, 0), (10.0, 0), (0.5, 0), (0.5, 1), (0.5, 1)]
+    for i, (scale, lv) in enumerate(steps):
+        g = torch.Generator(device="cuda").manual_seed(500 + i)
+        grads = (base + 0.05 * torch.randn(base.shape, generator=g, device="cuda") * (base != 0)) * scale
+        err = torch.zeros_like(grads)
+        level = torch.full((table.n_layers,), lv, dtype=torch.uint8, device="cuda")
+        e0 = err.clone()
+        ctx.acc_topk_step(grads, err, level, vals, idx, counts, out)
+        torch.cuda.synchronize()
+        H.check_topk_against_oracle(ctx, table, grads, e0, level, vals, idx, counts, out, err, 1000, 100)
