@@ -44,6 +44,7 @@ extern "C" {
 #define ACC_EWORKSPACE 3  /* workspace missing or too small                        */
 #define ACC_ECUDA 4       /* a CUDA runtime call or kernel launch reported an error */
 #define ACC_ETOOBIG 5     /* size beyond the fixed capacity of acc_sumsq_static    */
+#define ACC_ETIMEOUT 6    /* device side: a bounded wait on an asynchronous copy gave up (acc_device_status) */
 
 #define ACC_MATRIX 0
 #define ACC_VECTOR 1
@@ -161,6 +162,13 @@ int acc_powersgd_flush(acc_ctx* ctx, float* err, const float* q, const float* p_
  * idx [W*capacity] int32, counts [W*L] int32 (see acc_topk_layout).                                */
 int acc_topk_step(acc_ctx* ctx, const float* grads, float* err, const uint8_t* level, float* vals,
                   int32_t* idx, int32_t* counts, float* out, float* delta, void* stream);
+
+/* Device-side condition of the kernels launched so far on this context (no counterpart in the paper).
+ * The pipelined kernels wait for their asynchronous shared-memory copies with a bounded number of polls;
+ * should a wait ever give up, the block stores ACC_ETIMEOUT in a status word and returns instead of
+ * hanging, and the results of that call are undefined.  This call copies the status word to *status
+ * (HOST pointer; 0 = no such event) and blocks until the device has finished the work queued before it. */
+int acc_device_status(acc_ctx* ctx, int32_t* status);
 
 /* Floats one iteration communicates at the given HOST level array, following the "Data Sent"
  * accounting of Tables 1-4: PowerSGD r*(rows+cols) per MATRIX layer, TopK 2*k*W per MATRIX layer

@@ -43,7 +43,7 @@ class acc_config(C.Structure):
 EXPORTS = ["acc_workspace_bytes", "acc_create", "acc_destroy", "acc_factor_layout", "acc_topk_layout",
            "acc_error_feedback", "acc_layer_norms", "acc_detect_regime", "acc_powersgd_step", "acc_topk_step",
            "acc_floats_sent", "acc_last_launch_count", "acc_strerror", "acc_profile_enable", "acc_profile_read",
-           "acc_profile_kernel_count", "acc_profile_kernel_name", "acc_sumsq_static", "acc_powersgd_flush"]
+           "acc_profile_kernel_count", "acc_profile_kernel_name", "acc_sumsq_static", "acc_powersgd_flush", "acc_device_status"]
 
 _lib = None
 
@@ -83,6 +83,7 @@ def lib() -> C.CDLL:
     L.acc_profile_kernel_name.restype = C.c_char_p
     L.acc_sumsq_static.argtypes = [vp, i64, vp, vp]
     L.acc_powersgd_flush.argtypes = [vp, vp, vp, vp, vp]
+    L.acc_device_status.argtypes = [vp, C.POINTER(i32)]
     for name in EXPORTS:
         if name not in ("acc_floats_sent", "acc_last_launch_count", "acc_strerror", "acc_profile_kernel_count",
                         "acc_profile_kernel_name"):
@@ -225,6 +226,12 @@ class Context:
         ms, cnt = (C.c_double * n)(), (C.c_int32 * n)()
         self._check(lib().acc_profile_read(self._h, ms, cnt, n), "acc_profile_read")
         return {lib().acc_profile_kernel_name(i).decode(): (float(ms[i]), int(cnt[i])) for i in range(n) if cnt[i]}
+
+    def acc_device_status(self) -> int:
+        """Device-side status word (0 = fine); waits for the queued work of this device."""
+        v = C.c_int32(0)
+        self._check(lib().acc_device_status(self._h, C.byref(v)), "acc_device_status")
+        return int(v.value)
 
     def last_launch_count(self) -> int:
         return int(lib().acc_last_launch_count(self._h))

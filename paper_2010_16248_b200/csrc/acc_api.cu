@@ -63,6 +63,7 @@ static int make_plan(const acc_config* cfg, Plan& p) {
     for (long long e = 0; e < size; e += kTile) {
       Tile t{l, (int)e, (int)std::min<long long>(kTile, size - e)};
       if (d.kind == ACC_VECTOR) p.vec_tiles.push_back((int)p.tiles.size());
+      else p.mat_tiles.push_back((int)p.tiles.size());
       p.tiles.push_back(t);
     }
     o.ntiles = (int)p.tiles.size() - o.tile0;
@@ -99,6 +100,8 @@ static int make_plan(const acc_config* cfg, Plan& p) {
   p.o_tiles = take(sizeof(Tile) * nt);
   p.o_mat_layers = take(sizeof(int) * std::max<size_t>(1, p.mat_layers.size()));
   p.o_vec_tiles = take(sizeof(int) * std::max<size_t>(1, p.vec_tiles.size()));
+  p.o_mat_tiles = take(sizeof(int) * std::max<size_t>(1, p.mat_tiles.size()));
+  p.o_status = take(sizeof(int) * 64);
   p.o_part = take(sizeof(float4) * std::max<long long>(1, p.part_f4));
   p.o_ppart = take(sizeof(float4) * std::max<long long>(1, p.ppart_f4));
   p.o_pending = take(sizeof(int) * L);
@@ -158,6 +161,8 @@ int acc_create(const acc_config* cfg, void* workspace, size_t workspace_bytes, a
   ctx->d_tiles = reinterpret_cast<Tile*>(ws + p.o_tiles);
   ctx->d_mat_layers = reinterpret_cast<int*>(ws + p.o_mat_layers);
   ctx->d_vec_tiles = reinterpret_cast<int*>(ws + p.o_vec_tiles);
+  ctx->d_mat_tiles = reinterpret_cast<int*>(ws + p.o_mat_tiles);
+  ctx->d_status = reinterpret_cast<int*>(ws + p.o_status);
   ctx->d_part = reinterpret_cast<float4*>(ws + p.o_part);
   ctx->d_ppart = reinterpret_cast<float4*>(ws + p.o_ppart);
   ctx->d_pending = reinterpret_cast<int*>(ws + p.o_pending);
@@ -185,6 +190,8 @@ int acc_create(const acc_config* cfg, void* workspace, size_t workspace_bytes, a
   up(ctx->d_tiles, p.tiles.data(), sizeof(Tile) * p.tiles.size());
   up(ctx->d_mat_layers, p.mat_layers.data(), sizeof(int) * p.mat_layers.size());
   up(ctx->d_vec_tiles, p.vec_tiles.data(), sizeof(int) * p.vec_tiles.size());
+  up(ctx->d_mat_tiles, p.mat_tiles.data(), sizeof(int) * p.mat_tiles.size());
+  if (e == cudaSuccess) e = cudaMemset(ctx->d_status, 0, sizeof(int) * 64);
   if (e == cudaSuccess) e = cudaMemset(ctx->d_pending, 0, sizeof(int) * cfg->n_layers);
   if (e == cudaSuccess) e = cudaMemset(ctx->d_pred, 0xff, sizeof(unsigned) * 2 * seg);  // no prediction yet
   int dev = 0;
@@ -333,6 +340,14 @@ const char* acc_profile_kernel_name(int32_t i) {
   return (i >= 0 && i < PH_COUNT) ? names[i] : "";
 }
 
+int acc_device_status(acc_ctx* ctx, int32_t* status) {
+  if (!ctx || !status) return ACC_EINVAL;
+  int v = 0;
+  if (cudaMemcpy(&v, ctx->d_status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return ACC_ECUDA;
+  *status = v;
+  return ACC_OK;
+}
+
 int32_t acc_last_launch_count(const acc_ctx* ctx) { return ctx ? ctx->last_launches : -1; }
 
 const char* acc_strerror(int status) {
@@ -342,6 +357,7 @@ const char* acc_strerror(int status) {
     case ACC_EALIGN: return "pointer, offset or stride not 16-byte aligned";
     case ACC_EWORKSPACE: return "workspace missing or too small";
     case ACC_ECUDA: return "CUDA runtime or launch error";
+    case ACC_ETIMEOUT: return "a bounded device-side wait gave up (asynchronous copy did not complete)";
     case ACC_ETOOBIG: return "size exceeds the capacity of the built-in scratch array (ACC_STATIC_NORM_MAX_ELEMS)";
     default: return "unknown status";
   }

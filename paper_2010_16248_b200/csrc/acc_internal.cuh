@@ -64,10 +64,11 @@ struct Plan {
   std::vector<Tile> tiles;
   std::vector<int> mat_layers;   // layer index of each MATRIX layer
   std::vector<int> vec_tiles;    // tile indices that belong to VECTOR layers
+  std::vector<int> mat_tiles;    // tile indices that belong to MATRIX layers, in order
   long long q_rows = 0, p_rows = 0, capacity = 0, part_f4 = 0, cand_total = 0, ppart_f4 = 0;
   int n_mat = 0;
   // workspace offsets (bytes)
-  size_t o_layers = 0, o_col_items = 0, o_tiles = 0, o_mat_layers = 0, o_vec_tiles = 0,
+  size_t o_layers = 0, o_col_items = 0, o_tiles = 0, o_mat_layers = 0, o_vec_tiles = 0, o_mat_tiles = 0, o_status = 0,
          o_part = 0, o_ppart = 0, o_pending = 0, o_norm_part = 0, o_hist = 0, o_sel = 0, o_pred = 0, o_cand = 0, o_tile_cand = 0, o_tile_cnt = 0, o_tile_h3 = 0, o_tile_pre = 0,
          hist_bytes = 0, total = 0;
 };
@@ -90,6 +91,8 @@ struct acc_ctx {
   acc::Tile* d_tiles = nullptr;
   int* d_mat_layers = nullptr;
   int* d_vec_tiles = nullptr;
+  int* d_mat_tiles = nullptr;
+  int* d_status = nullptr;           // device-side error flag (0 = none), see acc_device_status
   float4* d_part = nullptr;
   float4* d_ppart = nullptr;         // partial rows of P, one slot per tile a row touches
   int* d_pending = nullptr;          // lazy PowerSGD: rank of the residual not yet applied to err, per layer

@@ -9,6 +9,9 @@
 // every access is a fully coalesced, 16-byte aligned float4 whatever the row length, and all blocks carry
 // the same load.  Row structure only enters through the factors: element i of a layer sits in row i / m,
 // column i % m, and the rows a tile cuts are reduced from shared memory afterwards.
+#include <cstdlib>
+
+#include "acc_async.cuh"
 #include "acc_internal.cuh"
 
 namespace acc {
@@ -148,6 +151,163 @@ psgd_project_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict_
     if (lane == 0)
       p_part[L.ppart_base + (long long)row * L.nslots + (tile_in_layer - row_begin / kTile)] =
           make_float4(a0, a1, a2, a3);
+  }
+}
+
+// Pass 1, pipelined.  Persistent blocks (one per SM, 512 threads), each with a contiguous range of MATRIX
+// tiles.  The sequence of (tile, worker) stages of a block is streamed through two shared-memory stage
+// buffers by bulk asynchronous copies: while the threads consume stage i (g_w and e_w of one tile,
+// 2 x 32 KB), the copy of stage i+1 is in flight and, once everybody has left stage i's buffer, stage i+2
+// is issued into it -- 64-128 KB per SM are in flight at all times without costing registers.
+// The arithmetic is that of the direct kernel (same operations in the same order).
+constexpr int kPipeThreads = 512;
+constexpr int kPipePos = kTile / 4 / kPipeThreads;  // float4 positions per thread and tile
+constexpr size_t kPipeSmemBytes = sizeof(float) * kTile * 5 + 64;
+
+template <bool LAZY>
+__global__ void __launch_bounds__(kPipeThreads, 1)
+psgd_project_pipe_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict__ tiles,
+                         const int* __restrict__ mat_tiles, int n_mat_tiles, const int* __restrict__ vec_tiles,
+                         int n_vec_tiles, const float* __restrict__ grads, float* __restrict__ err,
+                         const float* __restrict__ q, const float* __restrict__ p, float4* __restrict__ p_part,
+                         const int* __restrict__ pending, float* __restrict__ out, float* __restrict__ delta,
+                         long long stride, int W, int decider, float inv_w, int* __restrict__ status) {
+  extern __shared__ __align__(128) unsigned char smem_raw[];
+  float* stage = reinterpret_cast<float*>(smem_raw);                  // [2 buffers][g, e][kTile]
+  float* s_mbar = stage + 4 * kTile;                                  // [kTile]
+  uint64_t* bars = reinterpret_cast<uint64_t*>(s_mbar + kTile);       // [2]
+  for (int i = blockIdx.x; i < n_vec_tiles; i += gridDim.x) {
+    const Tile t = tiles[vec_tiles[i]];
+    vector_mean_tile(t, layers[t.layer], grads, out, delta, stride, W, decider, inv_w);
+  }
+  const int t0 = (int)((long long)n_mat_tiles * blockIdx.x / gridDim.x);
+  const int t1 = (int)((long long)n_mat_tiles * (blockIdx.x + 1) / gridDim.x);
+  const int n_stages = (t1 - t0) * W;
+  if (n_stages == 0) return;
+  if (threadIdx.x == 0) {
+    mbar_init(&bars[0], 1);
+    mbar_init(&bars[1], 1);
+    fence_mbar_init();
+  }
+  __syncthreads();
+  auto issue = [&](int it) {  // called by thread 0 only
+    const int ti = it / W, w = it - ti * W;
+    const Tile t = tiles[mat_tiles[t0 + ti]];
+    const long long base = (long long)w * stride + layers[t.layer].offset + t.elem0;
+    const unsigned bytes = (unsigned)((t.nelem + 3) / 4) * 16u;  // a ragged tile reads into the layer's padding
+    const int buf = it & 1;
+    mbar_arrive_expect_tx(&bars[buf], 2 * bytes);
+    bulk_copy_g2s(stage + (2 * buf) * kTile, grads + base, bytes, &bars[buf]);
+    bulk_copy_g2s(stage + (2 * buf + 1) * kTile, err + base, bytes, &bars[buf]);
+  };
+  if (threadIdx.x == 0) {
+    issue(0);
+    if (n_stages > 1) issue(1);
+  }
+  Tile t = tiles[mat_tiles[t0]];
+  DevLayer L = layers[t.layer];
+  float4 corr[kPipePos], mb[kPipePos];
+  int rp = 0;
+  for (int it = 0; it < n_stages; ++it) {
+    const int ti = it / W, w = it - ti * W;
+    const int buf = it & 1;
+    if (w == 0) {  // new tile: factors of the pending residual at this thread's positions
+      t = tiles[mat_tiles[t0 + ti]];
+      L = layers[t.layer];
+      rp = LAZY ? pending[t.layer] : 0;
+      const float4* Q4 = reinterpret_cast<const float4*>(q) + L.q_row;
+      const float4* P4 = reinterpret_cast<const float4*>(p) + L.p_row;
+#pragma unroll
+      for (int k = 0; k < kPipePos; ++k) {
+        const int e0 = 4 * (k * kPipeThreads + (int)threadIdx.x);
+        mb[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+        corr[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (LAZY && rp > 0 && e0 + 3 < t.nelem) corr[k] = lowrank4(P4, Q4, L.cols, t.elem0 + e0, rp);
+        else if (LAZY && rp > 0 && e0 < t.nelem) {  // ragged last float4 of a layer
+          float c[4] = {0.f, 0.f, 0.f, 0.f};
+          for (int e = 0; e0 + e < t.nelem; ++e) {
+            const int ei = t.elem0 + e0 + e, row = ei / L.cols;
+            c[e] = lowrank_entry(__ldg(P4 + row), __ldg(Q4 + (ei - row * L.cols)), rp);
+          }
+          corr[k] = make_float4(c[0], c[1], c[2], c[3]);
+        }
+      }
+    }
+    const bool arrived = __syncthreads_and(mbar_wait_bounded(&bars[buf], (unsigned)(it >> 1) & 1u));
+    if (!arrived) {  // a copy never completed: report and leave (uniformly for the whole block)
+      if (threadIdx.x == 0) atomicExch(status, ACC_ETIMEOUT);
+      return;
+    }
+    const float* sg = stage + (2 * buf) * kTile;
+    const float* se = sg + kTile;
+    const long long gbase = (long long)w * stride + L.offset + t.elem0;
+    const bool acc_delta = delta != nullptr && w == decider;
+#pragma unroll
+    for (int k = 0; k < kPipePos; ++k) {
+      const int e0 = 4 * (k * kPipeThreads + (int)threadIdx.x);
+      if (e0 >= t.nelem) continue;
+      const float4 gv = *reinterpret_cast<const float4*>(sg + e0);
+      float4 e = *reinterpret_cast<const float4*>(se + e0);
+      if (LAZY && rp > 0) { e.x -= corr[k].x; e.y -= corr[k].y; e.z -= corr[k].z; e.w -= corr[k].w; }
+      const float4 mw = make_float4(gv.x + e.x, gv.y + e.y, gv.z + e.z, gv.w + e.w);
+      mb[k].x += mw.x; mb[k].y += mw.y; mb[k].z += mw.z; mb[k].w += mw.w;
+      if (e0 + 3 < t.nelem) {
+        st_stream4(err + gbase + e0, mw);
+        if (acc_delta) {
+          float4 d = *reinterpret_cast<const float4*>(delta + L.offset + t.elem0 + e0);
+          d.x += gv.x; d.y += gv.y; d.z += gv.z; d.w += gv.w;
+          *reinterpret_cast<float4*>(delta + L.offset + t.elem0 + e0) = d;
+        }
+      } else {
+        const float mm[4] = {mw.x, mw.y, mw.z, mw.w}, gg[4] = {gv.x, gv.y, gv.z, gv.w};
+        for (int e2 = 0; e0 + e2 < t.nelem; ++e2) {
+          err[gbase + e0 + e2] = mm[e2];
+          if (acc_delta) delta[L.offset + t.elem0 + e0 + e2] += gg[e2];
+        }
+      }
+    }
+    __syncthreads();  // everybody has left this stage buffer
+    if (threadIdx.x == 0 && it + 2 < n_stages) {
+      fence_proxy_async_smem();
+      issue(it + 2);
+    }
+    if (w == W - 1) {  // tile complete: mean matrix out, partial rows of P from shared memory
+      const long long obase = L.offset + t.elem0;
+#pragma unroll
+      for (int k = 0; k < kPipePos; ++k) {
+        const int e0 = 4 * (k * kPipeThreads + (int)threadIdx.x);
+        if (e0 >= t.nelem) continue;
+        const float4 v = make_float4(mb[k].x * inv_w, mb[k].y * inv_w, mb[k].z * inv_w, mb[k].w * inv_w);
+        *reinterpret_cast<float4*>(s_mbar + e0) = v;
+        if (e0 + 3 < t.nelem) {
+          *reinterpret_cast<float4*>(out + obase + e0) = v;
+        } else {
+          const float vv[4] = {v.x, v.y, v.z, v.w};
+          for (int e2 = 0; e0 + e2 < t.nelem; ++e2) out[obase + e0 + e2] = vv[e2];
+        }
+      }
+      __syncthreads();
+      const int m = L.cols;
+      const float4* Q4 = reinterpret_cast<const float4*>(q) + L.q_row;
+      const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+      const int first_row = t.elem0 / m, last_row = (t.elem0 + t.nelem - 1) / m;
+      const int tile_in_layer = t.elem0 / kTile;
+      for (int row = first_row + warp; row <= last_row; row += kPipeThreads / 32) {
+        const int row_begin = row * m;
+        const int lo = max(row_begin, t.elem0) - t.elem0, hi = min(row_begin + m, t.elem0 + t.nelem) - t.elem0;
+        const float4* qr = Q4 + (t.elem0 + lo - row_begin);
+        float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+        for (int i = lo + lane; i < hi; i += 32) {
+          const float v = s_mbar[i];
+          const float4 qv = __ldg(qr + (i - lo));
+          a0 = fmaf(v, qv.x, a0); a1 = fmaf(v, qv.y, a1); a2 = fmaf(v, qv.z, a2); a3 = fmaf(v, qv.w, a3);
+        }
+        a0 = warp_sum(a0); a1 = warp_sum(a1); a2 = warp_sum(a2); a3 = warp_sum(a3);
+        if (lane == 0)
+          p_part[L.ppart_base + (long long)row * L.nslots + (tile_in_layer - row_begin / kTile)] =
+              make_float4(a0, a1, a2, a3);
+      }
+    }
   }
 }
 
@@ -346,7 +506,23 @@ cudaError_t launch_powersgd(acc_ctx* ctx, const float* grads, float* err, float*
   const int nt = (int)pl.tiles.size();
   const float inv_w = 1.0f / (float)c.n_workers;
   const bool lazy = (c.flags & ACC_FLAG_LAZY_RESIDUAL) != 0;
-  {
+  static const bool use_pipe = !(getenv("ACC_NOPIPE") && atoi(getenv("ACC_NOPIPE")));
+  if (use_pipe && pl.n_mat > 0) {
+    PhaseTimer pt(ctx, PH_PSGD_PROJECT, s);
+    const int n_mt = (int)pl.mat_tiles.size(), n_vt = (int)pl.vec_tiles.size();
+    const int grid = n_mt < ctx->sm_count ? n_mt : ctx->sm_count;
+    if (lazy) {
+      cudaFuncSetAttribute(psgd_project_pipe_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPipeSmemBytes);
+      psgd_project_pipe_kernel<true><<<grid, kPipeThreads, kPipeSmemBytes, s>>>(
+          ctx->d_layers, ctx->d_tiles, ctx->d_mat_tiles, n_mt, ctx->d_vec_tiles, n_vt, grads, err, q, p_hat,
+          ctx->d_ppart, ctx->d_pending, out, delta, c.worker_stride, c.n_workers, c.decider, inv_w, ctx->d_status);
+    } else {
+      cudaFuncSetAttribute(psgd_project_pipe_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPipeSmemBytes);
+      psgd_project_pipe_kernel<false><<<grid, kPipeThreads, kPipeSmemBytes, s>>>(
+          ctx->d_layers, ctx->d_tiles, ctx->d_mat_tiles, n_mt, ctx->d_vec_tiles, n_vt, grads, err, q, p_hat,
+          ctx->d_ppart, nullptr, out, delta, c.worker_stride, c.n_workers, c.decider, inv_w, ctx->d_status);
+    }
+  } else {
     PhaseTimer pt(ctx, PH_PSGD_PROJECT, s);
     if (lazy)
       psgd_project_kernel<4, true><<<nt, 256, 0, s>>>(ctx->d_layers, ctx->d_tiles, grads, err, q, p_hat, ctx->d_ppart,
