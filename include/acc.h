@@ -52,6 +52,11 @@ extern "C" {
 
 /* acc_config.flags */
 #define ACC_FLAG_LAZY_RESIDUAL 1 /* PowerSGD keeps M_w in err and applies -A on the next load (see acc_powersgd_step) */
+/* The first PowerSGD pass exists as a direct kernel and as a persistent kernel fed by bulk asynchronous
+ * copies; both compute the same values.  By default the library picks by problem size (the pipelined one
+ * needs a long queue of tiles per SM to pay off).  These two flags force the choice (tests, tuning). */
+#define ACC_FLAG_PIPELINE_ALWAYS 2
+#define ACC_FLAG_PIPELINE_NEVER 4
 
 #define ACC_COMPRESSOR_POWERSGD 0
 #define ACC_COMPRESSOR_TOPK 1
@@ -75,7 +80,7 @@ typedef struct {
   float eta;                    /* detection threshold of Algorithm 1 (the paper uses 0.5)       */
   float gs_eps;                 /* Gram-Schmidt divides by (norm + gs_eps)                       */
   int32_t decider;              /* worker whose raw gradient is accumulated for the detector     */
-  int32_t flags;                /* 0 or ACC_FLAG_LAZY_RESIDUAL                                   */
+  int32_t flags;                /* 0 or an OR of ACC_FLAG_* values                               */
 } acc_config;
 
 typedef struct acc_ctx acc_ctx;

@@ -19,6 +19,8 @@ ACC_OK = 0
 ACC_MATRIX, ACC_VECTOR = 0, 1
 ACC_MAX_RANK = 4
 ACC_FLAG_LAZY_RESIDUAL = 1
+ACC_FLAG_PIPELINE_ALWAYS = 2
+ACC_FLAG_PIPELINE_NEVER = 4
 POWERSGD, TOPK = 0, 1
 
 

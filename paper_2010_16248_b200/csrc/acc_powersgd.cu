@@ -9,8 +9,6 @@
 // every access is a fully coalesced, 16-byte aligned float4 whatever the row length, and all blocks carry
 // the same load.  Row structure only enters through the factors: element i of a layer sits in row i / m,
 // column i % m, and the rows a tile cuts are reduced from shared memory afterwards.
-#include <cstdlib>
-
 #include "acc_async.cuh"
 #include "acc_internal.cuh"
 
@@ -155,14 +153,17 @@ psgd_project_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict_
 }
 
 // Pass 1, pipelined.  Persistent blocks (one per SM, 512 threads), each with a contiguous range of MATRIX
-// tiles.  The sequence of (tile, worker) stages of a block is streamed through two shared-memory stage
+// tiles.  The sequence of (tile, worker) stages of a block is streamed through three shared-memory stage
 // buffers by bulk asynchronous copies: while the threads consume stage i (g_w and e_w of one tile,
-// 2 x 32 KB), the copy of stage i+1 is in flight and, once everybody has left stage i's buffer, stage i+2
-// is issued into it -- 64-128 KB per SM are in flight at all times without costing registers.
+// 2 x 32 KB), the copies of stages i+1 and i+2 are in flight and, once everybody has left stage i's buffer,
+// stage i+3 is issued into it -- 128-192 KB per SM are in flight at all times without costing registers.
 // The arithmetic is that of the direct kernel (same operations in the same order).
 constexpr int kPipeThreads = 512;
 constexpr int kPipePos = kTile / 4 / kPipeThreads;  // float4 positions per thread and tile
-constexpr size_t kPipeSmemBytes = sizeof(float) * kTile * 5 + 64;
+constexpr int kPipeStages = 2;
+constexpr int kPipeMinStagesPerSm = 200;  // below this the direct kernel is used
+constexpr int kPipeWarps = kPipeThreads / 32;
+constexpr size_t kPipeSmemBytes = sizeof(float) * kTile * (2 * kPipeStages + 1) + sizeof(float4) * 2 * kPipeWarps + 64;
 
 template <bool LAZY>
 __global__ void __launch_bounds__(kPipeThreads, 1)
@@ -173,9 +174,10 @@ psgd_project_pipe_kernel(const DevLayer* __restrict__ layers, const Tile* __rest
                          const int* __restrict__ pending, float* __restrict__ out, float* __restrict__ delta,
                          long long stride, int W, int decider, float inv_w, int* __restrict__ status) {
   extern __shared__ __align__(128) unsigned char smem_raw[];
-  float* stage = reinterpret_cast<float*>(smem_raw);                  // [2 buffers][g, e][kTile]
-  float* s_mbar = stage + 4 * kTile;                                  // [kTile]
-  uint64_t* bars = reinterpret_cast<uint64_t*>(s_mbar + kTile);       // [2]
+  float* stage = reinterpret_cast<float*>(smem_raw);                  // [kPipeStages buffers][g, e][kTile]
+  float* s_mbar = stage + 2 * kPipeStages * kTile;                    // [kTile]
+  float4* s_pp = reinterpret_cast<float4*>(s_mbar + kTile);           // [kPipeWarps][2] partial rows of P
+  uint64_t* bars = reinterpret_cast<uint64_t*>(s_pp + 2 * kPipeWarps);  // [kPipeStages]
   for (int i = blockIdx.x; i < n_vec_tiles; i += gridDim.x) {
     const Tile t = tiles[vec_tiles[i]];
     vector_mean_tile(t, layers[t.layer], grads, out, delta, stride, W, decider, inv_w);
@@ -185,8 +187,7 @@ psgd_project_pipe_kernel(const DevLayer* __restrict__ layers, const Tile* __rest
   const int n_stages = (t1 - t0) * W;
   if (n_stages == 0) return;
   if (threadIdx.x == 0) {
-    mbar_init(&bars[0], 1);
-    mbar_init(&bars[1], 1);
+    for (int b = 0; b < kPipeStages; ++b) mbar_init(&bars[b], 1);
     fence_mbar_init();
   }
   __syncthreads();
@@ -195,22 +196,20 @@ psgd_project_pipe_kernel(const DevLayer* __restrict__ layers, const Tile* __rest
     const Tile t = tiles[mat_tiles[t0 + ti]];
     const long long base = (long long)w * stride + layers[t.layer].offset + t.elem0;
     const unsigned bytes = (unsigned)((t.nelem + 3) / 4) * 16u;  // a ragged tile reads into the layer's padding
-    const int buf = it & 1;
+    const int buf = it % kPipeStages;
     mbar_arrive_expect_tx(&bars[buf], 2 * bytes);
     bulk_copy_g2s(stage + (2 * buf) * kTile, grads + base, bytes, &bars[buf]);
     bulk_copy_g2s(stage + (2 * buf + 1) * kTile, err + base, bytes, &bars[buf]);
   };
-  if (threadIdx.x == 0) {
-    issue(0);
-    if (n_stages > 1) issue(1);
-  }
+  if (threadIdx.x == 0)
+    for (int it = 0; it < kPipeStages && it < n_stages; ++it) issue(it);
   Tile t = tiles[mat_tiles[t0]];
   DevLayer L = layers[t.layer];
   float4 corr[kPipePos], mb[kPipePos];
   int rp = 0;
   for (int it = 0; it < n_stages; ++it) {
     const int ti = it / W, w = it - ti * W;
-    const int buf = it & 1;
+    const int buf = it % kPipeStages;
     if (w == 0) {  // new tile: factors of the pending residual at this thread's positions
       t = tiles[mat_tiles[t0 + ti]];
       L = layers[t.layer];
@@ -233,7 +232,7 @@ psgd_project_pipe_kernel(const DevLayer* __restrict__ layers, const Tile* __rest
         }
       }
     }
-    const bool arrived = __syncthreads_and(mbar_wait_bounded(&bars[buf], (unsigned)(it >> 1) & 1u));
+    const bool arrived = __syncthreads_and(mbar_wait_bounded(&bars[buf], (unsigned)(it / kPipeStages) & 1u));
     if (!arrived) {  // a copy never completed: report and leave (uniformly for the whole block)
       if (threadIdx.x == 0) atomicExch(status, ACC_ETIMEOUT);
       return;
@@ -267,9 +266,9 @@ psgd_project_pipe_kernel(const DevLayer* __restrict__ layers, const Tile* __rest
       }
     }
     __syncthreads();  // everybody has left this stage buffer
-    if (threadIdx.x == 0 && it + 2 < n_stages) {
+    if (threadIdx.x == 0 && it + kPipeStages < n_stages) {
       fence_proxy_async_smem();
-      issue(it + 2);
+      issue(it + kPipeStages);
     }
     if (w == W - 1) {  // tile complete: mean matrix out, partial rows of P from shared memory
       const long long obase = L.offset + t.elem0;
@@ -292,20 +291,54 @@ psgd_project_pipe_kernel(const DevLayer* __restrict__ layers, const Tile* __rest
       const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
       const int first_row = t.elem0 / m, last_row = (t.elem0 + t.nelem - 1) / m;
       const int tile_in_layer = t.elem0 / kTile;
-      for (int row = first_row + warp; row <= last_row; row += kPipeThreads / 32) {
-        const int row_begin = row * m;
-        const int lo = max(row_begin, t.elem0) - t.elem0, hi = min(row_begin + m, t.elem0 + t.nelem) - t.elem0;
-        const float4* qr = Q4 + (t.elem0 + lo - row_begin);
-        float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
-        for (int i = lo + lane; i < hi; i += 32) {
-          const float v = s_mbar[i];
-          const float4 qv = __ldg(qr + (i - lo));
-          a0 = fmaf(v, qv.x, a0); a1 = fmaf(v, qv.y, a1); a2 = fmaf(v, qv.z, a2); a3 = fmaf(v, qv.w, a3);
+      constexpr int kSpan = kTile / kPipeWarps;  // 512 elements of the tile per warp
+      if (m >= 2 * kSpan) {
+        // long rows (too few row pieces to occupy the warps): every warp reduces its own 512-element span of
+        // the tile (it meets at most two rows); the spans of a row are then added in span order
+        const int s0 = warp * kSpan, s1 = min(s0 + kSpan, t.nelem);
+        const int r_lo = (t.elem0 + s0) / m;
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+          const int row_begin = (r_lo + j) * m;
+          const int lo = max(row_begin - t.elem0, s0), hi = min(row_begin + m - t.elem0, s1);
+          float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+          for (int i = lo + lane; i < hi; i += 32) {
+            const float v = s_mbar[i];
+            const float4 qv = __ldg(Q4 + (t.elem0 + i - row_begin));
+            a0 = fmaf(v, qv.x, a0); a1 = fmaf(v, qv.y, a1); a2 = fmaf(v, qv.z, a2); a3 = fmaf(v, qv.w, a3);
+          }
+          a0 = warp_sum(a0); a1 = warp_sum(a1); a2 = warp_sum(a2); a3 = warp_sum(a3);
+          if (lane == 0) s_pp[2 * warp + j] = make_float4(a0, a1, a2, a3);
         }
-        a0 = warp_sum(a0); a1 = warp_sum(a1); a2 = warp_sum(a2); a3 = warp_sum(a3);
-        if (lane == 0)
-          p_part[L.ppart_base + (long long)row * L.nslots + (tile_in_layer - row_begin / kTile)] =
-              make_float4(a0, a1, a2, a3);
+        __syncthreads();
+        const int row = first_row + (int)threadIdx.x;
+        if (row <= last_row) {
+          const int row_begin = row * m;
+          const int lo = max(row_begin, t.elem0) - t.elem0, hi = min(row_begin + m, t.elem0 + t.nelem) - t.elem0;
+          float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+          for (int sp = lo / kSpan; sp <= (hi - 1) / kSpan; ++sp) {
+            const float4 v = s_pp[2 * sp + (row - (t.elem0 + sp * kSpan) / m)];
+            acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+          }
+          p_part[L.ppart_base + (long long)row * L.nslots + (tile_in_layer - row_begin / kTile)] = acc;
+        }
+      } else {
+        // short rows: one warp per row piece
+        for (int row = first_row + warp; row <= last_row; row += kPipeWarps) {
+          const int row_begin = row * m;
+          const int lo = max(row_begin, t.elem0) - t.elem0, hi = min(row_begin + m, t.elem0 + t.nelem) - t.elem0;
+          const float4* qr = Q4 + (t.elem0 + lo - row_begin);
+          float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+          for (int i = lo + lane; i < hi; i += 32) {
+            const float v = s_mbar[i];
+            const float4 qv = __ldg(qr + (i - lo));
+            a0 = fmaf(v, qv.x, a0); a1 = fmaf(v, qv.y, a1); a2 = fmaf(v, qv.z, a2); a3 = fmaf(v, qv.w, a3);
+          }
+          a0 = warp_sum(a0); a1 = warp_sum(a1); a2 = warp_sum(a2); a3 = warp_sum(a3);
+          if (lane == 0)
+            p_part[L.ppart_base + (long long)row * L.nslots + (tile_in_layer - row_begin / kTile)] =
+                make_float4(a0, a1, a2, a3);
+        }
       }
     }
   }
@@ -506,8 +539,13 @@ cudaError_t launch_powersgd(acc_ctx* ctx, const float* grads, float* err, float*
   const int nt = (int)pl.tiles.size();
   const float inv_w = 1.0f / (float)c.n_workers;
   const bool lazy = (c.flags & ACC_FLAG_LAZY_RESIDUAL) != 0;
-  static const bool use_pipe = !(getenv("ACC_NOPIPE") && atoi(getenv("ACC_NOPIPE")));
-  if (use_pipe && pl.n_mat > 0) {
+  // Two implementations of the same pass (same arithmetic, same results): the persistent pipelined kernel
+  // wins once every SM has a long queue of stages (measured: 330 stages/SM -> 0.95 ms against 1.11 ms);
+  // on small sets its one-block-per-SM static split loses a few percent to tile quantisation.
+  const long long stages_per_sm = (long long)pl.mat_tiles.size() * c.n_workers / (ctx->sm_count > 0 ? ctx->sm_count : 1);
+  const bool pipelined = (c.flags & ACC_FLAG_PIPELINE_ALWAYS) ||
+                         (!(c.flags & ACC_FLAG_PIPELINE_NEVER) && stages_per_sm >= kPipeMinStagesPerSm);
+  if (pipelined && pl.n_mat > 0) {
     PhaseTimer pt(ctx, PH_PSGD_PROJECT, s);
     const int n_mt = (int)pl.mat_tiles.size(), n_vt = (int)pl.vec_tiles.size();
     const int grid = n_mt < ctx->sm_count ? n_mt : ctx->sm_count;

@@ -113,10 +113,13 @@ def test_detect_regime_truth_table_and_random():
 
 
 # ------------------------------------------------------------------ PowerSGD
+@pytest.mark.parametrize("pipeline", [binding.ACC_FLAG_PIPELINE_NEVER, binding.ACC_FLAG_PIPELINE_ALWAYS])
 @pytest.mark.parametrize("W,rank_low,rank_high", [(1, 2, 1), (2, 2, 1), (3, 3, 2), (4, 4, 1), (8, 4, 4), (5, 1, 1)])
-def test_powersgd_step_matches_oracle(W, rank_low, rank_high):
+def test_powersgd_step_matches_oracle(W, rank_low, rank_high, pipeline):
+    """Both implementations of the first pass (direct, and persistent with bulk asynchronous copies) on a
+    table with ragged tiles, odd row lengths and vectors."""
     table = _table_mixed()
-    ctx = binding.Context(table, W, rank_low=rank_low, rank_high=rank_high, gs_eps=1e-8)
+    ctx = binding.Context(table, W, rank_low=rank_low, rank_high=rank_high, gs_eps=1e-8, flags=pipeline)
     grads, err = _random_inputs(table, W, 10 + W)
     q = ctx.new_q(wl.initial_q(table, 4, seed=W))  # ranks beyond rank_low hold values that must survive
     p = ctx.new_p()
@@ -131,6 +134,7 @@ def test_powersgd_step_matches_oracle(W, rank_low, rank_high):
         H.check_powersgd_against_oracle(ctx, table, grads, e0, q0, level, out, err, q, p, rank_low, rank_high, 1e-8)
         grads, _ = _random_inputs(table, W, 100 + it)
     assert ctx.last_launch_count() == 5
+    assert ctx.acc_device_status() == 0
 
 
 def test_powersgd_invariants_and_exact_recovery():
@@ -267,14 +271,16 @@ def test_bad_arguments_are_rejected():
 
 
 # ------------------------------------------------------------------ PowerSGD, lazy residual
+@pytest.mark.parametrize("pipeline", [binding.ACC_FLAG_PIPELINE_NEVER, binding.ACC_FLAG_PIPELINE_ALWAYS])
 @pytest.mark.parametrize("W,rank_low,rank_high", [(2, 2, 1), (8, 4, 1), (3, 3, 2)])
-def test_powersgd_lazy_residual_is_bit_identical_to_eager(W, rank_low, rank_high):
+def test_powersgd_lazy_residual_is_bit_identical_to_eager(W, rank_low, rank_high, pipeline):
     """With ACC_FLAG_LAZY_RESIDUAL err holds M_w between steps; out, q and p_hat of every step and the
     flushed error memory must equal the eager mode's bit for bit, also when the level (rank) changes
     between steps; the eager mode itself is checked against the oracle above."""
     table = _table_mixed()
-    eager = binding.Context(table, W, rank_low=rank_low, rank_high=rank_high)
-    lazy = binding.Context(table, W, rank_low=rank_low, rank_high=rank_high, flags=binding.ACC_FLAG_LAZY_RESIDUAL)
+    eager = binding.Context(table, W, rank_low=rank_low, rank_high=rank_high, flags=pipeline)
+    lazy = binding.Context(table, W, rank_low=rank_low, rank_high=rank_high,
+                           flags=binding.ACC_FLAG_LAZY_RESIDUAL | pipeline)
     grads, err0 = _random_inputs(table, W, 40 + W)
     state = []
     for ctx in (eager, lazy):
