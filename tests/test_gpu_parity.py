@@ -176,10 +176,11 @@ def test_powersgd_invariants_and_exact_recovery():
 
 
 # ------------------------------------------------------------------ TopK
+@pytest.mark.parametrize("pipeline", [binding.ACC_FLAG_PIPELINE_NEVER, binding.ACC_FLAG_PIPELINE_ALWAYS])
 @pytest.mark.parametrize("W,low_bp,high_bp", [(1, 1000, 100), (3, 1000, 100), (4, 2500, 200), (2, 10000, 9900), (2, 1, 1)])
-def test_topk_step_bit_exact(W, low_bp, high_bp):
+def test_topk_step_bit_exact(W, low_bp, high_bp, pipeline):
     table = _table_mixed()
-    ctx = binding.Context(table, W, topk_low_bp=low_bp, topk_high_bp=high_bp)
+    ctx = binding.Context(table, W, topk_low_bp=low_bp, topk_high_bp=high_bp, flags=pipeline)
     grads, err = _random_inputs(table, W, 20 + W)
     level = torch.tensor([(l * 5 + W) % 2 for l in range(table.n_layers)], dtype=torch.uint8, device="cuda")
     vals, idx, counts = ctx.new_topk_buffers()
@@ -191,9 +192,11 @@ def test_topk_step_bit_exact(W, low_bp, high_bp):
         H.check_topk_against_oracle(ctx, table, grads, e0, level, vals, idx, counts, out, err, low_bp, high_bp)
         grads, _ = _random_inputs(table, W, 200 + it)
     assert ctx.last_launch_count() == 11
+    assert ctx.acc_device_status() == 0
 
 
-def test_topk_ties_zeros_and_degenerate_layers():
+@pytest.mark.parametrize("pipeline", [binding.ACC_FLAG_PIPELINE_NEVER, binding.ACC_FLAG_PIPELINE_ALWAYS])
+def test_topk_ties_zeros_and_degenerate_layers(pipeline):
     table = wl.make_table([
         ("ties", (40, 650)),       # many exact duplicates around the threshold
         ("zeros", (30, 1000)),     # all zero: keeps the k lowest indices
@@ -203,7 +206,7 @@ def test_topk_ties_zeros_and_degenerate_layers():
         ("quant", (64, 640)),      # few distinct values: ties at every level of the radix select
     ])
     W = 3
-    ctx = binding.Context(table, W, topk_low_bp=1000, topk_high_bp=100)
+    ctx = binding.Context(table, W, topk_low_bp=1000, topk_high_bp=100, flags=pipeline)
     g = torch.Generator(device="cuda").manual_seed(7)
     grads = torch.zeros(W, table.stride, device="cuda")
     sl = {table.names[l]: s for l, s in table.slices()}
@@ -313,14 +316,15 @@ def test_powersgd_lazy_residual_is_bit_identical_to_eager(W, rank_low, rank_high
         eager.acc_powersgd_flush(state[0]["err"], state[0]["q"], state[0]["p"])
 
 
-def test_topk_threshold_prediction_hits_and_misses():
+@pytest.mark.parametrize("pipeline", [binding.ACC_FLAG_PIPELINE_NEVER, binding.ACC_FLAG_PIPELINE_ALWAYS])
+def test_topk_threshold_prediction_hits_and_misses(pipeline):
     """The step predicts the threshold's bucket from the previous step at the same level.  Sequence of
     gradient scales that makes the prediction hold (same scale), miss upwards (x10: exact list path),
     miss downwards (x0.1: the histogram below the predicted band was not counted, redo path) and switch
     level in between; every step must still match the oracle bit for bit."""
     table = _table_mixed()
     W = 2
-    ctx = binding.Context(table, W)
+    ctx = binding.Context(table, W, flags=pipeline)
     vals, idx, counts = ctx.new_topk_buffers()
     out = torch.zeros(table.stride, device="cuda")
     base, _ = _random_inputs(table, W, 77, err_scale=0.0)
