@@ -71,3 +71,56 @@ class AccordionStep:
         if "topk" in self.compressors:
             outs.append(self.out_topk)
         return outs
+
+
+class HostFedStep:
+    """Runs ``AccordionStep`` on gradients that live in pinned host memory.
+
+    Every call copies that step's gradients to the device and the step's averaged outputs back to pinned
+    host buffers.  The copies run on their own stream with two device staging buffers, so the upload of
+    step i+1 overlaps the kernels of step i; results are ordered by events, never by host synchronisation.
+    """
+
+    def __init__(self, engine: AccordionStep):
+        self.eng = engine
+        dev = engine.device
+        shape = (engine.W, engine.table.stride)
+        self.stage = [torch.empty(shape, dtype=torch.float32, device=dev) for _ in range(2)]
+        self.h2d = torch.cuda.Stream(device=dev)
+        self.d2h = torch.cuda.Stream(device=dev)
+        self.uploaded = [torch.cuda.Event() for _ in range(2)]
+        self.consumed = [torch.cuda.Event() for _ in range(2)]
+        self.downloaded = torch.cuda.Event()
+        self.outs_host = [torch.empty(engine.table.stride, dtype=torch.float32).pin_memory() for _ in engine.outputs()]
+        self.i = 0
+        self.h2d_bytes_per_step = 4 * shape[0] * shape[1]
+        self.d2h_bytes_per_step = 4 * engine.table.stride * len(self.outs_host)
+
+    def step(self, host_grads: torch.Tensor):
+        """Queues upload, compute and download of one step; returns the pinned host output tensors (valid
+        after ``synchronize`` or after the next call's download event)."""
+        assert host_grads.is_pinned() and host_grads.dtype == torch.float32
+        b = self.i & 1
+        main = torch.cuda.current_stream(self.eng.device)
+        with torch.cuda.stream(self.h2d):
+            if self.i >= 2:
+                self.h2d.wait_event(self.consumed[b])      # the step that read this staging buffer is done
+            self.stage[b].copy_(host_grads, non_blocking=True)
+            self.uploaded[b].record(self.h2d)
+        main.wait_event(self.uploaded[b])
+        if self.i >= 1:
+            main.wait_event(self.downloaded)               # previous outputs are safely on the host
+        self.eng.step(self.stage[b])
+        self.consumed[b].record(main)
+        with torch.cuda.stream(self.d2h):
+            self.d2h.wait_event(self.consumed[b])
+            for oh, od in zip(self.outs_host, self.eng.outputs()):
+                oh.copy_(od, non_blocking=True)
+            self.downloaded.record(self.d2h)
+        self.i += 1
+        return self.outs_host
+
+    def synchronize(self):
+        self.h2d.synchronize()
+        self.d2h.synchronize()
+        torch.cuda.current_stream(self.eng.device).synchronize()
