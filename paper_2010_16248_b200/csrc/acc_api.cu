@@ -113,6 +113,7 @@ static int make_plan(const acc_config* cfg, Plan& p) {
   take(sizeof(unsigned) * seg * kBins3);
   take(sizeof(unsigned) * seg);  // candidate counters, cleared with the histograms
   take(sizeof(unsigned) * seg);  // overflow flags of the predicted collection, likewise
+  take(sizeof(unsigned) * 64);   // "some segment needs the collect pass" flag, likewise
   p.hist_bytes = o - p.o_hist;
   p.o_sel = take(sizeof(Select) * seg);
   p.o_pred = take(sizeof(unsigned) * 2 * seg);
@@ -174,6 +175,7 @@ int acc_create(const acc_config* cfg, void* workspace, size_t workspace_bytes, a
   ctx->d_hist3 = ctx->d_hist2 + (align_up(sizeof(unsigned) * seg * kBins2, 256) / sizeof(unsigned));
   ctx->d_seg_cand = ctx->d_hist3 + (align_up(sizeof(unsigned) * seg * kBins3, 256) / sizeof(unsigned));
   ctx->d_seg_flag = ctx->d_seg_cand + (align_up(sizeof(unsigned) * seg, 256) / sizeof(unsigned));
+  ctx->d_any_list = ctx->d_seg_flag + (align_up(sizeof(unsigned) * seg, 256) / sizeof(unsigned));
   ctx->d_pred = reinterpret_cast<unsigned*>(ws + p.o_pred);
   ctx->d_sel = reinterpret_cast<Select*>(ws + p.o_sel);
   ctx->d_cand = reinterpret_cast<unsigned*>(ws + p.o_cand);

@@ -102,6 +102,7 @@ struct acc_ctx {
   unsigned* d_hist3 = nullptr;
   acc::Select* d_sel = nullptr;
   unsigned* d_seg_cand = nullptr;    // per (worker, layer): candidate slots handed out this step
+  unsigned* d_any_list = nullptr;    // 1 if some segment needs the collect pass this step
   unsigned* d_seg_flag = nullptr;    // per (worker, layer): 1 if pass A's collection overflowed this step
   unsigned* d_pred = nullptr;        // [2][W * n_mat]: predicted threshold bucket per level, kept across steps
   unsigned* d_cand = nullptr;        // candidate keys, [W][cand_total]

@@ -222,7 +222,8 @@ __global__ void __launch_bounds__(256)
 topk_pick1_kernel(const DevLayer* __restrict__ layers, const int* __restrict__ mat_layers, int n_mat, int n_layers,
                   int W, const uint8_t* __restrict__ level, const unsigned* __restrict__ hist1,
                   Select* __restrict__ sel, int32_t* __restrict__ counts, unsigned* __restrict__ pred,
-                  unsigned* __restrict__ seg_cand, const unsigned* __restrict__ seg_flag) {
+                  unsigned* __restrict__ seg_cand, const unsigned* __restrict__ seg_flag,
+                  unsigned* __restrict__ any_list) {
   __shared__ unsigned sums[256];
   __shared__ unsigned bin;
   __shared__ long long above;
@@ -245,6 +246,7 @@ topk_pick1_kernel(const DevLayer* __restrict__ layers, const int* __restrict__ m
     } else {
       seg_cand[seg] = 0;  // whatever pass A collected is of no use
       s.mode = fits ? kSelList : kSelDense;
+      if (fits) *any_list = 1u;
     }
     // next prediction: narrow the band after an overflow; none for the zero bucket or for buckets that
     // do not fit the list
@@ -326,36 +328,44 @@ __device__ __forceinline__ void collect_tile(const Tile& t, const Select& s, con
     tile_cnt_out->x = (int)(total >> 16);
   }
   __syncthreads();
-  if (inb == 0) return;
-  unsigned* dst = seg_list + *s_start + ((wbase + c - own) & 0xffffu);
+  if (inb != 0) {
+    unsigned* dst = seg_list + *s_start + ((wbase + c - own) & 0xffffu);
 #pragma unroll
-  for (int j = 0; j < 8; ++j) {
-    const float v[4] = {mv[j].x, mv[j].y, mv[j].z, mv[j].w};
+    for (int j = 0; j < 8; ++j) {
+      const float v[4] = {mv[j].x, mv[j].y, mv[j].z, mv[j].w};
 #pragma unroll
-    for (int e = 0; e < 4; ++e)
-      if ((inb >> (4 * j + e)) & 1u) *dst++ = key_of(v[e]);
+      for (int e = 0; e < 4; ++e)
+        if ((inb >> (4 * j + e)) & 1u) *dst++ = key_of(v[e]);
+    }
   }
+  __syncthreads();  // wsum and s_start are reused by the block's next tile
 }
 
+// Blocks walk the (worker, tile) pairs with a grid stride; when no segment of this step is in list mode
+// (every prediction of pass A held, or only dense segments remain) the kernel ends at once.
 __global__ void __launch_bounds__(256, 3)
 topk_collect_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict__ tiles, int n_tiles, int n_mat,
-                    const float* __restrict__ err, long long stride, const Select* __restrict__ sel,
-                    unsigned* __restrict__ seg_cand, unsigned* __restrict__ cand, int2* __restrict__ tile_cand,
-                    long long cand_total, int2* __restrict__ tile_cnt) {
+                    int W, const float* __restrict__ err, long long stride, const Select* __restrict__ sel,
+                    const unsigned* __restrict__ any_list, unsigned* __restrict__ seg_cand,
+                    unsigned* __restrict__ cand, int2* __restrict__ tile_cand, long long cand_total,
+                    int2* __restrict__ tile_cnt) {
   __shared__ unsigned wsum[8];
   __shared__ unsigned s_start;
-  const int ti = blockIdx.x, w = blockIdx.y;
-  const Tile t = tiles[ti];
-  const DevLayer L = layers[t.layer];
-  if (L.kind != ACC_MATRIX) return;
-  const int seg = w * n_mat + L.mat;
-  const Select s = sel[seg];
-  if (s.mode != kSelList) return;
-  const float* m = err + (long long)w * stride + L.offset + t.elem0;
-  unsigned* list = cand + (long long)w * cand_total + L.cand_base;
-  const long long v = (long long)w * n_tiles + ti;
-  if (t.nelem == kTile) collect_tile<true>(t, s, m, seg_cand + seg, list, tile_cand + v, tile_cnt + v, wsum, &s_start);
-  else collect_tile<false>(t, s, m, seg_cand + seg, list, tile_cand + v, tile_cnt + v, wsum, &s_start);
+  if (*any_list == 0) return;
+  const long long V = (long long)W * n_tiles;
+  for (long long v = blockIdx.x; v < V; v += gridDim.x) {
+    const int w = (int)(v / n_tiles), ti = (int)(v % n_tiles);
+    const Tile t = tiles[ti];
+    const DevLayer L = layers[t.layer];
+    if (L.kind != ACC_MATRIX) continue;
+    const int seg = w * n_mat + L.mat;
+    const Select s = sel[seg];
+    if (s.mode != kSelList) continue;
+    const float* m = err + (long long)w * stride + L.offset + t.elem0;
+    unsigned* list = cand + (long long)w * cand_total + L.cand_base;
+    if (t.nelem == kTile) collect_tile<true>(t, s, m, seg_cand + seg, list, tile_cand + v, tile_cnt + v, wsum, &s_start);
+    else collect_tile<false>(t, s, m, seg_cand + seg, list, tile_cand + v, tile_cnt + v, wsum, &s_start);
+  }
 }
 
 // Pass C.  Level-2 histogram of the keys whose level-1 bin is b1; per tile, how many keys lie in higher bins.
@@ -775,13 +785,14 @@ cudaError_t launch_topk(acc_ctx* ctx, const float* grads, float* err, const uint
       PhaseTimer pt(ctx, PH_TOPK_PICK1, s);
       topk_pick1_kernel<<<W * n_mat, 256, 0, s>>>(ctx->d_layers, ctx->d_mat_layers, n_mat, c.n_layers, W, level,
                                                   ctx->d_hist1, ctx->d_sel, counts, ctx->d_pred, ctx->d_seg_cand,
-                                                  ctx->d_seg_flag);
+                                                  ctx->d_seg_flag, ctx->d_any_list);
     }
     {
       PhaseTimer pt(ctx, PH_TOPK_COLLECT, s);
-      topk_collect_kernel<<<dim3(nt, W), 256, 0, s>>>(ctx->d_layers, ctx->d_tiles, nt, n_mat, err, c.worker_stride,
-                                                      ctx->d_sel, ctx->d_seg_cand, ctx->d_cand, ctx->d_tile_cand,
-                                                      pl.cand_total, ctx->d_tile_cnt);
+      const long long cap = (long long)ctx->sm_count * 12;
+      topk_collect_kernel<<<(unsigned)(V < cap ? V : cap), 256, 0, s>>>(
+          ctx->d_layers, ctx->d_tiles, nt, n_mat, W, err, c.worker_stride, ctx->d_sel, ctx->d_any_list,
+          ctx->d_seg_cand, ctx->d_cand, ctx->d_tile_cand, pl.cand_total, ctx->d_tile_cnt);
     }
     {
       PhaseTimer pt(ctx, PH_TOPK_HIST2, s);
