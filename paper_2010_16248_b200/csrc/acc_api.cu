@@ -339,7 +339,8 @@ const char* acc_profile_kernel_name(int32_t i) {
       "psgd_residual_kernel",
       "topk_ef_hist1_kernel", "topk_pick1_kernel", "topk_hist2_kernel", "topk_pick2_kernel", "topk_hist3_kernel",
       "topk_tile_scan_kernel", "topk_select_kernel", "topk_decompress_kernel", "psgd_flush_kernel",
-      "topk_collect_kernel", "topk_pick3_kernel", "topk_tile_counts_kernel"};
+      "topk_collect_kernel", "topk_pick3_kernel", "topk_tile_counts_kernel",
+      "topk_hist2_list_kernel", "topk_hist3_list_kernel"};
   return (i >= 0 && i < PH_COUNT) ? names[i] : "";
 }
 

@@ -52,7 +52,7 @@ enum Phase {
   PH_EF = 0, PH_NORM_PARTIAL, PH_NORM_FINAL, PH_DETECT,
   PH_PSGD_PROJECT, PH_PSGD_ORTHO, PH_PSGD_QPARTIAL, PH_PSGD_QREDUCE, PH_PSGD_RESIDUAL,
   PH_TOPK_EF_HIST1, PH_TOPK_PICK1, PH_TOPK_HIST2, PH_TOPK_PICK2, PH_TOPK_HIST3, PH_TOPK_PICK3_SCAN, PH_TOPK_SELECT,
-  PH_TOPK_DECOMPRESS, PH_PSGD_FLUSH, PH_TOPK_COLLECT, PH_TOPK_PICK3, PH_TOPK_TILE_COUNTS,
+  PH_TOPK_DECOMPRESS, PH_PSGD_FLUSH, PH_TOPK_COLLECT, PH_TOPK_PICK3, PH_TOPK_TILE_COUNTS, PH_TOPK_HIST2_LIST, PH_TOPK_HIST3_LIST,
   PH_COUNT
 };
 
@@ -102,7 +102,7 @@ struct acc_ctx {
   unsigned* d_hist3 = nullptr;
   acc::Select* d_sel = nullptr;
   unsigned* d_seg_cand = nullptr;    // per (worker, layer): candidate slots handed out this step
-  unsigned* d_any_list = nullptr;    // 1 if some segment needs the collect pass this step
+  unsigned* d_any_list = nullptr;    // [0]: some segment needs the collect pass this step; [1]: some segment is dense
   unsigned* d_seg_flag = nullptr;    // per (worker, layer): 1 if pass A's collection overflowed this step
   unsigned* d_pred = nullptr;        // [2][W * n_mat]: predicted threshold bucket per level, kept across steps
   unsigned* d_cand = nullptr;        // candidate keys, [W][cand_total]

@@ -9,12 +9,13 @@
 //   collect    (list path) keys of bucket b1 -> per-tile ranges of the segment's candidate list,
 //              per-tile count of keys above b1                                                  [reads M]
 //   hist2      level-2 histogram of the keys inside b1 (dense path: reads M and also counts the keys
-//              above b1 per tile; list path: reads the collected keys)
+//              above b1 per tile; list path, topk_hist_list_kernel: reads the segment's collected keys)
 //   pick2      bucket b2
-//   hist3      per-tile level-3 histogram of the keys with prefix (b1,b2), per-tile count above
-//              (dense path: reads M; list path: reads the collected keys)
+//   hist3      level-3 histogram of the keys with prefix (b1,b2) (dense path: reads M, keeps it per tile
+//              together with the per-tile count above; list path: per segment from the collected keys)
 //   pick3      threshold tau and the number of ties to keep
-//   tilecounts per tile (keys above tau, keys equal to tau);  tilescan: their exclusive prefix per layer
+//   tilecounts per tile (keys above tau, keys equal to tau), from the tile's level-3 histogram (dense) or from
+//              its collected keys (list);  tilescan: their exclusive prefix per layer
 //   select     keep key > tau and the lowest-index `need` of key == tau; write (val, idx) in index
 //              order, zero the kept entries of err                                              [reads M]
 //   decompress out = (1/W) sum_w scatter(idx_w, val_w), accumulated per tile in shared memory [reads packed]
@@ -246,7 +247,7 @@ topk_pick1_kernel(const DevLayer* __restrict__ layers, const int* __restrict__ m
     } else {
       seg_cand[seg] = 0;  // whatever pass A collected is of no use
       s.mode = fits ? kSelList : kSelDense;
-      if (fits) *any_list = 1u;
+      any_list[fits ? 0 : 1] = 1u;  // word 0: some segment needs the collect pass; word 1: some segment is dense
     }
     // next prediction: narrow the band after an overflow; none for the zero bucket or for buckets that
     // do not fit the list
@@ -372,10 +373,11 @@ topk_collect_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict_
 __global__ void __launch_bounds__(256)
 topk_hist2_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict__ tiles, int n_tiles, int n_mat,
                   const float* __restrict__ err, long long stride, int W, const Select* __restrict__ sel,
-                  const unsigned* __restrict__ cand, const int2* __restrict__ tile_cand, long long cand_total,
-                  unsigned* __restrict__ hist2, int2* __restrict__ tile_cnt) {
+                  const unsigned* __restrict__ any_dense, unsigned* __restrict__ hist2,
+                  int2* __restrict__ tile_cnt) {
   __shared__ unsigned h[kBins2];
   __shared__ int cnt;
+  if (*any_dense == 0) return;
   for (int b = threadIdx.x; b < kBins2; b += blockDim.x) h[b] = 0;
   if (threadIdx.x == 0) cnt = 0;
   __syncthreads();
@@ -401,15 +403,7 @@ topk_hist2_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict__ 
       b1 = sel[seg].b1;
       mode = sel[seg].mode;
     }
-    if (mode != kSelDense) {  // the tile's keys of bucket b1 were collected; its count above is already known
-      const int2 tc = tile_cand[(long long)w * n_tiles + ti];
-      const unsigned* c = cand + (long long)w * cand_total + L.cand_base + tc.x;
-      for (int i = threadIdx.x; i < tc.y; i += blockDim.x) {
-        const unsigned kk = c[i];  // a predicted band may hold keys of neighbouring buckets
-        if ((kk >> 19) == b1) atomicAdd(&h[(kk >> 7) & 0xfffu], 1u);
-      }
-      continue;
-    }
+    if (mode != kSelDense) continue;  // list segments are served by topk_hist_list_kernel
     const float* m = err + (long long)w * stride + L.offset + t.elem0;
     int above = 0;
     const int n4 = t.nelem >> 2;
@@ -447,31 +441,25 @@ topk_hist2_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict__ 
 __global__ void __launch_bounds__(256)
 topk_hist3_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict__ tiles, int n_tiles, int n_mat,
                   const float* __restrict__ err, long long stride, const Select* __restrict__ sel,
-                  const unsigned* __restrict__ cand, const int2* __restrict__ tile_cand, long long cand_total,
-                  unsigned* __restrict__ hist3, int2* __restrict__ tile_cnt, unsigned short* __restrict__ tile_h3) {
+                  const unsigned* __restrict__ any_dense, unsigned* __restrict__ hist3,
+                  int2* __restrict__ tile_cnt, unsigned short* __restrict__ tile_h3) {
   __shared__ unsigned h[kBins3];
   __shared__ int cnt;
+  if (*any_dense == 0) return;
   const int ti = blockIdx.x, w = blockIdx.y;
   const Tile t = tiles[ti];
   const DevLayer L = layers[t.layer];
   if (L.kind != ACC_MATRIX) return;
+  const int seg = w * n_mat + L.mat;
+  const Select s = sel[seg];
+  if (s.mode != kSelDense) return;  // list segments: topk_hist_list_kernel and topk_tile_counts_kernel
   if (threadIdx.x < kBins3) h[threadIdx.x] = 0;
   if (threadIdx.x == 0) cnt = 0;
   __syncthreads();
-  const int seg = w * n_mat + L.mat;
-  const Select s = sel[seg];
   const unsigned prefix = (s.b1 << 12) | s.b2;
   const float* m = err + (long long)w * stride + L.offset + t.elem0;
   int above = 0;
-  if (s.mode != kSelDense) {
-    const int2 tc = tile_cand[(long long)w * n_tiles + ti];
-    const unsigned* c = cand + (long long)w * cand_total + L.cand_base + tc.x;
-    for (int i = threadIdx.x; i < tc.y; i += blockDim.x) {
-      const unsigned k0 = c[i], p = k0 >> 7;  // collected keys: bucket b1, or a predicted band around it
-      above += p > prefix;
-      if (p == prefix) atomicAdd(&h[k0 & 127u], 1u);
-    }
-  } else {
+  {
     const int n4 = t.nelem >> 2;
 #pragma unroll 4
     for (int i = threadIdx.x; i < n4; i += blockDim.x) {
@@ -498,6 +486,52 @@ topk_hist3_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict__ 
     const unsigned c = h[threadIdx.x];
     tile_h3[((long long)w * n_tiles + ti) * kBins3 + threadIdx.x] = (unsigned short)c;
     if (c) atomicAdd(&hist3[(long long)seg * kBins3 + threadIdx.x], c);
+  }
+}
+
+// List path, levels 2 and 3.  The keys collected for a segment (by pass A or by the collect pass) sit in one
+// contiguous list; blocks (chunk, segment) histogram them.  LEVEL 2: keys of bucket b1 by their next 12 bits;
+// LEVEL 3: keys with the 24-bit prefix (b1, b2) by their last 7 bits.
+template <int LEVEL>
+__global__ void __launch_bounds__(256)
+topk_hist_list_kernel(const DevLayer* __restrict__ layers, const int* __restrict__ mat_layers, int n_mat,
+                      const Select* __restrict__ sel, const unsigned* __restrict__ seg_cand,
+                      const unsigned* __restrict__ cand, long long cand_total, unsigned* __restrict__ hist) {
+  constexpr int kBins = LEVEL == 2 ? kBins2 : kBins3;
+  constexpr unsigned kChunk = 4096;
+  __shared__ unsigned h[kBins];
+  const int seg = blockIdx.y;
+  const Select s = sel[seg];
+  if (s.mode == kSelDense) return;
+  const unsigned n = seg_cand[seg];
+  if (blockIdx.x * kChunk >= n) return;
+  for (int b = threadIdx.x; b < kBins; b += blockDim.x) h[b] = 0;
+  __syncthreads();
+  const DevLayer L = layers[mat_layers[seg % n_mat]];
+  const unsigned* keys = cand + (long long)(seg / n_mat) * cand_total + L.cand_base;
+  const unsigned prefix = (s.b1 << 12) | s.b2;
+  auto count = [&](unsigned kk) {
+    if (LEVEL == 2) {
+      if ((kk >> 19) == s.b1) atomicAdd(&h[(kk >> 7) & 0xfffu], 1u);
+    } else {
+      if ((kk >> 7) == prefix) atomicAdd(&h[kk & 127u], 1u);
+    }
+  };
+  for (unsigned c0 = blockIdx.x * kChunk; c0 < n; c0 += gridDim.x * kChunk) {
+    const unsigned c1 = min(c0 + kChunk, n);  // the list starts 16-byte aligned and kChunk is a multiple of 4
+    const unsigned n4 = (c1 - c0) >> 2;
+    const uint4* k4 = reinterpret_cast<const uint4*>(keys + c0);
+#pragma unroll 4
+    for (unsigned i = threadIdx.x; i < n4; i += blockDim.x) {
+      const uint4 kk = __ldcs(k4 + i);
+      count(kk.x); count(kk.y); count(kk.z); count(kk.w);
+    }
+    for (unsigned i = c0 + 4 * n4 + threadIdx.x; i < c1; i += blockDim.x) count(keys[i]);
+  }
+  __syncthreads();
+  for (int b = threadIdx.x; b < kBins; b += blockDim.x) {
+    const unsigned c = h[b];
+    if (c) atomicAdd(&hist[(long long)seg * kBins + b], c);
   }
 }
 
@@ -538,14 +572,30 @@ topk_pick3_kernel(int n_seg, const unsigned* __restrict__ hist3, Select* __restr
 __global__ void __launch_bounds__(256)
 topk_tile_counts_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict__ tiles, int n_tiles, int n_mat,
                         int W, const Select* __restrict__ sel, const int2* __restrict__ tile_cnt,
-                        const unsigned short* __restrict__ tile_h3, int2* __restrict__ tile_pre) {
+                        const unsigned short* __restrict__ tile_h3, const unsigned* __restrict__ cand,
+                        const int2* __restrict__ tile_cand, long long cand_total, int2* __restrict__ tile_pre) {
   const long long v = (long long)blockIdx.x * 8 + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
   if (v >= (long long)W * n_tiles) return;
   const int w = (int)(v / n_tiles), ti = (int)(v % n_tiles);
   const DevLayer L = layers[tiles[ti].layer];
   if (L.kind != ACC_MATRIX) return;
-  const unsigned b3 = sel[w * n_mat + L.mat].tau & 127u;
+  const Select s = sel[w * n_mat + L.mat];
+  if (s.mode != kSelDense) {  // list segment: count the tile's collected keys against the final threshold
+    const int2 tc = tile_cand[v];
+    const unsigned* keys = cand + (long long)w * cand_total + L.cand_base + tc.x;
+    int above = 0, ties = 0;
+    for (int i = lane; i < tc.y; i += 32) {
+      const unsigned kk = keys[i];
+      above += kk > s.tau;
+      ties += kk == s.tau;
+    }
+    above = __reduce_add_sync(0xffffffffu, above);
+    ties = __reduce_add_sync(0xffffffffu, ties);
+    if (lane == 0) tile_pre[v] = make_int2(tile_cnt[v].x + above, ties);
+    return;
+  }
+  const unsigned b3 = s.tau & 127u;
   const unsigned short* h = tile_h3 + v * kBins3;
   const uint2 raw = *reinterpret_cast<const uint2*>(h + 4 * lane);  // bins 4*lane .. 4*lane+3
   const unsigned c[4] = {raw.x & 0xffffu, raw.x >> 16, raw.y & 0xffffu, raw.y >> 16};
@@ -797,8 +847,13 @@ cudaError_t launch_topk(acc_ctx* ctx, const float* grads, float* err, const uint
     {
       PhaseTimer pt(ctx, PH_TOPK_HIST2, s);
       topk_hist2_kernel<<<grid, 256, 0, s>>>(ctx->d_layers, ctx->d_tiles, nt, n_mat, err, c.worker_stride, W,
-                                             ctx->d_sel, ctx->d_cand, ctx->d_tile_cand, pl.cand_total,
-                                             ctx->d_hist2, ctx->d_tile_cnt);
+                                             ctx->d_sel, ctx->d_any_list + 1, ctx->d_hist2, ctx->d_tile_cnt);
+    }
+    {
+      PhaseTimer pt(ctx, PH_TOPK_HIST2_LIST, s);
+      topk_hist_list_kernel<2><<<dim3(128, W * n_mat), 256, 0, s>>>(ctx->d_layers, ctx->d_mat_layers, n_mat, ctx->d_sel,
+                                                                   ctx->d_seg_cand, ctx->d_cand, pl.cand_total,
+                                                                   ctx->d_hist2);
     }
     {
       PhaseTimer pt(ctx, PH_TOPK_PICK2, s);
@@ -807,8 +862,14 @@ cudaError_t launch_topk(acc_ctx* ctx, const float* grads, float* err, const uint
     {
       PhaseTimer pt(ctx, PH_TOPK_HIST3, s);
       topk_hist3_kernel<<<dim3(nt, W), 256, 0, s>>>(ctx->d_layers, ctx->d_tiles, nt, n_mat, err, c.worker_stride,
-                                                    ctx->d_sel, ctx->d_cand, ctx->d_tile_cand, pl.cand_total,
-                                                    ctx->d_hist3, ctx->d_tile_cnt, ctx->d_tile_h3);
+                                                    ctx->d_sel, ctx->d_any_list + 1, ctx->d_hist3, ctx->d_tile_cnt,
+                                                    ctx->d_tile_h3);
+    }
+    {
+      PhaseTimer pt(ctx, PH_TOPK_HIST3_LIST, s);
+      topk_hist_list_kernel<3><<<dim3(128, W * n_mat), 256, 0, s>>>(ctx->d_layers, ctx->d_mat_layers, n_mat, ctx->d_sel,
+                                                                   ctx->d_seg_cand, ctx->d_cand, pl.cand_total,
+                                                                   ctx->d_hist3);
     }
     {
       PhaseTimer pt(ctx, PH_TOPK_PICK3, s);
@@ -817,7 +878,8 @@ cudaError_t launch_topk(acc_ctx* ctx, const float* grads, float* err, const uint
     {
       PhaseTimer pt(ctx, PH_TOPK_TILE_COUNTS, s);
       topk_tile_counts_kernel<<<(unsigned)(((long long)W * nt + 7) / 8), 256, 0, s>>>(
-          ctx->d_layers, ctx->d_tiles, nt, n_mat, W, ctx->d_sel, ctx->d_tile_cnt, ctx->d_tile_h3, ctx->d_tile_pre);
+          ctx->d_layers, ctx->d_tiles, nt, n_mat, W, ctx->d_sel, ctx->d_tile_cnt, ctx->d_tile_h3, ctx->d_cand,
+          ctx->d_tile_cand, pl.cand_total, ctx->d_tile_pre);
     }
     {
       PhaseTimer pt(ctx, PH_TOPK_PICK3_SCAN, s);
