@@ -56,6 +56,7 @@ static int make_plan(const acc_config* cfg, Plan& p) {
     DevLayer& o = p.layers[l];
     memset(&o, 0, sizeof(o));
     o.offset = d.offset; o.rows = d.rows; o.cols = d.cols; o.kind = d.kind;
+    o.inv_cols = 1.0 / (double)d.cols;
     o.q_row = o.p_row = o.mat = -1; o.seg_off = -1; o.part_base = -1;
     o.vec = (d.cols % 4 == 0) ? 4 : (d.cols % 2 == 0) ? 2 : 1;
     const long long size = (long long)d.rows * d.cols;

@@ -20,6 +20,7 @@ constexpr int kColBlockThreads = 256;
 struct DevLayer {
   long long offset;   // element offset inside a worker's slice
   int rows, cols, kind;
+  double inv_cols;    // 1.0 / cols, for row = index / cols without an integer division
   int q_row, p_row;   // first row of the layer's block in q / p_hat (MATRIX), else -1
   int vec;            // widest vector width (4, 2, 1) at which every row start is aligned
   int nslots;         // tiles a row of this layer can touch: (cols - 1) / 8192 + 2

@@ -23,9 +23,17 @@ __device__ __forceinline__ float lowrank_entry(const float4& pv, const float4& q
 }
 
 // A = P^[row] . Q[col] (first r ranks) for the four consecutive elements that start at layer element e_idx.
+// row = e_idx / m without an integer division: the double-precision reciprocal is exact to within one.
+__device__ __forceinline__ int row_of(int e_idx, int m, double inv_m) {
+  int row = (int)((double)e_idx * inv_m);
+  const int col = e_idx - row * m;
+  row += (col >= m) - (col < 0);
+  return row;
+}
+
 __device__ __forceinline__ float4 lowrank4(const float4* __restrict__ P4, const float4* __restrict__ Q4, int m,
-                                           int e_idx, int r) {
-  int row = e_idx / m, col = e_idx - row * m;
+                                           double inv_m, int e_idx, int r) {
+  int row = row_of(e_idx, m, inv_m), col = e_idx - row * m;
   float4 pv = __ldg(P4 + row);
   float a[4];
 #pragma unroll
@@ -82,7 +90,7 @@ psgd_project_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict_
   for (int f = threadIdx.x; f < n4; f += blockDim.x) {
     const long long idx = base + 4 * f;
     float4 corr = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (LAZY && rp > 0) corr = lowrank4(P4, Q4, m, t.elem0 + 4 * f, rp);
+    if (LAZY && rp > 0) corr = lowrank4(P4, Q4, m, L.inv_cols, t.elem0 + 4 * f, rp);
     float4 mb = make_float4(0.f, 0.f, 0.f, 0.f);
     for (int w0 = 0; w0 < W; w0 += WB) {
       float4 gv[WB], ev[WB];
@@ -221,7 +229,7 @@ psgd_project_pipe_kernel(const DevLayer* __restrict__ layers, const Tile* __rest
         const int e0 = 4 * (k * kPipeThreads + (int)threadIdx.x);
         mb[k] = make_float4(0.f, 0.f, 0.f, 0.f);
         corr[k] = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (LAZY && rp > 0 && e0 + 3 < t.nelem) corr[k] = lowrank4(P4, Q4, L.cols, t.elem0 + e0, rp);
+        if (LAZY && rp > 0 && e0 + 3 < t.nelem) corr[k] = lowrank4(P4, Q4, L.cols, L.inv_cols, t.elem0 + e0, rp);
         else if (LAZY && rp > 0 && e0 < t.nelem) {  // ragged last float4 of a layer
           float c[4] = {0.f, 0.f, 0.f, 0.f};
           for (int e = 0; e0 + e < t.nelem; ++e) {
@@ -501,7 +509,7 @@ psgd_residual_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict
   const int n4 = t.nelem >> 2;
   for (int f = threadIdx.x; f < n4; f += blockDim.x) {
     const long long idx = base + 4 * f;
-    const float4 a = lowrank4(P4, Q4, m, t.elem0 + 4 * f, r);
+    const float4 a = lowrank4(P4, Q4, m, L.inv_cols, t.elem0 + 4 * f, r);
     if (UPDATE_ERR) {
       for (int w0 = 0; w0 < W; w0 += WB) {
         float4 mw[WB];
