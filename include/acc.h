@@ -175,6 +175,18 @@ int acc_topk_step(acc_ctx* ctx, const float* grads, float* err, const uint8_t* l
  * (HOST pointer; 0 = no such event) and blocks until the device has finished the work queued before it. */
 int acc_device_status(acc_ctx* ctx, int32_t* status);
 
+/* Diagnostic (no counterpart in the paper): which selection path the last acc_topk_step took for every
+ * (worker, MATRIX layer) pair, in worker-major order, n >= W * (number of MATRIX layers) HOST ints:
+ *   0 dense (levels 2-3 of the radix select read M), 1 list built by the collect pass, 2 list built by the
+ *   first pass from a held prediction, 3 whole entries staged by the first pass (M not read again).
+ * Blocks until the device has finished the queued work.  All paths give identical results; tests use
+ * this to make sure each one is exercised.                                                          */
+#define ACC_TOPK_PATH_DENSE 0
+#define ACC_TOPK_PATH_LIST 1
+#define ACC_TOPK_PATH_LIST_PREDICTED 2
+#define ACC_TOPK_PATH_STAGED 3
+int acc_topk_last_paths(acc_ctx* ctx, int32_t* paths, int32_t n);
+
 /* Floats one iteration communicates at the given HOST level array, following the "Data Sent"
  * accounting of Tables 1-4: PowerSGD r*(rows+cols) per MATRIX layer, TopK 2*k*W per MATRIX layer
  * (values + indices gathered from every worker), plus every VECTOR element once.  Returns -1 on a

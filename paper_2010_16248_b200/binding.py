@@ -45,7 +45,7 @@ class acc_config(C.Structure):
 EXPORTS = ["acc_workspace_bytes", "acc_create", "acc_destroy", "acc_factor_layout", "acc_topk_layout",
            "acc_error_feedback", "acc_layer_norms", "acc_detect_regime", "acc_powersgd_step", "acc_topk_step",
            "acc_floats_sent", "acc_last_launch_count", "acc_strerror", "acc_profile_enable", "acc_profile_read",
-           "acc_profile_kernel_count", "acc_profile_kernel_name", "acc_sumsq_static", "acc_powersgd_flush", "acc_device_status"]
+           "acc_profile_kernel_count", "acc_profile_kernel_name", "acc_sumsq_static", "acc_powersgd_flush", "acc_device_status", "acc_topk_last_paths"]
 
 _lib = None
 
@@ -86,6 +86,7 @@ def lib() -> C.CDLL:
     L.acc_sumsq_static.argtypes = [vp, i64, vp, vp]
     L.acc_powersgd_flush.argtypes = [vp, vp, vp, vp, vp]
     L.acc_device_status.argtypes = [vp, C.POINTER(i32)]
+    L.acc_topk_last_paths.argtypes = [vp, C.POINTER(i32), i32]
     for name in EXPORTS:
         if name not in ("acc_floats_sent", "acc_last_launch_count", "acc_strerror", "acc_profile_kernel_count",
                         "acc_profile_kernel_name"):
@@ -228,6 +229,13 @@ class Context:
         ms, cnt = (C.c_double * n)(), (C.c_int32 * n)()
         self._check(lib().acc_profile_read(self._h, ms, cnt, n), "acc_profile_read")
         return {lib().acc_profile_kernel_name(i).decode(): (float(ms[i]), int(cnt[i])) for i in range(n) if cnt[i]}
+
+    def acc_topk_last_paths(self) -> np.ndarray:
+        """Selection path (0 dense, 1 list, 2 predicted list, 3 staged) per (worker, MATRIX layer) of the last TopK step."""
+        n = self.n_workers * int((self.q_row >= 0).sum())
+        buf = (C.c_int32 * max(n, 1))()
+        self._check(lib().acc_topk_last_paths(self._h, buf, n), "acc_topk_last_paths")
+        return np.array(buf[:n], np.int32).reshape(self.n_workers, -1)
 
     def acc_device_status(self) -> int:
         """Device-side status word (0 = fine); waits for the queued work of this device."""

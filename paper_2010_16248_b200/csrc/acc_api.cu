@@ -341,8 +341,20 @@ const char* acc_profile_kernel_name(int32_t i) {
       "topk_ef_hist1_kernel", "topk_pick1_kernel", "topk_hist2_kernel", "topk_pick2_kernel", "topk_hist3_kernel",
       "topk_tile_scan_kernel", "topk_select_kernel", "topk_decompress_kernel", "psgd_flush_kernel",
       "topk_collect_kernel", "topk_pick3_kernel", "topk_tile_counts_kernel",
-      "topk_hist2_list_kernel", "topk_hist3_list_kernel"};
+      "topk_hist2_list_kernel", "topk_hist3_list_kernel", "topk_finalize_staged_kernel"};
   return (i >= 0 && i < PH_COUNT) ? names[i] : "";
+}
+
+int acc_topk_last_paths(acc_ctx* ctx, int32_t* paths, int32_t n) {
+  if (!ctx || !paths) return ACC_EINVAL;
+  const int n_seg = ctx->cfg.n_workers * ctx->plan.n_mat;
+  if (n < n_seg) return ACC_EINVAL;
+  std::vector<Select> host((size_t)std::max(n_seg, 1));
+  if (n_seg > 0 &&
+      cudaMemcpy(host.data(), ctx->d_sel, sizeof(Select) * (size_t)n_seg, cudaMemcpyDeviceToHost) != cudaSuccess)
+    return ACC_ECUDA;
+  for (int i = 0; i < n_seg; ++i) paths[i] = host[i].mode;
+  return ACC_OK;
 }
 
 int acc_device_status(acc_ctx* ctx, int32_t* status) {

@@ -45,7 +45,8 @@ struct Select {
   int k, k1, k2, need;  // k wanted; still wanted inside bucket b1 / (b1,b2); ties (key == tau) to keep
   int mode;             // kSelDense: levels 2-3 read M;  kSelList: they read the collected keys of bucket b1
 };
-constexpr int kSelDense = 0, kSelList = 1, kSelListPred = 2;  // ListPred: the list was filled by pass A
+constexpr int kSelDense = 0, kSelList = 1, kSelListPred = 2, kSelStaged = 3;
+// ListPred: the key list was filled by pass A;  Staged: pass A staged whole (value, index) entries
 constexpr int kPredTileCap = 2048;  // keys one tile may hand to a predicted list (more: overflow, fall back)
 
 // Kernels of the library, for per-kernel timing (acc_profile_*).
@@ -53,7 +54,7 @@ enum Phase {
   PH_EF = 0, PH_NORM_PARTIAL, PH_NORM_FINAL, PH_DETECT,
   PH_PSGD_PROJECT, PH_PSGD_ORTHO, PH_PSGD_QPARTIAL, PH_PSGD_QREDUCE, PH_PSGD_RESIDUAL,
   PH_TOPK_EF_HIST1, PH_TOPK_PICK1, PH_TOPK_HIST2, PH_TOPK_PICK2, PH_TOPK_HIST3, PH_TOPK_PICK3_SCAN, PH_TOPK_SELECT,
-  PH_TOPK_DECOMPRESS, PH_PSGD_FLUSH, PH_TOPK_COLLECT, PH_TOPK_PICK3, PH_TOPK_TILE_COUNTS, PH_TOPK_HIST2_LIST, PH_TOPK_HIST3_LIST,
+  PH_TOPK_DECOMPRESS, PH_PSGD_FLUSH, PH_TOPK_COLLECT, PH_TOPK_PICK3, PH_TOPK_TILE_COUNTS, PH_TOPK_HIST2_LIST, PH_TOPK_HIST3_LIST, PH_TOPK_FINALIZE_STAGED,
   PH_COUNT
 };
 
@@ -103,7 +104,7 @@ struct acc_ctx {
   unsigned* d_hist3 = nullptr;
   acc::Select* d_sel = nullptr;
   unsigned* d_seg_cand = nullptr;    // per (worker, layer): candidate slots handed out this step
-  unsigned* d_any_list = nullptr;    // [0]: some segment needs the collect pass this step; [1]: some segment is dense
+  unsigned* d_any_list = nullptr;    // [0]: some segment needs the collect pass this step; [1]: some is dense; [2]: some needs the select pass
   unsigned* d_seg_flag = nullptr;    // per (worker, layer): 1 if pass A's collection overflowed this step
   unsigned* d_pred = nullptr;        // [2][W * n_mat]: predicted threshold bucket per level, kept across steps
   unsigned* d_cand = nullptr;        // candidate keys, [W][cand_total]

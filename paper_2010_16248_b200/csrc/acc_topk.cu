@@ -18,6 +18,7 @@
 //              its collected keys (list);  tilescan: their exclusive prefix per layer
 //   select     keep key > tau and the lowest-index `need` of key == tau; write (val, idx) in index
 //              order, zero the kept entries of err                                              [reads M]
+//   finalize   the same for segments whose pass A staged whole entries: from the list, M is not read
 //   decompress out = (1/W) sum_w scatter(idx_w, val_w), accumulated per tile in shared memory [reads packed]
 // No floating-point atomics and no inter-block waiting: same input, same bits.
 #include "acc_internal.cuh"
@@ -26,12 +27,15 @@ namespace acc {
 
 __device__ __forceinline__ unsigned key_of(float v) { return __float_as_uint(v) & 0x7fffffffu; }
 
-// A prediction word: level-1 bucket of the threshold at the segment's last step at this level, and the
-// half-width (in buckets) of the band collected around it.
+// A prediction word: level-1 bucket of the threshold at the segment's last step at this level (bits 0-15),
+// the half-width in buckets of the band collected around it (bits 16-23), and whether the next pass A may
+// stage whole entries instead of keys (bit 24, see below; bit 25 forbids it for good).
 constexpr unsigned kPredInvalid = 0xffffffffu;
-__device__ __forceinline__ bool pred_band(unsigned word, unsigned* lo, unsigned* hi) {
+__device__ __forceinline__ bool pred_band(unsigned word, unsigned* lo, unsigned* hi, bool* staged) {
+  *staged = false;
   if (word == kPredInvalid) return false;
-  const unsigned b = word & 0xffffu, hw = word >> 16;
+  const unsigned b = word & 0xffffu, hw = (word >> 16) & 0xffu;
+  *staged = (word >> 24) & 1u;
   *lo = b > hw ? b - hw : 1u;  // bucket 0 (zeros, denormals) is never collected
   *hi = b + hw < (unsigned)kBins1 ? b + hw : (unsigned)kBins1 - 1u;
   return *lo <= *hi;
@@ -42,6 +46,10 @@ __device__ __forceinline__ bool pred_band(unsigned word, unsigned* lo, unsigned*
 // (the bucket of the previous step at the same level), the keys of the buckets around it are collected
 // on the fly into the segment's candidate list, so that no further pass over M is needed to refine the
 // threshold when the prediction holds (checked exactly by pick1).
+// When few entries are expected at or above the band (high compression level), pass A stages them whole --
+// (value bits, layer-local index) for every key in a bucket >= the band's lowest -- so that, if the
+// prediction holds, the kept entries are produced from this list and M is never read again for the
+// segment (topk_finalize_staged_kernel instead of topk_select_kernel).
 __global__ void __launch_bounds__(256)
 topk_ef_hist1_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict__ tiles, int n_tiles, int n_mat,
                      const float* __restrict__ grads, float* __restrict__ err, float* __restrict__ delta,
@@ -63,7 +71,7 @@ topk_ef_hist1_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict
   const long long v0 = V * blockIdx.x / gridDim.x, v1 = V * (blockIdx.x + 1) / gridDim.x;
   int cur = -1;
   int cb = 0, pend = -1;  // staging buffer in use; buffer waiting to be copied out
-  bool collect = false;
+  bool collect = false, staged = false;
   unsigned blo = 1, bhi = 0;
   for (long long v = v0; v < v1; ++v) {
     const int w = (int)(v / n_tiles), ti = (int)(v % n_tiles);
@@ -80,7 +88,7 @@ topk_ef_hist1_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict
         }
       __syncthreads();
       cur = seg;
-      collect = pred_band(pred[(level[t.layer] ? 1 : 0) * W * n_mat + seg], &blo, &bhi);
+      collect = pred_band(pred[(level[t.layer] ? 1 : 0) * W * n_mat + seg], &blo, &bhi, &staged);
     }
     const long long base = L.offset + t.elem0;
     const float* g = grads + (long long)w * stride + base;
@@ -98,11 +106,20 @@ topk_ef_hist1_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict
       const float4 m = make_float4(gv.x + ev.x, gv.y + ev.y, gv.z + ev.z, gv.w + ev.w);
       *reinterpret_cast<float4*>(e + 4 * i) = m;
       const unsigned k[4] = {key_of(m.x), key_of(m.y), key_of(m.z), key_of(m.w)};
+      const float mm[4] = {m.x, m.y, m.z, m.w};
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
         const unsigned bin = k[q] >> 19;
         atomicAdd(&h[bin], 1u);
-        if (collect) {
+        if (staged) {
+          if (bin >= blo) {
+            const unsigned slot = atomicAdd(cnt, 1u);
+            if (slot < (unsigned)kPredTileCap / 2) {
+              buf[2 * slot] = __float_as_uint(mm[q]);
+              buf[2 * slot + 1] = (unsigned)(t.elem0 + 4 * i + q);
+            }
+          }
+        } else if (collect) {
           above += bin > bhi;
           if (bin - blo <= span) {
             const unsigned slot = atomicAdd(cnt, 1u);
@@ -122,7 +139,15 @@ topk_ef_hist1_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict
       e[i] = m;
       const unsigned kk = key_of(m), bin = kk >> 19;
       atomicAdd(&h[bin], 1u);
-      if (collect) {
+      if (staged) {
+        if (bin >= blo) {
+          const unsigned slot = atomicAdd(cnt, 1u);
+          if (slot < (unsigned)kPredTileCap / 2) {
+            buf[2 * slot] = __float_as_uint(m);
+            buf[2 * slot + 1] = (unsigned)(t.elem0 + i);
+          }
+        }
+      } else if (collect) {
         above += bin > bhi;
         if (bin - blo <= span) {
           const unsigned slot = atomicAdd(cnt, 1u);
@@ -139,20 +164,21 @@ topk_ef_hist1_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict
       __syncthreads();
       if (pend >= 0) {  // copy out the previous tile's keys (its range was published before this barrier)
         unsigned* dst = cand + s_dst[pend];
-        const unsigned n = s_n[pend];
+        const unsigned n = s_n[pend];  // in 4-byte words
         for (unsigned i = threadIdx.x; i < n; i += blockDim.x) dst[i] = s_buf[pend][i];
       }
       if (threadIdx.x == 0) {
+        const unsigned words = staged ? 2u : 1u;  // list slots are keys (one word) or entries (two words)
         unsigned n = s_cnt[cb], start = 0;
-        if (n > (unsigned)kPredTileCap) {
+        if (n * words > (unsigned)kPredTileCap) {
           atomicOr(&seg_flag[seg], 1u);
           n = 0;
         } else if (n) {
           start = atomicAdd(&seg_cand[seg], n);
-          if (start + n > (unsigned)L.cand_cap) { atomicOr(&seg_flag[seg], 1u); n = 0; }
+          if ((start + n) * words > (unsigned)L.cand_cap) { atomicOr(&seg_flag[seg], 1u); n = 0; }
         }
-        s_n[cb] = n;
-        s_dst[cb] = (long long)w * cand_total + L.cand_base + start;
+        s_n[cb] = n * words;
+        s_dst[cb] = (long long)w * cand_total + L.cand_base + (long long)start * words;
         tile_cand[(long long)w * n_tiles + ti] = make_int2((int)start, (int)n);
         tile_cnt[(long long)w * n_tiles + ti].x = s_above[cb];
       }
@@ -239,21 +265,35 @@ topk_pick1_kernel(const DevLayer* __restrict__ layers, const int* __restrict__ m
     unsigned* pw = pred + (long long)lv * W * n_mat + seg;
     const unsigned word = *pw;
     unsigned blo, bhi;
-    const bool had_band = pred_band(word, &blo, &bhi);
+    bool was_staged;
+    const bool had_band = pred_band(word, &blo, &bhi, &was_staged);
     const bool overflow = seg_flag[seg] != 0;
-    const bool fits = hist1[(long long)seg * kBins1 + bin] <= (unsigned)L.cand_cap;
+    const unsigned* hs = hist1 + (long long)seg * kBins1;
+    const bool fits = hs[bin] <= (unsigned)L.cand_cap;
     if (had_band && !overflow && bin >= blo && bin <= bhi) {
-      s.mode = kSelListPred;
+      s.mode = was_staged ? kSelStaged : kSelListPred;
+      if (!was_staged) any_list[2] = 1u;  // word 2: some segment still needs the select pass
     } else {
+      any_list[2] = 1u;
       seg_cand[seg] = 0;  // whatever pass A collected is of no use
       s.mode = fits ? kSelList : kSelDense;
       any_list[fits ? 0 : 1] = 1u;  // word 0: some segment needs the collect pass; word 1: some segment is dense
     }
     // next prediction: narrow the band after an overflow; none for the zero bucket or for buckets that
     // do not fit the list
-    unsigned hw = had_band ? (word >> 16) : 1u;
-    if (had_band && overflow) hw = 0;
-    *pw = (!fits || bin == 0) ? kPredInvalid : (bin | (hw << 16));
+    unsigned hw = had_band ? ((word >> 16) & 0xffu) : 1u;
+    if (had_band && overflow && !was_staged) hw = 0;
+    // staging whole entries pays when few keys lie at or above the band: the entries of buckets >= b1 - hw,
+    // with a margin, must fit half the list (two words each); after a staged overflow keys are collected again
+    long long n_ge = above;
+    for (unsigned b = bin > hw ? bin - hw : 1u; b <= bin; ++b) n_ge += hs[b];
+    // (bit 25, sticky: staging overflowed once for this segment and level -- e.g. a row-sparse layer whose
+    // non-zero rows fill whole tiles -- and is not tried again)
+    const bool no_stage = (word != kPredInvalid && ((word >> 25) & 1u)) || (had_band && overflow && was_staged);
+    const bool stage_next = !no_stage && n_ge * 5 / 2 <= (long long)L.cand_cap &&
+                            n_ge * 3 <= (long long)L.ntiles * (kPredTileCap / 2);
+    *pw = (!fits || bin == 0) ? kPredInvalid
+                              : (bin | (hw << 16) | ((stage_next ? 1u : 0u) << 24) | ((no_stage ? 1u : 0u) << 25));
     sel[seg] = s;
     counts[w * n_layers + l] = k;
   }
@@ -503,13 +543,14 @@ topk_hist_list_kernel(const DevLayer* __restrict__ layers, const int* __restrict
   const int seg = blockIdx.y;
   const Select s = sel[seg];
   if (s.mode == kSelDense) return;
-  const unsigned n = seg_cand[seg];
+  const unsigned n = seg_cand[seg] << (s.mode == kSelStaged ? 1 : 0);  // in 4-byte words
   if (blockIdx.x * kChunk >= n) return;
   for (int b = threadIdx.x; b < kBins; b += blockDim.x) h[b] = 0;
   __syncthreads();
   const DevLayer L = layers[mat_layers[seg % n_mat]];
   const unsigned* keys = cand + (long long)(seg / n_mat) * cand_total + L.cand_base;
   const unsigned prefix = (s.b1 << 12) | s.b2;
+  const bool staged = s.mode == kSelStaged;  // the list holds (value bits, index) pairs instead of keys
   auto count = [&](unsigned kk) {
     if (LEVEL == 2) {
       if ((kk >> 19) == s.b1) atomicAdd(&h[(kk >> 7) & 0xfffu], 1u);
@@ -524,9 +565,15 @@ topk_hist_list_kernel(const DevLayer* __restrict__ layers, const int* __restrict
 #pragma unroll 4
     for (unsigned i = threadIdx.x; i < n4; i += blockDim.x) {
       const uint4 kk = __ldcs(k4 + i);
-      count(kk.x); count(kk.y); count(kk.z); count(kk.w);
+      if (staged) {
+        count(kk.x & 0x7fffffffu); count(kk.z & 0x7fffffffu);
+      } else {
+        count(kk.x); count(kk.y); count(kk.z); count(kk.w);
+      }
     }
-    for (unsigned i = c0 + 4 * n4 + threadIdx.x; i < c1; i += blockDim.x) count(keys[i]);
+    for (unsigned i = c0 + 4 * n4 + threadIdx.x; i < c1; i += blockDim.x)
+      if (!staged) count(keys[i]);
+      else if ((i & 1u) == 0) count(keys[i] & 0x7fffffffu);
   }
   __syncthreads();
   for (int b = threadIdx.x; b < kBins; b += blockDim.x) {
@@ -583,10 +630,11 @@ topk_tile_counts_kernel(const DevLayer* __restrict__ layers, const Tile* __restr
   const Select s = sel[w * n_mat + L.mat];
   if (s.mode != kSelDense) {  // list segment: count the tile's collected keys against the final threshold
     const int2 tc = tile_cand[v];
-    const unsigned* keys = cand + (long long)w * cand_total + L.cand_base + tc.x;
+    const bool staged = s.mode == kSelStaged;
+    const unsigned* keys = cand + (long long)w * cand_total + L.cand_base + (staged ? 2 * tc.x : tc.x);
     int above = 0, ties = 0;
     for (int i = lane; i < tc.y; i += 32) {
-      const unsigned kk = keys[i];
+      const unsigned kk = staged ? (keys[2 * i] & 0x7fffffffu) : keys[i];
       above += kk > s.tau;
       ties += kk == s.tau;
     }
@@ -748,18 +796,97 @@ __device__ __forceinline__ void select_tile(const Tile& t, const DevLayer& L, co
 __global__ void __launch_bounds__(256, 3)
 topk_select_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict__ tiles, int n_tiles, int n_mat,
                    float* __restrict__ err, const Select* __restrict__ sel, const int2* __restrict__ tile_pre,
-                   float* __restrict__ vals, int32_t* __restrict__ idx, long long stride, long long capacity) {
+                   const unsigned* __restrict__ any_select, float* __restrict__ vals, int32_t* __restrict__ idx,
+                   long long stride, long long capacity) {
   __shared__ unsigned wtot[8];
+  if (*any_select == 0) return;  // every segment was served from staged entries
   const int ti = blockIdx.x, w = blockIdx.y;
   const Tile t = tiles[ti];
   const DevLayer L = layers[t.layer];
   if (L.kind != ACC_MATRIX) return;
   const Select s = sel[w * n_mat + L.mat];
+  if (s.mode == kSelStaged) return;
   const int2 pre = tile_pre[(long long)w * n_tiles + ti];
   float* m = err + (long long)w * stride + L.offset + t.elem0;
   const long long seg = (long long)w * capacity + L.seg_off;
   if (t.nelem == kTile) select_tile<true>(t, L, s, pre, m, vals, idx, seg, wtot);
   else select_tile<false>(t, L, s, pre, m, vals, idx, seg, wtot);
+}
+
+// Pass E', staged segments.  One warp per (tile, worker): the tile's staged entries (every element whose key
+// lies in a bucket at or above the predicted band) already hold all candidates, so the kept ones are written
+// from them and M is not read.  Index order inside the tile comes from two 8192-bit maps in shared memory
+// (keys above tau, keys equal to tau) with per-word prefix counts: an entry's rank is the number of set bits
+// below its index.
+__global__ void __launch_bounds__(256)
+topk_finalize_staged_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict__ tiles, int n_tiles,
+                            int n_mat, int W, float* __restrict__ err, const Select* __restrict__ sel,
+                            const int2* __restrict__ tile_pre, const unsigned* __restrict__ cand,
+                            const int2* __restrict__ tile_cand, long long cand_total, float* __restrict__ vals,
+                            int32_t* __restrict__ idx, long long stride, long long capacity) {
+  constexpr int kWords = kTile / 32;  // 256
+  __shared__ unsigned bits_a[8][kWords], bits_t[8][kWords];
+  __shared__ unsigned short pref_a[8][kWords], pref_t[8][kWords];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const long long v = (long long)blockIdx.x * 8 + warp;
+  if (v >= (long long)W * n_tiles) return;
+  const int w = (int)(v / n_tiles), ti = (int)(v % n_tiles);
+  const Tile t = tiles[ti];
+  const DevLayer L = layers[t.layer];
+  if (L.kind != ACC_MATRIX) return;
+  const Select s = sel[w * n_mat + L.mat];
+  if (s.mode != kSelStaged) return;
+  const int2 tc = tile_cand[v];
+  if (tc.y == 0) return;
+  const int2 pre = tile_pre[v];
+  const uint2* ent = reinterpret_cast<const uint2*>(cand + (long long)w * cand_total + L.cand_base) + tc.x;
+  unsigned* ba = bits_a[warp];
+  unsigned* bt = bits_t[warp];
+  for (int i = lane; i < kWords; i += 32) { ba[i] = 0; bt[i] = 0; }
+  __syncwarp();
+  for (int i = lane; i < tc.y; i += 32) {
+    const uint2 e = ent[i];
+    const unsigned kk = e.x & 0x7fffffffu, li = e.y - (unsigned)t.elem0;
+    if (kk > s.tau) atomicOr(&ba[li >> 5], 1u << (li & 31u));
+    else if (kk == s.tau) atomicOr(&bt[li >> 5], 1u << (li & 31u));
+  }
+  __syncwarp();
+  {  // per-word exclusive prefix counts: lane l owns words 8l .. 8l+7
+    unsigned ca = 0, ct = 0;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) { ca += __popc(ba[8 * lane + j]); ct += __popc(bt[8 * lane + j]); }
+    unsigned c = ca | (ct << 16), incl = c;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const unsigned n = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += n;
+    }
+    unsigned run = incl - c;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      pref_a[warp][8 * lane + j] = (unsigned short)(run & 0xffffu);
+      pref_t[warp][8 * lane + j] = (unsigned short)(run >> 16);
+      run += __popc(ba[8 * lane + j]) | (__popc(bt[8 * lane + j]) << 16);
+    }
+  }
+  __syncwarp();
+  const long long seg = (long long)w * capacity + L.seg_off;
+  float* m = err + (long long)w * stride + L.offset;
+  for (int i = lane; i < tc.y; i += 32) {
+    const uint2 e = ent[i];
+    const unsigned kk = e.x & 0x7fffffffu, li = e.y - (unsigned)t.elem0;
+    const bool is_a = kk > s.tau, is_t = kk == s.tau;
+    if (!is_a && !is_t) continue;
+    const unsigned wd = li >> 5, below = (1u << (li & 31u)) - 1u;
+    const int above_before = pre.x + (int)pref_a[warp][wd] + __popc(ba[wd] & below);
+    const int ties_before = pre.y + (int)pref_t[warp][wd] + __popc(bt[wd] & below);
+    if (is_a || ties_before < s.need) {
+      const int pos = above_before + min(ties_before, s.need);
+      vals[seg + pos] = __uint_as_float(e.x);
+      idx[seg + pos] = (int32_t)e.y;
+      m[e.y] = 0.f;
+    }
+  }
 }
 
 // Pass F.  Scatter-decompress and average: one block per tile; the tile of `out` is accumulated in shared
@@ -887,9 +1014,16 @@ cudaError_t launch_topk(acc_ctx* ctx, const float* grads, float* err, const uint
     }
   }
   if (n_mat > 0) {
+    {
+      PhaseTimer pt(ctx, PH_TOPK_FINALIZE_STAGED, s);
+      topk_finalize_staged_kernel<<<(unsigned)(((long long)W * nt + 7) / 8), 256, 0, s>>>(
+          ctx->d_layers, ctx->d_tiles, nt, n_mat, W, err, ctx->d_sel, ctx->d_tile_pre, ctx->d_cand, ctx->d_tile_cand,
+          pl.cand_total, vals, idx, c.worker_stride, pl.capacity);
+    }
     PhaseTimer pt(ctx, PH_TOPK_SELECT, s);
     topk_select_kernel<<<dim3(nt, W), 256, 0, s>>>(ctx->d_layers, ctx->d_tiles, nt, n_mat, err, ctx->d_sel,
-                                                   ctx->d_tile_pre, vals, idx, c.worker_stride, pl.capacity);
+                                                   ctx->d_tile_pre, ctx->d_any_list + 2, vals, idx, c.worker_stride,
+                                                   pl.capacity);
   }
   {
     PhaseTimer pt(ctx, PH_TOPK_DECOMPRESS, s);

@@ -191,7 +191,7 @@ def test_topk_step_bit_exact(W, low_bp, high_bp, pipeline):
         torch.cuda.synchronize()
         H.check_topk_against_oracle(ctx, table, grads, e0, level, vals, idx, counts, out, err, low_bp, high_bp)
         grads, _ = _random_inputs(table, W, 200 + it)
-    assert ctx.last_launch_count() == 13
+    assert ctx.last_launch_count() == 14
     assert ctx.acc_device_status() == 0
 
 
@@ -338,3 +338,33 @@ def test_topk_threshold_prediction_hits_and_misses(pipeline):
         ctx.acc_topk_step(grads, err, level, vals, idx, counts, out)
         torch.cuda.synchronize()
         H.check_topk_against_oracle(ctx, table, grads, e0, level, vals, idx, counts, out, err, 1000, 100)
+
+
+def test_topk_every_selection_path_is_exercised():
+    """All four selection paths give the same (oracle-checked) results; this run makes sure each of them is
+    actually taken: dense (a bucket too fat for a list: the all-zero layer), list (first step, no prediction),
+    predicted list (same gradients again) and staged entries (high compression level on a layer whose kept
+    entries stand far above the rest)."""
+    table = wl.make_table([("zeros", (64, 1024)), ("noise", (256, 1024)), ("spiky", (256, 1024))])
+    W = 2
+    ctx = binding.Context(table, W, topk_low_bp=1000, topk_high_bp=100)
+    g = torch.Generator(device="cuda").manual_seed(9)
+    grads = torch.zeros(W, table.stride, device="cuda")
+    sl = {table.names[l]: s for l, s in table.slices()}
+    grads[:, sl["noise"]] = torch.randn(W, 256 * 1024, generator=g, device="cuda")
+    spiky = 1e-3 * torch.randn(W, 256 * 1024, generator=g, device="cuda")
+    hot = torch.randperm(256 * 1024, generator=g, device="cuda")[:4000]
+    spiky[:, hot] = 5.0 + torch.rand(W, 4000, generator=g, device="cuda")
+    grads[:, sl["spiky"]] = spiky
+    vals, idx, counts = ctx.new_topk_buffers()
+    out = torch.zeros(table.stride, device="cuda")
+    seen = set()
+    for lv in (1, 1, 1, 0, 0, 0, 0):
+        level = torch.full((table.n_layers,), lv, dtype=torch.uint8, device="cuda")
+        err = torch.zeros_like(grads)
+        ctx.acc_topk_step(grads, err, level, vals, idx, counts, out)
+        torch.cuda.synchronize()
+        H.check_topk_against_oracle(ctx, table, grads, torch.zeros_like(grads), level, vals, idx, counts, out, err,
+                                    1000, 100)
+        seen.update(int(p) for p in ctx.acc_topk_last_paths().ravel())
+    assert seen == {0, 1, 2, 3}, seen
