@@ -195,6 +195,7 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=8)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--eager", action="store_true", help="PowerSGD: materialise the error memory every step")
+    ap.add_argument("--no-graphs", action="store_true", help="issue the timed steps call by call instead of as CUDA graphs")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -235,12 +236,17 @@ def main():
 
     step_no = 0
 
-    def run_steps(k, events=None):
+    use_graphs = not args.no_graphs
+
+    def run_steps(k, events=None, graphs=False):
         nonlocal step_no
         for i in range(k):
             if events is not None:
                 events[i][0].record()
-            eng.step(ring[step_no % RING])
+            if graphs:
+                eng.step_graph(step_no % RING)
+            else:
+                eng.step(ring[step_no % RING])
             if events is not None:
                 events[i][1].record()
             step_no += 1
@@ -248,6 +254,8 @@ def main():
     # ---- warm-up, then the timed region (device-resident inputs)
     run_steps(args.warmup)
     barrier()
+    if use_graphs:  # one CUDA graph per gradient buffer and per kind of iteration (with / without regime check)
+        eng.capture_graphs(ring)
     K = args.steps
     ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
     sampler = ClockSampler(local_rank) if rank == 0 else None
@@ -259,7 +267,7 @@ def main():
     t0 = time.time()
     start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     start.record()
-    run_steps(K, ev)
+    run_steps(K, ev, graphs=use_graphs)
     stop.record()
     barrier()
     t1 = time.time()
@@ -337,6 +345,7 @@ def main():
                            "gradient_bytes_per_step": grad_bytes_step,
                            "l2_policy": f"inputs larger than L2: {RING} gradient batches of "
                                         f"{4 * W * table.stride / 1e6:.0f} MB cycled, no flush",
+                           "launch": "CUDA graph replay per step" if use_graphs else "direct calls",
                            "multi_gpu": "independent replicas, no collective"},
                 "clocks": clocks, "e2e": e2e, "gpu_launches": gpu_launches,
                 "roofline": roofline, "cpu_baseline": cpu,

@@ -198,6 +198,7 @@ int acc_create(const acc_config* cfg, void* workspace, size_t workspace_bytes, a
   if (e == cudaSuccess) e = cudaMemset(ctx->d_status, 0, sizeof(int) * 64);
   if (e == cudaSuccess) e = cudaMemset(ctx->d_pending, 0, sizeof(int) * cfg->n_layers);
   if (e == cudaSuccess) e = cudaMemset(ctx->d_pred, 0xff, sizeof(unsigned) * 2 * seg);  // no prediction yet
+  if (e == cudaSuccess) e = prepare_powersgd();
   int dev = 0;
   if (e == cudaSuccess) e = cudaGetDevice(&dev);
   if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, dev);

@@ -125,6 +125,7 @@ cudaError_t launch_detect(acc_ctx* ctx, const double* n2c, double* n2p, float lr
                           uint8_t* level, cudaStream_t s);
 cudaError_t launch_powersgd(acc_ctx* ctx, const float* grads, float* err, float* q, float* p_hat,
                             const uint8_t* level, float* out, float* delta, cudaStream_t s);
+cudaError_t prepare_powersgd();
 cudaError_t launch_powersgd_flush(acc_ctx* ctx, float* err, const float* q, const float* p_hat, cudaStream_t s);
 cudaError_t launch_topk(acc_ctx* ctx, const float* grads, float* err, const uint8_t* level, float* vals,
                         int32_t* idx, int32_t* counts, float* out, float* delta, cudaStream_t s);

@@ -540,6 +540,17 @@ __global__ void psgd_clear_pending_kernel(int* __restrict__ pending, int n_layer
   if (l < n_layers) pending[l] = 0;
 }
 
+// Once per context, at creation (not a stream operation): the pipelined kernels need more than 48 KB of
+// dynamic shared memory.
+cudaError_t prepare_powersgd() {
+  cudaError_t e = cudaFuncSetAttribute(psgd_project_pipe_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       (int)kPipeSmemBytes);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(psgd_project_pipe_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)kPipeSmemBytes);
+  return e;
+}
+
 cudaError_t launch_powersgd(acc_ctx* ctx, const float* grads, float* err, float* q, float* p_hat,
                             const uint8_t* level, float* out, float* delta, cudaStream_t s) {
   const Plan& pl = ctx->plan;
@@ -558,12 +569,10 @@ cudaError_t launch_powersgd(acc_ctx* ctx, const float* grads, float* err, float*
     const int n_mt = (int)pl.mat_tiles.size(), n_vt = (int)pl.vec_tiles.size();
     const int grid = n_mt < ctx->sm_count ? n_mt : ctx->sm_count;
     if (lazy) {
-      cudaFuncSetAttribute(psgd_project_pipe_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPipeSmemBytes);
       psgd_project_pipe_kernel<true><<<grid, kPipeThreads, kPipeSmemBytes, s>>>(
           ctx->d_layers, ctx->d_tiles, ctx->d_mat_tiles, n_mt, ctx->d_vec_tiles, n_vt, grads, err, q, p_hat,
           ctx->d_ppart, ctx->d_pending, out, delta, c.worker_stride, c.n_workers, c.decider, inv_w, ctx->d_status);
     } else {
-      cudaFuncSetAttribute(psgd_project_pipe_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPipeSmemBytes);
       psgd_project_pipe_kernel<false><<<grid, kPipeThreads, kPipeSmemBytes, s>>>(
           ctx->d_layers, ctx->d_tiles, ctx->d_mat_tiles, n_mt, ctx->d_vec_tiles, n_vt, grads, err, q, p_hat,
           ctx->d_ppart, nullptr, out, delta, c.worker_stride, c.n_workers, c.decider, inv_w, ctx->d_status);

@@ -64,6 +64,40 @@ class AccordionStep:
             c.acc_detect_regime(self.norm2_curr, self.norm2_prev, lr_curr, lr_next, self.level, self.delta, stream)
             self.launches += c.last_launch_count()
 
+    def capture_graphs(self, grads_buffers, lr_curr: float = 0.1, lr_next: float = 0.1):
+        """Captures one iteration as CUDA graphs, for each of the given fixed device gradient buffers (the
+        caller refills them, or cycles through them, before every replay): one graph for an ordinary
+        iteration and one for an iteration that ends a detection window (with the norm and regime kernels).
+        Which rank or K a layer gets is decided on the device from ``level``, so the same graphs serve every
+        iteration.  ``step_graph(slot)`` replays the right one.  Every library call is asynchronous and
+        allocation-free, hence capturable."""
+        torch.cuda.synchronize(self.device)
+        saved_t, saved_launches = self.t, self.launches
+        side = torch.cuda.Stream(device=self.device)
+        self._graphs, self._graph_launches = [], []
+        with torch.cuda.stream(side):
+            for grads in grads_buffers:
+                pair, counts = [], []
+                for with_check in (False, True):
+                    g = torch.cuda.CUDAGraph()
+                    self.t = self.check_every - 1 if with_check else 0
+                    before = self.launches
+                    with torch.cuda.graph(g, stream=side):
+                        self.step(grads, lr_curr, lr_next, stream=side)
+                    pair.append(g)
+                    counts.append(self.launches - before)
+                self._graphs.append(pair)
+                self._graph_launches.append(counts)
+        torch.cuda.synchronize(self.device)
+        self.t, self.launches = saved_t, saved_launches
+
+    def step_graph(self, slot: int = 0):
+        """Replays the captured iteration that reads gradient buffer ``slot`` (see ``capture_graphs``)."""
+        self.t += 1
+        which = 1 if self.t % self.check_every == 0 else 0
+        self._graphs[slot][which].replay()
+        self.launches += self._graph_launches[slot][which]
+
     def outputs(self):
         outs = []
         if "powersgd" in self.compressors:
