@@ -115,13 +115,12 @@ def run_reference(args, rank, world):
         return
     from oracle import accordion_oracle as orc
     from paper_2010_16248_b200 import workloads as wl
-    from tests import helpers as H
     w = wl.workload(args.config)
     full = w.table
     li = full.names.index(REF_LAYER) if REF_LAYER in full.names else int(np.argmax(full.kind == wl.MATRIX))
     n, m = int(full.rows[li]), int(full.cols[li])
     sub = wl.make_table([(full.names[li], (n, m))])
-    layers = H.layers_of(sub)
+    layers = [(int(sub.offset[l]), int(sub.rows[l]), int(sub.cols[l]), int(sub.kind[l])) for l in range(sub.n_layers)]
     rng = np.random.default_rng(1234)
     W = w.n_workers
     batches = [rng.standard_normal((W, sub.stride)).astype(np.float32) for _ in range(2)]
