@@ -71,6 +71,7 @@ static int make_plan(const acc_config* cfg, Plan& p) {
     o.ntiles = (int)p.tiles.size() - o.tile0;
     if (d.kind != ACC_MATRIX) continue;
     o.mat = p.n_mat++;
+    p.max_rows = std::max(p.max_rows, d.rows);
     p.mat_layers.push_back(l);
     o.q_row = (int)p.q_rows; p.q_rows += d.cols;
     o.p_row = (int)p.p_rows; p.p_rows += d.rows;
@@ -342,7 +343,8 @@ const char* acc_profile_kernel_name(int32_t i) {
       "topk_ef_hist1_kernel", "topk_pick1_kernel", "topk_hist2_kernel", "topk_pick2_kernel", "topk_hist3_kernel",
       "topk_tile_scan_kernel", "topk_select_kernel", "topk_decompress_kernel", "psgd_flush_kernel",
       "topk_collect_kernel", "topk_pick3_kernel", "topk_tile_counts_kernel",
-      "topk_hist2_list_kernel", "topk_hist3_list_kernel", "topk_finalize_staged_kernel"};
+      "topk_hist2_list_kernel", "topk_hist3_list_kernel", "topk_finalize_staged_kernel",
+      "psgd_orthonormalise_block_kernel"};
   return (i >= 0 && i < PH_COUNT) ? names[i] : "";
 }
 

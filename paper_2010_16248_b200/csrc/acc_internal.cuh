@@ -54,7 +54,7 @@ enum Phase {
   PH_EF = 0, PH_NORM_PARTIAL, PH_NORM_FINAL, PH_DETECT,
   PH_PSGD_PROJECT, PH_PSGD_ORTHO, PH_PSGD_QPARTIAL, PH_PSGD_QREDUCE, PH_PSGD_RESIDUAL,
   PH_TOPK_EF_HIST1, PH_TOPK_PICK1, PH_TOPK_HIST2, PH_TOPK_PICK2, PH_TOPK_HIST3, PH_TOPK_PICK3_SCAN, PH_TOPK_SELECT,
-  PH_TOPK_DECOMPRESS, PH_PSGD_FLUSH, PH_TOPK_COLLECT, PH_TOPK_PICK3, PH_TOPK_TILE_COUNTS, PH_TOPK_HIST2_LIST, PH_TOPK_HIST3_LIST, PH_TOPK_FINALIZE_STAGED,
+  PH_TOPK_DECOMPRESS, PH_PSGD_FLUSH, PH_TOPK_COLLECT, PH_TOPK_PICK3, PH_TOPK_TILE_COUNTS, PH_TOPK_HIST2_LIST, PH_TOPK_HIST3_LIST, PH_TOPK_FINALIZE_STAGED, PH_PSGD_ORTHO_BLOCK,
   PH_COUNT
 };
 
@@ -69,6 +69,7 @@ struct Plan {
   std::vector<int> mat_tiles;    // tile indices that belong to MATRIX layers, in order
   long long q_rows = 0, p_rows = 0, capacity = 0, part_f4 = 0, cand_total = 0, ppart_f4 = 0;
   int n_mat = 0;
+  int max_rows = 0;  // most rows of any MATRIX layer
   // workspace offsets (bytes)
   size_t o_layers = 0, o_col_items = 0, o_tiles = 0, o_mat_layers = 0, o_vec_tiles = 0, o_mat_tiles = 0, o_status = 0,
          o_part = 0, o_ppart = 0, o_pending = 0, o_norm_part = 0, o_hist = 0, o_sel = 0, o_pred = 0, o_cand = 0, o_tile_cand = 0, o_tile_cnt = 0, o_tile_h3 = 0, o_tile_pre = 0,

@@ -9,10 +9,14 @@
 // every access is a fully coalesced, 16-byte aligned float4 whatever the row length, and all blocks carry
 // the same load.  Row structure only enters through the factors: element i of a layer sits in row i / m,
 // column i % m, and the rows a tile cuts are reduced from shared memory afterwards.
+#include <cooperative_groups.h>
+
 #include "acc_async.cuh"
 #include "acc_internal.cuh"
 
 namespace acc {
+
+namespace cg = cooperative_groups;
 
 __device__ __forceinline__ float lowrank_entry(const float4& pv, const float4& qv, int r) {
   float a = pv.x * qv.x;
@@ -364,7 +368,108 @@ __device__ __forceinline__ double block_sum(double v, double* sm) {
   return s;
 }
 
-// Pass 2.  One block per MATRIX layer: modified Gram-Schmidt on the first r columns of P, in place.
+// Pass 2, cluster version.  One thread-block cluster of 8 blocks per MATRIX layer: modified Gram-Schmidt on
+// the first r columns of P.  Every block keeps its eighth of the rows in registers (up to kOrthoRowsPerThread
+// per thread) for all passes; a pass is a block-level sum, an exchange of the eight partial sums through
+// distributed shared memory and one cluster barrier.  The eight partials are added in rank order by every
+// block, so all blocks see the same value and the result does not depend on scheduling.
+constexpr int kOrthoCluster = 8;
+constexpr int kOrthoThreads = 512;
+constexpr int kOrthoRowsPerThread = 12;
+constexpr int kOrthoMaxRows = kOrthoCluster * kOrthoThreads * kOrthoRowsPerThread;  // 49152; beyond: block kernel
+constexpr int kOrthoMinRows = 2048;  // below this one block is faster than a cluster (block barriers are cheaper)
+__host__ __device__ inline bool ortho_by_cluster(int rows) { return rows > kOrthoMinRows && rows <= kOrthoMaxRows; }
+
+__device__ __forceinline__ double cluster_sum(double v, double* sm_warp, double* slots, int phase,
+                                              cg::cluster_group& cluster) {
+  // block-level sum (fixed order), published in this block's slot of the current phase parity
+  v = warp_sum(v);
+  __syncthreads();
+  if ((threadIdx.x & 31) == 0) sm_warp[threadIdx.x >> 5] = v;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double s = 0.0;
+    for (int i = 0; i < kOrthoThreads / 32; ++i) s += sm_warp[i];
+    slots[phase & 1] = s;
+  }
+  cluster.sync();
+  double total = 0.0;
+  for (int r = 0; r < kOrthoCluster; ++r) total += cluster.map_shared_rank(slots, r)[phase & 1];
+  return total;
+}
+
+__global__ void __cluster_dims__(kOrthoCluster, 1, 1) __launch_bounds__(kOrthoThreads)
+psgd_orthonormalise_cluster_kernel(const DevLayer* __restrict__ layers, const int* __restrict__ mat_layers,
+                                   float* __restrict__ p, const float4* __restrict__ p_part,
+                                   const uint8_t* __restrict__ level, int* __restrict__ pending, int rank_low,
+                                   int rank_high, float eps) {
+  __shared__ double sm_warp[kOrthoThreads / 32];
+  __shared__ double slots[2];
+  cg::cluster_group cluster = cg::this_cluster();
+  const int l = mat_layers[blockIdx.x / kOrthoCluster];
+  const DevLayer L = layers[l];
+  if (!ortho_by_cluster(L.rows)) return;  // uniform over the cluster: such layers go to the block kernel
+  const int rank = (int)cluster.block_rank();
+  const int r = level[l] ? rank_low : rank_high;
+  if (pending != nullptr && rank == 0 && threadIdx.x == 0) pending[l] = r;
+  float4* P4 = reinterpret_cast<float4*>(p) + L.p_row;
+  const int per = (L.rows + kOrthoCluster - 1) / kOrthoCluster;
+  const int row_lo = rank * per, row_hi = min(L.rows, row_lo + per);
+  float4 v[kOrthoRowsPerThread];
+#pragma unroll
+  for (int k = 0; k < kOrthoRowsPerThread; ++k) {
+    const int i = row_lo + k * kOrthoThreads + (int)threadIdx.x;
+    v[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (i < row_hi) {
+      // P[i] = sum, in tile order, of the partial rows the project pass left; ranks beyond r keep their value
+      const int first_tile = (i * L.cols) / kTile, last_tile = (i * L.cols + L.cols - 1) / kTile;
+      const float4* pp = p_part + L.ppart_base + (long long)i * L.nslots;
+      float4 acc = pp[0];
+      for (int sl = 1; sl <= last_tile - first_tile; ++sl) {
+        acc.x += pp[sl].x; acc.y += pp[sl].y; acc.z += pp[sl].z; acc.w += pp[sl].w;
+      }
+      const float4 old = P4[i];
+      v[k] = make_float4(acc.x, r > 1 ? acc.y : old.y, r > 2 ? acc.z : old.z, r > 3 ? acc.w : old.w);
+    }
+  }
+  // columns as separate register arrays so that every index below is a compile-time constant
+  float col[ACC_MAX_RANK][kOrthoRowsPerThread];
+#pragma unroll
+  for (int k = 0; k < kOrthoRowsPerThread; ++k) { col[0][k] = v[k].x; col[1][k] = v[k].y; col[2][k] = v[k].z; col[3][k] = v[k].w; }
+  int phase = 0;
+#pragma unroll
+  for (int c = 0; c < ACC_MAX_RANK; ++c) {
+    if (c < r) {  // uniform over the cluster
+#pragma unroll
+      for (int j = 0; j < c; ++j) {
+        double part = 0.0;
+#pragma unroll
+        for (int k = 0; k < kOrthoRowsPerThread; ++k) part += (double)col[j][k] * (double)col[c][k];  // zeros outside the range
+        const float dot = (float)cluster_sum(part, sm_warp, slots, phase++, cluster);
+#pragma unroll
+        for (int k = 0; k < kOrthoRowsPerThread; ++k) col[c][k] = fmaf(-dot, col[j][k], col[c][k]);
+      }
+      double part = 0.0;
+#pragma unroll
+      for (int k = 0; k < kOrthoRowsPerThread; ++k) part += (double)col[c][k] * (double)col[c][k];
+      const double nrm = sqrt(cluster_sum(part, sm_warp, slots, phase++, cluster));
+      const float inv = (float)(1.0 / (nrm + (double)eps));
+#pragma unroll
+      for (int k = 0; k < kOrthoRowsPerThread; ++k) col[c][k] *= inv;
+    }
+  }
+#pragma unroll
+  for (int k = 0; k < kOrthoRowsPerThread; ++k) v[k] = make_float4(col[0][k], col[1][k], col[2][k], col[3][k]);
+#pragma unroll
+  for (int k = 0; k < kOrthoRowsPerThread; ++k) {
+    const int i = row_lo + k * kOrthoThreads + (int)threadIdx.x;
+    if (i < row_hi) P4[i] = v[k];
+  }
+  cluster.sync();  // no block may exit while another still reads its shared memory
+}
+
+// Pass 2, block version, for layers with few rows (or with more than the cluster version holds in registers).
+// One block per MATRIX layer: modified Gram-Schmidt on the first r columns of P, in place.
 __global__ void __launch_bounds__(1024)
 psgd_orthonormalise_kernel(const DevLayer* __restrict__ layers, const int* __restrict__ mat_layers,
                            float* __restrict__ p, const float4* __restrict__ p_part,
@@ -373,6 +478,7 @@ psgd_orthonormalise_kernel(const DevLayer* __restrict__ layers, const int* __res
   __shared__ double sm[32];
   const int l = mat_layers[blockIdx.x];
   const DevLayer L = layers[l];
+  if (ortho_by_cluster(L.rows)) return;  // served by the cluster kernel
   const int r = level[l] ? rank_low : rank_high;
   if (pending != nullptr && threadIdx.x == 0) pending[l] = r;  // lazy mode: this step's residual stays pending
   float* P = p + 4ll * L.p_row;
@@ -589,8 +695,16 @@ cudaError_t launch_powersgd(acc_ctx* ctx, const float* grads, float* err, float*
                                                        c.n_workers, c.decider, inv_w);
   }
   if (pl.n_mat > 0) {
-    {
+    bool any_cluster = false, any_block = false;
+    for (int l : pl.mat_layers) (ortho_by_cluster(pl.layers[l].rows) ? any_cluster : any_block) = true;
+    if (any_cluster) {
       PhaseTimer pt(ctx, PH_PSGD_ORTHO, s);
+      psgd_orthonormalise_cluster_kernel<<<pl.n_mat * kOrthoCluster, kOrthoThreads, 0, s>>>(
+          ctx->d_layers, ctx->d_mat_layers, p_hat, ctx->d_ppart, level, lazy ? ctx->d_pending : nullptr, c.rank_low,
+          c.rank_high, c.gs_eps);
+    }
+    if (any_block) {
+      PhaseTimer pt(ctx, PH_PSGD_ORTHO_BLOCK, s);
       psgd_orthonormalise_kernel<<<pl.n_mat, 1024, 0, s>>>(ctx->d_layers, ctx->d_mat_layers, p_hat, ctx->d_ppart,
                                                           level, lazy ? ctx->d_pending : nullptr, c.rank_low,
                                                           c.rank_high, c.gs_eps);

@@ -368,3 +368,28 @@ def test_topk_every_selection_path_is_exercised():
                                     1000, 100)
         seen.update(int(p) for p in ctx.acc_topk_last_paths().ravel())
     assert seen == {0, 1, 2, 3}, seen
+
+
+@pytest.mark.parametrize("lazy", [0, binding.ACC_FLAG_LAZY_RESIDUAL])
+def test_powersgd_tall_layers_orthonormalisation_paths(lazy):
+    """Gram-Schmidt runs on a thread-block cluster for layers of 2049..49152 rows and on one block otherwise;
+    a table with a layer of each kind (and one beyond the cluster's capacity) against the oracle."""
+    table = wl.make_table([("tall", (3000, 40)), ("b", (7,)), ("huge", (50000, 8)), ("short", (600, 16))])
+    W = 2
+    ctx = binding.Context(table, W, rank_low=4, rank_high=2, flags=lazy)
+    ref = binding.Context(table, W, rank_low=4, rank_high=2)  # eager twin supplies the true error memory
+    grads, err = _random_inputs(table, W, 91)
+    q0 = wl.initial_q(table, 4, seed=5)
+    st = [dict(err=err.clone(), q=c.new_q(q0), p=c.new_p(), out=torch.zeros(table.stride, device="cuda")) for c in (ctx, ref)]
+    for it in range(3):
+        level = torch.tensor([(l + it) % 2 for l in range(table.n_layers)], dtype=torch.uint8, device="cuda")
+        e0, qb = st[1]["err"].clone(), st[1]["q"].clone()
+        for c, s_ in zip((ctx, ref), st):
+            c.acc_powersgd_step(grads, s_["err"], s_["q"], s_["p"], level, s_["out"])
+        torch.cuda.synchronize()
+        H.check_powersgd_against_oracle(ref, table, grads, e0, qb, level, st[1]["out"], st[1]["err"], st[1]["q"],
+                                        st[1]["p"], 4, 2, 1e-8)
+        for name in ("out", "q", "p"):
+            assert torch.equal(st[0][name], st[1][name]), name
+        grads, _ = _random_inputs(table, W, 400 + it)
+    assert ctx.last_launch_count() == 6 and ctx.acc_device_status() == 0
