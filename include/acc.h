@@ -132,6 +132,21 @@ int acc_layer_norms(acc_ctx* ctx, const float* buf, int64_t buf_stride, int32_t 
 int acc_detect_regime(acc_ctx* ctx, const double* norm2_curr, double* norm2_prev, float lr_curr,
                       float lr_next, uint8_t* level, float* delta, void* stream);
 
+/* Variant of the regime test with the norm of the DIFFERENCE of the two accumulated gradients,
+ *   || D_prev - D_curr || >= eta * || D_prev ||,
+ * in place of the difference of their norms that the display equation of Section 4.2 and Algorithm 1 print.
+ * It needs the previous accumulated gradient itself (a second model-sized buffer), which Section 4.2 says the
+ * method does not keep; it is offered because the criterion is sometimes quoted in this form.
+ *   acc_layer_diff_norms:   norm2[l] = sum over layer l of (a - b)^2, fp64, fixed order (a, b: [worker_stride]).
+ *   acc_detect_regime_diff: level as in acc_detect_regime with sqrt(norm2_diff[l]) as the change; then
+ *                           norm2_prev <- norm2_curr, delta_prev <- delta, delta <- 0.
+ * Device pointers: a, b, delta, delta_prev [worker_stride] floats; norm2, norm2_diff, norm2_curr, norm2_prev
+ * [L] doubles; level [L] bytes.                                                                      */
+int acc_layer_diff_norms(acc_ctx* ctx, const float* a, const float* b, double* norm2, void* stream);
+int acc_detect_regime_diff(acc_ctx* ctx, const double* norm2_diff, const double* norm2_curr, double* norm2_prev,
+                           float lr_curr, float lr_next, uint8_t* level, float* delta, float* delta_prev,
+                           void* stream);
+
 /* One PowerSGD step with error feedback (the compressor of Section 5.2, applied per MATRIX layer at
  * rank r = rank_low if level[l] else rank_high), all workers, mean over workers (Section 3):
  *   M_w = g_w + e_w;  P = mean_w M_w Q[:, :r];  P^ = modified Gram-Schmidt(P) (divide by norm + gs_eps);

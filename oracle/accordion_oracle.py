@@ -73,6 +73,31 @@ def detect_regime(norm2_curr, norm2_prev, lr_curr, lr_next, eta):
     return level, np.array(norm2_curr, np.float64, copy=True)
 
 
+def layer_diff_norms2(a, b, layers):
+    """Squared L2 norm of (a - b) per layer."""
+    out = np.zeros(len(layers), np.float64)
+    for l, (off, rows, cols, kind) in enumerate(layers):
+        d = a[off:off + rows * cols].astype(np.float64) - b[off:off + rows * cols].astype(np.float64)
+        out[l] = float(np.sum(d * d))
+    return out
+
+
+def detect_regime_diff(norm2_diff, norm2_curr, norm2_prev, lr_curr, lr_next, eta):
+    """Variant of the criterion with the norm of the DIFFERENCE of the two accumulated gradients,
+    ||D_prev - D_curr|| / ||D_prev|| >= eta (a form in which the criterion is sometimes quoted; the paper's display
+    equation and Algorithm 1 use the difference of the norms, which ``detect_regime`` implements).
+    It needs the previous accumulated gradient itself, not only its norm.  Otherwise as Algorithm 1."""
+    L = len(norm2_curr)
+    level = np.zeros(L, np.uint8)
+    for l in range(L):
+        if norm2_prev[l] < 0.0:
+            level[l] = LOW
+            continue
+        critical = np.sqrt(np.float64(norm2_diff[l])) >= np.float64(eta) * np.sqrt(np.float64(norm2_prev[l]))
+        level[l] = LOW if (critical or lr_next < lr_curr) else HIGH
+    return level, np.array(norm2_curr, np.float64, copy=True)
+
+
 # --------------------------------------------------------------------------- #
 # Error feedback (the "memory term", Section 5.2 / Appendix A)
 # --------------------------------------------------------------------------- #

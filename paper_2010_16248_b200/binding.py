@@ -45,7 +45,8 @@ class acc_config(C.Structure):
 EXPORTS = ["acc_workspace_bytes", "acc_create", "acc_destroy", "acc_factor_layout", "acc_topk_layout",
            "acc_error_feedback", "acc_layer_norms", "acc_detect_regime", "acc_powersgd_step", "acc_topk_step",
            "acc_floats_sent", "acc_last_launch_count", "acc_strerror", "acc_profile_enable", "acc_profile_read",
-           "acc_profile_kernel_count", "acc_profile_kernel_name", "acc_sumsq_static", "acc_powersgd_flush", "acc_device_status", "acc_topk_last_paths"]
+           "acc_profile_kernel_count", "acc_profile_kernel_name", "acc_sumsq_static", "acc_powersgd_flush", "acc_device_status", "acc_topk_last_paths",
+           "acc_layer_diff_norms", "acc_detect_regime_diff"]
 
 _lib = None
 
@@ -87,6 +88,8 @@ def lib() -> C.CDLL:
     L.acc_powersgd_flush.argtypes = [vp, vp, vp, vp, vp]
     L.acc_device_status.argtypes = [vp, C.POINTER(i32)]
     L.acc_topk_last_paths.argtypes = [vp, C.POINTER(i32), i32]
+    L.acc_layer_diff_norms.argtypes = [vp, vp, vp, vp, vp]
+    L.acc_detect_regime_diff.argtypes = [vp, vp, vp, vp, f32, f32, vp, vp, vp, vp]
     for name in EXPORTS:
         if name not in ("acc_floats_sent", "acc_last_launch_count", "acc_strerror", "acc_profile_kernel_count",
                         "acc_profile_kernel_name"):
@@ -203,6 +206,18 @@ class Context:
         self._check(lib().acc_detect_regime(self._h, _ptr(norm2_curr, torch.float64), _ptr(norm2_prev, torch.float64),
                                             float(lr_curr), float(lr_next), _ptr(level, torch.uint8),
                                             _ptr(delta, torch.float32), _stream(stream)), "acc_detect_regime")
+
+    def acc_layer_diff_norms(self, a, b, norm2, stream=None):
+        self._check(lib().acc_layer_diff_norms(self._h, _ptr(a, torch.float32), _ptr(b, torch.float32),
+                                               _ptr(norm2, torch.float64), _stream(stream)), "acc_layer_diff_norms")
+
+    def acc_detect_regime_diff(self, norm2_diff, norm2_curr, norm2_prev, lr_curr, lr_next, level, delta, delta_prev,
+                               stream=None):
+        self._check(lib().acc_detect_regime_diff(self._h, _ptr(norm2_diff, torch.float64),
+                                                 _ptr(norm2_curr, torch.float64), _ptr(norm2_prev, torch.float64),
+                                                 float(lr_curr), float(lr_next), _ptr(level, torch.uint8),
+                                                 _ptr(delta, torch.float32), _ptr(delta_prev, torch.float32),
+                                                 _stream(stream)), "acc_detect_regime_diff")
 
     def acc_powersgd_step(self, grads, err, q, p_hat, level, out, delta=None, stream=None):
         self._check(lib().acc_powersgd_step(self._h, _ptr(grads, torch.float32), _ptr(err, torch.float32),

@@ -252,7 +252,14 @@ int acc_layer_norms(acc_ctx* ctx, const float* buf, int64_t buf_stride, int32_t 
   if (n_bufs > 1 && buf_stride < ctx->cfg.worker_stride) return ACC_EINVAL;
   if (!aligned16(buf) || (n_bufs > 1 && buf_stride % 4 != 0) || (reinterpret_cast<uintptr_t>(norm2) & 7u)) return ACC_EALIGN;
   ctx->last_launches = 0;
-  return finish(launch_layer_norms(ctx, buf, buf_stride, n_bufs, norm2, static_cast<cudaStream_t>(stream)));
+  return finish(launch_layer_norms(ctx, buf, buf_stride, n_bufs, nullptr, norm2, static_cast<cudaStream_t>(stream)));
+}
+
+int acc_layer_diff_norms(acc_ctx* ctx, const float* a, const float* b, double* norm2, void* stream) {
+  if (!ctx || !a || !b || !norm2) return ACC_EINVAL;
+  if (!aligned16(a) || !aligned16(b) || (reinterpret_cast<uintptr_t>(norm2) & 7u)) return ACC_EALIGN;
+  ctx->last_launches = 0;
+  return finish(launch_layer_norms(ctx, a, 0, 1, b, norm2, static_cast<cudaStream_t>(stream)));
 }
 
 int acc_detect_regime(acc_ctx* ctx, const double* norm2_curr, double* norm2_prev, float lr_curr, float lr_next,
@@ -261,8 +268,22 @@ int acc_detect_regime(acc_ctx* ctx, const double* norm2_curr, double* norm2_prev
   if (!aligned16(delta)) return ACC_EALIGN;
   ctx->last_launches = 0;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  cudaError_t e = launch_detect(ctx, norm2_curr, norm2_prev, lr_curr, lr_next, level, s);
+  cudaError_t e = launch_detect(ctx, norm2_curr, norm2_prev, nullptr, lr_curr, lr_next, level, s);
   if (e == cudaSuccess && delta) e = cudaMemsetAsync(delta, 0, sizeof(float) * (size_t)ctx->cfg.worker_stride, s);
+  return finish(e);
+}
+
+int acc_detect_regime_diff(acc_ctx* ctx, const double* norm2_diff, const double* norm2_curr, double* norm2_prev,
+                           float lr_curr, float lr_next, uint8_t* level, float* delta, float* delta_prev,
+                           void* stream) {
+  if (!ctx || !norm2_diff || !norm2_curr || !norm2_prev || !level || !delta || !delta_prev) return ACC_EINVAL;
+  if (!aligned16(delta) || !aligned16(delta_prev)) return ACC_EALIGN;
+  ctx->last_launches = 0;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const size_t bytes = sizeof(float) * (size_t)ctx->cfg.worker_stride;
+  cudaError_t e = launch_detect(ctx, norm2_curr, norm2_prev, norm2_diff, lr_curr, lr_next, level, s);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(delta_prev, delta, bytes, cudaMemcpyDeviceToDevice, s);
+  if (e == cudaSuccess) e = cudaMemsetAsync(delta, 0, bytes, s);
   return finish(e);
 }
 

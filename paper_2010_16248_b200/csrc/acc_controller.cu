@@ -41,21 +41,31 @@ __global__ void __launch_bounds__(256) ef_kernel(const DevLayer* __restrict__ la
 __global__ void __launch_bounds__(256) norm_partial_kernel(const DevLayer* __restrict__ layers,
                                                            const Tile* __restrict__ tiles,
                                                            const float* __restrict__ buf, long long stride,
+                                                           const float* __restrict__ minus,
                                                            double* __restrict__ part, int n_tiles) {
   __shared__ double sm[8];
   const Tile t = tiles[blockIdx.x];
   const int b = blockIdx.y;
-  const float* x = buf + (long long)b * stride + layers[t.layer].offset + t.elem0;
+  const long long base = layers[t.layer].offset + t.elem0;
+  const float* x = buf + (long long)b * stride + base;
+  const float* y = minus != nullptr ? minus + base : nullptr;  // norms of (buf - minus), one buffer only
   double acc = 0.0;
   const int n4 = t.nelem >> 2;
   for (int i = threadIdx.x; i < n4; i += blockDim.x) {
-    const float4 v = ld_stream4(x + 4 * i);
+    float4 v = ld_stream4(x + 4 * i);
+    if (y != nullptr) {
+      const float4 u = ld_stream4(y + 4 * i);
+      v.x -= u.x; v.y -= u.y; v.z -= u.z; v.w -= u.w;
+    }
     acc += (double)v.x * v.x;
     acc += (double)v.y * v.y;
     acc += (double)v.z * v.z;
     acc += (double)v.w * v.w;
   }
-  for (int i = 4 * n4 + threadIdx.x; i < t.nelem; i += blockDim.x) acc += (double)x[i] * x[i];
+  for (int i = 4 * n4 + threadIdx.x; i < t.nelem; i += blockDim.x) {
+    const float v = y != nullptr ? x[i] - y[i] : x[i];
+    acc += (double)v * v;
+  }
   acc = warp_sum(acc);
   if ((threadIdx.x & 31) == 0) sm[threadIdx.x >> 5] = acc;
   __syncthreads();
@@ -78,8 +88,11 @@ __global__ void norm_final_kernel(const DevLayer* __restrict__ layers, const dou
 }
 
 // Algorithm 1 per layer, in product form so that a zero previous norm needs no division.
-__global__ void detect_kernel(const double* __restrict__ n2c, double* __restrict__ n2p, float lr_curr, float lr_next,
-                              double eta, uint8_t* __restrict__ level, int n_layers) {
+// With n2d (squared norms of the difference of the two accumulated gradients) the variant criterion
+// ||D_prev - D_curr|| >= eta ||D_prev|| is used instead of | ||D_prev|| - ||D_curr|| | >= eta ||D_prev||.
+__global__ void detect_kernel(const double* __restrict__ n2c, double* __restrict__ n2p,
+                              const double* __restrict__ n2d, float lr_curr, float lr_next, double eta,
+                              uint8_t* __restrict__ level, int n_layers) {
   const int l = blockIdx.x * blockDim.x + threadIdx.x;
   if (l >= n_layers) return;
   const double cur = n2c[l], prev = n2p[l];
@@ -88,7 +101,8 @@ __global__ void detect_kernel(const double* __restrict__ n2c, double* __restrict
     lv = 1;
   } else {
     const double a = sqrt(prev), b = sqrt(cur);
-    lv = (fabs(a - b) >= eta * a || lr_next < lr_curr) ? 1 : 0;
+    const double change = n2d != nullptr ? sqrt(n2d[l]) : fabs(a - b);
+    lv = (change >= eta * a || lr_next < lr_curr) ? 1 : 0;
   }
   level[l] = lv;
   n2p[l] = cur;
@@ -104,13 +118,13 @@ cudaError_t launch_error_feedback(acc_ctx* ctx, const float* grads, float* err, 
   return cudaGetLastError();
 }
 
-cudaError_t launch_layer_norms(acc_ctx* ctx, const float* buf, long long stride, int n_bufs, double* norm2,
-                               cudaStream_t s) {
+cudaError_t launch_layer_norms(acc_ctx* ctx, const float* buf, long long stride, int n_bufs, const float* minus,
+                               double* norm2, cudaStream_t s) {
   const int nt = (int)ctx->plan.tiles.size();
   {
     PhaseTimer pt(ctx, PH_NORM_PARTIAL, s);
     norm_partial_kernel<<<dim3((unsigned)nt, (unsigned)n_bufs), 256, 0, s>>>(ctx->d_layers, ctx->d_tiles, buf, stride,
-                                                                            ctx->d_norm_part, nt);
+                                                                            minus, ctx->d_norm_part, nt);
   }
   {
     PhaseTimer pt(ctx, PH_NORM_FINAL, s);
@@ -120,12 +134,12 @@ cudaError_t launch_layer_norms(acc_ctx* ctx, const float* buf, long long stride,
   return cudaGetLastError();
 }
 
-cudaError_t launch_detect(acc_ctx* ctx, const double* n2c, double* n2p, float lr_curr, float lr_next, uint8_t* level,
-                          cudaStream_t s) {
+cudaError_t launch_detect(acc_ctx* ctx, const double* n2c, double* n2p, const double* n2d, float lr_curr,
+                          float lr_next, uint8_t* level, cudaStream_t s) {
   const int L = ctx->cfg.n_layers;
   {
     PhaseTimer pt(ctx, PH_DETECT, s);
-    detect_kernel<<<(L + 127) / 128, 128, 0, s>>>(n2c, n2p, lr_curr, lr_next, (double)ctx->cfg.eta, level, L);
+    detect_kernel<<<(L + 127) / 128, 128, 0, s>>>(n2c, n2p, n2d, lr_curr, lr_next, (double)ctx->cfg.eta, level, L);
   }
   return cudaGetLastError();
 }

@@ -120,10 +120,10 @@ namespace acc {
 // Kernel launchers (one per translation unit).  Each returns a cudaError_t from cudaGetLastError and
 // adds the number of kernels it launched to ctx->last_launches.
 cudaError_t launch_error_feedback(acc_ctx* ctx, const float* grads, float* err, float* delta, cudaStream_t s);
-cudaError_t launch_layer_norms(acc_ctx* ctx, const float* buf, long long stride, int n_bufs, double* norm2,
-                               cudaStream_t s);
-cudaError_t launch_detect(acc_ctx* ctx, const double* n2c, double* n2p, float lr_curr, float lr_next,
-                          uint8_t* level, cudaStream_t s);
+cudaError_t launch_layer_norms(acc_ctx* ctx, const float* buf, long long stride, int n_bufs, const float* minus,
+                               double* norm2, cudaStream_t s);
+cudaError_t launch_detect(acc_ctx* ctx, const double* n2c, double* n2p, const double* n2d, float lr_curr,
+                          float lr_next, uint8_t* level, cudaStream_t s);
 cudaError_t launch_powersgd(acc_ctx* ctx, const float* grads, float* err, float* q, float* p_hat,
                             const uint8_t* level, float* out, float* delta, cudaStream_t s);
 cudaError_t prepare_powersgd();

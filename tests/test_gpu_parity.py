@@ -8,7 +8,7 @@ import pytest
 import torch
 
 from oracle import accordion_oracle as orc
-from paper_2010_16248_b200 import binding, workloads as wl
+from paper_2010_16248_b200 import binding, pipeline, workloads as wl
 from tests import helpers as H
 
 pytestmark = pytest.mark.gpu
@@ -393,3 +393,84 @@ def test_powersgd_tall_layers_orthonormalisation_paths(lazy):
             assert torch.equal(st[0][name], st[1][name]), name
         grads, _ = _random_inputs(table, W, 400 + it)
     assert ctx.last_launch_count() == 6 and ctx.acc_device_status() == 0
+
+
+def test_difference_criterion_variant_matches_oracle():
+    table = _table_mixed()
+    ctx = binding.Context(table, 1, eta=0.5)
+    layers = H.layers_of(table)
+    g = torch.Generator(device="cuda").manual_seed(12)
+    prev = torch.zeros(table.stride, device="cuda")
+    curr = torch.zeros(table.stride, device="cuda")
+    for l, sl in table.slices():
+        base = torch.randn(sl.stop - sl.start, generator=g, device="cuda")
+        prev[sl] = base
+        # per layer a different relation: scaled copy, rotated (sign-flipped half), small perturbation
+        kind = l % 3
+        if kind == 0:
+            curr[sl] = base * (0.4 + 0.1 * l)
+        elif kind == 1:
+            flipped = base.clone(); flipped[::2] *= -1.0
+            curr[sl] = flipped
+        else:
+            curr[sl] = base + 0.1 * torch.randn(sl.stop - sl.start, generator=g, device="cuda")
+    L = table.n_layers
+    d2 = torch.zeros(L, dtype=torch.float64, device="cuda")
+    n2c = torch.zeros(L, dtype=torch.float64, device="cuda")
+    n2p = torch.zeros(L, dtype=torch.float64, device="cuda")
+    ctx.acc_layer_diff_norms(prev, curr, d2)
+    ctx.acc_layer_norms(curr, 1, n2c)
+    ctx.acc_layer_norms(prev, 1, n2p)
+    level = torch.full((L,), 9, dtype=torch.uint8, device="cuda")
+    delta, delta_prev = curr.clone(), prev.clone()
+    n2p_before = n2p.clone()
+    ctx.acc_detect_regime_diff(d2, n2c, n2p, 0.1, 0.1, level, delta, delta_prev)
+    torch.cuda.synchronize()
+    ph, ch = prev.cpu().numpy(), curr.cpu().numpy()
+    want_d2 = orc.layer_diff_norms2(ph, ch, layers)
+    assert np.allclose(d2.cpu().numpy(), want_d2, rtol=1e-6, atol=0)   # fp32 subtraction on the device
+    want, want_prev = orc.detect_regime_diff(d2.cpu().numpy(), n2c.cpu().numpy(), n2p_before.cpu().numpy(), 0.1, 0.1,
+                                             np.float32(0.5))
+    assert np.array_equal(level.cpu().numpy(), want) and 0 < want.sum() < L
+    assert np.array_equal(n2p.cpu().numpy(), want_prev)
+    assert torch.equal(delta_prev, curr) and float(delta.abs().max()) == 0.0
+    # the rotated layers are critical under this variant but not under Algorithm 1
+    lv1 = torch.zeros(L, dtype=torch.uint8, device="cuda")
+    ctx.acc_detect_regime(n2c, n2p_before.clone(), 0.1, 0.1, lv1)
+    torch.cuda.synchronize()
+    assert int(level[1]) == 1 and int(lv1[1]) == 0
+
+
+def test_checkpoint_resume_is_bit_identical():
+    """State of the path = caller buffers (error memories, Q, P^, accumulator, norms, levels).  Running 2k
+    iterations must equal k iterations + copying the state into a new context + k iterations.  In lazy mode
+    the residual pending inside the context is materialised with acc_powersgd_flush before the copy."""
+    w = wl.workload(5, scale=16)
+    table, W = w.table, w.n_workers
+    stream = wl.GradientStream(w, device="cuda")
+    names = ("level", "delta", "norm2_prev", "err_psgd", "q", "p_hat", "out_psgd", "err_topk", "out_topk")
+
+    def engine():
+        return pipeline.AccordionStep(table, W, w.compressors, w.rank_low, w.rank_high, w.topk_low_bp,
+                                      w.topk_high_bp, w.eta, 1e-8, 4, lazy_residual=True)
+
+    k = 6
+    full = engine()
+    for t in range(2 * k):
+        full.step(stream.grads(t))
+    first = engine()
+    for t in range(k):
+        first.step(stream.grads(t))
+    first.ctx.acc_powersgd_flush(first.err_psgd, first.q, first.p_hat)
+    torch.cuda.synchronize()
+    second = engine()
+    for n in names:
+        getattr(second, n).copy_(getattr(first, n))
+    second.t = first.t
+    for t in range(k, 2 * k):
+        second.step(stream.grads(t))
+    full.ctx.acc_powersgd_flush(full.err_psgd, full.q, full.p_hat)
+    second.ctx.acc_powersgd_flush(second.err_psgd, second.q, second.p_hat)
+    torch.cuda.synchronize()
+    for n in names:
+        assert torch.equal(getattr(full, n), getattr(second, n)), n

@@ -53,6 +53,33 @@ def test_detector_scale_invariance_and_per_layer_independence():
     assert 0 < l1.sum() < 50
 
 
+def test_difference_criterion_truth_table_and_contrast_with_algorithm1():
+    """The norm-of-difference variant on hand-computed vectors; the rotated case separates the two readings:
+    equal norms (Algorithm 1: not critical) but a large difference (variant: critical)."""
+    table = wl.make_table([("a", (2,)), ("b", (2,)), ("c", (2,)), ("d", (2,))])
+    layers = _layers(table)
+    prev = np.zeros(table.stride, np.float32)
+    curr = np.zeros(table.stride, np.float32)
+    vec = {0: ((1, 0), (0.5, 0)),     # ||diff|| = 0.5 = eta * 1      -> LOW (>=)
+           1: ((1, 0), (0.75, 0)),    # 0.25 < 0.5                    -> HIGH
+           2: ((1, 0), (0, 1)),       # rotated: sqrt(2) >= 0.5       -> LOW, while the norms are equal
+           3: ((0, 0), (0, 0))}       # zero previous gradient        -> LOW (0 >= 0)
+    for l, (p, c) in vec.items():
+        off = layers[l][0]
+        prev[off:off + 2], curr[off:off + 2] = p, c
+    d2 = orc.layer_diff_norms2(prev, curr, layers)
+    assert np.allclose(d2, [0.25, 0.0625, 2.0, 0.0])
+    n2p, n2c = orc.layer_norms2(prev, layers), orc.layer_norms2(curr, layers)
+    lv, new_prev = orc.detect_regime_diff(d2, n2c, n2p, 0.1, 0.1, 0.5)
+    assert list(lv) == [1, 0, 1, 1] and np.array_equal(new_prev, n2c)
+    lv0, _ = orc.detect_regime(n2c, n2p, 0.1, 0.1, 0.5)
+    assert list(lv0) == [1, 0, 0, 1]                      # Algorithm 1 does not see the rotation
+    lv, _ = orc.detect_regime_diff(d2, n2c, -np.ones(4), 0.1, 0.1, 0.5)
+    assert list(lv) == [1, 1, 1, 1]                       # no previous window
+    lv, _ = orc.detect_regime_diff(d2, n2c, n2p, 0.1, 0.05, 0.5)
+    assert list(lv) == [1, 1, 1, 1]                       # learning-rate decay
+
+
 def test_layer_norms_closed_form_and_library():
     table = wl.make_table([("a", (3, 5)), ("b", (7,)), ("c", (4, 4))])
     layers = _layers(table)
