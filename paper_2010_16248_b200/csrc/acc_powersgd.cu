@@ -560,6 +560,44 @@ psgd_qpartial_kernel(const DevLayer* __restrict__ layers, const ColItem* __restr
   else qpart_cols<1>(it, L, mbar, P4, part);
 }
 
+// Pass 5, lazy mode (out = A only).  Same items as the Q-partial pass: a thread owns `vec` adjacent columns,
+// keeps their rows of Q' in registers and walks the slab's rows, so the factor tables are read once per
+// (slab, column) instead of once per element; entries use the same lowrank_entry as every other pass.
+template <int VEC>
+__device__ __forceinline__ void decompress_cols(const ColItem& it, const DevLayer& L, const float4* __restrict__ Q4,
+                                                const float4* __restrict__ P4, float* __restrict__ out, int r) {
+  using V = typename VecT<VEC>::type;
+  const int col = it.col0 + (int)threadIdx.x * VEC;
+  if (col >= L.cols) return;
+  float4 qv[VEC];
+#pragma unroll
+  for (int e = 0; e < VEC; ++e) qv[e] = __ldg(Q4 + col + e);
+  float* base = out + L.offset + (long long)it.row0 * L.cols + col;
+  const float4* pr = P4 + it.row0;
+#pragma unroll 8
+  for (int i = 0; i < it.nrows; ++i) {
+    const float4 pv = __ldg(pr + i);
+    float a[VEC];
+#pragma unroll
+    for (int e = 0; e < VEC; ++e) a[e] = lowrank_entry(pv, qv[e], r);
+    __stcs(reinterpret_cast<V*>(base + (long long)i * L.cols), *reinterpret_cast<const V*>(a));
+  }
+}
+
+__global__ void __launch_bounds__(kColBlockThreads)
+psgd_decompress_kernel(const DevLayer* __restrict__ layers, const ColItem* __restrict__ items,
+                       const float* __restrict__ q, const float* __restrict__ p, const uint8_t* __restrict__ level,
+                       float* __restrict__ out, int rank_low, int rank_high) {
+  const ColItem it = items[blockIdx.x];
+  const DevLayer L = layers[it.layer];
+  const int r = level[it.layer] ? rank_low : rank_high;
+  const float4* Q4 = reinterpret_cast<const float4*>(q) + L.q_row;
+  const float4* P4 = reinterpret_cast<const float4*>(p) + L.p_row;
+  if (L.vec == 4) decompress_cols<4>(it, L, Q4, P4, out, r);
+  else if (L.vec == 2) decompress_cols<2>(it, L, Q4, P4, out, r);
+  else decompress_cols<1>(it, L, Q4, P4, out, r);
+}
+
 // Pass 4.  Sums the slab partials of 32 columns in a fixed order and stores the first r ranks of Q'.
 __global__ void __launch_bounds__(256)
 psgd_qreduce_kernel(const DevLayer* __restrict__ layers, const int* __restrict__ mat_layers,
@@ -724,9 +762,8 @@ cudaError_t launch_powersgd(acc_ctx* ctx, const float* grads, float* err, float*
     {
       PhaseTimer pt(ctx, PH_PSGD_RESIDUAL, s);
       if (lazy)
-        psgd_residual_kernel<4, true, false><<<nt, 256, 0, s>>>(ctx->d_layers, ctx->d_tiles, err, q, p_hat, level,
-                                                                nullptr, out, c.worker_stride, c.n_workers,
-                                                                c.rank_low, c.rank_high);
+        psgd_decompress_kernel<<<(unsigned)pl.col_items.size(), kColBlockThreads, 0, s>>>(
+            ctx->d_layers, ctx->d_col_items, q, p_hat, level, out, c.rank_low, c.rank_high);
       else
         psgd_residual_kernel<4, true, true><<<nt, 256, 0, s>>>(ctx->d_layers, ctx->d_tiles, err, q, p_hat, level,
                                                                nullptr, out, c.worker_stride, c.n_workers,
