@@ -214,28 +214,34 @@ __device__ void pick_from_top(const unsigned* __restrict__ hist, int nbins, long
   *above = cum;
 }
 
-// Block-parallel version for the 4096-bin levels: each of 256 threads owns 16 consecutive bins.
+// Block-parallel version for the 4096-bin levels: each of 256 threads owns 16 consecutive bins; a suffix scan
+// over the threads' sums finds the thread whose bins hold the `want`-th largest key, and that thread walks
+// its own 16 counters.  (want >= 1 and the histogram holds at least `want` keys.)
 __device__ void pick_from_top_block(const unsigned* __restrict__ hist, long long want, unsigned* bin,
                                     long long* above, unsigned* sm_sums) {
   const int tid = threadIdx.x;
+  unsigned c[16];
   unsigned s = 0;
-  for (int i = 0; i < 16; ++i) s += hist[tid * 16 + i];
+#pragma unroll
+  for (int i = 0; i < 16; ++i) { c[i] = hist[tid * 16 + i]; s += c[i]; }
   sm_sums[tid] = s;
+  if (tid == 0) { *bin = 0; *above = 0; }
   __syncthreads();
-  if (tid == 0) {
-    long long cum = 0;
-    int t = 255;
-    for (; t > 0; --t) {
-      if (cum + sm_sums[t] >= want) break;
-      cum += sm_sums[t];
+  for (int o = 1; o < 256; o <<= 1) {  // inclusive suffix sums: sm_sums[t] = keys in the bins of threads t..255
+    const unsigned v = tid + o < 256 ? sm_sums[tid + o] : 0u;
+    __syncthreads();
+    sm_sums[tid] += v;
+    __syncthreads();
+  }
+  const long long incl = sm_sums[tid], excl = incl - s;
+  if (excl < want && want <= incl) {
+    long long cum = excl;
+    int b = 15;
+    for (; b > 0; --b) {
+      if (cum + c[b] >= want) break;
+      cum += c[b];
     }
-    int b = t * 16 + 15;
-    for (; b > t * 16; --b) {
-      const long long c = hist[b];
-      if (cum + c >= want) break;
-      cum += c;
-    }
-    *bin = (unsigned)b;
+    *bin = (unsigned)(tid * 16 + b);
     *above = cum;
   }
   __syncthreads();
