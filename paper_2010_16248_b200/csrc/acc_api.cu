@@ -78,7 +78,7 @@ static int make_plan(const acc_config* cfg, Plan& p) {
     o.k_low = topk_count(size, cfg->topk_low_bp);
     o.k_high = topk_count(size, cfg->topk_high_bp);
     o.seg_off = p.capacity; p.capacity += o.k_low;
-    o.cand_cap = (int)std::max<long long>(64, (size / 8 + 3) / 4 * 4);
+    o.cand_cap = (int)std::max<long long>(64, (size / 4 + 3) / 4 * 4);
     o.cand_base = p.cand_total; p.cand_total += o.cand_cap;
     // row slabs of the row-wise passes: about kRowSlabElems elements per worker, whole rows,
     // a multiple of 8 rows (one row per warp of a 256-thread block) where the layer allows it
@@ -118,7 +118,7 @@ static int make_plan(const acc_config* cfg, Plan& p) {
   take(sizeof(unsigned) * 64);   // "some segment needs the collect pass" flag, likewise
   p.hist_bytes = o - p.o_hist;
   p.o_sel = take(sizeof(Select) * seg);
-  p.o_pred = take(sizeof(unsigned) * 2 * seg);
+  p.o_pred = take(sizeof(unsigned) * 4 * seg);  // [2] prediction words, [2] last buckets, per level
   p.o_cand = take(sizeof(unsigned) * (size_t)W * std::max<long long>(1, p.cand_total));
   p.o_tile_cand = take(sizeof(int2) * (size_t)W * nt);
   p.o_tile_cnt = take(sizeof(int2) * (size_t)W * nt);
@@ -198,7 +198,7 @@ int acc_create(const acc_config* cfg, void* workspace, size_t workspace_bytes, a
   up(ctx->d_mat_tiles, p.mat_tiles.data(), sizeof(int) * p.mat_tiles.size());
   if (e == cudaSuccess) e = cudaMemset(ctx->d_status, 0, sizeof(int) * 64);
   if (e == cudaSuccess) e = cudaMemset(ctx->d_pending, 0, sizeof(int) * cfg->n_layers);
-  if (e == cudaSuccess) e = cudaMemset(ctx->d_pred, 0xff, sizeof(unsigned) * 2 * seg);  // no prediction yet
+  if (e == cudaSuccess) e = cudaMemset(ctx->d_pred, 0xff, sizeof(unsigned) * 4 * seg);  // no prediction yet
   if (e == cudaSuccess) e = prepare_powersgd();
   int dev = 0;
   if (e == cudaSuccess) e = cudaGetDevice(&dev);

@@ -27,7 +27,8 @@ namespace acc {
 
 __device__ __forceinline__ unsigned key_of(float v) { return __float_as_uint(v) & 0x7fffffffu; }
 
-// A prediction word: level-1 bucket of the threshold at the segment's last step at this level (bits 0-15),
+// A prediction word: level-1 bucket expected for the threshold, extrapolated from the segment's last two steps
+// at this level (bits 0-15),
 // the half-width in buckets of the band collected around it (bits 16-23), and whether the next pass A may
 // stage whole entries instead of keys (bit 24, see below; bit 25 forbids it for good).
 constexpr unsigned kPredInvalid = 0xffffffffu;
@@ -294,12 +295,24 @@ topk_pick1_kernel(const DevLayer* __restrict__ layers, const int* __restrict__ m
     long long n_ge = above;
     for (unsigned b = bin > hw ? bin - hw : 1u; b <= bin; ++b) n_ge += hs[b];
     // (bit 25, sticky: staging overflowed once for this segment and level -- e.g. a row-sparse layer whose
-    // non-zero rows fill whole tiles -- and is not tried again)
-    const bool no_stage = (word != kPredInvalid && ((word >> 25) & 1u)) || (had_band && overflow && was_staged);
+    // non-zero rows fill whole tiles -- and is not tried again
+    // -- only when the prediction itself was right: a band that lay too low overflows for that reason alone)
+    const bool no_stage = (word != kPredInvalid && ((word >> 25) & 1u)) ||
+                          (had_band && overflow && was_staged && bin >= blo && bin <= bhi);
     const bool stage_next = !no_stage && n_ge * 5 / 2 <= (long long)L.cand_cap &&
-                            n_ge * 3 <= (long long)L.ntiles * (kPredTileCap / 2);
+                            n_ge * 3 / 2 <= (long long)L.ntiles * (kPredTileCap / 2);
+    // the band is centred on the bucket extrapolated from the last two steps at this level: under error
+    // feedback the threshold drifts steadily (it climbs for tens of steps after a switch to the high level)
+    unsigned* lb = pred + (long long)(2 + lv) * W * n_mat + seg;
+    const unsigned last = *lb;
+    int drift = last != kPredInvalid ? (int)bin - (int)last : 0;
+    drift = drift < -3 ? -3 : drift > 6 ? 6 : drift;
+    int centre = (int)bin + drift;
+    centre = centre < 1 ? 1 : centre > kBins1 - 1 ? kBins1 - 1 : centre;
+    *lb = bin;
     *pw = (!fits || bin == 0) ? kPredInvalid
-                              : (bin | (hw << 16) | ((stage_next ? 1u : 0u) << 24) | ((no_stage ? 1u : 0u) << 25));
+                              : ((unsigned)centre | (hw << 16) | ((stage_next ? 1u : 0u) << 24) |
+                                 ((no_stage ? 1u : 0u) << 25));
     sel[seg] = s;
     counts[w * n_layers + l] = k;
   }
