@@ -9,6 +9,9 @@ Precision: fp64 from fp32 inputs everywhere, except the TopK error-feedback add,
 which is one fp32 IEEE add because the packed values and every later selection
 are compared bit for bit.
 
+Besides the compression step the file holds the two extensions that follow it in the training
+loop: the optimiser tail (Nesterov momentum) and the batch-size mode of the controller.
+
 Conventions.  ``layers`` is a sequence of ``(offset, rows, cols, kind)`` with
 ``kind`` 0 = MATRIX (row-major ``rows x cols`` view: convolution weights as
 ``out x (in*k*k)``, the view that reproduces the "Data Sent" columns of Tables
@@ -259,3 +262,75 @@ def floats_sent_per_iteration(layers, level, compressor, n_workers, rank_low=2, 
         else:
             raise ValueError(compressor)
     return total
+
+
+# --------------------------------------------------------------------------- #
+# Optimiser tail (Appendix A, Table "Hyperparameters": Nesterov momentum 0.9)
+# --------------------------------------------------------------------------- #
+def sgd_nesterov(params, mom, d, layers, lr, momentum, weight_decay=0.0):
+    """One SGD step with Nesterov momentum on every layer, from the averaged (decompressed) gradient ``d``:
+
+        d' = d + weight_decay * x;   u <- momentum * u + d';   x <- x - lr * (d' + momentum * u)
+
+    (the paper names the optimiser and the momentum only; this is the usual statement of it, with no
+    dampening, and weight decay -- which the paper does not list -- added to the gradient when non-zero).
+    Elements outside the layers (padding) are left alone.  Returns new (params, mom) in fp64."""
+    x = np.array(params, np.float64, copy=True)
+    u = np.array(mom, np.float64, copy=True)
+    for (off, rows, cols, kind) in layers:
+        sl = slice(off, off + rows * cols)
+        dd = d[sl].astype(np.float64) + np.float64(weight_decay) * x[sl]
+        u[sl] = np.float64(momentum) * u[sl] + dd
+        x[sl] = x[sl] - np.float64(lr) * (dd + np.float64(momentum) * u[sl])
+    return x, u
+
+
+# --------------------------------------------------------------------------- #
+# Batch-size mode (Section 4.2, last paragraph before "Computational and memory overhead";
+# Section 5.1 "Hyperparameters"; Appendix A "Additional Details for Batch Size experiment")
+# --------------------------------------------------------------------------- #
+def batch_accumulate(acc, grads_micro, layers, first):
+    """Large batches are simulated by several backward passes whose gradients are added up before anything
+    is communicated (Appendix A): acc_w <- (0 if first else acc_w) + g_w for every worker and layer."""
+    W = grads_micro.shape[0]
+    a = np.array(acc, np.float64, copy=True)
+    for (off, rows, cols, kind) in layers:
+        sl = slice(off, off + rows * cols)
+        for w in range(W):
+            a[w, sl] = (0.0 if first else a[w, sl]) + grads_micro[w, sl].astype(np.float64)
+    return a
+
+
+def batch_average(acc, n_accum, layers):
+    """Uncompressed exchange of the accumulated gradients (all-reduce, Section 5.1):
+    out = (1 / (W * n_accum)) * sum_w acc_w, the mean over workers of the mean over the micro-batches."""
+    W, stride = acc.shape
+    out = np.zeros(stride, np.float64)
+    for (off, rows, cols, kind) in layers:
+        sl = slice(off, off + rows * cols)
+        s = np.zeros(rows * cols, np.float64)
+        for w in range(W):
+            s += acc[w, sl].astype(np.float64)
+        out[sl] = s / (W * n_accum)
+    return out
+
+
+def detect_batch(norm2_layers, norm2_prev, lr_curr, lr_next, eta, b_curr, b_low, b_high):
+    """Algorithm 1 at the granularity of the whole model (batch size is one setting for all layers): the
+    statistic is the norm of the whole accumulated gradient, ||D||^2 = sum over layers of ||D[l]||^2; the
+    small batch B_low takes the place of the low compression level and B_high of the high one.  The batch
+    size is only ever increased (Appendix A), so a critical regime found while already at B_high leaves
+    it there.  The learning rate scales in the same ratio as the batch size (Section 5.1).
+
+    ``norm2_prev`` < 0 means "no earlier window".  Returns (b_next, lr_scale, new norm2_prev) where
+    lr_scale = b_next / b_low multiplies the learning rate that belongs to B_low."""
+    curr = float(np.sum(np.asarray(norm2_layers, np.float64)))
+    if norm2_prev < 0.0:
+        critical = True
+    else:
+        a = np.sqrt(np.float64(norm2_prev))
+        b = np.sqrt(np.float64(curr))
+        critical = bool(abs(a - b) >= np.float64(eta) * a) or (lr_next < lr_curr)
+    want = b_low if critical else b_high
+    b_next = max(int(b_curr), int(want))
+    return b_next, float(b_next) / float(b_low), curr

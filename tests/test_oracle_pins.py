@@ -387,3 +387,100 @@ def test_data_sent_matches_tables():
             per_it = orc.floats_sent_per_iteration(layers, [1] * L, "topk", 4, topk_low_bp=1000)
             got = per_it * iters / 1e9
             assert abs(got - value) / value < 1e-3, (got, value)
+
+
+# ------------------------------------------------------------------ optimiser tail
+def _toy_table():
+    return wl.make_table([("w0", (6, 5)), ("b0", (7,)), ("w1", (3, 9))])
+
+
+@pytest.mark.parametrize("wd", [0.0, 5e-4])
+def test_sgd_nesterov_matches_library_optimiser(wd):
+    import torch
+    table = _toy_table()
+    layers = _layers(table)
+    rng = np.random.default_rng(3)
+    x0 = rng.standard_normal(table.stride)
+    xs, us = x0.copy(), np.zeros(table.stride)
+    ts = [torch.tensor(x0[o:o + r * c].copy(), dtype=torch.float64, requires_grad=True) for (o, r, c, k) in layers]
+    opt = torch.optim.SGD(ts, lr=0.1, momentum=0.9, nesterov=True, weight_decay=wd)
+    for step in range(4):
+        d = rng.standard_normal(table.stride)
+        xs, us = orc.sgd_nesterov(xs, us, d, layers, 0.1, 0.9, wd)
+        for t, (o, r, c, k) in zip(ts, layers):
+            t.grad = torch.tensor(d[o:o + r * c].copy(), dtype=torch.float64)
+        opt.step()
+        for t, (o, r, c, k) in zip(ts, layers):
+            np.testing.assert_allclose(xs[o:o + r * c], t.detach().numpy(), rtol=1e-12, atol=1e-14)
+    covered = np.zeros(table.stride, bool)
+    for (o, r, c, k) in layers:
+        covered[o:o + r * c] = True
+    assert np.array_equal(xs[~covered], x0[~covered])  # padding untouched
+    assert np.all(us[~covered] == 0.0)
+
+
+def test_sgd_nesterov_closed_form_constant_gradient():
+    table = wl.make_table([("w", (4, 4))])
+    layers = _layers(table)
+    g = np.full(table.stride, 2.0)
+    x, u = np.zeros(table.stride), np.zeros(table.stride)
+    lr, mu = 0.25, 0.5
+    want_x = 0.0
+    for t in range(1, 6):
+        x, u = orc.sgd_nesterov(x, u, g, layers, lr, mu)
+        want_u = 2.0 * (1.0 - mu ** t) / (1.0 - mu)  # geometric sum
+        want_x -= lr * (2.0 + mu * want_u)
+        assert np.allclose(u[:16], want_u, rtol=1e-14)
+        assert np.allclose(x[:16], want_x, rtol=1e-14)
+    # momentum 0 is plain gradient descent
+    x, u = orc.sgd_nesterov(np.ones(table.stride), np.zeros(table.stride), g, layers, 0.1, 0.0)
+    assert np.allclose(x[:16], 1.0 - 0.2) and np.allclose(u[:16], 2.0)
+
+
+# ------------------------------------------------------------------ batch-size mode
+def test_batch_accumulate_and_average_equal_the_mean_over_all_micro_batches():
+    table = _toy_table()
+    layers = _layers(table)
+    rng = np.random.default_rng(5)
+    W, n_accum = 3, 4
+    micro = rng.standard_normal((n_accum, W, table.stride)).astype(np.float32)
+    acc = rng.standard_normal((W, table.stride))  # stale content: the first micro-batch must overwrite it
+    for j in range(n_accum):
+        acc = orc.batch_accumulate(acc, micro[j], layers, first=(j == 0))
+    out = orc.batch_average(acc, n_accum, layers)
+    want = micro.astype(np.float64).mean(axis=(0, 1))
+    for (o, r, c, k) in layers:
+        np.testing.assert_allclose(out[o:o + r * c], want[o:o + r * c], rtol=1e-13, atol=1e-15)
+        np.testing.assert_allclose(acc[:, o:o + r * c], micro.astype(np.float64).sum(axis=0)[:, o:o + r * c],
+                                   rtol=1e-13, atol=1e-15)
+
+
+def test_detect_batch_truth_table():
+    n2 = np.array([9.0, 16.0])  # whole-model norm 5
+    # (prev norm, lr_curr, lr_next, b_curr) -> (b_next, lr_scale); eta = 0.5, B_low = 512, B_high = 4096
+    cases = [
+        (10.0, 0.1, 0.1, 512, 512, 1.0),    # |10-5| = 5 >= 0.5*10 exactly: critical, stay small
+        (6.0, 0.1, 0.1, 512, 4096, 8.0),    # |6-5| = 1 < 3: not critical, grow; LR x8 (512 -> 4096)
+        (4.0, 0.1, 0.1, 512, 4096, 8.0),    # |4-5| = 1 < 2
+        (2.0, 0.1, 0.1, 512, 512, 1.0),     # |2-5| = 3 >= 1: critical (growth counts)
+        (6.0, 0.1, 0.01, 512, 512, 1.0),    # LR decay declares a critical regime
+        (10.0, 0.1, 0.1, 4096, 4096, 8.0),  # critical, but the batch size is never decreased
+        (6.0, 0.1, 0.01, 4096, 4096, 8.0),
+        (0.0, 0.1, 0.1, 512, 512, 1.0),     # ||prev|| = 0
+    ]
+    for a, lc, ln, bc, want_b, want_s in cases:
+        b, s, prev = orc.detect_batch(n2, a * a, lc, ln, 0.5, bc, 512, 4096)
+        assert (b, s) == (want_b, want_s), (a, lc, ln, bc)
+        assert prev == 25.0
+    b, s, prev = orc.detect_batch(n2, -1.0, 0.1, 0.1, 0.5, 512, 512, 4096)
+    assert (b, s, prev) == (512, 1.0, 25.0)  # no earlier window: the early phase is critical
+
+
+def test_detect_batch_uses_the_whole_model_norm_not_the_layers():
+    # layer 0 collapses (per-layer test: critical) but carries little of the whole-model norm
+    prev_layers = np.array([1.0, 100.0])
+    curr_layers = np.array([0.01, 100.0])
+    lv, _ = orc.detect_regime(curr_layers, prev_layers, 0.1, 0.1, 0.5)
+    assert lv[0] == orc.LOW and lv[1] == orc.HIGH
+    b, s, _ = orc.detect_batch(curr_layers, float(prev_layers.sum()), 0.1, 0.1, 0.5, 128, 128, 1024)
+    assert (b, s) == (1024, 8.0)
