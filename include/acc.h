@@ -183,6 +183,49 @@ int acc_powersgd_flush(acc_ctx* ctx, float* err, const float* q, const float* p_
 int acc_topk_step(acc_ctx* ctx, const float* grads, float* err, const uint8_t* level, float* vals,
                   int32_t* idx, int32_t* counts, float* out, float* delta, void* stream);
 
+/* ---- Optimiser tail (Appendix A, hyper-parameter table: Nesterov momentum 0.9; the paper gives the name
+ * and the momentum only, the update below is the usual statement of it, without dampening) -------------
+ *   d' = d + weight_decay * x;   u <- momentum * u + d';   x <- x - lr * (d' + momentum * u)
+ * on every element of every layer (padding between layers is left alone), in fp32 with one fixed
+ * operation order.  hyper is a DEVICE array of three floats {lr, momentum, weight_decay}: the kernels read
+ * it, so a captured graph follows a learning-rate schedule by rewriting those floats.  (The paper lists no
+ * weight decay; 0 reproduces its setting.)
+ *
+ * acc_sgd_nesterov applies the tail on its own from a gradient d [worker_stride].
+ * acc_powersgd_step_sgd / acc_topk_step_sgd are acc_powersgd_step / acc_topk_step with the tail applied by the
+ * kernels that produce `out`, at each element as it is written, which saves a later pass over `out`;
+ * every other result (out, err, q, p_hat, vals, idx, counts, delta) is bit-identical to the plain step's,
+ * and params / mom are bit-identical to running acc_sgd_nesterov(out) after the plain step.
+ * Device pointers: params, mom [worker_stride] floats (in/out), 16-byte aligned; hyper 3 floats.       */
+int acc_sgd_nesterov(acc_ctx* ctx, const float* d, float* params, float* mom, const float* hyper, void* stream);
+int acc_powersgd_step_sgd(acc_ctx* ctx, const float* grads, float* err, float* q, float* p_hat,
+                          const uint8_t* level, float* out, float* delta, float* params, float* mom,
+                          const float* hyper, void* stream);
+int acc_topk_step_sgd(acc_ctx* ctx, const float* grads, float* err, const uint8_t* level, float* vals,
+                      int32_t* idx, int32_t* counts, float* out, float* delta, float* params, float* mom,
+                      const float* hyper, void* stream);
+
+/* ---- Batch-size mode (Section 4.2: "For batch size we use the same algorithm", switching between B_low and
+ * B_high at the granularity of the whole model; Section 5.1: the learning rate scales in the same ratio;
+ * Appendix A: large batches are simulated by accumulating several backward passes before the exchange, and
+ * the batch size is only ever increased) ---------------------------------------------------------------
+ * acc_batch_accumulate: acc_w <- (first ? 0 : acc_w) + g_w for every worker and layer (fp32);
+ *   delta += g_decider when delta != NULL.  grads, acc [W][worker_stride]; delta [worker_stride] or NULL.
+ * acc_batch_average: the uncompressed exchange, out = (1 / (W * n_accum)) * sum_w acc_w, workers added in
+ *   order; with params != NULL the optimiser tail above is applied to out as it is written.
+ * acc_detect_batch: whole-model statistic n2 = sum_l norm2_layers[l] (fp64, fixed order), then Algorithm 1:
+ *   critical = *norm2_prev < 0, or | sqrt(prev) - sqrt(n2) | >= eta * sqrt(prev), or lr_next < lr_curr;
+ *   *batch <- max(*batch, critical ? b_low : b_high);  *lr_scale <- *batch / b_low;  *norm2_prev <- n2;
+ *   delta <- 0 when delta != NULL (new window).
+ *   Device pointers: norm2_layers [L] doubles (e.g. from acc_layer_norms on delta), norm2_prev one double
+ *   (in/out, < 0 = none yet), batch one int32 (in/out), lr_scale one float (out).
+ *   1 <= b_low <= b_high, otherwise ACC_EINVAL.                                                        */
+int acc_batch_accumulate(acc_ctx* ctx, const float* grads, float* acc, float* delta, int32_t first, void* stream);
+int acc_batch_average(acc_ctx* ctx, const float* acc, int32_t n_accum, float* out, float* params, float* mom,
+                      const float* hyper, void* stream);
+int acc_detect_batch(acc_ctx* ctx, const double* norm2_layers, double* norm2_prev, float lr_curr, float lr_next,
+                     int32_t b_low, int32_t b_high, int32_t* batch, float* lr_scale, float* delta, void* stream);
+
 /* Device-side condition of the kernels launched so far on this context (no counterpart in the paper).
  * The pipelined kernels wait for their asynchronous shared-memory copies with a bounded number of polls;
  * should a wait ever give up, the block stores ACC_ETIMEOUT in a status word and returns instead of

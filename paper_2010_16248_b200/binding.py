@@ -46,7 +46,8 @@ EXPORTS = ["acc_workspace_bytes", "acc_create", "acc_destroy", "acc_factor_layou
            "acc_error_feedback", "acc_layer_norms", "acc_detect_regime", "acc_powersgd_step", "acc_topk_step",
            "acc_floats_sent", "acc_last_launch_count", "acc_strerror", "acc_profile_enable", "acc_profile_read",
            "acc_profile_kernel_count", "acc_profile_kernel_name", "acc_sumsq_static", "acc_powersgd_flush", "acc_device_status", "acc_topk_last_paths",
-           "acc_layer_diff_norms", "acc_detect_regime_diff"]
+           "acc_layer_diff_norms", "acc_detect_regime_diff", "acc_sgd_nesterov", "acc_powersgd_step_sgd",
+           "acc_topk_step_sgd", "acc_batch_accumulate", "acc_batch_average", "acc_detect_batch"]
 
 _lib = None
 
@@ -90,6 +91,12 @@ def lib() -> C.CDLL:
     L.acc_topk_last_paths.argtypes = [vp, C.POINTER(i32), i32]
     L.acc_layer_diff_norms.argtypes = [vp, vp, vp, vp, vp]
     L.acc_detect_regime_diff.argtypes = [vp, vp, vp, vp, f32, f32, vp, vp, vp, vp]
+    L.acc_sgd_nesterov.argtypes = [vp, vp, vp, vp, vp, vp]
+    L.acc_powersgd_step_sgd.argtypes = [vp] * 12
+    L.acc_topk_step_sgd.argtypes = [vp] * 13
+    L.acc_batch_accumulate.argtypes = [vp, vp, vp, vp, i32, vp]
+    L.acc_batch_average.argtypes = [vp, vp, i32, vp, vp, vp, vp, vp]
+    L.acc_detect_batch.argtypes = [vp, vp, vp, f32, f32, i32, i32, vp, vp, vp, vp]
     for name in EXPORTS:
         if name not in ("acc_floats_sent", "acc_last_launch_count", "acc_strerror", "acc_profile_kernel_count",
                         "acc_profile_kernel_name"):
@@ -234,6 +241,46 @@ class Context:
                                         _ptr(level, torch.uint8), _ptr(vals, torch.float32), _ptr(idx, torch.int32),
                                         _ptr(counts, torch.int32), _ptr(out, torch.float32),
                                         _ptr(delta, torch.float32), _stream(stream)), "acc_topk_step")
+
+    def acc_sgd_nesterov(self, d, params, mom, hyper, stream=None):
+        self._check(lib().acc_sgd_nesterov(self._h, _ptr(d, torch.float32), _ptr(params, torch.float32),
+                                           _ptr(mom, torch.float32), _ptr(hyper, torch.float32), _stream(stream)),
+                    "acc_sgd_nesterov")
+
+    def acc_powersgd_step_sgd(self, grads, err, q, p_hat, level, out, delta, params, mom, hyper, stream=None):
+        self._check(lib().acc_powersgd_step_sgd(self._h, _ptr(grads, torch.float32), _ptr(err, torch.float32),
+                                                _ptr(q, torch.float32), _ptr(p_hat, torch.float32),
+                                                _ptr(level, torch.uint8), _ptr(out, torch.float32),
+                                                _ptr(delta, torch.float32), _ptr(params, torch.float32),
+                                                _ptr(mom, torch.float32), _ptr(hyper, torch.float32),
+                                                _stream(stream)), "acc_powersgd_step_sgd")
+
+    def acc_topk_step_sgd(self, grads, err, level, vals, idx, counts, out, delta, params, mom, hyper, stream=None):
+        self._check(lib().acc_topk_step_sgd(self._h, _ptr(grads, torch.float32), _ptr(err, torch.float32),
+                                            _ptr(level, torch.uint8), _ptr(vals, torch.float32),
+                                            _ptr(idx, torch.int32), _ptr(counts, torch.int32),
+                                            _ptr(out, torch.float32), _ptr(delta, torch.float32),
+                                            _ptr(params, torch.float32), _ptr(mom, torch.float32),
+                                            _ptr(hyper, torch.float32), _stream(stream)), "acc_topk_step_sgd")
+
+    def acc_batch_accumulate(self, grads, acc, delta=None, first=False, stream=None):
+        self._check(lib().acc_batch_accumulate(self._h, _ptr(grads, torch.float32), _ptr(acc, torch.float32),
+                                               _ptr(delta, torch.float32), int(bool(first)), _stream(stream)),
+                    "acc_batch_accumulate")
+
+    def acc_batch_average(self, acc, n_accum, out, params=None, mom=None, hyper=None, stream=None):
+        self._check(lib().acc_batch_average(self._h, _ptr(acc, torch.float32), int(n_accum),
+                                            _ptr(out, torch.float32), _ptr(params, torch.float32),
+                                            _ptr(mom, torch.float32), _ptr(hyper, torch.float32), _stream(stream)),
+                    "acc_batch_average")
+
+    def acc_detect_batch(self, norm2_layers, norm2_prev, lr_curr, lr_next, b_low, b_high, batch, lr_scale,
+                         delta=None, stream=None):
+        self._check(lib().acc_detect_batch(self._h, _ptr(norm2_layers, torch.float64),
+                                           _ptr(norm2_prev, torch.float64), float(lr_curr), float(lr_next),
+                                           int(b_low), int(b_high), _ptr(batch, torch.int32),
+                                           _ptr(lr_scale, torch.float32), _ptr(delta, torch.float32),
+                                           _stream(stream)), "acc_detect_batch")
 
     def acc_profile_enable(self, enable: bool):
         self._check(lib().acc_profile_enable(self._h, int(bool(enable))), "acc_profile_enable")

@@ -9,7 +9,7 @@ PKG_DIR = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG_DIR)
 CSRC = os.path.join(PKG_DIR, "csrc")
 LIB_PATH = os.path.join(PKG_DIR, "libacc.so")
-SOURCES = ["acc_api.cu", "acc_controller.cu", "acc_powersgd.cu", "acc_topk.cu", "acc_static.cu"]
+SOURCES = ["acc_api.cu", "acc_controller.cu", "acc_powersgd.cu", "acc_topk.cu", "acc_batch.cu", "acc_static.cu"]
 
 
 def _nvcc() -> str:

@@ -294,7 +294,70 @@ int acc_powersgd_step(acc_ctx* ctx, const float* grads, float* err, float* q, fl
       !aligned16(delta))
     return ACC_EALIGN;
   ctx->last_launches = 0;
-  return finish(launch_powersgd(ctx, grads, err, q, p_hat, level, out, delta, static_cast<cudaStream_t>(stream)));
+  return finish(launch_powersgd(ctx, grads, err, q, p_hat, level, out, delta, SgdTail{nullptr, nullptr, nullptr},
+                                static_cast<cudaStream_t>(stream)));
+}
+
+static int check_tail(const float* params, const float* mom, const float* hyper) {
+  if (!params || !mom || !hyper) return ACC_EINVAL;
+  if (!aligned16(params) || !aligned16(mom) || (reinterpret_cast<uintptr_t>(hyper) & 3u)) return ACC_EALIGN;
+  return ACC_OK;
+}
+
+int acc_powersgd_step_sgd(acc_ctx* ctx, const float* grads, float* err, float* q, float* p_hat, const uint8_t* level,
+                          float* out, float* delta, float* params, float* mom, const float* hyper, void* stream) {
+  if (!ctx || !grads || !err || !q || !p_hat || !level || !out) return ACC_EINVAL;
+  if (!aligned16(grads) || !aligned16(err) || !aligned16(q) || !aligned16(p_hat) || !aligned16(out) ||
+      !aligned16(delta))
+    return ACC_EALIGN;
+  const int st = check_tail(params, mom, hyper);
+  if (st != ACC_OK) return st;
+  ctx->last_launches = 0;
+  return finish(launch_powersgd(ctx, grads, err, q, p_hat, level, out, delta, SgdTail{params, mom, hyper},
+                                static_cast<cudaStream_t>(stream)));
+}
+
+int acc_sgd_nesterov(acc_ctx* ctx, const float* d, float* params, float* mom, const float* hyper, void* stream) {
+  if (!ctx || !d) return ACC_EINVAL;
+  if (!aligned16(d)) return ACC_EALIGN;
+  const int st = check_tail(params, mom, hyper);
+  if (st != ACC_OK) return st;
+  ctx->last_launches = 0;
+  return finish(launch_sgd_tiles(ctx, nullptr, (int)ctx->plan.tiles.size(), d, SgdTail{params, mom, hyper},
+                                 static_cast<cudaStream_t>(stream)));
+}
+
+int acc_batch_accumulate(acc_ctx* ctx, const float* grads, float* acc, float* delta, int32_t first, void* stream) {
+  if (!ctx || !grads || !acc) return ACC_EINVAL;
+  if (!aligned16(grads) || !aligned16(acc) || !aligned16(delta)) return ACC_EALIGN;
+  ctx->last_launches = 0;
+  return finish(launch_batch_accumulate(ctx, grads, acc, delta, first != 0, static_cast<cudaStream_t>(stream)));
+}
+
+int acc_batch_average(acc_ctx* ctx, const float* acc, int32_t n_accum, float* out, float* params, float* mom,
+                      const float* hyper, void* stream) {
+  if (!ctx || !acc || !out || n_accum < 1) return ACC_EINVAL;
+  if (!aligned16(acc) || !aligned16(out)) return ACC_EALIGN;
+  SgdTail tail{nullptr, nullptr, nullptr};
+  if (params) {
+    const int st = check_tail(params, mom, hyper);
+    if (st != ACC_OK) return st;
+    tail = SgdTail{params, mom, hyper};
+  }
+  ctx->last_launches = 0;
+  return finish(launch_batch_average(ctx, acc, n_accum, out, tail, static_cast<cudaStream_t>(stream)));
+}
+
+int acc_detect_batch(acc_ctx* ctx, const double* norm2_layers, double* norm2_prev, float lr_curr, float lr_next,
+                     int32_t b_low, int32_t b_high, int32_t* batch, float* lr_scale, float* delta, void* stream) {
+  if (!ctx || !norm2_layers || !norm2_prev || !batch || !lr_scale) return ACC_EINVAL;
+  if (b_low < 1 || b_high < b_low) return ACC_EINVAL;
+  if (!aligned16(delta)) return ACC_EALIGN;
+  ctx->last_launches = 0;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  cudaError_t e = launch_detect_batch(ctx, norm2_layers, norm2_prev, lr_curr, lr_next, b_low, b_high, batch, lr_scale, s);
+  if (e == cudaSuccess && delta) e = cudaMemsetAsync(delta, 0, sizeof(float) * (size_t)ctx->cfg.worker_stride, s);
+  return finish(e);
 }
 
 int acc_powersgd_flush(acc_ctx* ctx, float* err, const float* q, const float* p_hat, void* stream) {
@@ -312,7 +375,22 @@ int acc_topk_step(acc_ctx* ctx, const float* grads, float* err, const uint8_t* l
       !aligned16(delta))
     return ACC_EALIGN;
   ctx->last_launches = 0;
-  return finish(launch_topk(ctx, grads, err, level, vals, idx, counts, out, delta, static_cast<cudaStream_t>(stream)));
+  return finish(launch_topk(ctx, grads, err, level, vals, idx, counts, out, delta, SgdTail{nullptr, nullptr, nullptr},
+                            static_cast<cudaStream_t>(stream)));
+}
+
+int acc_topk_step_sgd(acc_ctx* ctx, const float* grads, float* err, const uint8_t* level, float* vals, int32_t* idx,
+                      int32_t* counts, float* out, float* delta, float* params, float* mom, const float* hyper,
+                      void* stream) {
+  if (!ctx || !grads || !err || !level || !vals || !idx || !counts || !out) return ACC_EINVAL;
+  if (!aligned16(grads) || !aligned16(err) || !aligned16(vals) || !aligned16(idx) || !aligned16(out) ||
+      !aligned16(delta))
+    return ACC_EALIGN;
+  const int st = check_tail(params, mom, hyper);
+  if (st != ACC_OK) return st;
+  ctx->last_launches = 0;
+  return finish(launch_topk(ctx, grads, err, level, vals, idx, counts, out, delta, SgdTail{params, mom, hyper},
+                            static_cast<cudaStream_t>(stream)));
 }
 
 int64_t acc_floats_sent(const acc_config* cfg, const uint8_t* level_host, int32_t compressor) {
@@ -365,7 +443,8 @@ const char* acc_profile_kernel_name(int32_t i) {
       "topk_tile_scan_kernel", "topk_select_kernel", "topk_decompress_kernel", "psgd_flush_kernel",
       "topk_collect_kernel", "topk_pick3_kernel", "topk_tile_counts_kernel",
       "topk_hist2_list_kernel", "topk_hist3_list_kernel", "topk_finalize_staged_kernel",
-      "psgd_orthonormalise_block_kernel"};
+      "psgd_orthonormalise_block_kernel", "sgd_tiles_kernel", "batch_accumulate_kernel", "batch_average_kernel",
+      "detect_batch_kernel"};
   return (i >= 0 && i < PH_COUNT) ? names[i] : "";
 }
 

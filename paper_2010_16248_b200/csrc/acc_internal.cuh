@@ -54,7 +54,7 @@ enum Phase {
   PH_EF = 0, PH_NORM_PARTIAL, PH_NORM_FINAL, PH_DETECT,
   PH_PSGD_PROJECT, PH_PSGD_ORTHO, PH_PSGD_QPARTIAL, PH_PSGD_QREDUCE, PH_PSGD_RESIDUAL,
   PH_TOPK_EF_HIST1, PH_TOPK_PICK1, PH_TOPK_HIST2, PH_TOPK_PICK2, PH_TOPK_HIST3, PH_TOPK_PICK3_SCAN, PH_TOPK_SELECT,
-  PH_TOPK_DECOMPRESS, PH_PSGD_FLUSH, PH_TOPK_COLLECT, PH_TOPK_PICK3, PH_TOPK_TILE_COUNTS, PH_TOPK_HIST2_LIST, PH_TOPK_HIST3_LIST, PH_TOPK_FINALIZE_STAGED, PH_PSGD_ORTHO_BLOCK,
+  PH_TOPK_DECOMPRESS, PH_PSGD_FLUSH, PH_TOPK_COLLECT, PH_TOPK_PICK3, PH_TOPK_TILE_COUNTS, PH_TOPK_HIST2_LIST, PH_TOPK_HIST3_LIST, PH_TOPK_FINALIZE_STAGED, PH_PSGD_ORTHO_BLOCK, PH_SGD_TILES, PH_BATCH_ACCUMULATE, PH_BATCH_AVERAGE, PH_DETECT_BATCH,
   PH_COUNT
 };
 
@@ -117,6 +117,11 @@ struct acc_ctx {
 
 namespace acc {
 
+// Optimiser tail (Nesterov momentum, Appendix A) applied by the kernels that produce `out`, at the element
+// they have just computed.  params == nullptr: no tail.  hyper: three DEVICE floats (learning rate, momentum,
+// weight decay), read by the kernels so that a captured graph follows a learning-rate schedule.
+struct SgdTail { float* params; float* mom; const float* hyper; };
+
 // Kernel launchers (one per translation unit).  Each returns a cudaError_t from cudaGetLastError and
 // adds the number of kernels it launched to ctx->last_launches.
 cudaError_t launch_error_feedback(acc_ctx* ctx, const float* grads, float* err, float* delta, cudaStream_t s);
@@ -125,11 +130,19 @@ cudaError_t launch_layer_norms(acc_ctx* ctx, const float* buf, long long stride,
 cudaError_t launch_detect(acc_ctx* ctx, const double* n2c, double* n2p, const double* n2d, float lr_curr,
                           float lr_next, uint8_t* level, cudaStream_t s);
 cudaError_t launch_powersgd(acc_ctx* ctx, const float* grads, float* err, float* q, float* p_hat,
-                            const uint8_t* level, float* out, float* delta, cudaStream_t s);
+                            const uint8_t* level, float* out, float* delta, SgdTail tail, cudaStream_t s);
 cudaError_t prepare_powersgd();
 cudaError_t launch_powersgd_flush(acc_ctx* ctx, float* err, const float* q, const float* p_hat, cudaStream_t s);
 cudaError_t launch_topk(acc_ctx* ctx, const float* grads, float* err, const uint8_t* level, float* vals,
-                        int32_t* idx, int32_t* counts, float* out, float* delta, cudaStream_t s);
+                        int32_t* idx, int32_t* counts, float* out, float* delta, SgdTail tail, cudaStream_t s);
+// Optimiser tail on its own over the given tiles (tile_ids == nullptr: all tiles, in order).
+cudaError_t launch_sgd_tiles(acc_ctx* ctx, const int* tile_ids, int n, const float* d, SgdTail tail, cudaStream_t s);
+cudaError_t launch_batch_accumulate(acc_ctx* ctx, const float* grads, float* acc, float* delta, int first,
+                                    cudaStream_t s);
+cudaError_t launch_batch_average(acc_ctx* ctx, const float* acc, int n_accum, float* out, SgdTail tail,
+                                 cudaStream_t s);
+cudaError_t launch_detect_batch(acc_ctx* ctx, const double* n2_layers, double* n2_prev, float lr_curr, float lr_next,
+                                int b_low, int b_high, int32_t* batch, float* lr_scale, cudaStream_t s);
 
 // Brackets one kernel launch with CUDA events on its stream when profiling is on; counts the launch.
 struct PhaseTimer {
@@ -153,6 +166,32 @@ struct PhaseTimer {
 __device__ __forceinline__ float4 ld_stream4(const float* p) { return __ldcs(reinterpret_cast<const float4*>(p)); }
 __device__ __forceinline__ float ld_stream1(const float* p) { return __ldcs(p); }
 __device__ __forceinline__ void st_stream4(float* p, float4 v) { __stcs(reinterpret_cast<float4*>(p), v); }
+
+struct SgdHyper { float lr, mu, wd; };
+__device__ __forceinline__ SgdHyper sgd_hyper(const SgdTail& t) {
+  SgdHyper h;
+  h.lr = __ldg(t.hyper); h.mu = __ldg(t.hyper + 1); h.wd = __ldg(t.hyper + 2);
+  return h;
+}
+// d' = d + wd x;  u <- mu u + d';  x <- x - lr (d' + mu u).  One fixed fp32 operation order everywhere, so the
+// fused tails and the stand-alone kernel give the same bits.
+__device__ __forceinline__ void sgd_update(float d, float& x, float& u, const SgdHyper& h) {
+  const float dd = fmaf(h.wd, x, d);
+  u = fmaf(h.mu, u, dd);
+  x = fmaf(-h.lr, fmaf(h.mu, u, dd), x);
+}
+__device__ __forceinline__ void sgd_apply1(const SgdTail& t, const SgdHyper& h, long long i, float d) {
+  float x = t.params[i], u = t.mom[i];
+  sgd_update(d, x, u, h);
+  t.params[i] = x; t.mom[i] = u;
+}
+__device__ __forceinline__ void sgd_apply4(const SgdTail& t, const SgdHyper& h, long long i, const float4 d) {
+  float4 x = *reinterpret_cast<const float4*>(t.params + i), u = *reinterpret_cast<const float4*>(t.mom + i);
+  sgd_update(d.x, x.x, u.x, h); sgd_update(d.y, x.y, u.y, h);
+  sgd_update(d.z, x.z, u.z, h); sgd_update(d.w, x.w, u.w, h);
+  *reinterpret_cast<float4*>(t.params + i) = x;
+  *reinterpret_cast<float4*>(t.mom + i) = u;
+}
 
 __device__ __forceinline__ double warp_sum(double v) {
 #pragma unroll

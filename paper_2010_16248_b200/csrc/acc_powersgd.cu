@@ -563,17 +563,22 @@ psgd_qpartial_kernel(const DevLayer* __restrict__ layers, const ColItem* __restr
 // Pass 5, lazy mode (out = A only).  Same items as the Q-partial pass: a thread owns `vec` adjacent columns,
 // keeps their rows of Q' in registers and walks the slab's rows, so the factor tables are read once per
 // (slab, column) instead of once per element; entries use the same lowrank_entry as every other pass.
-template <int VEC>
+// SGD: the optimiser tail is applied to the element just computed (params and mom laid out like out).
+template <int VEC, bool SGD>
 __device__ __forceinline__ void decompress_cols(const ColItem& it, const DevLayer& L, const float4* __restrict__ Q4,
-                                                const float4* __restrict__ P4, float* __restrict__ out, int r) {
+                                                const float4* __restrict__ P4, float* __restrict__ out, int r,
+                                                const SgdTail& tail) {
   using V = typename VecT<VEC>::type;
   const int col = it.col0 + (int)threadIdx.x * VEC;
   if (col >= L.cols) return;
   float4 qv[VEC];
 #pragma unroll
   for (int e = 0; e < VEC; ++e) qv[e] = __ldg(Q4 + col + e);
-  float* base = out + L.offset + (long long)it.row0 * L.cols + col;
+  const long long first = L.offset + (long long)it.row0 * L.cols + col;
+  float* base = out + first;
   const float4* pr = P4 + it.row0;
+  SgdHyper h = {0.f, 0.f, 0.f};
+  if (SGD) h = sgd_hyper(tail);
 #pragma unroll 8
   for (int i = 0; i < it.nrows; ++i) {
     const float4 pv = __ldg(pr + i);
@@ -581,21 +586,32 @@ __device__ __forceinline__ void decompress_cols(const ColItem& it, const DevLaye
 #pragma unroll
     for (int e = 0; e < VEC; ++e) a[e] = lowrank_entry(pv, qv[e], r);
     __stcs(reinterpret_cast<V*>(base + (long long)i * L.cols), *reinterpret_cast<const V*>(a));
+    if (SGD) {
+      const long long at = first + (long long)i * L.cols;
+      V xv = *reinterpret_cast<const V*>(tail.params + at), uv = *reinterpret_cast<const V*>(tail.mom + at);
+      float* x = reinterpret_cast<float*>(&xv);
+      float* u = reinterpret_cast<float*>(&uv);
+#pragma unroll
+      for (int e = 0; e < VEC; ++e) sgd_update(a[e], x[e], u[e], h);
+      *reinterpret_cast<V*>(tail.params + at) = xv;
+      *reinterpret_cast<V*>(tail.mom + at) = uv;
+    }
   }
 }
 
+template <bool SGD>
 __global__ void __launch_bounds__(kColBlockThreads)
 psgd_decompress_kernel(const DevLayer* __restrict__ layers, const ColItem* __restrict__ items,
                        const float* __restrict__ q, const float* __restrict__ p, const uint8_t* __restrict__ level,
-                       float* __restrict__ out, int rank_low, int rank_high) {
+                       float* __restrict__ out, int rank_low, int rank_high, const SgdTail tail) {
   const ColItem it = items[blockIdx.x];
   const DevLayer L = layers[it.layer];
   const int r = level[it.layer] ? rank_low : rank_high;
   const float4* Q4 = reinterpret_cast<const float4*>(q) + L.q_row;
   const float4* P4 = reinterpret_cast<const float4*>(p) + L.p_row;
-  if (L.vec == 4) decompress_cols<4>(it, L, Q4, P4, out, r);
-  else if (L.vec == 2) decompress_cols<2>(it, L, Q4, P4, out, r);
-  else decompress_cols<1>(it, L, Q4, P4, out, r);
+  if (L.vec == 4) decompress_cols<4, SGD>(it, L, Q4, P4, out, r, tail);
+  else if (L.vec == 2) decompress_cols<2, SGD>(it, L, Q4, P4, out, r, tail);
+  else decompress_cols<1, SGD>(it, L, Q4, P4, out, r, tail);
 }
 
 // Pass 4.  Sums the slab partials of 32 columns in a fixed order and stores the first r ranks of Q'.
@@ -635,12 +651,13 @@ psgd_qreduce_kernel(const DevLayer* __restrict__ layers, const int* __restrict__
 // Pass 5.  One block per tile:  A = P^ Q'^T (first r ranks) at every element of the tile;
 //   WRITE_OUT: out = A;   UPDATE_ERR: err_w -= A for every worker.
 // Eager step: both (r from the level).  Lazy step: WRITE_OUT only.  Flush: UPDATE_ERR only, r = pending rank.
-template <int WB, bool WRITE_OUT, bool UPDATE_ERR>
+// SGD (with WRITE_OUT): the optimiser tail is applied to A where it is written.
+template <int WB, bool WRITE_OUT, bool UPDATE_ERR, bool SGD>
 __global__ void __launch_bounds__(256)
 psgd_residual_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict__ tiles, float* __restrict__ err,
                      const float* __restrict__ q, const float* __restrict__ p, const uint8_t* __restrict__ level,
                      const int* __restrict__ pending, float* __restrict__ out, long long stride, int W,
-                     int rank_low, int rank_high) {
+                     int rank_low, int rank_high, const SgdTail tail) {
   const Tile t = tiles[blockIdx.x];
   const DevLayer L = layers[t.layer];
   if (L.kind != ACC_MATRIX) return;
@@ -651,6 +668,8 @@ psgd_residual_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict
   const float4* __restrict__ P4 = reinterpret_cast<const float4*>(p) + L.p_row;
   const long long base = L.offset + t.elem0;
   const int n4 = t.nelem >> 2;
+  SgdHyper h = {0.f, 0.f, 0.f};
+  if (SGD) h = sgd_hyper(tail);
   for (int f = threadIdx.x; f < n4; f += blockDim.x) {
     const long long idx = base + 4 * f;
     const float4 a = lowrank4(P4, Q4, m, L.inv_cols, t.elem0 + 4 * f, r);
@@ -668,6 +687,7 @@ psgd_residual_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict
       }
     }
     if (WRITE_OUT) st_stream4(out + idx, a);
+    if (SGD) sgd_apply4(tail, h, idx, a);
   }
   for (int i = 4 * n4 + threadIdx.x; i < t.nelem; i += blockDim.x) {
     const int e_idx = t.elem0 + i, row = e_idx / m, col = e_idx - row * m;
@@ -675,7 +695,32 @@ psgd_residual_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict
     if (UPDATE_ERR)
       for (int w = 0; w < W; ++w) err[(long long)w * stride + base + i] -= a;
     if (WRITE_OUT) out[base + i] = a;
+    if (SGD) sgd_apply1(tail, h, base + i, a);
   }
+}
+
+// Optimiser tail on its own: x, u updated from d over the given flat tiles (tile_ids == nullptr: tile
+// blockIdx.x).  Used for the VECTOR layers of a fused PowerSGD step (their `out` comes from the first pass)
+// and as the stand-alone tail.
+__global__ void __launch_bounds__(256)
+sgd_tiles_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict__ tiles, const int* __restrict__ tile_ids,
+                 const float* __restrict__ d, const SgdTail tail) {
+  const Tile t = tiles[tile_ids != nullptr ? tile_ids[blockIdx.x] : (int)blockIdx.x];
+  const DevLayer L = layers[t.layer];
+  const long long base = L.offset + t.elem0;
+  const SgdHyper h = sgd_hyper(tail);
+  const int n4 = t.nelem >> 2;
+  for (int f = threadIdx.x; f < n4; f += blockDim.x)
+    sgd_apply4(tail, h, base + 4 * f, ld_stream4(d + base + 4 * f));
+  for (int i = 4 * n4 + threadIdx.x; i < t.nelem; i += blockDim.x) sgd_apply1(tail, h, base + i, d[base + i]);
+}
+
+cudaError_t launch_sgd_tiles(acc_ctx* ctx, const int* tile_ids, int n, const float* d, SgdTail tail, cudaStream_t s) {
+  if (n > 0) {
+    PhaseTimer pt(ctx, PH_SGD_TILES, s);
+    sgd_tiles_kernel<<<n, 256, 0, s>>>(ctx->d_layers, ctx->d_tiles, tile_ids, d, tail);
+  }
+  return cudaGetLastError();
 }
 
 // Lazy mode only: after a flush no residual is pending.
@@ -696,7 +741,7 @@ cudaError_t prepare_powersgd() {
 }
 
 cudaError_t launch_powersgd(acc_ctx* ctx, const float* grads, float* err, float* q, float* p_hat,
-                            const uint8_t* level, float* out, float* delta, cudaStream_t s) {
+                            const uint8_t* level, float* out, float* delta, SgdTail tail, cudaStream_t s) {
   const Plan& pl = ctx->plan;
   const acc_config& c = ctx->cfg;
   const int nt = (int)pl.tiles.size();
@@ -761,14 +806,27 @@ cudaError_t launch_powersgd(acc_ctx* ctx, const float* grads, float* err, float*
     }
     {
       PhaseTimer pt(ctx, PH_PSGD_RESIDUAL, s);
-      if (lazy)
-        psgd_decompress_kernel<<<(unsigned)pl.col_items.size(), kColBlockThreads, 0, s>>>(
-            ctx->d_layers, ctx->d_col_items, q, p_hat, level, out, c.rank_low, c.rank_high);
+      const unsigned n_items = (unsigned)pl.col_items.size();
+      if (lazy && tail.params)
+        psgd_decompress_kernel<true><<<n_items, kColBlockThreads, 0, s>>>(
+            ctx->d_layers, ctx->d_col_items, q, p_hat, level, out, c.rank_low, c.rank_high, tail);
+      else if (lazy)
+        psgd_decompress_kernel<false><<<n_items, kColBlockThreads, 0, s>>>(
+            ctx->d_layers, ctx->d_col_items, q, p_hat, level, out, c.rank_low, c.rank_high, tail);
+      else if (tail.params)
+        psgd_residual_kernel<4, true, true, true><<<nt, 256, 0, s>>>(ctx->d_layers, ctx->d_tiles, err, q, p_hat, level,
+                                                                     nullptr, out, c.worker_stride, c.n_workers,
+                                                                     c.rank_low, c.rank_high, tail);
       else
-        psgd_residual_kernel<4, true, true><<<nt, 256, 0, s>>>(ctx->d_layers, ctx->d_tiles, err, q, p_hat, level,
-                                                               nullptr, out, c.worker_stride, c.n_workers,
-                                                               c.rank_low, c.rank_high);
+        psgd_residual_kernel<4, true, true, false><<<nt, 256, 0, s>>>(ctx->d_layers, ctx->d_tiles, err, q, p_hat,
+                                                                      level, nullptr, out, c.worker_stride,
+                                                                      c.n_workers, c.rank_low, c.rank_high, tail);
     }
+  }
+  // VECTOR layers: their out (the plain mean) was written by the first pass
+  if (tail.params && !pl.vec_tiles.empty()) {
+    const cudaError_t e = launch_sgd_tiles(ctx, ctx->d_vec_tiles, (int)pl.vec_tiles.size(), out, tail, s);
+    if (e != cudaSuccess) return e;
   }
   return cudaGetLastError();
 }
@@ -780,9 +838,9 @@ cudaError_t launch_powersgd_flush(acc_ctx* ctx, float* err, const float* q, cons
   if (pl.n_mat > 0) {
     {
       PhaseTimer pt(ctx, PH_PSGD_FLUSH, s);
-      psgd_residual_kernel<4, false, true><<<nt, 256, 0, s>>>(ctx->d_layers, ctx->d_tiles, err, q, p_hat, nullptr,
-                                                              ctx->d_pending, nullptr, c.worker_stride, c.n_workers,
-                                                              c.rank_low, c.rank_high);
+      psgd_residual_kernel<4, false, true, false><<<nt, 256, 0, s>>>(
+          ctx->d_layers, ctx->d_tiles, err, q, p_hat, nullptr, ctx->d_pending, nullptr, c.worker_stride, c.n_workers,
+          c.rank_low, c.rank_high, SgdTail{nullptr, nullptr, nullptr});
     }
     ctx->last_launches += 1;
     psgd_clear_pending_kernel<<<(c.n_layers + 127) / 128, 128, 0, s>>>(ctx->d_pending, c.n_layers);

@@ -911,17 +911,21 @@ topk_finalize_staged_kernel(const DevLayer* __restrict__ layers, const Tile* __r
 // Pass F.  Scatter-decompress and average: one block per tile; the tile of `out` is accumulated in shared
 // memory from every worker's packed entries that fall into it, workers in order (fixed fp32 order), then
 // scaled by 1/W.  VECTOR tiles: out = mean_w g_w, delta += g_decider.
+// SGD: the optimiser tail is applied to every element of out where it is written.
+template <bool SGD>
 __global__ void __launch_bounds__(256)
 topk_decompress_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict__ tiles, int n_tiles, int n_mat,
                        const float* __restrict__ grads, const Select* __restrict__ sel,
                        const int2* __restrict__ tile_pre, const float* __restrict__ vals,
                        const int32_t* __restrict__ idx, float* __restrict__ out, float* __restrict__ delta,
-                       long long stride, long long capacity, int W, int decider, float inv_w) {
+                       long long stride, long long capacity, int W, int decider, float inv_w, const SgdTail tail) {
   __shared__ float acc[kTile];
   const int ti = blockIdx.x;
   const Tile t = tiles[ti];
   const DevLayer L = layers[t.layer];
   const long long base = L.offset + t.elem0;
+  SgdHyper h = {0.f, 0.f, 0.f};
+  if (SGD) h = sgd_hyper(tail);
   if (L.kind != ACC_MATRIX) {
     for (int i = threadIdx.x; i < t.nelem; i += blockDim.x) {
       float a = 0.f;
@@ -931,6 +935,7 @@ topk_decompress_kernel(const DevLayer* __restrict__ layers, const Tile* __restri
         if (delta != nullptr && w == decider) delta[base + i] += g;
       }
       out[base + i] = a * inv_w;
+      if (SGD) sgd_apply1(tail, h, base + i, a * inv_w);
     }
     return;
   }
@@ -951,14 +956,20 @@ topk_decompress_kernel(const DevLayer* __restrict__ layers, const Tile* __restri
     __syncthreads();
   }
   const int n4 = t.nelem >> 2;
-  for (int i = threadIdx.x; i < n4; i += blockDim.x)
-    st_stream4(out + base + 4 * i, make_float4(acc[4 * i] * inv_w, acc[4 * i + 1] * inv_w, acc[4 * i + 2] * inv_w,
-                                               acc[4 * i + 3] * inv_w));
-  for (int i = 4 * n4 + threadIdx.x; i < t.nelem; i += blockDim.x) out[base + i] = acc[i] * inv_w;
+  for (int i = threadIdx.x; i < n4; i += blockDim.x) {
+    const float4 v = make_float4(acc[4 * i] * inv_w, acc[4 * i + 1] * inv_w, acc[4 * i + 2] * inv_w,
+                                 acc[4 * i + 3] * inv_w);
+    st_stream4(out + base + 4 * i, v);
+    if (SGD) sgd_apply4(tail, h, base + 4 * i, v);
+  }
+  for (int i = 4 * n4 + threadIdx.x; i < t.nelem; i += blockDim.x) {
+    out[base + i] = acc[i] * inv_w;
+    if (SGD) sgd_apply1(tail, h, base + i, acc[i] * inv_w);
+  }
 }
 
 cudaError_t launch_topk(acc_ctx* ctx, const float* grads, float* err, const uint8_t* level, float* vals,
-                        int32_t* idx, int32_t* counts, float* out, float* delta, cudaStream_t s) {
+                        int32_t* idx, int32_t* counts, float* out, float* delta, SgdTail tail, cudaStream_t s) {
   const Plan& pl = ctx->plan;
   const acc_config& c = ctx->cfg;
   const int nt = (int)pl.tiles.size(), W = c.n_workers, n_mat = pl.n_mat;
@@ -1046,9 +1057,14 @@ cudaError_t launch_topk(acc_ctx* ctx, const float* grads, float* err, const uint
   }
   {
     PhaseTimer pt(ctx, PH_TOPK_DECOMPRESS, s);
-    topk_decompress_kernel<<<nt, 256, 0, s>>>(ctx->d_layers, ctx->d_tiles, nt, n_mat, grads, ctx->d_sel,
-                                              ctx->d_tile_pre, vals, idx, out, delta, c.worker_stride, pl.capacity,
-                                              W, c.decider, inv_w);
+    if (tail.params)
+      topk_decompress_kernel<true><<<nt, 256, 0, s>>>(ctx->d_layers, ctx->d_tiles, nt, n_mat, grads, ctx->d_sel,
+                                                      ctx->d_tile_pre, vals, idx, out, delta, c.worker_stride,
+                                                      pl.capacity, W, c.decider, inv_w, tail);
+    else
+      topk_decompress_kernel<false><<<nt, 256, 0, s>>>(ctx->d_layers, ctx->d_tiles, nt, n_mat, grads, ctx->d_sel,
+                                                       ctx->d_tile_pre, vals, idx, out, delta, c.worker_stride,
+                                                       pl.capacity, W, c.decider, inv_w, tail);
   }
   return cudaGetLastError();
 }

@@ -19,9 +19,14 @@ from . import workloads as wl
 class AccordionStep:
     def __init__(self, table: wl.LayerTable, n_workers: int, compressors: Sequence[str] = ("powersgd",),
                  rank_low=2, rank_high=1, topk_low_bp=1000, topk_high_bp=100, eta=0.5, gs_eps=1e-8,
-                 check_every=10, decider=0, q_init=None, device="cuda", lazy_residual=False):
+                 check_every=10, decider=0, q_init=None, device="cuda", lazy_residual=False, optimizer=None):
+        """``optimizer``: None, or a dict ``{"params": tensor [stride], "lr": .., "momentum": 0.9,
+        "weight_decay": 0.0}``: the Nesterov update (Appendix A) is then applied to ``params`` by the kernels
+        that produce the averaged gradient (one compressor only)."""
         self.table, self.W = table, n_workers
         self.compressors = tuple(compressors)
+        if optimizer is not None and len(self.compressors) != 1:
+            raise ValueError("the optimiser tail belongs to one compressor's output")
         self.check_every = check_every
         self.device = torch.device(device)
         self.ctx = binding.Context(table, n_workers, device=device, rank_low=rank_low, rank_high=rank_high,
@@ -35,6 +40,12 @@ class AccordionStep:
         self.norm2_prev = torch.full((L,), -1.0, dtype=torch.float64, device=dev)
         self.t = 0
         self.launches = 0
+        self.params = self.mom = self.hyper = None
+        if optimizer is not None:
+            self.params = optimizer["params"]
+            self.mom = torch.zeros(stride, device=dev)
+            self.hyper = torch.tensor([optimizer["lr"], optimizer.get("momentum", 0.9),
+                                       optimizer.get("weight_decay", 0.0)], dtype=torch.float32, device=dev)
         if "powersgd" in self.compressors:
             self.err_psgd = torch.zeros(n_workers, stride, device=dev)
             self.q = self.ctx.new_q(q_init if q_init is not None else wl.initial_q(table, rank_low, device=dev))
@@ -50,12 +61,21 @@ class AccordionStep:
         c = self.ctx
         delta: Optional[torch.Tensor] = self.delta  # accumulated once per iteration, by the first compressor
         if "powersgd" in self.compressors:
-            c.acc_powersgd_step(grads, self.err_psgd, self.q, self.p_hat, self.level, self.out_psgd, delta, stream)
+            if self.params is not None:
+                c.acc_powersgd_step_sgd(grads, self.err_psgd, self.q, self.p_hat, self.level, self.out_psgd, delta,
+                                        self.params, self.mom, self.hyper, stream)
+            else:
+                c.acc_powersgd_step(grads, self.err_psgd, self.q, self.p_hat, self.level, self.out_psgd, delta,
+                                    stream)
             self.launches += c.last_launch_count()
             delta = None
         if "topk" in self.compressors:
-            c.acc_topk_step(grads, self.err_topk, self.level, self.vals, self.idx, self.counts, self.out_topk,
-                            delta, stream)
+            if self.params is not None:
+                c.acc_topk_step_sgd(grads, self.err_topk, self.level, self.vals, self.idx, self.counts,
+                                    self.out_topk, delta, self.params, self.mom, self.hyper, stream)
+            else:
+                c.acc_topk_step(grads, self.err_topk, self.level, self.vals, self.idx, self.counts, self.out_topk,
+                                delta, stream)
             self.launches += c.last_launch_count()
         self.t += 1
         if self.t % self.check_every == 0:
@@ -63,6 +83,10 @@ class AccordionStep:
             self.launches += c.last_launch_count()
             c.acc_detect_regime(self.norm2_curr, self.norm2_prev, lr_curr, lr_next, self.level, self.delta, stream)
             self.launches += c.last_launch_count()
+
+    def set_lr(self, lr: float):
+        """Learning rate of the optimiser tail: a device scalar the kernels read, so captured graphs follow it."""
+        self.hyper[0:1].fill_(float(lr))
 
     def capture_graphs(self, grads_buffers, lr_curr: float = 0.1, lr_next: float = 0.1):
         """Captures one iteration as CUDA graphs, for each of the given fixed device gradient buffers (the
@@ -105,6 +129,57 @@ class AccordionStep:
         if "topk" in self.compressors:
             outs.append(self.out_topk)
         return outs
+
+
+class BatchSizeStep:
+    """Batch-size mode of the controller (Section 4.2, Appendix A): every backward pass adds its gradients to
+    per-worker accumulators; after ``n_accum = batch / micro_batch`` passes the accumulators are averaged
+    (the uncompressed exchange), optionally straight into the Nesterov update; at the end of every detection
+    window the whole-model norm of the accumulated decider gradient goes through Algorithm 1, which picks
+    B_low or B_high (never decreasing) and the matching learning-rate scale.  All arithmetic runs in the
+    library's kernels; the host reads back one integer per window (the batch size steers its loop)."""
+
+    def __init__(self, table: wl.LayerTable, n_workers: int, b_low: int, b_high: int, micro_batch: int, eta=0.5,
+                 decider=0, device="cuda", optimizer=None):
+        if b_low % micro_batch or b_high % micro_batch:
+            raise ValueError("batch sizes must be multiples of the micro-batch")
+        self.table, self.W = table, n_workers
+        self.b_low, self.b_high, self.micro_batch = b_low, b_high, micro_batch
+        self.device = dev = torch.device(device)
+        self.ctx = binding.Context(table, n_workers, device=device, eta=eta, decider=decider)
+        stride, L = table.stride, table.n_layers
+        self.acc = torch.zeros(n_workers, stride, device=dev)
+        self.delta = torch.zeros(stride, device=dev)
+        self.out = torch.zeros(stride, device=dev)
+        self.norm2_layers = torch.zeros(L, dtype=torch.float64, device=dev)
+        self.norm2_prev = torch.full((1,), -1.0, dtype=torch.float64, device=dev)
+        self.batch = torch.tensor([b_low], dtype=torch.int32, device=dev)  # the early phase is critical
+        self.lr_scale = torch.ones(1, device=dev)
+        self.pending = 0
+        self.params = self.mom = self.hyper = None
+        if optimizer is not None:
+            self.params = optimizer["params"]
+            self.mom = torch.zeros(stride, device=dev)
+            self.hyper = torch.tensor([optimizer["lr"], optimizer.get("momentum", 0.9),
+                                       optimizer.get("weight_decay", 0.0)], dtype=torch.float32, device=dev)
+
+    def micro_step(self, grads: torch.Tensor, stream=None):
+        """One backward pass worth of gradients ``[W, stride]`` (device)."""
+        self.ctx.acc_batch_accumulate(grads, self.acc, self.delta, first=(self.pending == 0), stream=stream)
+        self.pending += 1
+
+    def apply(self, stream=None):
+        """Ends the large batch: averages what was accumulated (and updates the parameters if asked)."""
+        self.ctx.acc_batch_average(self.acc, self.pending, self.out, self.params, self.mom, self.hyper, stream)
+        self.pending = 0
+        return self.out
+
+    def check(self, lr_curr: float, lr_next: float, stream=None) -> int:
+        """End of a detection window; returns the batch size to use from now on."""
+        self.ctx.acc_layer_norms(self.delta, 1, self.norm2_layers, stream=stream)
+        self.ctx.acc_detect_batch(self.norm2_layers, self.norm2_prev, lr_curr, lr_next, self.b_low, self.b_high,
+                                  self.batch, self.lr_scale, self.delta, stream)
+        return int(self.batch.item())
 
 
 class HostFedStep:
