@@ -195,6 +195,13 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--eager", action="store_true", help="PowerSGD: materialise the error memory every step")
     ap.add_argument("--no-graphs", action="store_true", help="issue the timed steps call by call instead of as CUDA graphs")
+    ap.add_argument("--sgd-tail", action="store_true",
+                    help="single-compressor configs: apply the Nesterov update inside the step (fused optimiser tail)")
+    ap.add_argument("--batch-mode", action="store_true",
+                    help="batch-size mode instead of compression: a step is n_accum micro-batch accumulations, the "
+                         "uncompressed average with the fused Nesterov update, and (every check_every steps) the "
+                         "whole-model detector")
+    ap.add_argument("--n-accum", type=int, default=8, help="--batch-mode: micro-batches per step (B_high / micro-batch)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -222,8 +229,16 @@ def main():
     stream_gen = wl.GradientStream(w, device=dev)
     # independent replicas: every rank draws its own gradient batches
     ring = [stream_gen.grads(dist_util.replica_seed_offset(rank) + t) for t in range(RING)]
+    if args.batch_mode:
+        run_batch_mode(args, w, ring, dev, rank, world, local_rank)
+        return
+    optimizer = None
+    if args.sgd_tail:
+        assert n_comp == 1, "--sgd-tail needs a single-compressor config (2, 3 or 4)"
+        optimizer = {"params": torch.zeros(table.stride, device=dev), "lr": 0.1, "momentum": 0.9}
     eng = pipeline.AccordionStep(table, W, w.compressors, w.rank_low, w.rank_high, w.topk_low_bp, w.topk_high_bp,
-                                 w.eta, 1e-8, w.check_every, device=dev, lazy_residual=not args.eager)
+                                 w.eta, 1e-8, w.check_every, device=dev, lazy_residual=not args.eager,
+                                 optimizer=optimizer)
     n_mat = table.n_matrix_params
     grad_bytes_step = n_comp * 4.0 * W * table.n_params
 
@@ -341,6 +356,7 @@ def main():
                            "compressors": list(w.compressors), "rank_low_high": [w.rank_low, w.rank_high],
                            "topk_bp_low_high": [w.topk_low_bp, w.topk_high_bp], "check_every": w.check_every,
                            "powersgd_residual": "eager" if args.eager else "lazy (applied on the next load)",
+                           "optimizer_tail": "Nesterov update fused into the step" if args.sgd_tail else "none",
                            "gradient_bytes_per_step": grad_bytes_step,
                            "l2_policy": f"inputs larger than L2: {RING} gradient batches of "
                                         f"{4 * W * table.stride / 1e6:.0f} MB cycled, no flush",
@@ -351,6 +367,142 @@ def main():
                 "step_ms": {"median": float(np.median(per_step)), "min": float(per_step.min()),
                             "max": float(per_step.max())},
                 "kernels": kernels}
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def run_batch_mode(args, w, ring, dev, rank, world, local_rank):
+    """Batch-size mode on the workload's layer table: a step = n_accum accumulations of [W, N] micro-batch
+    gradients, one average over workers fused with the Nesterov update, and the whole-model detector every
+    check_every steps.  Same timing rules and JSON keys as the compression bench."""
+    import torch.distributed as dist
+    from paper_2010_16248_b200 import dist_util, pipeline
+    table, W, n_accum = w.table, w.n_workers, args.n_accum
+    params = torch.zeros(table.stride, device=dev)
+    bs = pipeline.BatchSizeStep(table, W, b_low=512, b_high=512 * n_accum, micro_batch=512, eta=w.eta, device=dev,
+                                optimizer={"params": params, "lr": 0.1, "momentum": 0.9})
+    grad_bytes_step = 4.0 * W * table.n_params * n_accum
+    step_no = 0
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def one_step():
+        nonlocal step_no
+        n = 0
+        for j in range(n_accum):
+            bs.micro_step(ring[(step_no * n_accum + j) % RING])
+            n += bs.ctx.last_launch_count()
+        bs.apply()
+        n += bs.ctx.last_launch_count()
+        step_no += 1
+        if step_no % w.check_every == 0:
+            bs.ctx.acc_layer_norms(bs.delta, 1, bs.norm2_layers)
+            n += bs.ctx.last_launch_count()
+            bs.ctx.acc_detect_batch(bs.norm2_layers, bs.norm2_prev, 0.1, 0.1, bs.b_low, bs.b_high, bs.batch,
+                                    bs.lr_scale, bs.delta)
+            n += bs.ctx.last_launch_count()
+        return n
+
+    for _ in range(args.warmup):
+        one_step()
+    barrier()
+    K = args.steps
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    if sampler:
+        sampler.start()
+        time.sleep(0.25)
+    barrier()
+    t0 = time.time()
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    start.record()
+    gpu_launches = sum(one_step() for _ in range(K))
+    stop.record()
+    barrier()
+    t1 = time.time()
+    clocks = sampler.stop(t0, t1) if sampler else None
+    ms_per_step = dist_util.max_over_ranks(start.elapsed_time(stop), dev) / K
+    value = dist_util.whole_job_throughput(grad_bytes_step, ms_per_step, world) / 1e9
+
+    bs.ctx.acc_profile_enable(True)
+    for _ in range(K):
+        one_step()
+    torch.cuda.synchronize()
+    prof = bs.ctx.acc_profile_read()
+    bs.ctx.acc_profile_enable(False)
+    peak, peak_src = _peaks()
+    # algorithmic bytes per launch: accumulate reads g and acc and writes acc for every worker (the first
+    # micro-batch of a step skips the read of acc), plus the decider's read-modify-write of delta;
+    # average reads W accumulators, writes out, and reads + writes params and momentum
+    n = table.n_params
+    alg = {"batch_accumulate_kernel": (12.0 * W - 4.0 * W / n_accum + 8.0) * n,
+           "batch_average_kernel": (4.0 * W + 4.0 + 16.0) * n}
+    total_k_ms = sum(ms for ms, _ in prof.values())
+    kernels = {}
+    for name, (ms, cnt) in sorted(prof.items(), key=lambda kv: -kv[1][0]):
+        avg = ms / cnt
+        a = alg.get(name)
+        kernels[name] = {"launches": cnt, "ms_total": round(ms, 4), "share": round(ms / total_k_ms, 4),
+                         "avg_ms": round(avg, 5), "alg_gbs": round(a / (avg * 1e-3) / 1e9, 1) if a else None}
+    dom = next(iter(kernels))
+    achieved = alg[dom] / (prof[dom][0] / prof[dom][1] * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "kernel": dom, "achieved": round(achieved, 1), "peak": peak, "unit": "GB/s",
+                "frac": round(achieved / peak, 4), "peak_source": peak_src, "traffic": None,
+                "alg_bytes_per_launch": alg[dom]}
+
+    # end to end: each micro-batch uploaded from pinned host memory (copy stream, two staging buffers); the
+    # step's result (the updated parameters) read back to the host
+    ke = max(1, min(args.e2e_steps, K))
+    host = [torch.empty(W, table.stride, dtype=torch.float32).pin_memory() for _ in range(2)]
+    for i in range(2):
+        host[i].copy_(ring[i])
+    stage = [torch.empty(W, table.stride, device=dev) for _ in range(2)]
+    params_host = torch.empty(table.stride, dtype=torch.float32).pin_memory()
+    copy = torch.cuda.Stream(device=dev)
+    up = [torch.cuda.Event() for _ in range(2)]
+    used = [torch.cuda.Event() for _ in range(2)]
+    main = torch.cuda.current_stream(dev)
+    barrier()
+    s2, e2 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    s2.record()
+    i = 0
+    for _ in range(ke):
+        for j in range(n_accum):
+            b = i & 1
+            with torch.cuda.stream(copy):
+                if i >= 2:
+                    copy.wait_event(used[b])
+                stage[b].copy_(host[b], non_blocking=True)
+                up[b].record(copy)
+            main.wait_event(up[b])
+            bs.micro_step(stage[b])
+            used[b].record(main)
+            i += 1
+        bs.apply()
+        params_host.copy_(params, non_blocking=True)
+    e2.record()
+    barrier()
+    e2e_ms = dist_util.max_over_ranks(s2.elapsed_time(e2), dev)
+    e2e = {"value": dist_util.whole_job_throughput(grad_bytes_step, e2e_ms / ke, world) / 1e9, "unit": UNIT,
+           "steps": ke, "ms_per_step": e2e_ms / ke, "h2d_bytes_per_step": int(4 * W * table.stride * n_accum),
+           "d2h_bytes_per_step": int(4 * table.stride)}
+    if rank == 0:
+        line = {"metric": "batch_mode_gradient_throughput", "value": value, "unit": UNIT, "n_gpus": world, "steps": K,
+                "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+                "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+                "config": {"workload": w.name + " layer table, batch-size mode", "n_workers": W,
+                           "params": table.n_params, "n_accum": n_accum, "check_every": w.check_every,
+                           "optimizer_tail": "Nesterov update fused into the average",
+                           "gradient_bytes_per_step": grad_bytes_step,
+                           "l2_policy": f"inputs larger than L2: {RING} gradient batches cycled, no flush",
+                           "multi_gpu": "independent replicas, no collective"},
+                "clocks": clocks, "e2e": e2e, "gpu_launches": gpu_launches, "roofline": roofline,
+                "cpu_baseline": None, "kernels": kernels}
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.barrier()
