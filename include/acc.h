@@ -226,6 +226,49 @@ int acc_batch_average(acc_ctx* ctx, const float* acc, int32_t n_accum, float* ou
 int acc_detect_batch(acc_ctx* ctx, const double* norm2_layers, double* norm2_prev, float lr_curr, float lr_next,
                      int32_t b_low, int32_t b_high, int32_t* batch, float* lr_scale, float* delta, void* stream);
 
+/* ---- Real workers (Section 3: every worker computes its gradient on its own GPU; Section 5.1: the PowerSGD
+ * factors are exchanged by all-reduce, TopK's values and indices by all-gather) ------------------------------
+ * A context then holds this GPU's workers only (n_workers = workers on this GPU, the same on every GPU), and a
+ * step is split around the exchanges, which the caller performs with its collective library between the calls
+ * (sum over GPUs, in place):
+ *   acc_powersgd_phase1: first pass of acc_powersgd_step over this GPU's workers; then x1 <- this GPU's rows of
+ *                        the unnormalised P (ranks beyond r as zeros) followed by the VECTOR layers' local means.
+ *       -- all-reduce(sum) x1 --
+ *   acc_powersgd_phase2: P^ = Gram-Schmidt(scale * x1 rows); x2 <- this GPU's rows of Q' = Mbar^T P^.
+ *       -- all-reduce(sum) x2 --
+ *   acc_powersgd_phase3: Q[:, :r] <- scale * x2;  VECTOR out <- scale * x1 tail;  out = P^ Q^T and the residual as in
+ *                        acc_powersgd_step; with params != NULL the optimiser tail as in acc_powersgd_step_sgd.
+ * scale = 1 / (number of GPUs).  With one GPU and scale 1 the three calls give the results of acc_powersgd_step
+ * up to fp32 rounding (the fold of P changes the order of a few additions).
+ * acc_exchange_layout: lengths in floats of x1 (4*p_rows + packed VECTOR elements) and x2 (4*q_rows), and the
+ * length of the packed VECTOR region alone (each VECTOR layer, in order, starts at a multiple of 4 floats).
+ * Device pointers: x1, x2 16-byte aligned, caller-owned; the others as in acc_powersgd_step.                */
+int acc_exchange_layout(const acc_ctx* ctx, int64_t* x1_floats, int64_t* x2_floats, int64_t* vec_floats);
+int acc_powersgd_phase1(acc_ctx* ctx, const float* grads, float* err, float* q, float* p_hat,
+                        const uint8_t* level, float* out, float* delta, float* x1, void* stream);
+int acc_powersgd_phase2(acc_ctx* ctx, const float* x1, float scale, float* p_hat, const uint8_t* level,
+                        const float* out, float* x2, void* stream);
+int acc_powersgd_phase3(acc_ctx* ctx, float* err, float* q, const float* p_hat, const uint8_t* level,
+                        const float* x1, const float* x2, float scale, float* out, float* params, float* mom,
+                        const float* hyper, void* stream);
+
+/* TopK with real workers: values and indices are gathered from every worker (Section 5.1).
+ *   acc_topk_compress: acc_topk_step without its last pass, over this GPU's workers: vals / idx / counts and the
+ *                      error memories as in acc_topk_step; vec_packed <- this GPU's means of the VECTOR layers
+ *                      (packed as in acc_exchange_layout, vec_floats floats); delta += g_decider when != NULL.
+ *       -- all-gather vals, idx, counts (every GPU contributes its whole buffers); all-reduce(sum) vec_packed --
+ *   acc_topk_decompress: out[l] = (1/n_sets) sum_j scatter(idx_j, val_j) over the n_sets gathered packed sets
+ *                      (set j at entry j*capacity of vals_all / idx_all, its counts at counts_all[j*L ..]), sets
+ *                      added in order; VECTOR layers: out = vec_scale * vec_packed.  Each set's entries must be in
+ *                      ascending index order per layer (as acc_topk_compress writes them).  With params != NULL
+ *                      the optimiser tail is applied to out as it is written.
+ * With the sets of one GPU (n_sets = n_workers, vec_scale = 1) the pair gives the bits of acc_topk_step.    */
+int acc_topk_compress(acc_ctx* ctx, const float* grads, float* err, const uint8_t* level, float* vals,
+                      int32_t* idx, int32_t* counts, float* delta, float* vec_packed, void* stream);
+int acc_topk_decompress(acc_ctx* ctx, const float* vals_all, const int32_t* idx_all, const int32_t* counts_all,
+                        int32_t n_sets, const float* vec_packed, float vec_scale, float* out, float* params,
+                        float* mom, const float* hyper, void* stream);
+
 /* Device-side condition of the kernels launched so far on this context (no counterpart in the paper).
  * The pipelined kernels wait for their asynchronous shared-memory copies with a bounded number of polls;
  * should a wait ever give up, the block stores ACC_ETIMEOUT in a status word and returns instead of

@@ -47,7 +47,9 @@ EXPORTS = ["acc_workspace_bytes", "acc_create", "acc_destroy", "acc_factor_layou
            "acc_floats_sent", "acc_last_launch_count", "acc_strerror", "acc_profile_enable", "acc_profile_read",
            "acc_profile_kernel_count", "acc_profile_kernel_name", "acc_sumsq_static", "acc_powersgd_flush", "acc_device_status", "acc_topk_last_paths",
            "acc_layer_diff_norms", "acc_detect_regime_diff", "acc_sgd_nesterov", "acc_powersgd_step_sgd",
-           "acc_topk_step_sgd", "acc_batch_accumulate", "acc_batch_average", "acc_detect_batch"]
+           "acc_topk_step_sgd", "acc_batch_accumulate", "acc_batch_average", "acc_detect_batch",
+           "acc_exchange_layout", "acc_powersgd_phase1", "acc_powersgd_phase2", "acc_powersgd_phase3",
+           "acc_topk_compress", "acc_topk_decompress"]
 
 _lib = None
 
@@ -97,6 +99,12 @@ def lib() -> C.CDLL:
     L.acc_batch_accumulate.argtypes = [vp, vp, vp, vp, i32, vp]
     L.acc_batch_average.argtypes = [vp, vp, i32, vp, vp, vp, vp, vp]
     L.acc_detect_batch.argtypes = [vp, vp, vp, f32, f32, i32, i32, vp, vp, vp, vp]
+    L.acc_exchange_layout.argtypes = [vp, C.POINTER(i64), C.POINTER(i64), C.POINTER(i64)]
+    L.acc_powersgd_phase1.argtypes = [vp] * 10
+    L.acc_powersgd_phase2.argtypes = [vp, vp, f32, vp, vp, vp, vp, vp]
+    L.acc_powersgd_phase3.argtypes = [vp, vp, vp, vp, vp, vp, vp, f32, vp, vp, vp, vp, vp]
+    L.acc_topk_compress.argtypes = [vp] * 10
+    L.acc_topk_decompress.argtypes = [vp, vp, vp, vp, i32, vp, f32, vp, vp, vp, vp, vp]
     for name in EXPORTS:
         if name not in ("acc_floats_sent", "acc_last_launch_count", "acc_strerror", "acc_profile_kernel_count",
                         "acc_profile_kernel_name"):
@@ -183,6 +191,9 @@ class Context:
         L.acc_topk_layout(self._h, so, kl, kh, C.byref(cap))
         self.seg_offset, self.k_low, self.k_high = (np.array(a[:], np.int64) for a in (so, kl, kh))
         self.capacity = int(cap.value)
+        x1, x2, vf = C.c_int64(), C.c_int64(), C.c_int64()
+        L.acc_exchange_layout(self._h, C.byref(x1), C.byref(x2), C.byref(vf))
+        self.x1_floats, self.x2_floats, self.vec_floats = int(x1.value), int(x2.value), int(vf.value)
 
     def close(self):
         if getattr(self, "_h", None):
@@ -281,6 +292,41 @@ class Context:
                                            int(b_low), int(b_high), _ptr(batch, torch.int32),
                                            _ptr(lr_scale, torch.float32), _ptr(delta, torch.float32),
                                            _stream(stream)), "acc_detect_batch")
+
+    def acc_powersgd_phase1(self, grads, err, q, p_hat, level, out, delta, x1, stream=None):
+        f = torch.float32
+        self._check(lib().acc_powersgd_phase1(self._h, _ptr(grads, f), _ptr(err, f), _ptr(q, f), _ptr(p_hat, f),
+                                              _ptr(level, torch.uint8), _ptr(out, f), _ptr(delta, f), _ptr(x1, f),
+                                              _stream(stream)), "acc_powersgd_phase1")
+
+    def acc_powersgd_phase2(self, x1, scale, p_hat, level, out, x2, stream=None):
+        f = torch.float32
+        self._check(lib().acc_powersgd_phase2(self._h, _ptr(x1, f), float(scale), _ptr(p_hat, f),
+                                              _ptr(level, torch.uint8), _ptr(out, f), _ptr(x2, f), _stream(stream)),
+                    "acc_powersgd_phase2")
+
+    def acc_powersgd_phase3(self, err, q, p_hat, level, x1, x2, scale, out, params=None, mom=None, hyper=None,
+                            stream=None):
+        f = torch.float32
+        self._check(lib().acc_powersgd_phase3(self._h, _ptr(err, f), _ptr(q, f), _ptr(p_hat, f),
+                                              _ptr(level, torch.uint8), _ptr(x1, f), _ptr(x2, f), float(scale),
+                                              _ptr(out, f), _ptr(params, f), _ptr(mom, f), _ptr(hyper, f),
+                                              _stream(stream)), "acc_powersgd_phase3")
+
+    def acc_topk_compress(self, grads, err, level, vals, idx, counts, delta, vec_packed, stream=None):
+        f = torch.float32
+        self._check(lib().acc_topk_compress(self._h, _ptr(grads, f), _ptr(err, f), _ptr(level, torch.uint8),
+                                            _ptr(vals, f), _ptr(idx, torch.int32), _ptr(counts, torch.int32),
+                                            _ptr(delta, f), _ptr(vec_packed, f), _stream(stream)),
+                    "acc_topk_compress")
+
+    def acc_topk_decompress(self, vals_all, idx_all, counts_all, n_sets, vec_packed, vec_scale, out, params=None,
+                            mom=None, hyper=None, stream=None):
+        f = torch.float32
+        self._check(lib().acc_topk_decompress(self._h, _ptr(vals_all, f), _ptr(idx_all, torch.int32),
+                                              _ptr(counts_all, torch.int32), int(n_sets), _ptr(vec_packed, f),
+                                              float(vec_scale), _ptr(out, f), _ptr(params, f), _ptr(mom, f),
+                                              _ptr(hyper, f), _stream(stream)), "acc_topk_decompress")
 
     def acc_profile_enable(self, enable: bool):
         self._check(lib().acc_profile_enable(self._h, int(bool(enable))), "acc_profile_enable")

@@ -57,7 +57,7 @@ static int make_plan(const acc_config* cfg, Plan& p) {
     memset(&o, 0, sizeof(o));
     o.offset = d.offset; o.rows = d.rows; o.cols = d.cols; o.kind = d.kind;
     o.inv_cols = 1.0 / (double)d.cols;
-    o.q_row = o.p_row = o.mat = -1; o.seg_off = -1; o.part_base = -1;
+    o.q_row = o.p_row = o.mat = -1; o.seg_off = -1; o.part_base = -1; o.vec_off = -1;
     o.vec = (d.cols % 4 == 0) ? 4 : (d.cols % 2 == 0) ? 2 : 1;
     const long long size = (long long)d.rows * d.cols;
     // flat tiles
@@ -69,9 +69,14 @@ static int make_plan(const acc_config* cfg, Plan& p) {
       p.tiles.push_back(t);
     }
     o.ntiles = (int)p.tiles.size() - o.tile0;
-    if (d.kind != ACC_MATRIX) continue;
+    if (d.kind != ACC_MATRIX) {
+      o.vec_off = p.vec_floats;
+      p.vec_floats += (size + 3) / 4 * 4;
+      continue;
+    }
     o.mat = p.n_mat++;
     p.max_rows = std::max(p.max_rows, d.rows);
+    p.max_cols = std::max(p.max_cols, d.cols);
     p.mat_layers.push_back(l);
     o.q_row = (int)p.q_rows; p.q_rows += d.cols;
     o.p_row = (int)p.p_rows; p.p_rows += d.rows;
@@ -317,6 +322,79 @@ int acc_powersgd_step_sgd(acc_ctx* ctx, const float* grads, float* err, float* q
                                 static_cast<cudaStream_t>(stream)));
 }
 
+int acc_exchange_layout(const acc_ctx* ctx, int64_t* x1_floats, int64_t* x2_floats, int64_t* vec_floats) {
+  if (!ctx) return ACC_EINVAL;
+  if (x1_floats) *x1_floats = 4 * ctx->plan.p_rows + ctx->plan.vec_floats;
+  if (x2_floats) *x2_floats = 4 * ctx->plan.q_rows;
+  if (vec_floats) *vec_floats = ctx->plan.vec_floats;
+  return ACC_OK;
+}
+
+int acc_powersgd_phase1(acc_ctx* ctx, const float* grads, float* err, float* q, float* p_hat, const uint8_t* level,
+                        float* out, float* delta, float* x1, void* stream) {
+  if (!ctx || !grads || !err || !q || !p_hat || !level || !out || !x1) return ACC_EINVAL;
+  if (!aligned16(grads) || !aligned16(err) || !aligned16(q) || !aligned16(p_hat) || !aligned16(out) ||
+      !aligned16(delta) || !aligned16(x1))
+    return ACC_EALIGN;
+  ctx->last_launches = 0;
+  return finish(launch_powersgd_phase1(ctx, grads, err, q, p_hat, level, out, delta, x1,
+                                       static_cast<cudaStream_t>(stream)));
+}
+
+int acc_powersgd_phase2(acc_ctx* ctx, const float* x1, float scale, float* p_hat, const uint8_t* level,
+                        const float* out, float* x2, void* stream) {
+  if (!ctx || !x1 || !p_hat || !level || !out || !x2) return ACC_EINVAL;
+  if (!aligned16(x1) || !aligned16(p_hat) || !aligned16(out) || !aligned16(x2)) return ACC_EALIGN;
+  ctx->last_launches = 0;
+  return finish(launch_powersgd_phase2(ctx, x1, scale, p_hat, level, out, x2, static_cast<cudaStream_t>(stream)));
+}
+
+int acc_powersgd_phase3(acc_ctx* ctx, float* err, float* q, const float* p_hat, const uint8_t* level,
+                        const float* x1, const float* x2, float scale, float* out, float* params, float* mom,
+                        const float* hyper, void* stream) {
+  if (!ctx || !err || !q || !p_hat || !level || !x1 || !x2 || !out) return ACC_EINVAL;
+  if (!aligned16(err) || !aligned16(q) || !aligned16(p_hat) || !aligned16(x1) || !aligned16(x2) || !aligned16(out))
+    return ACC_EALIGN;
+  SgdTail tail{nullptr, nullptr, nullptr};
+  if (params) {
+    const int st = check_tail(params, mom, hyper);
+    if (st != ACC_OK) return st;
+    tail = SgdTail{params, mom, hyper};
+  }
+  ctx->last_launches = 0;
+  return finish(launch_powersgd_phase3(ctx, err, q, p_hat, level, x1, x2, scale, out, tail,
+                                       static_cast<cudaStream_t>(stream)));
+}
+
+int acc_topk_compress(acc_ctx* ctx, const float* grads, float* err, const uint8_t* level, float* vals, int32_t* idx,
+                      int32_t* counts, float* delta, float* vec_packed, void* stream) {
+  if (!ctx || !grads || !err || !level || !vals || !idx || !counts) return ACC_EINVAL;
+  if (!vec_packed && ctx->plan.vec_floats > 0) return ACC_EINVAL;
+  if (!aligned16(grads) || !aligned16(err) || !aligned16(vals) || !aligned16(idx) || !aligned16(delta) ||
+      !aligned16(vec_packed))
+    return ACC_EALIGN;
+  ctx->last_launches = 0;
+  return finish(launch_topk_compress(ctx, grads, err, level, vals, idx, counts, delta, vec_packed,
+                                     static_cast<cudaStream_t>(stream)));
+}
+
+int acc_topk_decompress(acc_ctx* ctx, const float* vals_all, const int32_t* idx_all, const int32_t* counts_all,
+                        int32_t n_sets, const float* vec_packed, float vec_scale, float* out, float* params,
+                        float* mom, const float* hyper, void* stream) {
+  if (!ctx || !vals_all || !idx_all || !counts_all || !out || n_sets < 1) return ACC_EINVAL;
+  if (!vec_packed && ctx->plan.vec_floats > 0) return ACC_EINVAL;
+  if (!aligned16(vals_all) || !aligned16(idx_all) || !aligned16(out) || !aligned16(vec_packed)) return ACC_EALIGN;
+  SgdTail tail{nullptr, nullptr, nullptr};
+  if (params) {
+    const int st = check_tail(params, mom, hyper);
+    if (st != ACC_OK) return st;
+    tail = SgdTail{params, mom, hyper};
+  }
+  ctx->last_launches = 0;
+  return finish(launch_topk_decompress_packed(ctx, vals_all, idx_all, counts_all, n_sets, vec_packed, vec_scale, out,
+                                              tail, static_cast<cudaStream_t>(stream)));
+}
+
 int acc_sgd_nesterov(acc_ctx* ctx, const float* d, float* params, float* mom, const float* hyper, void* stream) {
   if (!ctx || !d) return ACC_EINVAL;
   if (!aligned16(d)) return ACC_EALIGN;
@@ -444,7 +522,8 @@ const char* acc_profile_kernel_name(int32_t i) {
       "topk_collect_kernel", "topk_pick3_kernel", "topk_tile_counts_kernel",
       "topk_hist2_list_kernel", "topk_hist3_list_kernel", "topk_finalize_staged_kernel",
       "psgd_orthonormalise_block_kernel", "sgd_tiles_kernel", "batch_accumulate_kernel", "batch_average_kernel",
-      "detect_batch_kernel"};
+      "detect_batch_kernel", "psgd_pfold_kernel", "vec_exchange_kernel", "psgd_qmerge_kernel",
+      "topk_decompress_packed_kernel"};
   return (i >= 0 && i < PH_COUNT) ? names[i] : "";
 }
 

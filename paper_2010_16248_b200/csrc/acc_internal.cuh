@@ -33,6 +33,7 @@ struct DevLayer {
   int cand_cap;         // slots of that list (the list path is taken when bucket b1 fits)
   long long part_base;  // first float4 of the layer's Q partials
   int slab_rows, nslabs;  // row slabs of the Q-partial pass
+  long long vec_off;      // VECTOR layers: first float of the layer inside the packed exchange region, else -1
 };
 
 struct ColItem { int layer, slab, row0, nrows, col0; };  // (row slab, column block) of a MATRIX layer
@@ -55,6 +56,7 @@ enum Phase {
   PH_PSGD_PROJECT, PH_PSGD_ORTHO, PH_PSGD_QPARTIAL, PH_PSGD_QREDUCE, PH_PSGD_RESIDUAL,
   PH_TOPK_EF_HIST1, PH_TOPK_PICK1, PH_TOPK_HIST2, PH_TOPK_PICK2, PH_TOPK_HIST3, PH_TOPK_PICK3_SCAN, PH_TOPK_SELECT,
   PH_TOPK_DECOMPRESS, PH_PSGD_FLUSH, PH_TOPK_COLLECT, PH_TOPK_PICK3, PH_TOPK_TILE_COUNTS, PH_TOPK_HIST2_LIST, PH_TOPK_HIST3_LIST, PH_TOPK_FINALIZE_STAGED, PH_PSGD_ORTHO_BLOCK, PH_SGD_TILES, PH_BATCH_ACCUMULATE, PH_BATCH_AVERAGE, PH_DETECT_BATCH,
+  PH_PSGD_PFOLD, PH_VEC_EXCHANGE, PH_PSGD_QMERGE, PH_TOPK_DECOMPRESS_PACKED,
   PH_COUNT
 };
 
@@ -70,6 +72,8 @@ struct Plan {
   long long q_rows = 0, p_rows = 0, capacity = 0, part_f4 = 0, cand_total = 0, ppart_f4 = 0;
   int n_mat = 0;
   int max_rows = 0;  // most rows of any MATRIX layer
+  int max_cols = 0;  // most columns of any MATRIX layer
+  long long vec_floats = 0;  // packed VECTOR elements (each layer starts at a multiple of 4)
   // workspace offsets (bytes)
   size_t o_layers = 0, o_col_items = 0, o_tiles = 0, o_mat_layers = 0, o_vec_tiles = 0, o_mat_tiles = 0, o_status = 0,
          o_part = 0, o_ppart = 0, o_pending = 0, o_norm_part = 0, o_hist = 0, o_sel = 0, o_pred = 0, o_cand = 0, o_tile_cand = 0, o_tile_cnt = 0, o_tile_h3 = 0, o_tile_pre = 0,
@@ -132,9 +136,23 @@ cudaError_t launch_detect(acc_ctx* ctx, const double* n2c, double* n2p, const do
 cudaError_t launch_powersgd(acc_ctx* ctx, const float* grads, float* err, float* q, float* p_hat,
                             const uint8_t* level, float* out, float* delta, SgdTail tail, cudaStream_t s);
 cudaError_t prepare_powersgd();
+// Real workers: the step in three parts, around the two exchanges (x1: P rows + packed VECTOR means, x2: Q' rows).
+cudaError_t launch_powersgd_phase1(acc_ctx* ctx, const float* grads, float* err, float* q, float* p_hat,
+                                   const uint8_t* level, float* out, float* delta, float* x1, cudaStream_t s);
+cudaError_t launch_powersgd_phase2(acc_ctx* ctx, const float* x1, float scale, float* p_hat, const uint8_t* level,
+                                   const float* out, float* x2, cudaStream_t s);
+cudaError_t launch_powersgd_phase3(acc_ctx* ctx, float* err, float* q, const float* p_hat, const uint8_t* level,
+                                   const float* x1, const float* x2, float scale, float* out, SgdTail tail,
+                                   cudaStream_t s);
 cudaError_t launch_powersgd_flush(acc_ctx* ctx, float* err, const float* q, const float* p_hat, cudaStream_t s);
 cudaError_t launch_topk(acc_ctx* ctx, const float* grads, float* err, const uint8_t* level, float* vals,
                         int32_t* idx, int32_t* counts, float* out, float* delta, SgdTail tail, cudaStream_t s);
+// Real workers: the TopK step in two halves around the all-gather of the packed sets.
+cudaError_t launch_topk_compress(acc_ctx* ctx, const float* grads, float* err, const uint8_t* level, float* vals,
+                                 int32_t* idx, int32_t* counts, float* delta, float* vec_packed, cudaStream_t s);
+cudaError_t launch_topk_decompress_packed(acc_ctx* ctx, const float* vals, const int32_t* idx, const int32_t* counts,
+                                          int n_sets, const float* vec_packed, float vec_scale, float* out,
+                                          SgdTail tail, cudaStream_t s);
 // Optimiser tail on its own over the given tiles (tile_ids == nullptr: all tiles, in order).
 cudaError_t launch_sgd_tiles(acc_ctx* ctx, const int* tile_ids, int n, const float* d, SgdTail tail, cudaStream_t s);
 cudaError_t launch_batch_accumulate(acc_ctx* ctx, const float* grads, float* acc, float* delta, int first,

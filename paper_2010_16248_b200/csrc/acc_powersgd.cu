@@ -398,11 +398,29 @@ __device__ __forceinline__ double cluster_sum(double v, double* sm_warp, double*
   return total;
 }
 
+// Row i of the unnormalised P of layer L: the sum, in tile order, of the partial rows the project pass left for
+// the tiles the row touches -- or, when the rows were exchanged between GPUs (p_in != nullptr: the summed rows
+// of all ranks, [p_rows] float4), p_scale times the exchanged row.
+__device__ __forceinline__ float4 load_p_row(const DevLayer& L, int i, const float4* __restrict__ p_part,
+                                             const float4* __restrict__ p_in, float p_scale) {
+  if (p_in != nullptr) {
+    const float4 v = p_in[L.p_row + i];
+    return make_float4(v.x * p_scale, v.y * p_scale, v.z * p_scale, v.w * p_scale);
+  }
+  const int first_tile = (i * L.cols) / kTile, last_tile = (i * L.cols + L.cols - 1) / kTile;
+  const float4* pp = p_part + L.ppart_base + (long long)i * L.nslots;
+  float4 acc = pp[0];
+  for (int sl = 1; sl <= last_tile - first_tile; ++sl) {
+    acc.x += pp[sl].x; acc.y += pp[sl].y; acc.z += pp[sl].z; acc.w += pp[sl].w;
+  }
+  return acc;
+}
+
 __global__ void __cluster_dims__(kOrthoCluster, 1, 1) __launch_bounds__(kOrthoThreads)
 psgd_orthonormalise_cluster_kernel(const DevLayer* __restrict__ layers, const int* __restrict__ mat_layers,
                                    float* __restrict__ p, const float4* __restrict__ p_part,
                                    const uint8_t* __restrict__ level, int* __restrict__ pending, int rank_low,
-                                   int rank_high, float eps) {
+                                   int rank_high, float eps, const float4* __restrict__ p_in, float p_scale) {
   __shared__ double sm_warp[kOrthoThreads / 32];
   __shared__ double slots[2];
   cg::cluster_group cluster = cg::this_cluster();
@@ -421,13 +439,8 @@ psgd_orthonormalise_cluster_kernel(const DevLayer* __restrict__ layers, const in
     const int i = row_lo + k * kOrthoThreads + (int)threadIdx.x;
     v[k] = make_float4(0.f, 0.f, 0.f, 0.f);
     if (i < row_hi) {
-      // P[i] = sum, in tile order, of the partial rows the project pass left; ranks beyond r keep their value
-      const int first_tile = (i * L.cols) / kTile, last_tile = (i * L.cols + L.cols - 1) / kTile;
-      const float4* pp = p_part + L.ppart_base + (long long)i * L.nslots;
-      float4 acc = pp[0];
-      for (int sl = 1; sl <= last_tile - first_tile; ++sl) {
-        acc.x += pp[sl].x; acc.y += pp[sl].y; acc.z += pp[sl].z; acc.w += pp[sl].w;
-      }
+      // ranks beyond r keep their value
+      const float4 acc = load_p_row(L, i, p_part, p_in, p_scale);
       const float4 old = P4[i];
       v[k] = make_float4(acc.x, r > 1 ? acc.y : old.y, r > 2 ? acc.z : old.z, r > 3 ? acc.w : old.w);
     }
@@ -474,7 +487,7 @@ __global__ void __launch_bounds__(1024)
 psgd_orthonormalise_kernel(const DevLayer* __restrict__ layers, const int* __restrict__ mat_layers,
                            float* __restrict__ p, const float4* __restrict__ p_part,
                            const uint8_t* __restrict__ level, int* __restrict__ pending, int rank_low, int rank_high,
-                           float eps) {
+                           float eps, const float4* __restrict__ p_in, float p_scale) {
   __shared__ double sm[32];
   const int l = mat_layers[blockIdx.x];
   const DevLayer L = layers[l];
@@ -483,14 +496,8 @@ psgd_orthonormalise_kernel(const DevLayer* __restrict__ layers, const int* __res
   if (pending != nullptr && threadIdx.x == 0) pending[l] = r;  // lazy mode: this step's residual stays pending
   float* P = p + 4ll * L.p_row;
   const int n = L.rows;
-  // P[i] = sum, in tile order, of the partial rows the project pass left for the tiles row i touches
   for (int i = threadIdx.x; i < n; i += blockDim.x) {
-    const int first_tile = (i * L.cols) / kTile, last_tile = (i * L.cols + L.cols - 1) / kTile;
-    const float4* pp = p_part + L.ppart_base + (long long)i * L.nslots;
-    float4 acc = pp[0];
-    for (int sl = 1; sl <= last_tile - first_tile; ++sl) {
-      acc.x += pp[sl].x; acc.y += pp[sl].y; acc.z += pp[sl].z; acc.w += pp[sl].w;
-    }
+    const float4 acc = load_p_row(L, i, p_part, p_in, p_scale);
     P[4 * i] = acc.x;
     if (r > 1) P[4 * i + 1] = acc.y;
     if (r > 2) P[4 * i + 2] = acc.z;
@@ -618,7 +625,7 @@ psgd_decompress_kernel(const DevLayer* __restrict__ layers, const ColItem* __res
 __global__ void __launch_bounds__(256)
 psgd_qreduce_kernel(const DevLayer* __restrict__ layers, const int* __restrict__ mat_layers,
                     const float4* __restrict__ part, float* __restrict__ q, const uint8_t* __restrict__ level,
-                    int rank_low, int rank_high) {
+                    int rank_low, int rank_high, float4* __restrict__ q_sum) {
   __shared__ float4 sm[8][32];
   const int l = mat_layers[blockIdx.y];
   const DevLayer L = layers[l];
@@ -638,6 +645,10 @@ psgd_qreduce_kernel(const DevLayer* __restrict__ layers, const int* __restrict__
     float4 t = sm[0][cx];
     for (int g = 1; g < 8; ++g) { t.x += sm[g][cx].x; t.y += sm[g][cx].y; t.z += sm[g][cx].z; t.w += sm[g][cx].w; }
     const int r = level[l] ? rank_low : rank_high;
+    if (q_sum != nullptr) {  // real workers: this GPU's share goes to the exchange buffer, ranks beyond r as zeros
+      q_sum[L.q_row + col] = make_float4(t.x, r > 1 ? t.y : 0.f, r > 2 ? t.z : 0.f, r > 3 ? t.w : 0.f);
+      return;
+    }
     float4* Q4 = reinterpret_cast<float4*>(q) + L.q_row;
     float4 qv = Q4[col];
     qv.x = t.x;
@@ -740,21 +751,76 @@ cudaError_t prepare_powersgd() {
   return e;
 }
 
-cudaError_t launch_powersgd(acc_ctx* ctx, const float* grads, float* err, float* q, float* p_hat,
-                            const uint8_t* level, float* out, float* delta, SgdTail tail, cudaStream_t s) {
+// ---- real workers: the factors cross GPUs between the passes ---------------------------------------------
+// Exchange buffer 1: [p_rows] float4 rows of the unnormalised P (ranks beyond r as zeros), then the VECTOR
+// layers' means packed one after the other.  Exchange buffer 2: [q_rows] float4 rows of Q' (same convention).
+
+// One thread per row of P: folds the row's partials into exchange buffer 1.
+__global__ void __launch_bounds__(256)
+psgd_pfold_kernel(const DevLayer* __restrict__ layers, const int* __restrict__ mat_layers,
+                  const float4* __restrict__ p_part, const uint8_t* __restrict__ level, int rank_low, int rank_high,
+                  float4* __restrict__ p_sum) {
+  const int l = mat_layers[blockIdx.y];
+  const DevLayer L = layers[l];
+  const int i = blockIdx.x * 256 + threadIdx.x;
+  if (i >= L.rows) return;
+  const int r = level[l] ? rank_low : rank_high;
+  const float4 a = load_p_row(L, i, p_part, nullptr, 1.f);
+  p_sum[L.p_row + i] = make_float4(a.x, r > 1 ? a.y : 0.f, r > 2 ? a.z : 0.f, r > 3 ? a.w : 0.f);
+}
+
+// VECTOR tiles: packed <- out (PACK) or out <- scale * packed.
+template <bool PACK>
+__global__ void __launch_bounds__(256)
+vec_exchange_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict__ tiles,
+                    const int* __restrict__ vec_tiles, float* __restrict__ out, float* __restrict__ packed,
+                    float scale) {
+  const Tile t = tiles[vec_tiles[blockIdx.x]];
+  const DevLayer L = layers[t.layer];
+  float* o = out + L.offset + t.elem0;
+  float* x = packed + L.vec_off + t.elem0;
+  for (int i = threadIdx.x; i < t.nelem; i += blockDim.x) {
+    if (PACK) x[i] = o[i];
+    else o[i] = scale * x[i];
+  }
+}
+
+// One thread per column of Q: the first r ranks of Q' <- scale * exchanged sum.
+__global__ void __launch_bounds__(256)
+psgd_qmerge_kernel(const DevLayer* __restrict__ layers, const int* __restrict__ mat_layers,
+                   const float4* __restrict__ q_in, float scale, float* __restrict__ q,
+                   const uint8_t* __restrict__ level, int rank_low, int rank_high) {
+  const int l = mat_layers[blockIdx.y];
+  const DevLayer L = layers[l];
+  const int col = blockIdx.x * 256 + threadIdx.x;
+  if (col >= L.cols) return;
+  const int r = level[l] ? rank_low : rank_high;
+  const float4 t = q_in[L.q_row + col];
+  float4* Q4 = reinterpret_cast<float4*>(q) + L.q_row;
+  float4 qv = Q4[col];
+  qv.x = t.x * scale;
+  if (r > 1) qv.y = t.y * scale;
+  if (r > 2) qv.z = t.z * scale;
+  if (r > 3) qv.w = t.w * scale;
+  Q4[col] = qv;
+}
+
+// Pass 1 (both implementations of it; same arithmetic, same results).
+static void launch_psgd_project(acc_ctx* ctx, const float* grads, float* err, float* q, float* p_hat,
+                                const uint8_t* level, float* out, float* delta, cudaStream_t s) {
   const Plan& pl = ctx->plan;
   const acc_config& c = ctx->cfg;
   const int nt = (int)pl.tiles.size();
   const float inv_w = 1.0f / (float)c.n_workers;
   const bool lazy = (c.flags & ACC_FLAG_LAZY_RESIDUAL) != 0;
-  // Two implementations of the same pass (same arithmetic, same results): the persistent pipelined kernel
-  // wins once every SM has a long queue of stages (measured: 330 stages/SM -> 0.95 ms against 1.11 ms);
-  // on small sets its one-block-per-SM static split loses a few percent to tile quantisation.
+  // The persistent pipelined kernel wins once every SM has a long queue of stages (measured: 330 stages/SM ->
+  // 0.95 ms against 1.11 ms); on small sets its one-block-per-SM static split loses a few percent to tile
+  // quantisation.
   const long long stages_per_sm = (long long)pl.mat_tiles.size() * c.n_workers / (ctx->sm_count > 0 ? ctx->sm_count : 1);
   const bool pipelined = (c.flags & ACC_FLAG_PIPELINE_ALWAYS) ||
                          (!(c.flags & ACC_FLAG_PIPELINE_NEVER) && stages_per_sm >= kPipeMinStagesPerSm);
+  PhaseTimer pt(ctx, PH_PSGD_PROJECT, s);
   if (pipelined && pl.n_mat > 0) {
-    PhaseTimer pt(ctx, PH_PSGD_PROJECT, s);
     const int n_mt = (int)pl.mat_tiles.size(), n_vt = (int)pl.vec_tiles.size();
     const int grid = n_mt < ctx->sm_count ? n_mt : ctx->sm_count;
     if (lazy) {
@@ -766,62 +832,74 @@ cudaError_t launch_powersgd(acc_ctx* ctx, const float* grads, float* err, float*
           ctx->d_layers, ctx->d_tiles, ctx->d_mat_tiles, n_mt, ctx->d_vec_tiles, n_vt, grads, err, q, p_hat,
           ctx->d_ppart, nullptr, out, delta, c.worker_stride, c.n_workers, c.decider, inv_w, ctx->d_status);
     }
+  } else if (lazy) {
+    psgd_project_kernel<4, true><<<nt, 256, 0, s>>>(ctx->d_layers, ctx->d_tiles, grads, err, q, p_hat, ctx->d_ppart,
+                                                    level, ctx->d_pending, out, delta, c.worker_stride,
+                                                    c.n_workers, c.decider, inv_w);
   } else {
-    PhaseTimer pt(ctx, PH_PSGD_PROJECT, s);
-    if (lazy)
-      psgd_project_kernel<4, true><<<nt, 256, 0, s>>>(ctx->d_layers, ctx->d_tiles, grads, err, q, p_hat, ctx->d_ppart,
-                                                      level, ctx->d_pending, out, delta, c.worker_stride,
-                                                      c.n_workers, c.decider, inv_w);
-    else
-      psgd_project_kernel<4, false><<<nt, 256, 0, s>>>(ctx->d_layers, ctx->d_tiles, grads, err, q, p_hat,
-                                                       ctx->d_ppart, level, nullptr, out, delta, c.worker_stride,
-                                                       c.n_workers, c.decider, inv_w);
+    psgd_project_kernel<4, false><<<nt, 256, 0, s>>>(ctx->d_layers, ctx->d_tiles, grads, err, q, p_hat,
+                                                     ctx->d_ppart, level, nullptr, out, delta, c.worker_stride,
+                                                     c.n_workers, c.decider, inv_w);
   }
+}
+
+// Passes 2-4: P^ from the partial rows (or from exchanged rows p_in), Q' partials from Mbar (held in out),
+// their reduction into q (or into the exchange buffer q_sum).
+static void launch_psgd_ortho_q(acc_ctx* ctx, float* q, float* p_hat, const uint8_t* level, const float* out,
+                                const float4* p_in, float p_scale, float4* q_sum, cudaStream_t s) {
+  const Plan& pl = ctx->plan;
+  const acc_config& c = ctx->cfg;
+  const bool lazy = (c.flags & ACC_FLAG_LAZY_RESIDUAL) != 0;
+  bool any_cluster = false, any_block = false;
+  for (int l : pl.mat_layers) (ortho_by_cluster(pl.layers[l].rows) ? any_cluster : any_block) = true;
+  if (any_cluster) {
+    PhaseTimer pt(ctx, PH_PSGD_ORTHO, s);
+    psgd_orthonormalise_cluster_kernel<<<pl.n_mat * kOrthoCluster, kOrthoThreads, 0, s>>>(
+        ctx->d_layers, ctx->d_mat_layers, p_hat, ctx->d_ppart, level, lazy ? ctx->d_pending : nullptr, c.rank_low,
+        c.rank_high, c.gs_eps, p_in, p_scale);
+  }
+  if (any_block) {
+    PhaseTimer pt(ctx, PH_PSGD_ORTHO_BLOCK, s);
+    psgd_orthonormalise_kernel<<<pl.n_mat, 1024, 0, s>>>(ctx->d_layers, ctx->d_mat_layers, p_hat, ctx->d_ppart,
+                                                        level, lazy ? ctx->d_pending : nullptr, c.rank_low,
+                                                        c.rank_high, c.gs_eps, p_in, p_scale);
+  }
+  {
+    PhaseTimer pt(ctx, PH_PSGD_QPARTIAL, s);
+    psgd_qpartial_kernel<<<(unsigned)pl.col_items.size(), kColBlockThreads, 0, s>>>(
+        ctx->d_layers, ctx->d_col_items, out, p_hat, ctx->d_part);
+  }
+  {
+    PhaseTimer pt(ctx, PH_PSGD_QREDUCE, s);
+    psgd_qreduce_kernel<<<dim3((pl.max_cols + 31) / 32, pl.n_mat), 256, 0, s>>>(
+        ctx->d_layers, ctx->d_mat_layers, ctx->d_part, q, level, c.rank_low, c.rank_high, q_sum);
+  }
+}
+
+// Pass 5 (+ the optimiser tail): out = A, and in eager mode err_w -= A.
+static cudaError_t launch_psgd_finish(acc_ctx* ctx, float* err, const float* q, const float* p_hat,
+                                      const uint8_t* level, float* out, SgdTail tail, cudaStream_t s) {
+  const Plan& pl = ctx->plan;
+  const acc_config& c = ctx->cfg;
+  const int nt = (int)pl.tiles.size();
+  const bool lazy = (c.flags & ACC_FLAG_LAZY_RESIDUAL) != 0;
   if (pl.n_mat > 0) {
-    bool any_cluster = false, any_block = false;
-    for (int l : pl.mat_layers) (ortho_by_cluster(pl.layers[l].rows) ? any_cluster : any_block) = true;
-    if (any_cluster) {
-      PhaseTimer pt(ctx, PH_PSGD_ORTHO, s);
-      psgd_orthonormalise_cluster_kernel<<<pl.n_mat * kOrthoCluster, kOrthoThreads, 0, s>>>(
-          ctx->d_layers, ctx->d_mat_layers, p_hat, ctx->d_ppart, level, lazy ? ctx->d_pending : nullptr, c.rank_low,
-          c.rank_high, c.gs_eps);
-    }
-    if (any_block) {
-      PhaseTimer pt(ctx, PH_PSGD_ORTHO_BLOCK, s);
-      psgd_orthonormalise_kernel<<<pl.n_mat, 1024, 0, s>>>(ctx->d_layers, ctx->d_mat_layers, p_hat, ctx->d_ppart,
-                                                          level, lazy ? ctx->d_pending : nullptr, c.rank_low,
-                                                          c.rank_high, c.gs_eps);
-    }
-    {
-      PhaseTimer pt(ctx, PH_PSGD_QPARTIAL, s);
-      psgd_qpartial_kernel<<<(unsigned)pl.col_items.size(), kColBlockThreads, 0, s>>>(
-          ctx->d_layers, ctx->d_col_items, out, p_hat, ctx->d_part);
-    }
-    int max_cols = 0;
-    for (int l : pl.mat_layers) max_cols = max_cols > pl.layers[l].cols ? max_cols : pl.layers[l].cols;
-    {
-      PhaseTimer pt(ctx, PH_PSGD_QREDUCE, s);
-      psgd_qreduce_kernel<<<dim3((max_cols + 31) / 32, pl.n_mat), 256, 0, s>>>(
-          ctx->d_layers, ctx->d_mat_layers, ctx->d_part, q, level, c.rank_low, c.rank_high);
-    }
-    {
-      PhaseTimer pt(ctx, PH_PSGD_RESIDUAL, s);
-      const unsigned n_items = (unsigned)pl.col_items.size();
-      if (lazy && tail.params)
-        psgd_decompress_kernel<true><<<n_items, kColBlockThreads, 0, s>>>(
-            ctx->d_layers, ctx->d_col_items, q, p_hat, level, out, c.rank_low, c.rank_high, tail);
-      else if (lazy)
-        psgd_decompress_kernel<false><<<n_items, kColBlockThreads, 0, s>>>(
-            ctx->d_layers, ctx->d_col_items, q, p_hat, level, out, c.rank_low, c.rank_high, tail);
-      else if (tail.params)
-        psgd_residual_kernel<4, true, true, true><<<nt, 256, 0, s>>>(ctx->d_layers, ctx->d_tiles, err, q, p_hat, level,
-                                                                     nullptr, out, c.worker_stride, c.n_workers,
-                                                                     c.rank_low, c.rank_high, tail);
-      else
-        psgd_residual_kernel<4, true, true, false><<<nt, 256, 0, s>>>(ctx->d_layers, ctx->d_tiles, err, q, p_hat,
-                                                                      level, nullptr, out, c.worker_stride,
-                                                                      c.n_workers, c.rank_low, c.rank_high, tail);
-    }
+    PhaseTimer pt(ctx, PH_PSGD_RESIDUAL, s);
+    const unsigned n_items = (unsigned)pl.col_items.size();
+    if (lazy && tail.params)
+      psgd_decompress_kernel<true><<<n_items, kColBlockThreads, 0, s>>>(
+          ctx->d_layers, ctx->d_col_items, q, p_hat, level, out, c.rank_low, c.rank_high, tail);
+    else if (lazy)
+      psgd_decompress_kernel<false><<<n_items, kColBlockThreads, 0, s>>>(
+          ctx->d_layers, ctx->d_col_items, q, p_hat, level, out, c.rank_low, c.rank_high, tail);
+    else if (tail.params)
+      psgd_residual_kernel<4, true, true, true><<<nt, 256, 0, s>>>(ctx->d_layers, ctx->d_tiles, err, q, p_hat, level,
+                                                                   nullptr, out, c.worker_stride, c.n_workers,
+                                                                   c.rank_low, c.rank_high, tail);
+    else
+      psgd_residual_kernel<4, true, true, false><<<nt, 256, 0, s>>>(ctx->d_layers, ctx->d_tiles, err, q, p_hat,
+                                                                    level, nullptr, out, c.worker_stride,
+                                                                    c.n_workers, c.rank_low, c.rank_high, tail);
   }
   // VECTOR layers: their out (the plain mean) was written by the first pass
   if (tail.params && !pl.vec_tiles.empty()) {
@@ -829,6 +907,59 @@ cudaError_t launch_powersgd(acc_ctx* ctx, const float* grads, float* err, float*
     if (e != cudaSuccess) return e;
   }
   return cudaGetLastError();
+}
+
+cudaError_t launch_powersgd(acc_ctx* ctx, const float* grads, float* err, float* q, float* p_hat,
+                            const uint8_t* level, float* out, float* delta, SgdTail tail, cudaStream_t s) {
+  launch_psgd_project(ctx, grads, err, q, p_hat, level, out, delta, s);
+  if (ctx->plan.n_mat > 0) launch_psgd_ortho_q(ctx, q, p_hat, level, out, nullptr, 1.f, nullptr, s);
+  return launch_psgd_finish(ctx, err, q, p_hat, level, out, tail, s);
+}
+
+cudaError_t launch_powersgd_phase1(acc_ctx* ctx, const float* grads, float* err, float* q, float* p_hat,
+                                   const uint8_t* level, float* out, float* delta, float* x1, cudaStream_t s) {
+  const Plan& pl = ctx->plan;
+  const acc_config& c = ctx->cfg;
+  launch_psgd_project(ctx, grads, err, q, p_hat, level, out, delta, s);
+  if (pl.n_mat > 0) {
+    PhaseTimer pt(ctx, PH_PSGD_PFOLD, s);
+    psgd_pfold_kernel<<<dim3((pl.max_rows + 255) / 256, pl.n_mat), 256, 0, s>>>(
+        ctx->d_layers, ctx->d_mat_layers, ctx->d_ppart, level, c.rank_low, c.rank_high,
+        reinterpret_cast<float4*>(x1));
+  }
+  if (!pl.vec_tiles.empty()) {
+    PhaseTimer pt(ctx, PH_VEC_EXCHANGE, s);
+    vec_exchange_kernel<true><<<(unsigned)pl.vec_tiles.size(), 256, 0, s>>>(
+        ctx->d_layers, ctx->d_tiles, ctx->d_vec_tiles, out, x1 + 4 * pl.p_rows, 1.f);
+  }
+  return cudaGetLastError();
+}
+
+cudaError_t launch_powersgd_phase2(acc_ctx* ctx, const float* x1, float scale, float* p_hat, const uint8_t* level,
+                                   const float* out, float* x2, cudaStream_t s) {
+  if (ctx->plan.n_mat > 0)
+    launch_psgd_ortho_q(ctx, nullptr, p_hat, level, out, reinterpret_cast<const float4*>(x1), scale,
+                        reinterpret_cast<float4*>(x2), s);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_powersgd_phase3(acc_ctx* ctx, float* err, float* q, const float* p_hat, const uint8_t* level,
+                                   const float* x1, const float* x2, float scale, float* out, SgdTail tail,
+                                   cudaStream_t s) {
+  const Plan& pl = ctx->plan;
+  const acc_config& c = ctx->cfg;
+  if (pl.n_mat > 0) {
+    PhaseTimer pt(ctx, PH_PSGD_QMERGE, s);
+    psgd_qmerge_kernel<<<dim3((pl.max_cols + 255) / 256, pl.n_mat), 256, 0, s>>>(
+        ctx->d_layers, ctx->d_mat_layers, reinterpret_cast<const float4*>(x2), scale, q, level, c.rank_low,
+        c.rank_high);
+  }
+  if (!pl.vec_tiles.empty()) {
+    PhaseTimer pt(ctx, PH_VEC_EXCHANGE, s);
+    vec_exchange_kernel<false><<<(unsigned)pl.vec_tiles.size(), 256, 0, s>>>(
+        ctx->d_layers, ctx->d_tiles, ctx->d_vec_tiles, out, const_cast<float*>(x1) + 4 * pl.p_rows, scale);
+  }
+  return launch_psgd_finish(ctx, err, q, p_hat, level, out, tail, s);
 }
 
 cudaError_t launch_powersgd_flush(acc_ctx* ctx, float* err, const float* q, const float* p_hat, cudaStream_t s) {

@@ -968,12 +968,94 @@ topk_decompress_kernel(const DevLayer* __restrict__ layers, const Tile* __restri
   }
 }
 
-cudaError_t launch_topk(acc_ctx* ctx, const float* grads, float* err, const uint8_t* level, float* vals,
-                        int32_t* idx, int32_t* counts, float* out, float* delta, SgdTail tail, cudaStream_t s) {
+// Real workers.  VECTOR tiles of the compress half: this GPU's mean of the workers' gradients goes to the packed
+// exchange region; delta += g_decider.
+__global__ void __launch_bounds__(256)
+topk_vec_local_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict__ tiles,
+                      const int* __restrict__ vec_tiles, const float* __restrict__ grads,
+                      float* __restrict__ packed, float* __restrict__ delta, long long stride, int W, int decider,
+                      float inv_w) {
+  const Tile t = tiles[vec_tiles[blockIdx.x]];
+  const DevLayer L = layers[t.layer];
+  const long long base = L.offset + t.elem0;
+  for (int i = threadIdx.x; i < t.nelem; i += blockDim.x) {
+    float a = 0.f;
+    for (int w = 0; w < W; ++w) {
+      const float g = grads[(long long)w * stride + base + i];
+      a += g;
+      if (delta != nullptr && w == decider) delta[base + i] += g;
+    }
+    packed[L.vec_off + t.elem0 + i] = a * inv_w;
+  }
+}
+
+// First position in the ascending array a[0..n) whose value is >= key.
+__device__ __forceinline__ int lower_bound_i32(const int32_t* __restrict__ a, int n, int key) {
+  int lo = 0, hi = n;
+  while (lo < hi) {
+    const int mid = (lo + hi) >> 1;
+    if (a[mid] < key) lo = mid + 1; else hi = mid;
+  }
+  return lo;
+}
+
+// Real workers, decompress half.  One block per tile, from the gathered packed sets of all n_sets workers
+// (set j = worker j of the whole job: GPU-major, then the GPU's workers): each set's entries are in ascending
+// index order, so the tile's entries are a contiguous range found by binary search.  Sets are added in order
+// (bit-reproducible, and the same order as the single-GPU step), then scaled by 1/n_sets.
+// VECTOR tiles: out = vec_scale * (summed packed means).
+template <bool SGD>
+__global__ void __launch_bounds__(256)
+topk_decompress_packed_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict__ tiles, int n_layers,
+                              const float* __restrict__ vals, const int32_t* __restrict__ idx,
+                              const int32_t* __restrict__ counts, int n_sets, long long capacity,
+                              const float* __restrict__ packed, float vec_scale, float* __restrict__ out,
+                              const SgdTail tail) {
+  __shared__ float acc[kTile];
+  __shared__ int range[2];
+  const Tile t = tiles[blockIdx.x];
+  const DevLayer L = layers[t.layer];
+  const long long base = L.offset + t.elem0;
+  SgdHyper h = {0.f, 0.f, 0.f};
+  if (SGD) h = sgd_hyper(tail);
+  if (L.kind != ACC_MATRIX) {
+    for (int i = threadIdx.x; i < t.nelem; i += blockDim.x) {
+      const float v = vec_scale * packed[L.vec_off + t.elem0 + i];
+      out[base + i] = v;
+      if (SGD) sgd_apply1(tail, h, base + i, v);
+    }
+    return;
+  }
+  for (int i = threadIdx.x; i < kTile; i += blockDim.x) acc[i] = 0.f;
+  for (int j = 0; j < n_sets; ++j) {
+    const long long seg = (long long)j * capacity + L.seg_off;
+    const int n = counts[(long long)j * n_layers + t.layer];
+    __syncthreads();  // acc of the previous set complete; range free
+    if (threadIdx.x < 2)
+      range[threadIdx.x] = lower_bound_i32(idx + seg, n, threadIdx.x == 0 ? t.elem0 : t.elem0 + t.nelem);
+    __syncthreads();
+    for (int i = range[0] + (int)threadIdx.x; i < range[1]; i += blockDim.x) acc[idx[seg + i] - t.elem0] += vals[seg + i];
+  }
+  __syncthreads();
+  const float inv = 1.0f / (float)n_sets;
+  const int n4 = t.nelem >> 2;
+  for (int i = threadIdx.x; i < n4; i += blockDim.x) {
+    const float4 v = make_float4(acc[4 * i] * inv, acc[4 * i + 1] * inv, acc[4 * i + 2] * inv, acc[4 * i + 3] * inv);
+    st_stream4(out + base + 4 * i, v);
+    if (SGD) sgd_apply4(tail, h, base + 4 * i, v);
+  }
+  for (int i = 4 * n4 + threadIdx.x; i < t.nelem; i += blockDim.x) {
+    out[base + i] = acc[i] * inv;
+    if (SGD) sgd_apply1(tail, h, base + i, acc[i] * inv);
+  }
+}
+
+// Everything of the TopK step up to the packed sets (threshold, selection, error memory).
+static cudaError_t launch_topk_select_part(acc_ctx* ctx, const float* grads, float* err, const uint8_t* level,
+                                           float* vals, int32_t* idx, int32_t* counts, float* delta, cudaStream_t s) {
   const Plan& pl = ctx->plan;
   const acc_config& c = ctx->cfg;
   const int nt = (int)pl.tiles.size(), W = c.n_workers, n_mat = pl.n_mat;
-  const float inv_w = 1.0f / (float)W;
   cudaError_t e = cudaMemsetAsync(ctx->ws + pl.o_hist, 0, pl.hist_bytes, s);
   if (e != cudaSuccess) return e;
   e = cudaMemsetAsync(counts, 0, sizeof(int32_t) * (size_t)W * c.n_layers, s);
@@ -1055,6 +1137,17 @@ cudaError_t launch_topk(acc_ctx* ctx, const float* grads, float* err, const uint
                                                    ctx->d_tile_pre, ctx->d_any_list + 2, vals, idx, c.worker_stride,
                                                    pl.capacity);
   }
+  return cudaGetLastError();
+}
+
+cudaError_t launch_topk(acc_ctx* ctx, const float* grads, float* err, const uint8_t* level, float* vals,
+                        int32_t* idx, int32_t* counts, float* out, float* delta, SgdTail tail, cudaStream_t s) {
+  const Plan& pl = ctx->plan;
+  const acc_config& c = ctx->cfg;
+  const int nt = (int)pl.tiles.size(), W = c.n_workers, n_mat = pl.n_mat;
+  const float inv_w = 1.0f / (float)W;
+  const cudaError_t e = launch_topk_select_part(ctx, grads, err, level, vals, idx, counts, delta, s);
+  if (e != cudaSuccess) return e;
   {
     PhaseTimer pt(ctx, PH_TOPK_DECOMPRESS, s);
     if (tail.params)
@@ -1066,6 +1159,38 @@ cudaError_t launch_topk(acc_ctx* ctx, const float* grads, float* err, const uint
                                                        ctx->d_tile_pre, vals, idx, out, delta, c.worker_stride,
                                                        pl.capacity, W, c.decider, inv_w, tail);
   }
+  return cudaGetLastError();
+}
+
+cudaError_t launch_topk_compress(acc_ctx* ctx, const float* grads, float* err, const uint8_t* level, float* vals,
+                                 int32_t* idx, int32_t* counts, float* delta, float* vec_packed, cudaStream_t s) {
+  const Plan& pl = ctx->plan;
+  const acc_config& c = ctx->cfg;
+  const cudaError_t e = launch_topk_select_part(ctx, grads, err, level, vals, idx, counts, delta, s);
+  if (e != cudaSuccess) return e;
+  if (!pl.vec_tiles.empty()) {
+    PhaseTimer pt(ctx, PH_VEC_EXCHANGE, s);
+    topk_vec_local_kernel<<<(unsigned)pl.vec_tiles.size(), 256, 0, s>>>(
+        ctx->d_layers, ctx->d_tiles, ctx->d_vec_tiles, grads, vec_packed, delta, c.worker_stride, c.n_workers,
+        c.decider, 1.0f / (float)c.n_workers);
+  }
+  return cudaGetLastError();
+}
+
+cudaError_t launch_topk_decompress_packed(acc_ctx* ctx, const float* vals, const int32_t* idx, const int32_t* counts,
+                                          int n_sets, const float* vec_packed, float vec_scale, float* out,
+                                          SgdTail tail, cudaStream_t s) {
+  const Plan& pl = ctx->plan;
+  const unsigned nt = (unsigned)pl.tiles.size();
+  PhaseTimer pt(ctx, PH_TOPK_DECOMPRESS_PACKED, s);
+  if (tail.params)
+    topk_decompress_packed_kernel<true><<<nt, 256, 0, s>>>(ctx->d_layers, ctx->d_tiles, ctx->cfg.n_layers, vals, idx,
+                                                           counts, n_sets, pl.capacity, vec_packed, vec_scale, out,
+                                                           tail);
+  else
+    topk_decompress_packed_kernel<false><<<nt, 256, 0, s>>>(ctx->d_layers, ctx->d_tiles, ctx->cfg.n_layers, vals, idx,
+                                                            counts, n_sets, pl.capacity, vec_packed, vec_scale, out,
+                                                            tail);
   return cudaGetLastError();
 }
 

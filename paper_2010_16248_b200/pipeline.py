@@ -182,6 +182,94 @@ class BatchSizeStep:
         return int(self.batch.item())
 
 
+class DistributedStep:
+    """Real workers: every rank (GPU) holds ``n_local`` workers; the compressed factors are exchanged between the
+    kernels' phases (Section 5.1: all-reduce of P, then of Q, for PowerSGD; all-gather of the packed values and
+    indices for TopK; the VECTOR layers ride in the first all-reduce).  Every rank ends a step with the same
+    ``out``, ``q``, ``p_hat`` and ``level``: the decider's gradient is accumulated on the rank that holds it
+    (global worker ``decider``), and the detector's per-layer norms are broadcast from there by a sum in which
+    the other ranks contribute zeros."""
+
+    def __init__(self, table: wl.LayerTable, n_local: int, compressor: str = "powersgd", rank_low=2, rank_high=1,
+                 topk_low_bp=1000, topk_high_bp=100, eta=0.5, gs_eps=1e-8, check_every=10, decider=0, q_init=None,
+                 device="cuda", lazy_residual=False, optimizer=None, exchange=None):
+        from . import dist_util
+        self.table, self.n_local, self.compressor = table, n_local, compressor
+        self.x = exchange if exchange is not None else dist_util.Exchange()
+        self.world, self.rank = self.x.world, self.x.rank
+        self.check_every = check_every
+        self.device = dev = torch.device(device)
+        self.owns_decider = decider // n_local == self.rank
+        self.ctx = binding.Context(table, n_local, device=device, rank_low=rank_low, rank_high=rank_high,
+                                   topk_low_bp=topk_low_bp, topk_high_bp=topk_high_bp, eta=eta, gs_eps=gs_eps,
+                                   decider=decider % n_local,
+                                   flags=binding.ACC_FLAG_LAZY_RESIDUAL if lazy_residual else 0)
+        L, stride, c = table.n_layers, table.stride, self.ctx
+        self.level = torch.ones(L, dtype=torch.uint8, device=dev)
+        self.delta = torch.zeros(stride, device=dev) if self.owns_decider else None
+        self.norm2_curr = torch.zeros(L, dtype=torch.float64, device=dev)
+        self.norm2_prev = torch.full((L,), -1.0, dtype=torch.float64, device=dev)
+        self.err = torch.zeros(n_local, stride, device=dev)
+        self.out = torch.zeros(stride, device=dev)
+        self.t = 0
+        self.params = self.mom = self.hyper = None
+        if optimizer is not None:
+            self.params = optimizer["params"]
+            self.mom = torch.zeros(stride, device=dev)
+            self.hyper = torch.tensor([optimizer["lr"], optimizer.get("momentum", 0.9),
+                                       optimizer.get("weight_decay", 0.0)], dtype=torch.float32, device=dev)
+        if compressor == "powersgd":
+            self.q = c.new_q(q_init if q_init is not None else wl.initial_q(table, rank_low, device=dev))
+            self.p_hat = c.new_p()
+            self.x1 = torch.zeros(max(c.x1_floats, 4), device=dev)
+            self.x2 = torch.zeros(max(c.x2_floats, 4), device=dev)
+        elif compressor == "topk":
+            self.vals, self.idx, self.counts = c.new_topk_buffers()
+            self.vec = torch.zeros(max(c.vec_floats, 4), device=dev)
+            w = self.world
+            self.vals_all = torch.zeros(w * self.vals.numel(), device=dev)
+            self.idx_all = torch.zeros(w * self.idx.numel(), dtype=torch.int32, device=dev)
+            self.counts_all = torch.zeros(w * self.counts.numel(), dtype=torch.int32, device=dev)
+        else:
+            raise ValueError(compressor)
+
+    def bytes_exchanged_per_step(self) -> int:
+        """Bytes this rank hands to the collectives in one step (the method's communication volume)."""
+        if self.compressor == "powersgd":
+            return 4 * (self.x1.numel() + self.x2.numel())
+        return 4 * (self.vals.numel() + self.idx.numel() + self.counts.numel() + self.vec.numel())
+
+    def step(self, grads: torch.Tensor, lr_curr: float = 0.1, lr_next: float = 0.1, stream=None):
+        """One iteration on this rank's device-resident gradients ``[n_local, stride]``."""
+        c, x, scale = self.ctx, self.x, 1.0 / self.world
+        if self.compressor == "powersgd":
+            c.acc_powersgd_phase1(grads, self.err, self.q, self.p_hat, self.level, self.out, self.delta, self.x1,
+                                  stream)
+            x.sum_(self.x1)
+            c.acc_powersgd_phase2(self.x1, scale, self.p_hat, self.level, self.out, self.x2, stream)
+            x.sum_(self.x2)
+            c.acc_powersgd_phase3(self.err, self.q, self.p_hat, self.level, self.x1, self.x2, scale, self.out,
+                                  self.params, self.mom, self.hyper, stream)
+        else:
+            c.acc_topk_compress(grads, self.err, self.level, self.vals, self.idx, self.counts, self.delta, self.vec,
+                                stream)
+            x.gather_into(self.vals_all, self.vals)
+            x.gather_into(self.idx_all, self.idx)
+            x.gather_into(self.counts_all, self.counts)
+            x.sum_(self.vec)
+            c.acc_topk_decompress(self.vals_all, self.idx_all, self.counts_all, self.world * self.n_local, self.vec,
+                                  scale, self.out, self.params, self.mom, self.hyper, stream)
+        self.t += 1
+        if self.t % self.check_every == 0:
+            if self.owns_decider:
+                c.acc_layer_norms(self.delta, 1, self.norm2_curr, stream=stream)
+            else:
+                self.norm2_curr.zero_()
+            x.sum_(self.norm2_curr)  # a broadcast from the deciding rank (Section 3: one node decides for all)
+            c.acc_detect_regime(self.norm2_curr, self.norm2_prev, lr_curr, lr_next, self.level, self.delta, stream)
+        return self.out
+
+
 class HostFedStep:
     """Runs ``AccordionStep`` on gradients that live in pinned host memory.
 

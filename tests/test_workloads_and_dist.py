@@ -96,3 +96,61 @@ def test_two_rank_replicas_gloo():
     # whole-job throughput: both ranks' units over the slowest rank's time
     assert dist_util.whole_job_throughput(100.0, 15.0, world) == pytest.approx(2 * 100.0 / 0.015)
     assert dist_util.max_over_ranks(3.0) == 3.0                 # no process group: identity
+
+
+def _real_worker_rank_main(rank, world, port, out):
+    """Two ranks with two workers each: the exchange helper over gloo, and the algebra of the real-worker split
+    of the PowerSGD step (local P rows summed over ranks, Gram-Schmidt, local Q' rows summed) against the
+    oracle's step over all four workers."""
+    from oracle import accordion_oracle as orc
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        x = dist_util.Exchange()
+        t = torch.tensor([rank + 1.0, 2.0])
+        x.sum_(t)
+        gathered = torch.zeros(world * 3, dtype=torch.int32)
+        x.gather_into(gathered, torch.tensor([rank, 10 * rank, 7], dtype=torch.int32))
+        # the split step in numpy, exchanged through the real collectives
+        n, m, r, n_local = 12, 9, 2, 2
+        rng = np.random.default_rng(5)
+        g = rng.standard_normal((world * n_local, n * m)).astype(np.float32)
+        e = (0.3 * rng.standard_normal((world * n_local, n * m))).astype(np.float32)
+        q0 = rng.standard_normal((m, r)).astype(np.float32)
+        mine = slice(rank * n_local, (rank + 1) * n_local)
+        mbar = (g[mine].astype(np.float64) + e[mine].astype(np.float64)).mean(axis=0).reshape(n, m)
+        x1 = torch.from_numpy(mbar @ q0.astype(np.float64))
+        x.sum_(x1)
+        p_hat = orc.gram_schmidt(x1.numpy() / world, 1e-8)
+        x2 = torch.from_numpy(mbar.T @ p_hat)
+        x.sum_(x2)
+        q_new = x2.numpy() / world
+        layers = [(0, n, m, orc.MATRIX)]
+        o_out, _, o_q, o_p = orc.powersgd_step(g, e, [q0], np.ones(1, np.uint8), layers, r, r)
+        ok = (np.allclose(p_hat, o_p[0], rtol=1e-10, atol=1e-12) and np.allclose(q_new, o_q[0], rtol=1e-10, atol=1e-12)
+              and np.allclose((p_hat @ q_new.T).ravel(), o_out, rtol=1e-10, atol=1e-12))
+        out[rank] = (t.tolist(), gathered.tolist(), x.world, x.rank, bool(ok))
+    finally:
+        dist.destroy_process_group()
+
+
+def test_real_worker_exchange_and_split_algebra_gloo():
+    world = 2
+    ctx = mp.get_context("spawn")
+    out = ctx.Manager().dict()
+    port = 31500 + os.getpid() % 2000
+    procs = [ctx.Process(target=_real_worker_rank_main, args=(r, world, port, out)) for r in range(world)]
+    for p in procs:
+        p.start()
+    for p in procs:
+        p.join(180)
+        assert p.exitcode == 0
+    for r in range(world):
+        t, gathered, w, rk, ok = out[r]
+        assert t == [3.0, 4.0] and gathered == [0, 0, 7, 1, 10, 7] and (w, rk) == (world, r)
+        assert ok, "sum of local factor rows over ranks does not reproduce the all-worker step"
+    x = dist_util.Exchange()  # no process group: one-rank identity
+    a = torch.tensor([1.0, 2.0])
+    assert x.world == 1 and torch.equal(x.sum_(a.clone()), a)
+    assert torch.equal(x.gather_into(torch.zeros(2), a), a)
