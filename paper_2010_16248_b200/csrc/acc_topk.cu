@@ -1012,7 +1012,7 @@ topk_decompress_packed_kernel(const DevLayer* __restrict__ layers, const Tile* _
                               const float* __restrict__ packed, float vec_scale, float* __restrict__ out,
                               const SgdTail tail) {
   __shared__ float acc[kTile];
-  __shared__ int range[2];
+  __shared__ int range[256];
   const Tile t = tiles[blockIdx.x];
   const DevLayer L = layers[t.layer];
   const long long base = L.offset + t.elem0;
@@ -1027,14 +1027,23 @@ topk_decompress_packed_kernel(const DevLayer* __restrict__ layers, const Tile* _
     return;
   }
   for (int i = threadIdx.x; i < kTile; i += blockDim.x) acc[i] = 0.f;
-  for (int j = 0; j < n_sets; ++j) {
-    const long long seg = (long long)j * capacity + L.seg_off;
-    const int n = counts[(long long)j * n_layers + t.layer];
-    __syncthreads();  // acc of the previous set complete; range free
-    if (threadIdx.x < 2)
-      range[threadIdx.x] = lower_bound_i32(idx + seg, n, threadIdx.x == 0 ? t.elem0 : t.elem0 + t.nelem);
+  // the tile's range in every set: 128 sets at a time, one thread per bound, all searches in flight together
+  for (int j0 = 0; j0 < n_sets; j0 += 128) {
+    const int nj = min(128, n_sets - j0);
+    __syncthreads();  // acc cleared / previous chunk consumed
+    if ((int)threadIdx.x < 2 * nj) {
+      const int j = j0 + ((int)threadIdx.x >> 1);
+      const long long seg = (long long)j * capacity + L.seg_off;
+      const int n = counts[(long long)j * n_layers + t.layer];
+      range[threadIdx.x] = lower_bound_i32(idx + seg, n, (threadIdx.x & 1) ? t.elem0 + t.nelem : t.elem0);
+    }
     __syncthreads();
-    for (int i = range[0] + (int)threadIdx.x; i < range[1]; i += blockDim.x) acc[idx[seg + i] - t.elem0] += vals[seg + i];
+    for (int jj = 0; jj < nj; ++jj) {  // sets in order: the sum of an element's contributions has a fixed order
+      const long long seg = (long long)(j0 + jj) * capacity + L.seg_off;
+      const int lo = range[2 * jj], hi = range[2 * jj + 1];
+      for (int i = lo + (int)threadIdx.x; i < hi; i += blockDim.x) acc[idx[seg + i] - t.elem0] += vals[seg + i];
+      if (lo < hi) __syncthreads();  // lo, hi are uniform over the block
+    }
   }
   __syncthreads();
   const float inv = 1.0f / (float)n_sets;
