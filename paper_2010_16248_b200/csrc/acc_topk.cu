@@ -100,38 +100,50 @@ topk_ef_hist1_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict
     unsigned* buf = s_buf[cb];
     unsigned* cnt = &s_cnt[cb];
     int above = 0;
-#pragma unroll 4
-    for (int i = threadIdx.x; i < n4; i += blockDim.x) {
-      const float4 gv = ld_stream4(g + 4 * i);
-      const float4 ev = ld_stream4(e + 4 * i);
-      const float4 m = make_float4(gv.x + ev.x, gv.y + ev.y, gv.z + ev.z, gv.w + ev.w);
-      *reinterpret_cast<float4*>(e + 4 * i) = m;
-      const unsigned k[4] = {key_of(m.x), key_of(m.y), key_of(m.z), key_of(m.w)};
-      const float mm[4] = {m.x, m.y, m.z, m.w};
+    // batches of kBatch float4 per thread: all loads of a batch are issued before the first store, so that
+    // they are in flight together (a store to err in between would pin the later loads of err behind it)
+    constexpr int kBatch = 4, kThreads = 256;
+    for (int i0 = 0; i0 < n4; i0 += kBatch * kThreads) {
+      float4 gb[kBatch], eb[kBatch];
 #pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        const unsigned bin = k[q] >> 19;
-        atomicAdd(&h[bin], 1u);
-        if (staged) {
-          if (bin >= blo) {
-            const unsigned slot = atomicAdd(cnt, 1u);
-            if (slot < (unsigned)kPredTileCap / 2) {
-              buf[2 * slot] = __float_as_uint(mm[q]);
-              buf[2 * slot + 1] = (unsigned)(t.elem0 + 4 * i + q);
+      for (int u = 0; u < kBatch; ++u) {
+        const int i = i0 + u * kThreads + (int)threadIdx.x;
+        if (i < n4) { gb[u] = ld_stream4(g + 4 * i); eb[u] = ld_stream4(e + 4 * i); }
+      }
+#pragma unroll
+      for (int u = 0; u < kBatch; ++u) {
+        const int i = i0 + u * kThreads + (int)threadIdx.x;
+        if (i >= n4) break;
+        const float4 gv = gb[u], ev = eb[u];
+        const float4 m = make_float4(gv.x + ev.x, gv.y + ev.y, gv.z + ev.z, gv.w + ev.w);
+        *reinterpret_cast<float4*>(e + 4 * i) = m;
+        const unsigned k[4] = {key_of(m.x), key_of(m.y), key_of(m.z), key_of(m.w)};
+        const float mm[4] = {m.x, m.y, m.z, m.w};
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const unsigned bin = k[q] >> 19;
+          atomicAdd(&h[bin], 1u);
+          if (staged) {
+            if (bin >= blo) {
+              const unsigned slot = atomicAdd(cnt, 1u);
+              if (slot < (unsigned)kPredTileCap / 2) {
+                buf[2 * slot] = __float_as_uint(mm[q]);
+                buf[2 * slot + 1] = (unsigned)(t.elem0 + 4 * i + q);
+              }
+            }
+          } else if (collect) {
+            above += bin > bhi;
+            if (bin - blo <= span) {
+              const unsigned slot = atomicAdd(cnt, 1u);
+              if (slot < (unsigned)kPredTileCap) buf[slot] = k[q];
             }
           }
-        } else if (collect) {
-          above += bin > bhi;
-          if (bin - blo <= span) {
-            const unsigned slot = atomicAdd(cnt, 1u);
-            if (slot < (unsigned)kPredTileCap) buf[slot] = k[q];
-          }
         }
-      }
-      if (acc_delta) {
-        float4 d = *reinterpret_cast<const float4*>(delta + base + 4 * i);
-        d.x += gv.x; d.y += gv.y; d.z += gv.z; d.w += gv.w;
-        *reinterpret_cast<float4*>(delta + base + 4 * i) = d;
+        if (acc_delta) {
+          float4 d = *reinterpret_cast<const float4*>(delta + base + 4 * i);
+          d.x += gv.x; d.y += gv.y; d.z += gv.z; d.w += gv.w;
+          *reinterpret_cast<float4*>(delta + base + 4 * i) = d;
+        }
       }
     }
     for (int i = 4 * n4 + threadIdx.x; i < t.nelem; i += blockDim.x) {
