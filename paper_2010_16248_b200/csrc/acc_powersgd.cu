@@ -203,15 +203,24 @@ psgd_project_pipe_kernel(const DevLayer* __restrict__ layers, const Tile* __rest
     fence_mbar_init();
   }
   __syncthreads();
-  auto issue = [&](int it) {  // called by thread 0 only
+  // thread 0 only: the tile whose stages are being issued is kept in registers, so that issuing a stage costs
+  // no dependent global loads (they would sit on the critical path of every stage)
+  int is_ti = -1;
+  long long is_base = 0;
+  unsigned is_bytes = 0;
+  auto issue = [&](int it) {
     const int ti = it / W, w = it - ti * W;
-    const Tile t = tiles[mat_tiles[t0 + ti]];
-    const long long base = (long long)w * stride + layers[t.layer].offset + t.elem0;
-    const unsigned bytes = (unsigned)((t.nelem + 3) / 4) * 16u;  // a ragged tile reads into the layer's padding
+    if (ti != is_ti) {
+      const Tile tt = tiles[mat_tiles[t0 + ti]];
+      is_ti = ti;
+      is_base = layers[tt.layer].offset + tt.elem0;
+      is_bytes = (unsigned)((tt.nelem + 3) / 4) * 16u;  // a ragged tile reads into the layer's padding
+    }
+    const long long base = (long long)w * stride + is_base;
     const int buf = it % kPipeStages;
-    mbar_arrive_expect_tx(&bars[buf], 2 * bytes);
-    bulk_copy_g2s(stage + (2 * buf) * kTile, grads + base, bytes, &bars[buf]);
-    bulk_copy_g2s(stage + (2 * buf + 1) * kTile, err + base, bytes, &bars[buf]);
+    mbar_arrive_expect_tx(&bars[buf], 2 * is_bytes);
+    bulk_copy_g2s(stage + (2 * buf) * kTile, grads + base, is_bytes, &bars[buf]);
+    bulk_copy_g2s(stage + (2 * buf + 1) * kTile, err + base, is_bytes, &bars[buf]);
   };
   if (threadIdx.x == 0)
     for (int it = 0; it < kPipeStages && it < n_stages; ++it) issue(it);

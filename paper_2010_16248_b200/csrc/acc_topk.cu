@@ -828,7 +828,8 @@ __global__ void __launch_bounds__(256, 3)
 topk_select_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict__ tiles, int n_tiles, int n_mat,
                    float* __restrict__ err, const Select* __restrict__ sel, const int2* __restrict__ tile_pre,
                    const unsigned* __restrict__ any_select, float* __restrict__ vals, int32_t* __restrict__ idx,
-                   long long stride, long long capacity) {
+                   long long stride, long long capacity, const int2* __restrict__ tile_cnt,
+                   const int2* __restrict__ tile_cand) {
   __shared__ unsigned wtot[8];
   if (*any_select == 0) return;  // every segment was served from staged entries
   const int ti = blockIdx.x, w = blockIdx.y;
@@ -837,7 +838,12 @@ topk_select_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict__
   if (L.kind != ACC_MATRIX) return;
   const Select s = sel[w * n_mat + L.mat];
   if (s.mode == kSelStaged) return;
-  const int2 pre = tile_pre[(long long)w * n_tiles + ti];
+  const long long v = (long long)w * n_tiles + ti;
+  // list segments: the earlier pass counted the tile's keys above the collected bucket(s) and collected those
+  // inside; the threshold lies inside, so a tile with neither holds nothing to keep and is not read at all
+  // (most tiles of a row-sparse layer)
+  if (s.mode != kSelDense && tile_cnt[v].x == 0 && tile_cand[v].y == 0) return;
+  const int2 pre = tile_pre[v];
   float* m = err + (long long)w * stride + L.offset + t.elem0;
   const long long seg = (long long)w * capacity + L.seg_off;
   if (t.nelem == kTile) select_tile<true>(t, L, s, pre, m, vals, idx, seg, wtot);
@@ -1156,7 +1162,7 @@ static cudaError_t launch_topk_select_part(acc_ctx* ctx, const float* grads, flo
     PhaseTimer pt(ctx, PH_TOPK_SELECT, s);
     topk_select_kernel<<<dim3(nt, W), 256, 0, s>>>(ctx->d_layers, ctx->d_tiles, nt, n_mat, err, ctx->d_sel,
                                                    ctx->d_tile_pre, ctx->d_any_list + 2, vals, idx, c.worker_stride,
-                                                   pl.capacity);
+                                                   pl.capacity, ctx->d_tile_cnt, ctx->d_tile_cand);
   }
   return cudaGetLastError();
 }
