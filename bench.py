@@ -195,6 +195,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--eager", action="store_true", help="PowerSGD: materialise the error memory every step")
     ap.add_argument("--no-graphs", action="store_true", help="issue the timed steps call by call instead of as CUDA graphs")
+    ap.add_argument("--pipeline", default="auto", choices=["auto", "always", "never"],
+                    help="first PowerSGD pass: persistent bulk-copy pipeline, direct kernel, or the library's choice")
     ap.add_argument("--sgd-tail", action="store_true",
                     help="single-compressor configs: apply the Nesterov update inside the step (fused optimiser tail)")
     ap.add_argument("--batch-mode", action="store_true",
@@ -245,7 +247,7 @@ def main():
         optimizer = {"params": torch.zeros(table.stride, device=dev), "lr": 0.1, "momentum": 0.9}
     eng = pipeline.AccordionStep(table, W, w.compressors, w.rank_low, w.rank_high, w.topk_low_bp, w.topk_high_bp,
                                  w.eta, 1e-8, w.check_every, device=dev, lazy_residual=not args.eager,
-                                 optimizer=optimizer)
+                                 optimizer=optimizer, extra_flags={"auto": 0, "always": 2, "never": 4}[args.pipeline])
     n_mat = table.n_matrix_params
     grad_bytes_step = n_comp * 4.0 * W * table.n_params
 

@@ -19,8 +19,10 @@ from . import workloads as wl
 class AccordionStep:
     def __init__(self, table: wl.LayerTable, n_workers: int, compressors: Sequence[str] = ("powersgd",),
                  rank_low=2, rank_high=1, topk_low_bp=1000, topk_high_bp=100, eta=0.5, gs_eps=1e-8,
-                 check_every=10, decider=0, q_init=None, device="cuda", lazy_residual=False, optimizer=None):
-        """``optimizer``: None, or a dict ``{"params": tensor [stride], "lr": .., "momentum": 0.9,
+                 check_every=10, decider=0, q_init=None, device="cuda", lazy_residual=False, optimizer=None,
+                 extra_flags=0):
+        """``extra_flags``: further ACC_FLAG_* bits for the context (e.g. forcing one implementation of the first
+        PowerSGD pass).  ``optimizer``: None, or a dict ``{"params": tensor [stride], "lr": .., "momentum": 0.9,
         "weight_decay": 0.0}``: the Nesterov update (Appendix A) is then applied to ``params`` by the kernels
         that produce the averaged gradient (one compressor only)."""
         self.table, self.W = table, n_workers
@@ -32,7 +34,7 @@ class AccordionStep:
         self.ctx = binding.Context(table, n_workers, device=device, rank_low=rank_low, rank_high=rank_high,
                                    topk_low_bp=topk_low_bp, topk_high_bp=topk_high_bp, eta=eta, gs_eps=gs_eps,
                                    decider=decider,
-                                   flags=binding.ACC_FLAG_LAZY_RESIDUAL if lazy_residual else 0)
+                                   flags=(binding.ACC_FLAG_LAZY_RESIDUAL if lazy_residual else 0) | extra_flags)
         dev, L, stride = self.device, table.n_layers, table.stride
         self.level = torch.ones(L, dtype=torch.uint8, device=dev)  # before the first check: low compression
         self.delta = torch.zeros(stride, device=dev)
