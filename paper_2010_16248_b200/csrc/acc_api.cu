@@ -129,6 +129,7 @@ static int make_plan(const acc_config* cfg, Plan& p) {
   p.o_tile_cnt = take(sizeof(int2) * (size_t)W * nt);
   p.o_tile_h3 = take(sizeof(unsigned short) * (size_t)W * nt * kBins3);
   p.o_tile_pre = take(sizeof(int2) * (size_t)W * nt);
+  p.o_lists = take(sizeof(int2) * (size_t)kNumLists * W * nt);
   p.total = o;
   return ACC_OK;
 }
@@ -190,6 +191,7 @@ int acc_create(const acc_config* cfg, void* workspace, size_t workspace_bytes, a
   ctx->d_tile_cnt = reinterpret_cast<int2*>(ws + p.o_tile_cnt);
   ctx->d_tile_h3 = reinterpret_cast<unsigned short*>(ws + p.o_tile_h3);
   ctx->d_tile_pre = reinterpret_cast<int2*>(ws + p.o_tile_pre);
+  ctx->d_lists = reinterpret_cast<int2*>(ws + p.o_lists);
 
   cudaError_t e = cudaSuccess;
   auto up = [&](void* dst, const void* src, size_t bytes) {

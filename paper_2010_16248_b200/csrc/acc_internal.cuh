@@ -48,6 +48,11 @@ struct Select {
 };
 constexpr int kSelDense = 0, kSelList = 1, kSelListPred = 2, kSelStaged = 3;
 // ListPred: the key list was filled by pass A;  Staged: pass A staged whole (value, index) entries
+// Work lists of (worker, tile) pairs, rebuilt every step on the device, so that the passes that serve only some
+// segments launch as many blocks as there is work: tiles of segments whose bucket is collected by the collect
+// pass, tiles of dense segments, tiles the select pass must read, tiles served from staged entries.
+constexpr int kListCollect = 0, kListDense = 1, kListSelect = 2, kListStaged = 3, kNumLists = 4;
+constexpr int kListCountWord = 8;  // the lists' lengths live at words 8..11 of the per-step flag block
 constexpr int kPredTileCap = 2048;  // keys one tile may hand to a predicted list (more: overflow, fall back)
 
 // Kernels of the library, for per-kernel timing (acc_profile_*).
@@ -76,7 +81,7 @@ struct Plan {
   long long vec_floats = 0;  // packed VECTOR elements (each layer starts at a multiple of 4)
   // workspace offsets (bytes)
   size_t o_layers = 0, o_col_items = 0, o_tiles = 0, o_mat_layers = 0, o_vec_tiles = 0, o_mat_tiles = 0, o_status = 0,
-         o_part = 0, o_ppart = 0, o_pending = 0, o_norm_part = 0, o_hist = 0, o_sel = 0, o_pred = 0, o_cand = 0, o_tile_cand = 0, o_tile_cnt = 0, o_tile_h3 = 0, o_tile_pre = 0,
+         o_part = 0, o_ppart = 0, o_pending = 0, o_norm_part = 0, o_hist = 0, o_sel = 0, o_pred = 0, o_cand = 0, o_tile_cand = 0, o_tile_cnt = 0, o_tile_h3 = 0, o_tile_pre = 0, o_lists = 0,
          hist_bytes = 0, total = 0;
 };
 
@@ -117,6 +122,7 @@ struct acc_ctx {
   int2* d_tile_cnt = nullptr;
   unsigned short* d_tile_h3 = nullptr;
   int2* d_tile_pre = nullptr;
+  int2* d_lists = nullptr;           // [kNumLists][W * tiles] work lists of (worker, tile)
 };
 
 namespace acc {

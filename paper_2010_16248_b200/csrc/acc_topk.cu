@@ -21,6 +21,8 @@
 //   finalize   the same for segments whose pass A staged whole entries: from the list, M is not read
 //   decompress out = (1/W) sum_w scatter(idx_w, val_w), accumulated per tile in shared memory [reads packed]
 // No floating-point atomics and no inter-block waiting: same input, same bits.
+#include <algorithm>
+
 #include "acc_internal.cuh"
 
 namespace acc {
@@ -269,10 +271,12 @@ topk_pick1_kernel(const DevLayer* __restrict__ layers, const int* __restrict__ m
                   int W, const uint8_t* __restrict__ level, const unsigned* __restrict__ hist1,
                   Select* __restrict__ sel, int32_t* __restrict__ counts, unsigned* __restrict__ pred,
                   unsigned* __restrict__ seg_cand, const unsigned* __restrict__ seg_flag,
-                  unsigned* __restrict__ any_list) {
+                  unsigned* __restrict__ any_list, int2* __restrict__ lists, int n_tiles) {
   __shared__ unsigned sums[256];
   __shared__ unsigned bin;
   __shared__ long long above;
+  __shared__ int s_list;
+  __shared__ unsigned s_base;
   const int seg = blockIdx.x, w = seg / n_mat, l = mat_layers[seg % n_mat];
   const DevLayer L = layers[l];
   const int lv = level[l] ? 1 : 0;
@@ -327,6 +331,14 @@ topk_pick1_kernel(const DevLayer* __restrict__ layers, const int* __restrict__ m
                                  ((no_stage ? 1u : 0u) << 25));
     sel[seg] = s;
     counts[w * n_layers + l] = k;
+    // the segment's tiles join the work list of the pass that will read M for levels 2-3, as one run
+    s_list = s.mode == kSelList ? kListCollect : s.mode == kSelDense ? kListDense : -1;
+    if (s_list >= 0) s_base = atomicAdd(&any_list[kListCountWord + s_list], (unsigned)L.ntiles);
+  }
+  __syncthreads();
+  if (s_list >= 0) {
+    int2* dst = lists + (long long)s_list * W * n_tiles + s_base;
+    for (int i = threadIdx.x; i < L.ntiles; i += blockDim.x) dst[i] = make_int2(w, L.tile0 + i);
   }
 }
 
@@ -420,19 +432,19 @@ topk_collect_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict_
                     int W, const float* __restrict__ err, long long stride, const Select* __restrict__ sel,
                     const unsigned* __restrict__ any_list, unsigned* __restrict__ seg_cand,
                     unsigned* __restrict__ cand, int2* __restrict__ tile_cand, long long cand_total,
-                    int2* __restrict__ tile_cnt) {
+                    int2* __restrict__ tile_cnt, const int2* __restrict__ lists) {
   __shared__ unsigned wsum[8];
   __shared__ unsigned s_start;
-  if (*any_list == 0) return;
-  const long long V = (long long)W * n_tiles;
-  for (long long v = blockIdx.x; v < V; v += gridDim.x) {
-    const int w = (int)(v / n_tiles), ti = (int)(v % n_tiles);
+  const unsigned n_work = any_list[kListCountWord + kListCollect];
+  const int2* work = lists + (long long)kListCollect * W * n_tiles;
+  for (unsigned b = blockIdx.x; b < n_work; b += gridDim.x) {
+    __syncthreads();  // the shared words of the previous tile are no longer read
+    const int w = work[b].x, ti = work[b].y;
+    const long long v = (long long)w * n_tiles + ti;
     const Tile t = tiles[ti];
     const DevLayer L = layers[t.layer];
-    if (L.kind != ACC_MATRIX) continue;
     const int seg = w * n_mat + L.mat;
     const Select s = sel[seg];
-    if (s.mode != kSelList) continue;
     const float* m = err + (long long)w * stride + L.offset + t.elem0;
     unsigned* list = cand + (long long)w * cand_total + L.cand_base;
     if (t.nelem == kTile) collect_tile<true>(t, s, m, seg_cand + seg, list, tile_cand + v, tile_cnt + v, wsum, &s_start);
@@ -444,23 +456,24 @@ topk_collect_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict_
 __global__ void __launch_bounds__(256)
 topk_hist2_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict__ tiles, int n_tiles, int n_mat,
                   const float* __restrict__ err, long long stride, int W, const Select* __restrict__ sel,
-                  const unsigned* __restrict__ any_dense, unsigned* __restrict__ hist2,
-                  int2* __restrict__ tile_cnt) {
+                  const unsigned* __restrict__ any_list, unsigned* __restrict__ hist2,
+                  int2* __restrict__ tile_cnt, const int2* __restrict__ lists) {
   __shared__ unsigned h[kBins2];
   __shared__ int cnt;
-  if (*any_dense == 0) return;
+  // the dense segments' tiles, each segment one contiguous run of the list; a block takes a contiguous share
+  const long long V = any_list[kListCountWord + kListDense];
+  const long long v0 = V * blockIdx.x / gridDim.x, v1 = V * (blockIdx.x + 1) / gridDim.x;
+  if (v0 >= v1) return;
+  const int2* work = lists + (long long)kListDense * W * n_tiles;
   for (int b = threadIdx.x; b < kBins2; b += blockDim.x) h[b] = 0;
   if (threadIdx.x == 0) cnt = 0;
   __syncthreads();
-  const long long V = (long long)W * n_tiles;
-  const long long v0 = V * blockIdx.x / gridDim.x, v1 = V * (blockIdx.x + 1) / gridDim.x;
-  int cur = -1, mode = kSelDense;
+  int cur = -1;
   unsigned b1 = 0;
   for (long long v = v0; v < v1; ++v) {
-    const int w = (int)(v / n_tiles), ti = (int)(v % n_tiles);
+    const int w = work[v].x, ti = work[v].y;
     const Tile t = tiles[ti];
     const DevLayer L = layers[t.layer];
-    if (L.kind != ACC_MATRIX) continue;
     const int seg = w * n_mat + L.mat;
     if (seg != cur) {
       __syncthreads();
@@ -472,9 +485,7 @@ topk_hist2_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict__ 
       __syncthreads();
       cur = seg;
       b1 = sel[seg].b1;
-      mode = sel[seg].mode;
     }
-    if (mode != kSelDense) continue;  // list segments are served by topk_hist_list_kernel
     const float* m = err + (long long)w * stride + L.offset + t.elem0;
     int above = 0;
     const int n4 = t.nelem >> 2;
@@ -512,51 +523,54 @@ topk_hist2_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict__ 
 __global__ void __launch_bounds__(256)
 topk_hist3_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict__ tiles, int n_tiles, int n_mat,
                   const float* __restrict__ err, long long stride, const Select* __restrict__ sel,
-                  const unsigned* __restrict__ any_dense, unsigned* __restrict__ hist3,
-                  int2* __restrict__ tile_cnt, unsigned short* __restrict__ tile_h3) {
+                  const unsigned* __restrict__ any_list, unsigned* __restrict__ hist3,
+                  int2* __restrict__ tile_cnt, unsigned short* __restrict__ tile_h3, const int2* __restrict__ lists,
+                  int W) {
   __shared__ unsigned h[kBins3];
   __shared__ int cnt;
-  if (*any_dense == 0) return;
-  const int ti = blockIdx.x, w = blockIdx.y;
-  const Tile t = tiles[ti];
-  const DevLayer L = layers[t.layer];
-  if (L.kind != ACC_MATRIX) return;
-  const int seg = w * n_mat + L.mat;
-  const Select s = sel[seg];
-  if (s.mode != kSelDense) return;  // list segments: topk_hist_list_kernel and topk_tile_counts_kernel
-  if (threadIdx.x < kBins3) h[threadIdx.x] = 0;
-  if (threadIdx.x == 0) cnt = 0;
-  __syncthreads();
-  const unsigned prefix = (s.b1 << 12) | s.b2;
-  const float* m = err + (long long)w * stride + L.offset + t.elem0;
-  int above = 0;
-  {
-    const int n4 = t.nelem >> 2;
+  const unsigned n_work = any_list[kListCountWord + kListDense];
+  const int2* work = lists + (long long)kListDense * W * n_tiles;
+  for (unsigned b = blockIdx.x; b < n_work; b += gridDim.x) {
+    const int w = work[b].x, ti = work[b].y;
+    const Tile t = tiles[ti];
+    const DevLayer L = layers[t.layer];
+    const int seg = w * n_mat + L.mat;
+    const Select s = sel[seg];
+    __syncthreads();  // the previous tile's counters have been read
+    if (threadIdx.x < kBins3) h[threadIdx.x] = 0;
+    if (threadIdx.x == 0) cnt = 0;
+    __syncthreads();
+    const unsigned prefix = (s.b1 << 12) | s.b2;
+    const float* m = err + (long long)w * stride + L.offset + t.elem0;
+    int above = 0;
+    {
+      const int n4 = t.nelem >> 2;
 #pragma unroll 4
-    for (int i = threadIdx.x; i < n4; i += blockDim.x) {
-      const float4 mv = ld_stream4(m + 4 * i);
-      const unsigned k[4] = {key_of(mv.x), key_of(mv.y), key_of(mv.z), key_of(mv.w)};
+      for (int i = threadIdx.x; i < n4; i += blockDim.x) {
+        const float4 mv = ld_stream4(m + 4 * i);
+        const unsigned k[4] = {key_of(mv.x), key_of(mv.y), key_of(mv.z), key_of(mv.w)};
 #pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const unsigned p = k[e] >> 7;
+        for (int e = 0; e < 4; ++e) {
+          const unsigned p = k[e] >> 7;
+          above += ((p >> 12) == s.b1) && (p > prefix);
+          if (p == prefix) atomicAdd(&h[k[e] & 127u], 1u);
+        }
+      }
+      for (int i = 4 * n4 + threadIdx.x; i < t.nelem; i += blockDim.x) {
+        const unsigned k0 = key_of(m[i]), p = k0 >> 7;
         above += ((p >> 12) == s.b1) && (p > prefix);
-        if (p == prefix) atomicAdd(&h[k[e] & 127u], 1u);
+        if (p == prefix) atomicAdd(&h[k0 & 127u], 1u);
       }
     }
-    for (int i = 4 * n4 + threadIdx.x; i < t.nelem; i += blockDim.x) {
-      const unsigned k0 = key_of(m[i]), p = k0 >> 7;
-      above += ((p >> 12) == s.b1) && (p > prefix);
-      if (p == prefix) atomicAdd(&h[k0 & 127u], 1u);
+    above = __reduce_add_sync(0xffffffffu, above);
+    if ((threadIdx.x & 31) == 0 && above) atomicAdd(&cnt, above);
+    __syncthreads();
+    if (threadIdx.x == 0) tile_cnt[(long long)w * n_tiles + ti].y = cnt;
+    if (threadIdx.x < kBins3) {
+      const unsigned c = h[threadIdx.x];
+      tile_h3[((long long)w * n_tiles + ti) * kBins3 + threadIdx.x] = (unsigned short)c;
+      if (c) atomicAdd(&hist3[(long long)seg * kBins3 + threadIdx.x], c);
     }
-  }
-  above = __reduce_add_sync(0xffffffffu, above);
-  if ((threadIdx.x & 31) == 0 && above) atomicAdd(&cnt, above);
-  __syncthreads();
-  if (threadIdx.x == 0) tile_cnt[(long long)w * n_tiles + ti].y = cnt;
-  if (threadIdx.x < kBins3) {
-    const unsigned c = h[threadIdx.x];
-    tile_h3[((long long)w * n_tiles + ti) * kBins3 + threadIdx.x] = (unsigned short)c;
-    if (c) atomicAdd(&hist3[(long long)seg * kBins3 + threadIdx.x], c);
   }
 }
 
@@ -694,37 +708,52 @@ topk_tile_counts_kernel(const DevLayer* __restrict__ layers, const Tile* __restr
 }
 
 // One block per (worker, MATRIX layer): exclusive prefix, over the layer's tiles in index order, of the
-// per-tile (above, ties) counts, in place.
+// per-tile (above, ties) counts, in place.  The tiles that hold something to keep (above + ties > 0) join the
+// work list of the pass that will write their entries: the staged list or the select list.
 __global__ void __launch_bounds__(256)
 topk_tile_scan_kernel(const DevLayer* __restrict__ layers, const int* __restrict__ mat_layers, int n_mat,
-                      int n_tiles, int2* __restrict__ tile_pre) {
+                      int n_tiles, int W, const Select* __restrict__ sel, int2* __restrict__ tile_pre,
+                      unsigned* __restrict__ any_list, int2* __restrict__ lists) {
   __shared__ int2 chunk_sum[256];
+  __shared__ int chunk_act[256];
+  __shared__ unsigned s_base;
   const int seg = blockIdx.x, w = seg / n_mat, l = mat_layers[seg % n_mat];
   const DevLayer L = layers[l];
+  const int which = sel[seg].mode == kSelStaged ? kListStaged : kListSelect;
   const long long tb = (long long)w * n_tiles + L.tile0;
   const int per = (L.ntiles + 255) / 256;
   const int t0 = min(L.ntiles, (int)threadIdx.x * per), t1 = min(L.ntiles, t0 + per);
   int2 sum = make_int2(0, 0);
+  int act = 0;
   for (int t = t0; t < t1; ++t) {
     const int2 c = tile_pre[tb + t];
     sum.x += c.x; sum.y += c.y;
+    act += (c.x | c.y) != 0;
   }
   chunk_sum[threadIdx.x] = sum;
+  chunk_act[threadIdx.x] = act;
   __syncthreads();
   if (threadIdx.x == 0) {
     int2 run = make_int2(0, 0);
+    int ra = 0;
     for (int i = 0; i < 256; ++i) {
       const int2 c = chunk_sum[i];
+      const int a = chunk_act[i];
       chunk_sum[i] = run;
+      chunk_act[i] = ra;
       run.x += c.x; run.y += c.y;
+      ra += a;
     }
+    s_base = ra ? atomicAdd(&any_list[kListCountWord + which], (unsigned)ra) : 0u;
   }
   __syncthreads();
   int2 run = chunk_sum[threadIdx.x];
+  int2* dst = lists + (long long)which * W * n_tiles + s_base + chunk_act[threadIdx.x];
   for (int t = t0; t < t1; ++t) {
     const int2 c = tile_pre[tb + t];
     tile_pre[tb + t] = run;
     run.x += c.x; run.y += c.y;
+    if ((c.x | c.y) != 0) *dst++ = make_int2(w, L.tile0 + t);
   }
 }
 
@@ -827,27 +856,24 @@ __device__ __forceinline__ void select_tile(const Tile& t, const DevLayer& L, co
 __global__ void __launch_bounds__(256, 3)
 topk_select_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict__ tiles, int n_tiles, int n_mat,
                    float* __restrict__ err, const Select* __restrict__ sel, const int2* __restrict__ tile_pre,
-                   const unsigned* __restrict__ any_select, float* __restrict__ vals, int32_t* __restrict__ idx,
-                   long long stride, long long capacity, const int2* __restrict__ tile_cnt,
-                   const int2* __restrict__ tile_cand) {
+                   const unsigned* __restrict__ any_list, float* __restrict__ vals, int32_t* __restrict__ idx,
+                   long long stride, long long capacity, const int2* __restrict__ lists, int W) {
   __shared__ unsigned wtot[8];
-  if (*any_select == 0) return;  // every segment was served from staged entries
-  const int ti = blockIdx.x, w = blockIdx.y;
-  const Tile t = tiles[ti];
-  const DevLayer L = layers[t.layer];
-  if (L.kind != ACC_MATRIX) return;
-  const Select s = sel[w * n_mat + L.mat];
-  if (s.mode == kSelStaged) return;
-  const long long v = (long long)w * n_tiles + ti;
-  // list segments: the earlier pass counted the tile's keys above the collected bucket(s) and collected those
-  // inside; the threshold lies inside, so a tile with neither holds nothing to keep and is not read at all
-  // (most tiles of a row-sparse layer)
-  if (s.mode != kSelDense && tile_cnt[v].x == 0 && tile_cand[v].y == 0) return;
-  const int2 pre = tile_pre[v];
-  float* m = err + (long long)w * stride + L.offset + t.elem0;
-  const long long seg = (long long)w * capacity + L.seg_off;
-  if (t.nelem == kTile) select_tile<true>(t, L, s, pre, m, vals, idx, seg, wtot);
-  else select_tile<false>(t, L, s, pre, m, vals, idx, seg, wtot);
+  // the tiles of the non-staged segments that hold something to keep
+  const unsigned n_work = any_list[kListCountWord + kListSelect];
+  const int2* work = lists + (long long)kListSelect * W * n_tiles;
+  for (unsigned b = blockIdx.x; b < n_work; b += gridDim.x) {
+    __syncthreads();  // wtot of the previous tile is no longer read
+    const int w = work[b].x, ti = work[b].y;
+    const Tile t = tiles[ti];
+    const DevLayer L = layers[t.layer];
+    const Select s = sel[w * n_mat + L.mat];
+    const int2 pre = tile_pre[(long long)w * n_tiles + ti];
+    float* m = err + (long long)w * stride + L.offset + t.elem0;
+    const long long seg = (long long)w * capacity + L.seg_off;
+    if (t.nelem == kTile) select_tile<true>(t, L, s, pre, m, vals, idx, seg, wtot);
+    else select_tile<false>(t, L, s, pre, m, vals, idx, seg, wtot);
+  }
 }
 
 // Pass E', staged segments.  One warp per (tile, worker): the tile's staged entries (every element whose key
@@ -860,21 +886,22 @@ topk_finalize_staged_kernel(const DevLayer* __restrict__ layers, const Tile* __r
                             int n_mat, int W, float* __restrict__ err, const Select* __restrict__ sel,
                             const int2* __restrict__ tile_pre, const unsigned* __restrict__ cand,
                             const int2* __restrict__ tile_cand, long long cand_total, float* __restrict__ vals,
-                            int32_t* __restrict__ idx, long long stride, long long capacity) {
+                            int32_t* __restrict__ idx, long long stride, long long capacity,
+                            const unsigned* __restrict__ any_list, const int2* __restrict__ lists) {
   constexpr int kWords = kTile / 32;  // 256
   __shared__ unsigned bits_a[8][kWords], bits_t[8][kWords];
   __shared__ unsigned short pref_a[8][kWords], pref_t[8][kWords];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const long long v = (long long)blockIdx.x * 8 + warp;
-  if (v >= (long long)W * n_tiles) return;
-  const int w = (int)(v / n_tiles), ti = (int)(v % n_tiles);
+  const unsigned n_work = any_list[kListCountWord + kListStaged];
+  const int2* work = lists + (long long)kListStaged * W * n_tiles;
+  for (unsigned b = blockIdx.x * 8 + warp; b < n_work; b += gridDim.x * 8) {
+  __syncwarp();  // the maps of the previous tile are no longer read
+  const int w = work[b].x, ti = work[b].y;
+  const long long v = (long long)w * n_tiles + ti;
   const Tile t = tiles[ti];
   const DevLayer L = layers[t.layer];
-  if (L.kind != ACC_MATRIX) return;
   const Select s = sel[w * n_mat + L.mat];
-  if (s.mode != kSelStaged) return;
   const int2 tc = tile_cand[v];
-  if (tc.y == 0) return;
   const int2 pre = tile_pre[v];
   const uint2* ent = reinterpret_cast<const uint2*>(cand + (long long)w * cand_total + L.cand_base) + tc.x;
   unsigned* ba = bits_a[warp];
@@ -923,6 +950,7 @@ topk_finalize_staged_kernel(const DevLayer* __restrict__ layers, const Tile* __r
       idx[seg + pos] = (int32_t)e.y;
       m[e.y] = 0.f;
     }
+  }
   }
 }
 
@@ -1101,19 +1129,20 @@ static cudaError_t launch_topk_select_part(acc_ctx* ctx, const float* grads, flo
       PhaseTimer pt(ctx, PH_TOPK_PICK1, s);
       topk_pick1_kernel<<<W * n_mat, 256, 0, s>>>(ctx->d_layers, ctx->d_mat_layers, n_mat, c.n_layers, W, level,
                                                   ctx->d_hist1, ctx->d_sel, counts, ctx->d_pred, ctx->d_seg_cand,
-                                                  ctx->d_seg_flag, ctx->d_any_list);
+                                                  ctx->d_seg_flag, ctx->d_any_list, ctx->d_lists, nt);
     }
     {
       PhaseTimer pt(ctx, PH_TOPK_COLLECT, s);
       const long long cap = (long long)ctx->sm_count * 12;
       topk_collect_kernel<<<(unsigned)(V < cap ? V : cap), 256, 0, s>>>(
           ctx->d_layers, ctx->d_tiles, nt, n_mat, W, err, c.worker_stride, ctx->d_sel, ctx->d_any_list,
-          ctx->d_seg_cand, ctx->d_cand, ctx->d_tile_cand, pl.cand_total, ctx->d_tile_cnt);
+          ctx->d_seg_cand, ctx->d_cand, ctx->d_tile_cand, pl.cand_total, ctx->d_tile_cnt, ctx->d_lists);
     }
     {
       PhaseTimer pt(ctx, PH_TOPK_HIST2, s);
       topk_hist2_kernel<<<grid, 256, 0, s>>>(ctx->d_layers, ctx->d_tiles, nt, n_mat, err, c.worker_stride, W,
-                                             ctx->d_sel, ctx->d_any_list + 1, ctx->d_hist2, ctx->d_tile_cnt);
+                                             ctx->d_sel, ctx->d_any_list, ctx->d_hist2, ctx->d_tile_cnt,
+                                             ctx->d_lists);
     }
     {
       PhaseTimer pt(ctx, PH_TOPK_HIST2_LIST, s);
@@ -1127,9 +1156,9 @@ static cudaError_t launch_topk_select_part(acc_ctx* ctx, const float* grads, flo
     }
     {
       PhaseTimer pt(ctx, PH_TOPK_HIST3, s);
-      topk_hist3_kernel<<<dim3(nt, W), 256, 0, s>>>(ctx->d_layers, ctx->d_tiles, nt, n_mat, err, c.worker_stride,
-                                                    ctx->d_sel, ctx->d_any_list + 1, ctx->d_hist3, ctx->d_tile_cnt,
-                                                    ctx->d_tile_h3);
+      topk_hist3_kernel<<<grid, 256, 0, s>>>(ctx->d_layers, ctx->d_tiles, nt, n_mat, err, c.worker_stride,
+                                             ctx->d_sel, ctx->d_any_list, ctx->d_hist3, ctx->d_tile_cnt,
+                                             ctx->d_tile_h3, ctx->d_lists, W);
     }
     {
       PhaseTimer pt(ctx, PH_TOPK_HIST3_LIST, s);
@@ -1149,20 +1178,23 @@ static cudaError_t launch_topk_select_part(acc_ctx* ctx, const float* grads, flo
     }
     {
       PhaseTimer pt(ctx, PH_TOPK_PICK3_SCAN, s);
-      topk_tile_scan_kernel<<<W * n_mat, 256, 0, s>>>(ctx->d_layers, ctx->d_mat_layers, n_mat, nt, ctx->d_tile_pre);
+      topk_tile_scan_kernel<<<W * n_mat, 256, 0, s>>>(ctx->d_layers, ctx->d_mat_layers, n_mat, nt, W, ctx->d_sel,
+                                                      ctx->d_tile_pre, ctx->d_any_list, ctx->d_lists);
     }
   }
   if (n_mat > 0) {
     {
       PhaseTimer pt(ctx, PH_TOPK_FINALIZE_STAGED, s);
-      topk_finalize_staged_kernel<<<(unsigned)(((long long)W * nt + 7) / 8), 256, 0, s>>>(
+      const long long warps = (long long)W * nt, cap = (long long)ctx->sm_count * 8;
+      topk_finalize_staged_kernel<<<(unsigned)std::min((warps + 7) / 8, cap), 256, 0, s>>>(
           ctx->d_layers, ctx->d_tiles, nt, n_mat, W, err, ctx->d_sel, ctx->d_tile_pre, ctx->d_cand, ctx->d_tile_cand,
-          pl.cand_total, vals, idx, c.worker_stride, pl.capacity);
+          pl.cand_total, vals, idx, c.worker_stride, pl.capacity, ctx->d_any_list, ctx->d_lists);
     }
     PhaseTimer pt(ctx, PH_TOPK_SELECT, s);
-    topk_select_kernel<<<dim3(nt, W), 256, 0, s>>>(ctx->d_layers, ctx->d_tiles, nt, n_mat, err, ctx->d_sel,
-                                                   ctx->d_tile_pre, ctx->d_any_list + 2, vals, idx, c.worker_stride,
-                                                   pl.capacity, ctx->d_tile_cnt, ctx->d_tile_cand);
+    const long long blocks = (long long)W * nt, cap = (long long)ctx->sm_count * 12;
+    topk_select_kernel<<<(unsigned)std::min(blocks, cap), 256, 0, s>>>(
+        ctx->d_layers, ctx->d_tiles, nt, n_mat, err, ctx->d_sel, ctx->d_tile_pre, ctx->d_any_list, vals, idx,
+        c.worker_stride, pl.capacity, ctx->d_lists, W);
   }
   return cudaGetLastError();
 }
