@@ -908,11 +908,21 @@ topk_finalize_staged_kernel(const DevLayer* __restrict__ layers, const Tile* __r
   unsigned* bt = bits_t[warp];
   for (int i = lane; i < kWords; i += 32) { ba[i] = 0; bt[i] = 0; }
   __syncwarp();
-  for (int i = lane; i < tc.y; i += 32) {
-    const uint2 e = ent[i];
-    const unsigned kk = e.x & 0x7fffffffu, li = e.y - (unsigned)t.elem0;
-    if (kk > s.tau) atomicOr(&ba[li >> 5], 1u << (li & 31u));
-    else if (kk == s.tau) atomicOr(&bt[li >> 5], 1u << (li & 31u));
+  // entries are read four per lane at a time, so that the loads are in flight together (an absent entry reads
+  // as key 0, which lies below every staged threshold)
+  for (int i0 = 0; i0 < tc.y; i0 += 128) {
+    uint2 eb[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int i = i0 + 32 * u + lane;
+      eb[u] = i < tc.y ? ent[i] : make_uint2(0u, (unsigned)t.elem0);
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const unsigned kk = eb[u].x & 0x7fffffffu, li = eb[u].y - (unsigned)t.elem0;
+      if (kk > s.tau) atomicOr(&ba[li >> 5], 1u << (li & 31u));
+      else if (kk == s.tau) atomicOr(&bt[li >> 5], 1u << (li & 31u));
+    }
   }
   __syncwarp();
   {  // per-word exclusive prefix counts: lane l owns words 8l .. 8l+7
@@ -936,19 +946,28 @@ topk_finalize_staged_kernel(const DevLayer* __restrict__ layers, const Tile* __r
   __syncwarp();
   const long long seg = (long long)w * capacity + L.seg_off;
   float* m = err + (long long)w * stride + L.offset;
-  for (int i = lane; i < tc.y; i += 32) {
-    const uint2 e = ent[i];
-    const unsigned kk = e.x & 0x7fffffffu, li = e.y - (unsigned)t.elem0;
-    const bool is_a = kk > s.tau, is_t = kk == s.tau;
-    if (!is_a && !is_t) continue;
-    const unsigned wd = li >> 5, below = (1u << (li & 31u)) - 1u;
-    const int above_before = pre.x + (int)pref_a[warp][wd] + __popc(ba[wd] & below);
-    const int ties_before = pre.y + (int)pref_t[warp][wd] + __popc(bt[wd] & below);
-    if (is_a || ties_before < s.need) {
-      const int pos = above_before + min(ties_before, s.need);
-      vals[seg + pos] = __uint_as_float(e.x);
-      idx[seg + pos] = (int32_t)e.y;
-      m[e.y] = 0.f;
+  for (int i0 = 0; i0 < tc.y; i0 += 128) {
+    uint2 eb[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int i = i0 + 32 * u + lane;
+      eb[u] = i < tc.y ? ent[i] : make_uint2(0u, (unsigned)t.elem0);
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const uint2 e = eb[u];
+      const unsigned kk = e.x & 0x7fffffffu, li = e.y - (unsigned)t.elem0;
+      const bool is_a = kk > s.tau, is_t = kk == s.tau;
+      if (!is_a && !is_t) continue;
+      const unsigned wd = li >> 5, below = (1u << (li & 31u)) - 1u;
+      const int above_before = pre.x + (int)pref_a[warp][wd] + __popc(ba[wd] & below);
+      const int ties_before = pre.y + (int)pref_t[warp][wd] + __popc(bt[wd] & below);
+      if (is_a || ties_before < s.need) {
+        const int pos = above_before + min(ties_before, s.need);
+        vals[seg + pos] = __uint_as_float(e.x);
+        idx[seg + pos] = (int32_t)e.y;
+        m[e.y] = 0.f;
+      }
     }
   }
   }
@@ -1116,6 +1135,10 @@ static cudaError_t launch_topk_select_part(acc_ctx* ctx, const float* grads, flo
   e = cudaMemsetAsync(counts, 0, sizeof(int32_t) * (size_t)W * c.n_layers, s);
   if (e != cudaSuccess) return e;
   if (n_mat > 0) {
+    // blocks per segment of the list histograms: the longest possible list in 16 K-word pieces, 8..128
+    int max_cap = 0;
+    for (int l : pl.mat_layers) max_cap = std::max(max_cap, pl.layers[l].cand_cap);
+    const int list_chunks = std::min(128, std::max(8, max_cap / 16384));
     const long long V = (long long)W * nt;
     const int grid = (int)(V < (long long)ctx->sm_count * 8 ? V : (long long)ctx->sm_count * 8);
     {
@@ -1146,7 +1169,7 @@ static cudaError_t launch_topk_select_part(acc_ctx* ctx, const float* grads, flo
     }
     {
       PhaseTimer pt(ctx, PH_TOPK_HIST2_LIST, s);
-      topk_hist_list_kernel<2><<<dim3(128, W * n_mat), 256, 0, s>>>(ctx->d_layers, ctx->d_mat_layers, n_mat, ctx->d_sel,
+      topk_hist_list_kernel<2><<<dim3(list_chunks, W * n_mat), 256, 0, s>>>(ctx->d_layers, ctx->d_mat_layers, n_mat, ctx->d_sel,
                                                                    ctx->d_seg_cand, ctx->d_cand, pl.cand_total,
                                                                    ctx->d_hist2);
     }
@@ -1162,7 +1185,7 @@ static cudaError_t launch_topk_select_part(acc_ctx* ctx, const float* grads, flo
     }
     {
       PhaseTimer pt(ctx, PH_TOPK_HIST3_LIST, s);
-      topk_hist_list_kernel<3><<<dim3(128, W * n_mat), 256, 0, s>>>(ctx->d_layers, ctx->d_mat_layers, n_mat, ctx->d_sel,
+      topk_hist_list_kernel<3><<<dim3(list_chunks, W * n_mat), 256, 0, s>>>(ctx->d_layers, ctx->d_mat_layers, n_mat, ctx->d_sel,
                                                                    ctx->d_seg_cand, ctx->d_cand, pl.cand_total,
                                                                    ctx->d_hist3);
     }
@@ -1185,7 +1208,7 @@ static cudaError_t launch_topk_select_part(acc_ctx* ctx, const float* grads, flo
   if (n_mat > 0) {
     {
       PhaseTimer pt(ctx, PH_TOPK_FINALIZE_STAGED, s);
-      const long long warps = (long long)W * nt, cap = (long long)ctx->sm_count * 8;
+      const long long warps = (long long)W * nt, cap = (long long)ctx->sm_count * 32;
       topk_finalize_staged_kernel<<<(unsigned)std::min((warps + 7) / 8, cap), 256, 0, s>>>(
           ctx->d_layers, ctx->d_tiles, nt, n_mat, W, err, ctx->d_sel, ctx->d_tile_pre, ctx->d_cand, ctx->d_tile_cand,
           pl.cand_total, vals, idx, c.worker_stride, pl.capacity, ctx->d_any_list, ctx->d_lists);
