@@ -15,6 +15,7 @@ constexpr int kBins1 = 4096;       // radix-select level 1: key bits [30:19]
 constexpr int kBins2 = 4096;       // level 2: key bits [18:7]
 constexpr int kBins3 = 128;        // level 3: key bits [6:0]
 constexpr int kColBlockThreads = 256;
+constexpr int kMaxWorkers = 1024;  // workers per context
 
 // One layer, device-side view.
 struct DevLayer {

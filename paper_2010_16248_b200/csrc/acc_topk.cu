@@ -985,6 +985,7 @@ topk_decompress_kernel(const DevLayer* __restrict__ layers, const Tile* __restri
                        const int32_t* __restrict__ idx, float* __restrict__ out, float* __restrict__ delta,
                        long long stride, long long capacity, int W, int decider, float inv_w, const SgdTail tail) {
   __shared__ float acc[kTile];
+  __shared__ int r_lo[kMaxWorkers], r_hi[kMaxWorkers];
   const int ti = blockIdx.x;
   const Tile t = tiles[ti];
   const DevLayer L = layers[t.layer];
@@ -1005,19 +1006,44 @@ topk_decompress_kernel(const DevLayer* __restrict__ layers, const Tile* __restri
     return;
   }
   for (int i = threadIdx.x; i < kTile; i += blockDim.x) acc[i] = 0.f;
-  __syncthreads();
+  // the tile's range inside every worker's packed segment, all workers at once
   const bool last = ti == L.tile0 + L.ntiles - 1;
-  for (int w = 0; w < W; ++w) {
+  for (int w = threadIdx.x; w < W; w += blockDim.x) {
     const Select s = sel[w * n_mat + L.mat];
     const int2 p0 = tile_pre[(long long)w * n_tiles + ti];
-    const int start = p0.x + min(p0.y, s.need);
     int end = s.k;
     if (!last) {
       const int2 p1 = tile_pre[(long long)w * n_tiles + ti + 1];
       end = p1.x + min(p1.y, s.need);
     }
+    r_lo[w] = p0.x + min(p0.y, s.need);
+    r_hi[w] = end;
+  }
+  __syncthreads();
+  // workers are added one after the other (an element may be kept by several of them and the order of the sum
+  // is fixed); the first entry of the next worker is fetched before the barrier, so its latency is hidden
+  int ni = 0;
+  float nv = 0.f;
+  bool have = false;
+  {
+    const int i = r_lo[0] + (int)threadIdx.x;
+    have = i < r_hi[0];
+    if (have) { const long long seg = L.seg_off; ni = idx[seg + i]; nv = vals[seg + i]; }
+  }
+  for (int w = 0; w < W; ++w) {
     const long long seg = (long long)w * capacity + L.seg_off;
-    for (int i = start + threadIdx.x; i < end; i += blockDim.x) acc[idx[seg + i] - t.elem0] += vals[seg + i];
+    const int ci = ni;
+    const float cv = nv;
+    const bool chave = have;
+    if (w + 1 < W) {
+      const long long nseg = (long long)(w + 1) * capacity + L.seg_off;
+      const int i = r_lo[w + 1] + (int)threadIdx.x;
+      have = i < r_hi[w + 1];
+      if (have) { ni = idx[nseg + i]; nv = vals[nseg + i]; }
+    }
+    if (chave) acc[ci - t.elem0] += cv;
+    for (int i = r_lo[w] + (int)threadIdx.x + (int)blockDim.x; i < r_hi[w]; i += blockDim.x)
+      acc[idx[seg + i] - t.elem0] += vals[seg + i];
     __syncthreads();
   }
   const int n4 = t.nelem >> 2;
