@@ -189,7 +189,7 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=5)
-    ap.add_argument("--config", type=int, default=5, help="BASELINE config 1..5 (default: 5, the largest gradient set)")
+    ap.add_argument("--config", type=int, default=5, help="benchmark configuration 1..5 (default: 5, the largest gradient set)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=8)
     ap.add_argument("--no-cpu-baseline", action="store_true")

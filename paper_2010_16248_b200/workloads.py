@@ -148,7 +148,7 @@ def shapes_lstm(vocab: int = 33278, hidden: int = 650):
 
 
 # --------------------------------------------------------------------------- #
-# Workload descriptions (BASELINE configs 0..4 are c1..c5 here)
+# Workload descriptions (the five benchmark configurations, c1..c5)
 # --------------------------------------------------------------------------- #
 @dataclasses.dataclass
 class Workload:
@@ -173,7 +173,7 @@ class Workload:
 
 
 def workload(config: int, scale: int = 1) -> Workload:
-    """Return BASELINE config ``config`` (1..5).  ``scale`` > 1 shrinks widths /
+    """Return benchmark configuration ``config`` (1..5).  ``scale`` > 1 shrinks widths /
     vocabulary by that factor (CPU-sized versions of the same structure)."""
     if config == 1:
         n, m = max(256 // scale, 8), max(1152 // scale, 9)

@@ -7,7 +7,7 @@ import torch
 from oracle import accordion_oracle as orc
 
 # Float tolerance of the parity tests: relative Frobenius error per layer, fp32 kernels against the
-# fp64 oracle (the benchmark spec: <= 1e-4).
+# fp64 oracle (the target stated for this path: <= 1e-4).
 REL_TOL = 1e-4
 
 

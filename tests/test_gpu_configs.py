@@ -1,4 +1,4 @@
-"""The five BASELINE configurations on the GPU against the oracle.
+"""The five benchmark configurations on the GPU against the oracle.
 
 Protocol.  TopK and the controller are bit-reproducible, so they run free over the iterations and must
 match exactly (levels, indices, counts, packed value bits, error memory).  PowerSGD is compared per step
