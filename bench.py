@@ -197,6 +197,8 @@ def main():
     ap.add_argument("--no-graphs", action="store_true", help="issue the timed steps call by call instead of as CUDA graphs")
     ap.add_argument("--pipeline", default="auto", choices=["auto", "always", "never"],
                     help="first PowerSGD pass: persistent bulk-copy pipeline, direct kernel, or the library's choice")
+    ap.add_argument("--no-overlap", action="store_true",
+                    help="two-compressor configs: run the TopK step after the PowerSGD step instead of beside it")
     ap.add_argument("--sgd-tail", action="store_true",
                     help="single-compressor configs: apply the Nesterov update inside the step (fused optimiser tail)")
     ap.add_argument("--batch-mode", action="store_true",
@@ -247,7 +249,8 @@ def main():
         optimizer = {"params": torch.zeros(table.stride, device=dev), "lr": 0.1, "momentum": 0.9}
     eng = pipeline.AccordionStep(table, W, w.compressors, w.rank_low, w.rank_high, w.topk_low_bp, w.topk_high_bp,
                                  w.eta, 1e-8, w.check_every, device=dev, lazy_residual=not args.eager,
-                                 optimizer=optimizer, extra_flags={"auto": 0, "always": 2, "never": 4}[args.pipeline])
+                                 optimizer=optimizer, extra_flags={"auto": 0, "always": 2, "never": 4}[args.pipeline],
+                                 overlap=not args.no_overlap)
     n_mat = table.n_matrix_params
     grad_bytes_step = n_comp * 4.0 * W * table.n_params
 
@@ -303,11 +306,14 @@ def main():
     value = dist_util.whole_job_throughput(grad_bytes_step, ms_per_step, world) / 1e9
 
     # ---- same K steps again with per-kernel CUDA events (on the launching stream) for the roofline
+    # (the two compressors one after the other here, so that a kernel's events bracket that kernel alone)
+    overlap, eng.overlap = eng.overlap, False
     eng.ctx.acc_profile_enable(True)
     run_steps(K)
     torch.cuda.synchronize()
     prof = eng.ctx.acc_profile_read()
     eng.ctx.acc_profile_enable(False)
+    eng.overlap = overlap
     peak, peak_src = _peaks()
     units = W * n_mat
     total_k_ms = sum(ms for ms, _ in prof.values())
@@ -370,6 +376,8 @@ def main():
                            "l2_policy": f"inputs larger than L2: {RING} gradient batches of "
                                         f"{4 * W * table.stride / 1e6:.0f} MB cycled, no flush",
                            "launch": "CUDA graph replay per step" if use_graphs else "direct calls",
+                           "streams": ("TopK step beside the PowerSGD step on a second stream"
+                                       if (n_comp == 2 and not args.no_overlap) else "one stream"),
                            "multi_gpu": "independent replicas, no collective"},
                 "clocks": clocks, "e2e": e2e, "gpu_launches": gpu_launches,
                 "roofline": roofline, "cpu_baseline": cpu,

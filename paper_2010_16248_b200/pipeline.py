@@ -20,8 +20,11 @@ class AccordionStep:
     def __init__(self, table: wl.LayerTable, n_workers: int, compressors: Sequence[str] = ("powersgd",),
                  rank_low=2, rank_high=1, topk_low_bp=1000, topk_high_bp=100, eta=0.5, gs_eps=1e-8,
                  check_every=10, decider=0, q_init=None, device="cuda", lazy_residual=False, optimizer=None,
-                 extra_flags=0):
-        """``extra_flags``: further ACC_FLAG_* bits for the context (e.g. forcing one implementation of the first
+                 extra_flags=0, overlap=True):
+        """``overlap``: with two compressors, the TopK step runs on a second stream beside the PowerSGD step
+        (they share only the gradients and the level array, both read-only), so that the short, latency-bound
+        kernels of one hide behind the streaming kernels of the other; the results are the same bits.
+        ``extra_flags``: further ACC_FLAG_* bits for the context (e.g. forcing one implementation of the first
         PowerSGD pass).  ``optimizer``: None, or a dict ``{"params": tensor [stride], "lr": .., "momentum": 0.9,
         "weight_decay": 0.0}``: the Nesterov update (Appendix A) is then applied to ``params`` by the kernels
         that produce the averaged gradient (one compressor only)."""
@@ -42,6 +45,9 @@ class AccordionStep:
         self.norm2_prev = torch.full((L,), -1.0, dtype=torch.float64, device=dev)
         self.t = 0
         self.launches = 0
+        self.overlap = overlap
+        self._side = torch.cuda.Stream(device=dev)
+        self._fork, self._join = torch.cuda.Event(), torch.cuda.Event()
         self.params = self.mom = self.hyper = None
         if optimizer is not None:
             self.params = optimizer["params"]
@@ -62,6 +68,24 @@ class AccordionStep:
         """One iteration on device-resident gradients ``[W, stride]``."""
         c = self.ctx
         delta: Optional[torch.Tensor] = self.delta  # accumulated once per iteration, by the first compressor
+        if self.overlap and len(self.compressors) == 2:
+            main = stream if stream is not None else torch.cuda.current_stream(self.device)
+            self._fork.record(main)
+            self._side.wait_event(self._fork)
+            c.acc_topk_step(grads, self.err_topk, self.level, self.vals, self.idx, self.counts, self.out_topk,
+                            None, self._side)
+            self.launches += c.last_launch_count()
+            c.acc_powersgd_step(grads, self.err_psgd, self.q, self.p_hat, self.level, self.out_psgd, delta, main)
+            self.launches += c.last_launch_count()
+            self._join.record(self._side)
+            main.wait_event(self._join)
+            self.t += 1
+            if self.t % self.check_every == 0:
+                c.acc_layer_norms(self.delta, 1, self.norm2_curr, stream=main)
+                self.launches += c.last_launch_count()
+                c.acc_detect_regime(self.norm2_curr, self.norm2_prev, lr_curr, lr_next, self.level, self.delta, main)
+                self.launches += c.last_launch_count()
+            return
         if "powersgd" in self.compressors:
             if self.params is not None:
                 c.acc_powersgd_step_sgd(grads, self.err_psgd, self.q, self.p_hat, self.level, self.out_psgd, delta,

@@ -474,3 +474,26 @@ def test_checkpoint_resume_is_bit_identical():
     torch.cuda.synchronize()
     for n in names:
         assert torch.equal(getattr(full, n), getattr(second, n)), n
+
+
+def test_two_compressors_side_by_side_equal_one_after_the_other():
+    """With both compressors the engine runs the TopK step on a second stream beside the PowerSGD step; every
+    result must be the bits of the sequential order, directly and as replayed CUDA graphs."""
+    table = _table_mixed()
+    W = 3
+    q0 = wl.initial_q(table, 2, seed=31)
+    engines = [pipeline.AccordionStep(table, W, ("powersgd", "topk"), check_every=2, q_init=q0, lazy_residual=True,
+                                      overlap=ov) for ov in (False, True, True)]
+    bufs = [_random_inputs(table, W, 1200 + i)[0] for i in range(2)]
+    engines[2].capture_graphs(bufs)
+    for t in range(6):
+        engines[0].step(bufs[t % 2])
+        engines[1].step(bufs[t % 2])
+        engines[2].step_graph(t % 2)
+    torch.cuda.synchronize()
+    ref = engines[0]
+    for e in engines[1:]:
+        for name in ("out_psgd", "out_topk", "err_psgd", "err_topk", "q", "p_hat", "vals", "idx", "counts", "level",
+                     "delta", "norm2_prev"):
+            assert torch.equal(getattr(ref, name), getattr(e, name)), name
+        assert e.launches == ref.launches
