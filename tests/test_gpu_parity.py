@@ -497,3 +497,33 @@ def test_two_compressors_side_by_side_equal_one_after_the_other():
                      "delta", "norm2_prev"):
             assert torch.equal(getattr(ref, name), getattr(e, name)), name
         assert e.launches == ref.launches
+
+
+def test_topk_whole_model_selection_scope():
+    """Selection over the whole model instead of per layer is the same step on a table whose single MATRIX layer
+    spans all parameters: k = floor(N * K) entries are kept across what were the layers."""
+    per_layer = _table_mixed()
+    n = int(per_layer.stride)
+    table = wl.make_table([("model", (1, n))])
+    W = 2
+    ctx = binding.Context(table, W, topk_low_bp=500, topk_high_bp=50)
+    grads = torch.zeros(W, table.stride, device="cuda")
+    g, _ = _random_inputs(per_layer, W, 77)
+    grads[:, :n] = g
+    err = torch.zeros_like(grads)
+    vals, idx, counts = ctx.new_topk_buffers()
+    out = torch.zeros(table.stride, device="cuda")
+    for lv in (1, 0, 0):
+        level = torch.full((1,), lv, dtype=torch.uint8, device="cuda")
+        e0 = err.clone()
+        ctx.acc_topk_step(grads, err, level, vals, idx, counts, out)
+        torch.cuda.synchronize()
+        H.check_topk_against_oracle(ctx, table, grads, e0, level, vals, idx, counts, out, err, 500, 50)
+        assert int(counts[0]) == max(1, n * (500 if lv else 50) // 10000)
+    # the layers with the largest scale (10^0) carry nearly all kept entries: the scope really is global
+    kept = idx[:int(counts[0])].cpu().numpy()
+    big = np.zeros(n, bool)
+    for l, sl in per_layer.slices():
+        if l % 4 == 0:
+            big[sl] = True
+    assert big[kept].mean() > 0.9
