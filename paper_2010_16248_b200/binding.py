@@ -357,7 +357,8 @@ class Context:
     # --- buffer helpers (allocation and layout conversion only) -------------------------------
     def new_q(self, q_list=None):
         """Device q buffer ``[q_rows, 4]``; filled from per-layer ``[m, r]`` tensors when given."""
-        q = torch.zeros(self.q_rows, ACC_MAX_RANK, dtype=torch.float32, device=self.device)
+        # (at least one row, so that a table without MATRIX layers still has a buffer to point at)
+        q = torch.zeros(max(self.q_rows, 1), ACC_MAX_RANK, dtype=torch.float32, device=self.device)
         if q_list is not None:
             for l, ql in enumerate(q_list):
                 if ql is not None:
@@ -366,11 +367,11 @@ class Context:
         return q
 
     def new_p(self):
-        return torch.zeros(self.p_rows, ACC_MAX_RANK, dtype=torch.float32, device=self.device)
+        return torch.zeros(max(self.p_rows, 1), ACC_MAX_RANK, dtype=torch.float32, device=self.device)
 
     def new_topk_buffers(self):
         W = self.n_workers
-        vals = torch.zeros(W * self.capacity, dtype=torch.float32, device=self.device)
-        idx = torch.zeros(W * self.capacity, dtype=torch.int32, device=self.device)
+        vals = torch.zeros(max(W * self.capacity, 4), dtype=torch.float32, device=self.device)
+        idx = torch.zeros(max(W * self.capacity, 4), dtype=torch.int32, device=self.device)
         counts = torch.zeros(W * self.n_layers, dtype=torch.int32, device=self.device)
         return vals, idx, counts

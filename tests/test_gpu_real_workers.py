@@ -218,3 +218,28 @@ def test_one_rank_nccl_process_group():
         assert torch.equal(st.out, ref.out) and torch.equal(st.q, ref.q)
     finally:
         dist.destroy_process_group()
+
+
+@pytest.mark.parametrize("shapes", [[("w", (40, 30))], [("b", (100,))], [("w0", (9, 700)), ("b", (5,)), ("w1", (700, 9))]])
+@pytest.mark.parametrize("compressor", ["powersgd", "topk"])
+def test_degenerate_tables_two_ranks(shapes, compressor):
+    """Tables without VECTOR layers, without MATRIX layers, and with very flat / very tall matrices: two ranks of
+    one worker each against the single-context step over both workers."""
+    table = wl.make_table(shapes)
+    world, n_local = 2, 1
+    q0 = wl.initial_q(table, 2, seed=5)
+    batches = [_random_inputs(table, world, 1300 + it)[0] for it in range(3)]
+
+    def make_step(exchange):
+        return pipeline.DistributedStep(table, n_local, compressor, check_every=2, q_init=q0, exchange=exchange)
+
+    steps = _run_ranks(world, make_step, 3, lambda it, r: batches[it][r:r + 1].contiguous())
+    single = pipeline.AccordionStep(table, world, (compressor,), check_every=2, q_init=q0)
+    for it in range(3):
+        single.step(batches[it])
+    torch.cuda.synchronize()
+    ref = single.out_psgd if compressor == "powersgd" else single.out_topk
+    assert torch.equal(steps[0].out, steps[1].out) and torch.equal(steps[0].level, single.level)
+    for l, sl in table.slices():
+        got, want = steps[0].out[sl].cpu().numpy(), ref[sl].cpu().numpy()
+        assert H.rel_err(got, want, 1e-7 * np.linalg.norm(want) + 1e-12) <= 1e-4, (l, compressor)
