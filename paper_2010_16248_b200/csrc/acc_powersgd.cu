@@ -175,7 +175,8 @@ constexpr int kPipePos = kTile / 4 / kPipeThreads;  // float4 positions per thre
 constexpr int kPipeStages = 2;
 constexpr int kPipeMinStagesPerSm = 200;  // below this the direct kernel is used
 constexpr int kPipeWarps = kPipeThreads / 32;
-constexpr size_t kPipeSmemBytes = sizeof(float) * kTile * (2 * kPipeStages + 1) + sizeof(float4) * 2 * kPipeWarps + 64;
+// stage buffers, the mean matrix of the tile, the detector accumulator of the tile
+constexpr size_t kPipeSmemBytes = sizeof(float) * kTile * (2 * kPipeStages + 2) + sizeof(float4) * 2 * kPipeWarps + 64;
 
 template <bool LAZY>
 __global__ void __launch_bounds__(kPipeThreads, 1)
@@ -188,7 +189,8 @@ psgd_project_pipe_kernel(const DevLayer* __restrict__ layers, const Tile* __rest
   extern __shared__ __align__(128) unsigned char smem_raw[];
   float* stage = reinterpret_cast<float*>(smem_raw);                  // [kPipeStages buffers][g, e][kTile]
   float* s_mbar = stage + 2 * kPipeStages * kTile;                    // [kTile]
-  float4* s_pp = reinterpret_cast<float4*>(s_mbar + kTile);           // [kPipeWarps][2] partial rows of P
+  float* s_delta = s_mbar + kTile;                                    // [kTile] detector accumulator of the tile
+  float4* s_pp = reinterpret_cast<float4*>(s_delta + kTile);          // [kPipeWarps][2] partial rows of P
   uint64_t* bars = reinterpret_cast<uint64_t*>(s_pp + 2 * kPipeWarps);  // [kPipeStages]
   for (int i = blockIdx.x; i < n_vec_tiles; i += gridDim.x) {
     const Tile t = tiles[vec_tiles[i]];
@@ -203,6 +205,7 @@ psgd_project_pipe_kernel(const DevLayer* __restrict__ layers, const Tile* __rest
     fence_mbar_init();
   }
   __syncthreads();
+  const bool delta_by_copy = delta != nullptr && W >= 2;
   // thread 0 only: the tile whose stages are being issued is kept in registers, so that issuing a stage costs
   // no dependent global loads (they would sit on the critical path of every stage)
   int is_ti = -1;
@@ -218,9 +221,14 @@ psgd_project_pipe_kernel(const DevLayer* __restrict__ layers, const Tile* __rest
     }
     const long long base = (long long)w * stride + is_base;
     const int buf = it % kPipeStages;
-    mbar_arrive_expect_tx(&bars[buf], 2 * is_bytes);
+    // the deciding worker's stage also brings the tile of the detector's accumulator (single buffer: it is
+    // read once per tile, W stages apart; with W == 1 the next copy would overtake the read, so that case
+    // reads the accumulator with plain loads)
+    const bool with_delta = delta_by_copy && w == decider;
+    mbar_arrive_expect_tx(&bars[buf], (with_delta ? 3 : 2) * is_bytes);
     bulk_copy_g2s(stage + (2 * buf) * kTile, grads + base, is_bytes, &bars[buf]);
     bulk_copy_g2s(stage + (2 * buf + 1) * kTile, err + base, is_bytes, &bars[buf]);
+    if (with_delta) bulk_copy_g2s(s_delta, delta + is_base, is_bytes, &bars[buf]);
   };
   if (threadIdx.x == 0)
     for (int it = 0; it < kPipeStages && it < n_stages; ++it) issue(it);
@@ -274,7 +282,8 @@ psgd_project_pipe_kernel(const DevLayer* __restrict__ layers, const Tile* __rest
       if (e0 + 3 < t.nelem) {
         st_stream4(err + gbase + e0, mw);
         if (acc_delta) {
-          float4 d = *reinterpret_cast<const float4*>(delta + L.offset + t.elem0 + e0);
+          float4 d = delta_by_copy ? *reinterpret_cast<const float4*>(s_delta + e0)
+                                   : *reinterpret_cast<const float4*>(delta + L.offset + t.elem0 + e0);
           d.x += gv.x; d.y += gv.y; d.z += gv.z; d.w += gv.w;
           *reinterpret_cast<float4*>(delta + L.offset + t.elem0 + e0) = d;
         }
@@ -282,7 +291,8 @@ psgd_project_pipe_kernel(const DevLayer* __restrict__ layers, const Tile* __rest
         const float mm[4] = {mw.x, mw.y, mw.z, mw.w}, gg[4] = {gv.x, gv.y, gv.z, gv.w};
         for (int e2 = 0; e0 + e2 < t.nelem; ++e2) {
           err[gbase + e0 + e2] = mm[e2];
-          if (acc_delta) delta[L.offset + t.elem0 + e0 + e2] += gg[e2];
+          if (acc_delta)
+            delta[L.offset + t.elem0 + e0 + e2] = (delta_by_copy ? s_delta[e0 + e2] : delta[L.offset + t.elem0 + e0 + e2]) + gg[e2];
         }
       }
     }
