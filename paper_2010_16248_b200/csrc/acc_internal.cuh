@@ -218,6 +218,42 @@ __device__ __forceinline__ void sgd_apply4(const SgdTail& t, const SgdHyper& h, 
   *reinterpret_cast<float4*>(t.mom + i) = u;
 }
 
+// One VECTOR tile: mean over the workers of the tile's gradients, four elements per thread and step, the W loads
+// of a step in flight together; the deciding worker's values are added to delta after the loop (no
+// read-modify-write between the loads).  emit4(i, v) / emit1(i, v) receive the means of elements [i, i+4) / i.
+template <typename Emit4, typename Emit1>
+__device__ __forceinline__ void vector_tile_mean(const float* __restrict__ g /* worker 0, first element */,
+                                                 long long stride, int W, int decider, float inv_w, int nelem,
+                                                 float* __restrict__ delta /* first element, or nullptr */,
+                                                 Emit4 emit4, Emit1 emit1) {
+  const int n4 = nelem >> 2;
+  for (int f = threadIdx.x; f < n4; f += blockDim.x) {
+    float4 a = make_float4(0.f, 0.f, 0.f, 0.f), gd = a;
+#pragma unroll 8
+    for (int w = 0; w < W; ++w) {
+      const float4 v = ld_stream4(g + (long long)w * stride + 4 * f);
+      a.x += v.x; a.y += v.y; a.z += v.z; a.w += v.w;
+      if (w == decider) gd = v;
+    }
+    if (delta != nullptr) {
+      float4 d = *reinterpret_cast<const float4*>(delta + 4 * f);
+      d.x += gd.x; d.y += gd.y; d.z += gd.z; d.w += gd.w;
+      *reinterpret_cast<float4*>(delta + 4 * f) = d;
+    }
+    emit4(4 * f, make_float4(a.x * inv_w, a.y * inv_w, a.z * inv_w, a.w * inv_w));
+  }
+  for (int i = 4 * n4 + threadIdx.x; i < nelem; i += blockDim.x) {
+    float a = 0.f, gd = 0.f;
+    for (int w = 0; w < W; ++w) {
+      const float v = g[(long long)w * stride + i];
+      a += v;
+      gd = w == decider ? v : gd;
+    }
+    if (delta != nullptr) delta[i] += gd;
+    emit1(i, a * inv_w);
+  }
+}
+
 __device__ __forceinline__ double warp_sum(double v) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);

@@ -53,15 +53,9 @@ __device__ void vector_mean_tile(const Tile& t, const DevLayer& L, const float* 
                                  float* __restrict__ out, float* __restrict__ delta, long long stride, int W,
                                  int decider, float inv_w) {
   const long long base = L.offset + t.elem0;
-  for (int i = threadIdx.x; i < t.nelem; i += blockDim.x) {
-    float acc = 0.f;
-    for (int w = 0; w < W; ++w) {
-      const float g = grads[(long long)w * stride + base + i];
-      acc += g;
-      if (delta != nullptr && w == decider) delta[base + i] += g;
-    }
-    out[base + i] = acc * inv_w;
-  }
+  float* o = out + base;
+  vector_tile_mean(grads + base, stride, W, decider, inv_w, t.nelem, delta != nullptr ? delta + base : nullptr,
+                   [&](int i, float4 v) { *reinterpret_cast<float4*>(o + i) = v; }, [&](int i, float v) { o[i] = v; });
 }
 
 // Pass 1.  One block per tile, all workers:

@@ -141,10 +141,19 @@ topk_ef_hist1_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict
             }
           }
         }
-        if (acc_delta) {
-          float4 d = *reinterpret_cast<const float4*>(delta + base + 4 * i);
-          d.x += gv.x; d.y += gv.y; d.z += gv.z; d.w += gv.w;
-          *reinterpret_cast<float4*>(delta + base + 4 * i) = d;
+      }
+      if (acc_delta) {  // detector accumulator of the batch: its loads together too (err's registers are free now)
+#pragma unroll
+        for (int u = 0; u < kBatch; ++u) {
+          const int i = i0 + u * kThreads + (int)threadIdx.x;
+          if (i < n4) eb[u] = *reinterpret_cast<const float4*>(delta + base + 4 * i);
+        }
+#pragma unroll
+        for (int u = 0; u < kBatch; ++u) {
+          const int i = i0 + u * kThreads + (int)threadIdx.x;
+          if (i < n4)
+            *reinterpret_cast<float4*>(delta + base + 4 * i) =
+                make_float4(eb[u].x + gb[u].x, eb[u].y + gb[u].y, eb[u].z + gb[u].z, eb[u].w + gb[u].w);
         }
       }
     }
@@ -993,16 +1002,15 @@ topk_decompress_kernel(const DevLayer* __restrict__ layers, const Tile* __restri
   SgdHyper h = {0.f, 0.f, 0.f};
   if (SGD) h = sgd_hyper(tail);
   if (L.kind != ACC_MATRIX) {
-    for (int i = threadIdx.x; i < t.nelem; i += blockDim.x) {
-      float a = 0.f;
-      for (int w = 0; w < W; ++w) {
-        const float g = grads[(long long)w * stride + base + i];
-        a += g;
-        if (delta != nullptr && w == decider) delta[base + i] += g;
-      }
-      out[base + i] = a * inv_w;
-      if (SGD) sgd_apply1(tail, h, base + i, a * inv_w);
-    }
+    vector_tile_mean(grads + base, stride, W, decider, inv_w, t.nelem, delta != nullptr ? delta + base : nullptr,
+                     [&](int i, float4 v) {
+                       *reinterpret_cast<float4*>(out + base + i) = v;
+                       if (SGD) sgd_apply4(tail, h, base + i, v);
+                     },
+                     [&](int i, float v) {
+                       out[base + i] = v;
+                       if (SGD) sgd_apply1(tail, h, base + i, v);
+                     });
     return;
   }
   for (int i = threadIdx.x; i < kTile; i += blockDim.x) acc[i] = 0.f;
@@ -1069,15 +1077,9 @@ topk_vec_local_kernel(const DevLayer* __restrict__ layers, const Tile* __restric
   const Tile t = tiles[vec_tiles[blockIdx.x]];
   const DevLayer L = layers[t.layer];
   const long long base = L.offset + t.elem0;
-  for (int i = threadIdx.x; i < t.nelem; i += blockDim.x) {
-    float a = 0.f;
-    for (int w = 0; w < W; ++w) {
-      const float g = grads[(long long)w * stride + base + i];
-      a += g;
-      if (delta != nullptr && w == decider) delta[base + i] += g;
-    }
-    packed[L.vec_off + t.elem0 + i] = a * inv_w;
-  }
+  float* x = packed + L.vec_off + t.elem0;
+  vector_tile_mean(grads + base, stride, W, decider, inv_w, t.nelem, delta != nullptr ? delta + base : nullptr,
+                   [&](int i, float4 v) { *reinterpret_cast<float4*>(x + i) = v; }, [&](int i, float v) { x[i] = v; });
 }
 
 // First position in the ascending array a[0..n) whose value is >= key.
