@@ -849,9 +849,11 @@ __device__ __forceinline__ void select_tile(const Tile& t, const DevLayer& L, co
         const bool is_a = (a >> e) & 1u, is_t = (tt >> e) & 1u;
         if (is_a || (is_t && ties_before < s.need)) {
           const int pos = above_before + min(ties_before, s.need);
-          vals[seg + pos] = v[e];
-          idx[seg + pos] = t.elem0 + e0 + e;
-          m[e0 + e] = 0.f;
+          if ((unsigned)pos < (unsigned)s.k) {  // always true for consistent counts; keeps a write inside the segment
+            vals[seg + pos] = v[e];
+            idx[seg + pos] = t.elem0 + e0 + e;
+            m[e0 + e] = 0.f;
+          }
         }
         above_before += is_a;
         ties_before += is_t;
@@ -973,9 +975,11 @@ topk_finalize_staged_kernel(const DevLayer* __restrict__ layers, const Tile* __r
       const int ties_before = pre.y + (int)pref_t[warp][wd] + __popc(bt[wd] & below);
       if (is_a || ties_before < s.need) {
         const int pos = above_before + min(ties_before, s.need);
-        vals[seg + pos] = __uint_as_float(e.x);
-        idx[seg + pos] = (int32_t)e.y;
-        m[e.y] = 0.f;
+        if ((unsigned)pos < (unsigned)s.k && li < (unsigned)t.nelem) {  // always true for consistent lists
+          vals[seg + pos] = __uint_as_float(e.x);
+          idx[seg + pos] = (int32_t)e.y;
+          m[e.y] = 0.f;
+        }
       }
     }
   }
@@ -1024,8 +1028,8 @@ topk_decompress_kernel(const DevLayer* __restrict__ layers, const Tile* __restri
       const int2 p1 = tile_pre[(long long)w * n_tiles + ti + 1];
       end = p1.x + min(p1.y, s.need);
     }
-    r_lo[w] = p0.x + min(p0.y, s.need);
-    r_hi[w] = end;
+    r_lo[w] = min(p0.x + min(p0.y, s.need), s.k);  // (the clamps hold by construction)
+    r_hi[w] = min(end, s.k);
   }
   __syncthreads();
   // workers are added one after the other (an element may be kept by several of them and the order of the sum
@@ -1049,9 +1053,11 @@ topk_decompress_kernel(const DevLayer* __restrict__ layers, const Tile* __restri
       have = i < r_hi[w + 1];
       if (have) { ni = idx[nseg + i]; nv = vals[nseg + i]; }
     }
-    if (chave) acc[ci - t.elem0] += cv;
-    for (int i = r_lo[w] + (int)threadIdx.x + (int)blockDim.x; i < r_hi[w]; i += blockDim.x)
-      acc[idx[seg + i] - t.elem0] += vals[seg + i];
+    if (chave && (unsigned)(ci - t.elem0) < (unsigned)kTile) acc[ci - t.elem0] += cv;
+    for (int i = r_lo[w] + (int)threadIdx.x + (int)blockDim.x; i < r_hi[w]; i += blockDim.x) {
+      const unsigned li = (unsigned)(idx[seg + i] - t.elem0);
+      if (li < (unsigned)kTile) acc[li] += vals[seg + i];
+    }
     __syncthreads();
   }
   const int n4 = t.nelem >> 2;
@@ -1134,7 +1140,10 @@ topk_decompress_packed_kernel(const DevLayer* __restrict__ layers, const Tile* _
     for (int jj = 0; jj < nj; ++jj) {  // sets in order: the sum of an element's contributions has a fixed order
       const long long seg = (long long)(j0 + jj) * capacity + L.seg_off;
       const int lo = range[2 * jj], hi = range[2 * jj + 1];
-      for (int i = lo + (int)threadIdx.x; i < hi; i += blockDim.x) acc[idx[seg + i] - t.elem0] += vals[seg + i];
+      for (int i = lo + (int)threadIdx.x; i < hi; i += blockDim.x) {
+        const unsigned li = (unsigned)(idx[seg + i] - t.elem0);
+        if (li < (unsigned)kTile) acc[li] += vals[seg + i];
+      }
       if (lo < hi) __syncthreads();  // lo, hi are uniform over the block
     }
   }
