@@ -53,7 +53,7 @@ constexpr int kSelDense = 0, kSelList = 1, kSelListPred = 2, kSelStaged = 3;
 // segments launch as many blocks as there is work: tiles of segments whose bucket is collected by the collect
 // pass, tiles of dense segments, tiles the select pass must read, tiles served from staged entries.
 constexpr int kListCollect = 0, kListDense = 1, kListSelect = 2, kListStaged = 3, kNumLists = 4;
-constexpr int kListCountWord = 8;  // the lists' lengths live at words 8..11 of the per-step flag block
+constexpr int kListCountWord = 8;  // the lists' lengths live at words 8..11 of the per-step word block
 constexpr int kPredTileCap = 2048;  // keys one tile may hand to a predicted list (more: overflow, fall back)
 
 // Kernels of the library, for per-kernel timing (acc_profile_*).
@@ -115,7 +115,7 @@ struct acc_ctx {
   unsigned* d_hist3 = nullptr;
   acc::Select* d_sel = nullptr;
   unsigned* d_seg_cand = nullptr;    // per (worker, layer): candidate slots handed out this step
-  unsigned* d_any_list = nullptr;    // [0]: some segment needs the collect pass this step; [1]: some is dense; [2]: some needs the select pass
+  unsigned* d_any_list = nullptr;    // per-step word block, cleared with the histograms; words 8..11: lengths of the work lists
   unsigned* d_seg_flag = nullptr;    // per (worker, layer): 1 if pass A's collection overflowed this step
   unsigned* d_pred = nullptr;        // [4][W * n_mat]: prediction word per level, then last threshold bucket per level; kept across steps
   unsigned* d_cand = nullptr;        // candidate keys, [W][cand_total]

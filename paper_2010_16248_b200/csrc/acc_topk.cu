@@ -304,12 +304,9 @@ topk_pick1_kernel(const DevLayer* __restrict__ layers, const int* __restrict__ m
     const bool fits = hs[bin] <= (unsigned)L.cand_cap;
     if (had_band && !overflow && bin >= blo && bin <= bhi) {
       s.mode = was_staged ? kSelStaged : kSelListPred;
-      if (!was_staged) any_list[2] = 1u;  // word 2: some segment still needs the select pass
     } else {
-      any_list[2] = 1u;
       seg_cand[seg] = 0;  // whatever pass A collected is of no use
       s.mode = fits ? kSelList : kSelDense;
-      any_list[fits ? 0 : 1] = 1u;  // word 0: some segment needs the collect pass; word 1: some segment is dense
     }
     // next prediction: narrow the band after an overflow; none for the zero bucket or for buckets that
     // do not fit the list
