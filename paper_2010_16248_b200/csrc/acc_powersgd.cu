@@ -279,7 +279,7 @@ psgd_project_pipe_kernel(const DevLayer* __restrict__ layers, const Tile* __rest
           float4 d = delta_by_copy ? *reinterpret_cast<const float4*>(s_delta + e0)
                                    : *reinterpret_cast<const float4*>(delta + L.offset + t.elem0 + e0);
           d.x += gv.x; d.y += gv.y; d.z += gv.z; d.w += gv.w;
-          *reinterpret_cast<float4*>(delta + L.offset + t.elem0 + e0) = d;
+          st_stream4(delta + L.offset + t.elem0 + e0, d);
         }
       } else {
         const float mm[4] = {mw.x, mw.y, mw.z, mw.w}, gg[4] = {gv.x, gv.y, gv.z, gv.w};
