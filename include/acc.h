@@ -51,7 +51,8 @@ extern "C" {
 #define ACC_MAX_RANK 4    /* ranks are interleaved in groups of ACC_MAX_RANK floats  */
 
 /* acc_config.flags */
-#define ACC_FLAG_LAZY_RESIDUAL 1 /* PowerSGD keeps M_w in err and applies -A on the next load (see acc_powersgd_step) */
+#define ACC_FLAG_LAZY_RESIDUAL 1 /* err keeps M_w after a step; the compressed part is removed on the next load
+                                   (see acc_powersgd_step and acc_topk_step) */
 /* The first PowerSGD pass exists as a direct kernel and as a persistent kernel fed by bulk asynchronous
  * copies; both compute the same values.  By default the library picks by problem size (the pipelined one
  * needs a long queue of tiles per SM to pay off).  These two flags force the choice (tests, tuning). */
@@ -179,9 +180,18 @@ int acc_powersgd_flush(acc_ctx* ctx, float* err, const float* q, const float* p_
  *   out[l] = (1/W) sum_w scatter(idx_w, val_w)  (workers added in order, bit-reproducible).
  *   VECTOR layers: out[l] = mean_w g_w[l], counts = 0.  delta != NULL: delta += g_decider.
  * Device pointers: grads, err, level, out, delta as above; vals [W*capacity] floats,
- * idx [W*capacity] int32, counts [W*L] int32 (see acc_topk_layout).                                */
+ * idx [W*capacity] int32, counts [W*L] int32 (see acc_topk_layout).
+ *
+ * With ACC_FLAG_LAZY_RESIDUAL the kept entries above the threshold are not zeroed in err by the call: err keeps
+ * M_w there, the context remembers the threshold per (worker, layer), and the next acc_topk_step (or
+ * acc_topk_compress) reads every entry of err whose key lies above that threshold as +0.0 while it loads
+ * err -- the same value the eager mode would have stored -- so every later result is bit-identical and the
+ * scattered 4-byte stores into err (a DRAM sector read-modify-write each) are saved.  Kept entries equal to
+ * the threshold are zeroed at once in both modes.  Between steps the caller must leave err untouched;
+ * acc_topk_flush materialises the error memory (ACC_EINVAL without the flag).                         */
 int acc_topk_step(acc_ctx* ctx, const float* grads, float* err, const uint8_t* level, float* vals,
                   int32_t* idx, int32_t* counts, float* out, float* delta, void* stream);
+int acc_topk_flush(acc_ctx* ctx, float* err, void* stream);
 
 /* ---- Optimiser tail (Appendix A, hyper-parameter table: Nesterov momentum 0.9; the paper gives the name
  * and the momentum only, the update below is the usual statement of it, without dampening) -------------

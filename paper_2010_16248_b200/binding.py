@@ -49,7 +49,7 @@ EXPORTS = ["acc_workspace_bytes", "acc_create", "acc_destroy", "acc_factor_layou
            "acc_layer_diff_norms", "acc_detect_regime_diff", "acc_sgd_nesterov", "acc_powersgd_step_sgd",
            "acc_topk_step_sgd", "acc_batch_accumulate", "acc_batch_average", "acc_detect_batch",
            "acc_exchange_layout", "acc_powersgd_phase1", "acc_powersgd_phase2", "acc_powersgd_phase3",
-           "acc_topk_compress", "acc_topk_decompress"]
+           "acc_topk_compress", "acc_topk_decompress", "acc_topk_flush"]
 
 _lib = None
 
@@ -105,6 +105,7 @@ def lib() -> C.CDLL:
     L.acc_powersgd_phase3.argtypes = [vp, vp, vp, vp, vp, vp, vp, f32, vp, vp, vp, vp, vp]
     L.acc_topk_compress.argtypes = [vp] * 10
     L.acc_topk_decompress.argtypes = [vp, vp, vp, vp, i32, vp, f32, vp, vp, vp, vp, vp]
+    L.acc_topk_flush.argtypes = [vp, vp, vp]
     for name in EXPORTS:
         if name not in ("acc_floats_sent", "acc_last_launch_count", "acc_strerror", "acc_profile_kernel_count",
                         "acc_profile_kernel_name"):
@@ -327,6 +328,9 @@ class Context:
                                               _ptr(counts_all, torch.int32), int(n_sets), _ptr(vec_packed, f),
                                               float(vec_scale), _ptr(out, f), _ptr(params, f), _ptr(mom, f),
                                               _ptr(hyper, f), _stream(stream)), "acc_topk_decompress")
+
+    def acc_topk_flush(self, err, stream=None):
+        self._check(lib().acc_topk_flush(self._h, _ptr(err, torch.float32), _stream(stream)), "acc_topk_flush")
 
     def acc_profile_enable(self, enable: bool):
         self._check(lib().acc_profile_enable(self._h, int(bool(enable))), "acc_profile_enable")

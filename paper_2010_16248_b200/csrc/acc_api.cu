@@ -130,6 +130,7 @@ static int make_plan(const acc_config* cfg, Plan& p) {
   p.o_tile_h3 = take(sizeof(unsigned short) * (size_t)W * nt * kBins3);
   p.o_tile_pre = take(sizeof(int2) * (size_t)W * nt);
   p.o_lists = take(sizeof(int2) * (size_t)kNumLists * W * nt);
+  p.o_pend_tau = take(sizeof(unsigned) * seg);
   p.total = o;
   return ACC_OK;
 }
@@ -192,6 +193,7 @@ int acc_create(const acc_config* cfg, void* workspace, size_t workspace_bytes, a
   ctx->d_tile_h3 = reinterpret_cast<unsigned short*>(ws + p.o_tile_h3);
   ctx->d_tile_pre = reinterpret_cast<int2*>(ws + p.o_tile_pre);
   ctx->d_lists = reinterpret_cast<int2*>(ws + p.o_lists);
+  ctx->d_pend_tau = reinterpret_cast<unsigned*>(ws + p.o_pend_tau);
 
   cudaError_t e = cudaSuccess;
   auto up = [&](void* dst, const void* src, size_t bytes) {
@@ -206,6 +208,7 @@ int acc_create(const acc_config* cfg, void* workspace, size_t workspace_bytes, a
   if (e == cudaSuccess) e = cudaMemset(ctx->d_status, 0, sizeof(int) * 64);
   if (e == cudaSuccess) e = cudaMemset(ctx->d_pending, 0, sizeof(int) * cfg->n_layers);
   if (e == cudaSuccess) e = cudaMemset(ctx->d_pred, 0xff, sizeof(unsigned) * 4 * seg);  // no prediction yet
+  if (e == cudaSuccess) e = cudaMemset(ctx->d_pend_tau, 0xff, sizeof(unsigned) * seg);  // nothing pending
   if (e == cudaSuccess) e = prepare_powersgd();
   int dev = 0;
   if (e == cudaSuccess) e = cudaGetDevice(&dev);
@@ -368,6 +371,14 @@ int acc_powersgd_phase3(acc_ctx* ctx, float* err, float* q, const float* p_hat, 
                                        static_cast<cudaStream_t>(stream)));
 }
 
+int acc_topk_flush(acc_ctx* ctx, float* err, void* stream) {
+  if (!ctx || !err) return ACC_EINVAL;
+  if (!(ctx->cfg.flags & ACC_FLAG_LAZY_RESIDUAL)) return ACC_EINVAL;
+  if (!aligned16(err)) return ACC_EALIGN;
+  ctx->last_launches = 0;
+  return finish(launch_topk_flush(ctx, err, static_cast<cudaStream_t>(stream)));
+}
+
 int acc_topk_compress(acc_ctx* ctx, const float* grads, float* err, const uint8_t* level, float* vals, int32_t* idx,
                       int32_t* counts, float* delta, float* vec_packed, void* stream) {
   if (!ctx || !grads || !err || !level || !vals || !idx || !counts) return ACC_EINVAL;
@@ -525,7 +536,7 @@ const char* acc_profile_kernel_name(int32_t i) {
       "topk_hist2_list_kernel", "topk_hist3_list_kernel", "topk_finalize_staged_kernel",
       "psgd_orthonormalise_block_kernel", "sgd_tiles_kernel", "batch_accumulate_kernel", "batch_average_kernel",
       "detect_batch_kernel", "psgd_pfold_kernel", "vec_exchange_kernel", "psgd_qmerge_kernel",
-      "topk_decompress_packed_kernel"};
+      "topk_decompress_packed_kernel", "topk_flush_kernel"};
   return (i >= 0 && i < PH_COUNT) ? names[i] : "";
 }
 

@@ -54,6 +54,7 @@ constexpr int kSelDense = 0, kSelList = 1, kSelListPred = 2, kSelStaged = 3;
 // pass, tiles of dense segments, tiles the select pass must read, tiles served from staged entries.
 constexpr int kListCollect = 0, kListDense = 1, kListSelect = 2, kListStaged = 3, kNumLists = 4;
 constexpr int kListCountWord = 8;  // the lists' lengths live at words 8..11 of the per-step word block
+constexpr unsigned kNoPendingTau = 0xffffffffu;  // no key is larger: nothing pending
 constexpr int kPredTileCap = 2048;  // keys one tile may hand to a predicted list (more: overflow, fall back)
 
 // Kernels of the library, for per-kernel timing (acc_profile_*).
@@ -62,7 +63,7 @@ enum Phase {
   PH_PSGD_PROJECT, PH_PSGD_ORTHO, PH_PSGD_QPARTIAL, PH_PSGD_QREDUCE, PH_PSGD_RESIDUAL,
   PH_TOPK_EF_HIST1, PH_TOPK_PICK1, PH_TOPK_HIST2, PH_TOPK_PICK2, PH_TOPK_HIST3, PH_TOPK_PICK3_SCAN, PH_TOPK_SELECT,
   PH_TOPK_DECOMPRESS, PH_PSGD_FLUSH, PH_TOPK_COLLECT, PH_TOPK_PICK3, PH_TOPK_TILE_COUNTS, PH_TOPK_HIST2_LIST, PH_TOPK_HIST3_LIST, PH_TOPK_FINALIZE_STAGED, PH_PSGD_ORTHO_BLOCK, PH_SGD_TILES, PH_BATCH_ACCUMULATE, PH_BATCH_AVERAGE, PH_DETECT_BATCH,
-  PH_PSGD_PFOLD, PH_VEC_EXCHANGE, PH_PSGD_QMERGE, PH_TOPK_DECOMPRESS_PACKED,
+  PH_PSGD_PFOLD, PH_VEC_EXCHANGE, PH_PSGD_QMERGE, PH_TOPK_DECOMPRESS_PACKED, PH_TOPK_FLUSH,
   PH_COUNT
 };
 
@@ -82,7 +83,7 @@ struct Plan {
   long long vec_floats = 0;  // packed VECTOR elements (each layer starts at a multiple of 4)
   // workspace offsets (bytes)
   size_t o_layers = 0, o_col_items = 0, o_tiles = 0, o_mat_layers = 0, o_vec_tiles = 0, o_mat_tiles = 0, o_status = 0,
-         o_part = 0, o_ppart = 0, o_pending = 0, o_norm_part = 0, o_hist = 0, o_sel = 0, o_pred = 0, o_cand = 0, o_tile_cand = 0, o_tile_cnt = 0, o_tile_h3 = 0, o_tile_pre = 0, o_lists = 0,
+         o_part = 0, o_ppart = 0, o_pending = 0, o_norm_part = 0, o_hist = 0, o_sel = 0, o_pred = 0, o_cand = 0, o_tile_cand = 0, o_tile_cnt = 0, o_tile_h3 = 0, o_tile_pre = 0, o_lists = 0, o_pend_tau = 0,
          hist_bytes = 0, total = 0;
 };
 
@@ -124,6 +125,8 @@ struct acc_ctx {
   unsigned short* d_tile_h3 = nullptr;
   int2* d_tile_pre = nullptr;
   int2* d_lists = nullptr;           // [kNumLists][W * tiles] work lists of (worker, tile)
+  unsigned* d_pend_tau = nullptr;    // lazy TopK: per (worker, layer) threshold of the last step whose kept entries
+                                     // (key > threshold) are still to be zeroed in err; kNoPendingTau: none
 };
 
 namespace acc {
@@ -155,6 +158,7 @@ cudaError_t launch_powersgd_flush(acc_ctx* ctx, float* err, const float* q, cons
 cudaError_t launch_topk(acc_ctx* ctx, const float* grads, float* err, const uint8_t* level, float* vals,
                         int32_t* idx, int32_t* counts, float* out, float* delta, SgdTail tail, cudaStream_t s);
 // Real workers: the TopK step in two halves around the all-gather of the packed sets.
+cudaError_t launch_topk_flush(acc_ctx* ctx, float* err, cudaStream_t s);
 cudaError_t launch_topk_compress(acc_ctx* ctx, const float* grads, float* err, const uint8_t* level, float* vals,
                                  int32_t* idx, int32_t* counts, float* delta, float* vec_packed, cudaStream_t s);
 cudaError_t launch_topk_decompress_packed(acc_ctx* ctx, const float* vals, const int32_t* idx, const int32_t* counts,

@@ -59,7 +59,8 @@ topk_ef_hist1_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict
                      long long stride, int W, int decider, const uint8_t* __restrict__ level,
                      const unsigned* __restrict__ pred, unsigned* __restrict__ hist1,
                      unsigned* __restrict__ seg_cand, unsigned* __restrict__ seg_flag, unsigned* __restrict__ cand,
-                     int2* __restrict__ tile_cand, long long cand_total, int2* __restrict__ tile_cnt) {
+                     int2* __restrict__ tile_cand, long long cand_total, int2* __restrict__ tile_cnt,
+                     const unsigned* __restrict__ pend_tau) {
   __shared__ unsigned h[kBins1];
   // three staging buffers for the collected keys: a tile's keys are copied out while the next tile is
   // being processed and the buffer is reused two tiles later, so one barrier per tile is enough
@@ -76,6 +77,7 @@ topk_ef_hist1_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict
   int cb = 0, pend = -1;  // staging buffer in use; buffer waiting to be copied out
   bool collect = false, staged = false;
   unsigned blo = 1, bhi = 0;
+  unsigned ptau = kNoPendingTau;  // lazy residual: entries of err above this key were kept by the last step
   for (long long v = v0; v < v1; ++v) {
     const int w = (int)(v / n_tiles), ti = (int)(v % n_tiles);
     const Tile t = tiles[ti];
@@ -92,6 +94,7 @@ topk_ef_hist1_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict
       __syncthreads();
       cur = seg;
       collect = pred_band(pred[(level[t.layer] ? 1 : 0) * W * n_mat + seg], &blo, &bhi, &staged);
+      ptau = pend_tau != nullptr ? pend_tau[seg] : kNoPendingTau;
     }
     const long long base = L.offset + t.elem0;
     const float* g = grads + (long long)w * stride + base;
@@ -116,7 +119,13 @@ topk_ef_hist1_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict
       for (int u = 0; u < kBatch; ++u) {
         const int i = i0 + u * kThreads + (int)threadIdx.x;
         if (i >= n4) break;
-        const float4 gv = gb[u], ev = eb[u];
+        const float4 gv = gb[u];
+        float4 ev = eb[u];
+        // lazy residual: what the last step kept (key above its threshold) counts as +0.0
+        ev.x = key_of(ev.x) > ptau ? 0.f : ev.x;
+        ev.y = key_of(ev.y) > ptau ? 0.f : ev.y;
+        ev.z = key_of(ev.z) > ptau ? 0.f : ev.z;
+        ev.w = key_of(ev.w) > ptau ? 0.f : ev.w;
         const float4 m = make_float4(gv.x + ev.x, gv.y + ev.y, gv.z + ev.z, gv.w + ev.w);
         *reinterpret_cast<float4*>(e + 4 * i) = m;
         const unsigned k[4] = {key_of(m.x), key_of(m.y), key_of(m.z), key_of(m.w)};
@@ -159,7 +168,8 @@ topk_ef_hist1_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict
     }
     for (int i = 4 * n4 + threadIdx.x; i < t.nelem; i += blockDim.x) {
       const float gv = g[i];
-      const float m = gv + e[i];
+      const float ev = e[i];
+      const float m = gv + (key_of(ev) > ptau ? 0.f : ev);
       e[i] = m;
       const unsigned kk = key_of(m), bin = kk >> 19;
       atomicAdd(&h[bin], 1u);
@@ -636,7 +646,8 @@ topk_hist_list_kernel(const DevLayer* __restrict__ layers, const int* __restrict
 // One warp per (worker, MATRIX layer): bucket b3 of level 3, hence the threshold tau and the number of ties
 // (key == tau) to keep.  Lane l owns bins 4l..4l+3; a suffix sum over the lanes locates the bin.
 __global__ void __launch_bounds__(256)
-topk_pick3_kernel(int n_seg, const unsigned* __restrict__ hist3, Select* __restrict__ sel) {
+topk_pick3_kernel(int n_seg, const unsigned* __restrict__ hist3, Select* __restrict__ sel,
+                  unsigned* __restrict__ pend_tau) {
   const int seg = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
   if (seg >= n_seg) return;
   const uint4 c4 = *reinterpret_cast<const uint4*>(hist3 + (long long)seg * kBins3 + 4 * lane);
@@ -662,6 +673,7 @@ topk_pick3_kernel(int n_seg, const unsigned* __restrict__ hist3, Select* __restr
     s.tau = (s.b1 << 19) | (s.b2 << 7) | (unsigned)(4 * lane + i);
     s.need = s.k2 - (int)cum;
     sel[seg] = s;
+    if (pend_tau != nullptr) pend_tau[seg] = s.tau;  // lazy residual: keys above tau stay in err until the next load
   }
 }
 
@@ -776,7 +788,9 @@ __device__ __forceinline__ unsigned warp_incl_scan(unsigned c, int lane) {
 // handles float4 j*32+lane of that range for j = 0..7, so (j, lane, element) is index order.  Writes the
 // kept (value, index) pairs at their final positions and zeroes them in err.
 // Per-j lane counts are at most 4 and their warp prefixes at most 128, so four j share one 32-bit scan.
-template <bool FULL>
+// LAZY: entries above the threshold are not zeroed in err (the next first pass, or the flush, treats them as zero);
+// the kept ties are.
+template <bool FULL, bool LAZY>
 __device__ __forceinline__ void select_tile(const Tile& t, const DevLayer& L, const Select& s, const int2 pre,
                                             float* __restrict__ m, float* __restrict__ vals,
                                             int32_t* __restrict__ idx, long long seg, unsigned* wtot) {
@@ -849,7 +863,7 @@ __device__ __forceinline__ void select_tile(const Tile& t, const DevLayer& L, co
           if ((unsigned)pos < (unsigned)s.k) {  // always true for consistent counts; keeps a write inside the segment
             vals[seg + pos] = v[e];
             idx[seg + pos] = t.elem0 + e0 + e;
-            m[e0 + e] = 0.f;
+            if (!LAZY || !is_a) m[e0 + e] = 0.f;
           }
         }
         above_before += is_a;
@@ -861,6 +875,7 @@ __device__ __forceinline__ void select_tile(const Tile& t, const DevLayer& L, co
   }
 }
 
+template <bool LAZY>
 __global__ void __launch_bounds__(256, 3)
 topk_select_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict__ tiles, int n_tiles, int n_mat,
                    float* __restrict__ err, const Select* __restrict__ sel, const int2* __restrict__ tile_pre,
@@ -879,8 +894,8 @@ topk_select_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict__
     const int2 pre = tile_pre[(long long)w * n_tiles + ti];
     float* m = err + (long long)w * stride + L.offset + t.elem0;
     const long long seg = (long long)w * capacity + L.seg_off;
-    if (t.nelem == kTile) select_tile<true>(t, L, s, pre, m, vals, idx, seg, wtot);
-    else select_tile<false>(t, L, s, pre, m, vals, idx, seg, wtot);
+    if (t.nelem == kTile) select_tile<true, LAZY>(t, L, s, pre, m, vals, idx, seg, wtot);
+    else select_tile<false, LAZY>(t, L, s, pre, m, vals, idx, seg, wtot);
   }
 }
 
@@ -889,6 +904,7 @@ topk_select_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict__
 // from them and M is not read.  Index order inside the tile comes from two 8192-bit maps in shared memory
 // (keys above tau, keys equal to tau) with per-word prefix counts: an entry's rank is the number of set bits
 // below its index.
+template <bool LAZY>
 __global__ void __launch_bounds__(256)
 topk_finalize_staged_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict__ tiles, int n_tiles,
                             int n_mat, int W, float* __restrict__ err, const Select* __restrict__ sel,
@@ -975,7 +991,7 @@ topk_finalize_staged_kernel(const DevLayer* __restrict__ layers, const Tile* __r
         if ((unsigned)pos < (unsigned)s.k && li < (unsigned)t.nelem) {  // always true for consistent lists
           vals[seg + pos] = __uint_as_float(e.x);
           idx[seg + pos] = (int32_t)e.y;
-          m[e.y] = 0.f;
+          if (!LAZY || !is_a) m[e.y] = 0.f;
         }
       }
     }
@@ -1164,6 +1180,7 @@ static cudaError_t launch_topk_select_part(acc_ctx* ctx, const float* grads, flo
   const Plan& pl = ctx->plan;
   const acc_config& c = ctx->cfg;
   const int nt = (int)pl.tiles.size(), W = c.n_workers, n_mat = pl.n_mat;
+  const bool lazy = (c.flags & ACC_FLAG_LAZY_RESIDUAL) != 0;
   cudaError_t e = cudaMemsetAsync(ctx->ws + pl.o_hist, 0, pl.hist_bytes, s);
   if (e != cudaSuccess) return e;
   e = cudaMemsetAsync(counts, 0, sizeof(int32_t) * (size_t)W * c.n_layers, s);
@@ -1180,7 +1197,7 @@ static cudaError_t launch_topk_select_part(acc_ctx* ctx, const float* grads, flo
       topk_ef_hist1_kernel<<<grid, 256, 0, s>>>(ctx->d_layers, ctx->d_tiles, nt, n_mat, grads, err, delta,
                                                 c.worker_stride, W, c.decider, level, ctx->d_pred, ctx->d_hist1,
                                                 ctx->d_seg_cand, ctx->d_seg_flag, ctx->d_cand, ctx->d_tile_cand,
-                                                pl.cand_total, ctx->d_tile_cnt);
+                                                pl.cand_total, ctx->d_tile_cnt, lazy ? ctx->d_pend_tau : nullptr);
     }
     {
       PhaseTimer pt(ctx, PH_TOPK_PICK1, s);
@@ -1225,7 +1242,8 @@ static cudaError_t launch_topk_select_part(acc_ctx* ctx, const float* grads, flo
     }
     {
       PhaseTimer pt(ctx, PH_TOPK_PICK3, s);
-      topk_pick3_kernel<<<(W * n_mat + 7) / 8, 256, 0, s>>>(W * n_mat, ctx->d_hist3, ctx->d_sel);
+      topk_pick3_kernel<<<(W * n_mat + 7) / 8, 256, 0, s>>>(W * n_mat, ctx->d_hist3, ctx->d_sel,
+                                                            lazy ? ctx->d_pend_tau : nullptr);
     }
     {
       PhaseTimer pt(ctx, PH_TOPK_TILE_COUNTS, s);
@@ -1243,15 +1261,27 @@ static cudaError_t launch_topk_select_part(acc_ctx* ctx, const float* grads, flo
     {
       PhaseTimer pt(ctx, PH_TOPK_FINALIZE_STAGED, s);
       const long long warps = (long long)W * nt, cap = (long long)ctx->sm_count * 32;
-      topk_finalize_staged_kernel<<<(unsigned)std::min((warps + 7) / 8, cap), 256, 0, s>>>(
-          ctx->d_layers, ctx->d_tiles, nt, n_mat, W, err, ctx->d_sel, ctx->d_tile_pre, ctx->d_cand, ctx->d_tile_cand,
-          pl.cand_total, vals, idx, c.worker_stride, pl.capacity, ctx->d_any_list, ctx->d_lists);
+      const unsigned fgrid = (unsigned)std::min((warps + 7) / 8, cap);
+      if (lazy)
+        topk_finalize_staged_kernel<true><<<fgrid, 256, 0, s>>>(
+            ctx->d_layers, ctx->d_tiles, nt, n_mat, W, err, ctx->d_sel, ctx->d_tile_pre, ctx->d_cand,
+            ctx->d_tile_cand, pl.cand_total, vals, idx, c.worker_stride, pl.capacity, ctx->d_any_list, ctx->d_lists);
+      else
+        topk_finalize_staged_kernel<false><<<fgrid, 256, 0, s>>>(
+            ctx->d_layers, ctx->d_tiles, nt, n_mat, W, err, ctx->d_sel, ctx->d_tile_pre, ctx->d_cand,
+            ctx->d_tile_cand, pl.cand_total, vals, idx, c.worker_stride, pl.capacity, ctx->d_any_list, ctx->d_lists);
     }
     PhaseTimer pt(ctx, PH_TOPK_SELECT, s);
     const long long blocks = (long long)W * nt, cap = (long long)ctx->sm_count * 12;
-    topk_select_kernel<<<(unsigned)std::min(blocks, cap), 256, 0, s>>>(
-        ctx->d_layers, ctx->d_tiles, nt, n_mat, err, ctx->d_sel, ctx->d_tile_pre, ctx->d_any_list, vals, idx,
-        c.worker_stride, pl.capacity, ctx->d_lists, W);
+    const unsigned sgrid = (unsigned)std::min(blocks, cap);
+    if (lazy)
+      topk_select_kernel<true><<<sgrid, 256, 0, s>>>(ctx->d_layers, ctx->d_tiles, nt, n_mat, err, ctx->d_sel,
+                                                     ctx->d_tile_pre, ctx->d_any_list, vals, idx, c.worker_stride,
+                                                     pl.capacity, ctx->d_lists, W);
+    else
+      topk_select_kernel<false><<<sgrid, 256, 0, s>>>(ctx->d_layers, ctx->d_tiles, nt, n_mat, err, ctx->d_sel,
+                                                      ctx->d_tile_pre, ctx->d_any_list, vals, idx, c.worker_stride,
+                                                      pl.capacity, ctx->d_lists, W);
   }
   return cudaGetLastError();
 }
@@ -1274,6 +1304,55 @@ cudaError_t launch_topk(acc_ctx* ctx, const float* grads, float* err, const uint
       topk_decompress_kernel<false><<<nt, 256, 0, s>>>(ctx->d_layers, ctx->d_tiles, nt, n_mat, grads, ctx->d_sel,
                                                        ctx->d_tile_pre, vals, idx, out, delta, c.worker_stride,
                                                        pl.capacity, W, c.decider, inv_w, tail);
+  }
+  return cudaGetLastError();
+}
+
+// Lazy mode: err_w <- err_w with the entries the last step kept (key above the segment's pending threshold) set to
+// +0.0; afterwards nothing is pending.  One block per (tile, worker).
+__global__ void __launch_bounds__(256)
+topk_flush_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict__ tiles, int n_mat,
+                  float* __restrict__ err, long long stride, const unsigned* __restrict__ pend_tau) {
+  const Tile t = tiles[blockIdx.x];
+  const int w = blockIdx.y;
+  const DevLayer L = layers[t.layer];
+  if (L.kind != ACC_MATRIX) return;
+  const unsigned ptau = pend_tau[w * n_mat + L.mat];
+  if (ptau == kNoPendingTau) return;
+  float* e = err + (long long)w * stride + L.offset + t.elem0;
+  const int n4 = t.nelem >> 2;
+  for (int i = threadIdx.x; i < n4; i += blockDim.x) {
+    float4 v = ld_stream4(e + 4 * i);
+    const bool any = key_of(v.x) > ptau || key_of(v.y) > ptau || key_of(v.z) > ptau || key_of(v.w) > ptau;
+    if (any) {
+      v.x = key_of(v.x) > ptau ? 0.f : v.x;
+      v.y = key_of(v.y) > ptau ? 0.f : v.y;
+      v.z = key_of(v.z) > ptau ? 0.f : v.z;
+      v.w = key_of(v.w) > ptau ? 0.f : v.w;
+      *reinterpret_cast<float4*>(e + 4 * i) = v;
+    }
+  }
+  for (int i = 4 * n4 + threadIdx.x; i < t.nelem; i += blockDim.x)
+    if (key_of(e[i]) > ptau) e[i] = 0.f;
+}
+
+__global__ void topk_clear_pending_kernel(unsigned* __restrict__ pend_tau, int n) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) pend_tau[i] = kNoPendingTau;
+}
+
+cudaError_t launch_topk_flush(acc_ctx* ctx, float* err, cudaStream_t s) {
+  const Plan& pl = ctx->plan;
+  const acc_config& c = ctx->cfg;
+  if (pl.n_mat > 0) {
+    {
+      PhaseTimer pt(ctx, PH_TOPK_FLUSH, s);
+      topk_flush_kernel<<<dim3((unsigned)pl.tiles.size(), (unsigned)c.n_workers), 256, 0, s>>>(
+          ctx->d_layers, ctx->d_tiles, pl.n_mat, err, c.worker_stride, ctx->d_pend_tau);
+    }
+    const int n = c.n_workers * pl.n_mat;
+    ctx->last_launches += 1;
+    topk_clear_pending_kernel<<<(n + 127) / 128, 128, 0, s>>>(ctx->d_pend_tau, n);
   }
   return cudaGetLastError();
 }

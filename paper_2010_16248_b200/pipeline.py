@@ -45,6 +45,7 @@ class AccordionStep:
         self.norm2_prev = torch.full((L,), -1.0, dtype=torch.float64, device=dev)
         self.t = 0
         self.launches = 0
+        self.lazy_residual = lazy_residual
         self.overlap = overlap
         self._side = torch.cuda.Stream(device=dev)
         self._fork, self._join = torch.cuda.Event(), torch.cuda.Event()
@@ -109,6 +110,16 @@ class AccordionStep:
             self.launches += c.last_launch_count()
             c.acc_detect_regime(self.norm2_curr, self.norm2_prev, lr_curr, lr_next, self.level, self.delta, stream)
             self.launches += c.last_launch_count()
+
+    def flush(self, stream=None):
+        """Lazy mode: materialises the error memories (what the last step compressed is removed from ``err``), so
+        that the state buffers can be read, saved or copied into another engine.  A no-op in eager mode."""
+        if not self.lazy_residual:
+            return
+        if "powersgd" in self.compressors:
+            self.ctx.acc_powersgd_flush(self.err_psgd, self.q, self.p_hat, stream)
+        if "topk" in self.compressors:
+            self.ctx.acc_topk_flush(self.err_topk, stream)
 
     def set_lr(self, lr: float):
         """Learning rate of the optimiser tail: a device scalar the kernels read, so captured graphs follow it."""

@@ -41,15 +41,15 @@ def _run_config(w, iters, t0=0, lazy=False, topk_layers=None, topk_workers=None,
     """Runs `iters` iterations of workload `w` starting at stream iteration t0; checks every TopK step and
     every level decision exactly, and the PowerSGD steps listed in psgd_check (default: all).  With
     lazy=True a second engine in lazy-residual mode (the mode bench.py times) runs in lockstep and must
-    reproduce the eager engine's out, Q and P^ bit for bit at every step, and its error memory after a
-    final flush."""
+    reproduce the eager engine's outputs (out, Q, P^; packed TopK sets) bit for bit at every step, and its error
+    memories after a final flush."""
     table, W = w.table, w.n_workers
     stream = wl.GradientStream(w, device="cuda")
     eng = pipeline.AccordionStep(table, W, w.compressors, w.rank_low, w.rank_high, w.topk_low_bp, w.topk_high_bp,
                                  w.eta, 1e-8, w.check_every)
     lz = None
-    if lazy and "powersgd" in w.compressors:
-        lz = pipeline.AccordionStep(table, W, ("powersgd",), w.rank_low, w.rank_high, w.topk_low_bp, w.topk_high_bp,
+    if lazy:
+        lz = pipeline.AccordionStep(table, W, w.compressors, w.rank_low, w.rank_high, w.topk_low_bp, w.topk_high_bp,
                                     w.eta, 1e-8, w.check_every, lazy_residual=True)
     ctl = OracleController(table, w.check_every, w.eta)
     seen_levels = set()
@@ -68,7 +68,9 @@ def _run_config(w, iters, t0=0, lazy=False, topk_layers=None, topk_workers=None,
         torch.cuda.synchronize()
         if lz is not None:
             assert torch.equal(lz.level, eng.level)
-            for name in ("out_psgd", "q", "p_hat"):
+            names = (("out_psgd", "q", "p_hat") if "powersgd" in w.compressors else ()) + \
+                    (("out_topk", "vals", "idx", "counts") if "topk" in w.compressors else ())
+            for name in names:
                 assert torch.equal(getattr(lz, name), getattr(eng, name)), f"iteration {i}: lazy {name} differs"
         if "powersgd" in w.compressors and (psgd_check is None or i in psgd_check):
             H.check_powersgd_against_oracle(eng.ctx, table, grads, e0, q0, level_before, eng.out_psgd, eng.err_psgd,
@@ -79,9 +81,11 @@ def _run_config(w, iters, t0=0, lazy=False, topk_layers=None, topk_workers=None,
                                         layers_subset=topk_layers, workers_subset=topk_workers)
         ctl.step(grads[0].cpu().numpy())
     if lz is not None:
-        lz.ctx.acc_powersgd_flush(lz.err_psgd, lz.q, lz.p_hat)
+        lz.flush()
         torch.cuda.synchronize()
-        assert torch.equal(lz.err_psgd, eng.err_psgd), "flushed lazy error memory differs from the eager one"
+        for name in (("err_psgd",) if "powersgd" in w.compressors else ()) + \
+                (("err_topk",) if "topk" in w.compressors else ()):
+            assert torch.equal(getattr(lz, name), getattr(eng, name)), f"flushed lazy {name} differs from the eager one"
     return seen_levels
 
 
@@ -123,8 +127,9 @@ def test_reduced_configs_across_scale_jump(config, scale):
     assert seen == {0, 1}, "both compression levels must have been exercised"
 
 
-def test_reduced_config2_lazy_residual():
-    w = wl.workload(2, scale=4)
+@pytest.mark.parametrize("config,scale", [(2, 4), (3, 4), (5, 16)])
+def test_reduced_configs_lazy_residual(config, scale):
+    w = wl.workload(config, scale=scale)
     _run_config(w, iters=25, t0=90, lazy=True, psgd_check=set(range(25)))
 
 
@@ -142,7 +147,7 @@ def test_full_size_config3_topk():
     _run_config(w, iters=2, t0=0, topk_workers=[0])
     sizes = w.table.sizes
     sample = [big[0], int(np.argmax(sizes)), big[-1]]
-    _run_config(w, iters=2, t0=0, topk_layers=sample)
+    _run_config(w, iters=3, t0=0, lazy=True, topk_layers=sample)
 
 
 def test_full_size_config5_sampled():

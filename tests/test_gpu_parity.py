@@ -444,7 +444,7 @@ def test_difference_criterion_variant_matches_oracle():
 def test_checkpoint_resume_is_bit_identical():
     """State of the path = caller buffers (error memories, Q, P^, accumulator, norms, levels).  Running 2k
     iterations must equal k iterations + copying the state into a new context + k iterations.  In lazy mode
-    the residual pending inside the context is materialised with acc_powersgd_flush before the copy."""
+    what is pending inside the context is materialised (acc_powersgd_flush, acc_topk_flush) before the copy."""
     w = wl.workload(5, scale=16)
     table, W = w.table, w.n_workers
     stream = wl.GradientStream(w, device="cuda")
@@ -461,7 +461,7 @@ def test_checkpoint_resume_is_bit_identical():
     first = engine()
     for t in range(k):
         first.step(stream.grads(t))
-    first.ctx.acc_powersgd_flush(first.err_psgd, first.q, first.p_hat)
+    first.flush()
     torch.cuda.synchronize()
     second = engine()
     for n in names:
@@ -469,8 +469,8 @@ def test_checkpoint_resume_is_bit_identical():
     second.t = first.t
     for t in range(k, 2 * k):
         second.step(stream.grads(t))
-    full.ctx.acc_powersgd_flush(full.err_psgd, full.q, full.p_hat)
-    second.ctx.acc_powersgd_flush(second.err_psgd, second.q, second.p_hat)
+    full.flush()
+    second.flush()
     torch.cuda.synchronize()
     for n in names:
         assert torch.equal(getattr(full, n), getattr(second, n)), n
@@ -527,3 +527,44 @@ def test_topk_whole_model_selection_scope():
         if l % 4 == 0:
             big[sl] = True
     assert big[kept].mean() > 0.9
+
+
+@pytest.mark.parametrize("pipeline_flag", [binding.ACC_FLAG_PIPELINE_NEVER, binding.ACC_FLAG_PIPELINE_ALWAYS])
+def test_topk_lazy_residual_is_bit_identical_to_eager(pipeline_flag):
+    """Lazy mode leaves the kept entries above the threshold in err and reads them as +0.0 on the next load: packed
+    sets, outputs and -- after a flush -- the error memory are the eager mode's bits, through level switches,
+    exact ties at the threshold, zero-filled selections and every selection path."""
+    table = _table_mixed()
+    W = 3
+    eager = binding.Context(table, W, topk_low_bp=1000, topk_high_bp=100, flags=pipeline_flag)
+    lazy = binding.Context(table, W, topk_low_bp=1000, topk_high_bp=100,
+                           flags=pipeline_flag | binding.ACC_FLAG_LAZY_RESIDUAL)
+    _, err_e = _random_inputs(table, W, 5)
+    err_l = err_e.clone()
+    ve, ie, ce = eager.new_topk_buffers()
+    vl, il, cl = lazy.new_topk_buffers()
+    out_e, out_l = torch.zeros(table.stride, device="cuda"), torch.zeros(table.stride, device="cuda")
+    d_e, d_l = torch.zeros(table.stride, device="cuda"), torch.zeros(table.stride, device="cuda")
+    base, _ = _random_inputs(table, W, 1400)
+    for it in range(10):
+        level = torch.tensor([(l + it // 3) % 2 for l in range(table.n_layers)], dtype=torch.uint8, device="cuda")
+        noise, _ = _random_inputs(table, W, 1401 + it)
+        grads = base + 0.05 * noise  # similar steps: the threshold predictions hold, staged and list paths run
+        if it == 4:  # exact ties at and around the threshold; a worker with an all-zero gradient
+            grads = torch.round(grads * 4.0) / 4.0
+            grads[1].zero_()
+        eager.acc_topk_step(grads, err_e, level, ve, ie, ce, out_e, d_e)
+        lazy.acc_topk_step(grads, err_l, level, vl, il, cl, out_l, d_l)
+        torch.cuda.synchronize()
+        assert torch.equal(ie, il) and torch.equal(ce, cl) and torch.equal(out_e, out_l) and torch.equal(d_e, d_l), it
+        assert torch.equal(ve.view(torch.int32), vl.view(torch.int32)), it
+        if it in (2, 6):  # a flush in the middle changes nothing downstream
+            lazy.acc_topk_flush(err_l)
+            torch.cuda.synchronize()
+            assert torch.equal(err_e.view(torch.int32), err_l.view(torch.int32)), it
+    assert not torch.equal(err_e, err_l)  # something is pending: the modes differ in memory before the flush
+    lazy.acc_topk_flush(err_l)
+    torch.cuda.synchronize()
+    assert torch.equal(err_e.view(torch.int32), err_l.view(torch.int32))
+    with pytest.raises(binding.AccError):
+        eager.acc_topk_flush(err_e)
