@@ -18,7 +18,9 @@
  *   * Calls are asynchronous on `stream` (a cudaStream_t passed as void*; NULL = default stream),
  *     never synchronise the device, and return an int status: ACC_OK or one of the ACC_E* codes.
  *     Calls on one context must be ordered on one stream (or otherwise serialised by the caller):
- *     they share the context's scratch memory.
+ *     they share the context's scratch memory.  One exception: the PowerSGD calls and the TopK calls use
+ *     disjoint parts of it, so a PowerSGD step and a TopK step of the same iteration (different error
+ *     memories and outputs, the same gradients and levels) may run concurrently on two streams.
  *   * Layout.  All per-parameter buffers use one flat per-worker layout given by the layer table:
  *     layer l occupies elements [offset_l, offset_l + rows_l*cols_l) of each worker's slice, each
  *     offset a multiple of 4 elements; worker w's slice starts at element w*worker_stride
