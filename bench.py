@@ -92,20 +92,22 @@ class ClockSampler:
                 "reasons": sorted(reasons)}
 
 
-def _kernel_alg_bytes(name, units):
-    """Algorithmic bytes one launch of a streaming kernel must move, per MATRIX parameter-worker
-    (fp32): reads + writes that the method itself requires of that pass."""
+def _kernel_alg_bytes(name, units, n_workers=None, carries_delta=()):
+    """Algorithmic bytes one launch of a streaming kernel must move (fp32), for `units` MATRIX parameter-workers:
+    the reads and writes the method itself requires of that pass.  The first pass of a compressor reads g and e and
+    writes M (12 B per unit); the one that also accumulates the detector's gradient (the first compressor of the
+    step) reads and writes delta for one worker in W (8/W B per unit more).  The selection passes work on the
+    subsets their work lists name, so no per-launch figure is given for them."""
     per_unit = {
         "psgd_project_kernel": 12.0,    # read g, read e, write M
         "psgd_residual_kernel": 8.0,    # read M, write e' (eager mode; in lazy mode it only writes out)
         "topk_ef_hist1_kernel": 12.0,   # read g, read e, write M
-        "topk_collect_kernel": 4.0,     # read M
-        "topk_hist2_kernel": 4.0,       # read M (dense path only)
-        "topk_hist3_kernel": 4.0,       # read M
-        "topk_select_kernel": 4.0,      # read M (+ sparse writes, not counted)
         "ef_kernel": 12.0,
     }
-    return per_unit.get(name, 0.0) * units
+    b = per_unit.get(name, 0.0)
+    if b and name in carries_delta and n_workers:
+        b += 8.0 / n_workers
+    return b * units
 
 
 def run_reference(args, rank, world):
@@ -318,20 +320,26 @@ def main():
     units = W * n_mat
     total_k_ms = sum(ms for ms, _ in prof.values())
     kernels = {}
+    # the first compressor of the step carries the detector's accumulation in its first pass
+    carries = ("psgd_project_kernel",) if "powersgd" in w.compressors else ("topk_ef_hist1_kernel",)
     for name, (ms, cnt) in sorted(prof.items(), key=lambda kv: -kv[1][0]):
         alg = _kernel_alg_bytes(name, units)
+        if name == "psgd_residual_kernel" and not args.eager:
+            alg = 0.0  # lazy mode: this slot times the decompress kernel, which only writes out (4/W B per unit)
         avg = ms / cnt
         kernels[name] = {"launches": cnt, "ms_total": round(ms, 4), "share": round(ms / total_k_ms, 4),
                          "avg_ms": round(avg, 5),
                          "alg_gbs": round(alg / (avg * 1e-3) / 1e9, 1) if alg else None}
     dom = next(iter(kernels))
-    dom_alg = _kernel_alg_bytes(dom, units)
+    dom_alg = _kernel_alg_bytes(dom, units)  # 12 B per unit: the fraction is reported against the compulsory bytes
+    dom_alg_delta = _kernel_alg_bytes(dom, units, W, carries)  # ... and with the detector's accumulation counted
     dom_avg_ms = prof[dom][0] / prof[dom][1]
     achieved = dom_alg / (dom_avg_ms * 1e-3) / 1e9
     roofline = {"bound": "hbm", "kernel": dom, "achieved": round(achieved, 1), "peak": peak, "unit": "GB/s",
                 "frac": round(achieved / peak, 4), "peak_source": peak_src, "traffic": (TRAFFIC_PER_UNIT[dom] * units if dom in TRAFFIC_PER_UNIT else None),
                 "traffic_source": TRAFFIC_SOURCE.get(dom),
-                "alg_bytes_per_launch": dom_alg,
+                "alg_bytes_per_launch": dom_alg, "alg_bytes_per_unit": round(dom_alg / units, 3),
+                "frac_with_detector_bytes": round(dom_alg_delta / (dom_avg_ms * 1e-3) / 1e9 / peak, 4),
                 "step_frac_of_12B": round(n_comp * 12.0 * units / (ms_per_step * 1e-3) / 1e9 / peak, 4)}
 
     # ---- end to end: host (pinned) gradients -> device every step, results read back to the host.
