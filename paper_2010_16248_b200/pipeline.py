@@ -234,6 +234,7 @@ class DistributedStep:
         self.table, self.n_local, self.compressor = table, n_local, compressor
         self.x = exchange if exchange is not None else dist_util.Exchange()
         self.world, self.rank = self.x.world, self.x.rank
+        self.lazy_residual = lazy_residual
         self.check_every = check_every
         self.device = dev = torch.device(device)
         self.owns_decider = decider // n_local == self.rank
@@ -269,6 +270,15 @@ class DistributedStep:
             self.counts_all = torch.zeros(w * self.counts.numel(), dtype=torch.int32, device=dev)
         else:
             raise ValueError(compressor)
+
+    def flush(self, stream=None):
+        """Lazy mode: materialises this rank's error memories (see ``AccordionStep.flush``)."""
+        if not self.lazy_residual:
+            return
+        if self.compressor == "powersgd":
+            self.ctx.acc_powersgd_flush(self.err, self.q, self.p_hat, stream)
+        else:
+            self.ctx.acc_topk_flush(self.err, stream)
 
     def bytes_exchanged_per_step(self) -> int:
         """Bytes this rank hands to the collectives in one step (the method's communication volume)."""

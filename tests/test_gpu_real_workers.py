@@ -118,10 +118,9 @@ def test_powersgd_two_ranks_match_oracle_over_all_workers(lazy):
             level, prev = orc.detect_regime(orc.layer_norms2(delta, layers), prev, 0.1, 0.1, 0.5)
             delta[:] = 0.0
     assert np.array_equal(a.level.cpu().numpy(), level)
-    if lazy:
-        for st in steps:
-            st.ctx.acc_powersgd_flush(st.err, st.q, st.p_hat)
-        torch.cuda.synchronize()
+    for st in steps:
+        st.flush()  # lazy mode: materialise the error memories (a no-op in eager mode)
+    torch.cuda.synchronize()
     err_gpu = torch.cat([a.err, b.err]).cpu().numpy()
     out_h, x_h = a.out.cpu().numpy(), params[0].cpu().numpy()
     tol = 5e-4  # four chained steps in fp32 against fp64 (one step: 1e-4)
@@ -243,3 +242,23 @@ def test_degenerate_tables_two_ranks(shapes, compressor):
     for l, sl in table.slices():
         got, want = steps[0].out[sl].cpu().numpy(), ref[sl].cpu().numpy()
         assert H.rel_err(got, want, 1e-7 * np.linalg.norm(want) + 1e-12) <= 1e-4, (l, compressor)
+
+
+def test_topk_two_ranks_lazy_residual_equals_eager():
+    table = _table_mixed()
+    world, n_local, n_iters = 2, 2, 4
+    batches = [_random_inputs(table, world * n_local, 1500 + it)[0] for it in range(n_iters)]
+    results = []
+    for lazy in (False, True):
+        def make_step(exchange, lazy=lazy):
+            return pipeline.DistributedStep(table, n_local, "topk", check_every=2, decider=1, lazy_residual=lazy,
+                                            exchange=exchange)
+        steps = _run_ranks(world, make_step, n_iters,
+                           lambda it, r: batches[it][r * n_local:(r + 1) * n_local].contiguous())
+        for st in steps:
+            st.flush()
+        torch.cuda.synchronize()
+        results.append(steps)
+    for a, b in zip(*results):
+        for name in ("out", "err", "vals_all", "idx_all", "counts_all", "level"):
+            assert torch.equal(getattr(a, name), getattr(b, name)), name
