@@ -78,11 +78,21 @@ topk_ef_hist1_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict
   bool collect = false, staged = false;
   unsigned blo = 1, bhi = 0;
   unsigned ptau = kNoPendingTau;  // lazy residual: entries of err above this key were kept by the last step
+  // the layer record is kept while the tiles stay inside the layer (a tile's extent follows from its index), so
+  // that a tile does not start with a chain of dependent loads
+  DevLayer L;
+  int cur_layer = -1;
   for (long long v = v0; v < v1; ++v) {
     const int w = (int)(v / n_tiles), ti = (int)(v % n_tiles);
-    const Tile t = tiles[ti];
-    const DevLayer L = layers[t.layer];
+    if (cur_layer < 0 || ti < L.tile0 || ti >= L.tile0 + L.ntiles) {
+      cur_layer = tiles[ti].layer;
+      L = layers[cur_layer];
+    }
     if (L.kind != ACC_MATRIX) continue;
+    Tile t;
+    t.layer = cur_layer;
+    t.elem0 = (ti - L.tile0) * kTile;
+    t.nelem = (int)min((long long)kTile, (long long)L.rows * L.cols - t.elem0);
     const int seg = w * n_mat + L.mat;
     if (seg != cur) {
       __syncthreads();
@@ -114,6 +124,14 @@ topk_ef_hist1_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict
       for (int u = 0; u < kBatch; ++u) {
         const int i = i0 + u * kThreads + (int)threadIdx.x;
         if (i < n4) { gb[u] = ld_stream4(g + 4 * i); eb[u] = ld_stream4(e + 4 * i); }
+      }
+      // the next batch's lines are asked into L2 meanwhile (one request per 128-byte line)
+      if ((threadIdx.x & 7) == 0) {
+#pragma unroll
+        for (int u = 0; u < kBatch; ++u) {
+          const int i = i0 + (kBatch + u) * kThreads + (int)threadIdx.x;
+          if (i < n4) { prefetch_l2(g + 4 * i); prefetch_l2(e + 4 * i); }
+        }
       }
 #pragma unroll
       for (int u = 0; u < kBatch; ++u) {
