@@ -226,17 +226,27 @@ psgd_project_pipe_kernel(const DevLayer* __restrict__ layers, const Tile* __rest
   };
   if (threadIdx.x == 0)
     for (int it = 0; it < kPipeStages && it < n_stages; ++it) issue(it);
-  Tile t = tiles[mat_tiles[t0]];
+  int gt = mat_tiles[t0];  // the tile's index among all tiles
+  Tile t = tiles[gt];
   DevLayer L = layers[t.layer];
   float4 corr[kPipePos], mb[kPipePos];
-  int rp = 0;
+  int rp = LAZY ? pending[t.layer] : 0;
   for (int it = 0; it < n_stages; ++it) {
     const int ti = it / W, w = it - ti * W;
     const int buf = it % kPipeStages;
     if (w == 0) {  // new tile: factors of the pending residual at this thread's positions
-      t = tiles[mat_tiles[t0 + ti]];
-      L = layers[t.layer];
-      rp = LAZY ? pending[t.layer] : 0;
+      if (ti > 0) {
+        if (gt + 1 < L.tile0 + L.ntiles) {  // next tile of the same layer: no table look-ups
+          gt += 1;
+          t.elem0 += kTile;
+          t.nelem = (int)min((long long)kTile, (long long)L.rows * L.cols - t.elem0);
+        } else {
+          gt = mat_tiles[t0 + ti];
+          t = tiles[gt];
+          L = layers[t.layer];
+          rp = LAZY ? pending[t.layer] : 0;
+        }
+      }
       const float4* Q4 = reinterpret_cast<const float4*>(q) + L.q_row;
       const float4* P4 = reinterpret_cast<const float4*>(p) + L.p_row;
 #pragma unroll
