@@ -607,25 +607,46 @@ __device__ __forceinline__ void decompress_cols(const ColItem& it, const DevLaye
   const long long first = L.offset + (long long)it.row0 * L.cols + col;
   float* base = out + first;
   const float4* pr = P4 + it.row0;
-  SgdHyper h = {0.f, 0.f, 0.f};
-  if (SGD) h = sgd_hyper(tail);
+  if (!SGD) {
 #pragma unroll 8
-  for (int i = 0; i < it.nrows; ++i) {
-    const float4 pv = __ldg(pr + i);
-    float a[VEC];
+    for (int i = 0; i < it.nrows; ++i) {
+      const float4 pv = __ldg(pr + i);
+      float a[VEC];
 #pragma unroll
-    for (int e = 0; e < VEC; ++e) a[e] = lowrank_entry(pv, qv[e], r);
-    __stcs(reinterpret_cast<V*>(base + (long long)i * L.cols), *reinterpret_cast<const V*>(a));
-    if (SGD) {
-      const long long at = first + (long long)i * L.cols;
-      V xv = *reinterpret_cast<const V*>(tail.params + at), uv = *reinterpret_cast<const V*>(tail.mom + at);
-      float* x = reinterpret_cast<float*>(&xv);
-      float* u = reinterpret_cast<float*>(&uv);
-#pragma unroll
-      for (int e = 0; e < VEC; ++e) sgd_update(a[e], x[e], u[e], h);
-      *reinterpret_cast<V*>(tail.params + at) = xv;
-      *reinterpret_cast<V*>(tail.mom + at) = uv;
+      for (int e = 0; e < VEC; ++e) a[e] = lowrank_entry(pv, qv[e], r);
+      __stcs(reinterpret_cast<V*>(base + (long long)i * L.cols), *reinterpret_cast<const V*>(a));
     }
+    return;
+  }
+  // with the optimiser tail: rows in groups of kRows, the parameters and momenta of a group loaded before the
+  // group's first store (a store in between would hold the later loads back)
+  const SgdHyper h = sgd_hyper(tail);
+  constexpr int kRows = 4;
+  for (int i0 = 0; i0 < it.nrows; i0 += kRows) {
+    V xv[kRows], uv[kRows];
+#pragma unroll
+    for (int k = 0; k < kRows; ++k)
+      if (i0 + k < it.nrows) {
+        const long long at = first + (long long)(i0 + k) * L.cols;
+        xv[k] = *reinterpret_cast<const V*>(tail.params + at);
+        uv[k] = *reinterpret_cast<const V*>(tail.mom + at);
+      }
+#pragma unroll
+    for (int k = 0; k < kRows; ++k)
+      if (i0 + k < it.nrows) {
+        const long long at = first + (long long)(i0 + k) * L.cols;
+        const float4 pv = __ldg(pr + i0 + k);
+        float a[VEC];
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) a[e] = lowrank_entry(pv, qv[e], r);
+        __stcs(reinterpret_cast<V*>(out + at), *reinterpret_cast<const V*>(a));
+        float* x = reinterpret_cast<float*>(&xv[k]);
+        float* u = reinterpret_cast<float*>(&uv[k]);
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) sgd_update(a[e], x[e], u[e], h);
+        *reinterpret_cast<V*>(tail.params + at) = xv[k];
+        *reinterpret_cast<V*>(tail.mom + at) = uv[k];
+      }
   }
 }
 
@@ -744,8 +765,30 @@ sgd_tiles_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict__ t
   const long long base = L.offset + t.elem0;
   const SgdHyper h = sgd_hyper(tail);
   const int n4 = t.nelem >> 2;
-  for (int f = threadIdx.x; f < n4; f += blockDim.x)
-    sgd_apply4(tail, h, base + 4 * f, ld_stream4(d + base + 4 * f));
+  // four float4 per thread at a time: all loads of a group before its first store
+  constexpr int kGroup = 4, kThreads = 256;
+  for (int f0 = 0; f0 < n4; f0 += kGroup * kThreads) {
+    float4 dv[kGroup], xv[kGroup], uv[kGroup];
+#pragma unroll
+    for (int k = 0; k < kGroup; ++k) {
+      const int f = f0 + k * kThreads + (int)threadIdx.x;
+      if (f < n4) {
+        dv[k] = ld_stream4(d + base + 4 * f);
+        xv[k] = *reinterpret_cast<const float4*>(tail.params + base + 4 * f);
+        uv[k] = *reinterpret_cast<const float4*>(tail.mom + base + 4 * f);
+      }
+    }
+#pragma unroll
+    for (int k = 0; k < kGroup; ++k) {
+      const int f = f0 + k * kThreads + (int)threadIdx.x;
+      if (f < n4) {
+        sgd_update(dv[k].x, xv[k].x, uv[k].x, h); sgd_update(dv[k].y, xv[k].y, uv[k].y, h);
+        sgd_update(dv[k].z, xv[k].z, uv[k].z, h); sgd_update(dv[k].w, xv[k].w, uv[k].w, h);
+        *reinterpret_cast<float4*>(tail.params + base + 4 * f) = xv[k];
+        *reinterpret_cast<float4*>(tail.mom + base + 4 * f) = uv[k];
+      }
+    }
+  }
   for (int i = 4 * n4 + threadIdx.x; i < t.nelem; i += blockDim.x) sgd_apply1(tail, h, base + i, d[base + i]);
 }
 
