@@ -18,16 +18,30 @@ __global__ void __launch_bounds__(256) ef_kernel(const DevLayer* __restrict__ la
   float* e = err + (long long)w * stride + base;
   float* d = delta + base;
   const int n4 = t.nelem >> 2;
-  for (int i = threadIdx.x; i < n4; i += blockDim.x) {
-    const float4 gv = ld_stream4(g + 4 * i);
-    if (is_mat) {
-      const float4 ev = ld_stream4(e + 4 * i);
-      st_stream4(e + 4 * i, make_float4(gv.x + ev.x, gv.y + ev.y, gv.z + ev.z, gv.w + ev.w));
+  // four float4 per thread at a time: all loads of a group before its first store, so that they are in flight
+  // together (a store in between would hold the later loads of the same buffer back)
+  constexpr int kGroup = 4, kThreads = 256;
+  for (int i0 = 0; i0 < n4; i0 += kGroup * kThreads) {
+    float4 gv[kGroup], ev[kGroup], dv[kGroup];
+#pragma unroll
+    for (int k = 0; k < kGroup; ++k) {
+      const int i = i0 + k * kThreads + (int)threadIdx.x;
+      if (i < n4) {
+        gv[k] = ld_stream4(g + 4 * i);
+        if (is_mat) ev[k] = ld_stream4(e + 4 * i);
+        if (acc_delta) dv[k] = *reinterpret_cast<const float4*>(d + 4 * i);
+      }
     }
-    if (acc_delta) {
-      float4 dv = *reinterpret_cast<const float4*>(d + 4 * i);
-      dv.x += gv.x; dv.y += gv.y; dv.z += gv.z; dv.w += gv.w;
-      *reinterpret_cast<float4*>(d + 4 * i) = dv;
+#pragma unroll
+    for (int k = 0; k < kGroup; ++k) {
+      const int i = i0 + k * kThreads + (int)threadIdx.x;
+      if (i < n4) {
+        if (is_mat)
+          st_stream4(e + 4 * i, make_float4(gv[k].x + ev[k].x, gv[k].y + ev[k].y, gv[k].z + ev[k].z, gv[k].w + ev[k].w));
+        if (acc_delta)
+          *reinterpret_cast<float4*>(d + 4 * i) =
+              make_float4(dv[k].x + gv[k].x, dv[k].y + gv[k].y, dv[k].z + gv[k].z, dv[k].w + gv[k].w);
+      }
     }
   }
   for (int i = 4 * n4 + threadIdx.x; i < t.nelem; i += blockDim.x) {
