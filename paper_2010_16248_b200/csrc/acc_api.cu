@@ -210,6 +210,7 @@ int acc_create(const acc_config* cfg, void* workspace, size_t workspace_bytes, a
   if (e == cudaSuccess) e = cudaMemset(ctx->d_pred, 0xff, sizeof(unsigned) * 4 * seg);  // no prediction yet
   if (e == cudaSuccess) e = cudaMemset(ctx->d_pend_tau, 0xff, sizeof(unsigned) * seg);  // nothing pending
   if (e == cudaSuccess) e = prepare_powersgd();
+  if (e == cudaSuccess) e = prepare_topk(ctx);
   int dev = 0;
   if (e == cudaSuccess) e = cudaGetDevice(&dev);
   if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, dev);

@@ -95,6 +95,7 @@ struct acc_ctx {
   acc::Plan plan;
   char* ws = nullptr;
   int sm_count = 148;
+  int occ_topk_first_pass = 3;       // resident blocks per SM of topk_ef_hist1_kernel (queried at creation)
   int last_launches = 0;
   bool prof = false;                 // per-kernel event timing on
   std::vector<acc::ProfSlot> prof_slots;
@@ -159,6 +160,7 @@ cudaError_t launch_topk(acc_ctx* ctx, const float* grads, float* err, const uint
                         int32_t* idx, int32_t* counts, float* out, float* delta, SgdTail tail, cudaStream_t s);
 // Real workers: the TopK step in two halves around the all-gather of the packed sets.
 cudaError_t launch_topk_flush(acc_ctx* ctx, float* err, cudaStream_t s);
+cudaError_t prepare_topk(acc_ctx* ctx);
 cudaError_t launch_topk_compress(acc_ctx* ctx, const float* grads, float* err, const uint8_t* level, float* vals,
                                  int32_t* idx, int32_t* counts, float* delta, float* vec_packed, cudaStream_t s);
 cudaError_t launch_topk_decompress_packed(acc_ctx* ctx, const float* vals, const int32_t* idx, const int32_t* counts,

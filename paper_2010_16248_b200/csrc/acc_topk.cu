@@ -1210,9 +1210,15 @@ static cudaError_t launch_topk_select_part(acc_ctx* ctx, const float* grads, flo
     const int list_chunks = std::min(128, std::max(8, max_cap / 16384));
     const long long V = (long long)W * nt;
     const int grid = (int)(V < (long long)ctx->sm_count * 8 ? V : (long long)ctx->sm_count * 8);
+    // first pass: a whole number of waves of resident blocks (a grid that is not a multiple of what fits leaves the
+    // last wave of the static split short: 8 blocks per SM with 3 resident cost 4 %), two to six of them (finer
+    // shares even out the deciding worker's tiles, which also carry the detector's accumulator)
+    const long long per_wave = (long long)ctx->sm_count * ctx->occ_topk_first_pass;
+    const long long waves = std::min<long long>(6, std::max<long long>(2, V / (per_wave * 4)));
+    const int grid_a = (int)std::min(V, per_wave * waves);
     {
       PhaseTimer pt(ctx, PH_TOPK_EF_HIST1, s);
-      topk_ef_hist1_kernel<<<grid, 256, 0, s>>>(ctx->d_layers, ctx->d_tiles, nt, n_mat, grads, err, delta,
+      topk_ef_hist1_kernel<<<grid_a, 256, 0, s>>>(ctx->d_layers, ctx->d_tiles, nt, n_mat, grads, err, delta,
                                                 c.worker_stride, W, c.decider, level, ctx->d_pred, ctx->d_hist1,
                                                 ctx->d_seg_cand, ctx->d_seg_flag, ctx->d_cand, ctx->d_tile_cand,
                                                 pl.cand_total, ctx->d_tile_cnt, lazy ? ctx->d_pend_tau : nullptr);
@@ -1357,6 +1363,14 @@ topk_flush_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict__ 
 __global__ void topk_clear_pending_kernel(unsigned* __restrict__ pend_tau, int n) {
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i < n) pend_tau[i] = kNoPendingTau;
+}
+
+// Once per context, at creation: how many blocks of the first pass fit an SM.
+cudaError_t prepare_topk(acc_ctx* ctx) {
+  int occ = 0;
+  const cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, topk_ef_hist1_kernel, 256, 0);
+  ctx->occ_topk_first_pass = occ > 0 ? occ : 1;
+  return e;
 }
 
 cudaError_t launch_topk_flush(acc_ctx* ctx, float* err, cudaStream_t s) {
