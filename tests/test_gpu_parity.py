@@ -568,3 +568,52 @@ def test_topk_lazy_residual_is_bit_identical_to_eager(pipeline_flag):
     assert torch.equal(err_e.view(torch.int32), err_l.view(torch.int32))
     with pytest.raises(binding.AccError):
         eager.acc_topk_flush(err_e)
+
+
+@pytest.mark.parametrize("seed", [1, 2, 3, 4, 5, 6])
+def test_random_tables_both_compressors(seed):
+    """Seeded random layer tables (matrix shapes from 1 x 1 to a few tiles, odd row lengths, vectors in between,
+    unaligned sizes), random W, ranks, fractions, levels and flags: two steps of each compressor against the
+    oracle."""
+    rng = np.random.default_rng(1000 + seed)
+    shapes = []
+    for i in range(int(rng.integers(3, 9))):
+        kind = rng.integers(0, 4)
+        if kind == 0:
+            shapes.append((f"v{i}", (int(rng.integers(1, 9000)),)))
+        elif kind == 1:
+            shapes.append((f"m{i}", (int(rng.integers(1, 40)), int(rng.integers(1, 40)))))
+        elif kind == 2:
+            shapes.append((f"m{i}", (int(rng.integers(1, 12)), int(rng.integers(1000, 9000)))))
+        else:
+            shapes.append((f"m{i}", (int(rng.integers(100, 3000)), int(rng.integers(1, 24)))))
+    if not any(len(s) == 2 for _, s in shapes):
+        shapes.append(("m_last", (17, 19)))
+    table = wl.make_table(shapes)
+    W = int(rng.integers(1, 6))
+    rank_low = int(rng.integers(1, 5))
+    rank_high = int(rng.integers(1, rank_low + 1))
+    low_bp = int(rng.integers(50, 4000))
+    high_bp = int(rng.integers(1, low_bp + 1))
+    flags = int(rng.choice([0, binding.ACC_FLAG_PIPELINE_ALWAYS, binding.ACC_FLAG_PIPELINE_NEVER]))
+    ctx = binding.Context(table, W, rank_low=rank_low, rank_high=rank_high, topk_low_bp=low_bp, topk_high_bp=high_bp,
+                          decider=int(rng.integers(0, W)), flags=flags)
+    level = torch.tensor(rng.integers(0, 2, table.n_layers).astype(np.uint8), device="cuda")
+    _, err_p = _random_inputs(table, W, 2000 + seed)
+    err_t = err_p.clone()
+    q = ctx.new_q(wl.initial_q(table, 4, seed=seed))
+    p = ctx.new_p()
+    vals, idx, counts = ctx.new_topk_buffers()
+    out = torch.zeros(table.stride, device="cuda")
+    delta = torch.zeros(table.stride, device="cuda")
+    for it in range(2):
+        grads, _ = _random_inputs(table, W, 2100 + 10 * seed + it)
+        e0, q0 = err_p.clone(), q.clone()
+        ctx.acc_powersgd_step(grads, err_p, q, p, level, out, delta)
+        torch.cuda.synchronize()
+        H.check_powersgd_against_oracle(ctx, table, grads, e0, q0, level, out, err_p, q, p, rank_low, rank_high, 1e-8)
+        e0 = err_t.clone()
+        ctx.acc_topk_step(grads, err_t, level, vals, idx, counts, out, None)
+        torch.cuda.synchronize()
+        H.check_topk_against_oracle(ctx, table, grads, e0, level, vals, idx, counts, out, err_t, low_bp, high_bp)
+    assert ctx.acc_device_status() == 0
