@@ -281,6 +281,16 @@ int acc_topk_decompress(acc_ctx* ctx, const float* vals_all, const int32_t* idx_
                         int32_t n_sets, const float* vec_packed, float vec_scale, float* out, float* params,
                         float* mom, const float* hyper, void* stream);
 
+/* Host-fed operation (no counterpart in the paper: there the gradients are produced on the GPU).  For callers whose
+ * gradients arrive in HOST memory -- and for the end-to-end leg of the benchmark --
+ *   acc_upload_grads:  grads_dev [W][worker_stride] <- grads_host, one asynchronous copy on `stream`;
+ *   acc_download_out:  out_host [worker_stride] <- out_dev, likewise.
+ * grads_host / out_host are HOST pointers and should be page-locked (pinned), otherwise the copies are staged by
+ * the driver and block; grads_dev / out_dev are DEVICE pointers.  Issue the upload on a copy stream and order
+ * the step after it with an event to overlap it with the previous step's kernels.                     */
+int acc_upload_grads(acc_ctx* ctx, const float* grads_host, float* grads_dev, void* stream);
+int acc_download_out(acc_ctx* ctx, const float* out_dev, float* out_host, void* stream);
+
 /* Device-side condition of the kernels launched so far on this context (no counterpart in the paper).
  * The pipelined kernels wait for their asynchronous shared-memory copies with a bounded number of polls;
  * should a wait ever give up, the block stores ACC_ETIMEOUT in a status word and returns instead of

@@ -49,7 +49,8 @@ EXPORTS = ["acc_workspace_bytes", "acc_create", "acc_destroy", "acc_factor_layou
            "acc_layer_diff_norms", "acc_detect_regime_diff", "acc_sgd_nesterov", "acc_powersgd_step_sgd",
            "acc_topk_step_sgd", "acc_batch_accumulate", "acc_batch_average", "acc_detect_batch",
            "acc_exchange_layout", "acc_powersgd_phase1", "acc_powersgd_phase2", "acc_powersgd_phase3",
-           "acc_topk_compress", "acc_topk_decompress", "acc_topk_flush"]
+           "acc_topk_compress", "acc_topk_decompress", "acc_topk_flush",
+           "acc_upload_grads", "acc_download_out"]
 
 _lib = None
 
@@ -106,6 +107,8 @@ def lib() -> C.CDLL:
     L.acc_topk_compress.argtypes = [vp] * 10
     L.acc_topk_decompress.argtypes = [vp, vp, vp, vp, i32, vp, f32, vp, vp, vp, vp, vp]
     L.acc_topk_flush.argtypes = [vp, vp, vp]
+    L.acc_upload_grads.argtypes = [vp, vp, vp, vp]
+    L.acc_download_out.argtypes = [vp, vp, vp, vp]
     for name in EXPORTS:
         if name not in ("acc_floats_sent", "acc_last_launch_count", "acc_strerror", "acc_profile_kernel_count",
                         "acc_profile_kernel_name"):
@@ -331,6 +334,23 @@ class Context:
 
     def acc_topk_flush(self, err, stream=None):
         self._check(lib().acc_topk_flush(self._h, _ptr(err, torch.float32), _stream(stream)), "acc_topk_flush")
+
+    def acc_upload_grads(self, grads_host, grads_dev, stream=None):
+        """``grads_host``: CPU float32 tensor [W, stride] (pinned for an asynchronous copy)."""
+        if grads_host.is_cuda or grads_host.dtype != torch.float32 or not grads_host.is_contiguous():
+            raise ValueError("expected a contiguous float32 CPU tensor")
+        if grads_host.numel() != self.n_workers * self.stride or grads_dev.numel() != grads_host.numel():
+            raise ValueError("expected [n_workers, worker_stride] elements")
+        self._check(lib().acc_upload_grads(self._h, grads_host.data_ptr(), _ptr(grads_dev, torch.float32),
+                                           _stream(stream)), "acc_upload_grads")
+
+    def acc_download_out(self, out_dev, out_host, stream=None):
+        if out_host.is_cuda or out_host.dtype != torch.float32 or not out_host.is_contiguous():
+            raise ValueError("expected a contiguous float32 CPU tensor")
+        if out_host.numel() != self.stride or out_dev.numel() != self.stride:
+            raise ValueError("expected worker_stride elements")
+        self._check(lib().acc_download_out(self._h, _ptr(out_dev, torch.float32), out_host.data_ptr(),
+                                           _stream(stream)), "acc_download_out")
 
     def acc_profile_enable(self, enable: bool):
         self._check(lib().acc_profile_enable(self._h, int(bool(enable))), "acc_profile_enable")

@@ -372,6 +372,19 @@ int acc_powersgd_phase3(acc_ctx* ctx, float* err, float* q, const float* p_hat, 
                                        static_cast<cudaStream_t>(stream)));
 }
 
+int acc_upload_grads(acc_ctx* ctx, const float* grads_host, float* grads_dev, void* stream) {
+  if (!ctx || !grads_host || !grads_dev) return ACC_EINVAL;
+  if (!aligned16(grads_dev)) return ACC_EALIGN;
+  const size_t bytes = sizeof(float) * (size_t)ctx->cfg.n_workers * (size_t)ctx->cfg.worker_stride;
+  return finish(cudaMemcpyAsync(grads_dev, grads_host, bytes, cudaMemcpyHostToDevice, static_cast<cudaStream_t>(stream)));
+}
+
+int acc_download_out(acc_ctx* ctx, const float* out_dev, float* out_host, void* stream) {
+  if (!ctx || !out_dev || !out_host) return ACC_EINVAL;
+  const size_t bytes = sizeof(float) * (size_t)ctx->cfg.worker_stride;
+  return finish(cudaMemcpyAsync(out_host, out_dev, bytes, cudaMemcpyDeviceToHost, static_cast<cudaStream_t>(stream)));
+}
+
 int acc_topk_flush(acc_ctx* ctx, float* err, void* stream) {
   if (!ctx || !err) return ACC_EINVAL;
   if (!(ctx->cfg.flags & ACC_FLAG_LAZY_RESIDUAL)) return ACC_EINVAL;

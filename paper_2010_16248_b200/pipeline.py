@@ -321,7 +321,7 @@ class HostFedStep:
     """Runs ``AccordionStep`` on gradients that live in pinned host memory.
 
     Every call copies that step's gradients to the device and the step's averaged outputs back to pinned
-    host buffers.  The copies run on their own stream with two device staging buffers, so the upload of
+    host buffers (``acc_upload_grads`` / ``acc_download_out``: host pointers go straight to the library).  The copies run on their own stream with two device staging buffers, so the upload of
     step i+1 overlaps the kernels of step i; results are ordered by events, never by host synchronisation.
     """
 
@@ -349,7 +349,7 @@ class HostFedStep:
         with torch.cuda.stream(self.h2d):
             if self.i >= 2:
                 self.h2d.wait_event(self.consumed[b])      # the step that read this staging buffer is done
-            self.stage[b].copy_(host_grads, non_blocking=True)
+            self.eng.ctx.acc_upload_grads(host_grads, self.stage[b], self.h2d)
             self.uploaded[b].record(self.h2d)
         main.wait_event(self.uploaded[b])
         if self.i >= 1:
@@ -359,7 +359,7 @@ class HostFedStep:
         with torch.cuda.stream(self.d2h):
             self.d2h.wait_event(self.consumed[b])
             for oh, od in zip(self.outs_host, self.eng.outputs()):
-                oh.copy_(od, non_blocking=True)
+                self.eng.ctx.acc_download_out(od, oh, self.d2h)
             self.downloaded.record(self.d2h)
         self.i += 1
         return self.outs_host

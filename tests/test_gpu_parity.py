@@ -617,3 +617,26 @@ def test_random_tables_both_compressors(seed):
         torch.cuda.synchronize()
         H.check_topk_against_oracle(ctx, table, grads, e0, level, vals, idx, counts, out, err_t, low_bp, high_bp)
     assert ctx.acc_device_status() == 0
+
+
+def test_host_fed_step_uploads_and_downloads_through_the_library():
+    """Gradients in pinned host memory, uploaded by acc_upload_grads on a copy stream, outputs read back by
+    acc_download_out: the host copies of the outputs equal the device-resident run's."""
+    table = _table_mixed()
+    W = 2
+    q0 = wl.initial_q(table, 2, seed=41)
+    dev_eng = pipeline.AccordionStep(table, W, ("powersgd", "topk"), check_every=2, q_init=q0)
+    fed_eng = pipeline.AccordionStep(table, W, ("powersgd", "topk"), check_every=2, q_init=q0)
+    fed = pipeline.HostFedStep(fed_eng)
+    host = [torch.empty(W, table.stride).pin_memory() for _ in range(2)]
+    for t in range(5):
+        g, _ = _random_inputs(table, W, 3000 + t)
+        host[t % 2].copy_(g)
+        dev_eng.step(g)
+        outs = fed.step(host[t % 2])
+        fed.synchronize()
+        torch.cuda.synchronize()
+        for oh, od in zip(outs, dev_eng.outputs()):
+            assert torch.equal(oh, od.cpu())
+    with pytest.raises(ValueError):
+        fed_eng.ctx.acc_upload_grads(torch.empty(3), fed.stage[0])
