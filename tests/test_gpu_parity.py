@@ -640,3 +640,32 @@ def test_host_fed_step_uploads_and_downloads_through_the_library():
             assert torch.equal(oh, od.cpu())
     with pytest.raises(ValueError):
         fed_eng.ctx.acc_upload_grads(torch.empty(3), fed.stage[0])
+
+
+def test_many_workers():
+    """W = 37 (more workers than a warp has lanes, not a multiple of the kernels' worker batches) on a small table."""
+    table = wl.make_table([("w0", (50, 333)), ("b0", (77,)), ("w1", (9000, 3)), ("b1", (8195,))])
+    W = 37
+    ctx = binding.Context(table, W, rank_low=2, rank_high=1, topk_low_bp=700, topk_high_bp=70, decider=36)
+    level = torch.tensor([1, 0, 0, 1], dtype=torch.uint8, device="cuda")
+    _, err_p = _random_inputs(table, W, 3100)
+    err_t = err_p.clone()
+    q = ctx.new_q(wl.initial_q(table, 2, seed=3))
+    p = ctx.new_p()
+    vals, idx, counts = ctx.new_topk_buffers()
+    out = torch.zeros(table.stride, device="cuda")
+    delta = torch.zeros(table.stride, device="cuda")
+    for it in range(2):
+        grads, _ = _random_inputs(table, W, 3110 + it)
+        e0, q0 = err_p.clone(), q.clone()
+        ctx.acc_powersgd_step(grads, err_p, q, p, level, out, delta)
+        torch.cuda.synchronize()
+        H.check_powersgd_against_oracle(ctx, table, grads, e0, q0, level, out, err_p, q, p, 2, 1, 1e-8)
+        e0 = err_t.clone()
+        ctx.acc_topk_step(grads, err_t, level, vals, idx, counts, out, None)
+        torch.cuda.synchronize()
+        H.check_topk_against_oracle(ctx, table, grads, e0, level, vals, idx, counts, out, err_t, 700, 70)
+    # the accumulator holds the deciding worker's two gradients
+    want = sum(_random_inputs(table, W, 3110 + it)[0][36] for it in range(2))
+    for l, sl in table.slices():
+        assert torch.allclose(delta[sl], want[sl], rtol=1e-6, atol=1e-7), l
