@@ -298,6 +298,14 @@ int acc_download_out(acc_ctx* ctx, const float* out_dev, float* out_host, void* 
  * (HOST pointer; 0 = no such event) and blocks until the device has finished the work queued before it. */
 int acc_device_status(acc_ctx* ctx, int32_t* status);
 
+/* Failure-detection self-test (no counterpart in the paper).  acc_selftest_wait_timeout launches one small kernel
+ * that waits, with a short poll limit, on a barrier at which nothing ever arrives; the wait gives up, the kernel
+ * stores ACC_ETIMEOUT in the status word and returns normally -- the path a pipelined kernel takes should one of
+ * its copies never complete.  Nothing faults or hangs, and the context stays usable.  acc_reset_device_status
+ * clears the status word (asynchronously on `stream`).                                                 */
+int acc_selftest_wait_timeout(acc_ctx* ctx, void* stream);
+int acc_reset_device_status(acc_ctx* ctx, void* stream);
+
 /* Diagnostic (no counterpart in the paper): which selection path the last acc_topk_step took for every
  * (worker, MATRIX layer) pair, in worker-major order, n >= W * (number of MATRIX layers) HOST ints:
  *   0 dense (levels 2-3 of the radix select read M), 1 list built by the collect pass, 2 list built by the

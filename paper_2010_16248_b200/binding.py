@@ -50,7 +50,7 @@ EXPORTS = ["acc_workspace_bytes", "acc_create", "acc_destroy", "acc_factor_layou
            "acc_topk_step_sgd", "acc_batch_accumulate", "acc_batch_average", "acc_detect_batch",
            "acc_exchange_layout", "acc_powersgd_phase1", "acc_powersgd_phase2", "acc_powersgd_phase3",
            "acc_topk_compress", "acc_topk_decompress", "acc_topk_flush",
-           "acc_upload_grads", "acc_download_out"]
+           "acc_upload_grads", "acc_download_out", "acc_selftest_wait_timeout", "acc_reset_device_status"]
 
 _lib = None
 
@@ -108,6 +108,8 @@ def lib() -> C.CDLL:
     L.acc_topk_decompress.argtypes = [vp, vp, vp, vp, i32, vp, f32, vp, vp, vp, vp, vp]
     L.acc_topk_flush.argtypes = [vp, vp, vp]
     L.acc_upload_grads.argtypes = [vp, vp, vp, vp]
+    L.acc_selftest_wait_timeout.argtypes = [vp, vp]
+    L.acc_reset_device_status.argtypes = [vp, vp]
     L.acc_download_out.argtypes = [vp, vp, vp, vp]
     for name in EXPORTS:
         if name not in ("acc_floats_sent", "acc_last_launch_count", "acc_strerror", "acc_profile_kernel_count",
@@ -374,6 +376,12 @@ class Context:
         v = C.c_int32(0)
         self._check(lib().acc_device_status(self._h, C.byref(v)), "acc_device_status")
         return int(v.value)
+
+    def acc_selftest_wait_timeout(self, stream=None):
+        self._check(lib().acc_selftest_wait_timeout(self._h, _stream(stream)), "acc_selftest_wait_timeout")
+
+    def acc_reset_device_status(self, stream=None):
+        self._check(lib().acc_reset_device_status(self._h, _stream(stream)), "acc_reset_device_status")
 
     def last_launch_count(self) -> int:
         return int(lib().acc_last_launch_count(self._h))

@@ -574,6 +574,17 @@ int acc_device_status(acc_ctx* ctx, int32_t* status) {
   return ACC_OK;
 }
 
+int acc_selftest_wait_timeout(acc_ctx* ctx, void* stream) {
+  if (!ctx) return ACC_EINVAL;
+  ctx->last_launches = 0;
+  return finish(launch_selftest_wait(ctx, static_cast<cudaStream_t>(stream)));
+}
+
+int acc_reset_device_status(acc_ctx* ctx, void* stream) {
+  if (!ctx) return ACC_EINVAL;
+  return finish(cudaMemsetAsync(ctx->d_status, 0, sizeof(int), static_cast<cudaStream_t>(stream)));
+}
+
 int32_t acc_last_launch_count(const acc_ctx* ctx) { return ctx ? ctx->last_launches : -1; }
 
 const char* acc_strerror(int status) {

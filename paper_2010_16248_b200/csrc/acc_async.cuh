@@ -53,9 +53,9 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, unsigned parity) {
   return ok != 0;
 }
 
-// Waits for the phase with the given parity; false if it did not complete within kMaxBarrierPolls polls.
-__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, unsigned parity) {
-  for (unsigned i = 0; i < kMaxBarrierPolls; ++i)
+// Waits for the phase with the given parity; false if it did not complete within max_polls polls.
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, unsigned parity, unsigned max_polls = kMaxBarrierPolls) {
+  for (unsigned i = 0; i < max_polls; ++i)
     if (mbar_try_wait(bar, parity)) return true;
   return false;
 }

@@ -147,6 +147,7 @@ cudaError_t launch_detect(acc_ctx* ctx, const double* n2c, double* n2p, const do
 cudaError_t launch_powersgd(acc_ctx* ctx, const float* grads, float* err, float* q, float* p_hat,
                             const uint8_t* level, float* out, float* delta, SgdTail tail, cudaStream_t s);
 cudaError_t prepare_powersgd();
+cudaError_t launch_selftest_wait(acc_ctx* ctx, cudaStream_t s);
 // Real workers: the step in three parts, around the two exchanges (x1: P rows + packed VECTOR means, x2: Q' rows).
 cudaError_t launch_powersgd_phase1(acc_ctx* ctx, const float* grads, float* err, float* q, float* p_hat,
                                    const uint8_t* level, float* out, float* delta, float* x1, cudaStream_t s);

@@ -806,6 +806,25 @@ __global__ void psgd_clear_pending_kernel(int* __restrict__ pending, int n_layer
   if (l < n_layers) pending[l] = 0;
 }
 
+// Exercises the bounded wait: a barrier nobody arrives at, a short poll limit; the block reports ACC_ETIMEOUT in
+// the status word and returns normally (what a pipelined kernel does if a copy never completes).
+__global__ void selftest_wait_kernel(int* __restrict__ status) {
+  __shared__ uint64_t bar;
+  if (threadIdx.x == 0) {
+    mbar_init(&bar, 1);
+    fence_mbar_init();
+  }
+  __syncthreads();
+  const bool arrived = __syncthreads_and(mbar_wait_bounded(&bar, 0u, 2048u));
+  if (!arrived && threadIdx.x == 0) atomicExch(status, ACC_ETIMEOUT);
+}
+
+cudaError_t launch_selftest_wait(acc_ctx* ctx, cudaStream_t s) {
+  ctx->last_launches += 1;
+  selftest_wait_kernel<<<1, 64, 0, s>>>(ctx->d_status);
+  return cudaGetLastError();
+}
+
 // Once per context, at creation (not a stream operation): the pipelined kernels need more than 48 KB of
 // dynamic shared memory.
 cudaError_t prepare_powersgd() {

@@ -669,3 +669,27 @@ def test_many_workers():
     want = sum(_random_inputs(table, W, 3110 + it)[0][36] for it in range(2))
     for l, sl in table.slices():
         assert torch.allclose(delta[sl], want[sl], rtol=1e-6, atol=1e-7), l
+
+
+def test_bounded_wait_reports_timeout_and_context_stays_usable():
+    """Failure detection without a fault: a kernel waits, with a short poll limit, on a barrier nothing arrives at;
+    the wait gives up, the status word reads ACC_ETIMEOUT, the kernel has returned normally and later calls on the
+    same context work as before."""
+    table = _table_mixed()
+    W = 2
+    ctx = binding.Context(table, W, flags=binding.ACC_FLAG_PIPELINE_ALWAYS)
+    assert ctx.acc_device_status() == 0
+    ctx.acc_selftest_wait_timeout()
+    assert ctx.acc_device_status() == 6  # ACC_ETIMEOUT
+    grads, err = _random_inputs(table, W, 3200)
+    q = ctx.new_q(wl.initial_q(table, 2, seed=8))
+    p = ctx.new_p()
+    level = torch.ones(table.n_layers, dtype=torch.uint8, device="cuda")
+    out = torch.zeros(table.stride, device="cuda")
+    e0, q0 = err.clone(), q.clone()
+    ctx.acc_powersgd_step(grads, err, q, p, level, out)
+    torch.cuda.synchronize()
+    H.check_powersgd_against_oracle(ctx, table, grads, e0, q0, level, out, err, q, p, 2, 1, 1e-8)
+    assert ctx.acc_device_status() == 6  # sticky until it is reset
+    ctx.acc_reset_device_status()
+    assert ctx.acc_device_status() == 0
