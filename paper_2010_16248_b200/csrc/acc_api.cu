@@ -123,7 +123,7 @@ static int make_plan(const acc_config* cfg, Plan& p) {
   take(sizeof(unsigned) * 64);   // "some segment needs the collect pass" flag, likewise
   p.hist_bytes = o - p.o_hist;
   p.o_sel = take(sizeof(Select) * seg);
-  p.o_pred = take(sizeof(unsigned) * 4 * seg);  // [2] prediction words, [2] last buckets, per level
+  p.o_pred = take(sizeof(unsigned) * 6 * seg);  // [2] prediction words, [2] last buckets, [2] last moves, per level
   p.o_cand = take(sizeof(unsigned) * (size_t)W * std::max<long long>(1, p.cand_total));
   p.o_tile_cand = take(sizeof(int2) * (size_t)W * nt);
   p.o_tile_cnt = take(sizeof(int2) * (size_t)W * nt);
@@ -207,7 +207,7 @@ int acc_create(const acc_config* cfg, void* workspace, size_t workspace_bytes, a
   up(ctx->d_mat_tiles, p.mat_tiles.data(), sizeof(int) * p.mat_tiles.size());
   if (e == cudaSuccess) e = cudaMemset(ctx->d_status, 0, sizeof(int) * 64);
   if (e == cudaSuccess) e = cudaMemset(ctx->d_pending, 0, sizeof(int) * cfg->n_layers);
-  if (e == cudaSuccess) e = cudaMemset(ctx->d_pred, 0xff, sizeof(unsigned) * 4 * seg);  // no prediction yet
+  if (e == cudaSuccess) e = cudaMemset(ctx->d_pred, 0xff, sizeof(unsigned) * 6 * seg);  // no prediction yet
   if (e == cudaSuccess) e = cudaMemset(ctx->d_pend_tau, 0xff, sizeof(unsigned) * seg);  // nothing pending
   if (e == cudaSuccess) e = prepare_powersgd();
   if (e == cudaSuccess) e = prepare_topk(ctx);

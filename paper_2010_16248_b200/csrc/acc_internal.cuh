@@ -119,7 +119,7 @@ struct acc_ctx {
   unsigned* d_seg_cand = nullptr;    // per (worker, layer): candidate slots handed out this step
   unsigned* d_any_list = nullptr;    // per-step word block, cleared with the histograms; words 8..11: lengths of the work lists
   unsigned* d_seg_flag = nullptr;    // per (worker, layer): 1 if pass A's collection overflowed this step
-  unsigned* d_pred = nullptr;        // [4][W * n_mat]: prediction word per level, then last threshold bucket per level; kept across steps
+  unsigned* d_pred = nullptr;        // [6][W * n_mat]: prediction word, last threshold bucket, last move of the bucket, each per level; kept across steps
   unsigned* d_cand = nullptr;        // candidate keys, [W][cand_total]
   int2* d_tile_cand = nullptr;       // per (worker, tile): (first slot, count) inside the segment's list
   int2* d_tile_cnt = nullptr;

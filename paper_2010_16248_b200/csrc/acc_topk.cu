@@ -356,8 +356,14 @@ topk_pick1_kernel(const DevLayer* __restrict__ layers, const int* __restrict__ m
     unsigned* lb = pred + (long long)(2 + lv) * W * n_mat + seg;
     const unsigned last = *lb;
     int drift = last != kPredInvalid ? (int)bin - (int)last : 0;
-    drift = drift < -3 ? -3 : drift > 6 ? 6 : drift;
-    int centre = (int)bin + drift;
+    drift = drift < -12 ? -12 : drift > 12 ? 12 : drift;
+    // the mean of the last two moves (rounded toward zero): a threshold that hops between two neighbouring buckets
+    // keeps its band, a climb of one to two buckets a step with some jitter stays inside it, steady faster
+    // moves are followed
+    int* ld = reinterpret_cast<int*>(pred + (long long)(4 + lv) * W * n_mat + seg);
+    const int prev_drift = last != kPredInvalid ? *ld : 0;
+    *ld = drift;
+    int centre = (int)bin + (drift + prev_drift) / 2;
     centre = centre < 1 ? 1 : centre > kBins1 - 1 ? kBins1 - 1 : centre;
     *lb = bin;
     *pw = (!fits || bin == 0) ? kPredInvalid
