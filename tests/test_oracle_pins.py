@@ -107,6 +107,69 @@ def test_accumulate_sums_decider_gradients():
     assert delta[6] == 0.0 and delta[7] == 0.0  # padding between layers untouched
 
 
+def test_error_feedback_hand_values_vector_rule_and_precision_flag():
+    """M = g + e on MATRIX layers, M = g on VECTOR layers (1-D tensors carry no memory), padding stays zero;
+    with fp32=True the sum is ONE fp32 add, which the hand-picked operands distinguish from the fp64 sum."""
+    table = wl.make_table([("a", (2, 3)), ("v", (5,))])   # matrix at 0..5, padding 6..7, vector at 8..12
+    layers = _layers(table)
+    assert [l[0] for l in layers] == [0, 8]
+    tiny = np.float32(2.0 ** -24)                         # half an ulp of 1.0 in fp32
+    g = np.zeros((2, table.stride), np.float32)
+    e = np.zeros((2, table.stride), np.float32)
+    g[0, 0:6] = [1.0, 2.0, -3.0, 0.5, 1.0, 1.0]
+    e[0, 0:6] = [0.25, -2.0, 1.0, 0.125, tiny, 3 * tiny]
+    g[1, 0:6] = [10.0, 20.0, 30.0, 40.0, 50.0, 60.0]
+    e[1, 0:6] = [-1.0, -2.0, -3.0, -4.0, -5.0, -6.0]
+    g[:, 8:13] = [[1.0, 2.0, 3.0, 4.0, 5.0], [6.0, 7.0, 8.0, 9.0, 10.0]]
+    e[:, 8:13] = 100.0                                    # memory on a VECTOR layer must be ignored
+    e[:, 6:8] = 7.0                                       # so must anything in the padding
+    M64 = orc.error_feedback(g, e, layers)
+    assert M64.dtype == np.float64
+    assert M64[0, 0:4].tolist() == [1.25, 0.0, -2.0, 0.625]
+    assert M64[0, 4] == 1.0 + 2.0 ** -24 and M64[0, 5] == 1.0 + 3 * 2.0 ** -24      # exact in fp64
+    assert M64[1, 0:6].tolist() == [9.0, 18.0, 27.0, 36.0, 45.0, 54.0]
+    assert M64[0, 8:13].tolist() == [1.0, 2.0, 3.0, 4.0, 5.0] and M64[1, 8:13].tolist() == [6.0, 7.0, 8.0, 9.0, 10.0]
+    assert np.all(M64[:, 6:8] == 0.0) and np.all(M64[:, 13:] == 0.0)
+    M32 = orc.error_feedback(g, e, layers, fp32=True)
+    assert M32.dtype == np.float32
+    # 1 + 2^-24 is a tie between 1 and 1 + 2^-23: round-to-even gives 1; 1 + 3*2^-24 rounds up to 1 + 2^-22
+    assert M32[0, 4] == np.float32(1.0) and M32[0, 5] == np.float32(1.0 + 2.0 ** -22)
+    assert float(M32[0, 4]) != M64[0, 4] and float(M32[0, 5]) != M64[0, 5]
+    assert M32[0, 0:4].tolist() == [1.25, 0.0, -2.0, 0.625] and M32[0, 8:13].tolist() == [1.0, 2.0, 3.0, 4.0, 5.0]
+    assert np.all(M32[:, 6:8] == 0.0)
+
+
+def test_error_feedback_is_what_both_compressors_split():
+    """Invariant of error feedback: what a compressor sends plus what it keeps as memory is g + e.  Ties the
+    stand-alone accumulation to the two compressor steps (which were pinned independently of it)."""
+    rng = np.random.default_rng(21)
+    table = wl.make_table([("a", (9, 14)), ("v", (7,)), ("b", (12, 5))])
+    layers = _layers(table)
+    W = 3
+    grads = np.zeros((W, table.stride), np.float32)
+    err = np.zeros((W, table.stride), np.float32)
+    for (off, r, c, k) in layers:
+        grads[:, off:off + r * c] = rng.standard_normal((W, r * c))
+        if k == orc.MATRIX:
+            err[:, off:off + r * c] = 0.4 * rng.standard_normal((W, r * c))
+    level = [1, 0, 0]
+    M64 = orc.error_feedback(grads, err, layers)
+    M32 = orc.error_feedback(grads, err, layers, fp32=True)
+    q = [rng.standard_normal((c, 2)) if k == orc.MATRIX else None for (_, _, c, k) in layers]
+    out, e_p, _, _ = orc.powersgd_step(grads, err, q, level, layers, 2, 1)
+    vals, idx, counts, _, e_t = orc.topk_step(grads, err, level, layers, 1000, 100)
+    for l, (off, r, c, k) in enumerate(layers):
+        sl = slice(off, off + r * c)
+        if k == orc.VECTOR:
+            assert np.allclose(out[sl], M64[:, sl].mean(0), rtol=1e-15)   # the mean of the raw gradients
+            continue
+        for w in range(W):
+            assert np.allclose(out[sl] + e_p[w, sl], M64[w, sl], rtol=0, atol=1e-14)
+            rec = e_t[w, sl].copy()
+            rec[idx[w][l]] = vals[w][l]
+            assert np.array_equal(rec.view(np.uint32), M32[w, sl].view(np.uint32))   # bit for bit, fp32 add
+
+
 def test_c1_schedule_known_answer():
     """Config 1: scale doubles at iteration 10, checks after iterations 4, 9, 14, 19.
     Levels: LOW before the first check and after it (no previous window), HIGH after the
