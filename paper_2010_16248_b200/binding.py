@@ -144,21 +144,52 @@ def acc_sumsq_static(buf: torch.Tensor, n: int, norm2: torch.Tensor, stream=None
     For callers that cannot allocate device memory or supply a workspace: the reduction scratch is a
     fixed array inside the library, so this call allocates nothing (neither do these few lines).
     ``n`` is limited to 2**28 elements; calls that overlap on the GPU share the scratch and race."""
-    st = lib().acc_sumsq_static(_ptr(buf, torch.float32), int(n), _ptr(norm2, torch.float64), _stream(stream))
+    n = int(n)
+    st = lib().acc_sumsq_static(*_marshal(None, _Arg(buf, torch.float32, max(n, 0), "buf"), n,
+                                          _Arg(norm2, torch.float64, 1, "norm2")), _stream(stream))
     if st != ACC_OK:
         raise AccError(st, "acc_sumsq_static")
 
 
-def _ptr(t: Optional[torch.Tensor], dtype=None) -> Optional[int]:
-    if t is None:
-        return None
-    if not t.is_cuda:
-        raise ValueError("expected a CUDA tensor (the library has no CPU path)")
-    if not t.is_contiguous():
-        raise ValueError("expected a contiguous tensor")
-    if dtype is not None and t.dtype != dtype:
-        raise ValueError(f"expected dtype {dtype}, got {t.dtype}")
-    return t.data_ptr()
+class _Arg:
+    """One tensor argument of a call with what the call requires of it."""
+    __slots__ = ("t", "dtype", "min_numel", "what")
+
+    def __init__(self, t, dtype, min_numel, what):
+        self.t, self.dtype, self.min_numel, self.what = t, dtype, int(min_numel), what
+
+
+def _marshal(device, *items):
+    """Turns the ``_Arg`` items into device addresses (other items pass through) after checking what the C ABI
+    cannot see.  First every tensor's dtype, contiguity and length -- the kernels index by the context's layout, so
+    a short tensor would be an out-of-bounds device access, not an exception -- then that every tensor lives on
+    the GPU the call runs on (there is no CPU path)."""
+    for a in items:
+        if not isinstance(a, _Arg) or a.t is None:
+            continue
+        t = a.t
+        if not isinstance(t, torch.Tensor):
+            raise ValueError(f"{a.what}: expected a torch tensor")
+        if t.dtype != a.dtype:
+            raise ValueError(f"{a.what}: expected dtype {a.dtype}, got {t.dtype}")
+        if not t.is_contiguous():
+            raise ValueError(f"{a.what}: expected a contiguous tensor")
+        if t.numel() < a.min_numel:
+            raise ValueError(f"{a.what}: {t.numel()} elements, the call needs at least {a.min_numel}")
+    out = []
+    for a in items:
+        if not isinstance(a, _Arg):
+            out.append(a)
+            continue
+        if a.t is None:
+            out.append(None)
+            continue
+        if not a.t.is_cuda:
+            raise ValueError(f"{a.what}: expected a CUDA tensor (the library has no CPU path)")
+        if device is not None and device.index is not None and a.t.device.index != device.index:
+            raise ValueError(f"{a.what}: lives on {a.t.device}, the context on {device}")
+        out.append(a.t.data_ptr())
+    return out
 
 
 def _stream(stream) -> Optional[int]:
@@ -172,8 +203,13 @@ class Context:
     def __init__(self, table, n_workers, device="cuda", **cfg_kwargs):
         self.table = table
         self.device = torch.device(device)
+        if self.device.type == "cuda" and self.device.index is None:
+            self.device = torch.device("cuda", torch.cuda.current_device())
         self.cfg = make_config(table, n_workers, **cfg_kwargs)
         self.n_workers, self.n_layers, self.stride = n_workers, table.n_layers, int(self.cfg.worker_stride)
+        # elements of one worker's slice that the layer table reaches (<= worker_stride)
+        self.extent = int(max(int(table.offset[l]) + int(table.rows[l]) * int(table.cols[l])
+                              for l in range(table.n_layers)))
         L = lib()
         nbytes = C.c_size_t(0)
         st = L.acc_workspace_bytes(C.byref(self.cfg), C.byref(nbytes))
@@ -216,143 +252,164 @@ class Context:
         if st != ACC_OK:
             raise AccError(st, where)
 
+    def _call(self, name, *items, stream=None):
+        """Checks and marshals the tensor arguments, then calls entry point ``name`` on this context."""
+        self._check(getattr(lib(), name)(self._h, *_marshal(self.device, *items), _stream(stream)), name)
+
+    # --- argument checks: every device buffer must hold what the context's layout will index -----------------
+    def _f(self, t, n, what):
+        return _Arg(t, torch.float32, n, what)
+
+    def _d(self, t, n, what):
+        return _Arg(t, torch.float64, n, what)
+
+    def _i(self, t, n, what):
+        return _Arg(t, torch.int32, n, what)
+
+    def _lv(self, t):
+        return _Arg(t, torch.uint8, self.n_layers, "level")
+
+    @property
+    def _wn(self):  # elements of a [W][worker_stride] buffer
+        return self.n_workers * self.stride
+
+    def _tail(self, params, mom, hyper):
+        if params is None:
+            return None, None, None
+        if mom is None or hyper is None:
+            raise ValueError("the optimiser tail needs params, mom and hyper together")
+        return self._f(params, self.stride, "params"), self._f(mom, self.stride, "mom"), self._f(hyper, 3, "hyper")
+
     # --- entry points -------------------------------------------------------------------------
     def acc_error_feedback(self, grads, err, delta=None, stream=None):
-        self._check(lib().acc_error_feedback(self._h, _ptr(grads, torch.float32), _ptr(err, torch.float32),
-                                             _ptr(delta, torch.float32), _stream(stream)), "acc_error_feedback")
+        self._call("acc_error_feedback", self._f(grads, self._wn, "grads"), self._f(err, self._wn, "err"),
+                   self._f(delta, self.stride, "delta"), stream=stream)
 
     def acc_layer_norms(self, buf, n_bufs, norm2, buf_stride=None, stream=None):
         stride = int(buf_stride if buf_stride is not None else self.stride)
-        self._check(lib().acc_layer_norms(self._h, _ptr(buf, torch.float32), stride, n_bufs,
-                                          _ptr(norm2, torch.float64), _stream(stream)), "acc_layer_norms")
+        n_bufs = int(n_bufs)
+        need = (n_bufs - 1) * stride + self.extent if n_bufs >= 1 else 0
+        self._call("acc_layer_norms", self._f(buf, need, "buf"), stride, n_bufs,
+                   self._d(norm2, max(n_bufs, 0) * self.n_layers, "norm2"), stream=stream)
 
     def acc_detect_regime(self, norm2_curr, norm2_prev, lr_curr, lr_next, level, delta=None, stream=None):
-        self._check(lib().acc_detect_regime(self._h, _ptr(norm2_curr, torch.float64), _ptr(norm2_prev, torch.float64),
-                                            float(lr_curr), float(lr_next), _ptr(level, torch.uint8),
-                                            _ptr(delta, torch.float32), _stream(stream)), "acc_detect_regime")
+        L = self.n_layers
+        self._call("acc_detect_regime", self._d(norm2_curr, L, "norm2_curr"),
+                   self._d(norm2_prev, L, "norm2_prev"), float(lr_curr), float(lr_next), self._lv(level),
+                   self._f(delta, self.stride, "delta"), stream=stream)
 
     def acc_layer_diff_norms(self, a, b, norm2, stream=None):
-        self._check(lib().acc_layer_diff_norms(self._h, _ptr(a, torch.float32), _ptr(b, torch.float32),
-                                               _ptr(norm2, torch.float64), _stream(stream)), "acc_layer_diff_norms")
+        self._call("acc_layer_diff_norms", self._f(a, self.extent, "a"), self._f(b, self.extent, "b"),
+                   self._d(norm2, self.n_layers, "norm2"), stream=stream)
 
     def acc_detect_regime_diff(self, norm2_diff, norm2_curr, norm2_prev, lr_curr, lr_next, level, delta, delta_prev,
                                stream=None):
-        self._check(lib().acc_detect_regime_diff(self._h, _ptr(norm2_diff, torch.float64),
-                                                 _ptr(norm2_curr, torch.float64), _ptr(norm2_prev, torch.float64),
-                                                 float(lr_curr), float(lr_next), _ptr(level, torch.uint8),
-                                                 _ptr(delta, torch.float32), _ptr(delta_prev, torch.float32),
-                                                 _stream(stream)), "acc_detect_regime_diff")
+        L = self.n_layers
+        self._call("acc_detect_regime_diff", self._d(norm2_diff, L, "norm2_diff"),
+                   self._d(norm2_curr, L, "norm2_curr"), self._d(norm2_prev, L, "norm2_prev"), float(lr_curr),
+                   float(lr_next), self._lv(level), self._f(delta, self.stride, "delta"),
+                   self._f(delta_prev, self.stride, "delta_prev"), stream=stream)
+
+    def _psgd_args(self, grads, err, q, p_hat, level, out, delta):
+        return (self._f(grads, self._wn, "grads"), self._f(err, self._wn, "err"), self._f(q, 4 * self.q_rows, "q"),
+                self._f(p_hat, 4 * self.p_rows, "p_hat"), self._lv(level), self._f(out, self.stride, "out"),
+                self._f(delta, self.stride, "delta"))
+
+    def _topk_args(self, grads, err, level, vals, idx, counts):
+        cap = self.n_workers * self.capacity
+        return (self._f(grads, self._wn, "grads"), self._f(err, self._wn, "err"), self._lv(level),
+                self._f(vals, cap, "vals"), self._i(idx, cap, "idx"),
+                self._i(counts, self.n_workers * self.n_layers, "counts"))
 
     def acc_powersgd_step(self, grads, err, q, p_hat, level, out, delta=None, stream=None):
-        self._check(lib().acc_powersgd_step(self._h, _ptr(grads, torch.float32), _ptr(err, torch.float32),
-                                            _ptr(q, torch.float32), _ptr(p_hat, torch.float32),
-                                            _ptr(level, torch.uint8), _ptr(out, torch.float32),
-                                            _ptr(delta, torch.float32), _stream(stream)), "acc_powersgd_step")
+        self._call("acc_powersgd_step", *self._psgd_args(grads, err, q, p_hat, level, out, delta),
+                   stream=stream)
 
     def acc_powersgd_flush(self, err, q, p_hat, stream=None):
-        self._check(lib().acc_powersgd_flush(self._h, _ptr(err, torch.float32), _ptr(q, torch.float32),
-                                             _ptr(p_hat, torch.float32), _stream(stream)), "acc_powersgd_flush")
+        self._call("acc_powersgd_flush", self._f(err, self._wn, "err"), self._f(q, 4 * self.q_rows, "q"),
+                   self._f(p_hat, 4 * self.p_rows, "p_hat"), stream=stream)
 
     def acc_topk_step(self, grads, err, level, vals, idx, counts, out, delta=None, stream=None):
-        self._check(lib().acc_topk_step(self._h, _ptr(grads, torch.float32), _ptr(err, torch.float32),
-                                        _ptr(level, torch.uint8), _ptr(vals, torch.float32), _ptr(idx, torch.int32),
-                                        _ptr(counts, torch.int32), _ptr(out, torch.float32),
-                                        _ptr(delta, torch.float32), _stream(stream)), "acc_topk_step")
+        self._call("acc_topk_step", *self._topk_args(grads, err, level, vals, idx, counts),
+                   self._f(out, self.stride, "out"), self._f(delta, self.stride, "delta"), stream=stream)
 
     def acc_sgd_nesterov(self, d, params, mom, hyper, stream=None):
-        self._check(lib().acc_sgd_nesterov(self._h, _ptr(d, torch.float32), _ptr(params, torch.float32),
-                                           _ptr(mom, torch.float32), _ptr(hyper, torch.float32), _stream(stream)),
-                    "acc_sgd_nesterov")
+        self._call("acc_sgd_nesterov", self._f(d, self.stride, "d"), *self._tail(params, mom, hyper),
+                   stream=stream)
 
     def acc_powersgd_step_sgd(self, grads, err, q, p_hat, level, out, delta, params, mom, hyper, stream=None):
-        self._check(lib().acc_powersgd_step_sgd(self._h, _ptr(grads, torch.float32), _ptr(err, torch.float32),
-                                                _ptr(q, torch.float32), _ptr(p_hat, torch.float32),
-                                                _ptr(level, torch.uint8), _ptr(out, torch.float32),
-                                                _ptr(delta, torch.float32), _ptr(params, torch.float32),
-                                                _ptr(mom, torch.float32), _ptr(hyper, torch.float32),
-                                                _stream(stream)), "acc_powersgd_step_sgd")
+        self._call("acc_powersgd_step_sgd", *self._psgd_args(grads, err, q, p_hat, level, out, delta),
+                   *self._tail(params, mom, hyper), stream=stream)
 
     def acc_topk_step_sgd(self, grads, err, level, vals, idx, counts, out, delta, params, mom, hyper, stream=None):
-        self._check(lib().acc_topk_step_sgd(self._h, _ptr(grads, torch.float32), _ptr(err, torch.float32),
-                                            _ptr(level, torch.uint8), _ptr(vals, torch.float32),
-                                            _ptr(idx, torch.int32), _ptr(counts, torch.int32),
-                                            _ptr(out, torch.float32), _ptr(delta, torch.float32),
-                                            _ptr(params, torch.float32), _ptr(mom, torch.float32),
-                                            _ptr(hyper, torch.float32), _stream(stream)), "acc_topk_step_sgd")
+        self._call("acc_topk_step_sgd", *self._topk_args(grads, err, level, vals, idx, counts),
+                   self._f(out, self.stride, "out"), self._f(delta, self.stride, "delta"),
+                   *self._tail(params, mom, hyper), stream=stream)
 
     def acc_batch_accumulate(self, grads, acc, delta=None, first=False, stream=None):
-        self._check(lib().acc_batch_accumulate(self._h, _ptr(grads, torch.float32), _ptr(acc, torch.float32),
-                                               _ptr(delta, torch.float32), int(bool(first)), _stream(stream)),
-                    "acc_batch_accumulate")
+        self._call("acc_batch_accumulate", self._f(grads, self._wn, "grads"), self._f(acc, self._wn, "acc"),
+                   self._f(delta, self.stride, "delta"), int(bool(first)), stream=stream)
 
     def acc_batch_average(self, acc, n_accum, out, params=None, mom=None, hyper=None, stream=None):
-        self._check(lib().acc_batch_average(self._h, _ptr(acc, torch.float32), int(n_accum),
-                                            _ptr(out, torch.float32), _ptr(params, torch.float32),
-                                            _ptr(mom, torch.float32), _ptr(hyper, torch.float32), _stream(stream)),
-                    "acc_batch_average")
+        self._call("acc_batch_average", self._f(acc, self._wn, "acc"), int(n_accum),
+                   self._f(out, self.stride, "out"), *self._tail(params, mom, hyper), stream=stream)
 
     def acc_detect_batch(self, norm2_layers, norm2_prev, lr_curr, lr_next, b_low, b_high, batch, lr_scale,
                          delta=None, stream=None):
-        self._check(lib().acc_detect_batch(self._h, _ptr(norm2_layers, torch.float64),
-                                           _ptr(norm2_prev, torch.float64), float(lr_curr), float(lr_next),
-                                           int(b_low), int(b_high), _ptr(batch, torch.int32),
-                                           _ptr(lr_scale, torch.float32), _ptr(delta, torch.float32),
-                                           _stream(stream)), "acc_detect_batch")
+        self._call("acc_detect_batch", self._d(norm2_layers, self.n_layers, "norm2_layers"),
+                   self._d(norm2_prev, 1, "norm2_prev"), float(lr_curr), float(lr_next), int(b_low), int(b_high),
+                   self._i(batch, 1, "batch"), self._f(lr_scale, 1, "lr_scale"),
+                   self._f(delta, self.stride, "delta"), stream=stream)
 
     def acc_powersgd_phase1(self, grads, err, q, p_hat, level, out, delta, x1, stream=None):
-        f = torch.float32
-        self._check(lib().acc_powersgd_phase1(self._h, _ptr(grads, f), _ptr(err, f), _ptr(q, f), _ptr(p_hat, f),
-                                              _ptr(level, torch.uint8), _ptr(out, f), _ptr(delta, f), _ptr(x1, f),
-                                              _stream(stream)), "acc_powersgd_phase1")
+        self._call("acc_powersgd_phase1", *self._psgd_args(grads, err, q, p_hat, level, out, delta),
+                   self._f(x1, self.x1_floats, "x1"), stream=stream)
 
     def acc_powersgd_phase2(self, x1, scale, p_hat, level, out, x2, stream=None):
-        f = torch.float32
-        self._check(lib().acc_powersgd_phase2(self._h, _ptr(x1, f), float(scale), _ptr(p_hat, f),
-                                              _ptr(level, torch.uint8), _ptr(out, f), _ptr(x2, f), _stream(stream)),
-                    "acc_powersgd_phase2")
+        self._call("acc_powersgd_phase2", self._f(x1, self.x1_floats, "x1"), float(scale),
+                   self._f(p_hat, 4 * self.p_rows, "p_hat"), self._lv(level), self._f(out, self.stride, "out"),
+                   self._f(x2, self.x2_floats, "x2"), stream=stream)
 
     def acc_powersgd_phase3(self, err, q, p_hat, level, x1, x2, scale, out, params=None, mom=None, hyper=None,
                             stream=None):
-        f = torch.float32
-        self._check(lib().acc_powersgd_phase3(self._h, _ptr(err, f), _ptr(q, f), _ptr(p_hat, f),
-                                              _ptr(level, torch.uint8), _ptr(x1, f), _ptr(x2, f), float(scale),
-                                              _ptr(out, f), _ptr(params, f), _ptr(mom, f), _ptr(hyper, f),
-                                              _stream(stream)), "acc_powersgd_phase3")
+        self._call("acc_powersgd_phase3", self._f(err, self._wn, "err"), self._f(q, 4 * self.q_rows, "q"),
+                   self._f(p_hat, 4 * self.p_rows, "p_hat"), self._lv(level), self._f(x1, self.x1_floats, "x1"),
+                   self._f(x2, self.x2_floats, "x2"), float(scale), self._f(out, self.stride, "out"),
+                   *self._tail(params, mom, hyper), stream=stream)
 
     def acc_topk_compress(self, grads, err, level, vals, idx, counts, delta, vec_packed, stream=None):
-        f = torch.float32
-        self._check(lib().acc_topk_compress(self._h, _ptr(grads, f), _ptr(err, f), _ptr(level, torch.uint8),
-                                            _ptr(vals, f), _ptr(idx, torch.int32), _ptr(counts, torch.int32),
-                                            _ptr(delta, f), _ptr(vec_packed, f), _stream(stream)),
-                    "acc_topk_compress")
+        self._call("acc_topk_compress", *self._topk_args(grads, err, level, vals, idx, counts),
+                   self._f(delta, self.stride, "delta"), self._f(vec_packed, self.vec_floats, "vec_packed"),
+                   stream=stream)
 
     def acc_topk_decompress(self, vals_all, idx_all, counts_all, n_sets, vec_packed, vec_scale, out, params=None,
                             mom=None, hyper=None, stream=None):
-        f = torch.float32
-        self._check(lib().acc_topk_decompress(self._h, _ptr(vals_all, f), _ptr(idx_all, torch.int32),
-                                              _ptr(counts_all, torch.int32), int(n_sets), _ptr(vec_packed, f),
-                                              float(vec_scale), _ptr(out, f), _ptr(params, f), _ptr(mom, f),
-                                              _ptr(hyper, f), _stream(stream)), "acc_topk_decompress")
+        n_sets = int(n_sets)
+        cap = max(n_sets, 0) * self.capacity
+        self._call("acc_topk_decompress", self._f(vals_all, cap, "vals_all"), self._i(idx_all, cap, "idx_all"),
+                   self._i(counts_all, max(n_sets, 0) * self.n_layers, "counts_all"), n_sets,
+                   self._f(vec_packed, self.vec_floats, "vec_packed"), float(vec_scale),
+                   self._f(out, self.stride, "out"), *self._tail(params, mom, hyper), stream=stream)
 
     def acc_topk_flush(self, err, stream=None):
-        self._check(lib().acc_topk_flush(self._h, _ptr(err, torch.float32), _stream(stream)), "acc_topk_flush")
+        self._call("acc_topk_flush", self._f(err, self._wn, "err"), stream=stream)
 
     def acc_upload_grads(self, grads_host, grads_dev, stream=None):
         """``grads_host``: CPU float32 tensor [W, stride] (pinned for an asynchronous copy)."""
         if grads_host.is_cuda or grads_host.dtype != torch.float32 or not grads_host.is_contiguous():
             raise ValueError("expected a contiguous float32 CPU tensor")
-        if grads_host.numel() != self.n_workers * self.stride or grads_dev.numel() != grads_host.numel():
+        if grads_host.numel() != self._wn or grads_dev.numel() != grads_host.numel():
             raise ValueError("expected [n_workers, worker_stride] elements")
-        self._check(lib().acc_upload_grads(self._h, grads_host.data_ptr(), _ptr(grads_dev, torch.float32),
-                                           _stream(stream)), "acc_upload_grads")
+        self._call("acc_upload_grads", grads_host.data_ptr(), self._f(grads_dev, self._wn, "grads_dev"),
+                   stream=stream)
 
     def acc_download_out(self, out_dev, out_host, stream=None):
         if out_host.is_cuda or out_host.dtype != torch.float32 or not out_host.is_contiguous():
             raise ValueError("expected a contiguous float32 CPU tensor")
         if out_host.numel() != self.stride or out_dev.numel() != self.stride:
             raise ValueError("expected worker_stride elements")
-        self._check(lib().acc_download_out(self._h, _ptr(out_dev, torch.float32), out_host.data_ptr(),
-                                           _stream(stream)), "acc_download_out")
+        self._call("acc_download_out", self._f(out_dev, self.stride, "out_dev"), out_host.data_ptr(),
+                   stream=stream)
 
     def acc_profile_enable(self, enable: bool):
         self._check(lib().acc_profile_enable(self._h, int(bool(enable))), "acc_profile_enable")

@@ -92,3 +92,76 @@ def test_bench_reference_arm_prints_the_contract_line():
     assert line["impl"] == "reference" and line["steps"] == 2 and line["value"] > 0
     assert line["cpu_baseline"]["kind"] == "oracle" and line["cpu_baseline"]["cores"] >= 1
     assert line["e2e"]["h2d_bytes_per_step"] == 0 and line["e2e"]["d2h_bytes_per_step"] == 0
+
+
+def _hostless_context(table, W):
+    """A binding.Context with the layout fields filled in by hand and no library handle: the argument checks run
+    (and must raise) before any call into the library, so they can be tested without a GPU."""
+    import torch
+    c = binding.Context.__new__(binding.Context)
+    c.table, c.device, c._h = table, torch.device("cuda", 0), None
+    c.n_workers, c.n_layers, c.stride = W, table.n_layers, table.stride
+    c.extent = int(max(int(table.offset[l]) + int(table.rows[l]) * int(table.cols[l]) for l in range(table.n_layers)))
+    mat = table.kind == wl.MATRIX
+    c.q_rows, c.p_rows = int(table.cols[mat].sum()), int(table.rows[mat].sum())
+    c.capacity = int(sum(max(1, int(s) // 10) for s in table.sizes[mat]))
+    c.x1_floats, c.x2_floats, c.vec_floats = 4 * c.p_rows + 8, 4 * c.q_rows, 8
+    return c
+
+
+def test_binding_rejects_short_or_misplaced_tensors_before_calling_the_library():
+    """The C ABI takes bare pointers, so a tensor shorter than the context's layout would become an out-of-bounds
+    device access.  The binding refuses it (and wrong dtypes, non-contiguous views, CPU tensors) with ValueError."""
+    import torch
+    table = wl.make_table([("a", (6, 10)), ("v", (5,)), ("b", (4, 8))])
+    W, L, S = 2, table.n_layers, table.stride
+    c = _hostless_context(table, W)
+    f = lambda n: torch.zeros(n)                                   # noqa: E731
+    level = torch.zeros(L, dtype=torch.uint8)
+    ok = dict(grads=f(W * S), err=f(W * S), q=f(4 * c.q_rows), p_hat=f(4 * c.p_rows), level=level, out=f(S))
+    # every argument one element short, in turn: the message names it
+    for name in ok:
+        short = dict(ok)
+        short[name] = ok[name][:-1].clone()
+        with pytest.raises(ValueError, match=name):
+            c.acc_powersgd_step(**short)
+    with pytest.raises(ValueError, match="delta"):
+        c.acc_powersgd_step(**ok, delta=f(S - 1))
+    # right sizes on the CPU: refused as "not a CUDA tensor", after the size checks passed
+    with pytest.raises(ValueError, match="CUDA"):
+        c.acc_powersgd_step(**ok)
+    with pytest.raises(ValueError, match="dtype"):
+        c.acc_powersgd_step(**{**ok, "grads": torch.zeros(W * S, dtype=torch.float64)})
+    with pytest.raises(ValueError, match="contiguous"):
+        c.acc_powersgd_step(**{**ok, "out": torch.zeros(2 * S)[::2]})
+    vals, idx = f(W * c.capacity), torch.zeros(W * c.capacity, dtype=torch.int32)
+    counts = torch.zeros(W * L, dtype=torch.int32)
+    with pytest.raises(ValueError, match="vals"):
+        c.acc_topk_step(ok["grads"], ok["err"], level, vals[:-1].clone(), idx, counts, ok["out"])
+    with pytest.raises(ValueError, match="idx"):
+        c.acc_topk_step(ok["grads"], ok["err"], level, vals, idx[:-1].clone(), counts, ok["out"])
+    with pytest.raises(ValueError, match="counts"):
+        c.acc_topk_step(ok["grads"], ok["err"], level, vals, idx, counts[:-1].clone(), ok["out"])
+    with pytest.raises(ValueError, match="level"):
+        c.acc_topk_step(ok["grads"], ok["err"], level[:-1].clone(), vals, idx, counts, ok["out"])
+    n2 = torch.zeros(L, dtype=torch.float64)
+    with pytest.raises(ValueError, match="norm2"):
+        c.acc_layer_norms(f(S), 1, n2[:-1].clone())
+    with pytest.raises(ValueError, match="buf"):
+        c.acc_layer_norms(f(S + c.extent - 1), 2, torch.zeros(2 * L, dtype=torch.float64))
+    with pytest.raises(ValueError, match="norm2_prev"):
+        c.acc_detect_regime(n2, n2[:-1].clone(), 0.1, 0.1, level)
+    with pytest.raises(ValueError, match="hyper"):
+        c.acc_sgd_nesterov(f(S), f(S), f(S), f(2))
+    with pytest.raises(ValueError, match="together"):
+        c.acc_batch_average(f(W * S), 2, f(S), params=f(S))
+    with pytest.raises(ValueError, match="x1"):
+        c.acc_powersgd_phase2(f(c.x1_floats - 1), 1.0, ok["p_hat"], level, ok["out"], f(c.x2_floats))
+    with pytest.raises(ValueError, match="vals_all"):
+        c.acc_topk_decompress(f(3 * c.capacity - 1), torch.zeros(3 * c.capacity, dtype=torch.int32),
+                              torch.zeros(3 * L, dtype=torch.int32), 3, f(8), 1.0, f(S))
+    # the entry point without a context: n may not exceed what the tensor holds
+    with pytest.raises(ValueError, match="buf"):
+        binding.acc_sumsq_static(f(64), 1000, torch.zeros(1, dtype=torch.float64))
+    with pytest.raises(ValueError, match="norm2"):
+        binding.acc_sumsq_static(f(64), 64, torch.zeros(0, dtype=torch.float64))
