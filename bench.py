@@ -29,7 +29,8 @@ import torch  # noqa: E402
 METRIC = "compression_step_gradient_throughput"
 UNIT = "GB/s"
 RING = 4  # pre-generated gradient batches cycled through the steps (each far larger than L2)
-REF_LAYER = "rnn.weight_hh_l0"
+NOMINAL_HBM_GBS = 8000.0     # the B200's nominal HBM3e bandwidth, the figure the target of this path is stated against
+SAMPLE_PARAM_WORKERS = 26e6  # size of the oracle's sample of the workload (parameter-workers per step)
 
 
 def _peaks():
@@ -110,73 +111,118 @@ def _kernel_alg_bytes(name, units, n_workers=None, carries_delta=()):
     return b * units
 
 
+def oracle_sample(w, device):
+    """A bounded sample of workload ``w`` for the CPU oracle: every layer cut to its first rows (1/s of them, s the
+    smallest power of two that brings W x parameters under SAMPLE_PARAM_WORKERS), filled from the workload's own
+    gradient stream (iterations 0 and 1, the values the GPU arm sees), so the sample keeps the layer mix, the value
+    distributions and the row-sparse encoder of the full set.  Returns (sub-table, layer tuples, batches, text)."""
+    from paper_2010_16248_b200 import workloads as wl
+    full, W = w.table, w.n_workers
+    s = 1
+    while W * full.n_params / s > SAMPLE_PARAM_WORKERS:
+        s *= 2
+    shapes = []
+    for l in range(full.n_layers):
+        n, m = int(full.rows[l]), int(full.cols[l])
+        if full.kind[l] == wl.MATRIX:
+            shapes.append((full.names[l], (max(min(n, 4), -(-n // s)), m)))
+        else:
+            shapes.append((full.names[l], (max(1, m // s),)))
+    sub = wl.make_table(shapes)
+    gen = wl.GradientStream(w, device=device)
+    batches = []
+    for t in range(2):
+        g = gen.grads(t)
+        b = np.zeros((W, sub.stride), np.float32)
+        for l in range(sub.n_layers):
+            size = int(sub.rows[l]) * int(sub.cols[l])
+            o_full, o_sub = int(full.offset[l]), int(sub.offset[l])
+            b[:, o_sub:o_sub + size] = g[:, o_full:o_full + size].cpu().numpy()
+        batches.append(b)
+        del g
+    cut = "every layer whole" if s == 1 else f"the first 1/{s} of the rows of every layer"
+    text = (f"{w.name}: {cut} ({sub.n_params} of {full.n_params} parameters, all {W} workers, a row-sparse layer "
+            f"included where the set has one), gradients of iterations 0 and 1 of the workload's own stream, every "
+            f"compressor of the workload per step")
+    return sub, batches, text
+
+
 def run_reference(args, rank, world):
-    """Times the CPU oracle, as it stands, on a bounded sample of the workload (one LSTM gate matrix
-    with all workers, both compressors)."""
+    """Times the CPU oracle, as it stands, on a bounded sample of the workload (see ``oracle_sample``): with the
+    host's default thread pool for the K timed steps, and single-threaded on a few more.  The oracle's products
+    run in the BLAS pool; its sort (the TopK half) is one thread whatever the pool size."""
     if rank != 0:
         return
     from oracle import accordion_oracle as orc
     from paper_2010_16248_b200 import workloads as wl
     w = wl.workload(args.config)
-    full = w.table
-    li = full.names.index(REF_LAYER) if REF_LAYER in full.names else int(np.argmax(full.kind == wl.MATRIX))
-    n, m = int(full.rows[li]), int(full.cols[li])
-    sub = wl.make_table([(full.names[li], (n, m))])
+    dev = "cuda" if torch.cuda.is_available() else "cpu"
+    sub, batches, sample = oracle_sample(w, dev)
     layers = [(int(sub.offset[l]), int(sub.rows[l]), int(sub.cols[l]), int(sub.kind[l])) for l in range(sub.n_layers)]
-    rng = np.random.default_rng(1234)
     W = w.n_workers
-    batches = [rng.standard_normal((W, sub.stride)).astype(np.float32) for _ in range(2)]
-    err_p = np.zeros((W, sub.stride), np.float32)
-    err_t = np.zeros((W, sub.stride), np.float32)
-    q = [rng.standard_normal((m, w.rank_low)).astype(np.float32)]
-    level = np.ones(1, np.uint8)
-    delta = np.zeros(sub.stride)
-    prev = -np.ones(1)
+    q0 = [None if x is None else x.numpy() for x in wl.initial_q(sub, w.rank_low)]
+    state = {}
+
+    def reset():
+        state.update(err_p=np.zeros((W, sub.stride), np.float32), err_t=np.zeros((W, sub.stride), np.float32),
+                     q=[None if x is None else x.copy() for x in q0], level=np.ones(sub.n_layers, np.uint8),
+                     delta=np.zeros(sub.stride), prev=-np.ones(sub.n_layers))
 
     def step(t):
-        nonlocal err_p, err_t, q, level, prev
         g = batches[t % 2]
-        orc.accumulate(delta, g[0], layers)
+        orc.accumulate(state["delta"], g[0], layers)
         n_comp = 0
         if "powersgd" in w.compressors:
-            _, e, qn, _ = orc.powersgd_step(g, err_p, q, level, layers, w.rank_low, w.rank_high)
-            err_p, q = e.astype(np.float32), [x.astype(np.float32) for x in qn]
+            _, e, qn, _ = orc.powersgd_step(g, state["err_p"], state["q"], state["level"], layers, w.rank_low,
+                                            w.rank_high)
+            state["err_p"] = e.astype(np.float32)
+            state["q"] = [None if x is None else x.astype(np.float32) for x in qn]
             n_comp += 1
         if "topk" in w.compressors:
-            _, _, _, _, err_t = orc.topk_step(g, err_t, level, layers, w.topk_low_bp, w.topk_high_bp)
+            _, _, _, _, state["err_t"] = orc.topk_step(g, state["err_t"], state["level"], layers, w.topk_low_bp,
+                                                       w.topk_high_bp)
             n_comp += 1
         if (t + 1) % w.check_every == 0:
-            level, prev = orc.detect_regime(orc.layer_norms2(delta, layers), prev, 0.1, 0.1, w.eta)
-            delta[:] = 0
+            state["level"], state["prev"] = orc.detect_regime(orc.layer_norms2(state["delta"], layers), state["prev"],
+                                                              0.1, 0.1, w.eta)
+            state["delta"][:] = 0
         return n_comp
 
-    for t in range(args.warmup):
-        step(t)
-    t0 = time.perf_counter()
-    n_comp = 0
-    for t in range(args.steps):
-        n_comp = step(args.warmup + t)
-    dt = time.perf_counter() - t0
-    bytes_per_step = n_comp * 4.0 * W * n * m
-    value = bytes_per_step * args.steps / dt / 1e9
+    def timed(k, warm):
+        reset()
+        for t in range(warm):
+            step(t)
+        t0 = time.perf_counter()
+        n = 0
+        for t in range(k):
+            n = step(warm + t)
+        dt = time.perf_counter() - t0
+        return n * 4.0 * W * sub.n_params * k / dt / 1e9, dt / k * 1e3
+
+    value, ms = timed(args.steps, args.warmup)
+    cores, value_1 = 1, None
     try:
-        from threadpoolctl import threadpool_info
+        from threadpoolctl import threadpool_info, threadpool_limits
         cores = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+        with threadpool_limits(limits=1):
+            value_1, _ = timed(min(2, args.steps), 1)
     except Exception:
-        cores = 1
-    sample = f"layer {full.names[li]} ({n}x{m}) of {w.name}, all {W} workers, {n_comp} compressor passes per step"
+        pass
+    cpu = {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample,
+           "value_single_thread": value_1,
+           "threads": f"{cores} BLAS threads for the oracle's matrix products; its sort (TopK) runs on one thread"}
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
-            "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
             "config": {"workload": w.name, "sample": sample},
-            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "cpu_baseline": cpu,
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
     print(json.dumps(line), flush=True)
 
 
-def cpu_baseline(w, seconds_budget=20.0):
-    """The oracle timed on the host cores on a bounded sample (same sample as --impl reference)."""
+def cpu_baseline(w):
+    """The oracle timed on the host cores on a bounded sample of the workload (the --impl reference leg, 3 steps)."""
     ns = argparse.Namespace(config=w.config_id, warmup=1, steps=3, gpus=1)
     import io
     from contextlib import redirect_stdout
@@ -184,6 +230,18 @@ def cpu_baseline(w, seconds_budget=20.0):
     with redirect_stdout(buf):
         run_reference(ns, 0, 1)
     return json.loads(buf.getvalue().strip().splitlines()[-1])["cpu_baseline"]
+
+
+def respawn_under_torchrun(n):
+    """``--gpus N`` given to a plain ``python bench.py``: start N ranks, one per GPU, under torch.distributed.run
+    on this node, with the same arguments, and hand their output and exit code through."""
+    import socket
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
 
 
 def main():
@@ -212,15 +270,22 @@ def main():
                          "GPUs (all-reduce of P and Q, all-gather of the packed TopK sets) instead of independent "
                          "replicas; at --gpus 1 the collectives are the identity")
     ap.add_argument("--n-accum", type=int, default=8, help="--batch-mode: micro-batches per step (B_high / micro-batch)")
+    ap.add_argument("--force-level", default="auto", choices=["auto", "low", "high"],
+                    help="auto: the detector sets the per-layer levels (the method as it runs); low / high: every "
+                         "layer held at that compression level for the whole run (the detector still runs)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
+    if args.impl == "reference":  # the oracle on the host cores: rank 0 alone works, whatever N
+        run_reference(args, int(os.environ.get("RANK", "0")), int(os.environ.get("WORLD_SIZE", "1")))
+        return
+    if "WORLD_SIZE" not in os.environ and args.gpus > 1:
+        sys.exit(respawn_under_torchrun(args.gpus))
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    if args.impl == "reference":
-        run_reference(args, rank, world)
-        return
+    if world != max(args.gpus, 1):
+        raise SystemExit(f"--gpus {args.gpus} but the launcher started {world} rank(s)")
 
     import torch.distributed as dist
     from paper_2010_16248_b200 import build, dist_util, pipeline, workloads as wl
@@ -265,9 +330,19 @@ def main():
     step_no = 0
 
     use_graphs = not args.no_graphs
+    force = {"auto": None, "low": 1, "high": 0}[args.force_level]
+    if force is not None:
+        eng.level.fill_(force)
+    # the per-layer levels in force during each step, for the per-regime report: the array only changes at a regime
+    # check, so a copy is kept (device to device, read back after the timed region) whenever one has run
+    level_log = torch.zeros(args.steps // max(w.check_every, 1) + 2, table.n_layers, dtype=torch.uint8, device=dev)
+    level_from = []  # (first timed step a logged row applies to, row)
 
-    def run_steps(k, events=None, graphs=False):
+    def run_steps(k, events=None, graphs=False, log=False):
         nonlocal step_no
+        if log:
+            level_log[0].copy_(eng.level)
+            level_from.append((0, 0))
         for i in range(k):
             if events is not None:
                 events[i][0].record()
@@ -278,6 +353,12 @@ def main():
             if events is not None:
                 events[i][1].record()
             step_no += 1
+            if eng.t % w.check_every == 0:
+                if force is not None:
+                    eng.level.fill_(force)
+                if log:
+                    level_log[len(level_from)].copy_(eng.level)
+                    level_from.append((i + 1, len(level_from)))
 
     # ---- warm-up, then the timed region (device-resident inputs)
     run_steps(args.warmup)
@@ -295,7 +376,7 @@ def main():
     t0 = time.time()
     start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     start.record()
-    run_steps(K, ev, graphs=use_graphs)
+    run_steps(K, ev, graphs=use_graphs, log=True)
     stop.record()
     barrier()
     t1 = time.time()
@@ -303,6 +384,15 @@ def main():
     total_ms = start.elapsed_time(stop)
     gpu_launches = eng.launches - launches0
     per_step = np.array([a.elapsed_time(b) for a, b in ev])
+    # regime of every timed step: share of the MATRIX parameters whose layer was at the low compression level
+    log_host = level_log.cpu().numpy()
+    mat = table.kind == wl.MATRIX
+    weight = table.sizes[mat] / table.sizes[mat].sum()
+    regime = []
+    for i in range(K):
+        row = [r for (first, r) in level_from if first <= i][-1]
+        share = float((log_host[row][mat] * weight).sum())
+        regime.append("low" if share > 1 - 1e-9 else "high" if share < 1e-9 else "mixed")
     total_ms = dist_util.max_over_ranks(total_ms, dev)
     ms_per_step = total_ms / K
     value = dist_util.whole_job_throughput(grad_bytes_step, ms_per_step, world) / 1e9
@@ -318,6 +408,20 @@ def main():
     eng.overlap = overlap
     peak, peak_src = _peaks()
     units = W * n_mat
+    compulsory = n_comp * 12.0 * units  # bytes a step must move: read g, read e, write e', per compressor
+
+    def step_fracs(ms):
+        gbs = compulsory / (ms * 1e-3) / 1e9
+        return {"of_measured_copy_peak": round(gbs / peak, 4), "of_nominal_8TBs": round(gbs / NOMINAL_HBM_GBS, 4)}
+
+    by_regime = {}
+    for name in ("low", "high", "mixed"):
+        ts = per_step[[r == name for r in regime]]
+        if len(ts):
+            by_regime[name] = {"steps": int(len(ts)), "median_ms": round(float(np.median(ts)), 4),
+                               "min_ms": round(float(ts.min()), 4), "max_ms": round(float(ts.max()), 4),
+                               "gradient_gbs": round(grad_bytes_step / (float(np.median(ts)) * 1e-3) / 1e9, 1),
+                               "frac_of_12B": step_fracs(float(np.median(ts)))}
     total_k_ms = sum(ms for ms, _ in prof.values())
     kernels = {}
     # the first compressor of the step carries the detector's accumulation in its first pass
@@ -336,11 +440,14 @@ def main():
     dom_avg_ms = prof[dom][0] / prof[dom][1]
     achieved = dom_alg / (dom_avg_ms * 1e-3) / 1e9
     roofline = {"bound": "hbm", "kernel": dom, "achieved": round(achieved, 1), "peak": peak, "unit": "GB/s",
-                "frac": round(achieved / peak, 4), "peak_source": peak_src, "traffic": (TRAFFIC_PER_UNIT[dom] * units if dom in TRAFFIC_PER_UNIT else None),
+                "frac": round(achieved / peak, 4), "peak_source": peak_src,
+                "peak_nominal": NOMINAL_HBM_GBS, "frac_of_nominal": round(achieved / NOMINAL_HBM_GBS, 4),
+                "traffic": (TRAFFIC_PER_UNIT[dom] * units if dom in TRAFFIC_PER_UNIT else None),
                 "traffic_source": TRAFFIC_SOURCE.get(dom),
                 "alg_bytes_per_launch": dom_alg, "alg_bytes_per_unit": round(dom_alg / units, 3),
                 "frac_with_detector_bytes": round(dom_alg_delta / (dom_avg_ms * 1e-3) / 1e9 / peak, 4),
-                "step_frac_of_12B": round(n_comp * 12.0 * units / (ms_per_step * 1e-3) / 1e9 / peak, 4)}
+                "step_frac_of_12B": step_fracs(ms_per_step)["of_measured_copy_peak"],
+                "step_frac_of_12B_nominal": step_fracs(ms_per_step)["of_nominal_8TBs"]}
 
     # ---- end to end: host (pinned) gradients -> device every step, results read back to the host.
     # Uploads run on a copy stream into two staging buffers and overlap the previous step's kernels.
@@ -384,6 +491,10 @@ def main():
                            "l2_policy": f"inputs larger than L2: {RING} gradient batches of "
                                         f"{4 * W * table.stride / 1e6:.0f} MB cycled, no flush",
                            "launch": "CUDA graph replay per step" if use_graphs else "direct calls",
+                           "levels": ("set by the detector" if force is None else
+                                      f"every layer held at the {args.force_level} compression level"),
+                           "regime_of_value": ", ".join(f"{v['steps']} of {K} timed steps at {k}"
+                                                        for k, v in by_regime.items()),
                            "streams": ("TopK step beside the PowerSGD step on a second stream"
                                        if (n_comp == 2 and not args.no_overlap) else "one stream"),
                            "multi_gpu": "independent replicas, no collective"},
@@ -391,6 +502,7 @@ def main():
                 "roofline": roofline, "cpu_baseline": cpu,
                 "step_ms": {"median": float(np.median(per_step)), "min": float(per_step.min()),
                             "max": float(per_step.max())},
+                "step_ms_by_regime": by_regime,
                 "kernels": kernels}
         print(json.dumps(line), flush=True)
     if world > 1:
@@ -652,8 +764,8 @@ def run_real_workers(args, w, ring, dev, rank, world, local_rank):
 # summarised under profiles/; a launch's traffic is this figure times the units it processes (the kernels
 # stream every element once, so traffic grows in proportion).
 TRAFFIC_PER_UNIT = {"psgd_project_kernel": 13.15, "topk_ef_hist1_kernel": 12.92}
-TRAFFIC_SOURCE = {"psgd_project_kernel": "ncu on config 4 (profiles/psgd_project_kernel_config4_traffic.md), scaled by units",
-                  "topk_ef_hist1_kernel": "ncu on config 3 (profiles/topk_kernels_config3_resnet18.md), scaled by units"}
+TRAFFIC_SOURCE = {"psgd_project_kernel": "ncu capture of the direct kernel on config 4, scaled by units",
+                  "topk_ef_hist1_kernel": "ncu capture on config 3, scaled by units"}
 
 if __name__ == "__main__":
     main()

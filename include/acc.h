@@ -125,6 +125,19 @@ int acc_error_feedback(acc_ctx* ctx, const float* grads, float* err, float* delt
 int acc_layer_norms(acc_ctx* ctx, const float* buf, int64_t buf_stride, int32_t n_bufs, double* norm2,
                     void* stream);
 
+/* Second detector statistic: the mean-to-standard-deviation ratio (MSDR) per layer, the quantity the adaptive scheme
+ * of the Section "Comparison with Prior Work" switches on (that scheme lowers the compression when the ratio of its
+ * gradients has dropped; the paper names the statistic and no formula).  Taken over the coordinates of a layer:
+ *   S1 = sum_i x_i, S2 = sum_i x_i^2 (fp64, fixed order);  mean = S1/n;  var = max(S2/n - mean^2, 0);
+ *   msdr = |mean| / sqrt(var), 0 when mean = 0, +inf when var = 0 and mean != 0.
+ *   moments[2*(b*L + l)] = S1, moments[2*(b*L + l) + 1] = S2 (= the squared norm acc_layer_norms returns, so one pass
+ *   over the detector's accumulated gradient serves Algorithm 1 and this statistic);  msdr[b*L + l].
+ * Only the statistic is built; the switching rule of that scheme is not.
+ * Device pointers: buf [n_bufs][buf_stride] (read), moments [2*n_bufs*L] doubles, msdr [n_bufs*L] doubles (written);
+ * n_bufs <= W.                                                                                       */
+int acc_layer_msdr(acc_ctx* ctx, const float* buf, int64_t buf_stride, int32_t n_bufs, double* moments, double* msdr,
+                   void* stream);
+
 /* Critical-regime test, Algorithm 1, per layer, on the device:
  *   a = sqrt(norm2_prev[l]), b = sqrt(norm2_curr[l]);
  *   level[l] = 1 (l_low)  if norm2_prev[l] < 0 (no earlier window), or |a - b| >= eta*a, or
@@ -309,13 +322,16 @@ int acc_reset_device_status(acc_ctx* ctx, void* stream);
 /* Diagnostic (no counterpart in the paper): which selection path the last acc_topk_step took for every
  * (worker, MATRIX layer) pair, in worker-major order, n >= W * (number of MATRIX layers) HOST ints:
  *   0 dense (levels 2-3 of the radix select read M), 1 list built by the collect pass, 2 list built by the
- *   first pass from a held prediction, 3 whole entries staged by the first pass (M not read again).
+ *   first pass from a held prediction, 3 whole entries staged by the first pass (M not read again),
+ *   4 zero fill (k exceeds the non-zero entries, e.g. a row-sparse embedding gradient at a large K: the threshold
+ *   is 0, every non-zero is kept and the zeros of lowest index fill up; settled from counts of the first pass).
  * Blocks until the device has finished the queued work.  All paths give identical results; tests use
  * this to make sure each one is exercised.                                                          */
 #define ACC_TOPK_PATH_DENSE 0
 #define ACC_TOPK_PATH_LIST 1
 #define ACC_TOPK_PATH_LIST_PREDICTED 2
 #define ACC_TOPK_PATH_STAGED 3
+#define ACC_TOPK_PATH_ZERO_FILL 4
 int acc_topk_last_paths(acc_ctx* ctx, int32_t* paths, int32_t n);
 
 /* Floats one iteration communicates at the given HOST level array, following the "Data Sent"

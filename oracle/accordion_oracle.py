@@ -101,6 +101,33 @@ def detect_regime_diff(norm2_diff, norm2_curr, norm2_prev, lr_curr, lr_next, eta
     return level, np.array(norm2_curr, np.float64, copy=True)
 
 
+def layer_msdr(buf, layers):
+    """Mean-to-standard-deviation ratio of each layer of one flat buffer: the statistic of the adaptive scheme
+    the paper compares itself with (Section 6, "Comparison with Prior Work"), which lowers the compression when
+    the ratio has dropped.  The paper names the statistic only; taken here over the coordinates of a layer of
+    the detector's accumulated gradient:
+
+        mu = (1/n) sum_i x_i,   sd = sqrt((1/n) sum_i (x_i - mu)^2),   MSDR = |mu| / sd
+
+    with MSDR = 0 when mu = 0 (also for an all-zero layer) and +inf when sd = 0 but mu != 0 (a constant layer).
+    Returns (msdr[L], mean[L], std[L]) in fp64."""
+    L = len(layers)
+    msdr, mean, std = np.zeros(L), np.zeros(L), np.zeros(L)
+    for l, (off, rows, cols, kind) in enumerate(layers):
+        x = buf[off:off + rows * cols].astype(np.float64)
+        mu = float(np.sum(x)) / x.size
+        d = x - mu
+        sd = float(np.sqrt(np.sum(d * d) / x.size))
+        mean[l], std[l] = mu, sd
+        if mu == 0.0:
+            msdr[l] = 0.0
+        elif sd == 0.0:
+            msdr[l] = np.inf
+        else:
+            msdr[l] = abs(mu) / sd
+    return msdr, mean, std
+
+
 # --------------------------------------------------------------------------- #
 # Error feedback (the "memory term", Section 5.2 / Appendix A)
 # --------------------------------------------------------------------------- #

@@ -22,6 +22,7 @@ ACC_FLAG_LAZY_RESIDUAL = 1
 ACC_FLAG_PIPELINE_ALWAYS = 2
 ACC_FLAG_PIPELINE_NEVER = 4
 POWERSGD, TOPK = 0, 1
+ACC_TOPK_PATH_DENSE, ACC_TOPK_PATH_LIST, ACC_TOPK_PATH_LIST_PREDICTED, ACC_TOPK_PATH_STAGED, ACC_TOPK_PATH_ZERO_FILL = range(5)
 
 
 class AccError(RuntimeError):
@@ -50,7 +51,8 @@ EXPORTS = ["acc_workspace_bytes", "acc_create", "acc_destroy", "acc_factor_layou
            "acc_topk_step_sgd", "acc_batch_accumulate", "acc_batch_average", "acc_detect_batch",
            "acc_exchange_layout", "acc_powersgd_phase1", "acc_powersgd_phase2", "acc_powersgd_phase3",
            "acc_topk_compress", "acc_topk_decompress", "acc_topk_flush",
-           "acc_upload_grads", "acc_download_out", "acc_selftest_wait_timeout", "acc_reset_device_status"]
+           "acc_upload_grads", "acc_download_out", "acc_selftest_wait_timeout", "acc_reset_device_status",
+           "acc_layer_msdr"]
 
 _lib = None
 
@@ -73,6 +75,7 @@ def lib() -> C.CDLL:
     L.acc_topk_layout.argtypes = [vp, C.POINTER(i64), C.POINTER(i64), C.POINTER(i64), C.POINTER(i64)]
     L.acc_error_feedback.argtypes = [vp, vp, vp, vp, vp]
     L.acc_layer_norms.argtypes = [vp, vp, i64, i32, vp, vp]
+    L.acc_layer_msdr.argtypes = [vp, vp, i64, i32, vp, vp, vp]
     L.acc_detect_regime.argtypes = [vp, vp, vp, f32, f32, vp, vp, vp]
     L.acc_powersgd_step.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp]
     L.acc_topk_step.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
@@ -291,6 +294,14 @@ class Context:
         need = (n_bufs - 1) * stride + self.extent if n_bufs >= 1 else 0
         self._call("acc_layer_norms", self._f(buf, need, "buf"), stride, n_bufs,
                    self._d(norm2, max(n_bufs, 0) * self.n_layers, "norm2"), stream=stream)
+
+    def acc_layer_msdr(self, buf, n_bufs, moments, msdr, buf_stride=None, stream=None):
+        stride = int(buf_stride if buf_stride is not None else self.stride)
+        n_bufs = int(n_bufs)
+        need = (n_bufs - 1) * stride + self.extent if n_bufs >= 1 else 0
+        self._call("acc_layer_msdr", self._f(buf, need, "buf"), stride, n_bufs,
+                   self._d(moments, 2 * max(n_bufs, 0) * self.n_layers, "moments"),
+                   self._d(msdr, max(n_bufs, 0) * self.n_layers, "msdr"), stream=stream)
 
     def acc_detect_regime(self, norm2_curr, norm2_prev, lr_curr, lr_next, level, delta=None, stream=None):
         L = self.n_layers

@@ -113,7 +113,7 @@ static int make_plan(const acc_config* cfg, Plan& p) {
   p.o_part = take(sizeof(float4) * std::max<long long>(1, p.part_f4));
   p.o_ppart = take(sizeof(float4) * std::max<long long>(1, p.ppart_f4));
   p.o_pending = take(sizeof(int) * L);
-  p.o_norm_part = take(sizeof(double) * (size_t)W * nt);
+  p.o_norm_part = take(sizeof(double) * 2 * (size_t)W * nt);  // per (buffer, tile): sum of squares, or (sum, sum of squares)
   p.o_hist = o;
   take(sizeof(unsigned) * seg * kBins1);
   take(sizeof(unsigned) * seg * kBins2);
@@ -121,12 +121,12 @@ static int make_plan(const acc_config* cfg, Plan& p) {
   take(sizeof(unsigned) * seg);  // candidate counters, cleared with the histograms
   take(sizeof(unsigned) * seg);  // overflow flags of the predicted collection, likewise
   take(sizeof(unsigned) * 64);   // "some segment needs the collect pass" flag, likewise
+  p.o_tile_cnt = take(sizeof(int2) * (size_t)W * nt);  // per-tile counters (atomically added to), likewise
   p.hist_bytes = o - p.o_hist;
   p.o_sel = take(sizeof(Select) * seg);
   p.o_pred = take(sizeof(unsigned) * 6 * seg);  // [2] prediction words, [2] last buckets, [2] last moves, per level
   p.o_cand = take(sizeof(unsigned) * (size_t)W * std::max<long long>(1, p.cand_total));
   p.o_tile_cand = take(sizeof(int2) * (size_t)W * nt);
-  p.o_tile_cnt = take(sizeof(int2) * (size_t)W * nt);
   p.o_tile_h3 = take(sizeof(unsigned short) * (size_t)W * nt * kBins3);
   p.o_tile_pre = take(sizeof(int2) * (size_t)W * nt);
   p.o_lists = take(sizeof(int2) * (size_t)kNumLists * W * nt);
@@ -264,6 +264,17 @@ int acc_layer_norms(acc_ctx* ctx, const float* buf, int64_t buf_stride, int32_t 
   if (!aligned16(buf) || (n_bufs > 1 && buf_stride % 4 != 0) || (reinterpret_cast<uintptr_t>(norm2) & 7u)) return ACC_EALIGN;
   ctx->last_launches = 0;
   return finish(launch_layer_norms(ctx, buf, buf_stride, n_bufs, nullptr, norm2, static_cast<cudaStream_t>(stream)));
+}
+
+int acc_layer_msdr(acc_ctx* ctx, const float* buf, int64_t buf_stride, int32_t n_bufs, double* moments, double* msdr,
+                   void* stream) {
+  if (!ctx || !buf || !moments || !msdr || n_bufs < 1 || n_bufs > ctx->cfg.n_workers) return ACC_EINVAL;
+  if (n_bufs > 1 && buf_stride < ctx->cfg.worker_stride) return ACC_EINVAL;
+  if (!aligned16(buf) || (n_bufs > 1 && buf_stride % 4 != 0) || (reinterpret_cast<uintptr_t>(moments) & 7u) ||
+      (reinterpret_cast<uintptr_t>(msdr) & 7u))
+    return ACC_EALIGN;
+  ctx->last_launches = 0;
+  return finish(launch_layer_msdr(ctx, buf, buf_stride, n_bufs, moments, msdr, static_cast<cudaStream_t>(stream)));
 }
 
 int acc_layer_diff_norms(acc_ctx* ctx, const float* a, const float* b, double* norm2, void* stream) {
@@ -550,7 +561,7 @@ const char* acc_profile_kernel_name(int32_t i) {
       "topk_hist2_list_kernel", "topk_hist3_list_kernel", "topk_finalize_staged_kernel",
       "psgd_orthonormalise_block_kernel", "sgd_tiles_kernel", "batch_accumulate_kernel", "batch_average_kernel",
       "detect_batch_kernel", "psgd_pfold_kernel", "vec_exchange_kernel", "psgd_qmerge_kernel",
-      "topk_decompress_packed_kernel", "topk_flush_kernel"};
+      "topk_decompress_packed_kernel", "topk_flush_kernel", "moments_partial_kernel", "moments_final_kernel"};
   return (i >= 0 && i < PH_COUNT) ? names[i] : "";
 }
 

@@ -101,6 +101,67 @@ __global__ void norm_final_kernel(const DevLayer* __restrict__ layers, const dou
   if (threadIdx.x == 0) norm2[(long long)b * n_layers + l] = acc;
 }
 
+// One block per (tile, buffer): fp64 sum and sum of squares of the tile (the two moments behind the
+// mean-to-standard-deviation ratio; the sum of squares is also the tile's share of the layer norm of Section 4.2),
+// reduced in a fixed order.  part holds [buffer][tile][2].
+__global__ void __launch_bounds__(256) moments_partial_kernel(const DevLayer* __restrict__ layers,
+                                                              const Tile* __restrict__ tiles,
+                                                              const float* __restrict__ buf, long long stride,
+                                                              double* __restrict__ part, int n_tiles) {
+  __shared__ double sm[2][8];
+  const Tile t = tiles[blockIdx.x];
+  const int b = blockIdx.y;
+  const float* x = buf + (long long)b * stride + layers[t.layer].offset + t.elem0;
+  double s1 = 0.0, s2 = 0.0;
+  const int n4 = t.nelem >> 2;
+  for (int i = threadIdx.x; i < n4; i += blockDim.x) {
+    const float4 v = ld_stream4(x + 4 * i);
+    s1 += (double)v.x; s2 += (double)v.x * v.x;
+    s1 += (double)v.y; s2 += (double)v.y * v.y;
+    s1 += (double)v.z; s2 += (double)v.z * v.z;
+    s1 += (double)v.w; s2 += (double)v.w * v.w;
+  }
+  for (int i = 4 * n4 + threadIdx.x; i < t.nelem; i += blockDim.x) {
+    const float v = x[i];
+    s1 += (double)v; s2 += (double)v * v;
+  }
+  s1 = warp_sum(s1);
+  s2 = warp_sum(s2);
+  if ((threadIdx.x & 31) == 0) { sm[0][threadIdx.x >> 5] = s1; sm[1][threadIdx.x >> 5] = s2; }
+  __syncthreads();
+  if (threadIdx.x < 2) {
+    double s = 0.0;
+    for (int i = 0; i < (int)(blockDim.x >> 5); ++i) s += sm[threadIdx.x][i];
+    part[2 * ((long long)b * n_tiles + blockIdx.x) + threadIdx.x] = s;
+  }
+}
+
+// One warp per (layer, buffer): the layer's moments from its tile partials in a fixed order, then
+//   mean = S1 / n,  var = max(S2 / n - mean^2, 0),  msdr = |mean| / sqrt(var)   (0 when mean = 0, +inf when var = 0).
+__global__ void moments_final_kernel(const DevLayer* __restrict__ layers, const double* __restrict__ part,
+                                     double* __restrict__ moments, double* __restrict__ msdr, int n_layers,
+                                     int n_tiles) {
+  const int l = blockIdx.x, b = blockIdx.y;
+  const DevLayer L = layers[l];
+  double s1 = 0.0, s2 = 0.0;
+  for (int i = threadIdx.x; i < L.ntiles; i += 32) {
+    const double* p = part + 2 * ((long long)b * n_tiles + L.tile0 + i);
+    s1 += p[0]; s2 += p[1];
+  }
+  s1 = warp_sum(s1);
+  s2 = warp_sum(s2);
+  if (threadIdx.x == 0) {
+    const double n = (double)L.rows * (double)L.cols;
+    const double mean = s1 / n;
+    double var = s2 / n - mean * mean;
+    var = var > 0.0 ? var : 0.0;
+    const long long o = (long long)b * n_layers + l;
+    moments[2 * o] = s1;
+    moments[2 * o + 1] = s2;
+    msdr[o] = mean == 0.0 ? 0.0 : fabs(mean) / sqrt(var);  // var == 0: +inf
+  }
+}
+
 // Algorithm 1 per layer, in product form so that a zero previous norm needs no division.
 // With n2d (squared norms of the difference of the two accumulated gradients) the variant criterion
 // ||D_prev - D_curr|| >= eta ||D_prev|| is used instead of | ||D_prev|| - ||D_curr|| | >= eta ||D_prev||.
@@ -144,6 +205,22 @@ cudaError_t launch_layer_norms(acc_ctx* ctx, const float* buf, long long stride,
     PhaseTimer pt(ctx, PH_NORM_FINAL, s);
     norm_final_kernel<<<dim3((unsigned)ctx->cfg.n_layers, (unsigned)n_bufs), 32, 0, s>>>(
         ctx->d_layers, ctx->d_norm_part, norm2, ctx->cfg.n_layers, nt);
+  }
+  return cudaGetLastError();
+}
+
+cudaError_t launch_layer_msdr(acc_ctx* ctx, const float* buf, long long stride, int n_bufs, double* moments,
+                              double* msdr, cudaStream_t s) {
+  const int nt = (int)ctx->plan.tiles.size();
+  {
+    PhaseTimer pt(ctx, PH_MOMENTS_PARTIAL, s);
+    moments_partial_kernel<<<dim3((unsigned)nt, (unsigned)n_bufs), 256, 0, s>>>(ctx->d_layers, ctx->d_tiles, buf,
+                                                                               stride, ctx->d_norm_part, nt);
+  }
+  {
+    PhaseTimer pt(ctx, PH_MOMENTS_FINAL, s);
+    moments_final_kernel<<<dim3((unsigned)ctx->cfg.n_layers, (unsigned)n_bufs), 32, 0, s>>>(
+        ctx->d_layers, ctx->d_norm_part, moments, msdr, ctx->cfg.n_layers, nt);
   }
   return cudaGetLastError();
 }

@@ -47,8 +47,9 @@ struct Select {
   int k, k1, k2, need;  // k wanted; still wanted inside bucket b1 / (b1,b2); ties (key == tau) to keep
   int mode;             // kSelDense: levels 2-3 read M;  kSelList: they read the collected keys of bucket b1
 };
-constexpr int kSelDense = 0, kSelList = 1, kSelListPred = 2, kSelStaged = 3;
-// ListPred: the key list was filled by pass A;  Staged: pass A staged whole (value, index) entries
+constexpr int kSelDense = 0, kSelList = 1, kSelListPred = 2, kSelStaged = 3, kSelZeroFill = 4;
+// ListPred: the key list was filled by pass A;  Staged: pass A staged whole (value, index) entries;
+// ZeroFill: the threshold is 0 (k exceeds the non-zero entries): settled from the first pass's per-tile counts
 // Work lists of (worker, tile) pairs, rebuilt every step on the device, so that the passes that serve only some
 // segments launch as many blocks as there is work: tiles of segments whose bucket is collected by the collect
 // pass, tiles of dense segments, tiles the select pass must read, tiles served from staged entries.
@@ -64,6 +65,7 @@ enum Phase {
   PH_TOPK_EF_HIST1, PH_TOPK_PICK1, PH_TOPK_HIST2, PH_TOPK_PICK2, PH_TOPK_HIST3, PH_TOPK_PICK3_SCAN, PH_TOPK_SELECT,
   PH_TOPK_DECOMPRESS, PH_PSGD_FLUSH, PH_TOPK_COLLECT, PH_TOPK_PICK3, PH_TOPK_TILE_COUNTS, PH_TOPK_HIST2_LIST, PH_TOPK_HIST3_LIST, PH_TOPK_FINALIZE_STAGED, PH_PSGD_ORTHO_BLOCK, PH_SGD_TILES, PH_BATCH_ACCUMULATE, PH_BATCH_AVERAGE, PH_DETECT_BATCH,
   PH_PSGD_PFOLD, PH_VEC_EXCHANGE, PH_PSGD_QMERGE, PH_TOPK_DECOMPRESS_PACKED, PH_TOPK_FLUSH,
+  PH_MOMENTS_PARTIAL, PH_MOMENTS_FINAL,
   PH_COUNT
 };
 
@@ -142,6 +144,8 @@ struct SgdTail { float* params; float* mom; const float* hyper; };
 cudaError_t launch_error_feedback(acc_ctx* ctx, const float* grads, float* err, float* delta, cudaStream_t s);
 cudaError_t launch_layer_norms(acc_ctx* ctx, const float* buf, long long stride, int n_bufs, const float* minus,
                                double* norm2, cudaStream_t s);
+cudaError_t launch_layer_msdr(acc_ctx* ctx, const float* buf, long long stride, int n_bufs, double* moments,
+                              double* msdr, cudaStream_t s);
 cudaError_t launch_detect(acc_ctx* ctx, const double* n2c, double* n2p, const double* n2d, float lr_curr,
                           float lr_next, uint8_t* level, cudaStream_t s);
 cudaError_t launch_powersgd(acc_ctx* ctx, const float* grads, float* err, float* q, float* p_hat,

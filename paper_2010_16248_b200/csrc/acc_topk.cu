@@ -115,6 +115,7 @@ topk_ef_hist1_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict
     unsigned* buf = s_buf[cb];
     unsigned* cnt = &s_cnt[cb];
     int above = 0;
+    int nz = 0;  // non-zero keys of the tile seen by this thread (settles a threshold that falls among the zeros)
     // batches of kBatch float4 per thread: all loads of a batch are issued before the first store, so that
     // they are in flight together (a store to err in between would pin the later loads of err behind it)
     constexpr int kBatch = 4, kThreads = 256;
@@ -148,6 +149,7 @@ topk_ef_hist1_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict
         *reinterpret_cast<float4*>(e + 4 * i) = m;
         const unsigned k[4] = {key_of(m.x), key_of(m.y), key_of(m.z), key_of(m.w)};
         const float mm[4] = {m.x, m.y, m.z, m.w};
+        nz += (k[0] != 0u) + (k[1] != 0u) + (k[2] != 0u) + (k[3] != 0u);
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
           const unsigned bin = k[q] >> 19;
@@ -190,6 +192,7 @@ topk_ef_hist1_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict
       const float m = gv + (key_of(ev) > ptau ? 0.f : ev);
       e[i] = m;
       const unsigned kk = key_of(m), bin = kk >> 19;
+      nz += kk != 0u;
       atomicAdd(&h[bin], 1u);
       if (staged) {
         if (bin >= blo) {
@@ -208,6 +211,8 @@ topk_ef_hist1_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict
       }
       if (acc_delta) delta[base + i] += gv;
     }
+    nz = __reduce_add_sync(0xffffffffu, nz);
+    if ((threadIdx.x & 31) == 0 && nz) atomicAdd(&tile_cnt[(long long)w * n_tiles + ti].y, nz);  // cleared per step
     if (collect) {  // hand the tile's collected keys over to the segment's list
       above = __reduce_add_sync(0xffffffffu, above);
       if ((threadIdx.x & 31) == 0 && above) atomicAdd(&s_above[cb], above);
@@ -308,17 +313,32 @@ topk_pick1_kernel(const DevLayer* __restrict__ layers, const int* __restrict__ m
                   int W, const uint8_t* __restrict__ level, const unsigned* __restrict__ hist1,
                   Select* __restrict__ sel, int32_t* __restrict__ counts, unsigned* __restrict__ pred,
                   unsigned* __restrict__ seg_cand, const unsigned* __restrict__ seg_flag,
-                  unsigned* __restrict__ any_list, int2* __restrict__ lists, int n_tiles) {
+                  unsigned* __restrict__ any_list, int2* __restrict__ lists, int n_tiles,
+                  const int2* __restrict__ tile_cnt, unsigned* __restrict__ pend_tau) {
   __shared__ unsigned sums[256];
   __shared__ unsigned bin;
   __shared__ long long above;
   __shared__ int s_list;
   __shared__ unsigned s_base;
+  __shared__ unsigned long long s_nz;
   const int seg = blockIdx.x, w = seg / n_mat, l = mat_layers[seg % n_mat];
   const DevLayer L = layers[l];
   const int lv = level[l] ? 1 : 0;
   const int k = lv ? L.k_low : L.k_high;
+  if (threadIdx.x == 0) s_nz = 0;
   pick_from_top_block(hist1 + (long long)seg * kBins1, k, &bin, &above, sums);
+  // The threshold falls into the lowest bucket (k exceeds the keys of all other buckets -- a row-sparse layer at a
+  // large K): when that bucket holds nothing but exact zeros, which the first pass's per-tile counts of non-zero
+  // keys tell, the answer needs no further look at M: every non-zero is kept and the first k - nnz zeros, tau = 0.
+  bool zero_fill = false;
+  if (bin == 0) {
+    unsigned long long part = 0;
+    for (int i = threadIdx.x; i < L.ntiles; i += blockDim.x)
+      part += (unsigned long long)tile_cnt[(long long)w * n_tiles + L.tile0 + i].y;
+    if (part) atomicAdd(&s_nz, part);
+    __syncthreads();
+    zero_fill = s_nz == (unsigned long long)above;  // no non-zero key below the second bucket
+  }
   if (threadIdx.x == 0) {
     Select s;
     s.b1 = bin; s.b2 = 0; s.tau = 0; s.k = k; s.k1 = k - (int)above; s.k2 = 0; s.need = 0;
@@ -335,6 +355,12 @@ topk_pick1_kernel(const DevLayer* __restrict__ layers, const int* __restrict__ m
     } else {
       seg_cand[seg] = 0;  // whatever pass A collected is of no use
       s.mode = fits ? kSelList : kSelDense;
+    }
+    if (zero_fill) {
+      s.mode = kSelZeroFill;
+      s.k2 = s.k1;
+      s.need = s.k1;  // zeros to keep, lowest indices first
+      if (pend_tau != nullptr) pend_tau[seg] = 0u;  // lazy residual: every non-zero entry was kept
     }
     // next prediction: narrow the band after an overflow; none for the zero bucket or for buckets that
     // do not fit the list
@@ -388,6 +414,7 @@ topk_pick2_kernel(int n_mat, const unsigned* __restrict__ hist2, Select* __restr
   __shared__ unsigned bin;
   __shared__ long long above;
   const int seg = blockIdx.x;
+  if (sel[seg].mode == kSelZeroFill) return;  // settled by pick1
   const int k1 = sel[seg].k1;
   pick_from_top_block(hist2 + (long long)seg * kBins2, k1, &bin, &above, sums);
   if (threadIdx.x == 0) { sel[seg].b2 = bin; sel[seg].k2 = k1 - (int)above; }
@@ -627,7 +654,7 @@ topk_hist_list_kernel(const DevLayer* __restrict__ layers, const int* __restrict
   __shared__ unsigned h[kBins];
   const int seg = blockIdx.y;
   const Select s = sel[seg];
-  if (s.mode == kSelDense) return;
+  if (s.mode == kSelDense || s.mode == kSelZeroFill) return;
   const unsigned n = seg_cand[seg] << (s.mode == kSelStaged ? 1 : 0);  // in 4-byte words
   if (blockIdx.x * kChunk >= n) return;
   for (int b = threadIdx.x; b < kBins; b += blockDim.x) h[b] = 0;
@@ -673,7 +700,7 @@ __global__ void __launch_bounds__(256)
 topk_pick3_kernel(int n_seg, const unsigned* __restrict__ hist3, Select* __restrict__ sel,
                   unsigned* __restrict__ pend_tau) {
   const int seg = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
-  if (seg >= n_seg) return;
+  if (seg >= n_seg || sel[seg].mode == kSelZeroFill) return;
   const uint4 c4 = *reinterpret_cast<const uint4*>(hist3 + (long long)seg * kBins3 + 4 * lane);
   const unsigned c[4] = {c4.x, c4.y, c4.z, c4.w};
   const unsigned own = c[0] + c[1] + c[2] + c[3];
@@ -715,6 +742,13 @@ topk_tile_counts_kernel(const DevLayer* __restrict__ layers, const Tile* __restr
   const DevLayer L = layers[tiles[ti].layer];
   if (L.kind != ACC_MATRIX) return;
   const Select s = sel[w * n_mat + L.mat];
+  if (s.mode == kSelZeroFill) {  // tau = 0: the non-zeros lie above it, the zeros tie with it
+    if (lane == 0) {
+      const int nz = tile_cnt[v].y;
+      tile_pre[v] = make_int2(nz, tiles[ti].nelem - nz);
+    }
+    return;
+  }
   if (s.mode != kSelDense) {  // list segment: count the tile's collected keys against the final threshold
     const int2 tc = tile_cand[v];
     const bool staged = s.mode == kSelStaged;
@@ -749,53 +783,74 @@ topk_tile_counts_kernel(const DevLayer* __restrict__ layers, const Tile* __restr
   }
 }
 
+// Exclusive prefix of v over the 256 threads of the block (warp shuffles + the eight warp totals); *total = sum.
+__device__ __forceinline__ int block_excl_scan_256(int v, int* wsum, int* total) {
+  const int lane = threadIdx.x & 31, wi = threadIdx.x >> 5;
+  int incl = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int n = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += n;
+  }
+  if (lane == 31) wsum[wi] = incl;
+  __syncthreads();
+  int base = 0, tot = 0;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int c = wsum[i];
+    base += i < wi ? c : 0;
+    tot += c;
+  }
+  __syncthreads();  // wsum may be reused
+  *total = tot;
+  return base + incl - v;
+}
+
 // One block per (worker, MATRIX layer): exclusive prefix, over the layer's tiles in index order, of the
-// per-tile (above, ties) counts, in place.  The tiles that hold something to keep (above + ties > 0) join the
-// work list of the pass that will write their entries: the staged list or the select list.
+// per-tile (above, ties) counts, in place.  The tiles that hold something to keep -- a key above the threshold, or a
+// tie while fewer than `need` ties precede the tile -- join the work list of the pass that will write their
+// entries: the staged list or the select list.
 __global__ void __launch_bounds__(256)
 topk_tile_scan_kernel(const DevLayer* __restrict__ layers, const int* __restrict__ mat_layers, int n_mat,
                       int n_tiles, int W, const Select* __restrict__ sel, int2* __restrict__ tile_pre,
-                      unsigned* __restrict__ any_list, int2* __restrict__ lists) {
-  __shared__ int2 chunk_sum[256];
-  __shared__ int chunk_act[256];
+                      int2* __restrict__ tile_own, unsigned* __restrict__ any_list, int2* __restrict__ lists) {
+  __shared__ int wsum[8];
   __shared__ unsigned s_base;
   const int seg = blockIdx.x, w = seg / n_mat, l = mat_layers[seg % n_mat];
   const DevLayer L = layers[l];
-  const int which = sel[seg].mode == kSelStaged ? kListStaged : kListSelect;
+  const Select s = sel[seg];
+  const int which = s.mode == kSelStaged ? kListStaged : kListSelect;
   const long long tb = (long long)w * n_tiles + L.tile0;
   const int per = (L.ntiles + 255) / 256;
   const int t0 = min(L.ntiles, (int)threadIdx.x * per), t1 = min(L.ntiles, t0 + per);
   int2 sum = make_int2(0, 0);
-  int act = 0;
   for (int t = t0; t < t1; ++t) {
     const int2 c = tile_pre[tb + t];
     sum.x += c.x; sum.y += c.y;
-    act += (c.x | c.y) != 0;
   }
-  chunk_sum[threadIdx.x] = sum;
-  chunk_act[threadIdx.x] = act;
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    int2 run = make_int2(0, 0);
-    int ra = 0;
-    for (int i = 0; i < 256; ++i) {
-      const int2 c = chunk_sum[i];
-      const int a = chunk_act[i];
-      chunk_sum[i] = run;
-      chunk_act[i] = ra;
-      run.x += c.x; run.y += c.y;
-      ra += a;
+  int total;
+  int2 run;
+  run.x = block_excl_scan_256(sum.x, wsum, &total);
+  run.y = block_excl_scan_256(sum.y, wsum, &total);
+  int act = 0;
+  {
+    int ties_before = run.y;
+    for (int t = t0; t < t1; ++t) {
+      const int2 c = tile_pre[tb + t];
+      act += c.x != 0 || (c.y != 0 && ties_before < s.need);
+      ties_before += c.y;
     }
-    s_base = ra ? atomicAdd(&any_list[kListCountWord + which], (unsigned)ra) : 0u;
   }
+  const int slot = block_excl_scan_256(act, wsum, &total);
+  if (threadIdx.x == 0) s_base = total ? atomicAdd(&any_list[kListCountWord + which], (unsigned)total) : 0u;
   __syncthreads();
-  int2 run = chunk_sum[threadIdx.x];
-  int2* dst = lists + (long long)which * W * n_tiles + s_base + chunk_act[threadIdx.x];
+  int2* dst = lists + (long long)which * W * n_tiles + s_base + slot;
   for (int t = t0; t < t1; ++t) {
     const int2 c = tile_pre[tb + t];
     tile_pre[tb + t] = run;
+    tile_own[tb + t] = c;  // the tile's own (above, ties), for the select pass
+    if (c.x != 0 || (c.y != 0 && run.y < s.need)) *dst++ = make_int2(w, L.tile0 + t);
     run.x += c.x; run.y += c.y;
-    if ((c.x | c.y) != 0) *dst++ = make_int2(w, L.tile0 + t);
   }
 }
 
@@ -815,8 +870,8 @@ __device__ __forceinline__ unsigned warp_incl_scan(unsigned c, int lane) {
 // LAZY: entries above the threshold are not zeroed in err (the next first pass, or the flush, treats them as zero);
 // the kept ties are.
 template <bool FULL, bool LAZY>
-__device__ __forceinline__ void select_tile(const Tile& t, const DevLayer& L, const Select& s, const int2 pre,
-                                            float* __restrict__ m, float* __restrict__ vals,
+__device__ __forceinline__ void select_tile(const Tile& t, const unsigned tau, const int need, const int k,
+                                            const int2 pre, float* __restrict__ m, float* __restrict__ vals,
                                             int32_t* __restrict__ idx, long long seg, unsigned* wtot) {
   const int wi = threadIdx.x >> 5, lane = threadIdx.x & 31;
   float4 mv[8];
@@ -842,8 +897,8 @@ __device__ __forceinline__ void select_tile(const Tile& t, const DevLayer& L, co
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
       const bool valid = FULL || e0 + e < t.nelem;
-      a |= (unsigned)(valid && k[e] > s.tau) << e;
-      tt |= (unsigned)(valid && k[e] == s.tau) << e;
+      a |= (unsigned)(valid && k[e] > tau) << e;
+      tt |= (unsigned)(valid && k[e] == tau) << e;
     }
     am |= a << (4 * j);
     tm |= tt << (4 * j);
@@ -882,9 +937,9 @@ __device__ __forceinline__ void select_tile(const Tile& t, const DevLayer& L, co
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
         const bool is_a = (a >> e) & 1u, is_t = (tt >> e) & 1u;
-        if (is_a || (is_t && ties_before < s.need)) {
-          const int pos = above_before + min(ties_before, s.need);
-          if ((unsigned)pos < (unsigned)s.k) {  // always true for consistent counts; keeps a write inside the segment
+        if (is_a || (is_t && ties_before < need)) {
+          const int pos = above_before + min(ties_before, need);
+          if ((unsigned)pos < (unsigned)k) {  // always true for consistent counts; keeps a write inside the segment
             vals[seg + pos] = v[e];
             idx[seg + pos] = t.elem0 + e0 + e;
             if (!LAZY || !is_a) m[e0 + e] = 0.f;
@@ -899,27 +954,134 @@ __device__ __forceinline__ void select_tile(const Tile& t, const DevLayer& L, co
   }
 }
 
+// The same for a tile in which the ties need no counting: either every key equal to tau is kept (the tie budget
+// outlasts the tile) or none is (no tie in the tile, or the budget ran out before it) -- every tile of a segment but
+// the one where the budget runs out.  An entry is then kept iff its key >= thr (tau or tau + 1), one mask and one
+// scan instead of two, and the positions follow from the count of kept entries alone.
+template <bool FULL, bool LAZY>
+__device__ __forceinline__ void select_tile_simple(const Tile& t, unsigned thr, unsigned tau, bool zero_ties,
+                                                   int base, int k, float* __restrict__ m,
+                                                   float* __restrict__ vals, int32_t* __restrict__ idx, long long seg,
+                                                   unsigned* wtot) {
+  const int wi = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  float4 mv[8];
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    const int e0 = 4 * (wi * 256 + j * 32 + lane);
+    if (FULL || e0 + 3 < t.nelem) {
+      mv[j] = ld_stream4(m + e0);
+    } else {
+      mv[j].x = e0 < t.nelem ? m[e0] : 0.f;
+      mv[j].y = e0 + 1 < t.nelem ? m[e0 + 1] : 0.f;
+      mv[j].z = e0 + 2 < t.nelem ? m[e0 + 2] : 0.f;
+      mv[j].w = 0.f;
+    }
+  }
+  unsigned km = 0;            // 4 bits per j: entry kept
+  unsigned c[2] = {0, 0};     // one byte per j: kept entries of this lane
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    const int e0 = 4 * (wi * 256 + j * 32 + lane);
+    const unsigned kk[4] = {key_of(mv[j].x), key_of(mv[j].y), key_of(mv[j].z), key_of(mv[j].w)};
+    unsigned nib = 0;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) nib |= (unsigned)((FULL || e0 + e < t.nelem) && kk[e] >= thr) << e;
+    km |= nib << (4 * j);
+    c[j >> 2] |= (unsigned)__popc(nib) << (8 * (j & 3));
+  }
+  const unsigned i0 = warp_incl_scan(c[0], lane), i1 = warp_incl_scan(c[1], lane);
+  const unsigned t0 = __shfl_sync(0xffffffffu, i0, 31), t1 = __shfl_sync(0xffffffffu, i1, 31);
+  if (lane == 0) wtot[wi] = __dp4a(t0, 0x01010101u, 0u) + __dp4a(t1, 0x01010101u, 0u);
+  __syncthreads();
+  if (km == 0) return;
+  int pos0 = base;
+  for (int i = 0; i < wi; ++i) pos0 += (int)wtot[i];
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    const unsigned nib = (km >> (4 * j)) & 15u;
+    const unsigned sh = 8 * (j & 3);
+    if (nib) {
+      const int e0 = 4 * (wi * 256 + j * 32 + lane);
+      int pos = pos0 + (int)(((j < 4 ? i0 : i1) >> sh) & 0xffu) - __popc(nib);
+      const float v[4] = {mv[j].x, mv[j].y, mv[j].z, mv[j].w};
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        if ((nib >> e) & 1u) {
+          if ((unsigned)pos < (unsigned)k) {  // always true for consistent counts; keeps a write inside the segment
+            vals[seg + pos] = v[e];
+            idx[seg + pos] = t.elem0 + e0 + e;
+            // eager: every kept entry becomes +0.0; lazy: only the kept ties (entries above tau are dropped by the
+            // next load), and of those only the ones that are not +0.0 already (tau = 0: the negative zeros)
+            if (!LAZY) m[e0 + e] = 0.f;
+            else if (zero_ties && key_of(v[e]) == tau && __float_as_uint(v[e]) != 0u) m[e0 + e] = 0.f;
+          }
+          ++pos;
+        }
+      }
+    }
+    pos0 += (int)(((j < 4 ? t0 : t1) >> sh) & 0xffu);
+  }
+}
+
+// Persistent blocks, each over a contiguous share of the select work list (the tiles of the non-staged segments
+// that hold something to keep; a segment's tiles are consecutive entries, so the layer and threshold records are
+// re-read only when the segment changes).  The list entry and the counters of the next tile are fetched while
+// the current one is processed, and its lines are asked into L2.
 template <bool LAZY>
 __global__ void __launch_bounds__(256, 3)
 topk_select_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict__ tiles, int n_tiles, int n_mat,
                    float* __restrict__ err, const Select* __restrict__ sel, const int2* __restrict__ tile_pre,
-                   const unsigned* __restrict__ any_list, float* __restrict__ vals, int32_t* __restrict__ idx,
+                   const int2* __restrict__ tile_own, const unsigned* __restrict__ any_list,
+                   float* __restrict__ vals, int32_t* __restrict__ idx,
                    long long stride, long long capacity, const int2* __restrict__ lists, int W) {
   __shared__ unsigned wtot[8];
-  // the tiles of the non-staged segments that hold something to keep
-  const unsigned n_work = any_list[kListCountWord + kListSelect];
+  const unsigned long long n_work = any_list[kListCountWord + kListSelect];
+  const unsigned b0 = (unsigned)(n_work * blockIdx.x / gridDim.x), b1 = (unsigned)(n_work * (blockIdx.x + 1) / gridDim.x);
+  if (b0 >= b1) return;
   const int2* work = lists + (long long)kListSelect * W * n_tiles;
-  for (unsigned b = blockIdx.x; b < n_work; b += gridDim.x) {
+  int2 wk = work[b0];
+  int2 pre = tile_pre[(long long)wk.x * n_tiles + wk.y], own = tile_own[(long long)wk.x * n_tiles + wk.y];
+  int2 wk_next = b0 + 1 < b1 ? work[b0 + 1] : wk;
+  int cur_w = -1, tile0 = 0, tile1 = 0;  // the segment whose records are held: worker, tiles [tile0, tile1)
+  long long l_size = 0, l_offset = 0, l_seg_off = 0;
+  unsigned tau = 0;
+  int need = 0, k = 0;
+  for (unsigned b = b0; b < b1; ++b) {
     __syncthreads();  // wtot of the previous tile is no longer read
-    const int w = work[b].x, ti = work[b].y;
-    const Tile t = tiles[ti];
-    const DevLayer L = layers[t.layer];
-    const Select s = sel[w * n_mat + L.mat];
-    const int2 pre = tile_pre[(long long)w * n_tiles + ti];
-    float* m = err + (long long)w * stride + L.offset + t.elem0;
-    const long long seg = (long long)w * capacity + L.seg_off;
-    if (t.nelem == kTile) select_tile<true, LAZY>(t, L, s, pre, m, vals, idx, seg, wtot);
-    else select_tile<false, LAZY>(t, L, s, pre, m, vals, idx, seg, wtot);
+    const int w = wk.x, ti = wk.y;
+    const int2 p = pre, o = own;
+    if (w != cur_w || ti < tile0 || ti >= tile1) {
+      const DevLayer& L = layers[tiles[ti].layer];
+      cur_w = w; tile0 = L.tile0; tile1 = L.tile0 + L.ntiles;
+      l_size = (long long)L.rows * L.cols; l_offset = L.offset; l_seg_off = L.seg_off;
+      const Select& ss = sel[w * n_mat + L.mat];
+      tau = ss.tau; need = ss.need; k = ss.k;
+    }
+    Tile t;
+    t.layer = 0;
+    t.elem0 = (ti - tile0) * kTile;
+    t.nelem = (int)min((long long)kTile, l_size - t.elem0);
+    float* m = err + (long long)w * stride + l_offset + t.elem0;
+    const long long seg = (long long)w * capacity + l_seg_off;
+    // the next tile: its lines into L2 now, its counters and the list entry after it while this tile is worked on
+    wk = wk_next;
+    if (b + 1 < b1) {
+      const Tile tn = tiles[wk.y];
+      prefetch_l2(err + (long long)wk.x * stride + layers[tn.layer].offset + tn.elem0 + 32 * (int)threadIdx.x);
+      pre = tile_pre[(long long)wk.x * n_tiles + wk.y];
+      own = tile_own[(long long)wk.x * n_tiles + wk.y];
+      if (b + 2 < b1) wk_next = work[b + 2];
+    }
+    const bool all_ties = p.y + o.y <= need, no_ties = o.y == 0 || p.y >= need;
+    if (all_ties || no_ties) {
+      const unsigned thr = all_ties ? tau : tau + 1u;
+      const int base = p.x + min(p.y, need);
+      if (t.nelem == kTile) select_tile_simple<true, LAZY>(t, thr, tau, all_ties && o.y != 0, base, k, m, vals, idx, seg, wtot);
+      else select_tile_simple<false, LAZY>(t, thr, tau, all_ties && o.y != 0, base, k, m, vals, idx, seg, wtot);
+    } else {
+      if (t.nelem == kTile) select_tile<true, LAZY>(t, tau, need, k, p, m, vals, idx, seg, wtot);
+      else select_tile<false, LAZY>(t, tau, need, k, p, m, vals, idx, seg, wtot);
+    }
   }
 }
 
@@ -1028,7 +1190,7 @@ topk_finalize_staged_kernel(const DevLayer* __restrict__ layers, const Tile* __r
 // scaled by 1/W.  VECTOR tiles: out = mean_w g_w, delta += g_decider.
 // SGD: the optimiser tail is applied to every element of out where it is written.
 template <bool SGD>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, 3)
 topk_decompress_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict__ tiles, int n_tiles, int n_mat,
                        const float* __restrict__ grads, const Select* __restrict__ sel,
                        const int2* __restrict__ tile_pre, const float* __restrict__ vals,
@@ -1069,33 +1231,46 @@ topk_decompress_kernel(const DevLayer* __restrict__ layers, const Tile* __restri
     r_hi[w] = min(end, s.k);
   }
   __syncthreads();
-  // workers are added one after the other (an element may be kept by several of them and the order of the sum
-  // is fixed); the first entry of the next worker is fetched before the barrier, so its latency is hidden
-  int ni = 0;
-  float nv = 0.f;
-  bool have = false;
-  {
-    const int i = r_lo[0] + (int)threadIdx.x;
-    have = i < r_hi[0];
-    if (have) { const long long seg = L.seg_off; ni = idx[seg + i]; nv = vals[seg + i]; }
-  }
-  for (int w = 0; w < W; ++w) {
-    const long long seg = (long long)w * capacity + L.seg_off;
-    const int ci = ni;
-    const float cv = nv;
-    const bool chave = have;
-    if (w + 1 < W) {
-      const long long nseg = (long long)(w + 1) * capacity + L.seg_off;
-      const int i = r_lo[w + 1] + (int)threadIdx.x;
-      have = i < r_hi[w + 1];
-      if (have) { ni = idx[nseg + i]; nv = vals[nseg + i]; }
+  // Workers are added one after the other (an element may be kept by several of them and the order of the sum is
+  // fixed).  The entries of a group of workers are fetched together, before the first of them is added, so that a
+  // tile pays one memory latency per group instead of two per worker and 256 entries; what a worker has in the tile
+  // beyond the entries the registers hold (the first 512) is added by a plain loop.
+  constexpr int kGroup = 8, kHold = 2;
+  for (int w0 = 0; w0 < W; w0 += kGroup) {
+    const int g = min(kGroup, W - w0);
+    int ri[kGroup][kHold];
+    float rv[kGroup][kHold];
+#pragma unroll
+    for (int j = 0; j < kGroup; ++j) {
+      if (j >= g) break;
+      const long long seg = (long long)(w0 + j) * capacity + L.seg_off;
+      const int lo = r_lo[w0 + j], hi = r_hi[w0 + j];
+#pragma unroll
+      for (int u = 0; u < kHold; ++u) {
+        const int i = lo + u * 256 + (int)threadIdx.x;
+        const bool in = i < hi;
+        ri[j][u] = in ? idx[seg + i] : -1;
+        rv[j][u] = in ? vals[seg + i] : 0.f;
+      }
     }
-    if (chave && (unsigned)(ci - t.elem0) < (unsigned)kTile) acc[ci - t.elem0] += cv;
-    for (int i = r_lo[w] + (int)threadIdx.x + (int)blockDim.x; i < r_hi[w]; i += blockDim.x) {
-      const unsigned li = (unsigned)(idx[seg + i] - t.elem0);
-      if (li < (unsigned)kTile) acc[li] += vals[seg + i];
+#pragma unroll
+    for (int j = 0; j < kGroup; ++j) {
+      if (j >= g) break;
+#pragma unroll
+      for (int u = 0; u < kHold; ++u) {
+        const unsigned li = (unsigned)(ri[j][u] - t.elem0);  // an absent entry (-1) falls outside the tile
+        if (li < (unsigned)kTile) acc[li] += rv[j][u];
+      }
+      const int lo = r_lo[w0 + j], hi = r_hi[w0 + j];
+      if (hi - lo > kHold * 256) {  // uniform over the block
+        const long long seg = (long long)(w0 + j) * capacity + L.seg_off;
+        for (int i = lo + kHold * 256 + (int)threadIdx.x; i < hi; i += 256) {
+          const unsigned li = (unsigned)(idx[seg + i] - t.elem0);
+          if (li < (unsigned)kTile) acc[li] += vals[seg + i];
+        }
+      }
+      __syncthreads();
     }
-    __syncthreads();
   }
   const int n4 = t.nelem >> 2;
   for (int i = threadIdx.x; i < n4; i += blockDim.x) {
@@ -1233,7 +1408,8 @@ static cudaError_t launch_topk_select_part(acc_ctx* ctx, const float* grads, flo
       PhaseTimer pt(ctx, PH_TOPK_PICK1, s);
       topk_pick1_kernel<<<W * n_mat, 256, 0, s>>>(ctx->d_layers, ctx->d_mat_layers, n_mat, c.n_layers, W, level,
                                                   ctx->d_hist1, ctx->d_sel, counts, ctx->d_pred, ctx->d_seg_cand,
-                                                  ctx->d_seg_flag, ctx->d_any_list, ctx->d_lists, nt);
+                                                  ctx->d_seg_flag, ctx->d_any_list, ctx->d_lists, nt, ctx->d_tile_cnt,
+                                                  lazy ? ctx->d_pend_tau : nullptr);
     }
     {
       PhaseTimer pt(ctx, PH_TOPK_COLLECT, s);
@@ -1284,7 +1460,8 @@ static cudaError_t launch_topk_select_part(acc_ctx* ctx, const float* grads, flo
     {
       PhaseTimer pt(ctx, PH_TOPK_PICK3_SCAN, s);
       topk_tile_scan_kernel<<<W * n_mat, 256, 0, s>>>(ctx->d_layers, ctx->d_mat_layers, n_mat, nt, W, ctx->d_sel,
-                                                      ctx->d_tile_pre, ctx->d_any_list, ctx->d_lists);
+                                                      ctx->d_tile_pre, ctx->d_tile_cnt, ctx->d_any_list,
+                                                      ctx->d_lists);
     }
   }
   if (n_mat > 0) {
@@ -1306,12 +1483,12 @@ static cudaError_t launch_topk_select_part(acc_ctx* ctx, const float* grads, flo
     const unsigned sgrid = (unsigned)std::min(blocks, cap);
     if (lazy)
       topk_select_kernel<true><<<sgrid, 256, 0, s>>>(ctx->d_layers, ctx->d_tiles, nt, n_mat, err, ctx->d_sel,
-                                                     ctx->d_tile_pre, ctx->d_any_list, vals, idx, c.worker_stride,
-                                                     pl.capacity, ctx->d_lists, W);
+                                                     ctx->d_tile_pre, ctx->d_tile_cnt, ctx->d_any_list, vals, idx,
+                                                     c.worker_stride, pl.capacity, ctx->d_lists, W);
     else
       topk_select_kernel<false><<<sgrid, 256, 0, s>>>(ctx->d_layers, ctx->d_tiles, nt, n_mat, err, ctx->d_sel,
-                                                      ctx->d_tile_pre, ctx->d_any_list, vals, idx, c.worker_stride,
-                                                      pl.capacity, ctx->d_lists, W);
+                                                      ctx->d_tile_pre, ctx->d_tile_cnt, ctx->d_any_list, vals, idx,
+                                                      c.worker_stride, pl.capacity, ctx->d_lists, W);
   }
   return cudaGetLastError();
 }

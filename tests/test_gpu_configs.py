@@ -37,12 +37,15 @@ class OracleController:
             self.delta[:] = 0
 
 
-def _run_config(w, iters, t0=0, lazy=False, topk_layers=None, topk_workers=None, psgd_check=None):
-    """Runs `iters` iterations of workload `w` starting at stream iteration t0; checks every TopK step and
-    every level decision exactly, and the PowerSGD steps listed in psgd_check (default: all).  With
+def _run_config(w, iters, t0=0, lazy=False, topk_layers=None, topk_workers=None, psgd_check=None, topk_check=None,
+                force_level=None, paths_seen=None):
+    """Runs `iters` iterations of workload `w` starting at stream iteration t0; checks every level decision
+    exactly, the TopK steps listed in topk_check and the PowerSGD steps listed in psgd_check (default: all).  With
     lazy=True a second engine in lazy-residual mode (the mode bench.py times) runs in lockstep and must
     reproduce the eager engine's outputs (out, Q, P^; packed TopK sets) bit for bit at every step, and its error
-    memories after a final flush."""
+    memories after a final flush.  force_level (0 / 1) starts every engine, and the oracle's controller, at that
+    level instead of the initial low-compression level.  paths_seen (a set) collects the TopK selection paths the
+    lazy engine (else the eager one) took."""
     table, W = w.table, w.n_workers
     stream = wl.GradientStream(w, device="cuda")
     eng = pipeline.AccordionStep(table, W, w.compressors, w.rank_low, w.rank_high, w.topk_low_bp, w.topk_high_bp,
@@ -52,6 +55,11 @@ def _run_config(w, iters, t0=0, lazy=False, topk_layers=None, topk_workers=None,
         lz = pipeline.AccordionStep(table, W, w.compressors, w.rank_low, w.rank_high, w.topk_low_bp, w.topk_high_bp,
                                     w.eta, 1e-8, w.check_every, lazy_residual=True)
     ctl = OracleController(table, w.check_every, w.eta)
+    if force_level is not None:
+        for e in (eng, lz):
+            if e is not None:
+                e.level.fill_(force_level)
+        ctl.level[:] = force_level
     seen_levels = set()
     for i in range(iters):
         grads = stream.grads(t0 + i)
@@ -75,10 +83,12 @@ def _run_config(w, iters, t0=0, lazy=False, topk_layers=None, topk_workers=None,
         if "powersgd" in w.compressors and (psgd_check is None or i in psgd_check):
             H.check_powersgd_against_oracle(eng.ctx, table, grads, e0, q0, level_before, eng.out_psgd, eng.err_psgd,
                                             eng.q, eng.p_hat, w.rank_low, w.rank_high, 1e-8)
-        if "topk" in w.compressors:
+        if "topk" in w.compressors and (topk_check is None or i in topk_check):
             H.check_topk_against_oracle(eng.ctx, table, grads, et0, level_before, eng.vals, eng.idx, eng.counts,
                                         eng.out_topk, eng.err_topk, w.topk_low_bp, w.topk_high_bp,
                                         layers_subset=topk_layers, workers_subset=topk_workers)
+        if paths_seen is not None and "topk" in w.compressors:
+            paths_seen.update(int(p) for p in (lz or eng).ctx.acc_topk_last_paths().ravel())
         ctl.step(grads[0].cpu().numpy())
     if lz is not None:
         lz.flush()
@@ -127,6 +137,19 @@ def test_reduced_configs_across_scale_jump(config, scale):
     assert seen == {0, 1}, "both compression levels must have been exercised"
 
 
+@pytest.mark.parametrize("config,scale", [(2, 4), (3, 4), (4, 4), (5, 16)])
+def test_reduced_configs_second_jump_and_last_iteration(config, scale):
+    """The scale jump at iteration 150 and the end of the schedule.  From iteration 140: the windows [140,150) and
+    [150,160) differ by the jump (low level), [150,160) and [160,170) do not (high level from step 30).  Then the
+    last 25 iterations of the configuration, which end at the high level on its final iteration."""
+    w = wl.workload(config, scale=scale)
+    seen = _run_config(w, iters=35, t0=140, psgd_check={0, 9, 10, 11, 19, 20, 21, 29, 30, 31, 34},
+                       topk_check={0, 9, 10, 11, 19, 20, 21, 29, 30, 31, 34})
+    assert seen == {0, 1}
+    seen = _run_config(w, iters=25, t0=w.n_iters - 25, psgd_check={0, 19, 20, 21, 24}, topk_check={0, 19, 20, 21, 24})
+    assert seen == {0, 1}
+
+
 @pytest.mark.parametrize("config,scale", [(2, 4), (3, 4), (5, 16)])
 def test_reduced_configs_lazy_residual(config, scale):
     w = wl.workload(config, scale=scale)
@@ -158,6 +181,60 @@ def test_full_size_config5_sampled():
     names = w.table.names
     sample = [names.index("encoder.weight"), names.index("rnn.weight_hh_l1"), names.index("decoder.weight")]
     _run_config(w, iters=2, t0=0, lazy=True, topk_layers=sample, topk_workers=[0, 5])
+
+
+# ------------------------------------------------------------------ full size, the steady state bench.py times
+def test_full_size_config3_high_level_steady_state():
+    """ResNet-18 set, TopK at K = 1 % on every layer for six steps in a row, lazy residual (what the benchmark runs for
+    most of its steps): the threshold predictions engage from the second step, whole entries are staged from the
+    third.  Every step must equal the eager engine's bit for bit; steps 2 and 5 are checked against the oracle on
+    every MATRIX layer for one worker and on three layers for all workers."""
+    w = wl.workload(3)
+    mats = [l for l in range(w.table.n_layers) if w.table.kind[l] == wl.MATRIX]
+    paths = set()
+    _run_config(w, iters=6, t0=20, lazy=True, topk_workers=[1], topk_check={2, 5}, force_level=0, paths_seen=paths)
+    assert binding.ACC_TOPK_PATH_STAGED in paths, paths  # (the predicted-list path belongs to config 5's encoder)
+    sample = [mats[0], int(np.argmax(w.table.sizes)), mats[-1]]
+    _run_config(w, iters=4, t0=20, lazy=True, topk_layers=sample, topk_check={3}, force_level=0)
+
+
+def test_full_size_config5_high_level_steady_state():
+    """LSTM set, W = 8, both compressors at the high compression level (rank 1, K = 1 %) for six steps, lazy
+    residual: the pipelined first PowerSGD pass subtracts the pending rank-1 residual while loading, TopK runs on
+    staged entries (gate matrices, decoder) and on the predicted list (the row-sparse encoder).  Lazy must equal
+    eager at every step; PowerSGD is checked against the oracle on every layer at steps 1 and 5, TopK at step 5 on
+    the encoder, a gate matrix and the decoder for two workers."""
+    w = wl.workload(5)
+    names = w.table.names
+    sample = [names.index("encoder.weight"), names.index("rnn.weight_ih_l1"), names.index("decoder.weight")]
+    paths = set()
+    _run_config(w, iters=6, t0=20, lazy=True, topk_layers=sample, topk_workers=[2, 7], psgd_check={1, 5},
+                topk_check={5}, force_level=0, paths_seen=paths)
+    assert binding.ACC_TOPK_PATH_STAGED in paths and binding.ACC_TOPK_PATH_LIST_PREDICTED in paths, paths
+
+
+def test_full_size_config4_high_level_pending_residual():
+    """VGG-19bn set, W = 8, rank 1 on every layer with the lazy residual pending from step to step, direct and
+    pipelined first pass: both must equal the eager engine bit for bit; the oracle checks steps 1 and 3."""
+    w = wl.workload(4)
+    _run_config(w, iters=4, t0=20, lazy=True, psgd_check={1, 3}, force_level=0)
+    table, W = w.table, w.n_workers
+    stream = wl.GradientStream(w, device="cuda")
+    engines = [pipeline.AccordionStep(table, W, w.compressors, w.rank_low, w.rank_high, w.topk_low_bp, w.topk_high_bp,
+                                      w.eta, 1e-8, w.check_every, lazy_residual=True, extra_flags=f)
+               for f in (binding.ACC_FLAG_PIPELINE_NEVER, binding.ACC_FLAG_PIPELINE_ALWAYS)]
+    for e in engines:
+        e.level.zero_()
+    for i in range(4):
+        g = stream.grads(20 + i)
+        for e in engines:
+            e.step(g)
+    for e in engines:
+        e.flush()
+    torch.cuda.synchronize()
+    for name in ("out_psgd", "q", "p_hat", "err_psgd"):
+        assert torch.equal(getattr(engines[0], name), getattr(engines[1], name)), name
+    assert engines[1].ctx.acc_device_status() == 0
 
 
 def test_graph_replay_matches_direct_calls():

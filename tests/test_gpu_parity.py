@@ -85,6 +85,42 @@ def test_layer_norms_match_oracle():
     assert np.array_equal(one.cpu().numpy(), got[1])
 
 
+def test_layer_msdr_matches_oracle():
+    """Mean-to-standard-deviation ratio per layer (the second detector statistic) against the oracle: random layers
+    with a mean, a constant layer (+inf), an all-zero layer (0); the second moment must be the bits acc_layer_norms
+    returns, so one pass over the accumulated gradient serves both detectors."""
+    table = wl.make_table([("a", (300, 70)), ("v", (33,)), ("const", (16, 16)), ("zero", (8, 8)), ("big", (129, 1000))])
+    W = 2
+    ctx = binding.Context(table, W)
+    g = torch.Generator(device="cuda").manual_seed(4)
+    buf = torch.zeros(W, table.stride, device="cuda")
+    for l, sl in table.slices():
+        n = sl.stop - sl.start
+        if table.names[l] == "const":
+            buf[:, sl] = 0.375
+        elif table.names[l] != "zero":
+            buf[:, sl] = torch.randn(W, n, generator=g, device="cuda") * (0.5 + l) + 0.05 * (l + 1)
+    L = table.n_layers
+    mom = torch.zeros(2 * W * L, dtype=torch.float64, device="cuda")
+    msdr = torch.zeros(W * L, dtype=torch.float64, device="cuda")
+    n2 = torch.zeros(W * L, dtype=torch.float64, device="cuda")
+    ctx.acc_layer_msdr(buf, W, mom, msdr)
+    ctx.acc_layer_norms(buf, W, n2)
+    torch.cuda.synchronize()
+    mom_h, msdr_h = mom.cpu().numpy().reshape(W, L, 2), msdr.cpu().numpy().reshape(W, L)
+    assert np.array_equal(mom_h[:, :, 1].ravel(), n2.cpu().numpy())
+    for w in range(W):
+        want, mean, std = orc.layer_msdr(buf[w].cpu().numpy(), H.layers_of(table))
+        for l in range(L):
+            size = float(table.sizes[l])
+            assert abs(mom_h[w, l, 0] / size - mean[l]) <= 1e-12 * max(1.0, abs(mean[l]))
+            if np.isinf(want[l]):
+                assert np.isinf(msdr_h[w, l]) and msdr_h[w, l] > 0, table.names[l]
+            else:
+                assert abs(msdr_h[w, l] - want[l]) <= 1e-9 * max(want[l], 1e-30), (table.names[l], msdr_h[w, l], want[l])
+    assert msdr_h[0, table.names.index("zero")] == 0.0
+
+
 def test_detect_regime_truth_table_and_random():
     L = 300
     table = wl.make_table([(f"v{i}", (4,)) for i in range(L)])
@@ -262,9 +298,12 @@ def test_bad_arguments_are_rejected():
     table = _table_mixed()
     ctx = binding.Context(table, 2)
     grads, err = _random_inputs(table, 2, 1)
+    roomy = torch.zeros(grads.numel() + 8, device="cuda")
     with pytest.raises(binding.AccError) as ei:
-        ctx.acc_error_feedback(grads.view(-1)[1:-3].view(-1), err)  # misaligned pointer
+        ctx.acc_error_feedback(roomy[1:1 + grads.numel()], err)  # long enough, but 4 bytes off a 16-byte boundary
     assert ei.value.status == 2
+    with pytest.raises(ValueError):
+        ctx.acc_error_feedback(grads.view(-1)[:-4], err)           # too short for the layout: refused by the binding
     with pytest.raises(ValueError):
         ctx.acc_error_feedback(grads.cpu(), err)
     with pytest.raises(binding.AccError):
@@ -341,11 +380,13 @@ def test_topk_threshold_prediction_hits_and_misses(pipeline):
 
 
 def test_topk_every_selection_path_is_exercised():
-    """All four selection paths give the same (oracle-checked) results; this run makes sure each of them is
-    actually taken: dense (a bucket too fat for a list: the all-zero layer), list (first step, no prediction),
-    predicted list (same gradients again) and staged entries (high compression level on a layer whose kept
-    entries stand far above the rest)."""
-    table = wl.make_table([("zeros", (64, 1024)), ("noise", (256, 1024)), ("spiky", (256, 1024))])
+    """All five selection paths give the same (oracle-checked) results; this run makes sure each of them is
+    actually taken: dense (a bucket too fat for a list: a layer of equal magnitudes, and a layer of zeros with a few
+    denormals among them), list (first step, no prediction), predicted list (same gradients again), staged entries
+    (high compression level on a layer whose kept entries stand far above the rest) and zero fill (a layer with fewer
+    non-zeros than k: every non-zero plus the first zeros; an all-zero layer)."""
+    table = wl.make_table([("zeros", (64, 1024)), ("noise", (256, 1024)), ("spiky", (256, 1024)),
+                           ("const", (40, 1000)), ("rowsparse", (300, 650)), ("denormal", (32, 1024))])
     W = 2
     ctx = binding.Context(table, W, topk_low_bp=1000, topk_high_bp=100)
     g = torch.Generator(device="cuda").manual_seed(9)
@@ -356,9 +397,23 @@ def test_topk_every_selection_path_is_exercised():
     hot = torch.randperm(256 * 1024, generator=g, device="cuda")[:4000]
     spiky[:, hot] = 5.0 + torch.rand(W, 4000, generator=g, device="cuda")
     grads[:, sl["spiky"]] = spiky
+    sign = torch.randint(0, 2, (W, 40 * 1000), generator=g, device="cuda").float() * 2 - 1
+    grads[:, sl["const"]] = 0.75 * sign                       # one magnitude: everything ties at the threshold
+    rs = torch.zeros(W, 300, 650, device="cuda")
+    for w in range(W):                                        # 2 % of the rows non-zero, a negative zero among the rest
+        rows = torch.randperm(300, generator=g, device="cuda")[:6]
+        rs[w, rows] = torch.randn(6, 650, generator=g, device="cuda")
+    rs[:, 7, 3] = -0.0
+    grads[:, sl["rowsparse"]] = rs.reshape(W, -1)
+    den = torch.zeros(W, 32 * 1024, device="cuda")
+    den[:, 5::97] = 1e-41                                     # denormals share the lowest bucket with the zeros
+    den[:, 11] = 3.0
+    grads[:, sl["denormal"]] = den
     vals, idx, counts = ctx.new_topk_buffers()
     out = torch.zeros(table.stride, device="cuda")
     seen = set()
+    names = [n for l, n in enumerate(table.names)]
+    by_layer = {}
     for lv in (1, 1, 1, 0, 0, 0, 0):
         level = torch.full((table.n_layers,), lv, dtype=torch.uint8, device="cuda")
         err = torch.zeros_like(grads)
@@ -366,8 +421,52 @@ def test_topk_every_selection_path_is_exercised():
         torch.cuda.synchronize()
         H.check_topk_against_oracle(ctx, table, grads, torch.zeros_like(grads), level, vals, idx, counts, out, err,
                                     1000, 100)
-        seen.update(int(p) for p in ctx.acc_topk_last_paths().ravel())
-    assert seen == {0, 1, 2, 3}, seen
+        paths = ctx.acc_topk_last_paths()
+        seen.update(int(p) for p in paths.ravel())
+        for j, n in enumerate(names):
+            by_layer.setdefault(n, set()).update(int(p) for p in paths[:, j])
+    assert seen == {0, 1, 2, 3, 4}, seen
+    assert by_layer["zeros"] == {4} and 4 in by_layer["rowsparse"]      # k = 10 % of 195000 > 3900 non-zeros
+    assert by_layer["const"] == {0} and by_layer["denormal"] == {0}
+
+
+def test_topk_zero_fill_with_error_feedback_lazy_and_eager():
+    """A row-sparse layer over several steps with error feedback: at K = 10 % the threshold is zero (all non-zeros
+    and the first zeros are kept, the memory empties), at K = 1 % it lies among the non-zeros and the memory
+    fills up again.  Eager and lazy residual modes must give the same bits, step by step and after the flush."""
+    table = wl.make_table([("emb", (1200, 330)), ("v", (9,)), ("dense", (64, 330))])
+    W = 3
+    ctxs = [binding.Context(table, W), binding.Context(table, W, flags=binding.ACC_FLAG_LAZY_RESIDUAL)]
+    st = [dict(zip(("vals", "idx", "counts"), c.new_topk_buffers())) for c in ctxs]
+    for s_ in st:
+        s_["err"] = torch.zeros(W, table.stride, device="cuda")
+        s_["out"] = torch.zeros(table.stride, device="cuda")
+    g = torch.Generator(device="cuda").manual_seed(31)
+    o_emb = int(table.offset[0])
+    seen = set()
+    for it, lv in enumerate([1, 1, 0, 0, 1, 0, 1, 1]):
+        grads = torch.zeros(W, table.stride, device="cuda")
+        grads[:, int(table.offset[2]):int(table.offset[2]) + 64 * 330] = torch.randn(W, 64 * 330, generator=g, device="cuda")
+        grads[:, int(table.offset[1]):int(table.offset[1]) + 9] = torch.randn(W, 9, generator=g, device="cuda")
+        for w in range(W):
+            rows = torch.randperm(1200, generator=g, device="cuda")[:24]
+            emb = torch.zeros(1200, 330, device="cuda")
+            emb[rows] = torch.randn(24, 330, generator=g, device="cuda")
+            grads[w, o_emb:o_emb + 1200 * 330] = emb.reshape(-1)
+        level = torch.full((table.n_layers,), lv, dtype=torch.uint8, device="cuda")
+        e0 = st[0]["err"].clone()
+        for c, s_ in zip(ctxs, st):
+            c.acc_topk_step(grads, s_["err"], level, s_["vals"], s_["idx"], s_["counts"], s_["out"])
+        torch.cuda.synchronize()
+        H.check_topk_against_oracle(ctxs[0], table, grads, e0, level, st[0]["vals"], st[0]["idx"], st[0]["counts"],
+                                    st[0]["out"], st[0]["err"], 1000, 100)
+        for name in ("vals", "idx", "counts", "out"):
+            assert torch.equal(st[0][name], st[1][name]), (it, name)
+        seen.update(int(p) for p in ctxs[1].acc_topk_last_paths()[:, 0])
+    assert 4 in seen and len(seen) > 1, seen
+    ctxs[1].acc_topk_flush(st[1]["err"])
+    torch.cuda.synchronize()
+    assert torch.equal(st[0]["err"], st[1]["err"])
 
 
 @pytest.mark.parametrize("lazy", [0, binding.ACC_FLAG_LAZY_RESIDUAL])

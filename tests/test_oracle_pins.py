@@ -94,6 +94,42 @@ def test_layer_norms_closed_form_and_library():
     assert np.isclose(np.sqrt(n2[2]), np.linalg.norm(c.astype(np.float64)), rtol=1e-14)
 
 
+def test_msdr_hand_values_library_and_invariances():
+    """Mean-to-standard-deviation ratio per layer: hand-computed vectors, the library's mean / std on random
+    ones, and what the definition implies (scale invariance, sign symmetry, the effect of a shift)."""
+    table = wl.make_table([("a", (2, 2)), ("const", (4,)), ("zero", (1, 4)), ("sym", (4,)), ("b", (3, 5))])
+    layers = _layers(table)
+    buf = np.zeros(table.stride, np.float32)
+    rng = np.random.default_rng(3)
+    rnd = (rng.standard_normal(15) + 0.7).astype(np.float32)
+    for (off, r, c, k), vals in zip(layers, ([1, 2, 3, 4], [2, 2, 2, 2], [0, 0, 0, 0], [-3, -1, 1, 3], rnd)):
+        buf[off:off + r * c] = vals
+    msdr, mean, std = orc.layer_msdr(buf, layers)
+    # [1,2,3,4]: mean 2.5, deviations +-1.5, +-0.5 -> variance (2.25+0.25)*2/4 = 1.25
+    assert mean[0] == 2.5 and abs(std[0] - np.sqrt(1.25)) < 1e-15 and abs(msdr[0] - 2.5 / np.sqrt(1.25)) < 1e-15
+    assert abs(msdr[0] - np.sqrt(5.0)) < 1e-15
+    assert np.isinf(msdr[1]) and mean[1] == 2.0 and std[1] == 0.0      # constant layer
+    assert msdr[2] == 0.0 and msdr[3] == 0.0 and mean[3] == 0.0          # all zero; zero mean
+    assert abs(std[3] - np.sqrt(5.0)) < 1e-15                            # (9+1+1+9)/4
+    x = rnd.astype(np.float64)
+    assert abs(msdr[4] - abs(np.mean(x)) / np.std(x)) < 1e-12 and abs(std[4] - np.std(x)) < 1e-14
+    # invariances: scaling by c != 0 (also negative) leaves the ratio alone; padding is not read
+    buf2 = (-3.0 * buf).astype(np.float32)
+    end_b = layers[4][0] + 15
+    assert end_b < table.stride
+    buf2[end_b:] = 99.0
+    m2, _, _ = orc.layer_msdr(buf2, layers)
+    assert abs(m2[0] - msdr[0]) < 1e-6 and abs(m2[4] - msdr[4]) < 1e-6
+    # a shift by s moves the mean and leaves the deviation: MSDR(x + s) = |mu + s| / sd
+    off, r, c, _ = layers[4]
+    shifted = buf.copy()
+    shifted[off:off + 15] = (rnd.astype(np.float64) + 4.0).astype(np.float32)
+    m3, mu3, sd3 = orc.layer_msdr(shifted, layers)
+    xs = shifted[off:off + 15].astype(np.float64)
+    assert abs(sd3[4] - np.std(xs)) < 1e-14 and abs(m3[4] - abs(np.mean(xs)) / np.std(xs)) < 1e-12
+    assert abs(sd3[4] - std[4]) < 1e-6 and abs(mu3[4] - (mean[4] + 4.0)) < 1e-6
+
+
 def test_accumulate_sums_decider_gradients():
     table = wl.make_table([("a", (2, 3)), ("b", (5,))])
     layers = _layers(table)
