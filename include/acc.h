@@ -4,10 +4,10 @@
  * The library runs, for W simulated data-parallel workers whose gradients sit in one GPU's
  * memory, the per-iteration step that Accordion (arXiv 2010.16248) drives:
  *
- *   - error-feedback accumulation          M_w = g_w + e_w           (the "memory term", Section 5.2)
+ *   - error-feedback accumulation          M_w = g_w + e_w           (the "memory term", Section "Accordion with PowerSGD")
  *   - gradient accumulation + layer norms  for the critical-regime test (Section 4.2)
  *   - the regime test itself               Algorithm 1
- *   - the compressor at the chosen level   PowerSGD rank r, or TopK K%   (Section 5, first paragraph)
+ *   - the compressor at the chosen level   PowerSGD rank r, or TopK K%   (Section "Experimental evaluation", first paragraph)
  *   - the mean over workers of the compressed gradients   (update rule of Section 3)
  *
  * General rules, valid for every entry point unless it says otherwise:
@@ -56,8 +56,9 @@ extern "C" {
 #define ACC_FLAG_LAZY_RESIDUAL 1 /* err keeps M_w after a step; the compressed part is removed on the next load
                                    (see acc_powersgd_step and acc_topk_step) */
 /* The first PowerSGD pass exists as a direct kernel and as a persistent kernel fed by bulk asynchronous
- * copies; both compute the same values.  By default the library picks by problem size (the pipelined one
- * needs a long queue of tiles per SM to pay off).  These two flags force the choice (tests, tuning). */
+ * copies; both compute the same values up to the rounding order of a few additions (the last bits of P).
+ * By default the library picks by problem size (the pipelined one needs a long queue of tiles per SM to
+ * pay off).  These two flags force the choice (tests, tuning). */
 #define ACC_FLAG_PIPELINE_ALWAYS 2
 #define ACC_FLAG_PIPELINE_NEVER 4
 
@@ -110,7 +111,7 @@ int acc_factor_layout(const acc_ctx* ctx, int64_t* q_row /*[L]*/, int64_t* p_row
 int acc_topk_layout(const acc_ctx* ctx, int64_t* seg_offset /*[L]*/, int64_t* k_low /*[L]*/,
                     int64_t* k_high /*[L]*/, int64_t* capacity);
 
-/* Error-feedback accumulation on its own (Section 5.2: compressors run "with memory"):
+/* Error-feedback accumulation on its own (Section "Accordion with PowerSGD": the compressors run "with memory"):
  *   err_w <- g_w + err_w  on MATRIX layers, in fp32 (one IEEE add), for every worker;
  *   delta <- delta + g_decider on every layer when delta != NULL (gradient accumulation of the
  *   detector, Section 4.2 "Computational and memory overhead").
@@ -148,6 +149,13 @@ int acc_layer_msdr(acc_ctx* ctx, const float* buf, int64_t buf_stride, int32_t n
 int acc_detect_regime(acc_ctx* ctx, const double* norm2_curr, double* norm2_prev, float lr_curr,
                       float lr_next, uint8_t* level, float* delta, void* stream);
 
+/* acc_detect_regime with the two learning rates read from DEVICE memory (lr_pair[0] = current, lr_pair[1] = next) at
+ * the time the kernel runs, instead of from the arguments: a CUDA graph that captured the call then follows a
+ * learning-rate schedule -- the second condition of Algorithm 1 -- when the caller rewrites the two floats between
+ * replays.  Otherwise identical.  Device pointers: lr_pair 2 floats (read); the others as above.        */
+int acc_detect_regime_lr(acc_ctx* ctx, const double* norm2_curr, double* norm2_prev, const float* lr_pair,
+                         uint8_t* level, float* delta, void* stream);
+
 /* Variant of the regime test with the norm of the DIFFERENCE of the two accumulated gradients,
  *   || D_prev - D_curr || >= eta * || D_prev ||,
  * in place of the difference of their norms that the display equation of Section 4.2 and Algorithm 1 print.
@@ -163,7 +171,7 @@ int acc_detect_regime_diff(acc_ctx* ctx, const double* norm2_diff, const double*
                            float lr_curr, float lr_next, uint8_t* level, float* delta, float* delta_prev,
                            void* stream);
 
-/* One PowerSGD step with error feedback (the compressor of Section 5.2, applied per MATRIX layer at
+/* One PowerSGD step with error feedback (the compressor of the Section "Accordion with PowerSGD", applied per MATRIX layer at
  * rank r = rank_low if level[l] else rank_high), all workers, mean over workers (Section 3):
  *   M_w = g_w + e_w;  P = mean_w M_w Q[:, :r];  P^ = modified Gram-Schmidt(P) (divide by norm + gs_eps);
  *   Q[:, :r] <- mean_w M_w^T P^;  A = P^ Q[:, :r]^T;  out[l] = A;  e_w <- M_w - A.
@@ -187,7 +195,7 @@ int acc_powersgd_step(acc_ctx* ctx, const float* grads, float* err, float* q, fl
  * Device pointers: err [W][worker_stride] (in/out), q, p_hat (read).                                */
 int acc_powersgd_flush(acc_ctx* ctx, float* err, const float* q, const float* p_hat, void* stream);
 
-/* One TopK step with error feedback (the sparsifier of Section 5.3, per MATRIX layer and worker,
+/* One TopK step with error feedback (the sparsifier of the Section "Accordion with TopK", per MATRIX layer and worker,
  * k = max(1, floor(rows*cols*K_bp/10000)), K_bp = topk_low_bp if level[l] else topk_high_bp):
  *   M_w = g_w + e_w (fp32);  keep the k entries of largest |M_w| -- compared as 31-bit patterns,
  *   ties broken by lower index --;  vals/idx <- kept values (bit copies) and layer-local indices in

@@ -103,7 +103,7 @@ def detect_regime_diff(norm2_diff, norm2_curr, norm2_prev, lr_curr, lr_next, eta
 
 def layer_msdr(buf, layers):
     """Mean-to-standard-deviation ratio of each layer of one flat buffer: the statistic of the adaptive scheme
-    the paper compares itself with (Section 6, "Comparison with Prior Work"), which lowers the compression when
+    the paper compares itself with (Section "Comparison with Prior Work"), which lowers the compression when
     the ratio has dropped.  The paper names the statistic only; taken here over the coordinates of a layer of
     the detector's accumulated gradient:
 
@@ -129,7 +129,7 @@ def layer_msdr(buf, layers):
 
 
 # --------------------------------------------------------------------------- #
-# Error feedback (the "memory term", Section 5.2 / Appendix A)
+# Error feedback (the "memory term": Section "Accordion with PowerSGD", Appendix A)
 # --------------------------------------------------------------------------- #
 def error_feedback(grads, err, layers, fp32=False):
     """M_w = g_w + e_w on MATRIX layers (VECTOR layers carry no memory: M = g)."""

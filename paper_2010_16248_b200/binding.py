@@ -52,7 +52,7 @@ EXPORTS = ["acc_workspace_bytes", "acc_create", "acc_destroy", "acc_factor_layou
            "acc_exchange_layout", "acc_powersgd_phase1", "acc_powersgd_phase2", "acc_powersgd_phase3",
            "acc_topk_compress", "acc_topk_decompress", "acc_topk_flush",
            "acc_upload_grads", "acc_download_out", "acc_selftest_wait_timeout", "acc_reset_device_status",
-           "acc_layer_msdr"]
+           "acc_layer_msdr", "acc_detect_regime_lr"]
 
 _lib = None
 
@@ -77,6 +77,7 @@ def lib() -> C.CDLL:
     L.acc_layer_norms.argtypes = [vp, vp, i64, i32, vp, vp]
     L.acc_layer_msdr.argtypes = [vp, vp, i64, i32, vp, vp, vp]
     L.acc_detect_regime.argtypes = [vp, vp, vp, f32, f32, vp, vp, vp]
+    L.acc_detect_regime_lr.argtypes = [vp, vp, vp, vp, vp, vp, vp]
     L.acc_powersgd_step.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp]
     L.acc_topk_step.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
     L.acc_floats_sent.argtypes = [C.POINTER(acc_config), C.POINTER(C.c_uint8), i32]
@@ -308,6 +309,12 @@ class Context:
         self._call("acc_detect_regime", self._d(norm2_curr, L, "norm2_curr"),
                    self._d(norm2_prev, L, "norm2_prev"), float(lr_curr), float(lr_next), self._lv(level),
                    self._f(delta, self.stride, "delta"), stream=stream)
+
+    def acc_detect_regime_lr(self, norm2_curr, norm2_prev, lr_pair, level, delta=None, stream=None):
+        L = self.n_layers
+        self._call("acc_detect_regime_lr", self._d(norm2_curr, L, "norm2_curr"), self._d(norm2_prev, L, "norm2_prev"),
+                   self._f(lr_pair, 2, "lr_pair"), self._lv(level), self._f(delta, self.stride, "delta"),
+                   stream=stream)
 
     def acc_layer_diff_norms(self, a, b, norm2, stream=None):
         self._call("acc_layer_diff_norms", self._f(a, self.extent, "a"), self._f(b, self.extent, "b"),

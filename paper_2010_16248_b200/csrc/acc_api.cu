@@ -129,6 +129,7 @@ static int make_plan(const acc_config* cfg, Plan& p) {
   p.o_tile_cand = take(sizeof(int2) * (size_t)W * nt);
   p.o_tile_h3 = take(sizeof(unsigned short) * (size_t)W * nt * kBins3);
   p.o_tile_pre = take(sizeof(int2) * (size_t)W * nt);
+  p.o_tile_rng = take(sizeof(int2) * (size_t)W * nt);
   p.o_lists = take(sizeof(int2) * (size_t)kNumLists * W * nt);
   p.o_pend_tau = take(sizeof(unsigned) * seg);
   p.total = o;
@@ -192,6 +193,7 @@ int acc_create(const acc_config* cfg, void* workspace, size_t workspace_bytes, a
   ctx->d_tile_cnt = reinterpret_cast<int2*>(ws + p.o_tile_cnt);
   ctx->d_tile_h3 = reinterpret_cast<unsigned short*>(ws + p.o_tile_h3);
   ctx->d_tile_pre = reinterpret_cast<int2*>(ws + p.o_tile_pre);
+  ctx->d_tile_rng = reinterpret_cast<int2*>(ws + p.o_tile_rng);
   ctx->d_lists = reinterpret_cast<int2*>(ws + p.o_lists);
   ctx->d_pend_tau = reinterpret_cast<unsigned*>(ws + p.o_pend_tau);
 
@@ -290,7 +292,18 @@ int acc_detect_regime(acc_ctx* ctx, const double* norm2_curr, double* norm2_prev
   if (!aligned16(delta)) return ACC_EALIGN;
   ctx->last_launches = 0;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  cudaError_t e = launch_detect(ctx, norm2_curr, norm2_prev, nullptr, lr_curr, lr_next, level, s);
+  cudaError_t e = launch_detect(ctx, norm2_curr, norm2_prev, nullptr, lr_curr, lr_next, nullptr, level, s);
+  if (e == cudaSuccess && delta) e = cudaMemsetAsync(delta, 0, sizeof(float) * (size_t)ctx->cfg.worker_stride, s);
+  return finish(e);
+}
+
+int acc_detect_regime_lr(acc_ctx* ctx, const double* norm2_curr, double* norm2_prev, const float* lr_pair,
+                         uint8_t* level, float* delta, void* stream) {
+  if (!ctx || !norm2_curr || !norm2_prev || !lr_pair || !level) return ACC_EINVAL;
+  if (!aligned16(delta) || (reinterpret_cast<uintptr_t>(lr_pair) & 3u)) return ACC_EALIGN;
+  ctx->last_launches = 0;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  cudaError_t e = launch_detect(ctx, norm2_curr, norm2_prev, nullptr, 0.f, 0.f, lr_pair, level, s);
   if (e == cudaSuccess && delta) e = cudaMemsetAsync(delta, 0, sizeof(float) * (size_t)ctx->cfg.worker_stride, s);
   return finish(e);
 }
@@ -303,7 +316,7 @@ int acc_detect_regime_diff(acc_ctx* ctx, const double* norm2_diff, const double*
   ctx->last_launches = 0;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   const size_t bytes = sizeof(float) * (size_t)ctx->cfg.worker_stride;
-  cudaError_t e = launch_detect(ctx, norm2_curr, norm2_prev, norm2_diff, lr_curr, lr_next, level, s);
+  cudaError_t e = launch_detect(ctx, norm2_curr, norm2_prev, norm2_diff, lr_curr, lr_next, nullptr, level, s);
   if (e == cudaSuccess) e = cudaMemcpyAsync(delta_prev, delta, bytes, cudaMemcpyDeviceToDevice, s);
   if (e == cudaSuccess) e = cudaMemsetAsync(delta, 0, bytes, s);
   return finish(e);

@@ -165,11 +165,15 @@ __global__ void moments_final_kernel(const DevLayer* __restrict__ layers, const 
 // Algorithm 1 per layer, in product form so that a zero previous norm needs no division.
 // With n2d (squared norms of the difference of the two accumulated gradients) the variant criterion
 // ||D_prev - D_curr|| >= eta ||D_prev|| is used instead of | ||D_prev|| - ||D_curr|| | >= eta ||D_prev||.
+// With lr_dev (two DEVICE floats: current and next learning rate) the rates are read from there instead of the
+// arguments, so that a captured graph follows a learning-rate schedule.
 __global__ void detect_kernel(const double* __restrict__ n2c, double* __restrict__ n2p,
-                              const double* __restrict__ n2d, float lr_curr, float lr_next, double eta,
-                              uint8_t* __restrict__ level, int n_layers) {
+                              const double* __restrict__ n2d, float lr_curr, float lr_next,
+                              const float* __restrict__ lr_dev, double eta, uint8_t* __restrict__ level,
+                              int n_layers) {
   const int l = blockIdx.x * blockDim.x + threadIdx.x;
   if (l >= n_layers) return;
+  if (lr_dev != nullptr) { lr_curr = lr_dev[0]; lr_next = lr_dev[1]; }
   const double cur = n2c[l], prev = n2p[l];
   uint8_t lv;
   if (prev < 0.0) {
@@ -226,11 +230,12 @@ cudaError_t launch_layer_msdr(acc_ctx* ctx, const float* buf, long long stride, 
 }
 
 cudaError_t launch_detect(acc_ctx* ctx, const double* n2c, double* n2p, const double* n2d, float lr_curr,
-                          float lr_next, uint8_t* level, cudaStream_t s) {
+                          float lr_next, const float* lr_dev, uint8_t* level, cudaStream_t s) {
   const int L = ctx->cfg.n_layers;
   {
     PhaseTimer pt(ctx, PH_DETECT, s);
-    detect_kernel<<<(L + 127) / 128, 128, 0, s>>>(n2c, n2p, n2d, lr_curr, lr_next, (double)ctx->cfg.eta, level, L);
+    detect_kernel<<<(L + 127) / 128, 128, 0, s>>>(n2c, n2p, n2d, lr_curr, lr_next, lr_dev, (double)ctx->cfg.eta, level,
+                                                  L);
   }
   return cudaGetLastError();
 }

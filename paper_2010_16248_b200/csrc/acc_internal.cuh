@@ -55,6 +55,7 @@ constexpr int kSelDense = 0, kSelList = 1, kSelListPred = 2, kSelStaged = 3, kSe
 // pass, tiles of dense segments, tiles the select pass must read, tiles served from staged entries.
 constexpr int kListCollect = 0, kListDense = 1, kListSelect = 2, kListStaged = 3, kNumLists = 4;
 constexpr int kListCountWord = 8;  // the lists' lengths live at words 8..11 of the per-step word block
+constexpr int kTicketWord = 16;    // tile ticket of the decompress pass, same block (cleared at the start of a step)
 constexpr unsigned kNoPendingTau = 0xffffffffu;  // no key is larger: nothing pending
 constexpr int kPredTileCap = 2048;  // keys one tile may hand to a predicted list (more: overflow, fall back)
 
@@ -85,7 +86,7 @@ struct Plan {
   long long vec_floats = 0;  // packed VECTOR elements (each layer starts at a multiple of 4)
   // workspace offsets (bytes)
   size_t o_layers = 0, o_col_items = 0, o_tiles = 0, o_mat_layers = 0, o_vec_tiles = 0, o_mat_tiles = 0, o_status = 0,
-         o_part = 0, o_ppart = 0, o_pending = 0, o_norm_part = 0, o_hist = 0, o_sel = 0, o_pred = 0, o_cand = 0, o_tile_cand = 0, o_tile_cnt = 0, o_tile_h3 = 0, o_tile_pre = 0, o_lists = 0, o_pend_tau = 0,
+         o_part = 0, o_ppart = 0, o_pending = 0, o_norm_part = 0, o_hist = 0, o_sel = 0, o_pred = 0, o_cand = 0, o_tile_cand = 0, o_tile_cnt = 0, o_tile_h3 = 0, o_tile_pre = 0, o_tile_rng = 0, o_lists = 0, o_pend_tau = 0,
          hist_bytes = 0, total = 0;
 };
 
@@ -127,6 +128,7 @@ struct acc_ctx {
   int2* d_tile_cnt = nullptr;
   unsigned short* d_tile_h3 = nullptr;
   int2* d_tile_pre = nullptr;
+  int2* d_tile_rng = nullptr;        // per (worker, tile): the tile's entries [first, end) inside the worker's packed segment
   int2* d_lists = nullptr;           // [kNumLists][W * tiles] work lists of (worker, tile)
   unsigned* d_pend_tau = nullptr;    // lazy TopK: per (worker, layer) threshold of the last step whose kept entries
                                      // (key > threshold) are still to be zeroed in err; kNoPendingTau: none
@@ -147,7 +149,7 @@ cudaError_t launch_layer_norms(acc_ctx* ctx, const float* buf, long long stride,
 cudaError_t launch_layer_msdr(acc_ctx* ctx, const float* buf, long long stride, int n_bufs, double* moments,
                               double* msdr, cudaStream_t s);
 cudaError_t launch_detect(acc_ctx* ctx, const double* n2c, double* n2p, const double* n2d, float lr_curr,
-                          float lr_next, uint8_t* level, cudaStream_t s);
+                          float lr_next, const float* lr_dev, uint8_t* level, cudaStream_t s);
 cudaError_t launch_powersgd(acc_ctx* ctx, const float* grads, float* err, float* q, float* p_hat,
                             const uint8_t* level, float* out, float* delta, SgdTail tail, cudaStream_t s);
 cudaError_t prepare_powersgd();

@@ -1,4 +1,4 @@
-// PowerSGD rank-r step with error feedback over W workers (compressor of Section 5.2).
+// PowerSGD rank-r step with error feedback over W workers (compressor of the Section "Accordion with PowerSGD").
 //
 // Because every product of the step is linear in the workers' matrices, the factors only depend on
 // the mean matrix  Mbar = (1/W) sum_w (g_w + e_w):   P = Mbar Q,  Q' = Mbar^T P^,  A = P^ Q'^T.

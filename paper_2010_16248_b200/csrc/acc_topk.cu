@@ -1,4 +1,4 @@
-// TopK-K% sparsification with error feedback (sparsifier of Section 5.3), exact and order-preserving.
+// TopK-K% sparsification with error feedback (sparsifier of the Section "Accordion with TopK"), exact and order-preserving.
 //
 // Selection is a three-level radix select on the 31-bit magnitude pattern key = bits(M) & 0x7fffffff
 // (12 + 12 + 7 bits, shared-memory histograms), followed by an ordered compaction:
@@ -23,6 +23,7 @@
 // No floating-point atomics and no inter-block waiting: same input, same bits.
 #include <algorithm>
 
+#include "acc_async.cuh"
 #include "acc_internal.cuh"
 
 namespace acc {
@@ -813,7 +814,8 @@ __device__ __forceinline__ int block_excl_scan_256(int v, int* wsum, int* total)
 __global__ void __launch_bounds__(256)
 topk_tile_scan_kernel(const DevLayer* __restrict__ layers, const int* __restrict__ mat_layers, int n_mat,
                       int n_tiles, int W, const Select* __restrict__ sel, int2* __restrict__ tile_pre,
-                      int2* __restrict__ tile_own, unsigned* __restrict__ any_list, int2* __restrict__ lists) {
+                      int2* __restrict__ tile_own, int2* __restrict__ tile_rng, unsigned* __restrict__ any_list,
+                      int2* __restrict__ lists) {
   __shared__ int wsum[8];
   __shared__ unsigned s_base;
   const int seg = blockIdx.x, w = seg / n_mat, l = mat_layers[seg % n_mat];
@@ -850,7 +852,10 @@ topk_tile_scan_kernel(const DevLayer* __restrict__ layers, const int* __restrict
     tile_pre[tb + t] = run;
     tile_own[tb + t] = c;  // the tile's own (above, ties), for the select pass
     if (c.x != 0 || (c.y != 0 && run.y < s.need)) *dst++ = make_int2(w, L.tile0 + t);
+    const int lo = min(run.x + min(run.y, s.need), s.k);  // (the clamps hold by construction)
     run.x += c.x; run.y += c.y;
+    // the tile's entries inside the worker's packed segment, for the decompress pass
+    tile_rng[tb + t] = make_int2(lo, min(run.x + min(run.y, s.need), s.k));
   }
 }
 
@@ -958,7 +963,7 @@ __device__ __forceinline__ void select_tile(const Tile& t, const unsigned tau, c
 // outlasts the tile) or none is (no tie in the tile, or the budget ran out before it) -- every tile of a segment but
 // the one where the budget runs out.  An entry is then kept iff its key >= thr (tau or tau + 1), one mask and one
 // scan instead of two, and the positions follow from the count of kept entries alone.
-template <bool FULL, bool LAZY>
+template <bool FULL, bool LAZY, bool SPARSE>
 __device__ __forceinline__ void select_tile_simple(const Tile& t, unsigned thr, unsigned tau, bool zero_ties,
                                                    int base, int k, float* __restrict__ m,
                                                    float* __restrict__ vals, int32_t* __restrict__ idx, long long seg,
@@ -996,6 +1001,44 @@ __device__ __forceinline__ void select_tile_simple(const Tile& t, unsigned thr, 
   if (km == 0) return;
   int pos0 = base;
   for (int i = 0; i < wi; ++i) pos0 += (int)wtot[i];
+  if (SPARSE) {
+    // Few entries kept (the usual case: K of 1 % to 10 %): walk the set bits of the mask instead of all 32
+    // elements -- a warp runs as many rounds as its busiest lane has kept entries -- and read the kept values
+    // again (the lines were just loaded).  First position of this lane in each j: warp totals of the earlier j
+    // (running byte sums of t0 / t1) plus the lane's exclusive prefix inside j.
+    const unsigned e0x = i0 - c[0], e1x = i1 - c[1];  // exclusive prefixes over the lanes, one byte per j (< 128)
+    unsigned pj[4];  // kept entries of the warp in the earlier j, two 16-bit sums per word (a warp holds 1024 elements)
+    {
+      unsigned runj = 0;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        if ((j & 1) == 0) pj[j >> 1] = runj;
+        else pj[j >> 1] |= runj << 16;
+        runj += ((j < 4 ? t0 : t1) >> (8 * (j & 3))) & 0xffu;
+      }
+    }
+    unsigned rem = km;
+    int last_j = -1, run = 0;
+    while (rem) {
+      const int b = __ffs((int)rem) - 1;
+      rem &= rem - 1;
+      const int j = b >> 2, e = b & 3;
+      if (j != last_j) { last_j = j; run = 0; }
+      const int e0 = 4 * (wi * 256 + j * 32 + lane);
+      const unsigned pw = j < 4 ? (j < 2 ? pj[0] : pj[1]) : (j < 6 ? pj[2] : pj[3]);
+      const int pos = pos0 + (int)((pw >> (16 * (j & 1))) & 0xffffu) +
+                      (int)(((j < 4 ? e0x : e1x) >> (8 * (j & 3))) & 0xffu) + run;
+      ++run;
+      if ((unsigned)pos < (unsigned)k) {
+        const float v = m[e0 + e];
+        vals[seg + pos] = v;
+        idx[seg + pos] = t.elem0 + e0 + e;
+        if (!LAZY) m[e0 + e] = 0.f;
+        else if (zero_ties && key_of(v) == tau && __float_as_uint(v) != 0u) m[e0 + e] = 0.f;
+      }
+    }
+    return;
+  }
 #pragma unroll
   for (int j = 0; j < 8; ++j) {
     const unsigned nib = (km >> (4 * j)) & 15u;
@@ -1076,8 +1119,11 @@ topk_select_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict__
     if (all_ties || no_ties) {
       const unsigned thr = all_ties ? tau : tau + 1u;
       const int base = p.x + min(p.y, need);
-      if (t.nelem == kTile) select_tile_simple<true, LAZY>(t, thr, tau, all_ties && o.y != 0, base, k, m, vals, idx, seg, wtot);
-      else select_tile_simple<false, LAZY>(t, thr, tau, all_ties && o.y != 0, base, k, m, vals, idx, seg, wtot);
+      const bool zt = all_ties && o.y != 0;
+      const int kept = o.x + (all_ties ? o.y : 0);  // entries of the tile that will be written
+      if (t.nelem != kTile) select_tile_simple<false, LAZY, false>(t, thr, tau, zt, base, k, m, vals, idx, seg, wtot);
+      else if (kept <= kTile / 5) select_tile_simple<true, LAZY, true>(t, thr, tau, zt, base, k, m, vals, idx, seg, wtot);
+      else select_tile_simple<true, LAZY, false>(t, thr, tau, zt, base, k, m, vals, idx, seg, wtot);
     } else {
       if (t.nelem == kTile) select_tile<true, LAZY>(t, tau, need, k, p, m, vals, idx, seg, wtot);
       else select_tile<false, LAZY>(t, tau, need, k, p, m, vals, idx, seg, wtot);
@@ -1185,103 +1231,134 @@ topk_finalize_staged_kernel(const DevLayer* __restrict__ layers, const Tile* __r
   }
 }
 
-// Pass F.  Scatter-decompress and average: one block per tile; the tile of `out` is accumulated in shared
-// memory from every worker's packed entries that fall into it, workers in order (fixed fp32 order), then
+// Pass F.  Scatter-decompress and average: the tile of `out` is accumulated in shared memory from every worker's
+// packed entries that fall into it (their ranges come from the tile scan), workers in order (fixed fp32 order), then
 // scaled by 1/W.  VECTOR tiles: out = mean_w g_w, delta += g_decider.
+// The entries of all workers (as many as the staging area holds: always all of them for W <= 8 at K <= 12 %) are
+// brought into shared memory by asynchronous 4-byte copies issued back to back, so that a tile pays one memory
+// latency whatever the number of workers and entries; the adds then run from shared memory, one worker after the
+// other (an element may be kept by several workers and the order of its sum is fixed).
+// Persistent blocks take tiles by ticket (one atomic per tile, requested two tiles ahead), and the ranges of a
+// block's next tile are fetched while the current one is worked on.
 // SGD: the optimiser tail is applied to every element of out where it is written.
+constexpr int kDecStage = kTile;  // staged entries per round (a worker has at most kTile entries in a tile)
+constexpr size_t kDecSmemBytes = sizeof(float) * kTile + (sizeof(int) + sizeof(float)) * kDecStage +
+                                 sizeof(int) * 2 * kMaxWorkers + 16;
+
+__device__ __forceinline__ void cp_async4(void* dst_smem, const void* src) {
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(smem_u32(dst_smem)), "l"(__cvta_generic_to_global(src))
+               : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
+
 template <bool SGD>
-__global__ void __launch_bounds__(256, 3)
-topk_decompress_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict__ tiles, int n_tiles, int n_mat,
-                       const float* __restrict__ grads, const Select* __restrict__ sel,
-                       const int2* __restrict__ tile_pre, const float* __restrict__ vals,
-                       const int32_t* __restrict__ idx, float* __restrict__ out, float* __restrict__ delta,
-                       long long stride, long long capacity, int W, int decider, float inv_w, const SgdTail tail) {
-  __shared__ float acc[kTile];
-  __shared__ int r_lo[kMaxWorkers], r_hi[kMaxWorkers];
-  const int ti = blockIdx.x;
-  const Tile t = tiles[ti];
-  const DevLayer L = layers[t.layer];
-  const long long base = L.offset + t.elem0;
+__global__ void __launch_bounds__(256, 2)
+topk_decompress_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict__ tiles, int n_tiles,
+                       const float* __restrict__ grads, const int2* __restrict__ tile_rng,
+                       const float* __restrict__ vals, const int32_t* __restrict__ idx, float* __restrict__ out,
+                       float* __restrict__ delta, long long stride, long long capacity, int W, int decider,
+                       float inv_w, unsigned* __restrict__ ticket, const SgdTail tail) {
+  extern __shared__ __align__(16) unsigned char dec_smem[];
+  float* acc = reinterpret_cast<float*>(dec_smem);             // [kTile]
+  int* s_idx = reinterpret_cast<int*>(acc + kTile);            // [kDecStage]
+  float* s_val = reinterpret_cast<float*>(s_idx + kDecStage);  // [kDecStage]
+  int* r_lo = reinterpret_cast<int*>(s_val + kDecStage);       // [kMaxWorkers]
+  int* r_hi = r_lo + kMaxWorkers;                              // [kMaxWorkers]
+  int* s_tile = r_hi + kMaxWorkers;                            // [2]
+  constexpr int kRng = kMaxWorkers / 256;  // ranges a thread holds for the block's next tile
   SgdHyper h = {0.f, 0.f, 0.f};
   if (SGD) h = sgd_hyper(tail);
-  if (L.kind != ACC_MATRIX) {
-    vector_tile_mean(grads + base, stride, W, decider, inv_w, t.nelem, delta != nullptr ? delta + base : nullptr,
-                     [&](int i, float4 v) {
-                       *reinterpret_cast<float4*>(out + base + i) = v;
-                       if (SGD) sgd_apply4(tail, h, base + i, v);
-                     },
-                     [&](int i, float v) {
-                       out[base + i] = v;
-                       if (SGD) sgd_apply1(tail, h, base + i, v);
-                     });
-    return;
-  }
-  for (int i = threadIdx.x; i < kTile; i += blockDim.x) acc[i] = 0.f;
-  // the tile's range inside every worker's packed segment, all workers at once
-  const bool last = ti == L.tile0 + L.ntiles - 1;
-  for (int w = threadIdx.x; w < W; w += blockDim.x) {
-    const Select s = sel[w * n_mat + L.mat];
-    const int2 p0 = tile_pre[(long long)w * n_tiles + ti];
-    int end = s.k;
-    if (!last) {
-      const int2 p1 = tile_pre[(long long)w * n_tiles + ti + 1];
-      end = p1.x + min(p1.y, s.need);
-    }
-    r_lo[w] = min(p0.x + min(p0.y, s.need), s.k);  // (the clamps hold by construction)
-    r_hi[w] = min(end, s.k);
+  if (threadIdx.x == 0) {
+    s_tile[0] = (int)atomicAdd(ticket, 1u);
+    s_tile[1] = (int)atomicAdd(ticket, 1u);
   }
   __syncthreads();
-  // Workers are added one after the other (an element may be kept by several of them and the order of the sum is
-  // fixed).  The entries of a group of workers are fetched together, before the first of them is added, so that a
-  // tile pays one memory latency per group instead of two per worker and 256 entries; what a worker has in the tile
-  // beyond the entries the registers hold (the first 512) is added by a plain loop.
-  constexpr int kGroup = 8, kHold = 2;
-  for (int w0 = 0; w0 < W; w0 += kGroup) {
-    const int g = min(kGroup, W - w0);
-    int ri[kGroup][kHold];
-    float rv[kGroup][kHold];
+  int cur = s_tile[0], nxt = s_tile[1];
+  int2 rn[kRng];
 #pragma unroll
-    for (int j = 0; j < kGroup; ++j) {
-      if (j >= g) break;
-      const long long seg = (long long)(w0 + j) * capacity + L.seg_off;
-      const int lo = r_lo[w0 + j], hi = r_hi[w0 + j];
-#pragma unroll
-      for (int u = 0; u < kHold; ++u) {
-        const int i = lo + u * 256 + (int)threadIdx.x;
-        const bool in = i < hi;
-        ri[j][u] = in ? idx[seg + i] : -1;
-        rv[j][u] = in ? vals[seg + i] : 0.f;
-      }
+  for (int u = 0; u < kRng; ++u) {
+    const int w = u * 256 + (int)threadIdx.x;
+    rn[u] = (w < W && cur < n_tiles) ? tile_rng[(long long)w * n_tiles + cur] : make_int2(0, 0);
+  }
+  int l_tile0 = 0, l_tile1 = 0, l_kind = ACC_VECTOR;  // the layer whose record is held: tiles [l_tile0, l_tile1)
+  long long l_size = 0, l_offset = 0, l_seg_off = 0;
+  while (cur < n_tiles) {
+    __syncthreads();  // acc, the ranges and s_tile of the previous tile are no longer read
+    unsigned tick = 0;
+    if (threadIdx.x == 0) tick = atomicAdd(ticket, 1u);  // the tile after the next one
+    if (cur < l_tile0 || cur >= l_tile1) {
+      const DevLayer& L = layers[tiles[cur].layer];
+      l_tile0 = L.tile0; l_tile1 = L.tile0 + L.ntiles; l_kind = L.kind;
+      l_size = (long long)L.rows * L.cols; l_offset = L.offset; l_seg_off = L.seg_off;
     }
+    const int elem0 = (cur - l_tile0) * kTile;
+    const int nelem = (int)min((long long)kTile, l_size - elem0);
+    const long long base = l_offset + elem0;
 #pragma unroll
-    for (int j = 0; j < kGroup; ++j) {
-      if (j >= g) break;
-#pragma unroll
-      for (int u = 0; u < kHold; ++u) {
-        const unsigned li = (unsigned)(ri[j][u] - t.elem0);  // an absent entry (-1) falls outside the tile
-        if (li < (unsigned)kTile) acc[li] += rv[j][u];
-      }
-      const int lo = r_lo[w0 + j], hi = r_hi[w0 + j];
-      if (hi - lo > kHold * 256) {  // uniform over the block
-        const long long seg = (long long)(w0 + j) * capacity + L.seg_off;
-        for (int i = lo + kHold * 256 + (int)threadIdx.x; i < hi; i += 256) {
-          const unsigned li = (unsigned)(idx[seg + i] - t.elem0);
-          if (li < (unsigned)kTile) acc[li] += vals[seg + i];
+    for (int u = 0; u < kRng; ++u) {
+      const int w = u * 256 + (int)threadIdx.x;
+      if (w < W) { r_lo[w] = rn[u].x; r_hi[w] = rn[u].y; }
+      rn[u] = (w < W && nxt < n_tiles) ? tile_rng[(long long)w * n_tiles + nxt] : make_int2(0, 0);
+    }
+    if (l_kind != ACC_MATRIX) {
+      vector_tile_mean(grads + base, stride, W, decider, inv_w, nelem, delta != nullptr ? delta + base : nullptr,
+                       [&](int i, float4 v) {
+                         *reinterpret_cast<float4*>(out + base + i) = v;
+                         if (SGD) sgd_apply4(tail, h, base + i, v);
+                       },
+                       [&](int i, float v) {
+                         out[base + i] = v;
+                         if (SGD) sgd_apply1(tail, h, base + i, v);
+                       });
+    } else {
+      for (int i = threadIdx.x; i < kTile / 4; i += blockDim.x)
+        reinterpret_cast<float4*>(acc)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+      __syncthreads();  // the ranges are in place (and acc is clear)
+      for (int w0 = 0; w0 < W;) {
+        // the workers [w0, w1) whose entries in this tile fit the staging area together (at least one)
+        int w1 = w0, total = 0;
+        while (w1 < W && total + (r_hi[w1] - r_lo[w1]) <= kDecStage) { total += r_hi[w1] - r_lo[w1]; ++w1; }
+        if (w1 == w0) break;  // (cannot happen: a worker has at most kTile entries in a tile)
+        int o = 0;
+        for (int w = w0; w < w1; ++w) {
+          const long long seg = (long long)w * capacity + l_seg_off;
+          const int lo = r_lo[w], n = r_hi[w] - lo;
+          for (int i = threadIdx.x; i < n; i += 256) {
+            cp_async4(s_idx + o + i, idx + seg + lo + i);
+            cp_async4(s_val + o + i, vals + seg + lo + i);
+          }
+          o += n;
         }
+        cp_async_wait_all();
+        __syncthreads();
+        o = 0;
+        for (int w = w0; w < w1; ++w) {
+          const int n = r_hi[w] - r_lo[w];
+          for (int i = threadIdx.x; i < n; i += 256) {
+            const unsigned li = (unsigned)(s_idx[o + i] - elem0);
+            if (li < (unsigned)kTile) acc[li] += s_val[o + i];
+          }
+          o += n;
+          __syncthreads();  // the next worker may add to the same elements; the last one frees the staging area
+        }
+        w0 = w1;
       }
-      __syncthreads();
+      const int n4 = nelem >> 2;
+      for (int i = threadIdx.x; i < n4; i += blockDim.x) {
+        const float4 a = reinterpret_cast<const float4*>(acc)[i];
+        const float4 v = make_float4(a.x * inv_w, a.y * inv_w, a.z * inv_w, a.w * inv_w);
+        st_stream4(out + base + 4 * i, v);
+        if (SGD) sgd_apply4(tail, h, base + 4 * i, v);
+      }
+      for (int i = 4 * n4 + threadIdx.x; i < nelem; i += blockDim.x) {
+        out[base + i] = acc[i] * inv_w;
+        if (SGD) sgd_apply1(tail, h, base + i, acc[i] * inv_w);
+      }
     }
-  }
-  const int n4 = t.nelem >> 2;
-  for (int i = threadIdx.x; i < n4; i += blockDim.x) {
-    const float4 v = make_float4(acc[4 * i] * inv_w, acc[4 * i + 1] * inv_w, acc[4 * i + 2] * inv_w,
-                                 acc[4 * i + 3] * inv_w);
-    st_stream4(out + base + 4 * i, v);
-    if (SGD) sgd_apply4(tail, h, base + 4 * i, v);
-  }
-  for (int i = 4 * n4 + threadIdx.x; i < t.nelem; i += blockDim.x) {
-    out[base + i] = acc[i] * inv_w;
-    if (SGD) sgd_apply1(tail, h, base + i, acc[i] * inv_w);
+    if (threadIdx.x == 0) s_tile[0] = (int)tick;
+    __syncthreads();
+    cur = nxt;
+    nxt = s_tile[0];
   }
 }
 
@@ -1460,8 +1537,8 @@ static cudaError_t launch_topk_select_part(acc_ctx* ctx, const float* grads, flo
     {
       PhaseTimer pt(ctx, PH_TOPK_PICK3_SCAN, s);
       topk_tile_scan_kernel<<<W * n_mat, 256, 0, s>>>(ctx->d_layers, ctx->d_mat_layers, n_mat, nt, W, ctx->d_sel,
-                                                      ctx->d_tile_pre, ctx->d_tile_cnt, ctx->d_any_list,
-                                                      ctx->d_lists);
+                                                      ctx->d_tile_pre, ctx->d_tile_cnt, ctx->d_tile_rng,
+                                                      ctx->d_any_list, ctx->d_lists);
     }
   }
   if (n_mat > 0) {
@@ -1497,20 +1574,24 @@ cudaError_t launch_topk(acc_ctx* ctx, const float* grads, float* err, const uint
                         int32_t* idx, int32_t* counts, float* out, float* delta, SgdTail tail, cudaStream_t s) {
   const Plan& pl = ctx->plan;
   const acc_config& c = ctx->cfg;
-  const int nt = (int)pl.tiles.size(), W = c.n_workers, n_mat = pl.n_mat;
+  const int nt = (int)pl.tiles.size(), W = c.n_workers;
   const float inv_w = 1.0f / (float)W;
   const cudaError_t e = launch_topk_select_part(ctx, grads, err, level, vals, idx, counts, delta, s);
   if (e != cudaSuccess) return e;
   {
     PhaseTimer pt(ctx, PH_TOPK_DECOMPRESS, s);
+    // persistent blocks (two fit an SM), tiles handed out by ticket; the ticket word was cleared with the
+    // histograms at the start of the step
+    const int dgrid = std::min(nt, ctx->sm_count * 2);
+    unsigned* ticket = ctx->d_any_list + kTicketWord;
     if (tail.params)
-      topk_decompress_kernel<true><<<nt, 256, 0, s>>>(ctx->d_layers, ctx->d_tiles, nt, n_mat, grads, ctx->d_sel,
-                                                      ctx->d_tile_pre, vals, idx, out, delta, c.worker_stride,
-                                                      pl.capacity, W, c.decider, inv_w, tail);
+      topk_decompress_kernel<true><<<dgrid, 256, kDecSmemBytes, s>>>(ctx->d_layers, ctx->d_tiles, nt, grads, ctx->d_tile_rng, vals,
+                                                         idx, out, delta, c.worker_stride, pl.capacity, W, c.decider,
+                                                         inv_w, ticket, tail);
     else
-      topk_decompress_kernel<false><<<nt, 256, 0, s>>>(ctx->d_layers, ctx->d_tiles, nt, n_mat, grads, ctx->d_sel,
-                                                       ctx->d_tile_pre, vals, idx, out, delta, c.worker_stride,
-                                                       pl.capacity, W, c.decider, inv_w, tail);
+      topk_decompress_kernel<false><<<dgrid, 256, kDecSmemBytes, s>>>(ctx->d_layers, ctx->d_tiles, nt, grads, ctx->d_tile_rng, vals,
+                                                          idx, out, delta, c.worker_stride, pl.capacity, W, c.decider,
+                                                          inv_w, ticket, tail);
   }
   return cudaGetLastError();
 }
@@ -1551,8 +1632,15 @@ __global__ void topk_clear_pending_kernel(unsigned* __restrict__ pend_tau, int n
 // Once per context, at creation: how many blocks of the first pass fit an SM.
 cudaError_t prepare_topk(acc_ctx* ctx) {
   int occ = 0;
-  const cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, topk_ef_hist1_kernel, 256, 0);
+  cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, topk_ef_hist1_kernel, 256, 0);
   ctx->occ_topk_first_pass = occ > 0 ? occ : 1;
+  // the decompress pass stages its entries in more than 48 KB of dynamic shared memory
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(topk_decompress_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)kDecSmemBytes);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(topk_decompress_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)kDecSmemBytes);
   return e;
 }
 

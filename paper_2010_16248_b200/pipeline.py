@@ -45,6 +45,11 @@ class AccordionStep:
         self.norm2_prev = torch.full((L,), -1.0, dtype=torch.float64, device=dev)
         self.t = 0
         self.launches = 0
+        # the detector's learning-rate pair as device scalars (Algorithm 1 declares a critical regime when the rate
+        # is about to decay): the captured iteration reads them, ``set_detector_lr`` rewrites them between replays
+        self.lr_pair = torch.tensor([0.1, 0.1], dtype=torch.float32, device=dev)
+        self._lr_pair_host = (0.1, 0.1)
+        self._lr_from_device = False
         self.lazy_residual = lazy_residual
         self.overlap = overlap
         self._side = torch.cuda.Stream(device=dev)
@@ -84,8 +89,7 @@ class AccordionStep:
             if self.t % self.check_every == 0:
                 c.acc_layer_norms(self.delta, 1, self.norm2_curr, stream=main)
                 self.launches += c.last_launch_count()
-                c.acc_detect_regime(self.norm2_curr, self.norm2_prev, lr_curr, lr_next, self.level, self.delta, main)
-                self.launches += c.last_launch_count()
+                self._detect(lr_curr, lr_next, main)
             return
         if "powersgd" in self.compressors:
             if self.params is not None:
@@ -108,8 +112,23 @@ class AccordionStep:
         if self.t % self.check_every == 0:
             c.acc_layer_norms(self.delta, 1, self.norm2_curr, stream=stream)
             self.launches += c.last_launch_count()
-            c.acc_detect_regime(self.norm2_curr, self.norm2_prev, lr_curr, lr_next, self.level, self.delta, stream)
-            self.launches += c.last_launch_count()
+            self._detect(lr_curr, lr_next, stream)
+
+    def _detect(self, lr_curr, lr_next, stream):
+        if self._lr_from_device:
+            self.ctx.acc_detect_regime_lr(self.norm2_curr, self.norm2_prev, self.lr_pair, self.level, self.delta, stream)
+        else:
+            self.ctx.acc_detect_regime(self.norm2_curr, self.norm2_prev, lr_curr, lr_next, self.level, self.delta,
+                                       stream)
+        self.launches += self.ctx.last_launch_count()
+
+    def set_detector_lr(self, lr_curr: float, lr_next: float):
+        """Learning rates the captured regime test will see (current iteration's and the next one's)."""
+        pair = (float(lr_curr), float(lr_next))
+        if pair != self._lr_pair_host:
+            self.lr_pair[0:1].fill_(pair[0])
+            self.lr_pair[1:2].fill_(pair[1])
+            self._lr_pair_host = pair
 
     def flush(self, stream=None):
         """Lazy mode: materialises the error memories (what the last step compressed is removed from ``err``), so
@@ -129,10 +148,13 @@ class AccordionStep:
         """Captures one iteration as CUDA graphs, for each of the given fixed device gradient buffers (the
         caller refills them, or cycles through them, before every replay): one graph for an ordinary
         iteration and one for an iteration that ends a detection window (with the norm and regime kernels).
-        Which rank or K a layer gets is decided on the device from ``level``, so the same graphs serve every
-        iteration.  ``step_graph(slot)`` replays the right one.  Every library call is asynchronous and
+        Which rank or K a layer gets is decided on the device from ``level``, and the regime test reads its two
+        learning rates from device scalars, so the same graphs serve every iteration of a schedule.
+        ``step_graph(slot, lr_curr, lr_next)`` replays the right one.  Every library call is asynchronous and
         allocation-free, hence capturable."""
         torch.cuda.synchronize(self.device)
+        self.set_detector_lr(lr_curr, lr_next)
+        self._lr_from_device = True
         saved_t, saved_launches = self.t, self.launches
         side = torch.cuda.Stream(device=self.device)
         self._graphs, self._graph_launches = [], []
@@ -150,12 +172,16 @@ class AccordionStep:
                 self._graphs.append(pair)
                 self._graph_launches.append(counts)
         torch.cuda.synchronize(self.device)
+        self._lr_from_device = False
         self.t, self.launches = saved_t, saved_launches
 
-    def step_graph(self, slot: int = 0):
-        """Replays the captured iteration that reads gradient buffer ``slot`` (see ``capture_graphs``)."""
+    def step_graph(self, slot: int = 0, lr_curr: Optional[float] = None, lr_next: Optional[float] = None):
+        """Replays the captured iteration that reads gradient buffer ``slot`` (see ``capture_graphs``); the learning
+        rates, when given, are what the regime test of this iteration sees (unchanged otherwise)."""
         self.t += 1
         which = 1 if self.t % self.check_every == 0 else 0
+        if which and lr_curr is not None and lr_next is not None:
+            self.set_detector_lr(lr_curr, lr_next)
         self._graphs[slot][which].replay()
         self.launches += self._graph_launches[slot][which]
 
@@ -219,18 +245,84 @@ class BatchSizeStep:
         return int(self.batch.item())
 
 
+def _layer_groups(table: wl.LayerTable, n_groups: int):
+    """Contiguous runs of layers with about equal parameter counts (at least one layer each): the k-th cut falls
+    at the layer boundary whose cumulative size is nearest to k / n_groups of the total."""
+    sizes = [int(x) for x in table.sizes]
+    L = table.n_layers
+    n_groups = max(1, min(int(n_groups), L))
+    cum, run = [], 0
+    for sz in sizes:
+        run += sz
+        cum.append(run)
+    cuts, lo = [], 0
+    for k in range(1, n_groups):
+        want = run * k / n_groups
+        hi = L - (n_groups - k)  # leave a layer for each later group
+        best = min(range(lo, hi), key=lambda l: abs(cum[l] - want))
+        cuts.append(best + 1)
+        lo = best + 1
+    edges = [0] + cuts + [L]
+    return [list(range(edges[i], edges[i + 1])) for i in range(n_groups)]
+
+
+def _sub_table(table: wl.LayerTable, ids) -> wl.LayerTable:
+    """The layers ``ids`` of ``table`` at their offsets inside the same flat per-worker buffer."""
+    import numpy as np
+    ids = list(ids)
+    return wl.LayerTable([table.names[l] for l in ids], np.asarray(table.offset[ids], np.int64),
+                         np.asarray(table.rows[ids], np.int32), np.asarray(table.cols[ids], np.int32),
+                         np.asarray(table.kind[ids], np.int32), table.stride)
+
+
+class _Part:
+    """One layer group of a ``DistributedStep``: its own context (over the same flat buffers), factors or packed
+    sets, exchange buffers and the events that order its phases against its exchanges."""
+
+    def __init__(self, owner, ids, q_init):
+        self.ids = list(ids)
+        dev, n_local, world = owner.device, owner.n_local, owner.world
+        self.table = owner.table if len(self.ids) == owner.table.n_layers else _sub_table(owner.table, self.ids)
+        self.ctx = c = binding.Context(self.table, n_local, device=dev, **owner._cfg)
+        self.ids_dev = torch.tensor(self.ids, dtype=torch.long, device=dev)
+        self.level = torch.ones(len(self.ids), dtype=torch.uint8, device=dev)
+        if owner.compressor == "powersgd":
+            ql = None if q_init is None else [q_init[l] for l in self.ids]
+            self.q = c.new_q(ql if ql is not None else wl.initial_q(self.table, owner._cfg["rank_low"], device=dev))
+            self.p_hat = c.new_p()
+            self.x1 = torch.zeros(max(c.x1_floats, 4), device=dev)
+            self.x2 = torch.zeros(max(c.x2_floats, 4), device=dev)
+        else:
+            self.vals, self.idx, self.counts = c.new_topk_buffers()
+            self.vec = torch.zeros(max(c.vec_floats, 4), device=dev)
+            self.vals_all = torch.zeros(world * self.vals.numel(), device=dev)
+            self.idx_all = torch.zeros(world * self.idx.numel(), dtype=torch.int32, device=dev)
+            self.counts_all = torch.zeros(world * self.counts.numel(), dtype=torch.int32, device=dev)
+        self.done = [torch.cuda.Event() for _ in range(2)]       # a phase has produced an exchange buffer
+        self.exchanged = [torch.cuda.Event() for _ in range(2)]  # the exchange of that buffer has finished
+
+
 class DistributedStep:
     """Real workers: every rank (GPU) holds ``n_local`` workers; the compressed factors are exchanged between the
     kernels' phases (Section 5.1: all-reduce of P, then of Q, for PowerSGD; all-gather of the packed values and
     indices for TopK; the VECTOR layers ride in the first all-reduce).  Every rank ends a step with the same
     ``out``, ``q``, ``p_hat`` and ``level``: the decider's gradient is accumulated on the rank that holds it
     (global worker ``decider``), and the detector's per-layer norms are broadcast from there by a sum in which
-    the other ranks contribute zeros."""
+    the other ranks contribute zeros.
+
+    ``groups`` > 1 cuts the layers into that many contiguous groups of about equal size, each with its own
+    context over the same flat buffers, and runs the exchanges on a communication stream: while group i's rows of
+    P (or its packed sets) are in flight, the first pass of group i+1 runs, and likewise for Q'.  A layer's
+    arithmetic does not depend on the other layers of its context, so the results are those of ``groups = 1``
+    (bit for bit as long as the same implementation of the first PowerSGD pass serves both; ``extra_flags`` can
+    force one).  With one group the calls and the exchanges alternate on the caller's stream."""
 
     def __init__(self, table: wl.LayerTable, n_local: int, compressor: str = "powersgd", rank_low=2, rank_high=1,
                  topk_low_bp=1000, topk_high_bp=100, eta=0.5, gs_eps=1e-8, check_every=10, decider=0, q_init=None,
-                 device="cuda", lazy_residual=False, optimizer=None, exchange=None):
+                 device="cuda", lazy_residual=False, optimizer=None, exchange=None, groups=1, extra_flags=0):
         from . import dist_util
+        if compressor not in ("powersgd", "topk"):
+            raise ValueError(compressor)
         self.table, self.n_local, self.compressor = table, n_local, compressor
         self.x = exchange if exchange is not None else dist_util.Exchange()
         self.world, self.rank = self.x.world, self.x.rank
@@ -238,11 +330,10 @@ class DistributedStep:
         self.check_every = check_every
         self.device = dev = torch.device(device)
         self.owns_decider = decider // n_local == self.rank
-        self.ctx = binding.Context(table, n_local, device=device, rank_low=rank_low, rank_high=rank_high,
-                                   topk_low_bp=topk_low_bp, topk_high_bp=topk_high_bp, eta=eta, gs_eps=gs_eps,
-                                   decider=decider % n_local,
-                                   flags=binding.ACC_FLAG_LAZY_RESIDUAL if lazy_residual else 0)
-        L, stride, c = table.n_layers, table.stride, self.ctx
+        self._cfg = dict(rank_low=rank_low, rank_high=rank_high, topk_low_bp=topk_low_bp, topk_high_bp=topk_high_bp,
+                         eta=eta, gs_eps=gs_eps, decider=decider % n_local,
+                         flags=(binding.ACC_FLAG_LAZY_RESIDUAL if lazy_residual else 0) | extra_flags)
+        L, stride = table.n_layers, table.stride
         self.level = torch.ones(L, dtype=torch.uint8, device=dev)
         self.delta = torch.zeros(stride, device=dev) if self.owns_decider else None
         self.norm2_curr = torch.zeros(L, dtype=torch.float64, device=dev)
@@ -256,64 +347,94 @@ class DistributedStep:
             self.mom = torch.zeros(stride, device=dev)
             self.hyper = torch.tensor([optimizer["lr"], optimizer.get("momentum", 0.9),
                                        optimizer.get("weight_decay", 0.0)], dtype=torch.float32, device=dev)
-        if compressor == "powersgd":
-            self.q = c.new_q(q_init if q_init is not None else wl.initial_q(table, rank_low, device=dev))
-            self.p_hat = c.new_p()
-            self.x1 = torch.zeros(max(c.x1_floats, 4), device=dev)
-            self.x2 = torch.zeros(max(c.x2_floats, 4), device=dev)
-        elif compressor == "topk":
-            self.vals, self.idx, self.counts = c.new_topk_buffers()
-            self.vec = torch.zeros(max(c.vec_floats, 4), device=dev)
-            w = self.world
-            self.vals_all = torch.zeros(w * self.vals.numel(), device=dev)
-            self.idx_all = torch.zeros(w * self.idx.numel(), dtype=torch.int32, device=dev)
-            self.counts_all = torch.zeros(w * self.counts.numel(), dtype=torch.int32, device=dev)
-        else:
-            raise ValueError(compressor)
+        self.parts = [_Part(self, ids, q_init) for ids in _layer_groups(table, groups)]
+        # the whole table's context serves the detector (norms, Algorithm 1); with one group it is that group's
+        self.ctx = self.parts[0].ctx if len(self.parts) == 1 else binding.Context(table, n_local, device=dev,
+                                                                                   **self._cfg)
+        self._comm = torch.cuda.Stream(device=dev) if len(self.parts) > 1 else None
+        one = self.parts[0]
+        if len(self.parts) == 1:  # the single group's buffers under their plain names
+            for name in ("q", "p_hat", "x1", "x2", "vals", "idx", "counts", "vec", "vals_all", "idx_all",
+                         "counts_all"):
+                if hasattr(one, name):
+                    setattr(self, name, getattr(one, name))
+            one.level = self.level
 
     def flush(self, stream=None):
         """Lazy mode: materialises this rank's error memories (see ``AccordionStep.flush``)."""
         if not self.lazy_residual:
             return
-        if self.compressor == "powersgd":
-            self.ctx.acc_powersgd_flush(self.err, self.q, self.p_hat, stream)
-        else:
-            self.ctx.acc_topk_flush(self.err, stream)
+        for p in self.parts:
+            if self.compressor == "powersgd":
+                p.ctx.acc_powersgd_flush(self.err, p.q, p.p_hat, stream)
+            else:
+                p.ctx.acc_topk_flush(self.err, stream)
 
     def bytes_exchanged_per_step(self) -> int:
         """Bytes this rank hands to the collectives in one step (the method's communication volume)."""
         if self.compressor == "powersgd":
-            return 4 * (self.x1.numel() + self.x2.numel())
-        return 4 * (self.vals.numel() + self.idx.numel() + self.counts.numel() + self.vec.numel())
+            return 4 * sum(p.x1.numel() + p.x2.numel() for p in self.parts)
+        return 4 * sum(p.vals.numel() + p.idx.numel() + p.counts.numel() + p.vec.numel() for p in self.parts)
+
+    def _exchange(self, part, k, main, fn):
+        """Runs the exchange ``fn`` of ``part``'s k-th buffer: on the caller's stream with one group, else on the
+        communication stream, after the phase that filled the buffer and ahead of the phase that reads it."""
+        if self._comm is None:
+            with torch.cuda.stream(main):
+                fn()
+            return
+        part.done[k].record(main)
+        self._comm.wait_event(part.done[k])
+        with torch.cuda.stream(self._comm):
+            fn()
+        part.exchanged[k].record(self._comm)
+
+    def _await(self, part, k, main):
+        if self._comm is not None:
+            main.wait_event(part.exchanged[k])
 
     def step(self, grads: torch.Tensor, lr_curr: float = 0.1, lr_next: float = 0.1, stream=None):
         """One iteration on this rank's device-resident gradients ``[n_local, stride]``."""
-        c, x, scale = self.ctx, self.x, 1.0 / self.world
+        x, scale = self.x, 1.0 / self.world
+        main = stream if stream is not None else torch.cuda.current_stream(self.device)
         if self.compressor == "powersgd":
-            c.acc_powersgd_phase1(grads, self.err, self.q, self.p_hat, self.level, self.out, self.delta, self.x1,
-                                  stream)
-            x.sum_(self.x1)
-            c.acc_powersgd_phase2(self.x1, scale, self.p_hat, self.level, self.out, self.x2, stream)
-            x.sum_(self.x2)
-            c.acc_powersgd_phase3(self.err, self.q, self.p_hat, self.level, self.x1, self.x2, scale, self.out,
-                                  self.params, self.mom, self.hyper, stream)
+            for p in self.parts:
+                p.ctx.acc_powersgd_phase1(grads, self.err, p.q, p.p_hat, p.level, self.out, self.delta, p.x1, main)
+                self._exchange(p, 0, main, lambda p=p: x.sum_(p.x1))
+            for p in self.parts:
+                self._await(p, 0, main)
+                p.ctx.acc_powersgd_phase2(p.x1, scale, p.p_hat, p.level, self.out, p.x2, main)
+                self._exchange(p, 1, main, lambda p=p: x.sum_(p.x2))
+            for p in self.parts:
+                self._await(p, 1, main)
+                p.ctx.acc_powersgd_phase3(self.err, p.q, p.p_hat, p.level, p.x1, p.x2, scale, self.out, self.params,
+                                          self.mom, self.hyper, main)
         else:
-            c.acc_topk_compress(grads, self.err, self.level, self.vals, self.idx, self.counts, self.delta, self.vec,
-                                stream)
-            x.gather_into(self.vals_all, self.vals)
-            x.gather_into(self.idx_all, self.idx)
-            x.gather_into(self.counts_all, self.counts)
-            x.sum_(self.vec)
-            c.acc_topk_decompress(self.vals_all, self.idx_all, self.counts_all, self.world * self.n_local, self.vec,
-                                  scale, self.out, self.params, self.mom, self.hyper, stream)
+            def gather(p):
+                x.gather_into(p.vals_all, p.vals)
+                x.gather_into(p.idx_all, p.idx)
+                x.gather_into(p.counts_all, p.counts)
+                x.sum_(p.vec)
+            for p in self.parts:
+                p.ctx.acc_topk_compress(grads, self.err, p.level, p.vals, p.idx, p.counts, self.delta, p.vec, main)
+                self._exchange(p, 0, main, lambda p=p: gather(p))
+            for p in self.parts:
+                self._await(p, 0, main)
+                p.ctx.acc_topk_decompress(p.vals_all, p.idx_all, p.counts_all, self.world * self.n_local, p.vec,
+                                          scale, self.out, self.params, self.mom, self.hyper, main)
         self.t += 1
         if self.t % self.check_every == 0:
-            if self.owns_decider:
-                c.acc_layer_norms(self.delta, 1, self.norm2_curr, stream=stream)
-            else:
-                self.norm2_curr.zero_()
-            x.sum_(self.norm2_curr)  # a broadcast from the deciding rank (Section 3: one node decides for all)
-            c.acc_detect_regime(self.norm2_curr, self.norm2_prev, lr_curr, lr_next, self.level, self.delta, stream)
+            with torch.cuda.stream(main):
+                if self.owns_decider:
+                    self.ctx.acc_layer_norms(self.delta, 1, self.norm2_curr, stream=main)
+                else:
+                    self.norm2_curr.zero_()
+                x.sum_(self.norm2_curr)  # a broadcast from the deciding rank (Section 3: one node decides for all)
+                self.ctx.acc_detect_regime(self.norm2_curr, self.norm2_prev, lr_curr, lr_next, self.level, self.delta,
+                                           main)
+                if len(self.parts) > 1:
+                    for p in self.parts:
+                        torch.index_select(self.level, 0, p.ids_dev, out=p.level)
         return self.out
 
 

@@ -12,7 +12,7 @@ and 1-D tensors (biases, BatchNorm vectors) stay uncompressed, which is the
 convention that reproduces the "Data Sent" columns of Tables 1-2.
 
 The value distributions follow the qualitative structure the paper describes:
-low-rank-compressible layers plus noise for PowerSGD (Section 5.2), a fixed
+low-rank-compressible layers plus noise for PowerSGD (Section "Accordion with PowerSGD"), a fixed
 sparse mean plus dense noise for TopK (Section 4.3 and Appendix A.1), and a
 gradient-norm scale that changes at phase boundaries (Section 4.1).
 """

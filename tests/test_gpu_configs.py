@@ -38,22 +38,23 @@ class OracleController:
 
 
 def _run_config(w, iters, t0=0, lazy=False, topk_layers=None, topk_workers=None, psgd_check=None, topk_check=None,
-                force_level=None, paths_seen=None):
+                force_level=None, paths_seen=None, extra_flags=0):
     """Runs `iters` iterations of workload `w` starting at stream iteration t0; checks every level decision
     exactly, the TopK steps listed in topk_check and the PowerSGD steps listed in psgd_check (default: all).  With
     lazy=True a second engine in lazy-residual mode (the mode bench.py times) runs in lockstep and must
     reproduce the eager engine's outputs (out, Q, P^; packed TopK sets) bit for bit at every step, and its error
     memories after a final flush.  force_level (0 / 1) starts every engine, and the oracle's controller, at that
     level instead of the initial low-compression level.  paths_seen (a set) collects the TopK selection paths the
-    lazy engine (else the eager one) took."""
+    lazy engine (else the eager one) took.  extra_flags: further ACC_FLAG_* bits for both engines (e.g. forcing one
+    implementation of the first PowerSGD pass)."""
     table, W = w.table, w.n_workers
     stream = wl.GradientStream(w, device="cuda")
     eng = pipeline.AccordionStep(table, W, w.compressors, w.rank_low, w.rank_high, w.topk_low_bp, w.topk_high_bp,
-                                 w.eta, 1e-8, w.check_every)
+                                 w.eta, 1e-8, w.check_every, extra_flags=extra_flags)
     lz = None
     if lazy:
         lz = pipeline.AccordionStep(table, W, w.compressors, w.rank_low, w.rank_high, w.topk_low_bp, w.topk_high_bp,
-                                    w.eta, 1e-8, w.check_every, lazy_residual=True)
+                                    w.eta, 1e-8, w.check_every, lazy_residual=True, extra_flags=extra_flags)
     ctl = OracleController(table, w.check_every, w.eta)
     if force_level is not None:
         for e in (eng, lz):
@@ -213,28 +214,14 @@ def test_full_size_config5_high_level_steady_state():
     assert binding.ACC_TOPK_PATH_STAGED in paths and binding.ACC_TOPK_PATH_LIST_PREDICTED in paths, paths
 
 
-def test_full_size_config4_high_level_pending_residual():
-    """VGG-19bn set, W = 8, rank 1 on every layer with the lazy residual pending from step to step, direct and
-    pipelined first pass: both must equal the eager engine bit for bit; the oracle checks steps 1 and 3."""
+@pytest.mark.parametrize("first_pass", [binding.ACC_FLAG_PIPELINE_NEVER, binding.ACC_FLAG_PIPELINE_ALWAYS])
+def test_full_size_config4_high_level_pending_residual(first_pass):
+    """VGG-19bn set, W = 8, rank 1 on every layer with the lazy residual pending from step to step, with the direct
+    and with the pipelined first pass: the lazy engine must equal the eager one bit for bit at every step (the two
+    implementations of the pass differ from each other in the last bits: they sum the partial rows of P in
+    different orders); the oracle checks steps 1 and 3."""
     w = wl.workload(4)
-    _run_config(w, iters=4, t0=20, lazy=True, psgd_check={1, 3}, force_level=0)
-    table, W = w.table, w.n_workers
-    stream = wl.GradientStream(w, device="cuda")
-    engines = [pipeline.AccordionStep(table, W, w.compressors, w.rank_low, w.rank_high, w.topk_low_bp, w.topk_high_bp,
-                                      w.eta, 1e-8, w.check_every, lazy_residual=True, extra_flags=f)
-               for f in (binding.ACC_FLAG_PIPELINE_NEVER, binding.ACC_FLAG_PIPELINE_ALWAYS)]
-    for e in engines:
-        e.level.zero_()
-    for i in range(4):
-        g = stream.grads(20 + i)
-        for e in engines:
-            e.step(g)
-    for e in engines:
-        e.flush()
-    torch.cuda.synchronize()
-    for name in ("out_psgd", "q", "p_hat", "err_psgd"):
-        assert torch.equal(getattr(engines[0], name), getattr(engines[1], name)), name
-    assert engines[1].ctx.acc_device_status() == 0
+    _run_config(w, iters=4, t0=20, lazy=True, psgd_check={1, 3}, force_level=0, extra_flags=first_pass)
 
 
 def test_graph_replay_matches_direct_calls():
@@ -247,10 +234,16 @@ def test_graph_replay_matches_direct_calls():
     engines = [pipeline.AccordionStep(table, W, w.compressors, w.rank_low, w.rank_high, w.topk_low_bp,
                                       w.topk_high_bp, w.eta, 1e-8, 4, lazy_residual=True) for _ in range(2)]
     engines[1].capture_graphs(ring)
-    for i in range(14):  # crosses three regime checks
-        engines[0].step(ring[i % 3])
-        engines[1].step_graph(i % 3)
+    levels_after_decay = None
+    for i in range(14):  # crosses three regime checks; the second one sees a learning-rate decay (Algorithm 1)
+        lr = (0.1, 0.01) if i == 7 else (0.1, 0.1) if i < 7 else (0.01, 0.01)
+        engines[0].step(ring[i % 3], *lr)
+        engines[1].step_graph(i % 3, *lr)
+        if i == 7:
+            torch.cuda.synchronize()
+            levels_after_decay = engines[1].level.clone()
     torch.cuda.synchronize()
+    assert int(levels_after_decay.min()) == 1, "a learning-rate decay declares every layer critical"
     a, b = engines
     for name in ("level", "delta", "norm2_prev", "err_psgd", "q", "p_hat", "out_psgd", "err_topk", "vals", "idx",
                  "counts", "out_topk"):

@@ -98,6 +98,25 @@ def test_two_rank_replicas_gloo():
     assert dist_util.max_over_ranks(3.0) == 3.0                 # no process group: identity
 
 
+def test_layer_groups_partition_the_table_and_keep_the_offsets():
+    """Host logic of the grouped real-worker step: contiguous groups that cover every layer once, about equal in
+    size, and sub-tables that keep every layer at its place in the flat buffer."""
+    from paper_2010_16248_b200 import pipeline
+    for config, n_groups in ((2, 4), (4, 5), (5, 3), (1, 3)):
+        t = wl.workload(config, scale=4).table
+        groups = pipeline._layer_groups(t, n_groups)
+        assert [l for g in groups for l in g] == list(range(t.n_layers))
+        assert len(groups) == min(n_groups, t.n_layers) and all(len(g) >= 1 for g in groups)
+        for g in groups:
+            sub = pipeline._sub_table(t, g)
+            assert sub.stride == t.stride and sub.names == [t.names[l] for l in g]
+            assert np.array_equal(sub.offset, t.offset[g]) and np.array_equal(sub.rows, t.rows[g])
+            assert np.array_equal(sub.cols, t.cols[g]) and np.array_equal(sub.kind, t.kind[g])
+    t = wl.workload(5).table  # two huge layers and small ones between them: one group each side of the middle
+    sizes = [sum(int(t.sizes[l]) for l in g) for g in pipeline._layer_groups(t, 3)]
+    assert max(sizes) < 0.45 * t.n_params
+
+
 def _real_worker_rank_main(rank, world, port, out):
     """Two ranks with two workers each: the exchange helper over gloo, and the algebra of the real-worker split
     of the PowerSGD step (local P rows summed over ranks, Gram-Schmidt, local Q' rows summed) against the
