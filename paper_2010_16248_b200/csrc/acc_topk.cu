@@ -1004,8 +1004,8 @@ __device__ __forceinline__ void select_tile_simple(const Tile& t, unsigned thr, 
   if (SPARSE) {
     // Few entries kept (the usual case: K of 1 % to 10 %): walk the set bits of the mask instead of all 32
     // elements -- a warp runs as many rounds as its busiest lane has kept entries -- and read the kept values
-    // again (the lines were just loaded).  First position of this lane in each j: warp totals of the earlier j
-    // (running byte sums of t0 / t1) plus the lane's exclusive prefix inside j.
+    // again (the lines were just loaded).  First position of this lane in each j: the warp's kept entries in the
+    // earlier j (16-bit sums) plus the lane's exclusive prefix inside j.
     const unsigned e0x = i0 - c[0], e1x = i1 - c[1];  // exclusive prefixes over the lanes, one byte per j (< 128)
     unsigned pj[4];  // kept entries of the warp in the earlier j, two 16-bit sums per word (a warp holds 1024 elements)
     {
@@ -1037,8 +1037,7 @@ __device__ __forceinline__ void select_tile_simple(const Tile& t, unsigned thr, 
         else if (zero_ties && key_of(v) == tau && __float_as_uint(v) != 0u) m[e0 + e] = 0.f;
       }
     }
-    return;
-  }
+  } else {
 #pragma unroll
   for (int j = 0; j < 8; ++j) {
     const unsigned nib = (km >> (4 * j)) & 15u;
@@ -1064,6 +1063,7 @@ __device__ __forceinline__ void select_tile_simple(const Tile& t, unsigned thr, 
     }
     pos0 += (int)(((j < 4 ? t0 : t1) >> sh) & 0xffu);
   }
+  }
 }
 
 // Persistent blocks, each over a contiguous share of the select work list (the tiles of the non-staged segments
@@ -1071,7 +1071,7 @@ __device__ __forceinline__ void select_tile_simple(const Tile& t, unsigned thr, 
 // re-read only when the segment changes).  The list entry and the counters of the next tile are fetched while
 // the current one is processed, and its lines are asked into L2.
 template <bool LAZY>
-__global__ void __launch_bounds__(256, 3)
+__global__ void __launch_bounds__(256, 4)
 topk_select_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict__ tiles, int n_tiles, int n_mat,
                    float* __restrict__ err, const Select* __restrict__ sel, const int2* __restrict__ tile_pre,
                    const int2* __restrict__ tile_own, const unsigned* __restrict__ any_list,
@@ -1241,7 +1241,7 @@ topk_finalize_staged_kernel(const DevLayer* __restrict__ layers, const Tile* __r
 // Persistent blocks take tiles by ticket (one atomic per tile, requested two tiles ahead), and the ranges of a
 // block's next tile are fetched while the current one is worked on.
 // SGD: the optimiser tail is applied to every element of out where it is written.
-constexpr int kDecStage = kTile;  // staged entries per round (a worker has at most kTile entries in a tile)
+constexpr int kDecStage = kTile / 2;  // staged entries per round
 constexpr size_t kDecSmemBytes = sizeof(float) * kTile + (sizeof(int) + sizeof(float)) * kDecStage +
                                  sizeof(int) * 2 * kMaxWorkers + 16;
 
@@ -1252,7 +1252,7 @@ __device__ __forceinline__ void cp_async4(void* dst_smem, const void* src) {
 __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
 
 template <bool SGD>
-__global__ void __launch_bounds__(256, 2)
+__global__ void __launch_bounds__(256, 3)
 topk_decompress_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict__ tiles, int n_tiles,
                        const float* __restrict__ grads, const int2* __restrict__ tile_rng,
                        const float* __restrict__ vals, const int32_t* __restrict__ idx, float* __restrict__ out,
@@ -1314,34 +1314,37 @@ topk_decompress_kernel(const DevLayer* __restrict__ layers, const Tile* __restri
       for (int i = threadIdx.x; i < kTile / 4; i += blockDim.x)
         reinterpret_cast<float4*>(acc)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
       __syncthreads();  // the ranges are in place (and acc is clear)
-      for (int w0 = 0; w0 < W;) {
-        // the workers [w0, w1) whose entries in this tile fit the staging area together (at least one)
-        int w1 = w0, total = 0;
-        while (w1 < W && total + (r_hi[w1] - r_lo[w1]) <= kDecStage) { total += r_hi[w1] - r_lo[w1]; ++w1; }
-        if (w1 == w0) break;  // (cannot happen: a worker has at most kTile entries in a tile)
-        int o = 0;
-        for (int w = w0; w < w1; ++w) {
+      // rounds: the staging area is filled with the entries of as many workers as fit, in worker order (a worker
+      // with more entries in the tile than the area holds is cut into pieces that take a round each)
+      int w0 = 0, off0 = 0;  // first worker of the round and how many of its entries earlier rounds have taken
+      while (w0 < W) {
+        int w = w0, off = off0, o = 0;
+        while (w < W && o < kDecStage) {
+          const int lo = r_lo[w] + off, n = min(r_hi[w] - lo, kDecStage - o);
           const long long seg = (long long)w * capacity + l_seg_off;
-          const int lo = r_lo[w], n = r_hi[w] - lo;
           for (int i = threadIdx.x; i < n; i += 256) {
             cp_async4(s_idx + o + i, idx + seg + lo + i);
             cp_async4(s_val + o + i, vals + seg + lo + i);
           }
           o += n;
+          if (lo + n == r_hi[w]) { ++w; off = 0; } else { off += n; }
         }
         cp_async_wait_all();
         __syncthreads();
+        int w2 = w0, off2 = off0;
         o = 0;
-        for (int w = w0; w < w1; ++w) {
-          const int n = r_hi[w] - r_lo[w];
+        while (w2 < W && o < kDecStage) {
+          const int lo = r_lo[w2] + off2, n = min(r_hi[w2] - lo, kDecStage - o);
           for (int i = threadIdx.x; i < n; i += 256) {
             const unsigned li = (unsigned)(s_idx[o + i] - elem0);
             if (li < (unsigned)kTile) acc[li] += s_val[o + i];
           }
           o += n;
-          __syncthreads();  // the next worker may add to the same elements; the last one frees the staging area
+          if (lo + n == r_hi[w2]) { ++w2; off2 = 0; } else { off2 += n; }
+          __syncthreads();  // the next worker may add to the same elements; the last piece frees the staging area
         }
-        w0 = w1;
+        w0 = w;
+        off0 = off;
       }
       const int n4 = nelem >> 2;
       for (int i = threadIdx.x; i < n4; i += blockDim.x) {
@@ -1582,7 +1585,7 @@ cudaError_t launch_topk(acc_ctx* ctx, const float* grads, float* err, const uint
     PhaseTimer pt(ctx, PH_TOPK_DECOMPRESS, s);
     // persistent blocks (two fit an SM), tiles handed out by ticket; the ticket word was cleared with the
     // histograms at the start of the step
-    const int dgrid = std::min(nt, ctx->sm_count * 2);
+    const int dgrid = std::min(nt, ctx->sm_count * 3);
     unsigned* ticket = ctx->d_any_list + kTicketWord;
     if (tail.params)
       topk_decompress_kernel<true><<<dgrid, 256, kDecSmemBytes, s>>>(ctx->d_layers, ctx->d_tiles, nt, grads, ctx->d_tile_rng, vals,

@@ -43,9 +43,13 @@ def test_static_norm_matches_layer_norms_twice_in_a_row():
 def test_static_norm_rejects_bad_sizes_without_launching():
     x = torch.ones(64, device="cuda")
     o = torch.zeros(1, dtype=torch.float64, device="cuda")
+    with pytest.raises(ValueError):
+        binding.acc_sumsq_static(x, (1 << 28) + 1, o)   # more elements than the tensor holds: refused by the binding
+    big = torch.empty((1 << 28) + 1, device="cuda")     # 1 GiB + 4 bytes, never read
     with pytest.raises(binding.AccError) as ei:
-        binding.acc_sumsq_static(x, (1 << 28) + 1, o)   # beyond the built-in scratch: refused, nothing read
+        binding.acc_sumsq_static(big, big.numel(), o)   # beyond the built-in scratch: refused, nothing launched
     assert ei.value.status == 5 and "capacity" in str(ei.value)
+    del big
     with pytest.raises(binding.AccError):
         binding.acc_sumsq_static(x, 0, o)
     with pytest.raises(binding.AccError):
