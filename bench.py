@@ -439,11 +439,14 @@ def main():
     dom_alg_delta = _kernel_alg_bytes(dom, units, W, carries)  # ... and with the detector's accumulation counted
     dom_avg_ms = prof[dom][0] / prof[dom][1]
     achieved = dom_alg / (dom_avg_ms * 1e-3) / 1e9
+    tkey = traffic_key(dom, args, table, W, torch.cuda.get_device_properties(dev).multi_processor_count)
     roofline = {"bound": "hbm", "kernel": dom, "achieved": round(achieved, 1), "peak": peak, "unit": "GB/s",
                 "frac": round(achieved / peak, 4), "peak_source": peak_src,
                 "peak_nominal": NOMINAL_HBM_GBS, "frac_of_nominal": round(achieved / NOMINAL_HBM_GBS, 4),
-                "traffic": (TRAFFIC_PER_UNIT[dom] * units if dom in TRAFFIC_PER_UNIT else None),
-                "traffic_source": TRAFFIC_SOURCE.get(dom),
+                "traffic": (TRAFFIC_PER_UNIT[tkey] * units if tkey in TRAFFIC_PER_UNIT else None),
+                "traffic_source": TRAFFIC_SOURCE.get(tkey),
+                "traffic_over_algorithmic": (round(TRAFFIC_PER_UNIT[tkey] * units / dom_alg, 3)
+                                             if tkey in TRAFFIC_PER_UNIT and dom_alg else None),
                 "alg_bytes_per_launch": dom_alg, "alg_bytes_per_unit": round(dom_alg / units, 3),
                 "frac_with_detector_bytes": round(dom_alg_delta / (dom_avg_ms * 1e-3) / 1e9 / peak, 4),
                 "step_frac_of_12B": step_fracs(ms_per_step)["of_measured_copy_peak"],
@@ -763,9 +766,22 @@ def run_real_workers(args, w, ring, dev, rank, world, local_rank):
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per MATRIX parameter-worker, from the ncu captures
 # summarised under profiles/; a launch's traffic is this figure times the units it processes (the kernels
 # stream every element once, so traffic grows in proportion).
-TRAFFIC_PER_UNIT = {"psgd_project_kernel": 13.15, "topk_ef_hist1_kernel": 12.92}
+TRAFFIC_PER_UNIT = {"psgd_project_kernel": 13.15, "psgd_project_kernel/pipelined": 13.21, "topk_ef_hist1_kernel": 12.95}
 TRAFFIC_SOURCE = {"psgd_project_kernel": "ncu capture of the direct kernel on config 4, scaled by units",
+                  "psgd_project_kernel/pipelined": "ncu capture of the pipelined kernel on config 4, scaled by units",
                   "topk_ef_hist1_kernel": "ncu capture on config 3, scaled by units"}
+PIPE_MIN_STAGES_PER_SM = 200  # the library's rule for choosing the pipelined first PowerSGD pass (acc_powersgd.cu)
+
+
+def traffic_key(kernel, args, table, n_workers, sm_count):
+    """The traffic figure that belongs to the implementation of the first PowerSGD pass this run used."""
+    if kernel != "psgd_project_kernel":
+        return kernel
+    from paper_2010_16248_b200 import workloads as wl
+    tiles = sum(-(-int(table.sizes[l]) // 8192) for l in range(table.n_layers) if table.kind[l] == wl.MATRIX)
+    pipelined = args.pipeline == "always" or (args.pipeline == "auto" and
+                                              tiles * n_workers // max(sm_count, 1) >= PIPE_MIN_STAGES_PER_SM)
+    return kernel + "/pipelined" if pipelined else kernel
 
 if __name__ == "__main__":
     main()

@@ -1470,7 +1470,9 @@ static cudaError_t launch_topk_select_part(acc_ctx* ctx, const float* grads, flo
     for (int l : pl.mat_layers) max_cap = std::max(max_cap, pl.layers[l].cand_cap);
     const int list_chunks = std::min(128, std::max(8, max_cap / 16384));
     const long long V = (long long)W * nt;
-    const int grid = (int)(V < (long long)ctx->sm_count * 8 ? V : (long long)ctx->sm_count * 8);
+    // grids of the passes that usually find an empty work list: the blocks resident at once and no more (an idle
+    // block costs about 5 ns: 1776 of them were 10 us of an otherwise empty launch)
+    const int grid = (int)(V < (long long)ctx->sm_count * 4 ? V : (long long)ctx->sm_count * 4);
     // first pass: a whole number of waves of resident blocks (a grid that is not a multiple of what fits leaves the
     // last wave of the static split short: 8 blocks per SM with 3 resident cost 4 %), two to six of them (finer
     // shares even out the deciding worker's tiles, which also carry the detector's accumulator)
@@ -1493,7 +1495,7 @@ static cudaError_t launch_topk_select_part(acc_ctx* ctx, const float* grads, flo
     }
     {
       PhaseTimer pt(ctx, PH_TOPK_COLLECT, s);
-      const long long cap = (long long)ctx->sm_count * 12;
+      const long long cap = (long long)ctx->sm_count * 3;
       topk_collect_kernel<<<(unsigned)(V < cap ? V : cap), 256, 0, s>>>(
           ctx->d_layers, ctx->d_tiles, nt, n_mat, W, err, c.worker_stride, ctx->d_sel, ctx->d_any_list,
           ctx->d_seg_cand, ctx->d_cand, ctx->d_tile_cand, pl.cand_total, ctx->d_tile_cnt, ctx->d_lists);
@@ -1559,8 +1561,14 @@ static cudaError_t launch_topk_select_part(acc_ctx* ctx, const float* grads, flo
             ctx->d_tile_cand, pl.cand_total, vals, idx, c.worker_stride, pl.capacity, ctx->d_any_list, ctx->d_lists);
     }
     PhaseTimer pt(ctx, PH_TOPK_SELECT, s);
-    const long long blocks = (long long)W * nt, cap = (long long)ctx->sm_count * 12;
-    const unsigned sgrid = (unsigned)std::min(blocks, cap);
+    // contiguous shares of the select work list.  Large sets: shares of about four tiles, fine enough that a run of
+    // expensive tiles (the fully kept head of a zero-filled layer) spreads over many blocks (config 5 at K = 10 %:
+    // 0.68 ms with 592 blocks, 0.51 ms with 1776, 0.46 ms with 4736).  Small sets: the blocks resident at once,
+    // so that a launch which finds an empty list stays cheap (an idle block costs about 5 ns).
+    const long long blocks = (long long)W * nt;
+    const long long sm = ctx->sm_count;
+    const long long want = blocks >= sm * 128 ? std::min(blocks / 4, sm * 64) : sm * 4;
+    const unsigned sgrid = (unsigned)std::min(blocks, want);
     if (lazy)
       topk_select_kernel<true><<<sgrid, 256, 0, s>>>(ctx->d_layers, ctx->d_tiles, nt, n_mat, err, ctx->d_sel,
                                                      ctx->d_tile_pre, ctx->d_tile_cnt, ctx->d_any_list, vals, idx,

@@ -94,6 +94,35 @@ def test_bench_reference_arm_prints_the_contract_line():
     assert line["e2e"]["h2d_bytes_per_step"] == 0 and line["e2e"]["d2h_bytes_per_step"] == 0
 
 
+def test_bench_gpus_argument_reaches_both_arms(monkeypatch):
+    """`--gpus N`: the reference arm (the oracle on the host) echoes N and prints one line whatever N is; the GPU
+    arm, started without a launcher, re-executes itself under torch.distributed.run with N ranks on 127.0.0.1 and
+    the same arguments."""
+    import importlib
+    import json
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    res = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--impl", "reference", "--gpus", "2",
+                          "--config", "1", "--steps", "1", "--warmup", "0"], capture_output=True, text=True,
+                         timeout=600)
+    assert res.returncode == 0, res.stderr[-2000:]
+    lines = [l for l in res.stdout.strip().splitlines() if l.startswith("{")]
+    assert len(lines) == 1 and json.loads(lines[0])["n_gpus"] == 2
+    cpu = json.loads(lines[0])["cpu_baseline"]
+    assert cpu["value_single_thread"] > 0 and "stream" in cpu["sample"] and cpu["cores"] >= 1
+    sys.path.insert(0, root)
+    bench = importlib.import_module("bench")
+    seen = {}
+    monkeypatch.setattr(bench.subprocess, "call", lambda cmd: seen.setdefault("cmd", cmd) and 0)
+    monkeypatch.setattr(sys, "argv", ["bench.py", "--gpus", "2", "--steps", "7"])
+    assert bench.respawn_under_torchrun(2) == 0
+    cmd = seen["cmd"]
+    assert cmd[1:3] == ["-m", "torch.distributed.run"] and "--nproc-per-node=2" in cmd and "--nnodes=1" in cmd
+    assert cmd[cmd.index("--master-addr") + 1] == "127.0.0.1" and int(cmd[cmd.index("--master-port") + 1]) > 0
+    assert cmd[-4:] == ["--gpus", "2", "--steps", "7"] and cmd[-5].endswith("bench.py")
+
+
 def _hostless_context(table, W):
     """A binding.Context with the layout fields filled in by hand and no library handle: the argument checks run
     (and must raise) before any call into the library, so they can be tested without a GPU."""
