@@ -269,6 +269,9 @@ def main():
                     help="every GPU holds the config's W workers and the compressed factors are exchanged between "
                          "GPUs (all-reduce of P and Q, all-gather of the packed TopK sets) instead of independent "
                          "replicas; at --gpus 1 the collectives are the identity")
+    ap.add_argument("--groups", type=int, default=1,
+                    help="--real-workers: layer groups whose exchanges run on a communication stream beside the next "
+                         "group's first pass")
     ap.add_argument("--n-accum", type=int, default=8, help="--batch-mode: micro-batches per step (B_high / micro-batch)")
     ap.add_argument("--force-level", default="auto", choices=["auto", "low", "high"],
                     help="auto: the detector sets the per-layer levels (the method as it runs); low / high: every "
@@ -656,7 +659,8 @@ def run_real_workers(args, w, ring, dev, rank, world, local_rank):
     from paper_2010_16248_b200 import dist_util, pipeline
     table, W = w.table, w.n_workers
     engines = [pipeline.DistributedStep(table, W, comp, w.rank_low, w.rank_high, w.topk_low_bp, w.topk_high_bp, w.eta,
-                                        1e-8, w.check_every, device=dev, lazy_residual=not args.eager)
+                                        1e-8, w.check_every, device=dev, lazy_residual=not args.eager,
+                                        groups=args.groups)
                for comp in w.compressors]
     n_comp = len(engines)
     grad_bytes_step = n_comp * 4.0 * W * table.n_params
@@ -695,17 +699,18 @@ def run_real_workers(args, w, ring, dev, rank, world, local_rank):
     ms_per_step = dist_util.max_over_ranks(start.elapsed_time(stop), dev) / K
     value = dist_util.whole_job_throughput(grad_bytes_step, ms_per_step, world) / 1e9
 
-    for e in engines:
-        e.ctx.acc_profile_enable(True)
+    contexts = list({id(c): c for e in engines for c in [p.ctx for p in e.parts] + [e.ctx]}.values())
+    for c in contexts:
+        c.acc_profile_enable(True)
     for _ in range(K):
         one_step(ring[step_no % RING])
     torch.cuda.synchronize()
     prof = {}
-    for e in engines:
-        for name, (ms, cnt) in e.ctx.acc_profile_read().items():
+    for c in contexts:
+        for name, (ms, cnt) in c.acc_profile_read().items():
             a = prof.get(name, (0.0, 0))
             prof[name] = (a[0] + ms, a[1] + cnt)
-        e.ctx.acc_profile_enable(False)
+        c.acc_profile_enable(False)
     gpu_launches = sum(cnt for _, cnt in prof.values())  # the profiled pass repeats the timed pass launch for launch
     peak, peak_src = _peaks()
     units = W * table.n_matrix_params
@@ -754,6 +759,7 @@ def run_real_workers(args, w, ring, dev, rank, world, local_rank):
                            "exchange_bytes_per_step_per_gpu": sum(e.bytes_exchanged_per_step() for e in engines),
                            "l2_policy": f"inputs larger than L2: {RING} gradient batches cycled, no flush",
                            "launch": "direct calls (collectives between the phases)",
+                           "layer_groups": args.groups,
                            "multi_gpu": "NCCL all-reduce of the PowerSGD factors, all-gather of the packed TopK sets"},
                 "clocks": clocks, "e2e": e2e, "gpu_launches": gpu_launches, "roofline": roofline,
                 "cpu_baseline": None, "kernels": kernels}

@@ -14,7 +14,8 @@
  *   * Pointers named in "Device pointers" below are DEVICE pointers owned by the caller; the library
  *     never allocates or frees device memory.  `cfg`, `layers`, and every `int64_t*` / `size_t*`
  *     out-parameter are HOST pointers.
- *   * Every device buffer must be 16-byte aligned (ACC_EALIGN otherwise).
+ *   * Every device buffer of floats or indices must be 16-byte aligned (ACC_EALIGN otherwise); arrays of doubles
+ *     need 8 bytes, level arrays (bytes) no alignment at all.
  *   * Calls are asynchronous on `stream` (a cudaStream_t passed as void*; NULL = default stream),
  *     never synchronise the device, and return an int status: ACC_OK or one of the ACC_E* codes.
  *     Calls on one context must be ordered on one stream (or otherwise serialised by the caller):

@@ -284,8 +284,9 @@ class _Part:
         dev, n_local, world = owner.device, owner.n_local, owner.world
         self.table = owner.table if len(self.ids) == owner.table.n_layers else _sub_table(owner.table, self.ids)
         self.ctx = c = binding.Context(self.table, n_local, device=dev, **owner._cfg)
-        self.ids_dev = torch.tensor(self.ids, dtype=torch.long, device=dev)
-        self.level = torch.ones(len(self.ids), dtype=torch.uint8, device=dev)
+        # the group's layers are a contiguous run, so its levels are a slice of the step's level array: what the
+        # regime test writes there is what the group's kernels read
+        self.level = owner.level[self.ids[0]:self.ids[-1] + 1]
         if owner.compressor == "powersgd":
             ql = None if q_init is None else [q_init[l] for l in self.ids]
             self.q = c.new_q(ql if ql is not None else wl.initial_q(self.table, owner._cfg["rank_low"], device=dev))
@@ -358,7 +359,6 @@ class DistributedStep:
                          "counts_all"):
                 if hasattr(one, name):
                     setattr(self, name, getattr(one, name))
-            one.level = self.level
 
     def flush(self, stream=None):
         """Lazy mode: materialises this rank's error memories (see ``AccordionStep.flush``)."""
@@ -432,9 +432,6 @@ class DistributedStep:
                 x.sum_(self.norm2_curr)  # a broadcast from the deciding rank (Section 3: one node decides for all)
                 self.ctx.acc_detect_regime(self.norm2_curr, self.norm2_prev, lr_curr, lr_next, self.level, self.delta,
                                            main)
-                if len(self.parts) > 1:
-                    for p in self.parts:
-                        torch.index_select(self.level, 0, p.ids_dev, out=p.level)
         return self.out
 
 
