@@ -4,8 +4,11 @@
 // (12 + 12 + 7 bits, shared-memory histograms), followed by an ordered compaction:
 //   ef_hist1   M = g + e -> err, level-1 histogram per (worker, layer)                [reads g, e; writes M]
 //              (+ keys of the buckets around the predicted threshold bucket -> candidate list)
-//   pick1      bucket b1 holding the k-th largest key; predicted-list path if pass A's prediction held,
-//              else list path if the keys of b1 fit the candidate list, else dense path
+//              (+ per-tile counts of non-zero keys)
+//   pick1      bucket b1 holding the k-th largest key; zero fill if the threshold falls among exact zeros (every
+//              non-zero kept, the zeros of lowest index fill up: settled from the non-zero counts, levels 2-3 skipped);
+//              predicted-list / staged path if pass A's prediction held, else list path if the keys of b1 fit the
+//              candidate list, else dense path
 //   collect    (list path) keys of bucket b1 -> per-tile ranges of the segment's candidate list,
 //              per-tile count of keys above b1                                                  [reads M]
 //   hist2      level-2 histogram of the keys inside b1 (dense path: reads M and also counts the keys
@@ -14,12 +17,14 @@
 //   hist3      level-3 histogram of the keys with prefix (b1,b2) (dense path: reads M, keeps it per tile
 //              together with the per-tile count above; list path: per segment from the collected keys)
 //   pick3      threshold tau and the number of ties to keep
-//   tilecounts per tile (keys above tau, keys equal to tau), from the tile's level-3 histogram (dense) or from
-//              its collected keys (list);  tilescan: their exclusive prefix per layer
+//   tilecounts per tile (keys above tau, keys equal to tau), from the tile's level-3 histogram (dense), its collected
+//              keys (list) or its non-zero count (zero fill);  tilescan: their exclusive prefix per layer, every
+//              tile's range inside the packed segment, and the work lists of select / finalize
 //   select     keep key > tau and the lowest-index `need` of key == tau; write (val, idx) in index
 //              order, zero the kept entries of err                                              [reads M]
 //   finalize   the same for segments whose pass A staged whole entries: from the list, M is not read
-//   decompress out = (1/W) sum_w scatter(idx_w, val_w), accumulated per tile in shared memory [reads packed]
+//   decompress out = (1/W) sum_w scatter(idx_w, val_w), accumulated per tile in shared memory from the workers'
+//              entries staged there by asynchronous copies                                      [reads packed]
 // No floating-point atomics and no inter-block waiting: same input, same bits.
 #include <algorithm>
 
