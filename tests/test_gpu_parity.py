@@ -770,6 +770,25 @@ def test_many_workers():
         assert torch.allclose(delta[sl], want[sl], rtol=1e-6, atol=1e-7), l
 
 
+def test_topk_three_hundred_workers():
+    """W = 300: more workers than the decompress pass has threads in a block (it keeps a tile's ranges for up to
+    four workers per thread) and than its staging area holds at once at K = 50 % (several rounds per tile)."""
+    table = wl.make_table([("w", (40, 300)), ("b", (5,)), ("tall", (2100, 4))])
+    W = 300
+    ctx = binding.Context(table, W, topk_low_bp=5000, topk_high_bp=100, decider=299)
+    vals, idx, counts = ctx.new_topk_buffers()
+    out = torch.zeros(table.stride, device="cuda")
+    _, err = _random_inputs(table, W, 4100)
+    for it, lv in enumerate(([1, 0, 0], [0, 0, 1])):
+        level = torch.tensor(lv, dtype=torch.uint8, device="cuda")
+        grads, _ = _random_inputs(table, W, 4110 + it)
+        e0 = err.clone()
+        ctx.acc_topk_step(grads, err, level, vals, idx, counts, out, None)
+        torch.cuda.synchronize()
+        H.check_topk_against_oracle(ctx, table, grads, e0, level, vals, idx, counts, out, err, 5000, 100)
+    assert ctx.acc_device_status() == 0
+
+
 def test_bounded_wait_reports_timeout_and_context_stays_usable():
     """Failure detection without a fault: a kernel waits, with a short poll limit, on a barrier nothing arrives at;
     the wait gives up, the status word reads ACC_ETIMEOUT, the kernel has returned normally and later calls on the
