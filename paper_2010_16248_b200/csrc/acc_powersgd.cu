@@ -58,38 +58,162 @@ __device__ void vector_mean_tile(const Tile& t, const DevLayer& L, const float* 
                    [&](int i, float4 v) { *reinterpret_cast<float4*>(o + i) = v; }, [&](int i, float v) { o[i] = v; });
 }
 
-// Pass 1.  One block per tile, all workers:
-//   e_w = err_w                                 (eager: err holds the error memory)
-//   e_w = err_w - P^_prev Q^T  (first rp ranks) (lazy: err holds last step's M_w, residual still pending)
-//   M_w = g_w + e_w -> err;  Mbar = mean_w M_w -> out and shared memory;  delta += g_decider;
-// then, for every row the tile cuts, the partial dot products Mbar[row, cols in tile] . Q go to the row's
-// slot for this tile in p_part (a row touches (m-1)/8192 + 2 tiles at most; the orthonormalise pass adds
-// the slots in order).
-template <int WB, bool LAZY>
-__global__ void __launch_bounds__(256, 3)
-psgd_project_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict__ tiles,
-                    const float* __restrict__ grads, float* __restrict__ err, const float* __restrict__ q,
-                    const float* __restrict__ p, float4* __restrict__ p_part, const uint8_t* __restrict__ level,
-                    const int* __restrict__ pending, float* __restrict__ out, float* __restrict__ delta,
-                    long long stride, int W, int decider, float inv_w) {
-  __shared__ __align__(16) float s_mbar[kTile];
-  const Tile t = tiles[blockIdx.x];
-  const DevLayer L = layers[t.layer];
-  if (L.kind != ACC_MATRIX) {
-    vector_mean_tile(t, L, grads, out, delta, stride, W, decider, inv_w);
-    return;
-  }
-  const int rp = LAZY ? pending[t.layer] : 0;
+// Partial rows of P from a tile's mean matrix in shared memory: for every row the tile cuts, the dot products of
+// Mbar[row, columns inside the tile] with the columns of Q go to the row's slot for this tile in p_part.  Both
+// first-pass kernels end a tile with it (NWARPS warps, all threads of the block; s_mbar complete and visible),
+// so they give the same bits.  s_pp: 2 * kTile / kSpan float4 of shared memory.
+constexpr int kSpan = 512;
+constexpr int kSpans = kTile / kSpan;
+template <int NWARPS>
+__device__ __forceinline__ void tile_p_partials(const float* s_mbar, float4* s_pp, const Tile& t, const DevLayer& L,
+                                                const float4* __restrict__ Q4, float4* __restrict__ p_part) {
   const int m = L.cols;
-  const float4* __restrict__ Q4 = reinterpret_cast<const float4*>(q) + L.q_row;
-  const float4* __restrict__ P4 = reinterpret_cast<const float4*>(p) + L.p_row;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int first_row = t.elem0 / m, last_row = (t.elem0 + t.nelem - 1) / m;
+  const int tile_in_layer = t.elem0 / kTile;
+  if (m >= 2 * kSpan) {
+    // long rows (too few row pieces to occupy the warps): the tile is cut into 512-element spans, a warp reduces
+    // a span at a time (a span meets at most two rows); the spans of a row are then added in span order
+    for (int sp = warp; sp < kSpans; sp += NWARPS) {
+      const int s0 = sp * kSpan, s1 = min(s0 + kSpan, t.nelem);
+      const int r_lo = (t.elem0 + s0) / m;
+#pragma unroll
+      for (int j = 0; j < 2; ++j) {
+        const int row_begin = (r_lo + j) * m;
+        const int lo = max(row_begin - t.elem0, s0), hi = min(row_begin + m - t.elem0, s1);
+        float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+        for (int i = lo + lane; i < hi; i += 32) {
+          const float v = s_mbar[i];
+          const float4 qv = __ldg(Q4 + (t.elem0 + i - row_begin));
+          a0 = fmaf(v, qv.x, a0); a1 = fmaf(v, qv.y, a1); a2 = fmaf(v, qv.z, a2); a3 = fmaf(v, qv.w, a3);
+        }
+        a0 = warp_sum(a0); a1 = warp_sum(a1); a2 = warp_sum(a2); a3 = warp_sum(a3);
+        if (lane == 0) s_pp[2 * sp + j] = make_float4(a0, a1, a2, a3);
+      }
+    }
+    __syncthreads();
+    const int row = first_row + (int)threadIdx.x;
+    if (row <= last_row) {
+      const int row_begin = row * m;
+      const int lo = max(row_begin, t.elem0) - t.elem0, hi = min(row_begin + m, t.elem0 + t.nelem) - t.elem0;
+      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+      for (int sp = lo / kSpan; sp <= (hi - 1) / kSpan; ++sp) {
+        const float4 v = s_pp[2 * sp + (row - (t.elem0 + sp * kSpan) / m)];
+        acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+      }
+      p_part[L.ppart_base + (long long)row * L.nslots + (tile_in_layer - row_begin / kTile)] = acc;
+    }
+  } else {
+    // short rows: one warp per row piece
+    for (int row = first_row + warp; row <= last_row; row += NWARPS) {
+      const int row_begin = row * m;
+      const int lo = max(row_begin, t.elem0) - t.elem0, hi = min(row_begin + m, t.elem0 + t.nelem) - t.elem0;
+      const float4* qr = Q4 + (t.elem0 + lo - row_begin);
+      float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+      for (int i = lo + lane; i < hi; i += 32) {
+        const float v = s_mbar[i];
+        const float4 qv = __ldg(qr + (i - lo));
+        a0 = fmaf(v, qv.x, a0); a1 = fmaf(v, qv.y, a1); a2 = fmaf(v, qv.z, a2); a3 = fmaf(v, qv.w, a3);
+      }
+      a0 = warp_sum(a0); a1 = warp_sum(a1); a2 = warp_sum(a2); a3 = warp_sum(a3);
+      if (lane == 0)
+        p_part[L.ppart_base + (long long)row * L.nslots + (tile_in_layer - row_begin / kTile)] =
+            make_float4(a0, a1, a2, a3);
+    }
+  }
+}
+
+constexpr int kProjThreads = 256;
+
+// The same for a tile whose shared memory holds, per group of four consecutive elements, the group's dot products
+// with its four rows of Q (rows whose length is a multiple of four: a group never meets two rows).  Only adds are
+// left: a quarter of the shared-memory reads of the element version and no loads of Q.
+template <int NWARPS>
+__device__ __forceinline__ void tile_p_partials_grouped(const float4* s_grp, float4* s_pp, const Tile& t,
+                                                        const DevLayer& L, float4* __restrict__ p_part) {
+  const int m = L.cols;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int first_row = t.elem0 / m, last_row = (t.elem0 + t.nelem - 1) / m;
+  const int tile_in_layer = t.elem0 / kTile;
+  if (m >= 2 * kSpan) {
+    for (int sp = warp; sp < kSpans; sp += NWARPS) {
+      const int s0 = sp * kSpan, s1 = min(s0 + kSpan, t.nelem);
+      const int r_lo = (t.elem0 + s0) / m;
+#pragma unroll
+      for (int j = 0; j < 2; ++j) {
+        const int row_begin = (r_lo + j) * m;
+        const int lo = max(row_begin - t.elem0, s0), hi = min(row_begin + m - t.elem0, s1);
+        float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int i = (lo >> 2) + lane; i < (hi >> 2); i += 32) {
+          const float4 v = s_grp[i];
+          a.x += v.x; a.y += v.y; a.z += v.z; a.w += v.w;
+        }
+        a.x = warp_sum(a.x); a.y = warp_sum(a.y); a.z = warp_sum(a.z); a.w = warp_sum(a.w);
+        if (lane == 0) s_pp[2 * sp + j] = a;
+      }
+    }
+    __syncthreads();
+    const int row = first_row + (int)threadIdx.x;
+    if (row <= last_row) {
+      const int row_begin = row * m;
+      const int lo = max(row_begin, t.elem0) - t.elem0, hi = min(row_begin + m, t.elem0 + t.nelem) - t.elem0;
+      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+      for (int sp = lo / kSpan; sp <= (hi - 1) / kSpan; ++sp) {
+        const float4 v = s_pp[2 * sp + (row - (t.elem0 + sp * kSpan) / m)];
+        acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+      }
+      p_part[L.ppart_base + (long long)row * L.nslots + (tile_in_layer - row_begin / kTile)] = acc;
+    }
+  } else {
+    for (int row = first_row + warp; row <= last_row; row += NWARPS) {
+      const int row_begin = row * m;
+      const int lo = max(row_begin, t.elem0) - t.elem0, hi = min(row_begin + m, t.elem0 + t.nelem) - t.elem0;
+      float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+      for (int i = (lo >> 2) + lane; i < (hi >> 2); i += 32) {
+        const float4 v = s_grp[i];
+        a.x += v.x; a.y += v.y; a.z += v.z; a.w += v.w;
+      }
+      a.x = warp_sum(a.x); a.y = warp_sum(a.y); a.z = warp_sum(a.z); a.w = warp_sum(a.w);
+      if (lane == 0) p_part[L.ppart_base + (long long)row * L.nslots + (tile_in_layer - row_begin / kTile)] = a;
+    }
+  }
+}
+
+// The streaming part of pass 1 on one MATRIX tile (all threads of the block).  GROUPED (rows of a multiple of four
+// elements): the thread that holds four consecutive means multiplies them with their rows of Q at once and leaves
+// the four-rank sum in shared memory, and the pending residual comes from one row of P^ and the same rows of Q,
+// with no branch between the loads; otherwise the means themselves go to shared memory.
+template <int WB, bool LAZY, bool GROUPED>
+__device__ __forceinline__ void project_tile_stream(const Tile& t, const DevLayer& L, int rp,
+                                                    const float4* __restrict__ Q4, const float4* __restrict__ P4,
+                                                    const float* __restrict__ grads, float* __restrict__ err,
+                                                    float* __restrict__ out, float* __restrict__ delta,
+                                                    long long stride, int W, int decider, float inv_w,
+                                                    float* s_mbar) {
+  const int m = L.cols;
   const long long base = L.offset + t.elem0;
   const int n4 = t.nelem >> 2;
   for (int f = threadIdx.x; f < n4; f += blockDim.x) {
     const long long idx = base + 4 * f;
     float4 corr = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (LAZY && rp > 0) corr = lowrank4(P4, Q4, m, L.inv_cols, t.elem0 + 4 * f, rp);
+    int col = 0;
+    if (GROUPED) {
+      const int e_idx = t.elem0 + 4 * f, row = row_of(e_idx, m, L.inv_cols);
+      col = e_idx - row * m;
+      if (LAZY && rp > 0) {
+        const float4 pv = __ldg(P4 + row);
+        corr.x = lowrank_entry(pv, __ldg(Q4 + col), rp);
+        corr.y = lowrank_entry(pv, __ldg(Q4 + col + 1), rp);
+        corr.z = lowrank_entry(pv, __ldg(Q4 + col + 2), rp);
+        corr.w = lowrank_entry(pv, __ldg(Q4 + col + 3), rp);
+      }
+    } else if (LAZY && rp > 0) {
+      corr = lowrank4(P4, Q4, m, L.inv_cols, t.elem0 + 4 * f, rp);
+    }
     float4 mb = make_float4(0.f, 0.f, 0.f, 0.f);
+    // the detector's accumulator is asked for together with the first batch
+    float4 dv = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (delta != nullptr) dv = *reinterpret_cast<const float4*>(delta + idx);
     for (int w0 = 0; w0 < W; w0 += WB) {
       float4 gv[WB], ev[WB];
 #pragma unroll
@@ -108,16 +232,62 @@ psgd_project_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict_
           else *reinterpret_cast<float4*>(err + (long long)(w0 + b) * stride + idx) = mw;
           mb.x += mw.x; mb.y += mw.y; mb.z += mw.z; mb.w += mw.w;
           if (delta != nullptr && w0 + b == decider) {
-            float4 d = *reinterpret_cast<const float4*>(delta + idx);
-            d.x += gv[b].x; d.y += gv[b].y; d.z += gv[b].z; d.w += gv[b].w;
-            *reinterpret_cast<float4*>(delta + idx) = d;
+            dv.x += gv[b].x; dv.y += gv[b].y; dv.z += gv[b].z; dv.w += gv[b].w;
+            *reinterpret_cast<float4*>(delta + idx) = dv;
           }
         }
     }
     mb.x *= inv_w; mb.y *= inv_w; mb.z *= inv_w; mb.w *= inv_w;
     *reinterpret_cast<float4*>(out + idx) = mb;
-    *reinterpret_cast<float4*>(s_mbar + 4 * f) = mb;
+    if (GROUPED) {
+      const float4 q0 = __ldg(Q4 + col), q1 = __ldg(Q4 + col + 1), q2 = __ldg(Q4 + col + 2), q3 = __ldg(Q4 + col + 3);
+      float4 g;
+      g.x = fmaf(mb.w, q3.x, fmaf(mb.z, q2.x, fmaf(mb.y, q1.x, mb.x * q0.x)));
+      g.y = fmaf(mb.w, q3.y, fmaf(mb.z, q2.y, fmaf(mb.y, q1.y, mb.x * q0.y)));
+      g.z = fmaf(mb.w, q3.z, fmaf(mb.z, q2.z, fmaf(mb.y, q1.z, mb.x * q0.z)));
+      g.w = fmaf(mb.w, q3.w, fmaf(mb.z, q2.w, fmaf(mb.y, q1.w, mb.x * q0.w)));
+      *reinterpret_cast<float4*>(s_mbar + 4 * f) = g;
+    } else {
+      *reinterpret_cast<float4*>(s_mbar + 4 * f) = mb;
+    }
   }
+}
+
+// Pass 1.  One block per tile, all workers:
+//   e_w = err_w                                 (eager: err holds the error memory)
+//   e_w = err_w - P^_prev Q^T  (first rp ranks) (lazy: err holds last step's M_w, residual still pending)
+//   M_w = g_w + e_w -> err;  Mbar = mean_w M_w -> out and shared memory;  delta += g_decider;
+// then, for every row the tile cuts, the partial dot products Mbar[row, cols in tile] . Q go to the row's
+// slot for this tile in p_part (a row touches (m-1)/8192 + 2 tiles at most; the orthonormalise pass adds
+// the slots in order).
+template <int WB, bool LAZY>
+__global__ void __launch_bounds__(kProjThreads, 768 / kProjThreads)
+psgd_project_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict__ tiles,
+                    const float* __restrict__ grads, float* __restrict__ err, const float* __restrict__ q,
+                    const float* __restrict__ p, float4* __restrict__ p_part, const uint8_t* __restrict__ level,
+                    const int* __restrict__ pending, float* __restrict__ out, float* __restrict__ delta,
+                    long long stride, int W, int decider, float inv_w) {
+  __shared__ __align__(16) float s_mbar[kTile];
+  __shared__ float4 s_pp[2 * kSpans];
+  const Tile t = tiles[blockIdx.x];
+  const DevLayer L = layers[t.layer];
+  if (L.kind != ACC_MATRIX) {
+    vector_mean_tile(t, L, grads, out, delta, stride, W, decider, inv_w);
+    return;
+  }
+  const int rp = LAZY ? pending[t.layer] : 0;
+  const int m = L.cols;
+  const float4* __restrict__ Q4 = reinterpret_cast<const float4*>(q) + L.q_row;
+  const float4* __restrict__ P4 = reinterpret_cast<const float4*>(p) + L.p_row;
+  if ((m & 3) == 0) {
+    project_tile_stream<WB, LAZY, true>(t, L, rp, Q4, P4, grads, err, out, delta, stride, W, decider, inv_w, s_mbar);
+    __syncthreads();
+    tile_p_partials_grouped<kProjThreads / 32>(reinterpret_cast<const float4*>(s_mbar), s_pp, t, L, p_part);
+    return;
+  }
+  project_tile_stream<WB, LAZY, false>(t, L, rp, Q4, P4, grads, err, out, delta, stride, W, decider, inv_w, s_mbar);
+  const long long base = L.offset + t.elem0;
+  const int n4 = t.nelem >> 2;
   for (int i = 4 * n4 + threadIdx.x; i < t.nelem; i += blockDim.x) {  // last 1-3 elements of the layer
     const long long idx = base + i;
     const int e_idx = t.elem0 + i, row = e_idx / m, col = e_idx - row * m;
@@ -137,25 +307,7 @@ psgd_project_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict_
     s_mbar[i] = mb;
   }
   __syncthreads();
-  // partial rows of P from the tile in shared memory: one warp per row piece
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int first_row = t.elem0 / m, last_row = (t.elem0 + t.nelem - 1) / m;
-  const int tile_in_layer = t.elem0 / kTile;
-  for (int row = first_row + warp; row <= last_row; row += 8) {
-    const int row_begin = row * m;
-    const int lo = max(row_begin, t.elem0) - t.elem0, hi = min(row_begin + m, t.elem0 + t.nelem) - t.elem0;
-    const float4* qr = Q4 + (t.elem0 + lo - row_begin);
-    float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
-    for (int i = lo + lane; i < hi; i += 32) {
-      const float v = s_mbar[i];
-      const float4 qv = __ldg(qr + (i - lo));
-      a0 = fmaf(v, qv.x, a0); a1 = fmaf(v, qv.y, a1); a2 = fmaf(v, qv.z, a2); a3 = fmaf(v, qv.w, a3);
-    }
-    a0 = warp_sum(a0); a1 = warp_sum(a1); a2 = warp_sum(a2); a3 = warp_sum(a3);
-    if (lane == 0)
-      p_part[L.ppart_base + (long long)row * L.nslots + (tile_in_layer - row_begin / kTile)] =
-          make_float4(a0, a1, a2, a3);
-  }
+  tile_p_partials<kProjThreads / 32>(s_mbar, s_pp, t, L, Q4, p_part);
 }
 
 // Pass 1, pipelined.  Persistent blocks (one per SM, 512 threads), each with a contiguous range of MATRIX
@@ -321,60 +473,7 @@ psgd_project_pipe_kernel(const DevLayer* __restrict__ layers, const Tile* __rest
         }
       }
       __syncthreads();
-      const int m = L.cols;
-      const float4* Q4 = reinterpret_cast<const float4*>(q) + L.q_row;
-      const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-      const int first_row = t.elem0 / m, last_row = (t.elem0 + t.nelem - 1) / m;
-      const int tile_in_layer = t.elem0 / kTile;
-      constexpr int kSpan = kTile / kPipeWarps;  // 512 elements of the tile per warp
-      if (m >= 2 * kSpan) {
-        // long rows (too few row pieces to occupy the warps): every warp reduces its own 512-element span of
-        // the tile (it meets at most two rows); the spans of a row are then added in span order
-        const int s0 = warp * kSpan, s1 = min(s0 + kSpan, t.nelem);
-        const int r_lo = (t.elem0 + s0) / m;
-#pragma unroll
-        for (int j = 0; j < 2; ++j) {
-          const int row_begin = (r_lo + j) * m;
-          const int lo = max(row_begin - t.elem0, s0), hi = min(row_begin + m - t.elem0, s1);
-          float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
-          for (int i = lo + lane; i < hi; i += 32) {
-            const float v = s_mbar[i];
-            const float4 qv = __ldg(Q4 + (t.elem0 + i - row_begin));
-            a0 = fmaf(v, qv.x, a0); a1 = fmaf(v, qv.y, a1); a2 = fmaf(v, qv.z, a2); a3 = fmaf(v, qv.w, a3);
-          }
-          a0 = warp_sum(a0); a1 = warp_sum(a1); a2 = warp_sum(a2); a3 = warp_sum(a3);
-          if (lane == 0) s_pp[2 * warp + j] = make_float4(a0, a1, a2, a3);
-        }
-        __syncthreads();
-        const int row = first_row + (int)threadIdx.x;
-        if (row <= last_row) {
-          const int row_begin = row * m;
-          const int lo = max(row_begin, t.elem0) - t.elem0, hi = min(row_begin + m, t.elem0 + t.nelem) - t.elem0;
-          float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-          for (int sp = lo / kSpan; sp <= (hi - 1) / kSpan; ++sp) {
-            const float4 v = s_pp[2 * sp + (row - (t.elem0 + sp * kSpan) / m)];
-            acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
-          }
-          p_part[L.ppart_base + (long long)row * L.nslots + (tile_in_layer - row_begin / kTile)] = acc;
-        }
-      } else {
-        // short rows: one warp per row piece
-        for (int row = first_row + warp; row <= last_row; row += kPipeWarps) {
-          const int row_begin = row * m;
-          const int lo = max(row_begin, t.elem0) - t.elem0, hi = min(row_begin + m, t.elem0 + t.nelem) - t.elem0;
-          const float4* qr = Q4 + (t.elem0 + lo - row_begin);
-          float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
-          for (int i = lo + lane; i < hi; i += 32) {
-            const float v = s_mbar[i];
-            const float4 qv = __ldg(qr + (i - lo));
-            a0 = fmaf(v, qv.x, a0); a1 = fmaf(v, qv.y, a1); a2 = fmaf(v, qv.z, a2); a3 = fmaf(v, qv.w, a3);
-          }
-          a0 = warp_sum(a0); a1 = warp_sum(a1); a2 = warp_sum(a2); a3 = warp_sum(a3);
-          if (lane == 0)
-            p_part[L.ppart_base + (long long)row * L.nslots + (tile_in_layer - row_begin / kTile)] =
-                make_float4(a0, a1, a2, a3);
-        }
-      }
+      tile_p_partials<kPipeWarps>(s_mbar, s_pp, t, L, reinterpret_cast<const float4*>(q) + L.q_row, p_part);
     }
   }
 }
@@ -918,11 +1017,11 @@ static void launch_psgd_project(acc_ctx* ctx, const float* grads, float* err, fl
           ctx->d_ppart, nullptr, out, delta, c.worker_stride, c.n_workers, c.decider, inv_w, ctx->d_status);
     }
   } else if (lazy) {
-    psgd_project_kernel<4, true><<<nt, 256, 0, s>>>(ctx->d_layers, ctx->d_tiles, grads, err, q, p_hat, ctx->d_ppart,
+    psgd_project_kernel<4, true><<<nt, kProjThreads, 0, s>>>(ctx->d_layers, ctx->d_tiles, grads, err, q, p_hat, ctx->d_ppart,
                                                     level, ctx->d_pending, out, delta, c.worker_stride,
                                                     c.n_workers, c.decider, inv_w);
   } else {
-    psgd_project_kernel<4, false><<<nt, 256, 0, s>>>(ctx->d_layers, ctx->d_tiles, grads, err, q, p_hat,
+    psgd_project_kernel<4, false><<<nt, kProjThreads, 0, s>>>(ctx->d_layers, ctx->d_tiles, grads, err, q, p_hat,
                                                      ctx->d_ppart, level, nullptr, out, delta, c.worker_stride,
                                                      c.n_workers, c.decider, inv_w);
   }
