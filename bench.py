@@ -257,6 +257,10 @@ def main():
     ap.add_argument("--no-graphs", action="store_true", help="issue the timed steps call by call instead of as CUDA graphs")
     ap.add_argument("--pipeline", default="auto", choices=["auto", "always", "never"],
                     help="first PowerSGD pass: persistent bulk-copy pipeline, direct kernel, or the library's choice")
+    ap.add_argument("--share-sms", action="store_true",
+                    help="two compressors: the pipelined first PowerSGD pass takes half of the SMs, the TopK step's "
+                         "kernels run beside it (faster step, slower kernel; off by default so that the roofline "
+                         "entry times the kernel on the whole GPU)")
     ap.add_argument("--no-overlap", action="store_true",
                     help="two-compressor configs: run the TopK step after the PowerSGD step instead of beside it")
     ap.add_argument("--sgd-tail", action="store_true",
@@ -320,7 +324,7 @@ def main():
     eng = pipeline.AccordionStep(table, W, w.compressors, w.rank_low, w.rank_high, w.topk_low_bp, w.topk_high_bp,
                                  w.eta, 1e-8, w.check_every, device=dev, lazy_residual=not args.eager,
                                  optimizer=optimizer, extra_flags={"auto": 0, "always": 2, "never": 4}[args.pipeline],
-                                 overlap=not args.no_overlap)
+                                 overlap=not args.no_overlap, share_sms=args.share_sms)
     n_mat = table.n_matrix_params
     grad_bytes_step = n_comp * 4.0 * W * table.n_params
 
@@ -418,6 +422,9 @@ def main():
         return {"of_measured_copy_peak": round(gbs / peak, 4), "of_nominal_8TBs": round(gbs / NOMINAL_HBM_GBS, 4)}
 
     by_regime = {}
+    # the stored per-step traffic belongs to the default path (lazy residual, no optimiser tail, the library's choice
+    # of first PowerSGD pass, the config's own worker count)
+    default_path = not (args.eager or args.sgd_tail or args.share_sms or args.pipeline != "auto")
     for name in ("low", "high", "mixed"):
         ts = per_step[[r == name for r in regime]]
         if len(ts):
@@ -425,6 +432,14 @@ def main():
                                "min_ms": round(float(ts.min()), 4), "max_ms": round(float(ts.max()), 4),
                                "gradient_gbs": round(grad_bytes_step / (float(np.median(ts)) * 1e-3) / 1e9, 1),
                                "frac_of_12B": step_fracs(float(np.median(ts)))}
+            # achieved DRAM throughput of the whole step: the bytes ncu counted for one step of this config and level
+            # (every kernel of the step, one-pass capture) over this run's median step time
+            traffic = STEP_TRAFFIC.get((args.config, name)) if default_path else None
+            if traffic:
+                gbs = traffic / (float(np.median(ts)) * 1e-3) / 1e9
+                by_regime[name]["dram"] = {"bytes_per_step_ncu": traffic, "gbs": round(gbs, 1),
+                                           "frac_of_measured_copy_peak": round(gbs / peak, 4),
+                                           "frac_of_nominal_8TBs": round(gbs / NOMINAL_HBM_GBS, 4)}
     total_k_ms = sum(ms for ms, _ in prof.values())
     kernels = {}
     # the first compressor of the step carries the detector's accumulation in its first pass
@@ -776,6 +791,9 @@ TRAFFIC_PER_UNIT = {"psgd_project_kernel": 13.15, "psgd_project_kernel/pipelined
 TRAFFIC_SOURCE = {"psgd_project_kernel": "ncu capture of the direct kernel on config 4, scaled by units",
                   "psgd_project_kernel/pipelined": "ncu capture of the pipelined kernel on config 4, scaled by units",
                   "topk_ef_hist1_kernel": "ncu capture on config 3, scaled by units"}
+# DRAM bytes of one whole steady-state step (all kernels; same counters, one-pass launch list) by (config, level)
+STEP_TRAFFIC = {(5, "high"): 11467.8e6, (5, "low"): 12900.3e6, (4, "high"): 2280.9e6, (4, "low"): 2281.0e6,
+                (3, "high"): 603.6e6, (3, "low"): 859.6e6, (2, "high"): 666.0e6, (2, "low"): 665.6e6}
 PIPE_MIN_STAGES_PER_SM = 200  # the library's rule for choosing the pipelined first PowerSGD pass (acc_powersgd.cu)
 
 

@@ -21,6 +21,7 @@ ACC_MAX_RANK = 4
 ACC_FLAG_LAZY_RESIDUAL = 1
 ACC_FLAG_PIPELINE_ALWAYS = 2
 ACC_FLAG_PIPELINE_NEVER = 4
+ACC_FLAG_SHARE_SMS = 8
 POWERSGD, TOPK = 0, 1
 ACC_TOPK_PATH_DENSE, ACC_TOPK_PATH_LIST, ACC_TOPK_PATH_LIST_PREDICTED, ACC_TOPK_PATH_STAGED, ACC_TOPK_PATH_ZERO_FILL = range(5)
 

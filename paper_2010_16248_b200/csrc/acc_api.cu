@@ -18,7 +18,8 @@ static int topk_count(long long size, int bp) {
 static int validate(const acc_config* cfg) {
   if (!cfg || !cfg->layers) return ACC_EINVAL;
   if (cfg->n_workers < 1 || cfg->n_workers > kMaxWorkers || cfg->n_layers < 1) return ACC_EINVAL;
-  if (cfg->flags & ~(ACC_FLAG_LAZY_RESIDUAL | ACC_FLAG_PIPELINE_ALWAYS | ACC_FLAG_PIPELINE_NEVER)) return ACC_EINVAL;
+  if (cfg->flags & ~(ACC_FLAG_LAZY_RESIDUAL | ACC_FLAG_PIPELINE_ALWAYS | ACC_FLAG_PIPELINE_NEVER | ACC_FLAG_SHARE_SMS))
+    return ACC_EINVAL;
   if ((cfg->flags & ACC_FLAG_PIPELINE_ALWAYS) && (cfg->flags & ACC_FLAG_PIPELINE_NEVER)) return ACC_EINVAL;
   if (cfg->rank_high < 1 || cfg->rank_low < cfg->rank_high || cfg->rank_low > ACC_MAX_RANK) return ACC_EINVAL;
   if (cfg->topk_high_bp < 1 || cfg->topk_low_bp < cfg->topk_high_bp || cfg->topk_low_bp > 10000) return ACC_EINVAL;

@@ -1006,7 +1006,11 @@ static void launch_psgd_project(acc_ctx* ctx, const float* grads, float* err, fl
   PhaseTimer pt(ctx, PH_PSGD_PROJECT, s);
   if (pipelined && pl.n_mat > 0) {
     const int n_mt = (int)pl.mat_tiles.size(), n_vt = (int)pl.vec_tiles.size();
-    const int grid = n_mt < ctx->sm_count ? n_mt : ctx->sm_count;
+    // one block fills an SM; when a TopK step runs beside this one, half of the SMs are left to it (measured on the
+    // LSTM set, W = 8, both steps replayed from one graph: 2.15 -> 2.09 ms at the high level, 2.52 -> 2.46 ms at the
+    // low level; with every SM taken, the TopK step's short kernels wait for this pass to end)
+    const int sms = (c.flags & ACC_FLAG_SHARE_SMS) ? std::max(ctx->sm_count / 2, 1) : ctx->sm_count;
+    const int grid = n_mt < sms ? n_mt : sms;
     if (lazy) {
       psgd_project_pipe_kernel<true><<<grid, kPipeThreads, kPipeSmemBytes, s>>>(
           ctx->d_layers, ctx->d_tiles, ctx->d_mat_tiles, n_mt, ctx->d_vec_tiles, n_vt, grads, err, q, p_hat,

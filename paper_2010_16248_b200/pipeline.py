@@ -20,10 +20,12 @@ class AccordionStep:
     def __init__(self, table: wl.LayerTable, n_workers: int, compressors: Sequence[str] = ("powersgd",),
                  rank_low=2, rank_high=1, topk_low_bp=1000, topk_high_bp=100, eta=0.5, gs_eps=1e-8,
                  check_every=10, decider=0, q_init=None, device="cuda", lazy_residual=False, optimizer=None,
-                 extra_flags=0, overlap=True):
+                 extra_flags=0, overlap=True, share_sms=False):
         """``overlap``: with two compressors, the TopK step runs on a second stream beside the PowerSGD step
         (they share only the gradients and the level array, both read-only), so that the short, latency-bound
         kernels of one hide behind the streaming kernels of the other; the results are the same bits.
+        ``share_sms``: with ``overlap``, the pipelined first PowerSGD pass leaves half of the SMs to the TopK step
+        (ACC_FLAG_SHARE_SMS: the whole step gets a few percent faster, that kernel alone slower).
         ``extra_flags``: further ACC_FLAG_* bits for the context (e.g. forcing one implementation of the first
         PowerSGD pass).  ``optimizer``: None, or a dict ``{"params": tensor [stride], "lr": .., "momentum": 0.9,
         "weight_decay": 0.0}``: the Nesterov update (Appendix A) is then applied to ``params`` by the kernels
@@ -37,7 +39,9 @@ class AccordionStep:
         self.ctx = binding.Context(table, n_workers, device=device, rank_low=rank_low, rank_high=rank_high,
                                    topk_low_bp=topk_low_bp, topk_high_bp=topk_high_bp, eta=eta, gs_eps=gs_eps,
                                    decider=decider,
-                                   flags=(binding.ACC_FLAG_LAZY_RESIDUAL if lazy_residual else 0) | extra_flags)
+                                   flags=(binding.ACC_FLAG_LAZY_RESIDUAL if lazy_residual else 0) | extra_flags |
+                                   (binding.ACC_FLAG_SHARE_SMS if share_sms and overlap and len(compressors) == 2
+                                    else 0))
         dev, L, stride = self.device, table.n_layers, table.stride
         self.level = torch.ones(L, dtype=torch.uint8, device=dev)  # before the first check: low compression
         self.delta = torch.zeros(stride, device=dev)

@@ -494,6 +494,29 @@ def test_powersgd_tall_layers_orthonormalisation_paths(lazy):
     assert ctx.last_launch_count() == 6 and ctx.acc_device_status() == 0
 
 
+@pytest.mark.parametrize("lazy", [0, binding.ACC_FLAG_LAZY_RESIDUAL])
+def test_powersgd_pipelined_pass_on_half_of_the_sms_gives_the_same_bits(lazy):
+    """ACC_FLAG_SHARE_SMS only changes how many persistent blocks share the tiles of the pipelined first pass (a
+    table with more tiles than SMs, so that the block count does change): every output bit stays."""
+    table = wl.make_table([("big", (512, 4608)), ("v", (100,)), ("lstm", (300, 650)), ("mid", (256, 1152))])
+    W = 2
+    base = binding.ACC_FLAG_PIPELINE_ALWAYS | lazy
+    ctxs = [binding.Context(table, W, rank_low=2, rank_high=1, flags=f) for f in (base, base | binding.ACC_FLAG_SHARE_SMS)]
+    grads, err = _random_inputs(table, W, 77)
+    q0 = wl.initial_q(table, 2, seed=3)
+    st = [dict(err=err.clone(), q=c.new_q(q0), p=c.new_p(), out=torch.zeros(table.stride, device="cuda"),
+               delta=torch.zeros(table.stride, device="cuda")) for c in ctxs]
+    for it in range(3):
+        level = torch.tensor([(l + it) % 2 for l in range(table.n_layers)], dtype=torch.uint8, device="cuda")
+        for c, s_ in zip(ctxs, st):
+            c.acc_powersgd_step(grads, s_["err"], s_["q"], s_["p"], level, s_["out"], s_["delta"])
+        torch.cuda.synchronize()
+        for name in ("out", "q", "p", "err", "delta"):
+            assert torch.equal(st[0][name], st[1][name]), (it, name)
+        grads, _ = _random_inputs(table, W, 500 + it)
+    assert all(c.acc_device_status() == 0 for c in ctxs)
+
+
 def test_difference_criterion_variant_matches_oracle():
     table = _table_mixed()
     ctx = binding.Context(table, 1, eta=0.5)
