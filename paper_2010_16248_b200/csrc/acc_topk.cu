@@ -326,7 +326,7 @@ topk_pick1_kernel(const DevLayer* __restrict__ layers, const int* __restrict__ m
   __shared__ long long above;
   __shared__ int s_list;
   __shared__ unsigned s_base;
-  __shared__ unsigned long long s_nz;
+  __shared__ unsigned s_nz;
   const int seg = blockIdx.x, w = seg / n_mat, l = mat_layers[seg % n_mat];
   const DevLayer L = layers[l];
   const int lv = level[l] ? 1 : 0;
@@ -338,12 +338,16 @@ topk_pick1_kernel(const DevLayer* __restrict__ layers, const int* __restrict__ m
   // keys tell, the answer needs no further look at M: every non-zero is kept and the first k - nnz zeros, tau = 0.
   bool zero_fill = false;
   if (bin == 0) {
-    unsigned long long part = 0;
-    for (int i = threadIdx.x; i < L.ntiles; i += blockDim.x)
-      part += (unsigned long long)tile_cnt[(long long)w * n_tiles + L.tile0 + i].y;
-    if (part) atomicAdd(&s_nz, part);
+    // (a layer holds fewer than 2^31 elements, so 32 bits do; the loads of a thread are independent and go out
+    // together, the warps add their sums with one native shared-memory atomic each)
+    const int2* tc = tile_cnt + (long long)w * n_tiles + L.tile0;
+    unsigned part = 0;
+#pragma unroll 4
+    for (int i = threadIdx.x; i < L.ntiles; i += blockDim.x) part += (unsigned)__ldg(&tc[i].y);
+    part = __reduce_add_sync(0xffffffffu, part);
+    if ((threadIdx.x & 31) == 0 && part) atomicAdd(&s_nz, part);
     __syncthreads();
-    zero_fill = s_nz == (unsigned long long)above;  // no non-zero key below the second bucket
+    zero_fill = (long long)s_nz == above;  // no non-zero key below the second bucket
   }
   if (threadIdx.x == 0) {
     Select s;
