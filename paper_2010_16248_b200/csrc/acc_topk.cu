@@ -972,7 +972,7 @@ __device__ __forceinline__ void select_tile(const Tile& t, const unsigned tau, c
 // outlasts the tile) or none is (no tie in the tile, or the budget ran out before it) -- every tile of a segment but
 // the one where the budget runs out.  An entry is then kept iff its key >= thr (tau or tau + 1), one mask and one
 // scan instead of two, and the positions follow from the count of kept entries alone.
-template <bool FULL, bool LAZY, bool SPARSE>
+template <bool FULL, bool LAZY>
 __device__ __forceinline__ void select_tile_simple(const Tile& t, unsigned thr, unsigned tau, bool zero_ties,
                                                    int base, int k, float* __restrict__ m,
                                                    float* __restrict__ vals, int32_t* __restrict__ idx, long long seg,
@@ -1010,43 +1010,6 @@ __device__ __forceinline__ void select_tile_simple(const Tile& t, unsigned thr, 
   if (km == 0) return;
   int pos0 = base;
   for (int i = 0; i < wi; ++i) pos0 += (int)wtot[i];
-  if (SPARSE) {
-    // Few entries kept (the usual case: K of 1 % to 10 %): walk the set bits of the mask instead of all 32
-    // elements -- a warp runs as many rounds as its busiest lane has kept entries -- and read the kept values
-    // again (the lines were just loaded).  First position of this lane in each j: the warp's kept entries in the
-    // earlier j (16-bit sums) plus the lane's exclusive prefix inside j.
-    const unsigned e0x = i0 - c[0], e1x = i1 - c[1];  // exclusive prefixes over the lanes, one byte per j (< 128)
-    unsigned pj[4];  // kept entries of the warp in the earlier j, two 16-bit sums per word (a warp holds 1024 elements)
-    {
-      unsigned runj = 0;
-#pragma unroll
-      for (int j = 0; j < 8; ++j) {
-        if ((j & 1) == 0) pj[j >> 1] = runj;
-        else pj[j >> 1] |= runj << 16;
-        runj += ((j < 4 ? t0 : t1) >> (8 * (j & 3))) & 0xffu;
-      }
-    }
-    unsigned rem = km;
-    int last_j = -1, run = 0;
-    while (rem) {
-      const int b = __ffs((int)rem) - 1;
-      rem &= rem - 1;
-      const int j = b >> 2, e = b & 3;
-      if (j != last_j) { last_j = j; run = 0; }
-      const int e0 = 4 * (wi * 256 + j * 32 + lane);
-      const unsigned pw = j < 4 ? (j < 2 ? pj[0] : pj[1]) : (j < 6 ? pj[2] : pj[3]);
-      const int pos = pos0 + (int)((pw >> (16 * (j & 1))) & 0xffffu) +
-                      (int)(((j < 4 ? e0x : e1x) >> (8 * (j & 3))) & 0xffu) + run;
-      ++run;
-      if ((unsigned)pos < (unsigned)k) {
-        const float v = m[e0 + e];
-        vals[seg + pos] = v;
-        idx[seg + pos] = t.elem0 + e0 + e;
-        if (!LAZY) m[e0 + e] = 0.f;
-        else if (zero_ties && key_of(v) == tau && __float_as_uint(v) != 0u) m[e0 + e] = 0.f;
-      }
-    }
-  } else {
 #pragma unroll
   for (int j = 0; j < 8; ++j) {
     const unsigned nib = (km >> (4 * j)) & 15u;
@@ -1072,6 +1035,62 @@ __device__ __forceinline__ void select_tile_simple(const Tile& t, unsigned thr, 
     }
     pos0 += (int)(((j < 4 ? t0 : t1) >> sh) & 0xffu);
   }
+}
+
+// The same for a full tile with few entries to keep (the usual case: K of 1 % to 10 %), every lane owning 32
+// CONSECUTIVE elements: the warp's 1024 elements go through shared memory (coalesced 16-byte loads in, one padded
+// row of 32 per lane out), so that an entry's position is the lane's exclusive prefix plus a running count -- the
+// kept entries are found by walking the set bits of one 32-bit mask, a dozen instructions each, instead of deriving
+// the position of every entry from per-row prefixes (the walk was half of the pass).  A warp runs as many rounds
+// as its busiest lane has kept entries.
+constexpr int kRowWords = 36;  // 32 elements + 4 words of padding: 16-byte reads of consecutive rows hit distinct banks
+template <bool LAZY>
+__device__ __forceinline__ void select_tile_rows(const Tile& t, unsigned thr, unsigned tau, bool zero_ties, int base,
+                                                 int k, float* __restrict__ m, float* __restrict__ vals,
+                                                 int32_t* __restrict__ idx, long long seg, unsigned* wtot,
+                                                 float* rows) {
+  const int wi = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  float* wr = rows + wi * (32 * kRowWords);
+  float4 mv[8];
+#pragma unroll
+  for (int j = 0; j < 8; ++j) mv[j] = ld_stream4(m + 4 * (wi * 256 + j * 32 + lane));
+#pragma unroll
+  for (int j = 0; j < 8; ++j)  // float4 number j * 32 + lane of the warp: row 4 j + lane / 8, column 4 (lane % 8)
+    *reinterpret_cast<float4*>(wr + kRowWords * (4 * j + (lane >> 3)) + 4 * (lane & 7)) = mv[j];
+  __syncwarp();
+  const float* my = wr + kRowWords * lane;
+  unsigned km = 0;  // bit i: element 32 * lane + i of the warp's share is kept
+#pragma unroll
+  for (int q = 0; q < 8; ++q) {
+    const float4 v = *reinterpret_cast<const float4*>(my + 4 * q);
+    km |= ((unsigned)(key_of(v.x) >= thr) | ((unsigned)(key_of(v.y) >= thr) << 1) |
+           ((unsigned)(key_of(v.z) >= thr) << 2) | ((unsigned)(key_of(v.w) >= thr) << 3)) << (4 * q);
+  }
+  const unsigned cnt = __popc(km);
+  unsigned incl = cnt;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const unsigned n = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += n;
+  }
+  if (lane == 31) wtot[wi] = incl;
+  __syncthreads();
+  if (km == 0) return;
+  int pos = base + (int)(incl - cnt);
+  for (int i = 0; i < wi; ++i) pos += (int)wtot[i];
+  const int ebase = wi * 1024 + 32 * lane;
+  unsigned rem = km;
+  while (rem) {
+    const int b = __ffs((int)rem) - 1;
+    rem &= rem - 1;
+    if ((unsigned)pos < (unsigned)k) {  // always true for consistent counts; keeps a write inside the segment
+      const float v = my[b];
+      vals[seg + pos] = v;
+      idx[seg + pos] = t.elem0 + ebase + b;
+      if (!LAZY) m[ebase + b] = 0.f;
+      else if (zero_ties && key_of(v) == tau && __float_as_uint(v) != 0u) m[ebase + b] = 0.f;
+    }
+    ++pos;
   }
 }
 
@@ -1087,6 +1106,7 @@ topk_select_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict__
                    float* __restrict__ vals, int32_t* __restrict__ idx,
                    long long stride, long long capacity, const int2* __restrict__ lists, int W) {
   __shared__ unsigned wtot[8];
+  __shared__ __align__(16) float rows[8 * 32 * kRowWords];
   const unsigned long long n_work = any_list[kListCountWord + kListSelect];
   const unsigned b0 = (unsigned)(n_work * blockIdx.x / gridDim.x), b1 = (unsigned)(n_work * (blockIdx.x + 1) / gridDim.x);
   if (b0 >= b1) return;
@@ -1130,9 +1150,9 @@ topk_select_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict__
       const int base = p.x + min(p.y, need);
       const bool zt = all_ties && o.y != 0;
       const int kept = o.x + (all_ties ? o.y : 0);  // entries of the tile that will be written
-      if (t.nelem != kTile) select_tile_simple<false, LAZY, false>(t, thr, tau, zt, base, k, m, vals, idx, seg, wtot);
-      else if (kept <= kTile / 5) select_tile_simple<true, LAZY, true>(t, thr, tau, zt, base, k, m, vals, idx, seg, wtot);
-      else select_tile_simple<true, LAZY, false>(t, thr, tau, zt, base, k, m, vals, idx, seg, wtot);
+      if (t.nelem != kTile) select_tile_simple<false, LAZY>(t, thr, tau, zt, base, k, m, vals, idx, seg, wtot);
+      else if (kept <= kTile / 5) select_tile_rows<LAZY>(t, thr, tau, zt, base, k, m, vals, idx, seg, wtot, rows);
+      else select_tile_simple<true, LAZY>(t, thr, tau, zt, base, k, m, vals, idx, seg, wtot);
     } else {
       if (t.nelem == kTile) select_tile<true, LAZY>(t, tau, need, k, p, m, vals, idx, seg, wtot);
       else select_tile<false, LAZY>(t, tau, need, k, p, m, vals, idx, seg, wtot);
