@@ -311,16 +311,19 @@ psgd_project_kernel(const DevLayer* __restrict__ layers, const Tile* __restrict_
 }
 
 // Pass 1, pipelined.  Persistent blocks (one per SM, 512 threads), each with a contiguous range of MATRIX
-// tiles.  The sequence of (tile, worker) stages of a block is streamed through three shared-memory stage
-// buffers by bulk asynchronous copies: while the threads consume stage i (g_w and e_w of one tile,
-// 2 x 32 KB), the copies of stages i+1 and i+2 are in flight and, once everybody has left stage i's buffer,
-// stage i+3 is issued into it -- 128-192 KB per SM are in flight at all times without costing registers.
-// The arithmetic is that of the direct kernel (same operations in the same order).
+// tiles and, at the end, a few tiles drawn by ticket.  The sequence of (tile, worker) stages of a block is streamed
+// through two shared-memory stage buffers by bulk asynchronous copies: while the threads consume stage i (g_w and
+// e_w of one tile, 2 x 32 KB), the copy of stage i+1 is in flight and, once everybody has left stage i's buffer,
+// stage i+2 is issued into it -- 64-128 KB per SM are in flight at all times without costing registers.
+// The arithmetic is that of the direct kernel's element path (same operations in the same order).
 constexpr int kPipeThreads = 512;
 constexpr int kPipePos = kTile / 4 / kPipeThreads;  // float4 positions per thread and tile
 constexpr int kPipeStages = 2;
 constexpr int kPipeMinStagesPerSm = 200;  // below this the direct kernel is used
 constexpr int kPipeWarps = kPipeThreads / 32;
+constexpr int kPipeDynamicTiles = 3;  // tiles per block handed out by ticket instead of the even split (LSTM set, W = 8:
+                                      // 0.858 ms with 0, 0.851 with 1, 0.838 with 2, 0.835 with 3, 0.832-0.839 with 4 to all)
+constexpr int kPipeTicketWord = 8;    // status block, words 8-9: ticket and count of finished blocks
 // stage buffers, the mean matrix of the tile, the detector accumulator of the tile
 constexpr size_t kPipeSmemBytes = sizeof(float) * kTile * (2 * kPipeStages + 2) + sizeof(float4) * 2 * kPipeWarps + 64;
 
@@ -331,7 +334,8 @@ psgd_project_pipe_kernel(const DevLayer* __restrict__ layers, const Tile* __rest
                          int n_vec_tiles, const float* __restrict__ grads, float* __restrict__ err,
                          const float* __restrict__ q, const float* __restrict__ p, float4* __restrict__ p_part,
                          const int* __restrict__ pending, float* __restrict__ out, float* __restrict__ delta,
-                         long long stride, int W, int decider, float inv_w, int* __restrict__ status) {
+                         long long stride, int W, int decider, float inv_w, int* __restrict__ status,
+                         int dyn_tiles) {
   extern __shared__ __align__(128) unsigned char smem_raw[];
   float* stage = reinterpret_cast<float*>(smem_raw);                  // [kPipeStages buffers][g, e][kTile]
   float* s_mbar = stage + 2 * kPipeStages * kTile;                    // [kTile]
@@ -342,10 +346,17 @@ psgd_project_pipe_kernel(const DevLayer* __restrict__ layers, const Tile* __rest
     const Tile t = tiles[vec_tiles[i]];
     vector_mean_tile(t, layers[t.layer], grads, out, delta, stride, W, decider, inv_w);
   }
-  const int t0 = (int)((long long)n_mat_tiles * blockIdx.x / gridDim.x);
-  const int t1 = (int)((long long)n_mat_tiles * (blockIdx.x + 1) / gridDim.x);
-  const int n_stages = (t1 - t0) * W;
-  if (n_stages == 0) return;
+  // The tiles of a block: a contiguous range of the first n_static tiles (an even split), then tiles of the rest
+  // handed out one at a time by ticket -- blocks do not take the same time per tile (ragged tiles, rows of the
+  // factor tables in L1 or not, the SM's share of DRAM), and with an even split of everything the SMs were idle for
+  // 5 % of the kernel on average (8 % on the VGG set) while the slowest blocks finished.  ticket[0] hands out the
+  // tiles, ticket[1] counts the blocks that are through; the last one clears both for the next launch.
+  int* ticket = status + kPipeTicketWord;
+  const int n_dynamic = min(n_mat_tiles, (int)gridDim.x * dyn_tiles);
+  const int n_static = n_mat_tiles - n_dynamic;
+  const int t0 = (int)((long long)n_static * blockIdx.x / gridDim.x);
+  const int n_own = (int)((long long)n_static * (blockIdx.x + 1) / gridDim.x) - t0;
+  int* s_seq = reinterpret_cast<int*>(bars + kPipeStages);  // [4] ring: the block's i-th tile (index into mat_tiles), -1 = none
   if (threadIdx.x == 0) {
     for (int b = 0; b < kPipeStages; ++b) mbar_init(&bars[b], 1);
     fence_mbar_init();
@@ -357,10 +368,19 @@ psgd_project_pipe_kernel(const DevLayer* __restrict__ layers, const Tile* __rest
   int is_ti = -1;
   long long is_base = 0;
   unsigned is_bytes = 0;
+  bool ended = false;  // the block's sequence of tiles is complete (a ticket beyond the last tile was drawn)
   auto issue = [&](int it) {
+    if (ended) return;
     const int ti = it / W, w = it - ti * W;
     if (ti != is_ti) {
-      const Tile tt = tiles[mat_tiles[t0 + ti]];
+      int g = t0 + ti;
+      if (ti >= n_own) {
+        const int k = atomicAdd(&ticket[0], 1);
+        g = k < n_dynamic ? n_static + k : -1;
+      }
+      s_seq[ti & 3] = g;  // read by everybody at the first stage of the tile, at least one barrier later
+      if (g < 0) { ended = true; return; }
+      const Tile tt = tiles[mat_tiles[g]];
       is_ti = ti;
       is_base = layers[tt.layer].offset + tt.elem0;
       is_bytes = (unsigned)((tt.nelem + 3) / 4) * 16u;  // a ragged tile reads into the layer's padding
@@ -376,29 +396,36 @@ psgd_project_pipe_kernel(const DevLayer* __restrict__ layers, const Tile* __rest
     bulk_copy_g2s(stage + (2 * buf + 1) * kTile, err + base, is_bytes, &bars[buf]);
     if (with_delta) bulk_copy_g2s(s_delta, delta + is_base, is_bytes, &bars[buf]);
   };
+  auto leave = [&]() {  // thread 0, once per block
+    __threadfence();
+    if (atomicAdd(&ticket[1], 1) == (int)gridDim.x - 1) { ticket[0] = 0; ticket[1] = 0; }
+  };
   if (threadIdx.x == 0)
-    for (int it = 0; it < kPipeStages && it < n_stages; ++it) issue(it);
-  int gt = mat_tiles[t0];  // the tile's index among all tiles
-  Tile t = tiles[gt];
-  DevLayer L = layers[t.layer];
+    for (int it = 0; it < kPipeStages; ++it) issue(it);
+  __syncthreads();  // s_seq of the first tile(s) is in place
+  int gt = 0;  // the tile's index among all tiles
+  Tile t;
+  DevLayer L;
+  t.layer = -1; t.elem0 = 0; t.nelem = 0;
   float4 corr[kPipePos], mb[kPipePos];
-  int rp = LAZY ? pending[t.layer] : 0;
-  for (int it = 0; it < n_stages; ++it) {
-    const int ti = it / W, w = it - ti * W;
+  int rp = 0;
+  int last_g = -2;
+  for (int it = 0, ti = 0, w = 0;; ++it) {
     const int buf = it % kPipeStages;
     if (w == 0) {  // new tile: factors of the pending residual at this thread's positions
-      if (ti > 0) {
-        if (gt + 1 < L.tile0 + L.ntiles) {  // next tile of the same layer: no table look-ups
-          gt += 1;
-          t.elem0 += kTile;
-          t.nelem = (int)min((long long)kTile, (long long)L.rows * L.cols - t.elem0);
-        } else {
-          gt = mat_tiles[t0 + ti];
-          t = tiles[gt];
-          L = layers[t.layer];
-          rp = LAZY ? pending[t.layer] : 0;
-        }
+      const int g = s_seq[ti & 3];
+      if (g < 0) break;  // (uniform over the block)
+      if (g == last_g + 1 && gt + 1 < L.tile0 + L.ntiles) {  // next tile of the same layer: no table look-ups
+        gt += 1;
+        t.elem0 += kTile;
+        t.nelem = (int)min((long long)kTile, (long long)L.rows * L.cols - t.elem0);
+      } else {
+        gt = mat_tiles[g];
+        t = tiles[gt];
+        L = layers[t.layer];
+        rp = LAZY ? pending[t.layer] : 0;
       }
+      last_g = g;
       const float4* Q4 = reinterpret_cast<const float4*>(q) + L.q_row;
       const float4* P4 = reinterpret_cast<const float4*>(p) + L.p_row;
 #pragma unroll
@@ -419,7 +446,7 @@ psgd_project_pipe_kernel(const DevLayer* __restrict__ layers, const Tile* __rest
     }
     const bool arrived = __syncthreads_and(mbar_wait_bounded(&bars[buf], (unsigned)(it / kPipeStages) & 1u));
     if (!arrived) {  // a copy never completed: report and leave (uniformly for the whole block)
-      if (threadIdx.x == 0) atomicExch(status, ACC_ETIMEOUT);
+      if (threadIdx.x == 0) { atomicExch(status, ACC_ETIMEOUT); leave(); }
       return;
     }
     const float* sg = stage + (2 * buf) * kTile;
@@ -453,7 +480,7 @@ psgd_project_pipe_kernel(const DevLayer* __restrict__ layers, const Tile* __rest
       }
     }
     __syncthreads();  // everybody has left this stage buffer
-    if (threadIdx.x == 0 && it + kPipeStages < n_stages) {
+    if (threadIdx.x == 0 && !ended) {
       fence_proxy_async_smem();
       issue(it + kPipeStages);
     }
@@ -475,7 +502,9 @@ psgd_project_pipe_kernel(const DevLayer* __restrict__ layers, const Tile* __rest
       __syncthreads();
       tile_p_partials<kPipeWarps>(s_mbar, s_pp, t, L, reinterpret_cast<const float4*>(q) + L.q_row, p_part);
     }
+    if (++w == W) { w = 0; ++ti; }
   }
+  if (threadIdx.x == 0) leave();
 }
 
 // Deterministic block-wide sum of doubles; every thread gets the result.
@@ -1011,14 +1040,16 @@ static void launch_psgd_project(acc_ctx* ctx, const float* grads, float* err, fl
     // low level; with every SM taken, the TopK step's short kernels wait for this pass to end)
     const int sms = (c.flags & ACC_FLAG_SHARE_SMS) ? std::max(ctx->sm_count / 2, 1) : ctx->sm_count;
     const int grid = n_mt < sms ? n_mt : sms;
+    const int dyn_tiles = kPipeDynamicTiles;
     if (lazy) {
       psgd_project_pipe_kernel<true><<<grid, kPipeThreads, kPipeSmemBytes, s>>>(
           ctx->d_layers, ctx->d_tiles, ctx->d_mat_tiles, n_mt, ctx->d_vec_tiles, n_vt, grads, err, q, p_hat,
-          ctx->d_ppart, ctx->d_pending, out, delta, c.worker_stride, c.n_workers, c.decider, inv_w, ctx->d_status);
+          ctx->d_ppart, ctx->d_pending, out, delta, c.worker_stride, c.n_workers, c.decider, inv_w, ctx->d_status,
+          dyn_tiles);
     } else {
       psgd_project_pipe_kernel<false><<<grid, kPipeThreads, kPipeSmemBytes, s>>>(
           ctx->d_layers, ctx->d_tiles, ctx->d_mat_tiles, n_mt, ctx->d_vec_tiles, n_vt, grads, err, q, p_hat,
-          ctx->d_ppart, nullptr, out, delta, c.worker_stride, c.n_workers, c.decider, inv_w, ctx->d_status);
+          ctx->d_ppart, nullptr, out, delta, c.worker_stride, c.n_workers, c.decider, inv_w, ctx->d_status, dyn_tiles);
     }
   } else if (lazy) {
     psgd_project_kernel<4, true><<<nt, kProjThreads, 0, s>>>(ctx->d_layers, ctx->d_tiles, grads, err, q, p_hat, ctx->d_ppart,
