@@ -516,7 +516,9 @@ def main():
                                       f"every layer held at the {args.force_level} compression level"),
                            "regime_of_value": ", ".join(f"{v['steps']} of {K} timed steps at {k}"
                                                         for k, v in by_regime.items()),
-                           "streams": ("TopK step beside the PowerSGD step on a second stream"
+                           "streams": (("TopK step beside the PowerSGD step on a second stream" +
+                                        ("; pipelined first PowerSGD pass on half of the SMs" if args.share_sms
+                                         else ""))
                                        if (n_comp == 2 and not args.no_overlap) else "one stream"),
                            "multi_gpu": "independent replicas, no collective"},
                 "clocks": clocks, "e2e": e2e, "gpu_launches": gpu_launches,
