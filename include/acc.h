@@ -63,9 +63,9 @@ extern "C" {
 #define ACC_FLAG_PIPELINE_ALWAYS 2
 #define ACC_FLAG_PIPELINE_NEVER 4
 /* The caller issues this context's PowerSGD step and TopK step at the same time on two streams.  The pipelined
- * first PowerSGD pass then starts one persistent block on every second SM only (a block fills an SM, so that
- * nothing else runs beside it): the TopK step's kernels get the other half instead of waiting for the pass to
- * end.  Same results; a PowerSGD step that runs alone is slower with it.  No effect on the direct kernel. */
+ * first PowerSGD pass then starts half as many persistent blocks as the GPU has SMs (a block fills an SM, so
+ * nothing else runs beside it): the TopK step's kernels get the other SMs instead of waiting for the pass to end.
+ * Same results bit for bit; a PowerSGD step that runs alone is slower with it.  No effect on the direct kernel. */
 #define ACC_FLAG_SHARE_SMS 8
 
 #define ACC_COMPRESSOR_POWERSGD 0
