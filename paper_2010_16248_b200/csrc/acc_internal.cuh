@@ -110,7 +110,8 @@ struct acc_ctx {
   int* d_mat_layers = nullptr;
   int* d_vec_tiles = nullptr;
   int* d_mat_tiles = nullptr;
-  int* d_status = nullptr;           // device-side error flag (0 = none), see acc_device_status
+  int* d_status = nullptr;           // 64 words: [0] device-side error flag (0 = none), see acc_device_status;
+                                     // [8], [9] tile ticket and finished-block count of the pipelined first PowerSGD pass
   float4* d_part = nullptr;
   float4* d_ppart = nullptr;         // partial rows of P, one slot per tile a row touches
   int* d_pending = nullptr;          // lazy PowerSGD: rank of the residual not yet applied to err, per layer
