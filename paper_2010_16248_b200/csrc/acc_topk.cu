@@ -1271,11 +1271,16 @@ topk_finalize_staged_kernel(const DevLayer* __restrict__ layers, const Tile* __r
 // block's next tile are fetched while the current one is worked on.
 // SGD: the optimiser tail is applied to every element of out where it is written.
 constexpr int kDecStage = kTile / 2;  // staged entries per round
+constexpr int kDecWide = 256;         // tiles in which worker 0 has this many entries move them in 16-byte copies
 constexpr size_t kDecSmemBytes = sizeof(float) * kTile + (sizeof(int) + sizeof(float)) * kDecStage +
                                  sizeof(int) * 2 * kMaxWorkers + 16;
 
 __device__ __forceinline__ void cp_async4(void* dst_smem, const void* src) {
   asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(smem_u32(dst_smem)), "l"(__cvta_generic_to_global(src))
+               : "memory");
+}
+__device__ __forceinline__ void cp_async16(void* dst_smem, const void* src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(dst_smem)), "l"(__cvta_generic_to_global(src))
                : "memory");
 }
 __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
@@ -1343,37 +1348,103 @@ topk_decompress_kernel(const DevLayer* __restrict__ layers, const Tile* __restri
       for (int i = threadIdx.x; i < kTile / 4; i += blockDim.x)
         reinterpret_cast<float4*>(acc)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
       __syncthreads();  // the ranges are in place (and acc is clear)
-      // rounds: the staging area is filled with the entries of as many workers as fit, in worker order (a worker
-      // with more entries in the tile than the area holds is cut into pieces that take a round each)
-      int w0 = 0, off0 = 0;  // first worker of the round and how many of its entries earlier rounds have taken
-      while (w0 < W) {
-        int w = w0, off = off0, o = 0;
-        while (w < W && o < kDecStage) {
-          const int lo = r_lo[w] + off, n = min(r_hi[w] - lo, kDecStage - o);
-          const long long seg = (long long)w * capacity + l_seg_off;
-          for (int i = threadIdx.x; i < n; i += 256) {
-            cp_async4(s_idx + o + i, idx + seg + lo + i);
-            cp_async4(s_val + o + i, vals + seg + lo + i);
+      // Long ranges (a low compression level; told by worker 0's range): a piece is placed so that its first entry
+      // on a 16-byte boundary of the packed arrays also lies on one in shared memory; everything between the
+      // boundaries then moves in 16-byte copies (four entries each), at most three entries at either end in 4-byte
+      // copies.  Short ranges are not worth the placement arithmetic.
+      if (r_hi[0] - r_lo[0] >= kDecWide) {
+        const int cap3 = (int)(capacity & 3), seg3 = (int)(l_seg_off & 3);
+        auto piece = [&](int w, int off, int o, int* lo, int* take, int* os, int* lead, bool* whole) {
+          *lo = r_lo[w] + off;
+          const int rem = r_hi[w] - *lo;
+          // (the last two bits of the piece's first position, w * capacity + seg_off + lo, in 32-bit arithmetic)
+          *lead = -((w & 3) * cap3 + seg3 + *lo) & 3;
+          *os = o + (-(o + *lead) & 3);
+          *take = rem > 0 ? max(0, min(rem, kDecStage - *os)) : 0;
+          *whole = *take == rem;  // (an empty range is whole; a range that finds the area full is not)
+        };
+        int w0 = 0, off0 = 0;  // first worker of the round and how many of its entries earlier rounds have taken
+        while (w0 < W) {
+          int w = w0, off = off0, o = 0;
+          while (w < W) {
+            int lo, take, os, lead;
+            bool whole;
+            piece(w, off, o, &lo, &take, &os, &lead, &whole);
+            if (take > 0) {
+              const long long g0 = (long long)w * capacity + l_seg_off + lo;
+              const int32_t* gi = idx + g0;
+              const float* gv = vals + g0;
+              const int ld = min(lead, take), nq = (take - ld) >> 2, tail0 = ld + 4 * nq;
+              for (int i = threadIdx.x; i < nq; i += 256) {
+                cp_async16(s_idx + os + ld + 4 * i, gi + ld + 4 * i);
+                cp_async16(s_val + os + ld + 4 * i, gv + ld + 4 * i);
+              }
+              const int ne = ld + (take - tail0);  // the entries outside the boundaries: at most six
+              if ((int)threadIdx.x < ne) {
+                const int j = (int)threadIdx.x < ld ? (int)threadIdx.x : tail0 + ((int)threadIdx.x - ld);
+                cp_async4(s_idx + os + j, gi + j);
+                cp_async4(s_val + os + j, gv + j);
+              }
+              o = os + take;
+            }
+            if (!whole) { off += take; break; }
+            ++w;
+            off = 0;
           }
-          o += n;
-          if (lo + n == r_hi[w]) { ++w; off = 0; } else { off += n; }
-        }
-        cp_async_wait_all();
-        __syncthreads();
-        int w2 = w0, off2 = off0;
-        o = 0;
-        while (w2 < W && o < kDecStage) {
-          const int lo = r_lo[w2] + off2, n = min(r_hi[w2] - lo, kDecStage - o);
-          for (int i = threadIdx.x; i < n; i += 256) {
-            const unsigned li = (unsigned)(s_idx[o + i] - elem0);
-            if (li < (unsigned)kTile) acc[li] += s_val[o + i];
+          cp_async_wait_all();
+          __syncthreads();
+          int w2 = w0, off2 = off0;
+          o = 0;
+          while (w2 < W) {
+            int lo, take, os, lead;
+            bool whole;
+            piece(w2, off2, o, &lo, &take, &os, &lead, &whole);
+            for (int i = threadIdx.x; i < take; i += 256) {
+              const unsigned li = (unsigned)(s_idx[os + i] - elem0);
+              if (li < (unsigned)kTile) acc[li] += s_val[os + i];
+            }
+            if (take > 0) o = os + take;
+            __syncthreads();  // the next worker may add to the same elements; the last piece frees the staging area
+            if (!whole) break;
+            ++w2;
+            off2 = 0;
           }
-          o += n;
-          if (lo + n == r_hi[w2]) { ++w2; off2 = 0; } else { off2 += n; }
-          __syncthreads();  // the next worker may add to the same elements; the last piece frees the staging area
+          w0 = w;
+          off0 = off;
         }
-        w0 = w;
-        off0 = off;
+      } else {
+        // rounds: the staging area is filled with the entries of as many workers as fit, in worker order (a worker
+        // with more entries in the tile than the area holds is cut into pieces that take a round each)
+        int w0 = 0, off0 = 0;  // first worker of the round and how many of its entries earlier rounds have taken
+        while (w0 < W) {
+          int w = w0, off = off0, o = 0;
+          while (w < W && o < kDecStage) {
+            const int lo = r_lo[w] + off, n = min(r_hi[w] - lo, kDecStage - o);
+            const long long seg = (long long)w * capacity + l_seg_off;
+            for (int i = threadIdx.x; i < n; i += 256) {
+              cp_async4(s_idx + o + i, idx + seg + lo + i);
+              cp_async4(s_val + o + i, vals + seg + lo + i);
+            }
+            o += n;
+            if (lo + n == r_hi[w]) { ++w; off = 0; } else { off += n; }
+          }
+          cp_async_wait_all();
+          __syncthreads();
+          int w2 = w0, off2 = off0;
+          o = 0;
+          while (w2 < W && o < kDecStage) {
+            const int lo = r_lo[w2] + off2, n = min(r_hi[w2] - lo, kDecStage - o);
+            for (int i = threadIdx.x; i < n; i += 256) {
+              const unsigned li = (unsigned)(s_idx[o + i] - elem0);
+              if (li < (unsigned)kTile) acc[li] += s_val[o + i];
+            }
+            o += n;
+            if (lo + n == r_hi[w2]) { ++w2; off2 = 0; } else { off2 += n; }
+            __syncthreads();  // the next worker may add to the same elements; the last piece frees the staging area
+          }
+          w0 = w;
+          off0 = off;
+        }
       }
       const int n4 = nelem >> 2;
       for (int i = threadIdx.x; i < n4; i += blockDim.x) {
