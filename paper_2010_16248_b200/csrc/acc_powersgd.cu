@@ -687,18 +687,26 @@ __device__ __forceinline__ void qpart_cols(const ColItem& it, const DevLayer& L,
   for (int e = 0; e < VEC; ++e) acc[e][0] = acc[e][1] = acc[e][2] = acc[e][3] = 0.f;
   const float* base = mbar + L.offset + (long long)it.row0 * L.cols + col;
   const float4* pr = P4 + it.row0;
-#pragma unroll 8
-  for (int i = 0; i < it.nrows; ++i) {
-    const V mv = *reinterpret_cast<const V*>(base + (long long)i * L.cols);
-    const float4 pv = __ldg(pr + i);
-    const float* m = reinterpret_cast<const float*>(&mv);
+  // rows in batches of kRows: the batch's loads of the mean matrix go out together (the rows are added in order)
+  constexpr int kRows = 16 / VEC;  // 64 bytes of every row batch per thread
+  for (int i0 = 0; i0 < it.nrows; i0 += kRows) {
+    V mv[kRows];
 #pragma unroll
-    for (int e = 0; e < VEC; ++e) {
-      acc[e][0] = fmaf(m[e], pv.x, acc[e][0]);
-      acc[e][1] = fmaf(m[e], pv.y, acc[e][1]);
-      acc[e][2] = fmaf(m[e], pv.z, acc[e][2]);
-      acc[e][3] = fmaf(m[e], pv.w, acc[e][3]);
-    }
+    for (int k = 0; k < kRows; ++k)
+      if (i0 + k < it.nrows) mv[k] = *reinterpret_cast<const V*>(base + (long long)(i0 + k) * L.cols);
+#pragma unroll
+    for (int k = 0; k < kRows; ++k)
+      if (i0 + k < it.nrows) {
+        const float4 pv = __ldg(pr + i0 + k);
+        const float* m = reinterpret_cast<const float*>(&mv[k]);
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) {
+          acc[e][0] = fmaf(m[e], pv.x, acc[e][0]);
+          acc[e][1] = fmaf(m[e], pv.y, acc[e][1]);
+          acc[e][2] = fmaf(m[e], pv.z, acc[e][2]);
+          acc[e][3] = fmaf(m[e], pv.w, acc[e][3]);
+        }
+      }
   }
   float4* dst = part + L.part_base + (long long)it.slab * L.cols + col;
 #pragma unroll
