@@ -684,13 +684,24 @@ topk_hist_list_kernel(const DevLayer* __restrict__ layers, const int* __restrict
     const unsigned c1 = min(c0 + kChunk, n);  // the list starts 16-byte aligned and kChunk is a multiple of 4
     const unsigned n4 = (c1 - c0) >> 2;
     const uint4* k4 = reinterpret_cast<const uint4*>(keys + c0);
-#pragma unroll 4
-    for (unsigned i = threadIdx.x; i < n4; i += blockDim.x) {
-      const uint4 kk = __ldcs(k4 + i);
-      if (staged) {
-        count(kk.x & 0x7fffffffu); count(kk.z & 0x7fffffffu);
-      } else {
-        count(kk.x); count(kk.y); count(kk.z); count(kk.w);
+    // (the chunk's loads of a thread -- four 16-byte words -- go out together, then the counting)
+    constexpr int kLoads = kChunk / 4 / 256;
+    uint4 kb[kLoads];
+#pragma unroll
+    for (int u = 0; u < kLoads; ++u) {
+      const unsigned i = threadIdx.x + u * 256u;
+      if (i < n4) kb[u] = __ldcs(k4 + i);
+    }
+#pragma unroll
+    for (int u = 0; u < kLoads; ++u) {
+      const unsigned i = threadIdx.x + u * 256u;
+      if (i < n4) {
+        const uint4 kk = kb[u];
+        if (staged) {
+          count(kk.x & 0x7fffffffu); count(kk.z & 0x7fffffffu);
+        } else {
+          count(kk.x); count(kk.y); count(kk.z); count(kk.w);
+        }
       }
     }
     for (unsigned i = c0 + 4 * n4 + threadIdx.x; i < c1; i += blockDim.x)
