@@ -99,6 +99,7 @@ static int make_plan(const acc_config* cfg, Plan& p) {
     for (int s = 0; s < o.nslabs; ++s)
       for (int c0 = 0; c0 < d.cols; c0 += cb)
         p.col_items.push_back(ColItem{l, s, s * o.slab_rows, std::min(o.slab_rows, d.rows - s * o.slab_rows), c0});
+    for (int c0 = 0; c0 < d.cols; c0 += 32) p.qred_items.push_back(make_int2(l, c0 / 32));
   }
   const size_t nt = p.tiles.size();
   const size_t seg = (size_t)W * std::max(p.n_mat, 1);
@@ -106,6 +107,7 @@ static int make_plan(const acc_config* cfg, Plan& p) {
   auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes, 256); return at; };
   p.o_layers = take(sizeof(DevLayer) * L);
   p.o_col_items = take(sizeof(ColItem) * std::max<size_t>(1, p.col_items.size()));
+  p.o_qred_items = take(sizeof(int2) * std::max<size_t>(1, p.qred_items.size()));
   p.o_tiles = take(sizeof(Tile) * nt);
   p.o_mat_layers = take(sizeof(int) * std::max<size_t>(1, p.mat_layers.size()));
   p.o_vec_tiles = take(sizeof(int) * std::max<size_t>(1, p.vec_tiles.size()));
@@ -171,6 +173,7 @@ int acc_create(const acc_config* cfg, void* workspace, size_t workspace_bytes, a
   char* ws = ctx->ws;
   ctx->d_layers = reinterpret_cast<DevLayer*>(ws + p.o_layers);
   ctx->d_col_items = reinterpret_cast<ColItem*>(ws + p.o_col_items);
+  ctx->d_qred_items = reinterpret_cast<int2*>(ws + p.o_qred_items);
   ctx->d_tiles = reinterpret_cast<Tile*>(ws + p.o_tiles);
   ctx->d_mat_layers = reinterpret_cast<int*>(ws + p.o_mat_layers);
   ctx->d_vec_tiles = reinterpret_cast<int*>(ws + p.o_vec_tiles);
@@ -204,6 +207,7 @@ int acc_create(const acc_config* cfg, void* workspace, size_t workspace_bytes, a
   };
   up(ctx->d_layers, p.layers.data(), sizeof(DevLayer) * p.layers.size());
   up(ctx->d_col_items, p.col_items.data(), sizeof(ColItem) * p.col_items.size());
+  up(ctx->d_qred_items, p.qred_items.data(), sizeof(int2) * p.qred_items.size());
   up(ctx->d_tiles, p.tiles.data(), sizeof(Tile) * p.tiles.size());
   up(ctx->d_mat_layers, p.mat_layers.data(), sizeof(int) * p.mat_layers.size());
   up(ctx->d_vec_tiles, p.vec_tiles.data(), sizeof(int) * p.vec_tiles.size());

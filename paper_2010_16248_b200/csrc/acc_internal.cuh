@@ -75,6 +75,7 @@ struct ProfSlot { int phase; cudaEvent_t a, b; };
 struct Plan {
   std::vector<DevLayer> layers;
   std::vector<ColItem> col_items;
+  std::vector<int2> qred_items;  // (layer, block of 32 columns) of every MATRIX layer: the grid of the Q-reduce pass
   std::vector<Tile> tiles;
   std::vector<int> mat_layers;   // layer index of each MATRIX layer
   std::vector<int> vec_tiles;    // tile indices that belong to VECTOR layers
@@ -85,6 +86,7 @@ struct Plan {
   int max_cols = 0;  // most columns of any MATRIX layer
   long long vec_floats = 0;  // packed VECTOR elements (each layer starts at a multiple of 4)
   // workspace offsets (bytes)
+  size_t o_qred_items = 0;
   size_t o_layers = 0, o_col_items = 0, o_tiles = 0, o_mat_layers = 0, o_vec_tiles = 0, o_mat_tiles = 0, o_status = 0,
          o_part = 0, o_ppart = 0, o_pending = 0, o_norm_part = 0, o_hist = 0, o_sel = 0, o_pred = 0, o_cand = 0, o_tile_cand = 0, o_tile_cnt = 0, o_tile_h3 = 0, o_tile_pre = 0, o_tile_rng = 0, o_lists = 0, o_pend_tau = 0,
          hist_bytes = 0, total = 0;
@@ -106,6 +108,7 @@ struct acc_ctx {
   // device views into the workspace
   acc::DevLayer* d_layers = nullptr;
   acc::ColItem* d_col_items = nullptr;
+  int2* d_qred_items = nullptr;
   acc::Tile* d_tiles = nullptr;
   int* d_mat_layers = nullptr;
   int* d_vec_tiles = nullptr;

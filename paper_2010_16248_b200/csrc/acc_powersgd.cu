@@ -803,15 +803,15 @@ psgd_decompress_kernel(const DevLayer* __restrict__ layers, const ColItem* __res
 
 // Pass 4.  Sums the slab partials of 32 columns in a fixed order and stores the first r ranks of Q'.
 __global__ void __launch_bounds__(256)
-psgd_qreduce_kernel(const DevLayer* __restrict__ layers, const int* __restrict__ mat_layers,
+psgd_qreduce_kernel(const DevLayer* __restrict__ layers, const int2* __restrict__ items,
                     const float4* __restrict__ part, float* __restrict__ q, const uint8_t* __restrict__ level,
                     int rank_low, int rank_high, float4* __restrict__ q_sum) {
   __shared__ float4 sm[8][32];
-  const int l = mat_layers[blockIdx.y];
+  const int2 it = items[blockIdx.x];  // (layer, block of 32 columns)
+  const int l = it.x;
   const DevLayer L = layers[l];
-  if ((int)blockIdx.x * 32 >= L.cols) return;
   const int cx = threadIdx.x & 31, gy = threadIdx.x >> 5;
-  const int col = blockIdx.x * 32 + cx;
+  const int col = it.y * 32 + cx;
   float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
   if (col < L.cols) {
     for (int s = gy; s < L.nslabs; s += 8) {
@@ -1098,8 +1098,8 @@ static void launch_psgd_ortho_q(acc_ctx* ctx, float* q, float* p_hat, const uint
   }
   {
     PhaseTimer pt(ctx, PH_PSGD_QREDUCE, s);
-    psgd_qreduce_kernel<<<dim3((pl.max_cols + 31) / 32, pl.n_mat), 256, 0, s>>>(
-        ctx->d_layers, ctx->d_mat_layers, ctx->d_part, q, level, c.rank_low, c.rank_high, q_sum);
+    psgd_qreduce_kernel<<<(unsigned)pl.qred_items.size(), 256, 0, s>>>(
+        ctx->d_layers, ctx->d_qred_items, ctx->d_part, q, level, c.rank_low, c.rank_high, q_sum);
   }
 }
 
